@@ -1,0 +1,362 @@
+"""CPU oracle of the expert-cached MoE layer.  TEST INFRASTRUCTURE ONLY.
+
+A plain, slow, obviously-correct numpy/fp64 statement of what the layer
+computes, written from the paper's description of the method (Sec. 3 intro:
+host expert pool = source of truth, HBM slots = cache; Sec. 3.2: hit set,
+miss partition Eq. 1, residual bandwidth Eq. 2, branch times Eq. 3, fill count
+q* Eq. 4, "always retains at least one fill", LRU residency; Sec. 4.1: one
+pass yields the K least-recently-used candidate slots).  It shares no code
+with the CUDA library and must never be imported by the product path: only
+tests, the smoke check and the benchmark's CPU-baseline leg use it.
+
+Values are exact by definition (the method preserves the MoE output without
+approximation, Sec. 3.2), so the value part of the oracle is simply the
+definition of a top-k softmax MoE layer with SwiGLU experts, evaluated from the
+*pool* by expert id and therefore independent of any cache state.  Residency
+is a deterministic integer state machine; it is written out step by step.
+
+Where the paper is silent the readings are (each also listed in the design
+notes): top-k order = (logit descending, expert id ascending); gate weights =
+softmax over the k selected logits; the permutation is stable in pair index
+p = t*k + j; one recency stamp per plan call; experts hit in this step cannot
+be evicted in this step; free slots are consumed first (ascending index), then
+occupied ones by (stamp ascending, resident expert id ascending); the fill set
+is taken from the eligible misses by (token count descending, id ascending);
+q* is rounded half up in integer arithmetic; misses that get no slot are served
+in place (zero-copy) and leave residency unchanged.
+
+Every function is pinned by tests that do not re-use its own formula: brute
+force over subsets, library softmax / stable sort, the worked split of the
+paper's overview figure, closed forms (B_r = 0 gives q = m), a naive
+move-to-front LRU, a hand-worked trace and the dense (uncached) MoE.
+Parity unpinned: nothing.
+"""
+from __future__ import annotations
+
+import dataclasses
+
+import numpy as np
+
+GROUP = 128
+
+LOC_NOT_ROUTED = -1
+LOC_ZERO_COPY = -2
+
+
+# ---------------------------------------------------------------------------
+# Step 1: routing (Sec. 3.2: "the router and cache lookup run on the GPU")
+# ---------------------------------------------------------------------------
+
+def route(logits: np.ndarray, k: int) -> tuple[np.ndarray, np.ndarray]:
+    """Top-k experts and gate weights per token.
+
+    ids[t, :] are the k experts with the largest logits, ordered by
+    (logit descending, id ascending); w[t, j] = exp(z_j) / sum_{i<k} exp(z_i)
+    over the selected logits.  Non-finite logits are invalid input.
+    """
+    z = np.asarray(logits, dtype=np.float32)
+    if z.ndim != 2:
+        raise ValueError("logits must be [T, E]")
+    T, E = z.shape
+    if not (1 <= k <= E):
+        raise ValueError("top_k out of range")
+    if not np.all(np.isfinite(z)):
+        raise ValueError("non-finite logits")
+    ids = np.empty((T, k), dtype=np.int32)
+    w = np.empty((T, k), dtype=np.float32)
+    for t in range(T):
+        order = sorted(range(E), key=lambda e: (-float(z[t, e]), e))
+        sel = order[:k]
+        zs = np.array([float(z[t, e]) for e in sel], dtype=np.float64)
+        ex = np.exp(zs - zs[0])
+        ids[t] = sel
+        w[t] = (ex / ex.sum()).astype(np.float32)
+    return ids, w
+
+
+# ---------------------------------------------------------------------------
+# Step 2: permutation of (token, choice) pairs by expert ("grouped evaluation")
+# ---------------------------------------------------------------------------
+
+def permute(ids: np.ndarray, n_experts: int):
+    """count[E], offset[E+1], perm[P], inv[P] of the stable expert-sorted order."""
+    keys = np.asarray(ids, dtype=np.int32).reshape(-1)
+    P = keys.shape[0]
+    count = np.zeros(n_experts, dtype=np.int32)
+    for p in range(P):
+        count[keys[p]] += 1
+    offset = np.zeros(n_experts + 1, dtype=np.int32)
+    for e in range(n_experts):
+        offset[e + 1] = offset[e] + count[e]
+    seen = np.zeros(n_experts, dtype=np.int32)
+    perm = np.empty(P, dtype=np.int32)
+    inv = np.empty(P, dtype=np.int32)
+    for p in range(P):
+        e = keys[p]
+        pos = offset[e] + seen[e]
+        seen[e] += 1
+        perm[pos] = p
+        inv[p] = pos
+    return count, offset, perm, inv
+
+
+# ---------------------------------------------------------------------------
+# Step 3: slot table, LRU bookkeeping and the miss split
+# ---------------------------------------------------------------------------
+
+@dataclasses.dataclass(frozen=True)
+class CostModel:
+    """Frozen integer constants of the plan (bandwidths in MB/s = 1e6 B/s)."""
+    expert_bytes: int
+    bw_fill: int                 # B_f : copy-engine fill rate (the paper's B_PCIe)
+    bw_zc_residual: int          # B_r : zero-copy rate left while fills saturate the link (Eq. 2)
+    bw_zc: int                   # B_z : zero-copy rate alone
+    bw_hbm: int                  # B_h : HBM streaming rate
+    reuse_credit: int = 1        # R   : future link passes a fill is credited with saving
+    zc_tokens_per_pass: int = 64     # T_z
+    hbm_tokens_per_pass: int = 128   # T_g
+
+    def ns(self, bw: int) -> int:
+        return (self.expert_bytes * 1000) // bw
+
+
+def fill_count_bw(m: int, bw_fill: int, bw_zc_residual: int) -> int:
+    """Eq. 4 with B_PCIe := B_f and B_Host := B_f + B_r, rounded half up, at least 1."""
+    if m <= 0:
+        return 0
+    bt = bw_fill + bw_zc_residual
+    return max(1, (2 * m * bw_fill + bt) // (2 * bt))
+
+
+@dataclasses.dataclass
+class Plan:
+    step: int
+    routed: list      # U, ascending
+    hit: list         # H, ascending
+    miss: list        # M, ascending
+    fill: list        # F, ascending
+    zc: list          # Z, ascending
+    fill_order: list  # F in priority order
+    fill_slot: list   # slot of fill_order[i]
+    fill_evicted: list  # expert evicted from that slot, -1 if it was free
+    loc: np.ndarray   # [E]: slot >= 0 | -1 not routed | -2 zero-copy
+
+
+class CacheState:
+    """Per-layer residency table (Sec. 3.2 "shared LRU residency space", here one per layer)."""
+
+    def __init__(self, n_experts: int, n_slots: int):
+        self.n_experts = n_experts
+        self.n_slots = n_slots
+        self.slot_expert = np.full(n_slots, -1, dtype=np.int32)
+        self.slot_stamp = np.full(n_slots, -1, dtype=np.int64)
+        self.expert_slot = np.full(n_experts, -1, dtype=np.int32)
+        self.step = 0
+
+    def reset(self):
+        self.slot_expert[:] = -1
+        self.slot_stamp[:] = -1
+        self.expert_slot[:] = -1
+        self.step = 0
+
+
+def plan(state: CacheState, count: np.ndarray, cm: CostModel) -> Plan | None:
+    """One step of the cache state machine.  Returns None (and changes nothing) if no
+    pair was routed (T = 0)."""
+    E = state.n_experts
+    count = np.asarray(count)
+    if int(count.sum()) == 0:
+        return None
+    t = state.step
+    # 1. unique routed experts, ascending
+    U = [e for e in range(E) if count[e] > 0]
+    # 2. hits refresh recency; the rest are the m unique misses
+    H = [e for e in U if state.expert_slot[e] >= 0]
+    M = [e for e in U if state.expert_slot[e] < 0]
+    for e in H:
+        state.slot_stamp[state.expert_slot[e]] = t
+    m = len(M)
+    # 3. victim candidates: every slot not touched in this step; free ones first
+    free = [s for s in range(state.n_slots) if state.slot_expert[s] < 0]
+    occ = [s for s in range(state.n_slots) if state.slot_expert[s] >= 0 and state.slot_stamp[s] < t]
+    occ.sort(key=lambda s: (int(state.slot_stamp[s]), int(state.slot_expert[s])))
+    V = free + occ
+    K = len(V)
+    # 4. per-expert eligibility: is filling cheaper than serving in place, counting R future passes
+    ns_z, ns_f, ns_h = cm.ns(cm.bw_zc), cm.ns(cm.bw_fill), cm.ns(cm.bw_hbm)
+    eligible = []
+    for e in M:
+        n_e = int(count[e])
+        pz = -(-n_e // cm.zc_tokens_per_pass)
+        pg = -(-n_e // cm.hbm_tokens_per_pass)
+        c_zc = pz * ns_z
+        c_fill = ns_f + pg * ns_h
+        v = c_zc - c_fill + cm.reuse_credit * (ns_z - ns_h)
+        if v > 0:
+            eligible.append(e)
+    # 5. how many to fill
+    q = min(fill_count_bw(m, cm.bw_fill, cm.bw_zc_residual), len(eligible), K)
+    # 6. which: most demanded first
+    eligible.sort(key=lambda e: (-int(count[e]), e))
+    F_order = eligible[:q]
+    Fset = set(F_order)
+    Z = [e for e in M if e not in Fset]
+    # 7. assignment: i-th fill takes the i-th candidate slot
+    fill_slot, fill_evicted = [], []
+    for i, e in enumerate(F_order):
+        s = V[i]
+        old = int(state.slot_expert[s])
+        if old >= 0:
+            state.expert_slot[old] = -1
+        state.slot_expert[s] = e
+        state.expert_slot[e] = s
+        state.slot_stamp[s] = t
+        fill_slot.append(s)
+        fill_evicted.append(old)
+    # 8. location of every expert for the execution step
+    loc = np.full(E, LOC_NOT_ROUTED, dtype=np.int32)
+    for e in H + F_order:
+        loc[e] = state.expert_slot[e]
+    for e in Z:
+        loc[e] = LOC_ZERO_COPY
+    state.step = t + 1
+    return Plan(step=t, routed=U, hit=H, miss=M, fill=sorted(F_order), zc=Z, fill_order=F_order,
+                fill_slot=fill_slot, fill_evicted=fill_evicted, loc=loc)
+
+
+# ---------------------------------------------------------------------------
+# Expert records -> matrices (the oracle's own reader of the pool format)
+# ---------------------------------------------------------------------------
+
+def _bf16_bits_to_f64(u16: np.ndarray) -> np.ndarray:
+    return (u16.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+
+
+def bf16_to_f64(a) -> np.ndarray:
+    """bf16 payload given as uint16 bit patterns (any shape) -> float64."""
+    return _bf16_bits_to_f64(np.asarray(a, dtype=np.uint16))
+
+
+def unpack_record(rec: np.ndarray, d: int, inter: int, wdtype: str):
+    """Record bytes -> (W_gate [d, I], W_up [d, I], W_down [I, d]) in float64.
+
+    bf16 record: three row-major [I][d] bf16 matrices (gate and up stored transposed,
+    i.e. one row per intermediate neuron), then nothing.
+    int4 record: the same three [I][d] matrices as 4-bit two's-complement codes, two per
+    byte along d (low nibble = even column), followed by bf16 scales sg[I][d/128],
+    su[I][d/128] (groups along the hidden index) and sd[I/128][d] (groups along the
+    neuron index); weight = scale * code.
+    """
+    rec = np.ascontiguousarray(rec).view(np.uint8).reshape(-1)
+    n = inter * d
+    if wdtype == "bf16":
+        assert rec.size == 3 * n * 2
+        m = _bf16_bits_to_f64(rec.view(np.uint16)).reshape(3, inter, d)
+        return m[0].T.copy(), m[1].T.copy(), m[2].copy()
+    if wdtype == "int4":
+        nb = n // 2
+        codes = []
+        for which in range(3):
+            b = rec[which * nb:(which + 1) * nb].reshape(inter, d // 2)
+            lo = (b & 0xF).astype(np.int16)
+            hi = (b >> 4).astype(np.int16)
+            q = np.empty((inter, d), dtype=np.int16)
+            q[:, 0::2] = lo
+            q[:, 1::2] = hi
+            q = np.where(q >= 8, q - 16, q)
+            codes.append(q.astype(np.float64))
+        off = 3 * nb
+        ng = inter * (d // GROUP)
+        sg = _bf16_bits_to_f64(rec[off:off + 2 * ng].view(np.uint16)).reshape(inter, d // GROUP)
+        off += 2 * ng
+        su = _bf16_bits_to_f64(rec[off:off + 2 * ng].view(np.uint16)).reshape(inter, d // GROUP)
+        off += 2 * ng
+        nd = (inter // GROUP) * d
+        sd = _bf16_bits_to_f64(rec[off:off + 2 * nd].view(np.uint16)).reshape(inter // GROUP, d)
+        off += 2 * nd
+        assert off == rec.size
+        wg = codes[0] * np.repeat(sg, GROUP, axis=1)
+        wu = codes[1] * np.repeat(su, GROUP, axis=1)
+        wd = codes[2] * np.repeat(sd, GROUP, axis=0)
+        return wg.T.copy(), wu.T.copy(), wd
+    raise ValueError(wdtype)
+
+
+# ---------------------------------------------------------------------------
+# Steps 5 and 6: SwiGLU expert FFN and the gate-weighted combine
+# ---------------------------------------------------------------------------
+
+def expert_ffn(x: np.ndarray, wg: np.ndarray, wu: np.ndarray, wd: np.ndarray) -> np.ndarray:
+    """o = (SiLU(x W_gate) * (x W_up)) W_down for rows of x; float64."""
+    g = x @ wg
+    u = x @ wu
+    h = g / (1.0 + np.exp(-g)) * u
+    return h @ wd
+
+
+def moe_layer(x_f64: np.ndarray, ids: np.ndarray, w: np.ndarray, get_expert, shared=()) -> np.ndarray:
+    """y[t] = sum_j w[t,j] * FFN_{ids[t,j]}(x[t]) + sum over shared experts FFN(x[t]).
+
+    ``get_expert(e)`` returns (W_gate, W_up, W_down) read from the *pool* by expert id,
+    so the result cannot depend on residency.  Accumulates in ascending j.
+    """
+    T, k = ids.shape
+    d = x_f64.shape[1]
+    outs = np.zeros((T, k, d), dtype=np.float64)
+    for e in sorted(set(int(v) for v in ids.reshape(-1))):
+        tj = np.argwhere(ids == e)
+        wg, wu, wd = get_expert(e)
+        o = expert_ffn(x_f64[tj[:, 0]], wg, wu, wd)
+        for r, (t, j) in enumerate(tj):
+            outs[t, j] = o[r]
+    y = np.zeros((T, d), dtype=np.float64)
+    for j in range(k):
+        y += w[:, j].astype(np.float64)[:, None] * outs[:, j]
+    for (wg, wu, wd) in shared:
+        y += expert_ffn(x_f64, wg, wu, wd)
+    return y
+
+
+# ---------------------------------------------------------------------------
+# The whole layer, step by step
+# ---------------------------------------------------------------------------
+
+@dataclasses.dataclass
+class StepResult:
+    ids: np.ndarray
+    w: np.ndarray
+    count: np.ndarray
+    offset: np.ndarray
+    perm: np.ndarray
+    inv: np.ndarray
+    plan: Plan | None
+    y: np.ndarray | None
+
+
+class OracleLayer:
+    """One MoE layer with its cache: route -> permute -> plan -> (fill) -> FFN -> combine."""
+
+    def __init__(self, d: int, inter: int, n_experts: int, top_k: int, n_slots: int,
+                 wdtype: str, pool_records, cm: CostModel, shared_records=()):
+        self.d, self.inter, self.E, self.k = d, inter, n_experts, top_k
+        self.wdtype = wdtype
+        self.pool = pool_records          # indexable by expert id -> record bytes
+        self.cm = cm
+        self.state = CacheState(n_experts, n_slots)
+        self.slots = [None] * n_slots     # bytes each slot would hold after the fills
+        self.shared = [unpack_record(r, d, inter, wdtype) for r in shared_records]
+
+    def get_expert(self, e: int):
+        return unpack_record(np.asarray(self.pool[e]), self.d, self.inter, self.wdtype)
+
+    def step(self, logits: np.ndarray, x_bf16_bits: np.ndarray | None, compute_y: bool = True) -> StepResult:
+        ids, w = route(logits, self.k)
+        count, offset, perm, inv = permute(ids, self.E)
+        p = plan(self.state, count, self.cm)
+        if p is not None:
+            for e, s in zip(p.fill_order, p.fill_slot):
+                self.slots[s] = e      # step 4: slot s now mirrors pool record e
+        y = None
+        if compute_y and x_bf16_bits is not None and ids.shape[0] > 0:
+            y = moe_layer(bf16_to_f64(x_bf16_bits), ids, w, self.get_expert, self.shared)
+        return StepResult(ids, w, count, offset, perm, inv, p, y)

@@ -1,0 +1,232 @@
+"""Seeded synthetic inputs for the expert-cached MoE layer.
+
+This module only *draws inputs*: expert-weight records, router logits and
+activations.  It contains none of the layer's arithmetic (no routing, no cache
+logic, no FFN, no dequantisation) so that the CPU oracle and the CUDA library
+can both be fed from it without sharing any of the method's code.  Everything
+is a pure function of an integer seed.
+
+Expert record formats (one contiguous record per (layer, expert); the pool is
+``n_layers * n_experts`` records back to back, record index ``l * E + e``, the
+flattened identifier of Sec. 4.2 of the paper):
+
+``bf16``  three row-major ``[I][d]`` bf16 matrices, in this order
+          ``Wg_t`` (``Wg_t[n][i] = W_gate[i][n]``), ``Wu_t`` (same for W_up),
+          ``Wd`` (``Wd[n][c] = W_down[n][c]``).  ``S = 3*I*d*2`` bytes.
+``int4``  the same three ``[I][d]`` matrices as 4-bit two's-complement codes
+          in [-8, 7], two per byte along ``d`` (low nibble = even column), then
+          bf16 scales: ``sg[I][d/128]``, ``su[I][d/128]`` (groups of 128
+          consecutive ``i``: the contraction dimension of gate/up) and
+          ``sd[I/128][d]`` (groups of 128 consecutive ``n``: the contraction
+          dimension of down).  ``S = 3*I*d/2 + (2*I*d/128 + (I/128)*d)*2``.
+
+The routing-logit recipes follow the workload descriptions: a Zipf-style
+popularity bias ``b_e = -alpha * ln(rank_e)`` with ``rank`` a seeded permutation
+of ``1..E`` per layer, and an AR(1) chain per (layer, batch row) with unit
+stationary variance, ``u_t = rho*u_{t-1} + sqrt(1-rho^2)*eps_t``, ``z_t = u_t + b``.
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+
+import numpy as np
+import torch
+
+GROUP = 128  # int4 quantisation group length along the contraction dimension
+
+
+@dataclasses.dataclass(frozen=True)
+class LayerShape:
+    d: int            # hidden size
+    inter: int        # expert intermediate size I
+    n_experts: int    # routed experts E
+    top_k: int
+    wdtype: str = "bf16"   # "bf16" | "int4"
+    n_shared: int = 0      # always-resident shared experts (0 or 1)
+
+    @property
+    def expert_bytes(self) -> int:
+        if self.wdtype == "bf16":
+            return 3 * self.inter * self.d * 2
+        if self.wdtype == "int4":
+            payload = 3 * self.inter * self.d // 2
+            scales = (2 * self.inter * (self.d // GROUP) + (self.inter // GROUP) * self.d) * 2
+            return payload + scales
+        raise ValueError(self.wdtype)
+
+
+# The shapes of the five workload configurations.
+TINY = LayerShape(d=256, inter=128, n_experts=8, top_k=2)
+QWEN3_30B = LayerShape(d=2048, inter=768, n_experts=128, top_k=8)
+DSV3_INT4 = LayerShape(d=7168, inter=2048, n_experts=256, top_k=8, wdtype="int4", n_shared=1)
+
+
+def mix64(*vals: int) -> int:
+    """splitmix64-style mix of a tuple of small integers into one 63-bit seed."""
+    h = 0x9E3779B97F4A7C15
+    for v in vals:
+        h = (h ^ (int(v) & 0xFFFFFFFFFFFFFFFF)) & 0xFFFFFFFFFFFFFFFF
+        h = (h + 0x9E3779B97F4A7C15) & 0xFFFFFFFFFFFFFFFF
+        h = ((h ^ (h >> 30)) * 0xBF58476D1CE4E5B9) & 0xFFFFFFFFFFFFFFFF
+        h = ((h ^ (h >> 27)) * 0x94D049BB133111EB) & 0xFFFFFFFFFFFFFFFF
+        h ^= h >> 31
+    return h & 0x7FFFFFFFFFFFFFFF
+
+
+_TAG_W, _TAG_RANK, _TAG_U0, _TAG_EPS, _TAG_X, _TAG_LOGIT = 1, 2, 3, 4, 5, 6
+
+
+def slots_for_fraction(frac: float, n_experts: int) -> int:
+    """Cache fraction -> slots per layer (rounded up)."""
+    return int(math.ceil(frac * n_experts - 1e-9))
+
+
+# --------------------------------------------------------------------------
+# expert weights
+# --------------------------------------------------------------------------
+
+def _gen(device, seed: int) -> torch.Generator:
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    return g
+
+
+def _quantise_int4(w: torch.Tensor, group_axis: int) -> tuple[torch.Tensor, torch.Tensor]:
+    """Symmetric int4 quantiser used to *produce* the synthetic pool.
+
+    ``w``: fp32 ``[n, I, d]``; groups of 128 along ``group_axis`` (1 or 2).
+    Returns (codes int8 in [-8,7] with w's shape, scales bf16 with the group
+    axis reduced by 128).
+    """
+    n, I, d = w.shape
+    if group_axis == 2:
+        wg = w.reshape(n, I, d // GROUP, GROUP)
+        amax = wg.abs().amax(dim=3)                              # [n, I, d/128]
+        scale = (amax / 7.0).to(torch.bfloat16)
+        sf = scale.to(torch.float32).unsqueeze(3)
+        q = torch.where(sf > 0, torch.round(wg / torch.where(sf > 0, sf, torch.ones_like(sf))),
+                        torch.zeros_like(wg))
+        q = q.clamp_(-8, 7).reshape(n, I, d)
+    else:
+        wg = w.reshape(n, I // GROUP, GROUP, d)
+        amax = wg.abs().amax(dim=2)                              # [n, I/128, d]
+        scale = (amax / 7.0).to(torch.bfloat16)
+        sf = scale.to(torch.float32).unsqueeze(2)
+        q = torch.where(sf > 0, torch.round(wg / torch.where(sf > 0, sf, torch.ones_like(sf))),
+                        torch.zeros_like(wg))
+        q = q.clamp_(-8, 7).reshape(n, I, d)
+    return q.to(torch.int8), scale
+
+
+def _pack_nibbles(q: torch.Tensor) -> torch.Tensor:
+    """int8 codes ``[..., d]`` -> uint8 ``[..., d/2]``, low nibble = even column."""
+    u = (q.to(torch.int16) & 0xF).to(torch.uint8)
+    return u[..., 0::2] | (u[..., 1::2] << 4)
+
+
+def make_records(shape: LayerShape, seed: int, layer: int, first: int, count: int,
+                 device="cpu", std: float = 0.02) -> torch.Tensor:
+    """Records of experts ``first .. first+count-1`` of ``layer`` as uint8 ``[count, S]``.
+
+    Record ``e`` depends only on (seed, layer, e) for a given device type, so a
+    pool may be produced in chunks of any size.
+    """
+    I, d = shape.inter, shape.d
+    out = torch.empty((count, shape.expert_bytes), dtype=torch.uint8, device=device)
+    for j in range(count):
+        g = _gen(device, mix64(seed, _TAG_W, layer, first + j))
+        w = torch.randn((3, I, d), generator=g, device=device, dtype=torch.float32) * std
+        if shape.wdtype == "bf16":
+            out[j] = w.to(torch.bfloat16).reshape(-1).view(torch.uint8)
+        else:
+            qg, sg = _quantise_int4(w[0:1], 2)
+            qu, su = _quantise_int4(w[1:2], 2)
+            qd, sd = _quantise_int4(w[2:3], 1)
+            parts = [_pack_nibbles(qg).reshape(-1), _pack_nibbles(qu).reshape(-1),
+                     _pack_nibbles(qd).reshape(-1),
+                     sg.reshape(-1).view(torch.uint8), su.reshape(-1).view(torch.uint8),
+                     sd.reshape(-1).view(torch.uint8)]
+            out[j] = torch.cat(parts)
+    return out
+
+
+def fill_pool(pool: torch.Tensor, shape: LayerShape, n_layers: int, seed: int,
+              device="cpu", chunk: int = 16, n_per_layer: int | None = None) -> None:
+    """Write all records of ``n_layers`` layers into ``pool`` (uint8, host)."""
+    S = shape.expert_bytes
+    E = shape.n_experts if n_per_layer is None else n_per_layer
+    assert pool.dtype == torch.uint8 and pool.numel() >= n_layers * E * S
+    view = pool[: n_layers * E * S].view(n_layers * E, S)
+    for l in range(n_layers):
+        for first in range(0, E, chunk):
+            cnt = min(chunk, E - first)
+            rec = make_records(shape, seed, l, first, cnt, device=device)
+            view[l * E + first: l * E + first + cnt].copy_(rec)
+    if torch.device(device).type == "cuda":
+        torch.cuda.synchronize()
+
+
+def make_shared_records(shape: LayerShape, n_layers: int, seed: int, device="cpu") -> torch.Tensor:
+    """Records of the always-resident shared expert of each layer, uint8 ``[L, S]`` (host)."""
+    recs = [make_records(shape, seed, l, shape.n_experts, 1, device=device).cpu() for l in range(n_layers)]
+    return torch.cat(recs, dim=0).contiguous()
+
+
+# --------------------------------------------------------------------------
+# router logits
+# --------------------------------------------------------------------------
+
+def zipf_bias(n_experts: int, alpha: float, seed: int, layer: int) -> np.ndarray:
+    """``b_e = -alpha * ln(rank_e)``, rank a seeded permutation of 1..E (float64)."""
+    rng = np.random.Generator(np.random.PCG64(mix64(seed, _TAG_RANK, layer)))
+    rank = rng.permutation(n_experts) + 1
+    return -alpha * np.log(rank.astype(np.float64))
+
+
+def ar1_logits(n_layers: int, n_steps: int, batch: int, n_experts: int, rho: float,
+               alpha: float, seed: int) -> np.ndarray:
+    """Decode logits, float32 ``[n_steps, n_layers, batch, E]``.
+
+    One chain per (layer, batch row): ``u_0 ~ N(0,1)``,
+    ``u_t = rho*u_{t-1} + sqrt(1-rho^2)*eps_t``, ``z_t = u_t + b_layer``.
+    """
+    out = np.empty((n_steps, n_layers, batch, n_experts), dtype=np.float32)
+    s = math.sqrt(max(0.0, 1.0 - rho * rho))
+    for l in range(n_layers):
+        b = zipf_bias(n_experts, alpha, seed, l)
+        rng = np.random.Generator(np.random.PCG64(mix64(seed, _TAG_U0, l, batch)))
+        u = rng.standard_normal((batch, n_experts))
+        for t in range(n_steps):
+            if t > 0:
+                u = rho * u + s * rng.standard_normal((batch, n_experts))
+            out[t, l] = (u + b).astype(np.float32)
+    return out
+
+
+def prefill_logits(n_layers: int, n_tokens: int, n_experts: int, alpha: float, seed: int,
+                   step: int = 0) -> np.ndarray:
+    """Prefill logits ``eps + b``, float32 ``[n_layers, T, E]``."""
+    out = np.empty((n_layers, n_tokens, n_experts), dtype=np.float32)
+    for l in range(n_layers):
+        b = zipf_bias(n_experts, alpha, seed, l)
+        rng = np.random.Generator(np.random.PCG64(mix64(seed, _TAG_LOGIT, l, step)))
+        out[l] = (rng.standard_normal((n_tokens, n_experts)) + b).astype(np.float32)
+    return out
+
+
+def normal_logits(n_tokens: int, n_experts: int, seed: int, step: int) -> np.ndarray:
+    """Fresh ``N(0,1)`` logits per step (the tiny configuration), float32 ``[T, E]``."""
+    rng = np.random.Generator(np.random.PCG64(mix64(seed, _TAG_LOGIT, 0, step)))
+    return rng.standard_normal((n_tokens, n_experts)).astype(np.float32)
+
+
+# --------------------------------------------------------------------------
+# activations
+# --------------------------------------------------------------------------
+
+def noise_x(n_tokens: int, d: int, seed: int, step: int, layer: int, device="cpu") -> torch.Tensor:
+    """``N(0,1)`` noise rows as bf16 ``[T, d]``; the layer input is this noise plus
+    (for layer > 0) the previous layer's output, rounded to bf16 by the caller."""
+    g = _gen(device, mix64(seed, _TAG_X, step, layer))
+    return torch.randn((n_tokens, d), generator=g, device=device, dtype=torch.float32).to(torch.bfloat16)

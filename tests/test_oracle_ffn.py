@@ -1,0 +1,160 @@
+"""Pins for the oracle's record reader, expert FFN and combine (CPU only)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ftmoe_oracle as O
+from paper_2608_16157_b200 import workload as W
+
+
+def _bf16_bits(a: np.ndarray) -> np.ndarray:
+    """float -> bf16 bit patterns via torch's round-to-nearest-even (a library routine)."""
+    t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(torch.bfloat16)
+    return t.view(torch.int16).numpy().view(np.uint16)
+
+
+def _record_bf16_by_definition(wg, wu, wd):
+    """Build a record straight from the documented layout with explicit loops over (n, i)."""
+    d, I = wg.shape
+    rec = np.zeros(3 * I * d, dtype=np.uint16)
+    gb, ub, db = _bf16_bits(wg), _bf16_bits(wu), _bf16_bits(wd)
+    for n in range(I):
+        for i in range(d):
+            rec[0 * I * d + n * d + i] = gb[i, n]
+            rec[1 * I * d + n * d + i] = ub[i, n]
+            rec[2 * I * d + n * d + i] = db[n, i]
+    return rec.view(np.uint8)
+
+
+def test_unpack_bf16_record_orientation():
+    d, I = 16, 8
+    wg = np.arange(d * I, dtype=np.float32).reshape(d, I) / 4.0        # all exactly representable
+    wu = -np.arange(d * I, dtype=np.float32).reshape(d, I) / 8.0
+    wd = (np.arange(I * d, dtype=np.float32).reshape(I, d) % 31) - 15.0
+    g, u, dn = O.unpack_record(_record_bf16_by_definition(wg, wu, wd), d, I, "bf16")
+    assert np.array_equal(g, wg) and np.array_equal(u, wu) and np.array_equal(dn, wd)
+
+
+def _record_int4_by_definition(qg, qu, qd, sg, su, sd):
+    """qX: int codes [I][d] in stored orientation; sg/su [I][d/128]; sd [I/128][d] (floats, bf16-exact)."""
+    I, d = qg.shape
+    out = bytearray()
+    for q in (qg, qu, qd):
+        for n in range(I):
+            for c in range(0, d, 2):
+                out.append((int(q[n, c]) & 0xF) | ((int(q[n, c + 1]) & 0xF) << 4))
+    for s in (sg, su, sd):
+        out += _bf16_bits(s).tobytes()
+    return np.frombuffer(bytes(out), dtype=np.uint8)
+
+
+def test_unpack_int4_record_by_definition():
+    rng = np.random.default_rng(0)
+    d, I = 256, 128
+    qg, qu, qd = (rng.integers(-8, 8, size=(I, d)) for _ in range(3))
+    sg = rng.integers(1, 9, size=(I, d // 128)).astype(np.float32) / 64.0
+    su = rng.integers(1, 9, size=(I, d // 128)).astype(np.float32) / 32.0
+    sd = rng.integers(1, 9, size=(I // 128, d)).astype(np.float32) / 16.0
+    rec = _record_int4_by_definition(qg, qu, qd, sg, su, sd)
+    assert rec.size == W.LayerShape(d, I, 1, 1, "int4").expert_bytes
+    wg, wu, wd = O.unpack_record(rec, d, I, "int4")
+    for n in (0, 5, 127):
+        for i in (0, 1, 127, 128, 255):
+            assert wg[i, n] == qg[n, i] * sg[n, i // 128]
+            assert wu[i, n] == qu[n, i] * su[n, i // 128]
+            assert wd[n, i] == qd[n, i] * sd[n // 128, i]
+    # all-zero codes give zero weights; code 1 with scale 1 gives column sums of x
+    z = np.zeros((I, d), dtype=np.int64)
+    one = np.ones((I, d), dtype=np.int64)
+    s1g = np.ones((I, d // 128), dtype=np.float32)
+    s1d = np.ones((I // 128, d), dtype=np.float32)
+    wg0, wu0, wd0 = O.unpack_record(_record_int4_by_definition(z, z, z, s1g, s1g, s1d), d, I, "int4")
+    assert not wg0.any() and not wu0.any() and not wd0.any()
+    wg1, _, _ = O.unpack_record(_record_int4_by_definition(one, one, one, s1g, s1g, s1d), d, I, "int4")
+    x = rng.standard_normal((3, d))
+    np.testing.assert_allclose(x @ wg1, np.repeat(x.sum(axis=1, keepdims=True), I, axis=1), rtol=1e-12)
+
+
+def test_generated_int4_pool_quantiser_error_bound():
+    shape = W.LayerShape(d=256, inter=128, n_experts=2, top_k=1, wdtype="int4")
+    rec = W.make_records(shape, seed=0, layer=0, first=0, count=1)[0].numpy()
+    wg, wu, wd = O.unpack_record(rec, 256, 128, "int4")
+    # regenerate the fp32 draws and check |w - deq(w)| <= scale/2 (+ bf16 rounding of the scale)
+    g = torch.Generator().manual_seed(W.mix64(0, 1, 0, 0))
+    w = (torch.randn((3, 128, 256), generator=g) * 0.02).double().numpy()
+    for got, ref, axis in ((wg.T, w[0], 1), (wu.T, w[1], 1), (wd, w[2], 0)):
+        amax = np.abs(ref).reshape((128, 2, 128) if axis == 1 else (1, 128, 256)).max(axis=2 if axis == 1 else 1)
+        bound = np.repeat(amax / 7.0, 128, axis=axis) * (0.5 + 7 * 2.0 ** -8) + 1e-12
+        assert np.all(np.abs(got - ref) <= bound)
+
+
+def test_single_expert_is_library_swiglu_mlp():
+    rng = np.random.default_rng(1)
+    d, I, T = 32, 24, 5
+    x = rng.standard_normal((T, d))
+    wg, wu, wd = rng.standard_normal((d, I)), rng.standard_normal((d, I)), rng.standard_normal((I, d))
+    xt = torch.from_numpy(x)
+    ref = (torch.nn.functional.silu(xt @ torch.from_numpy(wg)) * (xt @ torch.from_numpy(wu))) @ torch.from_numpy(wd)
+    np.testing.assert_allclose(O.expert_ffn(x, wg, wu, wd), ref.numpy(), rtol=1e-12, atol=1e-12)
+    ids = np.zeros((T, 1), dtype=np.int32)
+    w = np.ones((T, 1), dtype=np.float32)
+    y = O.moe_layer(x, ids, w, lambda e: (wg, wu, wd))
+    np.testing.assert_allclose(y, ref.numpy(), rtol=1e-12, atol=1e-12)
+
+
+def _dense_moe(x, logits, k, experts):
+    """Uncached dense MoE: every expert evaluated for every token, weighted by the masked gate."""
+    T, E = logits.shape
+    z = torch.from_numpy(logits).double()
+    top = torch.topk(z, k, dim=1)
+    gate = torch.zeros(T, E, dtype=torch.float64)
+    gate.scatter_(1, top.indices, torch.softmax(top.values, dim=1))
+    y = np.zeros_like(x)
+    for e, (wg, wu, wd) in enumerate(experts):
+        xt = torch.from_numpy(x)
+        o = (torch.nn.functional.silu(xt @ torch.from_numpy(wg)) * (xt @ torch.from_numpy(wu))) @ torch.from_numpy(wd)
+        y += gate[:, e:e + 1].numpy() * o.numpy()
+    return y
+
+
+def test_cached_layer_equals_dense_uncached_moe_for_any_slot_count():
+    shape = W.LayerShape(d=256, inter=128, n_experts=8, top_k=2)
+    pool = W.make_records(shape, seed=0, layer=0, first=0, count=8).numpy()
+    experts = [O.unpack_record(pool[e], 256, 128, "bf16") for e in range(8)]
+    cm = O.CostModel(shape.expert_bytes, 50000, 0, 50000, 6000000)
+    ys = {}
+    for n_slots in (0, 4, 8):
+        layer = O.OracleLayer(256, 128, 8, 2, n_slots, "bf16", pool, cm)
+        out = []
+        for step in range(3):
+            logits = W.normal_logits(8, 8, 0, step)      # continuous: no ties, torch.topk agrees
+            xb = W.noise_x(8, 256, 0, step, 0).view(torch.int16).numpy().view(np.uint16)
+            r = layer.step(logits, xb)
+            ref = _dense_moe(O.bf16_to_f64(xb), logits, 2, experts)
+            np.testing.assert_allclose(r.y, ref, rtol=1e-6, atol=1e-8)   # gate weights are rounded to fp32
+            out.append(r.y)
+        ys[n_slots] = out
+    for step in range(3):
+        assert np.array_equal(ys[0][step], ys[4][step]) and np.array_equal(ys[4][step], ys[8][step])
+
+
+def test_algebraic_properties_of_the_layer():
+    rng = np.random.default_rng(2)
+    d, I, E, k, T = 16, 12, 5, 3, 7
+    x = rng.standard_normal((T, d))
+    logits = rng.standard_normal((T, E)).astype(np.float32)
+    ids, w = O.route(logits, k)
+    same = (rng.standard_normal((d, I)), rng.standard_normal((d, I)), rng.standard_normal((I, d)))
+    # identical experts: the gate weights sum to one, so y = FFN(x)
+    y = O.moe_layer(x, ids, w, lambda e: same)
+    np.testing.assert_allclose(y, O.expert_ffn(x, *same), rtol=1e-6, atol=1e-6)
+    # W_down = 0 -> 0 ; scaling W_down scales y
+    experts = [(rng.standard_normal((d, I)), rng.standard_normal((d, I)), rng.standard_normal((I, d))) for _ in range(E)]
+    y0 = O.moe_layer(x, ids, w, lambda e: (experts[e][0], experts[e][1], 0 * experts[e][2]))
+    assert not y0.any()
+    y1 = O.moe_layer(x, ids, w, lambda e: experts[e])
+    y3 = O.moe_layer(x, ids, w, lambda e: (experts[e][0], experts[e][1], 3.0 * experts[e][2]))
+    np.testing.assert_allclose(y3, 3.0 * y1, rtol=1e-12)
+    # a shared expert adds its FFN with weight one
+    ys = O.moe_layer(x, ids, w, lambda e: experts[e], shared=[same])
+    np.testing.assert_allclose(ys - y1, O.expert_ffn(x, *same), rtol=1e-9, atol=1e-9)
