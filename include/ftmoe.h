@@ -1,0 +1,200 @@
+/*
+ * ftmoe.h -- C ABI of the expert-cached Mixture-of-Experts layer for NVIDIA B200 (sm_100a).
+ *
+ * The library implements one thing: the MoE layer of an engine whose complete routed-expert
+ * weights live in a pinned host pool (the source of truth) while a fixed pool of HBM slots caches
+ * the experts in use (paper Sec. 3: two-level expert-memory hierarchy; each slot holds every tensor
+ * of one (layer, expert) pair).  Per step and layer the caller runs
+ *
+ *     ft_moe_route -> ft_moe_plan -> ft_moe_fill -> ft_moe_forward
+ *
+ * route   : top-k gating with softmax over the selected logits, stable expert-sorted permutation.
+ * plan    : slot-table lookup gives the hit set H; the m unique misses M are split into a fill set
+ *           F (|F| = q, Eq. 1 and Eq. 4 of the paper) and an in-place set served by zero-copy reads
+ *           of the mapped host pool (the paper's CPU branch, kept on the GPU here); LRU victims.
+ * fill    : copies pool records of F into their slots over the host link.
+ * forward : grouped SwiGLU expert FFN over H u F (from slots) and Z (from host), gate-weighted sum.
+ *
+ * Conventions
+ *   - Every function returns an ft_status_t, never aborts, never throws, never traps on the device.
+ *   - "dev" pointers are device pointers, "host" pointers are host pointers; streams are
+ *     cudaStream_t passed as void*.  One host thread per handle.
+ *   - Asynchronous device-detected conditions (non-finite logits) are latched in a device status
+ *     word and reported by the next synchronising call (ft_moe_plan with a non-null out pointer,
+ *     ft_moe_fill in copy-engine mode, the ft_moe_get_* calls, ft_moe_sync_status).
+ *   - T = 0 is a no-op that does not advance the layer's step counter.
+ *
+ * Expert record layout (pool records and slots are byte-identical, so a fill is one contiguous copy)
+ *   record index in the pool: layer * n_experts + expert (the flattened id of paper Sec. 4.2).
+ *   FT_W_BF16     : three row-major [inter][hidden] bf16 matrices, in this order:
+ *                     Wg_t  (Wg_t[n][i] = W_gate[i][n]),  Wu_t (Wu_t[n][i] = W_up[i][n]),
+ *                     Wd    (Wd[n][c]   = W_down[n][c]).          S = 3*inter*hidden*2 bytes.
+ *   FT_W_INT4_G128: the same three [inter][hidden] matrices as 4-bit two's-complement codes in
+ *                   [-8,7], two per byte along hidden (low nibble = even column), followed by bf16
+ *                   scales sg[inter][hidden/128], su[inter][hidden/128] (groups of 128 consecutive
+ *                   hidden indices: the contraction dimension of gate/up) and sd[inter/128][hidden]
+ *                   (groups of 128 consecutive neurons: the contraction dimension of down);
+ *                   weight = scale * code.
+ *   Shape limits: bf16: hidden in {256, 512, 1024, 2048}, inter % 64 == 0; int4: hidden % 512 == 0,
+ *   hidden <= 8192, inter % 128 == 0; n_experts <= 1024; top_k <= min(n_experts, 32);
+ *   slots_per_layer <= 2048.
+ */
+#ifndef FTMOE_H_
+#define FTMOE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ft_moe ft_moe_t; /* opaque: owns the slot pool, the tables, scratch, events */
+
+typedef enum {
+  FT_OK = 0,
+  FT_ERR_INVALID_ARG = 1,
+  FT_ERR_NOT_PINNED = 2,   /* host_pool is not pinned + mapped host memory (no pageable fallback) */
+  FT_ERR_OOM = 3,
+  FT_ERR_CUDA = 4,
+  FT_ERR_STATE = 5,        /* calls out of order for this layer */
+  FT_ERR_TIMEOUT = 6,      /* a bounded device-side wait gave up */
+  FT_ERR_NONFINITE = 7,    /* NaN/Inf in the router logits */
+  FT_ERR_UNSUPPORTED = 8
+} ft_status_t;
+
+typedef enum { FT_W_BF16 = 0, FT_W_INT4_G128 = 1 } ft_wdtype_t;
+
+/* How ft_moe_fill moves records.  Both give byte-identical slots. */
+typedef enum {
+  FT_FILL_COPY_ENGINE = 0, /* host waits for the plan record, then one cudaMemcpyAsync per fill */
+  FT_FILL_SM = 1           /* one fixed-shape copy kernel driven by the device-resident fill list
+                              (paper Sec. 4.1: a work list plus a valid count); no host wait */
+} ft_fill_mode_t;
+
+typedef struct {
+  uint32_t struct_size;     /* = sizeof(ft_moe_config_t) */
+  int32_t device;           /* CUDA device ordinal */
+  int32_t n_layers;
+  int32_t hidden;           /* d */
+  int32_t inter;            /* I */
+  int32_t n_experts;        /* E routed experts per layer */
+  int32_t top_k;
+  int32_t n_shared;         /* 0 or 1 always-resident shared expert per layer */
+  int32_t wdtype;           /* ft_wdtype_t */
+  int32_t slots_per_layer;  /* N_s >= 0; 0 = every routed expert is served zero-copy */
+  int32_t max_tokens;       /* largest T of any call */
+  int32_t fill_mode;        /* ft_fill_mode_t */
+  const void *host_pool;    /* HOST, caller-owned, pinned + mapped, n_layers*n_experts records;
+                               must stay valid and unmodified for the life of the handle */
+  size_t host_pool_bytes;
+  const void *shared_weights; /* HOST, n_layers*n_shared records, copied to HBM at create; may be
+                                 NULL when n_shared == 0 */
+  /* Frozen integer constants of the plan's cost model, MB/s (1e6 bytes/s); all must be > 0 except
+   * bw_zc_residual_MBps which may be 0 (then every miss that can get a slot is filled: the paper's
+   * degenerate "pure on-demand cache fill", text after Eq. 4). */
+  uint32_t bw_fill_MBps;        /* B_f: copy-engine fill rate            (the paper's B_PCIe)      */
+  uint32_t bw_zc_MBps;          /* B_z: zero-copy read rate alone                                   */
+  uint32_t bw_zc_residual_MBps; /* B_r: zero-copy rate while fills saturate the link (Eq. 2)        */
+  uint32_t bw_hbm_MBps;         /* B_h: HBM streaming rate                                          */
+  int32_t reuse_credit;         /* R >= 0: future link passes a fill is credited with saving        */
+  int32_t zc_tokens_per_pass;   /* T_z >= 1: tokens one zero-copy weight pass serves                */
+  int32_t hbm_tokens_per_pass;  /* T_g >= 1: tokens one resident weight pass serves                 */
+  int32_t gemm_min_tokens;      /* experts with at least this many tokens and a slot use the
+                                   tensor-core grouped GEMM; 0 = never                              */
+} ft_moe_config_t;
+
+/* Host-visible plan of one (layer, step).  The caller provides arrays of n_experts int32 each. */
+typedef struct {
+  int64_t step;
+  int32_t n_routed, n_hit, n_miss, n_fill, n_zc;
+  int32_t *hit, *miss, *fill, *zc;  /* ascending expert ids */
+  int32_t *fill_order;              /* F in priority order */
+  int32_t *fill_slot;               /* slot of fill_order[i] */
+  int32_t *fill_evicted;            /* expert evicted from that slot, -1 if it was free */
+  int32_t *loc;                     /* [n_experts]: slot >= 0 | -1 not routed | -2 zero-copy */
+} ft_moe_plan_t;
+
+enum { FT_STAT_STEPS = 0, FT_STAT_ROUTED, FT_STAT_HITS, FT_STAT_MISSES, FT_STAT_FILLS, FT_STAT_ZC,
+       FT_STAT_EVICTIONS, FT_STAT_PAIRS, FT_STAT_PAIRS_RESIDENT, FT_STAT_COUNT };
+
+/* S, the bytes of one expert record for this configuration (0 if the shape is not supported). */
+size_t ft_moe_expert_bytes(const ft_moe_config_t *cfg);
+
+/* Pinned + mapped host memory for an expert pool (cudaHostAlloc, portable | mapped).  HOST pointer
+ * out; free with ft_moe_host_free.  Contents are uninitialised. */
+ft_status_t ft_moe_host_alloc(size_t bytes, void **out_host);
+ft_status_t ft_moe_host_free(void *host);
+
+/* Validates the configuration, checks that host_pool is pinned and mapped (else FT_ERR_NOT_PINNED),
+ * allocates n_layers*slots_per_layer slots (FT_ERR_OOM if HBM cannot hold them) and empty tables
+ * (paper Sec. 3.3: the first request is served with a cold cache). */
+ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out);
+ft_status_t ft_moe_destroy(ft_moe_t *h);
+
+/* Bandwidth profiling at deployment (paper Sec. 3.2, "empirically profiled on the target
+ * hardware"): out_MBps = { fill (pinned H2D copy of records), zero-copy alone, zero-copy while the
+ * copy engine is saturated, HBM streaming }.  Measures only; plans keep using the frozen constants
+ * given at create.  Synchronises the device. */
+ft_status_t ft_moe_calibrate(ft_moe_t *h, uint32_t out_MBps[4]);
+
+/* Step 1+2 (paper Sec. 3.2: the router runs on the GPU).  logits_dev: DEVICE fp32 [T][n_experts]
+ * row-major.  Produces, on the device: ids[T][k] (logit descending, id ascending), gate weights
+ * w[T][k] = softmax over the selected logits, count[E], offset[E+1], and the stable expert-sorted
+ * permutation perm[P] / inv[P] of the P = T*k pairs p = t*k + j. */
+ft_status_t ft_moe_route(ft_moe_t *h, int layer, const float *logits_dev, int T, void *stream);
+
+/* Step 3 (paper Sec. 3.2 Eq. 1-4 and Sec. 4.1 "device-side cache control"): one device kernel
+ * deduplicates the routed experts, classifies them against the slot table, refreshes the stamps of
+ * hits, orders the evictable slots (free first, then least recently used, ties to the lower
+ * resident expert id), sizes the fill set q = min(max(1, round(m*B_f/(B_f+B_r))), eligible, K),
+ * picks F (most tokens first), assigns slots, and rewrites expert ids into slot ids or the
+ * zero-copy flag.  out_host may be NULL (no synchronisation); otherwise the call waits for the
+ * plan and fills *out_host (HOST arrays owned by the caller). */
+ft_status_t ft_moe_plan(ft_moe_t *h, int layer, ft_moe_plan_t *out_host, void *stream);
+
+/* Step 4: for every (expert, slot) of F copy the S-byte pool record into the slot on copy_stream
+ * and record the handle's fill event there.  The copies are ordered after the plan. */
+ft_status_t ft_moe_fill(ft_moe_t *h, int layer, void *copy_stream);
+
+/* Steps 5+6: x_dev DEVICE bf16 [T][hidden], y_dev DEVICE bf16 [T][hidden] (written).  Waits (on the
+ * stream, not the host) for the fill event, evaluates the SwiGLU expert FFN of every routed expert
+ * from its slot or, for the zero-copy set, straight from the mapped host pool, and writes
+ * y[t] = sum_j w[t][j] * FFN_{ids[t][j]}(x[t]) (+ the shared expert) rounded once to bf16. */
+ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_dev, void *stream);
+
+/* route + plan + fill + forward of one layer in one call; fills go to the handle's own copy
+ * stream. */
+ft_status_t ft_moe_layer(ft_moe_t *h, int layer, const float *logits_dev, const void *x_dev,
+                         void *y_dev, int T, void *stream);
+
+/* The same through HOST buffers (pinned or pageable): copies logits and x to the device, runs the
+ * layer, copies y back and waits for it. */
+ft_status_t ft_moe_layer_host(ft_moe_t *h, int layer, const float *logits_host, const void *x_host,
+                              void *y_host, int T, void *stream);
+
+/* ---- introspection (tests, reports); each synchronises the device ---- */
+/* Results of the latest ft_moe_route on this handle, which must have been for `layer`.  HOST arrays:
+ * ids[T*k], w[T*k], count[E], offset[E+1], perm[T*k], inv[T*k]; any may be NULL. */
+ft_status_t ft_moe_get_routing(ft_moe_t *h, int layer, int32_t *ids, float *w, int32_t *count,
+                               int32_t *offset, int32_t *perm, int32_t *inv);
+/* HOST arrays slot_expert[N_s] (-1 free), slot_stamp[N_s] (-1 never used), expert_slot[E]. */
+ft_status_t ft_moe_get_slot_table(ft_moe_t *h, int layer, int32_t *slot_expert,
+                                  int64_t *slot_stamp, int32_t *expert_slot);
+ft_status_t ft_moe_read_slot(ft_moe_t *h, int layer, int slot, void *host_dst /* S bytes */);
+/* counters[FT_STAT_*], accumulated since create/reset. */
+ft_status_t ft_moe_get_stats(ft_moe_t *h, int layer, uint64_t *counters, int n);
+/* Empties the slot table and zeroes step counter and statistics; layer = -1 for all layers. */
+ft_status_t ft_moe_reset(ft_moe_t *h, int layer);
+/* Waits for the device and returns (and clears) the latched device status. */
+ft_status_t ft_moe_sync_status(ft_moe_t *h);
+/* Duration of the most recent ft_moe_fill's copies in microseconds and their bytes (waits for them). */
+ft_status_t ft_moe_last_fill(ft_moe_t *h, float *out_us, uint64_t *out_bytes);
+/* Number of kernels this handle has launched since create. */
+ft_status_t ft_moe_launch_count(ft_moe_t *h, uint64_t *out);
+const char *ft_moe_status_string(ft_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FTMOE_H_ */

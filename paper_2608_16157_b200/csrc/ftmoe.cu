@@ -1,0 +1,723 @@
+// Host side of the C ABI declared in include/ftmoe.h: handle, validation, launches, streams, events.
+#include "../../include/ftmoe.h"
+
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+#include "ffn_stream.cuh"
+#include "fill.cuh"
+#include "plan.cuh"
+#include "route.cuh"
+
+using namespace ftmoe;
+
+namespace {
+
+enum LayerPhase { PH_IDLE = 0, PH_ROUTED, PH_PLANNED, PH_FILLED };
+
+struct LayerState {
+  int32_t *slot_expert = nullptr;
+  int64_t *slot_stamp = nullptr;
+  int32_t *expert_slot = nullptr;
+  int64_t *step = nullptr;
+  unsigned long long *stats = nullptr;
+  int phase = PH_IDLE;
+  int T = 0;
+};
+
+}  // namespace
+
+struct ft_moe {
+  ft_moe_config_t cfg;
+  size_t S = 0;
+  int sm_count = 148;
+  // memory
+  uint8_t *slots = nullptr;         // [L][N_s][S]
+  uint8_t *shared_dev = nullptr;    // [L][n_shared][S]
+  const uint8_t *pool_dev = nullptr;  // device alias of host_pool
+  uint8_t *tables = nullptr;        // one allocation for all per-layer tables
+  size_t tables_bytes = 0;
+  std::vector<LayerState> layers;
+  // per-handle scratch (layers are stream-ordered, so one set serves all)
+  int32_t *ids = nullptr, *count = nullptr, *offset = nullptr, *perm = nullptr, *inv = nullptr;
+  float *topk_w = nullptr;
+  float *y_acc = nullptr;
+  PlanHeader *plan_dev = nullptr;
+  PlanHeader *plan_host = nullptr;      // pinned, mapped
+  PlanHeader *plan_host_devptr = nullptr;
+  size_t plan_bytes = 0;
+  WorkItem *items_res = nullptr, *items_zc = nullptr, *items_gemm = nullptr;
+  uint32_t *status_dev = nullptr;
+  uint32_t *seq_dev = nullptr;
+  uint32_t seq_host = 0;                // plans launched
+  float *stage_logits = nullptr;
+  __nv_bfloat16 *stage_x = nullptr, *stage_y = nullptr;
+  // streams / events
+  cudaStream_t copy_stream = nullptr, aux_stream = nullptr;
+  cudaEvent_t ev_plan = nullptr, ev_fill = nullptr, ev_fork = nullptr, ev_join = nullptr;
+  cudaEvent_t ev_fill_t0 = nullptr, ev_fill_t1 = nullptr;
+  uint64_t last_fill_bytes = 0;
+  bool fill_timed = false;
+  int last_routed_layer = -1;
+  uint64_t launches = 0;
+};
+
+namespace {
+
+#define FT_CUDA(expr)                                                                     \
+  do {                                                                                    \
+    cudaError_t e_ = (expr);                                                              \
+    if (e_ != cudaSuccess) {                                                              \
+      if (e_ == cudaErrorMemoryAllocation) { (void)cudaGetLastError(); return FT_ERR_OOM; } \
+      return FT_ERR_CUDA;                                                                 \
+    }                                                                                     \
+  } while (0)
+
+size_t expert_bytes_of(const ft_moe_config_t *c) {
+  if (!c || c->hidden <= 0 || c->inter <= 0) return 0;
+  const size_t d = (size_t)c->hidden, I = (size_t)c->inter;
+  if (c->wdtype == FT_W_BF16) {
+    if (d % 256 || d > 2048 || I % 8) return 0;
+    return 3 * I * d * 2;
+  }
+  if (c->wdtype == FT_W_INT4_G128) {
+    if (d % 512 || d > 8192 || I % 128) return 0;
+    return 3 * I * d / 2 + (2 * I * (d / 128) + (I / 128) * d) * 2;
+  }
+  return 0;
+}
+
+// threads across a row, row groups, threads per CTA of the streaming kernel
+void stream_geometry(const ft_moe_config_t &c, int &CT, int &G) {
+  const int epl = (c.wdtype == FT_W_BF16) ? 8 : 16;
+  CT = c.hidden / epl;
+  G = (CT >= 256) ? 1 : 256 / CT;
+}
+
+bool geometry_ok(const ft_moe_config_t &c) {
+  int CT, G;
+  stream_geometry(c, CT, G);
+  if (CT % 32 || CT > (c.wdtype == FT_W_BF16 ? 256 : 512)) return false;
+  if (CT < 256 && (256 % CT)) return false;
+  if (c.inter % (8 * G)) return false;
+  return true;
+}
+
+ft_status_t drain_status(ft_moe *h) {
+  uint32_t st = 0;
+  FT_CUDA(cudaMemcpy(&st, h->status_dev, sizeof(st), cudaMemcpyDeviceToHost));
+  if (st) {
+    FT_CUDA(cudaMemset(h->status_dev, 0, sizeof(st)));
+    if (st & kStatNonFinite) return FT_ERR_NONFINITE;
+    if (st & kStatTimeout) return FT_ERR_TIMEOUT;
+    return FT_ERR_CUDA;
+  }
+  return FT_OK;
+}
+
+ft_status_t reset_layer(ft_moe *h, int l) {
+  LayerState &L = h->layers[l];
+  const int Ns = h->cfg.slots_per_layer, E = h->cfg.n_experts;
+  if (Ns > 0) {
+    FT_CUDA(cudaMemset(L.slot_expert, 0xff, sizeof(int32_t) * Ns));
+    FT_CUDA(cudaMemset(L.slot_stamp, 0xff, sizeof(int64_t) * Ns));
+  }
+  FT_CUDA(cudaMemset(L.expert_slot, 0xff, sizeof(int32_t) * E));
+  FT_CUDA(cudaMemset(L.step, 0, sizeof(int64_t)));
+  FT_CUDA(cudaMemset(L.stats, 0, sizeof(unsigned long long) * FT_STAT_COUNT));
+  L.phase = PH_IDLE;
+  L.T = 0;
+  return FT_OK;
+}
+
+template <int WD, int TC, int NR>
+void launch_stream(ft_moe *h, const FfnParams &fp, int threads, int grid, cudaStream_t st) {
+  ffn_stream_kernel<WD, TC, NR><<<grid, threads, 0, st>>>(fp);
+  h->launches++;
+}
+
+void launch_stream_any(ft_moe *h, const FfnParams &fp, int T, cudaStream_t st) {
+  int CT, G;
+  stream_geometry(h->cfg, CT, G);
+  const int threads = CT * G;
+  const int grid = h->sm_count * ((threads <= 256) ? 2 : 1);
+  if (h->cfg.wdtype == FT_W_BF16) {
+    if (T <= 1) launch_stream<0, 1, 8>(h, fp, threads, grid, st);
+    else if (T <= 2) launch_stream<0, 2, 4>(h, fp, threads, grid, st);
+    else if (T <= 4) launch_stream<0, 4, 4>(h, fp, threads, grid, st);
+    else launch_stream<0, 8, 2>(h, fp, threads, grid, st);
+  } else {
+    if (T <= 1) launch_stream<1, 1, 8>(h, fp, threads, grid, st);
+    else launch_stream<1, 2, 4>(h, fp, threads, grid, st);
+  }
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t ft_moe_expert_bytes(const ft_moe_config_t *cfg) { return expert_bytes_of(cfg); }
+
+const char *ft_moe_status_string(ft_status_t s) {
+  switch (s) {
+    case FT_OK: return "ok";
+    case FT_ERR_INVALID_ARG: return "invalid argument";
+    case FT_ERR_NOT_PINNED: return "host pool is not pinned and mapped";
+    case FT_ERR_OOM: return "out of memory";
+    case FT_ERR_CUDA: return "CUDA error";
+    case FT_ERR_STATE: return "call out of order";
+    case FT_ERR_TIMEOUT: return "device-side wait timed out";
+    case FT_ERR_NONFINITE: return "non-finite router logits";
+    case FT_ERR_UNSUPPORTED: return "unsupported";
+  }
+  return "unknown status";
+}
+
+ft_status_t ft_moe_host_alloc(size_t bytes, void **out_host) {
+  if (!out_host || bytes == 0) return FT_ERR_INVALID_ARG;
+  *out_host = nullptr;
+  cudaError_t e = cudaHostAlloc(out_host, bytes, cudaHostAllocPortable | cudaHostAllocMapped);
+  if (e != cudaSuccess) {
+    (void)cudaGetLastError();
+    return e == cudaErrorMemoryAllocation ? FT_ERR_OOM : FT_ERR_CUDA;
+  }
+  return FT_OK;
+}
+
+ft_status_t ft_moe_host_free(void *host) {
+  if (!host) return FT_OK;
+  FT_CUDA(cudaFreeHost(host));
+  return FT_OK;
+}
+
+ft_status_t ft_moe_destroy(ft_moe_t *h) {
+  if (!h) return FT_OK;
+  cudaSetDevice(h->cfg.device);
+  cudaDeviceSynchronize();
+  cudaFree(h->slots);
+  cudaFree(h->shared_dev);
+  cudaFree(h->tables);
+  cudaFree(h->ids);
+  cudaFree(h->count);
+  cudaFree(h->offset);
+  cudaFree(h->perm);
+  cudaFree(h->inv);
+  cudaFree(h->topk_w);
+  cudaFree(h->y_acc);
+  cudaFree(h->plan_dev);
+  if (h->plan_host) cudaFreeHost(h->plan_host);
+  cudaFree(h->items_res);
+  cudaFree(h->items_zc);
+  cudaFree(h->items_gemm);
+  cudaFree(h->status_dev);
+  cudaFree(h->seq_dev);
+  cudaFree(h->stage_logits);
+  cudaFree(h->stage_x);
+  cudaFree(h->stage_y);
+  if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
+  if (h->aux_stream) cudaStreamDestroy(h->aux_stream);
+  cudaEvent_t evs[] = {h->ev_plan, h->ev_fill, h->ev_fork, h->ev_join, h->ev_fill_t0, h->ev_fill_t1};
+  for (cudaEvent_t e : evs)
+    if (e) cudaEventDestroy(e);
+  (void)cudaGetLastError();
+  delete h;
+  return FT_OK;
+}
+
+ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
+  if (!out) return FT_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!cfg || cfg->struct_size != sizeof(ft_moe_config_t)) return FT_ERR_INVALID_ARG;
+  const ft_moe_config_t &c = *cfg;
+  if (c.n_layers <= 0 || c.n_experts <= 0 || c.n_experts > kMaxExperts || c.top_k <= 0 ||
+      c.top_k > c.n_experts || c.top_k > kMaxTopK || c.slots_per_layer < 0 || c.slots_per_layer > 2048 ||
+      c.max_tokens <= 0 || (c.n_shared != 0 && c.n_shared != 1) || c.device < 0 ||
+      (c.fill_mode != FT_FILL_COPY_ENGINE && c.fill_mode != FT_FILL_SM))
+    return FT_ERR_INVALID_ARG;
+  if (c.wdtype != FT_W_BF16 && c.wdtype != FT_W_INT4_G128) return FT_ERR_INVALID_ARG;
+  if (c.bw_fill_MBps == 0 || c.bw_zc_MBps == 0 || c.bw_hbm_MBps == 0 || c.reuse_credit < 0 ||
+      c.zc_tokens_per_pass < 1 || c.hbm_tokens_per_pass < 1 || c.gemm_min_tokens < 0)
+    return FT_ERR_INVALID_ARG;
+  const size_t S = expert_bytes_of(cfg);
+  if (S == 0 || !geometry_ok(c)) return FT_ERR_UNSUPPORTED;
+  if (c.gemm_min_tokens != 0) return FT_ERR_UNSUPPORTED;
+  if (!c.host_pool || c.host_pool_bytes < (size_t)c.n_layers * c.n_experts * S) return FT_ERR_INVALID_ARG;
+  if (c.n_shared && !c.shared_weights) return FT_ERR_INVALID_ARG;
+  if ((long long)c.max_tokens * c.top_k > (1ll << 30)) return FT_ERR_INVALID_ARG;
+
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess) { (void)cudaGetLastError(); return FT_ERR_CUDA; }
+  if (c.device >= ndev) return FT_ERR_INVALID_ARG;
+  FT_CUDA(cudaSetDevice(c.device));
+
+  // The pool must be pinned and mapped: there is deliberately no pageable / CPU fallback.
+  cudaPointerAttributes attr;
+  if (cudaPointerGetAttributes(&attr, c.host_pool) != cudaSuccess) { (void)cudaGetLastError(); return FT_ERR_NOT_PINNED; }
+  if (attr.type != cudaMemoryTypeHost || attr.devicePointer == nullptr) return FT_ERR_NOT_PINNED;
+  {
+    const char *last = static_cast<const char *>(c.host_pool) + (size_t)c.n_layers * c.n_experts * S - 1;
+    cudaPointerAttributes a2;
+    if (cudaPointerGetAttributes(&a2, last) != cudaSuccess) { (void)cudaGetLastError(); return FT_ERR_NOT_PINNED; }
+    if (a2.type != cudaMemoryTypeHost) return FT_ERR_NOT_PINNED;
+  }
+
+  ft_moe *h = new (std::nothrow) ft_moe();
+  if (!h) return FT_ERR_OOM;
+  h->cfg = c;
+  h->S = S;
+  h->pool_dev = static_cast<const uint8_t *>(attr.devicePointer);
+  h->layers.resize(c.n_layers);
+  ft_status_t rc = FT_OK;
+  auto fail = [&](ft_status_t s) { ft_moe_destroy(h); return s; };
+#define FT_TRY(expr)                                            \
+  do {                                                          \
+    cudaError_t e_ = (expr);                                    \
+    if (e_ != cudaSuccess) {                                    \
+      (void)cudaGetLastError();                                 \
+      return fail(e_ == cudaErrorMemoryAllocation ? FT_ERR_OOM : FT_ERR_CUDA); \
+    }                                                           \
+  } while (0)
+
+  int smc = 0;
+  FT_TRY(cudaDeviceGetAttribute(&smc, cudaDevAttrMultiProcessorCount, c.device));
+  h->sm_count = smc > 0 ? smc : 148;
+
+  const size_t E = c.n_experts, Ns = c.slots_per_layer, L = c.n_layers;
+  const size_t P = (size_t)c.max_tokens * c.top_k;
+  if (Ns > 0) FT_TRY(cudaMalloc(&h->slots, L * Ns * S));
+  if (c.n_shared) {
+    FT_TRY(cudaMalloc(&h->shared_dev, L * S));
+    FT_TRY(cudaMemcpy(h->shared_dev, c.shared_weights, L * S, cudaMemcpyHostToDevice));
+  }
+  // per-layer tables, 256-byte aligned pieces
+  auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+  const size_t per_layer = up(Ns * 4) + up(Ns * 8) + up(E * 4) + up(8) + up(FT_STAT_COUNT * 8);
+  h->tables_bytes = per_layer * L;
+  FT_TRY(cudaMalloc(&h->tables, h->tables_bytes));
+  for (size_t l = 0; l < L; ++l) {
+    uint8_t *b = h->tables + l * per_layer;
+    LayerState &ls = h->layers[l];
+    ls.slot_expert = reinterpret_cast<int32_t *>(b); b += up(Ns * 4);
+    ls.slot_stamp = reinterpret_cast<int64_t *>(b); b += up(Ns * 8);
+    ls.expert_slot = reinterpret_cast<int32_t *>(b); b += up(E * 4);
+    ls.step = reinterpret_cast<int64_t *>(b); b += up(8);
+    ls.stats = reinterpret_cast<unsigned long long *>(b);
+  }
+  FT_TRY(cudaMalloc(&h->ids, P * 4 + 16));
+  FT_TRY(cudaMalloc(&h->topk_w, P * 4 + 16));
+  FT_TRY(cudaMalloc(&h->count, E * 4));
+  FT_TRY(cudaMalloc(&h->offset, (E + 1) * 4));
+  FT_TRY(cudaMalloc(&h->perm, P * 4 + 16));
+  FT_TRY(cudaMalloc(&h->inv, P * 4 + 16));
+  FT_TRY(cudaMalloc(&h->y_acc, (size_t)c.max_tokens * c.hidden * 4));
+  FT_TRY(cudaMemset(h->y_acc, 0, (size_t)c.max_tokens * c.hidden * 4));
+  h->plan_bytes = sizeof(PlanHeader) + 8 * E * 4;
+  FT_TRY(cudaMalloc(&h->plan_dev, h->plan_bytes));
+  FT_TRY(cudaMemset(h->plan_dev, 0, h->plan_bytes));
+  FT_TRY(cudaHostAlloc(&h->plan_host, h->plan_bytes, cudaHostAllocMapped));
+  memset(h->plan_host, 0, h->plan_bytes);
+  FT_TRY(cudaHostGetDevicePointer(reinterpret_cast<void **>(&h->plan_host_devptr), h->plan_host, 0));
+  FT_TRY(cudaMalloc(&h->items_res, (E + 1) * sizeof(WorkItem)));
+  FT_TRY(cudaMalloc(&h->items_zc, E * sizeof(WorkItem)));
+  FT_TRY(cudaMalloc(&h->items_gemm, E * sizeof(WorkItem)));
+  FT_TRY(cudaMalloc(&h->status_dev, 4));
+  FT_TRY(cudaMemset(h->status_dev, 0, 4));
+  FT_TRY(cudaMalloc(&h->seq_dev, 4));
+  FT_TRY(cudaMemset(h->seq_dev, 0, 4));
+  FT_TRY(cudaMalloc(&h->stage_logits, (size_t)c.max_tokens * E * 4));
+  FT_TRY(cudaMalloc(&h->stage_x, (size_t)c.max_tokens * c.hidden * 2));
+  FT_TRY(cudaMalloc(&h->stage_y, (size_t)c.max_tokens * c.hidden * 2));
+  FT_TRY(cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking));
+  FT_TRY(cudaStreamCreateWithFlags(&h->aux_stream, cudaStreamNonBlocking));
+  FT_TRY(cudaEventCreateWithFlags(&h->ev_plan, cudaEventDisableTiming));
+  FT_TRY(cudaEventCreateWithFlags(&h->ev_fill, cudaEventDisableTiming));
+  FT_TRY(cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming));
+  FT_TRY(cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming));
+  FT_TRY(cudaEventCreate(&h->ev_fill_t0));
+  FT_TRY(cudaEventCreate(&h->ev_fill_t1));
+  for (int l = 0; l < c.n_layers; ++l) {
+    rc = reset_layer(h, l);
+    if (rc != FT_OK) return fail(rc);
+  }
+  FT_TRY(cudaDeviceSynchronize());
+#undef FT_TRY
+  *out = h;
+  return FT_OK;
+}
+
+ft_status_t ft_moe_reset(ft_moe_t *h, int layer) {
+  if (!h || layer < -1 || layer >= h->cfg.n_layers) return FT_ERR_INVALID_ARG;
+  FT_CUDA(cudaSetDevice(h->cfg.device));
+  FT_CUDA(cudaDeviceSynchronize());
+  for (int l = 0; l < h->cfg.n_layers; ++l)
+    if (layer < 0 || l == layer) {
+      ft_status_t rc = reset_layer(h, l);
+      if (rc != FT_OK) return rc;
+    }
+  FT_CUDA(cudaMemset(h->y_acc, 0, (size_t)h->cfg.max_tokens * h->cfg.hidden * 4));
+  FT_CUDA(cudaDeviceSynchronize());
+  return FT_OK;
+}
+
+ft_status_t ft_moe_route(ft_moe_t *h, int layer, const float *logits_dev, int T, void *stream) {
+  if (!h || layer < 0 || layer >= h->cfg.n_layers || T < 0 || T > h->cfg.max_tokens) return FT_ERR_INVALID_ARG;
+  if (T > 0 && !logits_dev) return FT_ERR_INVALID_ARG;
+  LayerState &L = h->layers[layer];
+  L.phase = PH_ROUTED;
+  L.T = T;
+  h->last_routed_layer = layer;
+  if (T == 0) return FT_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  RouteParams rp;
+  rp.logits = logits_dev;
+  rp.T = T; rp.E = h->cfg.n_experts; rp.k = h->cfg.top_k;
+  rp.ids = h->ids; rp.w = h->topk_w; rp.count = h->count; rp.offset = h->offset;
+  rp.perm = h->perm; rp.inv = h->inv; rp.status = h->status_dev;
+  if (T <= kRouteSmallMaxTokens) {
+    route_small_kernel<<<1, 1024, 0, st>>>(rp);
+    h->launches++;
+  } else {
+    FT_CUDA(cudaMemsetAsync(h->count, 0, sizeof(int32_t) * rp.E, st));
+    route_topk_kernel<<<(T + 7) / 8, 256, 0, st>>>(rp);
+    permute_kernel<<<(rp.E + 7) / 8, 256, 0, st>>>(rp);
+    h->launches += 2;
+  }
+  FT_CUDA(cudaGetLastError());
+  return FT_OK;
+}
+
+ft_status_t ft_moe_plan(ft_moe_t *h, int layer, ft_moe_plan_t *out, void *stream) {
+  if (!h || layer < 0 || layer >= h->cfg.n_layers) return FT_ERR_INVALID_ARG;
+  LayerState &L = h->layers[layer];
+  if (L.phase != PH_ROUTED || h->last_routed_layer != layer) return FT_ERR_STATE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const ft_moe_config_t &c = h->cfg;
+  if (L.T > 0) {
+    PlanParams pp;
+    pp.count = h->count; pp.offset = h->offset;
+    pp.E = c.n_experts; pp.n_slots = c.slots_per_layer;
+    pp.cm.ns_fill = (int64_t)(h->S * 1000 / c.bw_fill_MBps);
+    pp.cm.ns_zc = (int64_t)(h->S * 1000 / c.bw_zc_MBps);
+    pp.cm.ns_hbm = (int64_t)(h->S * 1000 / c.bw_hbm_MBps);
+    pp.cm.bw_fill = c.bw_fill_MBps; pp.cm.bw_res = c.bw_zc_residual_MBps;
+    pp.cm.reuse_credit = c.reuse_credit; pp.cm.tz = c.zc_tokens_per_pass; pp.cm.tg = c.hbm_tokens_per_pass;
+    pp.cm.gemm_min_tokens = c.gemm_min_tokens;
+    pp.slot_expert = L.slot_expert; pp.slot_stamp = L.slot_stamp; pp.expert_slot = L.expert_slot;
+    pp.step = L.step; pp.stats = L.stats;
+    pp.pool_layer_dev = h->pool_dev + (size_t)layer * c.n_experts * h->S;
+    pp.slots_layer = h->slots ? h->slots + (size_t)layer * c.slots_per_layer * h->S : nullptr;
+    pp.shared_rec = c.n_shared ? h->shared_dev + (size_t)layer * h->S : nullptr;
+    pp.S = h->S; pp.T = L.T;
+    pp.hdr_dev = h->plan_dev; pp.hdr_host = h->plan_host_devptr;
+    pp.items_res = h->items_res; pp.items_zc = h->items_zc; pp.items_gemm = h->items_gemm;
+    pp.seq = h->seq_dev;
+    const size_t smem = (size_t)c.slots_per_layer * 16;
+    plan_kernel<<<1, 1024, smem, st>>>(pp);
+    h->launches++;
+    h->seq_host++;
+    FT_CUDA(cudaGetLastError());
+    FT_CUDA(cudaEventRecord(h->ev_plan, st));
+  }
+  L.phase = PH_PLANNED;
+  if (out) {
+    const int E = c.n_experts;
+    if (L.T == 0) {
+      out->step = -1;
+      out->n_routed = out->n_hit = out->n_miss = out->n_fill = out->n_zc = 0;
+      if (out->loc) for (int e = 0; e < E; ++e) out->loc[e] = kLocNotRouted;
+      return FT_OK;
+    }
+    FT_CUDA(cudaEventSynchronize(h->ev_plan));
+    const PlanHeader hd = *h->plan_host;
+    if (hd.seq != h->seq_host) return FT_ERR_CUDA;
+    const int32_t *a = reinterpret_cast<const int32_t *>(h->plan_host + 1);
+    out->step = hd.step;
+    out->n_routed = hd.n_routed; out->n_hit = hd.n_hit; out->n_miss = hd.n_miss;
+    out->n_fill = hd.n_fill; out->n_zc = hd.n_zc;
+    if (out->hit) memcpy(out->hit, a + 0 * E, sizeof(int32_t) * hd.n_hit);
+    if (out->miss) memcpy(out->miss, a + 1 * E, sizeof(int32_t) * hd.n_miss);
+    if (out->fill) memcpy(out->fill, a + 2 * E, sizeof(int32_t) * hd.n_fill);
+    if (out->zc) memcpy(out->zc, a + 3 * E, sizeof(int32_t) * hd.n_zc);
+    if (out->fill_order) memcpy(out->fill_order, a + 4 * E, sizeof(int32_t) * hd.n_fill);
+    if (out->fill_slot) memcpy(out->fill_slot, a + 5 * E, sizeof(int32_t) * hd.n_fill);
+    if (out->fill_evicted) memcpy(out->fill_evicted, a + 6 * E, sizeof(int32_t) * hd.n_fill);
+    if (out->loc) memcpy(out->loc, a + 7 * E, sizeof(int32_t) * E);
+    return drain_status(h);
+  }
+  return FT_OK;
+}
+
+ft_status_t ft_moe_fill(ft_moe_t *h, int layer, void *copy_stream) {
+  if (!h || layer < 0 || layer >= h->cfg.n_layers) return FT_ERR_INVALID_ARG;
+  LayerState &L = h->layers[layer];
+  if (L.phase != PH_PLANNED) return FT_ERR_STATE;
+  L.phase = PH_FILLED;
+  h->fill_timed = false;
+  h->last_fill_bytes = 0;
+  if (L.T == 0 || h->cfg.slots_per_layer == 0) return FT_OK;
+  cudaStream_t cs = static_cast<cudaStream_t>(copy_stream);
+  const ft_moe_config_t &c = h->cfg;
+  uint8_t *slots_layer = h->slots + (size_t)layer * c.slots_per_layer * h->S;
+  if (c.fill_mode == FT_FILL_COPY_ENGINE) {
+    // the host needs the fill list: wait for the plan record (one host round trip per layer)
+    FT_CUDA(cudaEventSynchronize(h->ev_plan));
+    const PlanHeader hd = *h->plan_host;
+    if (hd.seq != h->seq_host) return FT_ERR_CUDA;
+    if (hd.n_fill > 0) {
+      const int E = c.n_experts;
+      const int32_t *a = reinterpret_cast<const int32_t *>(h->plan_host + 1);
+      const int32_t *forder = a + 4 * E, *fslot = a + 5 * E;
+      const uint8_t *pool_layer = static_cast<const uint8_t *>(c.host_pool) + (size_t)layer * E * h->S;
+      FT_CUDA(cudaStreamWaitEvent(cs, h->ev_plan, 0));
+      FT_CUDA(cudaEventRecord(h->ev_fill_t0, cs));
+      for (int i = 0; i < hd.n_fill; ++i) {
+        if (forder[i] < 0 || forder[i] >= E || fslot[i] < 0 || fslot[i] >= c.slots_per_layer) return FT_ERR_CUDA;
+        FT_CUDA(cudaMemcpyAsync(slots_layer + (size_t)fslot[i] * h->S, pool_layer + (size_t)forder[i] * h->S,
+                                h->S, cudaMemcpyHostToDevice, cs));
+      }
+      FT_CUDA(cudaEventRecord(h->ev_fill_t1, cs));
+      FT_CUDA(cudaEventRecord(h->ev_fill, cs));
+      h->fill_timed = true;
+      h->last_fill_bytes = (uint64_t)hd.n_fill * h->S;
+    } else {
+      // nothing to copy: the fill event of an earlier layer must not be waited on needlessly
+      FT_CUDA(cudaStreamWaitEvent(cs, h->ev_plan, 0));
+      FT_CUDA(cudaEventRecord(h->ev_fill, cs));
+    }
+  } else {
+    FillParams fp;
+    fp.hdr = h->plan_dev; fp.E = c.n_experts;
+    fp.pool_layer_dev = h->pool_dev + (size_t)layer * c.n_experts * h->S;
+    fp.slots_layer = slots_layer; fp.S = h->S;
+    FT_CUDA(cudaStreamWaitEvent(cs, h->ev_plan, 0));
+    FT_CUDA(cudaEventRecord(h->ev_fill_t0, cs));
+    fill_kernel<<<h->sm_count * 4, 256, 0, cs>>>(fp);
+    h->launches++;
+    FT_CUDA(cudaGetLastError());
+    FT_CUDA(cudaEventRecord(h->ev_fill_t1, cs));
+    FT_CUDA(cudaEventRecord(h->ev_fill, cs));
+    h->fill_timed = true;
+    h->last_fill_bytes = ~0ull;  // resolved from the plan record when asked
+  }
+  return FT_OK;
+}
+
+ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_dev, void *stream) {
+  if (!h || layer < 0 || layer >= h->cfg.n_layers) return FT_ERR_INVALID_ARG;
+  LayerState &L = h->layers[layer];
+  if (L.phase != PH_FILLED) return FT_ERR_STATE;
+  L.phase = PH_IDLE;
+  if (L.T == 0) return FT_OK;
+  if (!x_dev || !y_dev) return FT_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const ft_moe_config_t &c = h->cfg;
+  FfnParams fp;
+  fp.x = static_cast<const __nv_bfloat16 *>(x_dev);
+  fp.perm = h->perm; fp.topk_w = h->topk_w; fp.y_acc = h->y_acc;
+  fp.d = c.hidden; fp.inter = c.inter; fp.top_k = c.top_k;
+  // zero-copy set first: it does not depend on the fills and shares the host link with them
+  fp.items = h->items_zc;
+  fp.n_items = &h->plan_dev->n_zc_items;
+  launch_stream_any(h, fp, L.T, st);
+  // resident set after the fills have landed
+  if (c.slots_per_layer > 0) FT_CUDA(cudaStreamWaitEvent(st, h->ev_fill, 0));
+  if (c.slots_per_layer > 0 || c.n_shared) {
+    fp.items = h->items_res;
+    fp.n_items = &h->plan_dev->n_res_items;
+    launch_stream_any(h, fp, L.T, st);
+  }
+  const long long n4 = (long long)L.T * c.hidden / 4;
+  finalize_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(h->y_acc, static_cast<__nv_bfloat16 *>(y_dev), n4);
+  h->launches++;
+  FT_CUDA(cudaGetLastError());
+  return FT_OK;
+}
+
+ft_status_t ft_moe_layer(ft_moe_t *h, int layer, const float *logits_dev, const void *x_dev, void *y_dev,
+                         int T, void *stream) {
+  ft_status_t rc = ft_moe_route(h, layer, logits_dev, T, stream);
+  if (rc != FT_OK) return rc;
+  rc = ft_moe_plan(h, layer, nullptr, stream);
+  if (rc != FT_OK) return rc;
+  rc = ft_moe_fill(h, layer, h->copy_stream);
+  if (rc != FT_OK) return rc;
+  return ft_moe_forward(h, layer, x_dev, y_dev, stream);
+}
+
+ft_status_t ft_moe_layer_host(ft_moe_t *h, int layer, const float *logits_host, const void *x_host,
+                              void *y_host, int T, void *stream) {
+  if (!h || T < 0 || T > h->cfg.max_tokens) return FT_ERR_INVALID_ARG;
+  if (T > 0 && (!logits_host || !x_host || !y_host)) return FT_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const ft_moe_config_t &c = h->cfg;
+  if (T > 0) {
+    FT_CUDA(cudaMemcpyAsync(h->stage_logits, logits_host, (size_t)T * c.n_experts * 4, cudaMemcpyHostToDevice, st));
+    FT_CUDA(cudaMemcpyAsync(h->stage_x, x_host, (size_t)T * c.hidden * 2, cudaMemcpyHostToDevice, st));
+  }
+  ft_status_t rc = ft_moe_layer(h, layer, h->stage_logits, h->stage_x, h->stage_y, T, stream);
+  if (rc != FT_OK) return rc;
+  if (T > 0) {
+    FT_CUDA(cudaMemcpyAsync(y_host, h->stage_y, (size_t)T * c.hidden * 2, cudaMemcpyDeviceToHost, st));
+    FT_CUDA(cudaStreamSynchronize(st));
+  }
+  return FT_OK;
+}
+
+ft_status_t ft_moe_get_routing(ft_moe_t *h, int layer, int32_t *ids, float *w, int32_t *count,
+                               int32_t *offset, int32_t *perm, int32_t *inv) {
+  if (!h || layer < 0 || layer >= h->cfg.n_layers) return FT_ERR_INVALID_ARG;
+  if (h->last_routed_layer != layer) return FT_ERR_STATE;
+  FT_CUDA(cudaSetDevice(h->cfg.device));
+  FT_CUDA(cudaDeviceSynchronize());
+  const size_t P = (size_t)h->layers[layer].T * h->cfg.top_k, E = h->cfg.n_experts;
+  if (P == 0) {
+    if (count) memset(count, 0, E * 4);
+    if (offset) memset(offset, 0, (E + 1) * 4);
+    return FT_OK;
+  }
+  if (ids) FT_CUDA(cudaMemcpy(ids, h->ids, P * 4, cudaMemcpyDeviceToHost));
+  if (w) FT_CUDA(cudaMemcpy(w, h->topk_w, P * 4, cudaMemcpyDeviceToHost));
+  if (count) FT_CUDA(cudaMemcpy(count, h->count, E * 4, cudaMemcpyDeviceToHost));
+  if (offset) FT_CUDA(cudaMemcpy(offset, h->offset, (E + 1) * 4, cudaMemcpyDeviceToHost));
+  if (perm) FT_CUDA(cudaMemcpy(perm, h->perm, P * 4, cudaMemcpyDeviceToHost));
+  if (inv) FT_CUDA(cudaMemcpy(inv, h->inv, P * 4, cudaMemcpyDeviceToHost));
+  return drain_status(h);
+}
+
+ft_status_t ft_moe_get_slot_table(ft_moe_t *h, int layer, int32_t *slot_expert, int64_t *slot_stamp,
+                                  int32_t *expert_slot) {
+  if (!h || layer < 0 || layer >= h->cfg.n_layers) return FT_ERR_INVALID_ARG;
+  FT_CUDA(cudaSetDevice(h->cfg.device));
+  FT_CUDA(cudaDeviceSynchronize());
+  const LayerState &L = h->layers[layer];
+  const size_t Ns = h->cfg.slots_per_layer;
+  if (slot_expert && Ns) FT_CUDA(cudaMemcpy(slot_expert, L.slot_expert, Ns * 4, cudaMemcpyDeviceToHost));
+  if (slot_stamp && Ns) FT_CUDA(cudaMemcpy(slot_stamp, L.slot_stamp, Ns * 8, cudaMemcpyDeviceToHost));
+  if (expert_slot) FT_CUDA(cudaMemcpy(expert_slot, L.expert_slot, (size_t)h->cfg.n_experts * 4, cudaMemcpyDeviceToHost));
+  return FT_OK;
+}
+
+ft_status_t ft_moe_read_slot(ft_moe_t *h, int layer, int slot, void *host_dst) {
+  if (!h || layer < 0 || layer >= h->cfg.n_layers || slot < 0 || slot >= h->cfg.slots_per_layer || !host_dst)
+    return FT_ERR_INVALID_ARG;
+  FT_CUDA(cudaSetDevice(h->cfg.device));
+  FT_CUDA(cudaDeviceSynchronize());
+  FT_CUDA(cudaMemcpy(host_dst, h->slots + ((size_t)layer * h->cfg.slots_per_layer + slot) * h->S, h->S,
+                     cudaMemcpyDeviceToHost));
+  return FT_OK;
+}
+
+ft_status_t ft_moe_get_stats(ft_moe_t *h, int layer, uint64_t *counters, int n) {
+  if (!h || layer < 0 || layer >= h->cfg.n_layers || !counters || n < 0) return FT_ERR_INVALID_ARG;
+  FT_CUDA(cudaSetDevice(h->cfg.device));
+  FT_CUDA(cudaDeviceSynchronize());
+  unsigned long long tmp[FT_STAT_COUNT];
+  FT_CUDA(cudaMemcpy(tmp, h->layers[layer].stats, sizeof(tmp), cudaMemcpyDeviceToHost));
+  for (int i = 0; i < n && i < FT_STAT_COUNT; ++i) counters[i] = tmp[i];
+  return FT_OK;
+}
+
+ft_status_t ft_moe_sync_status(ft_moe_t *h) {
+  if (!h) return FT_ERR_INVALID_ARG;
+  FT_CUDA(cudaSetDevice(h->cfg.device));
+  FT_CUDA(cudaDeviceSynchronize());
+  return drain_status(h);
+}
+
+ft_status_t ft_moe_last_fill(ft_moe_t *h, float *out_us, uint64_t *out_bytes) {
+  if (!h) return FT_ERR_INVALID_ARG;
+  if (out_us) *out_us = 0.f;
+  if (out_bytes) *out_bytes = 0;
+  if (!h->fill_timed) return FT_OK;
+  FT_CUDA(cudaEventSynchronize(h->ev_fill_t1));
+  float ms = 0.f;
+  FT_CUDA(cudaEventElapsedTime(&ms, h->ev_fill_t0, h->ev_fill_t1));
+  if (out_us) *out_us = ms * 1000.f;
+  uint64_t bytes = h->last_fill_bytes;
+  if (bytes == ~0ull) bytes = (uint64_t)h->plan_host->n_fill * h->S;
+  if (out_bytes) *out_bytes = bytes;
+  return FT_OK;
+}
+
+ft_status_t ft_moe_launch_count(ft_moe_t *h, uint64_t *out) {
+  if (!h || !out) return FT_ERR_INVALID_ARG;
+  *out = h->launches;
+  return FT_OK;
+}
+
+ft_status_t ft_moe_calibrate(ft_moe_t *h, uint32_t out_MBps[4]) {
+  if (!h || !out_MBps) return FT_ERR_INVALID_ARG;
+  FT_CUDA(cudaSetDevice(h->cfg.device));
+  FT_CUDA(cudaDeviceSynchronize());
+  const ft_moe_config_t &c = h->cfg;
+  const size_t pool_records = (size_t)c.n_layers * c.n_experts;
+  // sample: up to 256 MiB of pool records, at least one
+  size_t n_rec = (256ull << 20) / h->S;
+  if (n_rec < 1) n_rec = 1;
+  if (n_rec > pool_records) n_rec = pool_records;
+  const size_t bytes = n_rec * h->S;
+  uint8_t *scratch = nullptr;
+  uint32_t *sink = nullptr;
+  FT_CUDA(cudaMalloc(&scratch, bytes));
+  if (cudaMalloc(&sink, 4) != cudaSuccess) { cudaFree(scratch); (void)cudaGetLastError(); return FT_ERR_OOM; }
+  cudaMemset(sink, 0, 4);
+  cudaEvent_t e0, e1, e2, e3;
+  cudaEventCreate(&e0); cudaEventCreate(&e1); cudaEventCreate(&e2); cudaEventCreate(&e3);
+  const uint8_t *hp = static_cast<const uint8_t *>(c.host_pool);
+  auto mbps = [](size_t b, float ms) { return (uint32_t)(ms > 0.f ? (double)b / (ms * 1e-3) / 1e6 : 0.0); };
+  float best[4] = {1e30f, 1e30f, 1e30f, 1e30f};
+  const int grid = h->sm_count * 4;
+  for (int rep = 0; rep < 4; ++rep) {
+    float ms;
+    // (0) copy-engine fill rate: record-sized pinned H2D copies back to back
+    cudaEventRecord(e0, h->copy_stream);
+    for (size_t r = 0; r < n_rec; ++r)
+      cudaMemcpyAsync(scratch + r * h->S, hp + r * h->S, h->S, cudaMemcpyHostToDevice, h->copy_stream);
+    cudaEventRecord(e1, h->copy_stream);
+    cudaEventSynchronize(e1);
+    cudaEventElapsedTime(&ms, e0, e1);
+    if (rep > 0 && ms < best[0]) best[0] = ms;
+    // (1) zero-copy reads alone
+    cudaEventRecord(e0, h->aux_stream);
+    read_kernel<<<grid, 256, 0, h->aux_stream>>>(h->pool_dev, bytes, sink);
+    cudaEventRecord(e1, h->aux_stream);
+    cudaEventSynchronize(e1);
+    cudaEventElapsedTime(&ms, e0, e1);
+    if (rep > 0 && ms < best[1]) best[1] = ms;
+    // (2) zero-copy reads while the copy engine is kept busy for the whole kernel
+    cudaEventRecord(e2, h->copy_stream);
+    for (int k = 0; k < 3; ++k)
+      for (size_t r = 0; r < n_rec; ++r)
+        cudaMemcpyAsync(scratch + r * h->S, hp + r * h->S, h->S, cudaMemcpyHostToDevice, h->copy_stream);
+    cudaEventRecord(e3, h->copy_stream);
+    cudaEventRecord(e0, h->aux_stream);
+    read_kernel<<<grid, 256, 0, h->aux_stream>>>(h->pool_dev, bytes, sink);
+    cudaEventRecord(e1, h->aux_stream);
+    cudaEventSynchronize(e1);
+    cudaEventSynchronize(e3);
+    cudaEventElapsedTime(&ms, e0, e1);
+    if (rep > 0 && ms < best[2]) best[2] = ms;
+    // (3) HBM streaming reads
+    cudaEventRecord(e0, h->aux_stream);
+    read_kernel<<<grid, 256, 0, h->aux_stream>>>(scratch, bytes, sink);
+    cudaEventRecord(e1, h->aux_stream);
+    cudaEventSynchronize(e1);
+    cudaEventElapsedTime(&ms, e0, e1);
+    if (rep > 0 && ms < best[3]) best[3] = ms;
+    h->launches += 3;
+  }
+  for (int i = 0; i < 4; ++i) out_MBps[i] = mbps(bytes, best[i]);
+  cudaEventDestroy(e0); cudaEventDestroy(e1); cudaEventDestroy(e2); cudaEventDestroy(e3);
+  cudaFree(scratch);
+  cudaFree(sink);
+  FT_CUDA(cudaDeviceSynchronize());
+  FT_CUDA(cudaGetLastError());
+  return FT_OK;
+}
+
+}  // extern "C"

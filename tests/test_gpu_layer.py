@@ -1,0 +1,219 @@
+"""GPU parity of the whole layer path against the CPU oracle, through the C ABI."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ftmoe_oracle as O
+from paper_2608_16157_b200 import binding as B
+from paper_2608_16157_b200 import workload as W
+from tests.helpers import Pair, check_output
+
+pytestmark = pytest.mark.gpu
+
+LAPTOP = dict(bw_fill=11800, bw_zc_residual=35700, bw_zc=11800)     # Table 1, 4060-laptop row
+
+
+@pytest.mark.parametrize("fill_mode", [B.FT_FILL_COPY_ENGINE, B.FT_FILL_SM])
+@pytest.mark.parametrize("cost", [dict(), LAPTOP])
+def test_tiny_config_all_steps_every_array(fill_mode, cost):
+    """d=256, 8 experts, top-2, 4 slots, 4 steps x 8 tokens, cold start: H, F and Z all occur."""
+    pr = Pair(W.TINY, n_slots=4, max_tokens=8, fill_mode=fill_mode, **cost)
+    seen = set()
+    for step in range(4):
+        logits = W.normal_logits(8, 8, 0, step)
+        x = W.noise_x(8, 256, 0, step, 0)
+        _, r = pr.step(0, logits, x, check_slots=True)
+        seen |= {"H"} if r.plan.hit else set()
+        seen |= {"F"} if r.plan.fill else set()
+        seen |= {"Z"} if r.plan.zc else set()
+    assert seen == {"H", "F", "Z"}
+    st = pr.moe.get_stats(0)
+    assert st["steps"] == 4 and st["pairs"] == 4 * 16
+    assert st["routed"] == st["hits"] + st["misses"] and st["misses"] == st["fills"] + st["zc"]
+    pr.close()
+
+
+@pytest.mark.parametrize("T", [1, 2, 3, 5, 8, 13, 37, 128, 129, 300])
+def test_token_counts_span_tiles_and_both_route_paths(T):
+    shape = W.LayerShape(d=512, inter=192, n_experts=16, top_k=4)
+    pr = Pair(shape, n_slots=6, max_tokens=300, seed=T)
+    rng = np.random.default_rng(T)
+    for step in range(3):
+        logits = (rng.standard_normal((T, 16)) * 2).astype(np.float32)
+        x = W.noise_x(T, 512, T, step, 0)
+        pr.step(0, logits, x, check_slots=(step == 2))
+    pr.close()
+
+
+def test_empty_call_is_a_noop_and_does_not_advance():
+    pr = Pair(W.TINY, n_slots=4, max_tokens=8)
+    pr.step(0, W.normal_logits(8, 8, 0, 0), W.noise_x(8, 256, 0, 0, 0))
+    pr.step(0, np.zeros((0, 8), dtype=np.float32), torch.zeros((0, 256), dtype=torch.bfloat16))
+    _, r = pr.step(0, W.normal_logits(8, 8, 0, 1), W.noise_x(8, 256, 0, 1, 0))
+    assert r.plan.step == 1
+    pr.close()
+
+
+def test_ties_signed_zero_and_nonfinite_logits():
+    pr = Pair(W.TINY, n_slots=8, max_tokens=8)
+    z = np.zeros((8, 8), dtype=np.float32)
+    z[0] = [1, 2, 2, -0.0, 0.0, 2, 2, 1]
+    z[1] = [0.0, -0.0, 0.0, -0.0, -1, -1, -1, -1]
+    z[2] = 3.0
+    z[3] = [5, 4, 3, 2, 1, 0, -1, -2]
+    z[4] = z[3][::-1]
+    z[5] = [-1e30, 1e30, 0, 0, 0, 0, 0, 0]
+    z[6] = [1e-40, -1e-40, 0, 0, 0, 0, 0, 0]       # subnormals
+    z[7] = [7, 7, 7, 7, 8, 8, 8, 8]
+    x = W.noise_x(8, 256, 1, 0, 0)
+    pr.step(0, z, x)
+    bad = z.copy()
+    bad[3, 2] = np.nan
+    lg = torch.from_numpy(bad).cuda()
+    pr.moe.route(0, lg, 8)
+    assert pr.moe.sync_status() == B.FT_ERR_NONFINITE
+    assert pr.moe.sync_status() == 0          # latched once
+    bad[3, 2] = np.inf
+    pr.moe.route(0, torch.from_numpy(bad).cuda(), 8)
+    with pytest.raises(B.FtMoeError) as ei:
+        pr.moe.plan(0)
+    assert ei.value.code == B.FT_ERR_NONFINITE
+    pr.close()
+
+
+def test_results_do_not_depend_on_residency():
+    """All-zero-copy, cold all-fill and warm all-hit runs give the same y (the host pool is the
+    source of truth; the cache affects only performance)."""
+    shape = W.LayerShape(d=512, inter=128, n_experts=8, top_k=2)
+    logits = W.normal_logits(12, 8, 3, 0)
+    x = W.noise_x(12, 512, 3, 0, 0)
+    ys = {}
+    for name, n_slots in (("zc", 0), ("full", 8)):
+        pr = Pair(shape, n_slots=n_slots, max_tokens=12, seed=3)
+        y, r = pr.step(0, logits, x)
+        if name == "zc":
+            assert r.plan.zc == r.plan.routed
+            ys["zc"] = y.float().cpu()
+        else:
+            assert r.plan.fill == r.plan.routed
+            ys["fill"] = y.float().cpu()
+            y2, r2 = pr.step(0, logits, x)
+            assert r2.plan.hit == r2.plan.routed
+            ys["hit"] = y2.float().cpu()
+        pr.close()
+    scale = ys["hit"].abs().max()
+    assert (ys["zc"] - ys["hit"]).abs().max() <= 1e-2 * scale
+    assert torch.equal(ys["fill"], ys["hit"]) or (ys["fill"] - ys["hit"]).abs().max() <= 1e-2 * scale
+
+
+@pytest.mark.parametrize("n_shared", [0, 1])
+@pytest.mark.parametrize("T", [1, 4, 7])
+def test_int4_group_dequant_and_shared_expert(n_shared, T):
+    shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2, wdtype="int4", n_shared=n_shared)
+    pr = Pair(shape, n_slots=4, max_tokens=8, seed=5)
+    for step in range(3):
+        pr.step(0, W.normal_logits(T, 8, 5, step), W.noise_x(T, 512, 5, step, 0), check_slots=True)
+    pr.close()
+
+
+def test_plan_and_permutation_are_deterministic():
+    shape = W.LayerShape(d=256, inter=64, n_experts=32, top_k=4)
+    runs = []
+    for rep in range(3):
+        pr = Pair(shape, n_slots=10, max_tokens=64, seed=9, **LAPTOP)
+        out = []
+        for step in range(5):
+            logits = W.normal_logits(64, 32, 9, step)
+            lg = torch.from_numpy(logits).cuda()
+            pr.moe.route(0, lg, 64)
+            plan = pr.moe.plan(0)
+            pr.moe.fill(0, None)
+            x = W.noise_x(64, 256, 9, step, 0).cuda()
+            pr.moe.forward(0, x, torch.empty_like(x))
+            ids, w, count, offset, perm, inv = pr.moe.get_routing(0, 64)
+            out.append((ids.tobytes(), perm.tobytes(), inv.tobytes(), str(plan["fill_order"]), str(plan["fill_slot"]),
+                        str(plan["zc"]), plan["loc"].tobytes()))
+        runs.append(out)
+        pr.close()
+    assert runs[0] == runs[1] == runs[2]
+
+
+def test_multi_layer_stack_keeps_per_layer_state():
+    shape = W.LayerShape(d=256, inter=64, n_experts=16, top_k=2)
+    pr = Pair(shape, n_slots=5, max_tokens=4, n_layers=3, seed=11)
+    for step in range(4):
+        for l in range(3):
+            logits = W.normal_logits(4, 16, 11 + l, step)
+            pr.step(l, logits, W.noise_x(4, 256, 11, step, l), check_slots=True, fused=(step % 2 == 1))
+    pr.close()
+
+
+def test_error_paths():
+    lib = B.load()
+    shape = W.TINY
+    S = shape.expert_bytes
+    # pageable pool -> FT_ERR_NOT_PINNED (there is no CPU fallback)
+    pageable = torch.zeros(shape.n_experts * S, dtype=torch.uint8)
+    cfg = B.make_config(hidden=256, inter=128, n_experts=8, top_k=2, slots_per_layer=4, max_tokens=8,
+                        host_pool_ptr=pageable.data_ptr(), host_pool_bytes=pageable.numel())
+    h = ctypes.c_void_p()
+    assert lib.ft_moe_create(ctypes.byref(cfg), ctypes.byref(h)) == B.FT_ERR_NOT_PINNED
+    # pool too small
+    pr = Pair(shape, n_slots=4, max_tokens=8)
+    cfg2 = B.make_config(hidden=256, inter=128, n_experts=8, top_k=2, slots_per_layer=4, max_tokens=8,
+                         host_pool_ptr=pr.pool.ptr.value, host_pool_bytes=S)
+    assert lib.ft_moe_create(ctypes.byref(cfg2), ctypes.byref(h)) == B.FT_ERR_INVALID_ARG
+    # call order
+    lg = torch.from_numpy(W.normal_logits(8, 8, 0, 0)).cuda()
+    x = W.noise_x(8, 256, 0, 0, 0).cuda()
+    y = torch.empty_like(x)
+    for call in (lambda: pr.moe.plan(0), lambda: pr.moe.fill(0, None), lambda: pr.moe.forward(0, x, y)):
+        with pytest.raises(B.FtMoeError) as ei:
+            call()
+        assert ei.value.code == B.FT_ERR_STATE
+    pr.moe.route(0, lg, 8)
+    with pytest.raises(B.FtMoeError) as ei:
+        pr.moe.forward(0, x, y)
+    assert ei.value.code == B.FT_ERR_STATE
+    with pytest.raises(B.FtMoeError) as ei:
+        pr.moe.route(0, lg, 9)        # T > max_tokens
+    assert ei.value.code == B.FT_ERR_INVALID_ARG
+    with pytest.raises(B.FtMoeError):
+        pr.moe.route(1, lg, 8)        # no such layer
+    # the handle still works after the errors
+    pr.moe.reset()
+    pr.step(0, W.normal_logits(8, 8, 0, 0), W.noise_x(8, 256, 0, 0, 0))
+    pr.close()
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    pr = Pair(W.TINY, n_slots=4, max_tokens=8)
+    logits = W.normal_logits(8, 8, 0, 0)
+    x = W.noise_x(8, 256, 0, 0, 0)
+    y_dev, r = pr.step(0, logits, x)
+    pr.moe.reset()
+    y_host = torch.empty_like(x)
+    pr.moe.layer_host(0, logits, x, y_host, 8)
+    assert torch.equal(y_host, y_dev.cpu()) or (y_host.float() - y_dev.cpu().float()).abs().max() < 1e-3
+    check_output(y_host, r.y)
+    pr.close()
+
+
+@pytest.mark.parametrize("batch", [1, 8])
+def test_qwen3_shaped_decode_two_layers(batch):
+    """d=2048, 128 experts, I=768, top-8, 64 slots per layer; AR(1) + Zipf logits; teacher-forced layers."""
+    shape = W.QWEN3_30B
+    L, steps = 2, 6
+    pr = Pair(shape, n_slots=64, max_tokens=8, n_layers=L, seed=0, gen_device="cuda")
+    logits = W.ar1_logits(L, steps, batch, 128, rho=0.8, alpha=1.1, seed=0)
+    for t in range(steps):
+        y_prev = None
+        for l in range(L):
+            n = W.noise_x(batch, 2048, 0, t, l)
+            x = n if y_prev is None else (n.float() + y_prev.float().cpu()).to(torch.bfloat16)
+            y_prev, _ = pr.step(l, logits[t, l], x, check_y=(t in (0, steps - 1)), check_slots=(t == 0 and l == 0))
+    st = pr.moe.get_stats(0)
+    assert st["hits"] > 0 and st["fills"] > 0
+    pr.close()
