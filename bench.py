@@ -1,0 +1,422 @@
+#!/usr/bin/env python
+"""Decode throughput of the expert-cached MoE stack on B200 (one JSON line on stdout).
+
+Workload (the Qwen3-30B-A3B-shaped decode configuration): 48 independent MoE layers, d=2048,
+128 SwiGLU experts of intermediate 768, top-8, bf16 weights ~N(0,0.02) in a pinned host pool
+(54 GiB), HBM cache of 64 slots per layer (50 %), router logits from an AR(1) chain (rho 0.8) plus a
+Zipf-style bias (alpha 1.1), layer inputs x_l = bf16(noise_l + y_{l-1}).  A step is one decode step
+of `--batch` tokens through all layers: route -> plan -> fill -> expert FFN -> combine per layer.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--batch 8]
+
+`value` is whole-job tokens/s with inputs resident in HBM; `e2e` is the same through the
+host-buffer entry point (logits and x copied host->device and y device->host every layer).
+`roofline` is the resident-expert streaming kernel: algorithmic bytes = resident experts x record
+bytes, duration from CUDA events on the launching stream, peak from MEASURED_PEAKS.json.
+With N > 1 every rank runs an independent replica (the path has no exchange step).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+SEED = 0
+RHO, ALPHA = 0.8, 1.1
+FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock/throttle samples during the timed region."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.path = index, None, f"/tmp/ftmoe_clocks_{os.getpid()}.csv"
+
+    def start(self):
+        try:
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for ln in open(self.path):
+                parts = [p.strip() for p in ln.split(",")]
+                if len(parts) < 7:
+                    continue
+                try:
+                    sm.append(float(parts[0]))
+                    mx.append(float(parts[1]))
+                except ValueError:
+                    continue
+                for n, v in zip(names, parts[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            os.remove(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def oracle_sample_seconds(pool_np, shape, n_slots, cm_args, logits_step, x_bits_by_layer, layers):
+    """Times the CPU oracle (as it stands) on `layers` layers of one decode step."""
+    from oracle import ftmoe_oracle as O
+    cm = O.CostModel(*cm_args)
+    t0 = time.perf_counter()
+    for l in layers:
+        ora = O.OracleLayer(shape.d, shape.inter, shape.n_experts, shape.top_k, n_slots, shape.wdtype,
+                            pool_np[l], cm)
+        ora.step(logits_step[l], x_bits_by_layer[l])
+    return time.perf_counter() - t0
+
+
+def run_reference(args):
+    """The reference arm of this tier is the CPU oracle, timed as it stands on the host cores."""
+    import torch
+    from paper_2608_16157_b200 import workload as W
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    shape = W.QWEN3_30B
+    B = args.batch
+    S = shape.expert_bytes
+    n_layers_pool = 2                      # the sample never needs more than two layers of weights
+    pool = torch.empty(n_layers_pool * shape.n_experts * S, dtype=torch.uint8)
+    W.fill_pool(pool, shape, n_layers_pool, SEED)
+    pool_np = pool.view(n_layers_pool, shape.n_experts, S).numpy()
+    steps_total = args.steps + args.warmup
+    logits = W.ar1_logits(n_layers_pool, steps_total, B, shape.n_experts, RHO, ALPHA, SEED)
+    cm_args = (S, 50000, 0, 50000, 6000000, 1, 64, 128)
+    from oracle import ftmoe_oracle as O
+    cm = O.CostModel(*cm_args)
+    ora = O.OracleLayer(shape.d, shape.inter, shape.n_experts, shape.top_k, 64, "bf16", pool_np[0], cm)
+    # size the per-step sample (batch rows of one layer) so the whole run stays within ~2.5 minutes
+    x0 = W.noise_x(B, shape.d, SEED, 0, 0).view(torch.int16).numpy().view(np.uint16)
+    t0 = time.perf_counter()
+    ora.step(logits[0, 0][:1], x0[:1])
+    t_row = time.perf_counter() - t0
+    rows = int(max(1, min(B, 150.0 / max(steps_total, 1) / max(t_row, 1e-6))))
+    ora.state.reset()
+    times = []
+    for s in range(steps_total):
+        x = W.noise_x(B, shape.d, SEED, s, 0).view(torch.int16).numpy().view(np.uint16)
+        t0 = time.perf_counter()
+        ora.step(logits[s, 0][:rows], x[:rows])
+        dt = time.perf_counter() - t0
+        if s >= args.warmup:
+            times.append(dt)
+    per_step = sum(times) / max(len(times), 1) * 48            # one layer timed, 48 in the stack
+    value = rows / per_step
+    cores = len(os.sched_getaffinity(0))
+    sample = f"{rows} of {B} batch rows through 1 of 48 layers per step, time scaled x48"
+    line = {"impl": "reference", "metric": "moe_decode_tok_per_s", "value": value, "unit": "tok/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic",
+            "config": {"workload": "decode Qwen3-30B-A3B-shaped MoE stack (config 1)", "batch": B,
+                       "layers": 48, "hidden": shape.d, "experts": shape.n_experts, "inter": shape.inter,
+                       "top_k": shape.top_k, "slots_per_layer": 64},
+            "cpu_baseline": {"value": value, "unit": "tok/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "tok/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args):
+    import torch
+    from paper_2608_16157_b200 import binding as Bd
+    from paper_2608_16157_b200 import workload as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    shape = W.QWEN3_30B
+    L, E, k, d = args.layers, shape.n_experts, shape.top_k, shape.d
+    S = shape.expert_bytes
+    Ns = W.slots_for_fraction(args.cache_frac, E)
+    B = args.batch
+    Wn, K = args.warmup, args.steps
+    t_setup = time.perf_counter()
+    pool = Bd.HostPool(L * E * S)
+    W.fill_pool(pool.tensor, shape, L, SEED, device=dev, chunk=32)
+    log(f"[rank {rank}] pool {L * E * S / 2**30:.1f} GiB pinned+filled in {time.perf_counter() - t_setup:.1f}s")
+
+    fill_mode = Bd.FT_FILL_SM if args.fill == "sm" else Bd.FT_FILL_COPY_ENGINE
+
+    def make(bw):
+        cfg = Bd.make_config(hidden=d, inter=shape.inter, n_experts=E, top_k=k, n_layers=L, slots_per_layer=Ns,
+                             max_tokens=max(B, 8), host_pool_ptr=pool.ptr.value, host_pool_bytes=pool.n_bytes,
+                             fill_mode=fill_mode, device=local, **bw)
+        return Bd.FtMoe(cfg)
+
+    # bandwidth profiling at deployment, then frozen into the plan's cost model
+    moe = make({})
+    cal = moe.calibrate()
+    moe.destroy()
+    log(f"[rank {rank}] calibrate MB/s: {cal}")
+    bw = dict(bw_fill=max(cal["fill_MBps"], 1), bw_zc=max(cal["zc_MBps"], 1),
+              bw_zc_residual=cal["zc_residual_MBps"] if args.residual else 0, bw_hbm=max(cal["hbm_MBps"], 1))
+    moe = make(bw)
+
+    stream = torch.cuda.current_stream()
+    n_total = Wn + K + args.prof_steps + 8
+
+    def gen_inputs(batch):
+        lg = torch.from_numpy(W.ar1_logits(L, n_total, batch, E, RHO, ALPHA, SEED)).to(dev)
+        g = torch.Generator(device=dev)
+        g.manual_seed(W.mix64(SEED, 77, batch))
+        noise = torch.randn((n_total, L, batch, d), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        return lg, noise
+
+    xbuf = torch.empty((L, max(B, 8), d), dtype=torch.bfloat16, device=dev)
+    ybuf = torch.empty((L, max(B, 8), d), dtype=torch.bfloat16, device=dev)
+
+    def step(lg, noise, s, batch):
+        for l in range(L):
+            if l == 0:
+                x = noise[s, 0]
+            else:
+                x = xbuf[l, :batch]
+                torch.add(noise[s, l], ybuf[l - 1, :batch], out=x)
+            moe.layer(l, lg[s, l], x, ybuf[l, :batch], batch, stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(lg, noise, batch, first, count, sample_clocks=False):
+        sampler = ClockSampler(local) if sample_clocks else None
+        barrier()
+        if sampler:
+            sampler.start()
+            time.sleep(0.3)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0 = moe.launch_count()
+        e0.record(stream)
+        for s in range(first, first + count):
+            step(lg, noise, s, batch)
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        clocks = sampler.stop() if sampler else None
+        launches = moe.launch_count() - l0 + count * (L - 1)     # + the harness's x = noise + y kernels
+        if dist is not None:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, clocks, launches
+
+    def stats_sum():
+        tot = {}
+        for l in range(L):
+            for kk, v in moe.get_stats(l).items():
+                tot[kk] = tot.get(kk, 0) + v
+        return tot
+
+    results = {}
+    for batch in ([B] if args.only_batch else [B, 1] if B != 1 else [1]):
+        lg, noise = gen_inputs(batch)
+        moe.reset()
+        for s in range(Wn):
+            step(lg, noise, s, batch)
+        torch.cuda.synchronize()
+        st0 = stats_sum()
+        ms, clocks, launches = timed(lg, noise, batch, Wn, K, sample_clocks=(batch == B))
+        st1 = stats_sum()
+        dst = {kk: st1[kk] - st0[kk] for kk in st1}
+        # per-kernel durations with CUDA events on the launching stream (separate pass: events perturb)
+        moe.timing_enable(True)
+        st2 = stats_sum()
+        for s in range(Wn + K, Wn + K + args.prof_steps):
+            step(lg, noise, s, batch)
+        tim = moe.timing_read()
+        st3 = stats_sum()
+        moe.timing_enable(False)
+        res_bytes = (st3["hits"] - st2["hits"] + st3["fills"] - st2["fills"]) * S
+        results[batch] = dict(ms=ms, clocks=clocks, launches=launches, dstats=dst, timing=tim,
+                              res_bytes=res_bytes, prof_fill_bytes=(st3["fills"] - st2["fills"]) * S,
+                              lg=lg, noise=noise)
+        log(f"[rank {rank}] batch {batch}: {ms / K:.3f} ms/step, {batch * K * world / (ms * 1e-3):.1f} tok/s, "
+            f"per step: hits {dst['hits'] / K:.1f} fills {dst['fills'] / K:.2f} zc {dst['zc'] / K:.2f}")
+        log(f"[rank {rank}]   kernel timing (us total, launches): {tim}")
+
+    main = results[B]
+    value = B * K * world / (main["ms"] * 1e-3)
+    hbm_peak, peak_kind = peaks()
+    tim = main["timing"]
+    ffn_us, ffn_n = tim["ffn_res"]
+    achieved = main["res_bytes"] / (ffn_us * 1e-6) / 1e9 if ffn_us > 0 else 0.0
+    fill_us, fill_n = tim["fill"]
+
+    # end to end through the host-buffer entry point
+    e2e = None
+    if args.e2e_steps > 0:
+        lg, noise = main["lg"], main["noise"]
+        lg_h = lg.cpu().pin_memory()
+        noise_h = noise.cpu().pin_memory()
+        xh = torch.empty((L, B, d), dtype=torch.bfloat16).pin_memory()
+        yh = torch.empty((L, B, d), dtype=torch.bfloat16).pin_memory()
+        Ke = min(K, args.e2e_steps)
+
+        def step_host(s):
+            for l in range(L):
+                if l == 0:
+                    x = noise_h[s, 0]
+                else:
+                    x = xh[l]
+                    torch.add(noise_h[s, l], yh[l - 1], out=x)
+                moe.layer_host(l, lg_h[s, l], x, yh[l], B, stream)
+
+        for s in range(Wn + K, Wn + K + 3):
+            step_host(s)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for s in range(Wn, Wn + Ke):
+            step_host(s)
+        e1.record(stream)
+        barrier()
+        ms_e = e0.elapsed_time(e1)
+        if dist is not None:
+            t = torch.tensor([ms_e], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e = float(t.item())
+        e2e = {"value": B * Ke * world / (ms_e * 1e-3), "unit": "tok/s",
+               "h2d_bytes_per_step": L * (B * E * 4 + B * d * 2), "d2h_bytes_per_step": L * B * d * 2,
+               "steps": Ke}
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        lg, noise = main["lg"], main["noise"]
+        n_samp = args.cpu_layers
+        pool_np = pool.tensor.view(L, E, S).numpy()
+        lg_np = lg[Wn].cpu().numpy()
+        xb = [noise[Wn, l].cpu().view(torch.int16).numpy().view(np.uint16) for l in range(n_samp)]
+        cm_args = (S, bw["bw_fill"], bw["bw_zc_residual"], bw["bw_zc"], bw["bw_hbm"], 1, 64, 128)
+        sec = oracle_sample_seconds(pool_np, shape, Ns, cm_args, lg_np, xb, range(n_samp))
+        cpu_baseline = {"value": B / (sec * L / n_samp), "unit": "tok/s", "cores": len(os.sched_getaffinity(0)),
+                        "kind": "oracle",
+                        "sample": f"{n_samp} of {L} layers of one decode step at batch {B} "
+                                  f"({sec:.1f} s), time scaled x{L / n_samp:.0f}"}
+
+    if rank == 0:
+        dst = main["dstats"]
+        line = {
+            "metric": "moe_decode_tok_per_s", "value": value, "unit": "tok/s", "n_gpus": world, "steps": K,
+            "warmup": Wn, "ms_per_step": main["ms"] / K, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "decode Qwen3-30B-A3B-shaped MoE stack (config 1)", "batch": B, "layers": L,
+                       "hidden": d, "experts": E, "inter": shape.inter, "top_k": k, "slots_per_layer": Ns,
+                       "fill_mode": args.fill, "rho": RHO, "zipf_alpha": ALPHA,
+                       "l2": "inputs larger than L2: each step streams >= 3.4 GB of distinct expert records "
+                             "from a 27 GiB slot pool, no L2 flush needed",
+                       "parallelism": "replicas" if world > 1 else "single"},
+            "clocks": main["clocks"],
+            "e2e": e2e,
+            "gpu_launches": main["launches"],
+            "roofline": {"bound": "hbm", "kernel": "ffn_stream_kernel (resident experts)",
+                         "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
+                         "frac": achieved / hbm_peak if hbm_peak else None, "peak_source": peak_kind,
+                         "launches_timed": ffn_n, "avg_launch_us": ffn_us / ffn_n if ffn_n else None,
+                         "bytes_per_launch": main["res_bytes"] / ffn_n if ffn_n else None,
+                         "traffic": None},
+            "cpu_baseline": cpu_baseline,
+            "per_step": {"hits": dst["hits"] / K, "fills": dst["fills"] / K, "zero_copy": dst["zc"] / K,
+                         "routed_unique": dst["routed"] / K, "fill_bytes": dst["fills"] / K * S},
+            "fill": {"GBps": (main["prof_fill_bytes"] / (fill_us * 1e-6) / 1e9) if fill_us > 0 else None,
+                     "link_GBps_measured": cal["fill_MBps"] / 1e3, "zero_copy_GBps_measured": cal["zc_MBps"] / 1e3,
+                     "zero_copy_residual_GBps_measured": cal["zc_residual_MBps"] / 1e3,
+                     "hbm_read_GBps_measured": cal["hbm_MBps"] / 1e3},
+            "kernel_us_per_launch": {kk: (v[0] / v[1] if v[1] else None) for kk, v in tim.items()},
+        }
+        if 1 in results and B != 1:
+            r1 = results[1]
+            t1 = r1["timing"]
+            a1 = r1["res_bytes"] / (t1["ffn_res"][0] * 1e-6) / 1e9 if t1["ffn_res"][0] > 0 else 0.0
+            line["batch1"] = {"value": K * world / (r1["ms"] * 1e-3), "unit": "tok/s", "ms_per_step": r1["ms"] / K,
+                              "ffn_res_GBps": a1, "ffn_res_frac": a1 / hbm_peak,
+                              "fills_per_step": r1["dstats"]["fills"] / K}
+        print(json.dumps(line), flush=True)
+    moe.destroy()
+    pool.free()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--warmup", type=int, default=32)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=8)
+    ap.add_argument("--layers", type=int, default=48)
+    ap.add_argument("--cache-frac", type=float, default=0.5)
+    ap.add_argument("--fill", default="ce", choices=["ce", "sm"])
+    ap.add_argument("--residual", type=int, default=0, help="use the measured residual zero-copy rate in the plan")
+    ap.add_argument("--prof-steps", type=int, default=16)
+    ap.add_argument("--e2e-steps", type=int, default=32)
+    ap.add_argument("--cpu-layers", type=int, default=4)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--only-batch", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

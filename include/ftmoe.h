@@ -190,6 +190,14 @@ ft_status_t ft_moe_reset(ft_moe_t *h, int layer);
 ft_status_t ft_moe_sync_status(ft_moe_t *h);
 /* Duration of the most recent ft_moe_fill's copies in microseconds and their bytes (waits for them). */
 ft_status_t ft_moe_last_fill(ft_moe_t *h, float *out_us, uint64_t *out_bytes);
+/* Per-kernel device timing with CUDA events on the launching stream.  enable(1) clears the
+ * accumulators and brackets every later launch with two events; read() waits for the device and
+ * returns, per kind FT_TIME_*, the summed microseconds and the number of timed launches since
+ * enable.  Timing adds two event records per launch, so throughput is measured with it off. */
+enum { FT_TIME_ROUTE = 0, FT_TIME_PLAN, FT_TIME_FFN_ZC, FT_TIME_FFN_RES, FT_TIME_FINALIZE, FT_TIME_FILL,
+       FT_TIME_COUNT };
+ft_status_t ft_moe_timing_enable(ft_moe_t *h, int on);
+ft_status_t ft_moe_timing_read(ft_moe_t *h, double *out_us, uint64_t *out_launches, int n);
 /* Number of kernels this handle has launched since create. */
 ft_status_t ft_moe_launch_count(ft_moe_t *h, uint64_t *out);
 const char *ft_moe_status_string(ft_status_t s);

@@ -25,8 +25,9 @@ SYMBOLS = (
     "ft_moe_calibrate", "ft_moe_route", "ft_moe_plan", "ft_moe_fill", "ft_moe_forward", "ft_moe_layer",
     "ft_moe_layer_host", "ft_moe_get_routing", "ft_moe_get_slot_table", "ft_moe_read_slot",
     "ft_moe_get_stats", "ft_moe_reset", "ft_moe_sync_status", "ft_moe_last_fill", "ft_moe_launch_count",
-    "ft_moe_status_string",
+    "ft_moe_status_string", "ft_moe_timing_enable", "ft_moe_timing_read",
 )
+TIME_NAMES = ("route", "plan", "ffn_zc", "ffn_res", "finalize", "fill")
 
 
 class Config(C.Structure):
@@ -93,6 +94,8 @@ def load(rebuild: bool = False):
         "ft_moe_last_fill": (i32, [vp, C.POINTER(C.c_float), C.POINTER(C.c_uint64)]),
         "ft_moe_launch_count": (i32, [vp, C.POINTER(C.c_uint64)]),
         "ft_moe_status_string": (C.c_char_p, [i32]),
+        "ft_moe_timing_enable": (i32, [vp, i32]),
+        "ft_moe_timing_read": (i32, [vp, vp, vp, i32]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -279,6 +282,16 @@ class FtMoe:
         us, b = C.c_float(), C.c_uint64()
         _check(self._lib.ft_moe_last_fill(self._h, C.byref(us), C.byref(b)), "ft_moe_last_fill")
         return float(us.value), int(b.value)
+
+    def timing_enable(self, on=True):
+        _check(self._lib.ft_moe_timing_enable(self._h, 1 if on else 0), "ft_moe_timing_enable")
+
+    def timing_read(self):
+        """{kind: (total microseconds, timed launches)} since timing was enabled."""
+        us = np.zeros(len(TIME_NAMES), dtype=np.float64)
+        n = np.zeros(len(TIME_NAMES), dtype=np.uint64)
+        _check(self._lib.ft_moe_timing_read(self._h, _ptr(us), _ptr(n), len(TIME_NAMES)), "ft_moe_timing_read")
+        return {k: (float(a), int(b)) for k, a, b in zip(TIME_NAMES, us, n)}
 
     def launch_count(self):
         n = C.c_uint64()

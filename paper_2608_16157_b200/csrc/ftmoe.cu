@@ -65,6 +65,13 @@ struct ft_moe {
   bool fill_timed = false;
   int last_routed_layer = -1;
   uint64_t launches = 0;
+  // optional per-kernel timing (CUDA events on the launching stream)
+  bool timing = false;
+  struct Pending { int kind; cudaEvent_t e0, e1; };
+  std::vector<Pending> pending;
+  std::vector<cudaEvent_t> free_events;
+  double time_us[FT_TIME_COUNT] = {0};
+  uint64_t time_n[FT_TIME_COUNT] = {0};
 };
 
 namespace {
@@ -119,6 +126,53 @@ ft_status_t drain_status(ft_moe *h) {
   }
   return FT_OK;
 }
+
+cudaEvent_t timing_event(ft_moe *h) {
+  if (!h->free_events.empty()) {
+    cudaEvent_t e = h->free_events.back();
+    h->free_events.pop_back();
+    return e;
+  }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+
+void timing_flush(ft_moe *h) {
+  for (auto &p : h->pending) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(p.e1) == cudaSuccess && cudaEventElapsedTime(&ms, p.e0, p.e1) == cudaSuccess) {
+      h->time_us[p.kind] += (double)ms * 1000.0;
+      h->time_n[p.kind] += 1;
+    }
+    h->free_events.push_back(p.e0);
+    h->free_events.push_back(p.e1);
+  }
+  h->pending.clear();
+  (void)cudaGetLastError();
+}
+
+// Brackets the launches issued in its lifetime on `st` with two events when timing is on.
+struct TimeScope {
+  ft_moe *h;
+  cudaStream_t st;
+  int kind;
+  cudaEvent_t e0 = nullptr;
+  TimeScope(ft_moe *h_, cudaStream_t st_, int kind_) : h(h_), st(st_), kind(kind_) {
+    if (h->timing) {
+      if (h->pending.size() >= 4096) timing_flush(h);
+      e0 = timing_event(h);
+      cudaEventRecord(e0, st);
+    }
+  }
+  ~TimeScope() {
+    if (e0) {
+      cudaEvent_t e1 = timing_event(h);
+      cudaEventRecord(e1, st);
+      h->pending.push_back({kind, e0, e1});
+    }
+  }
+};
 
 ft_status_t reset_layer(ft_moe *h, int l) {
   LayerState &L = h->layers[l];
@@ -224,6 +278,8 @@ ft_status_t ft_moe_destroy(ft_moe_t *h) {
   cudaEvent_t evs[] = {h->ev_plan, h->ev_fill, h->ev_fork, h->ev_join, h->ev_fill_t0, h->ev_fill_t1};
   for (cudaEvent_t e : evs)
     if (e) cudaEventDestroy(e);
+  for (auto &p : h->pending) { cudaEventDestroy(p.e0); cudaEventDestroy(p.e1); }
+  for (cudaEvent_t e : h->free_events) cudaEventDestroy(e);
   (void)cudaGetLastError();
   delete h;
   return FT_OK;
@@ -378,6 +434,7 @@ ft_status_t ft_moe_route(ft_moe_t *h, int layer, const float *logits_dev, int T,
   rp.T = T; rp.E = h->cfg.n_experts; rp.k = h->cfg.top_k;
   rp.ids = h->ids; rp.w = h->topk_w; rp.count = h->count; rp.offset = h->offset;
   rp.perm = h->perm; rp.inv = h->inv; rp.status = h->status_dev;
+  TimeScope ts(h, st, FT_TIME_ROUTE);
   if (T <= kRouteSmallMaxTokens) {
     route_small_kernel<<<1, 1024, 0, st>>>(rp);
     h->launches++;
@@ -417,7 +474,10 @@ ft_status_t ft_moe_plan(ft_moe_t *h, int layer, ft_moe_plan_t *out, void *stream
     pp.items_res = h->items_res; pp.items_zc = h->items_zc; pp.items_gemm = h->items_gemm;
     pp.seq = h->seq_dev;
     const size_t smem = (size_t)c.slots_per_layer * 16;
-    plan_kernel<<<1, 1024, smem, st>>>(pp);
+    {
+      TimeScope ts(h, st, FT_TIME_PLAN);
+      plan_kernel<<<1, 1024, smem, st>>>(pp);
+    }
     h->launches++;
     h->seq_host++;
     FT_CUDA(cudaGetLastError());
@@ -475,10 +535,13 @@ ft_status_t ft_moe_fill(ft_moe_t *h, int layer, void *copy_stream) {
       const uint8_t *pool_layer = static_cast<const uint8_t *>(c.host_pool) + (size_t)layer * E * h->S;
       FT_CUDA(cudaStreamWaitEvent(cs, h->ev_plan, 0));
       FT_CUDA(cudaEventRecord(h->ev_fill_t0, cs));
-      for (int i = 0; i < hd.n_fill; ++i) {
-        if (forder[i] < 0 || forder[i] >= E || fslot[i] < 0 || fslot[i] >= c.slots_per_layer) return FT_ERR_CUDA;
-        FT_CUDA(cudaMemcpyAsync(slots_layer + (size_t)fslot[i] * h->S, pool_layer + (size_t)forder[i] * h->S,
-                                h->S, cudaMemcpyHostToDevice, cs));
+      {
+        TimeScope ts(h, cs, FT_TIME_FILL);
+        for (int i = 0; i < hd.n_fill; ++i) {
+          if (forder[i] < 0 || forder[i] >= E || fslot[i] < 0 || fslot[i] >= c.slots_per_layer) return FT_ERR_CUDA;
+          FT_CUDA(cudaMemcpyAsync(slots_layer + (size_t)fslot[i] * h->S, pool_layer + (size_t)forder[i] * h->S,
+                                  h->S, cudaMemcpyHostToDevice, cs));
+        }
       }
       FT_CUDA(cudaEventRecord(h->ev_fill_t1, cs));
       FT_CUDA(cudaEventRecord(h->ev_fill, cs));
@@ -496,7 +559,10 @@ ft_status_t ft_moe_fill(ft_moe_t *h, int layer, void *copy_stream) {
     fp.slots_layer = slots_layer; fp.S = h->S;
     FT_CUDA(cudaStreamWaitEvent(cs, h->ev_plan, 0));
     FT_CUDA(cudaEventRecord(h->ev_fill_t0, cs));
-    fill_kernel<<<h->sm_count * 4, 256, 0, cs>>>(fp);
+    {
+      TimeScope ts(h, cs, FT_TIME_FILL);
+      fill_kernel<<<h->sm_count * 4, 256, 0, cs>>>(fp);
+    }
     h->launches++;
     FT_CUDA(cudaGetLastError());
     FT_CUDA(cudaEventRecord(h->ev_fill_t1, cs));
@@ -523,16 +589,23 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   // zero-copy set first: it does not depend on the fills and shares the host link with them
   fp.items = h->items_zc;
   fp.n_items = &h->plan_dev->n_zc_items;
-  launch_stream_any(h, fp, L.T, st);
+  {
+    TimeScope ts(h, st, FT_TIME_FFN_ZC);
+    launch_stream_any(h, fp, L.T, st);
+  }
   // resident set after the fills have landed
   if (c.slots_per_layer > 0) FT_CUDA(cudaStreamWaitEvent(st, h->ev_fill, 0));
   if (c.slots_per_layer > 0 || c.n_shared) {
     fp.items = h->items_res;
     fp.n_items = &h->plan_dev->n_res_items;
+    TimeScope ts(h, st, FT_TIME_FFN_RES);
     launch_stream_any(h, fp, L.T, st);
   }
   const long long n4 = (long long)L.T * c.hidden / 4;
-  finalize_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(h->y_acc, static_cast<__nv_bfloat16 *>(y_dev), n4);
+  {
+    TimeScope ts(h, st, FT_TIME_FINALIZE);
+    finalize_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(h->y_acc, static_cast<__nv_bfloat16 *>(y_dev), n4);
+  }
   h->launches++;
   FT_CUDA(cudaGetLastError());
   return FT_OK;
@@ -647,6 +720,25 @@ ft_status_t ft_moe_last_fill(ft_moe_t *h, float *out_us, uint64_t *out_bytes) {
 ft_status_t ft_moe_launch_count(ft_moe_t *h, uint64_t *out) {
   if (!h || !out) return FT_ERR_INVALID_ARG;
   *out = h->launches;
+  return FT_OK;
+}
+
+ft_status_t ft_moe_timing_enable(ft_moe_t *h, int on) {
+  if (!h) return FT_ERR_INVALID_ARG;
+  FT_CUDA(cudaSetDevice(h->cfg.device));
+  FT_CUDA(cudaDeviceSynchronize());
+  timing_flush(h);
+  for (int i = 0; i < FT_TIME_COUNT; ++i) { h->time_us[i] = 0.0; h->time_n[i] = 0; }
+  h->timing = on != 0;
+  return FT_OK;
+}
+
+ft_status_t ft_moe_timing_read(ft_moe_t *h, double *out_us, uint64_t *out_n, int n) {
+  if (!h || !out_us || !out_n || n < 0) return FT_ERR_INVALID_ARG;
+  FT_CUDA(cudaSetDevice(h->cfg.device));
+  FT_CUDA(cudaDeviceSynchronize());
+  timing_flush(h);
+  for (int i = 0; i < n && i < FT_TIME_COUNT; ++i) { out_us[i] = h->time_us[i]; out_n[i] = h->time_n[i]; }
   return FT_OK;
 }
 
