@@ -1,0 +1,330 @@
+// Steps 5+6 for resident bf16 experts at decode-sized token counts: an HBM-streaming SwiGLU FFN.
+//
+// One persistent CTA per SM.  A producer warp streams the expert records through a 3-stage shared
+// memory ring with bulk asynchronous copies (cp.async.bulk + mbarrier complete_tx), one 16-neuron
+// tile of one matrix per stage, so ~190 KB per SM are in flight and HBM never waits for arithmetic.
+// Eight consumer warps turn each tile into tensor-core MMAs (mma.sync m16n8k16, bf16 x bf16 -> fp32)
+// with up to 8 tokens in the N dimension, so the arithmetic cost does not grow with the token count:
+//   gate/up tile: warp w owns the k-slice [w*d/8, (w+1)*d/8); partial [16 neurons x 8 tokens] sums are
+//                 reduced across warps through shared memory, then h = SiLU(g) * u.
+//   down tile   : warp w owns the output columns [w*d/8, (w+1)*d/8); A = Wd^T through
+//                 ldmatrix.trans, B = h; fp32 accumulators persist across the CTA's neuron range.
+// The gate-weighted combine is a red.global.add into the fp32 [T][d] accumulator; the last CTA to
+// finish rounds it once to bf16 and clears it.  Every mbarrier wait is bounded: on expiry the CTA
+// latches a timeout status, stops waiting and runs to completion.
+#pragma once
+#include "common.cuh"
+
+namespace ftmoe {
+
+constexpr int kMmaStages = 3;
+constexpr int kMmaTileRows = 16;
+constexpr int kMmaConsumers = 256;
+constexpr int kMmaThreads = kMmaConsumers + 32;
+constexpr int kMmaTokens = 8;  // tokens per weight pass
+
+struct FfnMmaParams {
+  const WorkItem *items;
+  const int32_t *n_items;
+  const __nv_bfloat16 *x;   // [T][d]
+  const int32_t *perm;
+  const float *topk_w;
+  float *y_acc;             // [T][d]
+  __nv_bfloat16 *y;         // [T][d], written by the last CTA when finalize != 0
+  uint32_t *done;           // CTA completion counter, zero between launches
+  uint32_t *status;
+  int d, inter, top_k, T, finalize;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait; returns false (after latching the abort flag) if the phase never completes.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status) {
+  if (*abort_flag) return false;
+  for (uint32_t i = 0; i < (1u << 22); ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 1023u) == 1023u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  atomicOr(status, kStatTimeout);
+  return false;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+
+// Dynamic shared memory layout (bytes): [stages][16 rows x (2d+64)] | red [8][2][16][8] f32 | hs [8][16] bf16
+// | pref [kMaxExperts+2] i32 | mbarriers full[3], empty[3] | abort flag.
+template <int KB>  // KB = d / 256: 32-wide k-blocks per warp in the gate/up phase
+__global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p) {
+  constexpr int CTW = 2 * KB;  // 16-column tiles per warp in the down phase
+  extern __shared__ __align__(128) unsigned char smem[];
+  const int d = p.d;
+  const uint32_t row_bytes = 2u * d;
+  const uint32_t stride_gu = row_bytes + 64;   // = 64 mod 128: conflict-free 16-byte fragment loads
+  const uint32_t stride_d = row_bytes + 16;    // = 16 mod 128: conflict-free ldmatrix rows
+  const uint32_t stage_bytes = kMmaTileRows * stride_gu;
+  unsigned char *sp = smem + (size_t)kMmaStages * stage_bytes;
+  float *s_red = reinterpret_cast<float *>(sp); sp += 8 * 2 * 16 * 8 * 4;
+  __nv_bfloat16 *s_h = reinterpret_cast<__nv_bfloat16 *>(sp); sp += 8 * 16 * 2;
+  int32_t *s_pref = reinterpret_cast<int32_t *>(sp); sp += (kMaxExperts + 2) * 4;
+  uint64_t *s_bar = reinterpret_cast<uint64_t *>(sp); sp += 2 * kMmaStages * 8;
+  volatile int *s_abort = reinterpret_cast<volatile int *>(sp);
+  __shared__ int s_last;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n_items = *p.n_items;
+  const int NBLK = p.inter / kMmaTileRows;
+  const uint32_t smem_base = smem_u32(smem);
+  const uint32_t bar_base = smem_u32(s_bar);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (kMmaStages + s); };
+
+  if (tid == 0) {
+    for (int s = 0; s < kMmaStages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 8);
+    }
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  // passes per item (8 tokens per pass) and their prefix sums
+  for (int i = tid; i < n_items; i += blockDim.x) s_pref[i + 1] = (p.items[i].n_tok + kMmaTokens - 1) / kMmaTokens;
+  __syncthreads();
+  if (tid == 0) {
+    s_pref[0] = 0;
+    for (int i = 0; i < n_items; ++i) s_pref[i + 1] += s_pref[i];
+  }
+  __syncthreads();
+  const long long total = (long long)s_pref[n_items] * NBLK;
+  long long u = total * blockIdx.x / gridDim.x;
+  const long long u1 = total * (blockIdx.x + 1) / gridDim.x;
+  int item = 0;
+  uint32_t tile = 0;  // tiles consumed / produced so far by this CTA
+
+  if (warp == 8) {
+    // ------------------------------ producer ------------------------------
+    if (lane == 0) {
+      while (u < u1) {
+        const long long pu = u / NBLK;
+        while (s_pref[item + 1] <= pu) ++item;
+        const int b_begin = (int)(u - pu * NBLK);
+        const long long left = u1 - u;
+        const int b_end = (left < (long long)(NBLK - b_begin)) ? b_begin + (int)left : NBLK;
+        const uint8_t *rec = p.items[item].w;
+        const size_t mat_bytes = (size_t)row_bytes * p.inter;
+        for (int b = b_begin; b < b_end; ++b) {
+#pragma unroll 1
+          for (int which = 0; which < 3; ++which) {
+            const int s = tile % kMmaStages;
+            const uint32_t ph = (tile / kMmaStages) & 1u;
+            mbar_wait(empty_bar(s), ph ^ 1u, s_abort, p.status);
+            if (*s_abort) break;
+            mbar_expect_tx(full_bar(s), kMmaTileRows * row_bytes);
+            const uint8_t *src = rec + which * mat_bytes + (size_t)b * kMmaTileRows * row_bytes;
+            const uint32_t dst = smem_base + s * stage_bytes;
+            const uint32_t stride = (which == 2) ? stride_d : stride_gu;
+#pragma unroll 4
+            for (int r = 0; r < kMmaTileRows; ++r) bulk_g2s(dst + r * stride, src + (size_t)r * row_bytes, row_bytes, full_bar(s));
+            ++tile;
+          }
+        }
+        u += (b_end - b_begin);
+      }
+    }
+  } else {
+    // ------------------------------ consumers ------------------------------
+    const int g = lane >> 2, q = lane & 3;
+    const int kslice = warp * (d / 8);      // first k of this warp's slice (gate/up) and first column (down)
+    while (u < u1) {
+      const long long pu = u / NBLK;
+      while (s_pref[item + 1] <= pu) ++item;
+      const int pass = (int)(pu - s_pref[item]);
+      const int b_begin = (int)(u - pu * NBLK);
+      const long long left = u1 - u;
+      const int b_end = (left < (long long)(NBLK - b_begin)) ? b_begin + (int)left : NBLK;
+      const WorkItem it = p.items[item];
+      const int nt = min(kMmaTokens, it.n_tok - kMmaTokens * pass);
+      // token g of this pass: row of x and gate weight
+      int tok_g = -1;
+      float gw_g = 0.f;
+      if (g < nt) {
+        if (it.expert >= 0) {
+          const int pr = p.perm[it.off + kMmaTokens * pass + g];
+          tok_g = pr / p.top_k;
+          gw_g = p.topk_w[pr];
+        } else {
+          tok_g = kMmaTokens * pass + g;
+          gw_g = 1.f;
+        }
+      }
+      uint32_t xf[KB][4];
+#pragma unroll
+      for (int kb = 0; kb < KB; ++kb) {
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (tok_g >= 0) v = *reinterpret_cast<const uint4 *>(p.x + (size_t)tok_g * d + kslice + 32 * kb + 8 * q);
+        xf[kb][0] = v.x; xf[kb][1] = v.y; xf[kb][2] = v.z; xf[kb][3] = v.w;
+      }
+      float dacc[CTW][4];
+#pragma unroll
+      for (int c = 0; c < CTW; ++c) { dacc[c][0] = dacc[c][1] = dacc[c][2] = dacc[c][3] = 0.f; }
+
+      for (int b = b_begin; b < b_end; ++b) {
+        float cgu[2][4];
+#pragma unroll
+        for (int which = 0; which < 2; ++which) {
+          const int s = tile % kMmaStages;
+          const uint32_t ph = (tile / kMmaStages) & 1u;
+          cgu[which][0] = cgu[which][1] = cgu[which][2] = cgu[which][3] = 0.f;
+          const bool ok = mbar_wait(full_bar(s), ph, s_abort, p.status);
+          if (ok) {
+            const uint32_t base = smem_base + s * stage_bytes + (uint32_t)(kslice + 8 * q) * 2u;
+#pragma unroll
+            for (int kb = 0; kb < KB; ++kb) {
+              const uint4 lo = lds_v4(base + g * stride_gu + kb * 64);
+              const uint4 hi = lds_v4(base + (g + 8) * stride_gu + kb * 64);
+              mma_bf16(cgu[which], lo.x, hi.x, lo.y, hi.y, xf[kb][0], xf[kb][1]);
+              mma_bf16(cgu[which], lo.z, hi.z, lo.w, hi.w, xf[kb][2], xf[kb][3]);
+            }
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(empty_bar(s));
+          ++tile;
+        }
+        // cross-warp reduction of the [16 neurons][8 tokens] partial sums
+        {
+          float *r0 = s_red + ((warp * 2 + 0) * 16) * 8;
+          float *r1 = s_red + ((warp * 2 + 1) * 16) * 8;
+          *reinterpret_cast<float2 *>(r0 + g * 8 + 2 * q) = make_float2(cgu[0][0], cgu[0][1]);
+          *reinterpret_cast<float2 *>(r0 + (g + 8) * 8 + 2 * q) = make_float2(cgu[0][2], cgu[0][3]);
+          *reinterpret_cast<float2 *>(r1 + g * 8 + 2 * q) = make_float2(cgu[1][0], cgu[1][1]);
+          *reinterpret_cast<float2 *>(r1 + (g + 8) * 8 + 2 * q) = make_float2(cgu[1][2], cgu[1][3]);
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (tid < 128) {
+          const int n = tid >> 3, t = tid & 7;
+          float a = 0.f, c = 0.f;
+#pragma unroll
+          for (int w = 0; w < 8; ++w) {
+            a += s_red[((w * 2 + 0) * 16 + n) * 8 + t];
+            c += s_red[((w * 2 + 1) * 16 + n) * 8 + t];
+          }
+          const float h = a / (1.f + __expf(-a)) * c;
+          s_h[t * 16 + n] = __float2bfloat16_rn(h);
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        // down tile
+        {
+          const int s = tile % kMmaStages;
+          const uint32_t ph = (tile / kMmaStages) & 1u;
+          const bool ok = mbar_wait(full_bar(s), ph, s_abort, p.status);
+          if (ok) {
+            const uint32_t *h32 = reinterpret_cast<const uint32_t *>(s_h);
+            const uint32_t b0 = h32[g * 8 + q], b1 = h32[g * 8 + q + 4];
+            // ldmatrix.x4.trans: lanes 0-7 / 8-15 / 16-23 / 24-31 address the four 8x8 blocks
+            const int mat = lane >> 3, r = lane & 7;
+            const uint32_t abase = smem_base + s * stage_bytes + (uint32_t)(r + 8 * (mat >> 1)) * stride_d +
+                                   (uint32_t)(kslice + 8 * (mat & 1)) * 2u;
+#pragma unroll
+            for (int c = 0; c < CTW; ++c) {
+              uint32_t a[4];
+              ldmatrix_x4_trans(a, abase + c * 32);
+              mma_bf16(dacc[c], a[0], a[1], a[2], a[3], b0, b1);
+            }
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(empty_bar(s));
+          ++tile;
+        }
+      }
+      // gate-weighted combine: D fragment = [column g / g+8 of the tile][tokens 2q, 2q+1]
+      {
+        const int tok_a = __shfl_sync(0xffffffffu, tok_g, (2 * q) * 4);
+        const int tok_b = __shfl_sync(0xffffffffu, tok_g, (2 * q + 1) * 4);
+        const float gw_a = __shfl_sync(0xffffffffu, gw_g, (2 * q) * 4);
+        const float gw_b = __shfl_sync(0xffffffffu, gw_g, (2 * q + 1) * 4);
+#pragma unroll
+        for (int c = 0; c < CTW; ++c) {
+          const int col = kslice + 16 * c + g;
+          if (tok_a >= 0) {
+            atomicAdd(p.y_acc + (size_t)tok_a * d + col, gw_a * dacc[c][0]);
+            atomicAdd(p.y_acc + (size_t)tok_a * d + col + 8, gw_a * dacc[c][2]);
+          }
+          if (tok_b >= 0) {
+            atomicAdd(p.y_acc + (size_t)tok_b * d + col, gw_b * dacc[c][1]);
+            atomicAdd(p.y_acc + (size_t)tok_b * d + col + 8, gw_b * dacc[c][3]);
+          }
+        }
+      }
+      u += (b_end - b_begin);
+    }
+  }
+
+  // ---- the last CTA to finish rounds the accumulator to bf16 and clears it ----
+  if (!p.finalize) return;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const uint32_t prev = atomicAdd(p.done, 1u);
+    s_last = (prev == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const long long n4 = (long long)p.T * d / 4;
+  for (long long i = tid; i < n4; i += blockDim.x) {
+    const float4 v = __ldcg(reinterpret_cast<const float4 *>(p.y_acc) + i);
+    __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+    uint2 o;
+    o.x = *reinterpret_cast<uint32_t *>(&a);
+    o.y = *reinterpret_cast<uint32_t *>(&b);
+    reinterpret_cast<uint2 *>(p.y)[i] = o;
+    reinterpret_cast<float4 *>(p.y_acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  if (tid == 0) *p.done = 0u;
+}
+
+inline size_t ffn_mma_smem_bytes(int d) {
+  return (size_t)kMmaStages * kMmaTileRows * (2 * (size_t)d + 64) + 8 * 2 * 16 * 8 * 4 + 8 * 16 * 2 +
+         (kMaxExperts + 2) * 4 + 2 * kMmaStages * 8 + 16;
+}
+
+}  // namespace ftmoe

@@ -9,6 +9,7 @@
 #include <vector>
 
 #include "common.cuh"
+#include "ffn_mma.cuh"
 #include "ffn_stream.cuh"
 #include "fill.cuh"
 #include "plan.cuh"
@@ -54,6 +55,7 @@ struct ft_moe {
   WorkItem *items_res = nullptr, *items_zc = nullptr, *items_gemm = nullptr;
   uint32_t *status_dev = nullptr;
   uint32_t *seq_dev = nullptr;
+  uint32_t *done_dev = nullptr;          // CTA completion counter of the streaming MMA kernel
   uint32_t seq_host = 0;                // plans launched
   float *stage_logits = nullptr;
   __nv_bfloat16 *stage_x = nullptr, *stage_y = nullptr;
@@ -89,7 +91,7 @@ size_t expert_bytes_of(const ft_moe_config_t *c) {
   if (!c || c->hidden <= 0 || c->inter <= 0) return 0;
   const size_t d = (size_t)c->hidden, I = (size_t)c->inter;
   if (c->wdtype == FT_W_BF16) {
-    if (d % 256 || d > 2048 || I % 8) return 0;
+    if ((d != 256 && d != 512 && d != 1024 && d != 2048) || I % 16) return 0;
     return 3 * I * d * 2;
   }
   if (c->wdtype == FT_W_INT4_G128) {
@@ -270,6 +272,7 @@ ft_status_t ft_moe_destroy(ft_moe_t *h) {
   cudaFree(h->items_gemm);
   cudaFree(h->status_dev);
   cudaFree(h->seq_dev);
+  cudaFree(h->done_dev);
   cudaFree(h->stage_logits);
   cudaFree(h->stage_x);
   cudaFree(h->stage_y);
@@ -385,6 +388,15 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
   FT_TRY(cudaMemset(h->status_dev, 0, 4));
   FT_TRY(cudaMalloc(&h->seq_dev, 4));
   FT_TRY(cudaMemset(h->seq_dev, 0, 4));
+  FT_TRY(cudaMalloc(&h->done_dev, 4));
+  FT_TRY(cudaMemset(h->done_dev, 0, 4));
+  if (c.wdtype == FT_W_BF16) {
+    const int smem = (int)ffn_mma_smem_bytes(c.hidden);
+    FT_TRY(cudaFuncSetAttribute(ffn_mma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    FT_TRY(cudaFuncSetAttribute(ffn_mma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    FT_TRY(cudaFuncSetAttribute(ffn_mma_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    FT_TRY(cudaFuncSetAttribute(ffn_mma_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  }
   FT_TRY(cudaMalloc(&h->stage_logits, (size_t)c.max_tokens * E * 4));
   FT_TRY(cudaMalloc(&h->stage_x, (size_t)c.max_tokens * c.hidden * 2));
   FT_TRY(cudaMalloc(&h->stage_y, (size_t)c.max_tokens * c.hidden * 2));
@@ -595,6 +607,29 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   }
   // resident set after the fills have landed
   if (c.slots_per_layer > 0) FT_CUDA(cudaStreamWaitEvent(st, h->ev_fill, 0));
+  if (c.wdtype == FT_W_BF16) {
+    // resident experts: bulk-copy pipelined tensor-core streaming kernel; its last CTA finalizes y
+    FfnMmaParams mp;
+    mp.items = h->items_res;
+    mp.n_items = &h->plan_dev->n_res_items;
+    mp.x = fp.x; mp.perm = h->perm; mp.topk_w = h->topk_w; mp.y_acc = h->y_acc;
+    mp.y = static_cast<__nv_bfloat16 *>(y_dev);
+    mp.done = h->done_dev; mp.status = h->status_dev;
+    mp.d = c.hidden; mp.inter = c.inter; mp.top_k = c.top_k; mp.T = L.T; mp.finalize = 1;
+    const size_t smem = ffn_mma_smem_bytes(c.hidden);
+    {
+      TimeScope ts(h, st, FT_TIME_FFN_RES);
+      switch (c.hidden / 256) {
+        case 1: ffn_mma_kernel<1><<<h->sm_count, kMmaThreads, smem, st>>>(mp); break;
+        case 2: ffn_mma_kernel<2><<<h->sm_count, kMmaThreads, smem, st>>>(mp); break;
+        case 4: ffn_mma_kernel<4><<<h->sm_count, kMmaThreads, smem, st>>>(mp); break;
+        default: ffn_mma_kernel<8><<<h->sm_count, kMmaThreads, smem, st>>>(mp); break;
+      }
+    }
+    h->launches++;
+    FT_CUDA(cudaGetLastError());
+    return FT_OK;
+  }
   if (c.slots_per_layer > 0 || c.n_shared) {
     fp.items = h->items_res;
     fp.n_items = &h->plan_dev->n_res_items;
