@@ -26,6 +26,7 @@ constexpr int kMmaTokens = 8;  // tokens per weight pass
 struct FfnMmaParams {
   const WorkItem *items;
   const int32_t *n_items;
+  const int32_t *pref;      // [n_items+1] exclusive prefix of the weight passes per item (from the plan)
   const __nv_bfloat16 *x;   // [T][d]
   const int32_t *perm;
   const float *topk_w;
@@ -126,13 +127,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  // passes per item (8 tokens per pass) and their prefix sums
-  for (int i = tid; i < n_items; i += blockDim.x) s_pref[i + 1] = (p.items[i].n_tok + kMmaTokens - 1) / kMmaTokens;
-  __syncthreads();
-  if (tid == 0) {
-    s_pref[0] = 0;
-    for (int i = 0; i < n_items; ++i) s_pref[i + 1] += s_pref[i];
-  }
+  // prefix sums of the weight passes per item (8 tokens per pass), written by the plan kernel
+  for (int i = tid; i <= n_items; i += blockDim.x) s_pref[i] = p.pref[i];
   __syncthreads();
   const long long total = (long long)s_pref[n_items] * NBLK;
   long long u = total * blockIdx.x / gridDim.x;

@@ -12,8 +12,7 @@
 #include "ffn_mma.cuh"
 #include "ffn_stream.cuh"
 #include "fill.cuh"
-#include "plan.cuh"
-#include "route.cuh"
+#include "route_plan.cuh"
 
 using namespace ftmoe;
 
@@ -53,6 +52,8 @@ struct ft_moe {
   PlanHeader *plan_host_devptr = nullptr;
   size_t plan_bytes = 0;
   WorkItem *items_res = nullptr, *items_zc = nullptr, *items_gemm = nullptr;
+  int32_t *res_pref = nullptr;
+  bool plan_mirrored = false;
   uint32_t *status_dev = nullptr;
   uint32_t *seq_dev = nullptr;
   uint32_t *done_dev = nullptr;          // CTA completion counter of the streaming MMA kernel
@@ -270,6 +271,7 @@ ft_status_t ft_moe_destroy(ft_moe_t *h) {
   cudaFree(h->items_res);
   cudaFree(h->items_zc);
   cudaFree(h->items_gemm);
+  cudaFree(h->res_pref);
   cudaFree(h->status_dev);
   cudaFree(h->seq_dev);
   cudaFree(h->done_dev);
@@ -384,12 +386,19 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
   FT_TRY(cudaMalloc(&h->items_res, (E + 1) * sizeof(WorkItem)));
   FT_TRY(cudaMalloc(&h->items_zc, E * sizeof(WorkItem)));
   FT_TRY(cudaMalloc(&h->items_gemm, E * sizeof(WorkItem)));
+  FT_TRY(cudaMalloc(&h->res_pref, (E + 2) * 4));
+  FT_TRY(cudaMemset(h->res_pref, 0, (E + 2) * 4));
   FT_TRY(cudaMalloc(&h->status_dev, 4));
   FT_TRY(cudaMemset(h->status_dev, 0, 4));
   FT_TRY(cudaMalloc(&h->seq_dev, 4));
   FT_TRY(cudaMemset(h->seq_dev, 0, 4));
   FT_TRY(cudaMalloc(&h->done_dev, 4));
   FT_TRY(cudaMemset(h->done_dev, 0, 4));
+  if ((size_t)c.slots_per_layer * 16 + 36 * 1024 > 48 * 1024) {
+    const int dyn = c.slots_per_layer * 16;
+    FT_TRY(cudaFuncSetAttribute(plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn));
+    FT_TRY(cudaFuncSetAttribute(route_plan_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn));
+  }
   if (c.wdtype == FT_W_BF16) {
     const int smem = (int)ffn_mma_smem_bytes(c.hidden);
     FT_TRY(cudaFuncSetAttribute(ffn_mma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
@@ -432,6 +441,42 @@ ft_status_t ft_moe_reset(ft_moe_t *h, int layer) {
   return FT_OK;
 }
 
+static RouteParams make_route_params(ft_moe *h, const float *logits_dev, int T) {
+  RouteParams rp;
+  rp.logits = logits_dev;
+  rp.T = T; rp.E = h->cfg.n_experts; rp.k = h->cfg.top_k;
+  rp.ids = h->ids; rp.w = h->topk_w; rp.count = h->count; rp.offset = h->offset;
+  rp.perm = h->perm; rp.inv = h->inv; rp.status = h->status_dev;
+  return rp;
+}
+
+static PlanParams make_plan_params(ft_moe *h, int layer, bool mirror_to_host) {
+  const ft_moe_config_t &c = h->cfg;
+  LayerState &L = h->layers[layer];
+  PlanParams pp;
+  pp.count = h->count; pp.offset = h->offset;
+  pp.E = c.n_experts; pp.n_slots = c.slots_per_layer;
+  pp.cm.ns_fill = (int64_t)(h->S * 1000 / c.bw_fill_MBps);
+  pp.cm.ns_zc = (int64_t)(h->S * 1000 / c.bw_zc_MBps);
+  pp.cm.ns_hbm = (int64_t)(h->S * 1000 / c.bw_hbm_MBps);
+  pp.cm.bw_fill = c.bw_fill_MBps; pp.cm.bw_res = c.bw_zc_residual_MBps;
+  pp.cm.reuse_credit = c.reuse_credit; pp.cm.tz = c.zc_tokens_per_pass; pp.cm.tg = c.hbm_tokens_per_pass;
+  pp.cm.gemm_min_tokens = c.gemm_min_tokens;
+  pp.slot_expert = L.slot_expert; pp.slot_stamp = L.slot_stamp; pp.expert_slot = L.expert_slot;
+  pp.step = L.step; pp.stats = L.stats;
+  pp.pool_layer_dev = h->pool_dev + (size_t)layer * c.n_experts * h->S;
+  pp.slots_layer = h->slots ? h->slots + (size_t)layer * c.slots_per_layer * h->S : nullptr;
+  pp.shared_rec = c.n_shared ? h->shared_dev + (size_t)layer * h->S : nullptr;
+  pp.S = h->S; pp.T = L.T;
+  pp.tokens_per_pass = kMmaTokens;
+  pp.hdr_dev = h->plan_dev;
+  pp.hdr_host = mirror_to_host ? h->plan_host_devptr : nullptr;
+  pp.items_res = h->items_res; pp.res_pref = h->res_pref;
+  pp.items_zc = h->items_zc; pp.items_gemm = h->items_gemm;
+  pp.seq = h->seq_dev;
+  return pp;
+}
+
 ft_status_t ft_moe_route(ft_moe_t *h, int layer, const float *logits_dev, int T, void *stream) {
   if (!h || layer < 0 || layer >= h->cfg.n_layers || T < 0 || T > h->cfg.max_tokens) return FT_ERR_INVALID_ARG;
   if (T > 0 && !logits_dev) return FT_ERR_INVALID_ARG;
@@ -441,11 +486,7 @@ ft_status_t ft_moe_route(ft_moe_t *h, int layer, const float *logits_dev, int T,
   h->last_routed_layer = layer;
   if (T == 0) return FT_OK;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  RouteParams rp;
-  rp.logits = logits_dev;
-  rp.T = T; rp.E = h->cfg.n_experts; rp.k = h->cfg.top_k;
-  rp.ids = h->ids; rp.w = h->topk_w; rp.count = h->count; rp.offset = h->offset;
-  rp.perm = h->perm; rp.inv = h->inv; rp.status = h->status_dev;
+  const RouteParams rp = make_route_params(h, logits_dev, T);
   TimeScope ts(h, st, FT_TIME_ROUTE);
   if (T <= kRouteSmallMaxTokens) {
     route_small_kernel<<<1, 1024, 0, st>>>(rp);
@@ -467,31 +508,18 @@ ft_status_t ft_moe_plan(ft_moe_t *h, int layer, ft_moe_plan_t *out, void *stream
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const ft_moe_config_t &c = h->cfg;
   if (L.T > 0) {
-    PlanParams pp;
-    pp.count = h->count; pp.offset = h->offset;
-    pp.E = c.n_experts; pp.n_slots = c.slots_per_layer;
-    pp.cm.ns_fill = (int64_t)(h->S * 1000 / c.bw_fill_MBps);
-    pp.cm.ns_zc = (int64_t)(h->S * 1000 / c.bw_zc_MBps);
-    pp.cm.ns_hbm = (int64_t)(h->S * 1000 / c.bw_hbm_MBps);
-    pp.cm.bw_fill = c.bw_fill_MBps; pp.cm.bw_res = c.bw_zc_residual_MBps;
-    pp.cm.reuse_credit = c.reuse_credit; pp.cm.tz = c.zc_tokens_per_pass; pp.cm.tg = c.hbm_tokens_per_pass;
-    pp.cm.gemm_min_tokens = c.gemm_min_tokens;
-    pp.slot_expert = L.slot_expert; pp.slot_stamp = L.slot_stamp; pp.expert_slot = L.expert_slot;
-    pp.step = L.step; pp.stats = L.stats;
-    pp.pool_layer_dev = h->pool_dev + (size_t)layer * c.n_experts * h->S;
-    pp.slots_layer = h->slots ? h->slots + (size_t)layer * c.slots_per_layer * h->S : nullptr;
-    pp.shared_rec = c.n_shared ? h->shared_dev + (size_t)layer * h->S : nullptr;
-    pp.S = h->S; pp.T = L.T;
-    pp.hdr_dev = h->plan_dev; pp.hdr_host = h->plan_host_devptr;
-    pp.items_res = h->items_res; pp.items_zc = h->items_zc; pp.items_gemm = h->items_gemm;
-    pp.seq = h->seq_dev;
+    const bool mirror = (out != nullptr) || c.fill_mode == FT_FILL_COPY_ENGINE;
+    const PlanParams pp = make_plan_params(h, layer, mirror);
     const size_t smem = (size_t)c.slots_per_layer * 16;
+    int threads = ((c.n_experts + 31) / 32) * 32;
+    if (threads < 128) threads = 128;
     {
       TimeScope ts(h, st, FT_TIME_PLAN);
-      plan_kernel<<<1, 1024, smem, st>>>(pp);
+      plan_kernel<<<1, threads, smem, st>>>(pp);
     }
     h->launches++;
     h->seq_host++;
+    h->plan_mirrored = mirror;
     FT_CUDA(cudaGetLastError());
     FT_CUDA(cudaEventRecord(h->ev_plan, st));
   }
@@ -612,6 +640,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     FfnMmaParams mp;
     mp.items = h->items_res;
     mp.n_items = &h->plan_dev->n_res_items;
+    mp.pref = h->res_pref;
     mp.x = fp.x; mp.perm = h->perm; mp.topk_w = h->topk_w; mp.y_acc = h->y_acc;
     mp.y = static_cast<__nv_bfloat16 *>(y_dev);
     mp.done = h->done_dev; mp.status = h->status_dev;
@@ -648,10 +677,34 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
 
 ft_status_t ft_moe_layer(ft_moe_t *h, int layer, const float *logits_dev, const void *x_dev, void *y_dev,
                          int T, void *stream) {
-  ft_status_t rc = ft_moe_route(h, layer, logits_dev, T, stream);
-  if (rc != FT_OK) return rc;
-  rc = ft_moe_plan(h, layer, nullptr, stream);
-  if (rc != FT_OK) return rc;
+  ft_status_t rc;
+  if (h && layer >= 0 && layer < h->cfg.n_layers && T > 0 && T <= kRouteSmallMaxTokens && T <= h->cfg.max_tokens &&
+      logits_dev) {
+    // decode-sized call: route, permute and plan in one single-CTA launch
+    LayerState &L = h->layers[layer];
+    const ft_moe_config_t &c = h->cfg;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    L.T = T;
+    h->last_routed_layer = layer;
+    const bool mirror = c.fill_mode == FT_FILL_COPY_ENGINE;
+    const RouteParams rp = make_route_params(h, logits_dev, T);
+    const PlanParams pp = make_plan_params(h, layer, mirror);
+    {
+      TimeScope ts(h, st, FT_TIME_PLAN);
+      route_plan_small_kernel<<<1, 1024, (size_t)c.slots_per_layer * 16, st>>>(rp, pp);
+    }
+    h->launches++;
+    h->seq_host++;
+    h->plan_mirrored = mirror;
+    FT_CUDA(cudaGetLastError());
+    FT_CUDA(cudaEventRecord(h->ev_plan, st));
+    L.phase = PH_PLANNED;
+  } else {
+    rc = ft_moe_route(h, layer, logits_dev, T, stream);
+    if (rc != FT_OK) return rc;
+    rc = ft_moe_plan(h, layer, nullptr, stream);
+    if (rc != FT_OK) return rc;
+  }
   rc = ft_moe_fill(h, layer, h->copy_stream);
   if (rc != FT_OK) return rc;
   return ft_moe_forward(h, layer, x_dev, y_dev, stream);
@@ -747,7 +800,11 @@ ft_status_t ft_moe_last_fill(ft_moe_t *h, float *out_us, uint64_t *out_bytes) {
   FT_CUDA(cudaEventElapsedTime(&ms, h->ev_fill_t0, h->ev_fill_t1));
   if (out_us) *out_us = ms * 1000.f;
   uint64_t bytes = h->last_fill_bytes;
-  if (bytes == ~0ull) bytes = (uint64_t)h->plan_host->n_fill * h->S;
+  if (bytes == ~0ull) {
+    PlanHeader hd;
+    FT_CUDA(cudaMemcpy(&hd, h->plan_dev, sizeof(hd), cudaMemcpyDeviceToHost));
+    bytes = (uint64_t)hd.n_fill * h->S;
+  }
   if (out_bytes) *out_bytes = bytes;
   return FT_OK;
 }

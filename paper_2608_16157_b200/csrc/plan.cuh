@@ -27,34 +27,36 @@ struct PlanParams {
   const uint8_t *shared_rec;      // shared-expert record of this layer or nullptr
   size_t S;
   int T;
+  int tokens_per_pass;   // tokens one weight pass of the resident streaming kernel serves
   // outputs
   PlanHeader *hdr_dev;   // device plan record (header + 8 arrays of E)
-  PlanHeader *hdr_host;  // mapped host mirror
+  PlanHeader *hdr_host;  // mapped host mirror, or nullptr when the host does not read the plan
   WorkItem *items_res;   // [E+1]  experts evaluated from slots by the streaming kernel
+  int32_t *res_pref;     // [E+2]  exclusive prefix of the weight passes of items_res
   WorkItem *items_zc;    // [E]    experts evaluated from the mapped host pool
   WorkItem *items_gemm;  // [E]    experts evaluated from slots by the grouped GEMM
   uint32_t *seq;         // [1] plan sequence number
 };
 
-// Block-wide exclusive scan of one int per thread (blockDim = 1024); returns the exclusive prefix and
-// the total through `total`.
-__device__ __forceinline__ int block_excl_scan(int v, int *s_w /*[33]*/, int &total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int incl = v;
+// Block-wide exclusive scan of one 64-bit value per thread (several small counters packed into it).
+__device__ __forceinline__ unsigned long long block_excl_scan64(unsigned long long v, unsigned long long *s_w /*[33]*/,
+                                                                unsigned long long &total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = (blockDim.x + 31) >> 5;
+  unsigned long long incl = v;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
-    const int n = __shfl_up_sync(0xffffffffu, incl, o);
+    const unsigned long long n = __shfl_up_sync(0xffffffffu, incl, o);
     if (lane >= o) incl += n;
   }
   __syncthreads();  // protects s_w against the previous use
   if (lane == 31) s_w[warp] = incl;
   __syncthreads();
   if (warp == 0) {
-    const int ws = s_w[lane];
-    int wincl = ws;
+    const unsigned long long ws = (lane < nwarps) ? s_w[lane] : 0ull;
+    unsigned long long wincl = ws;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const int n = __shfl_up_sync(0xffffffffu, wincl, o);
+      const unsigned long long n = __shfl_up_sync(0xffffffffu, wincl, o);
       if (lane >= o) wincl += n;
     }
     s_w[lane] = wincl - ws;
@@ -65,47 +67,65 @@ __device__ __forceinline__ int block_excl_scan(int v, int *s_w /*[33]*/, int &to
   return incl - v + s_w[warp];
 }
 
-// Dynamic shared memory: int64 stamp[n_slots]; int32 sexp[n_slots]; int32 victim[n_slots].
-__global__ void __launch_bounds__(1024) plan_kernel(PlanParams p) {
-  extern __shared__ __align__(16) unsigned char s_raw[];
-  int64_t *s_stamp = reinterpret_cast<int64_t *>(s_raw);
+constexpr int kPlanField = 11;  // bits per packed counter (values <= 1024)
+__device__ __forceinline__ unsigned long long pack4(int a, int b, int c, int d) {
+  return (unsigned long long)a | ((unsigned long long)b << kPlanField) | ((unsigned long long)c << (2 * kPlanField)) |
+         ((unsigned long long)d << (3 * kPlanField));
+}
+__device__ __forceinline__ int unpack(unsigned long long v, int i) {
+  return (int)((v >> (i * kPlanField)) & ((1u << kPlanField) - 1u));
+}
+
+// Shared memory the plan needs besides the dynamic part (stamp/expert/victim per slot).
+struct PlanSmem {
+  unsigned long long w[33];
+  int32_t cnt[kMaxExperts];
+  uint8_t elig[kMaxExperts];
+  int32_t forder[kMaxExperts];
+  int K;
+};
+
+// One plan step.  Thread `tid` < E owns expert `tid`: `c` = its token count, `off` = its offset in the
+// expert-sorted pair order, `n_pairs` = all pairs of the call.  blockDim.x >= E, a multiple of 32.
+// s_dyn: int64 stamp[n_slots]; int32 sexp[n_slots]; int32 victim[n_slots].
+__device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, unsigned char *s_dyn, int c, int off,
+                                          int n_pairs) {
+  int64_t *s_stamp = reinterpret_cast<int64_t *>(s_dyn);
   int32_t *s_sexp = reinterpret_cast<int32_t *>(s_stamp + p.n_slots);
   int32_t *s_victim = s_sexp + p.n_slots;
-  __shared__ int s_w[33];
-  __shared__ int32_t s_cnt[kMaxExperts];
-  __shared__ uint8_t s_elig[kMaxExperts];
-  __shared__ int32_t s_forder[kMaxExperts];
-  __shared__ int s_K;
-
   const int tid = threadIdx.x;
   const int E = p.E;
-  if (p.offset[E] == 0) return;  // nothing routed: the step does not advance
+  if (n_pairs == 0) return;  // nothing routed: the step does not advance
   const int64_t t = *p.step;
 
   int32_t *a_hit = reinterpret_cast<int32_t *>(p.hdr_dev + 1);
   int32_t *a_miss = a_hit + E, *a_fill = a_miss + E, *a_zc = a_fill + E, *a_forder = a_zc + E;
   int32_t *a_fslot = a_forder + E, *a_fevict = a_fslot + E, *a_loc = a_fevict + E;
 
-  // ---- 1/2: classify, refresh recency of hits
-  int c = 0, slot = -1, cls = 0;
+  // ---- 1/2: classify, refresh recency of hits; 4: which misses are worth a fill
+  int slot = -1, cls = 0, elig = 0;
   if (tid < E) {
-    c = p.count[tid];
     slot = p.expert_slot[tid];
     cls = (c > 0) ? (slot >= 0 ? 1 : 2) : 0;
     if (cls == 1) p.slot_stamp[slot] = t;
-    s_cnt[tid] = c;
+    if (cls == 2) {
+      const int64_t pz = (c + p.cm.tz - 1) / p.cm.tz, pg = (c + p.cm.tg - 1) / p.cm.tg;
+      const int64_t v = pz * p.cm.ns_zc - (p.cm.ns_fill + pg * p.cm.ns_hbm) +
+                        (int64_t)p.cm.reuse_credit * (p.cm.ns_zc - p.cm.ns_hbm);
+      elig = v > 0;
+    }
+    sm.cnt[tid] = c;
+    sm.elig[tid] = (uint8_t)elig;
   }
-  if (tid == 0) s_K = 0;
-  __syncthreads();  // stamps of hits are visible to this block (global writes + barrier)
-
-  int n_routed, n_hit, n_miss;
-  block_excl_scan(cls != 0, s_w, n_routed);
-  const int hpos = block_excl_scan(cls == 1, s_w, n_hit);
-  if (cls == 1) a_hit[hpos] = tid;
-  const int mpos = block_excl_scan(cls == 2, s_w, n_miss);
-  if (cls == 2) a_miss[mpos] = tid;
+  if (tid == 0) sm.K = 0;
+  unsigned long long totA;
+  const unsigned long long exA = block_excl_scan64(pack4(cls != 0, cls == 1, cls == 2, elig), sm.w, totA);
+  const int n_routed = unpack(totA, 0), n_hit = unpack(totA, 1), n_miss = unpack(totA, 2), n_elig = unpack(totA, 3);
+  if (cls == 1) a_hit[unpack(exA, 1)] = tid;
+  if (cls == 2) a_miss[unpack(exA, 2)] = tid;
 
   // ---- 3: victim candidates, ordered in one pass by counting how many candidates precede each
+  // (the scan's barriers make the refreshed stamps visible to the whole block)
   for (int s = tid; s < p.n_slots; s += blockDim.x) {
     s_stamp[s] = p.slot_stamp[s];
     s_sexp[s] = p.slot_expert[s];
@@ -128,22 +148,10 @@ __global__ void __launch_bounds__(1024) plan_kernel(PlanParams p) {
       rank += before ? 1 : 0;
     }
     s_victim[rank] = s;
-    atomicAdd(&s_K, 1);  // a count
+    atomicAdd(&sm.K, 1);  // a count
   }
   __syncthreads();
-  const int K = s_K;
-
-  // ---- 4: which misses are worth a fill
-  int elig = 0;
-  if (cls == 2) {
-    const int64_t pz = (c + p.cm.tz - 1) / p.cm.tz, pg = (c + p.cm.tg - 1) / p.cm.tg;
-    const int64_t v = pz * p.cm.ns_zc - (p.cm.ns_fill + pg * p.cm.ns_hbm) +
-                      (int64_t)p.cm.reuse_credit * (p.cm.ns_zc - p.cm.ns_hbm);
-    elig = v > 0;
-  }
-  if (tid < E) s_elig[tid] = (uint8_t)elig;
-  int n_elig;
-  block_excl_scan(elig, s_w, n_elig);  // (also orders the s_elig writes before the reads below)
+  const int K = sm.K;
 
   // ---- 5: fill count
   int q = 0;
@@ -161,17 +169,19 @@ __global__ void __launch_bounds__(1024) plan_kernel(PlanParams p) {
   if (elig) {
     int rank = 0;
     for (int o = 0; o < E; ++o) {
-      if (!s_elig[o] || o == tid) continue;
-      const int oc = s_cnt[o];
+      if (!sm.elig[o] || o == tid) continue;
+      const int oc = sm.cnt[o];
       rank += (oc > c || (oc == c && o < tid)) ? 1 : 0;
     }
-    if (rank < q) { is_fill = 1; s_forder[rank] = tid; }
+    if (rank < q) { is_fill = 1; sm.forder[rank] = tid; }
   }
   __syncthreads();
 
   // ---- 7: the i-th fill takes the i-th candidate slot
+  int loc = kLocNotRouted;
+  if (cls == 1) loc = slot;
   if (tid < q) {
-    const int e = s_forder[tid];
+    const int e = sm.forder[tid];
     const int s = s_victim[tid];
     const int old = s_sexp[s];
     if (old >= 0) p.expert_slot[old] = -1;
@@ -181,51 +191,54 @@ __global__ void __launch_bounds__(1024) plan_kernel(PlanParams p) {
     a_forder[tid] = e;
     a_fslot[tid] = s;
     a_fevict[tid] = old;
+    sm.cnt[e] = -1 - s;   // hands the slot to the thread that owns expert e (negative marks "filled")
   }
   __syncthreads();
+  if (is_fill) loc = -1 - sm.cnt[tid];
 
   // ---- 8: lists and locations
-  int n_fill, n_zc;
-  const int fpos = block_excl_scan(is_fill, s_w, n_fill);
-  if (is_fill) a_fill[fpos] = tid;
   const int is_zc = (cls == 2 && !is_fill);
-  const int zpos = block_excl_scan(is_zc, s_w, n_zc);
-  if (is_zc) a_zc[zpos] = tid;
-  int loc = kLocNotRouted;
-  if (cls == 1) loc = slot;
-  else if (is_fill) loc = p.expert_slot[tid];  // written in step 7 by this block, barrier above
-  else if (is_zc) loc = kLocZeroCopy;
-  if (tid < E) a_loc[tid] = loc;
-
-  // work lists for the execution step
+  if (is_zc) loc = kLocZeroCopy;
   const int resident = (cls == 1 || is_fill);
   const int use_gemm = resident && p.cm.gemm_min_tokens > 0 && c >= p.cm.gemm_min_tokens;
-  int n_res, n_gemm;
-  const int rpos = block_excl_scan(resident && !use_gemm, s_w, n_res);
-  const int gpos = block_excl_scan(use_gemm, s_w, n_gemm);
+  const int res_stream = resident && !use_gemm;
+  unsigned long long totB;
+  const unsigned long long exB = block_excl_scan64(pack4(is_fill, is_zc, res_stream, use_gemm), sm.w, totB);
+  const int n_fill = unpack(totB, 0), n_zc = unpack(totB, 1), n_res = unpack(totB, 2), n_gemm = unpack(totB, 3);
+  const int passes = res_stream ? (c + p.tokens_per_pass - 1) / p.tokens_per_pass : 0;
+  unsigned long long totC;
+  const unsigned long long exC =
+      block_excl_scan64(((unsigned long long)(resident ? c : 0) << 32) | (unsigned long long)passes, sm.w, totC);
+  if (is_fill) a_fill[unpack(exB, 0)] = tid;
+  if (is_zc) a_zc[unpack(exB, 1)] = tid;
+  if (tid < E) a_loc[tid] = loc;
   if (resident) {
     WorkItem it;
     it.w = p.slots_layer + (size_t)loc * p.S;
     it.expert = tid;
     it.n_tok = c;
-    it.off = p.offset[tid];
+    it.off = off;
     it.slot = loc;
-    if (use_gemm) p.items_gemm[gpos] = it; else p.items_res[rpos] = it;
+    if (use_gemm) {
+      p.items_gemm[unpack(exB, 3)] = it;
+    } else {
+      p.items_res[unpack(exB, 2)] = it;
+      p.res_pref[unpack(exB, 2)] = (int32_t)(exC & 0xffffffffull);
+    }
   }
   if (is_zc) {
     WorkItem it;
     it.w = p.pool_layer_dev + (size_t)tid * p.S;
     it.expert = tid;
     it.n_tok = c;
-    it.off = p.offset[tid];
+    it.off = off;
     it.slot = -1;
-    p.items_zc[zpos] = it;
+    p.items_zc[unpack(exB, 1)] = it;
   }
-  int pairs_res;
-  block_excl_scan(resident ? c : 0, s_w, pairs_res);
 
   if (tid == 0) {
     int n_res_items = n_res;
+    int pass_total = (int)(totC & 0xffffffffull);
     if (p.shared_rec != nullptr) {
       WorkItem it;
       it.w = p.shared_rec;
@@ -233,8 +246,12 @@ __global__ void __launch_bounds__(1024) plan_kernel(PlanParams p) {
       it.n_tok = p.T;
       it.off = 0;
       it.slot = -1;
-      p.items_res[n_res_items++] = it;
+      p.items_res[n_res_items] = it;
+      p.res_pref[n_res_items] = pass_total;
+      pass_total += (p.T + p.tokens_per_pass - 1) / p.tokens_per_pass;
+      ++n_res_items;
     }
+    p.res_pref[n_res_items] = pass_total;
     PlanHeader h;
     h.step = t;
     h.n_routed = n_routed; h.n_hit = n_hit; h.n_miss = n_miss; h.n_fill = n_fill; h.n_zc = n_zc;
@@ -245,7 +262,7 @@ __global__ void __launch_bounds__(1024) plan_kernel(PlanParams p) {
     *p.seq = h.seq;
     *p.step = t + 1;
     int evictions = 0;
-    for (int i = 0; i < n_fill; ++i) evictions += (a_fevict[i] >= 0);
+    for (int i = 0; i < n_fill; ++i) evictions += (s_sexp[s_victim[i]] >= 0);
     p.stats[0] += 1;
     p.stats[1] += n_routed;
     p.stats[2] += n_hit;
@@ -253,22 +270,28 @@ __global__ void __launch_bounds__(1024) plan_kernel(PlanParams p) {
     p.stats[4] += n_fill;
     p.stats[5] += n_zc;
     p.stats[6] += evictions;
-    p.stats[7] += p.offset[E];
-    p.stats[8] += pairs_res;
+    p.stats[7] += n_pairs;
+    p.stats[8] += (unsigned long long)(totC >> 32);
   }
-  __syncthreads();
-  // mirror the record into mapped host memory for the copy-engine fill path and for reports
+  // mirror the record into mapped host memory when the host reads the plan (copy-engine fills)
   if (p.hdr_host != nullptr) {
+    __syncthreads();
     const int n_words = (int)(sizeof(PlanHeader) / 4) + 8 * E;
     const uint32_t *src = reinterpret_cast<const uint32_t *>(p.hdr_dev);
     volatile uint32_t *dst = reinterpret_cast<volatile uint32_t *>(p.hdr_host);
-    // arrays first, header (with the sequence number) last
-    for (int i = (int)(sizeof(PlanHeader) / 4) + tid; i < n_words; i += blockDim.x) dst[i] = src[i];
-    __threadfence_system();
-    __syncthreads();
-    if (tid < (int)(sizeof(PlanHeader) / 4)) dst[tid] = src[tid];
-    __threadfence_system();
+    for (int i = tid; i < n_words; i += blockDim.x) dst[i] = src[i];
   }
+}
+
+// Stand-alone plan kernel: blockDim.x = E rounded up to a warp multiple (at least 128).
+__global__ void __launch_bounds__(1024) plan_kernel(PlanParams p) {
+  extern __shared__ __align__(16) unsigned char s_dyn[];
+  __shared__ PlanSmem sm;
+  const int tid = threadIdx.x;
+  const int n_pairs = p.offset[p.E];
+  int c = 0, off = 0;
+  if (tid < p.E) { c = p.count[tid]; off = p.offset[tid]; }
+  plan_body(p, sm, s_dyn, c, off, n_pairs);
 }
 
 }  // namespace ftmoe

@@ -86,15 +86,20 @@ __device__ __forceinline__ void route_token_any(const RouteParams &p, int t, int
   else route_token_dispatch<32>(p, t, lane, id, w);
 }
 
-// Decode-sized calls: one CTA (1024 threads) routes all tokens, counts, scans and permutes.
-__global__ void __launch_bounds__(1024) route_small_kernel(RouteParams p) {
-  __shared__ int32_t s_cnt[kMaxExperts];
-  __shared__ int32_t s_off[kMaxExperts + 1];
-  __shared__ int16_t s_key[kRouteSmallMaxTokens * kMaxTopK];
-  __shared__ int32_t s_wsum[32];
+// Shared memory of the single-CTA route + permute.
+struct RouteSmem {
+  int32_t cnt[kMaxExperts];
+  int32_t off[kMaxExperts + 1];
+  int16_t key[kRouteSmallMaxTokens * kMaxTopK];
+  int32_t wsum[32];
+};
+
+// Decode-sized calls: one CTA (1024 threads) routes all tokens, counts, scans and permutes.  On
+// return (after a barrier) s.cnt / s.off hold count[] and offset[] for the caller.
+__device__ __forceinline__ void route_small_body(const RouteParams &p, RouteSmem &s) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int P = p.T * p.k;
-  for (int e = tid; e < p.E; e += blockDim.x) s_cnt[e] = 0;
+  for (int e = tid; e < p.E; e += blockDim.x) s.cnt[e] = 0;
   __syncthreads();
   for (int t = warp; t < p.T; t += 32) {
     int id;
@@ -103,49 +108,49 @@ __global__ void __launch_bounds__(1024) route_small_kernel(RouteParams p) {
     if (lane < p.k) {
       p.ids[t * p.k + lane] = id;
       p.w[t * p.k + lane] = w;
-      s_key[t * p.k + lane] = (int16_t)id;
-      atomicAdd(&s_cnt[id], 1);  // a count: the result does not depend on the order of the adds
+      s.key[t * p.k + lane] = (int16_t)id;
+      atomicAdd(&s.cnt[id], 1);  // a count: the result does not depend on the order of the adds
     }
   }
   __syncthreads();
   // exclusive scan of the counts (one expert per thread)
   {
-    const int c = (tid < p.E) ? s_cnt[tid] : 0;
+    const int c = (tid < p.E) ? s.cnt[tid] : 0;
     int incl = c;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const int n = __shfl_up_sync(0xffffffffu, incl, o);
       if (lane >= o) incl += n;
     }
-    if (lane == 31) s_wsum[warp] = incl;
+    if (lane == 31) s.wsum[warp] = incl;
     __syncthreads();
     if (warp == 0) {
-      int ws = s_wsum[lane];
+      int ws = s.wsum[lane];
       int wincl = ws;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
         const int n = __shfl_up_sync(0xffffffffu, wincl, o);
         if (lane >= o) wincl += n;
       }
-      s_wsum[lane] = wincl - ws;
+      s.wsum[lane] = wincl - ws;
     }
     __syncthreads();
-    const int excl = incl - c + s_wsum[warp];
+    const int excl = incl - c + s.wsum[warp];
     if (tid < p.E) {
-      s_off[tid] = excl;
+      s.off[tid] = excl;
       p.count[tid] = c;
       p.offset[tid] = excl;
-      if (tid == p.E - 1) { s_off[p.E] = excl + c; p.offset[p.E] = excl + c; }
+      if (tid == p.E - 1) { s.off[p.E] = excl + c; p.offset[p.E] = excl + c; }
     }
   }
   __syncthreads();
   // one warp per expert walks the pairs in index order: rank = number of earlier pairs with this key
   for (int e = warp; e < p.E; e += 32) {
-    if (s_cnt[e] == 0) continue;
-    int run = s_off[e];
+    if (s.cnt[e] == 0) continue;
+    int run = s.off[e];
     for (int base = 0; base < P; base += 32) {
       const int q = base + lane;
-      const bool mine = (q < P) && (s_key[q] == e);
+      const bool mine = (q < P) && (s.key[q] == e);
       const unsigned m = __ballot_sync(0xffffffffu, mine);
       if (mine) {
         const int pos = run + __popc(m & ((1u << lane) - 1u));
@@ -155,6 +160,11 @@ __global__ void __launch_bounds__(1024) route_small_kernel(RouteParams p) {
       run += __popc(m);
     }
   }
+}
+
+__global__ void __launch_bounds__(1024) route_small_kernel(RouteParams p) {
+  __shared__ RouteSmem s;
+  route_small_body(p, s);
 }
 
 // Prefill-sized calls, kernel 1: one warp per token; counts by integer atomics (order-free result).
