@@ -202,6 +202,43 @@ ft_status_t ft_moe_timing_read(ft_moe_t *h, double *out_us, uint64_t *out_launch
 ft_status_t ft_moe_launch_count(ft_moe_t *h, uint64_t *out);
 const char *ft_moe_status_string(ft_status_t s);
 
+/* An expert FFN for callers that are not allowed to allocate.  (The paper has no counterpart: this
+ * is a convenience of this library.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a serving loop with a frozen memory
+ * budget, a plug-in inside a process whose device memory pool belongs to the host application, a
+ * component started after the application has already claimed all of HBM.  Such a caller cannot
+ * create an ft_moe_t handle (ft_moe_create allocates slots, tables and scratch), but it can still
+ * evaluate one expert on weights it already holds in device memory.
+ *
+ * What it does: y[t] = (SiLU(x[t] W_gate) * (x[t] W_up)) W_down for t < T, with the same streaming
+ * tensor-core kernel ft_moe_forward uses for resident bf16 experts.
+ *   record_dev : DEVICE, one FT_W_BF16 expert record (layout above), 16-byte aligned, caller-owned
+ *   x_dev      : DEVICE bf16 [T][hidden], caller-owned, read only
+ *   y_dev      : DEVICE bf16 [T][hidden], caller-owned, written
+ *   stream     : cudaStream_t; the call only enqueues work
+ * The kernel's scratch (an fp32 [T][hidden] accumulator and a few control words) lives in a fixed
+ * array of FT_NOALLOC_MAX_TOKENS * FT_NOALLOC_MAX_HIDDEN * 4 + 256 bytes (512.25 KiB) in the library's
+ * device data segment; every GPU that loads the library holds it until the process exits.  The
+ * call makes no cudaMalloc / cudaFree and uses no allocating library routine.
+ *
+ * Limits and errors: T in [1, FT_NOALLOC_MAX_TOKENS] and hidden <= FT_NOALLOC_MAX_HIDDEN, otherwise
+ * FT_ERR_INVALID_ARG (the scratch cannot be grown); hidden in {256, 512, 1024, 2048} and
+ * inter % 16 == 0, otherwise FT_ERR_UNSUPPORTED; null pointers FT_ERR_INVALID_ARG.
+ *
+ * First call on a device: looks up the device address of the scratch array and raises the kernel's
+ * shared-memory limit for that device (no allocation, but not stream work either), so make the
+ * first call on each device before any stream capture begins.
+ *
+ * Sharing: all calls on a device use the same array, which keeps whatever the last call left; each
+ * call clears the part it needs on its own stream before use.  Two calls that can overlap on the GPU
+ * (different streams without an ordering between them, or several host threads) race on the array
+ * and give wrong results: order them. */
+#define FT_NOALLOC_MAX_TOKENS 64
+#define FT_NOALLOC_MAX_HIDDEN 2048
+ft_status_t ft_moe_ffn_noalloc(int device, const void *record_dev, int hidden, int inter,
+                               const void *x_dev, void *y_dev, int T, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -25,8 +25,9 @@ SYMBOLS = (
     "ft_moe_calibrate", "ft_moe_route", "ft_moe_plan", "ft_moe_fill", "ft_moe_forward", "ft_moe_layer",
     "ft_moe_layer_host", "ft_moe_get_routing", "ft_moe_get_slot_table", "ft_moe_read_slot",
     "ft_moe_get_stats", "ft_moe_reset", "ft_moe_sync_status", "ft_moe_last_fill", "ft_moe_launch_count",
-    "ft_moe_status_string", "ft_moe_timing_enable", "ft_moe_timing_read",
+    "ft_moe_status_string", "ft_moe_timing_enable", "ft_moe_timing_read", "ft_moe_ffn_noalloc",
 )
+NOALLOC_MAX_TOKENS, NOALLOC_MAX_HIDDEN = 64, 2048
 TIME_NAMES = ("route", "plan", "ffn_zc", "ffn_res", "finalize", "fill")
 
 
@@ -96,6 +97,7 @@ def load(rebuild: bool = False):
         "ft_moe_status_string": (C.c_char_p, [i32]),
         "ft_moe_timing_enable": (i32, [vp, i32]),
         "ft_moe_timing_read": (i32, [vp, vp, vp, i32]),
+        "ft_moe_ffn_noalloc": (i32, [i32, vp, i32, i32, vp, vp, i32, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -133,6 +135,13 @@ def make_config(*, hidden, inter, n_experts, top_k, n_layers=1, slots_per_layer,
 
 def ft_moe_expert_bytes(cfg: Config) -> int:
     return int(load().ft_moe_expert_bytes(C.byref(cfg)))
+
+
+def ft_moe_ffn_noalloc(device, record_dev, hidden, inter, x_dev, y_dev, T, stream=None) -> int:
+    """One expert FFN on caller-held device memory without any allocation (scratch is a fixed array
+    inside the library).  Returns the status code; see ``include/ftmoe.h`` for the limits."""
+    return int(load().ft_moe_ffn_noalloc(device, _ptr(record_dev), hidden, inter, _ptr(x_dev), _ptr(y_dev), T,
+                                         _stream(stream)))
 
 
 class HostPool:
