@@ -395,8 +395,101 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_prefill(args):
+    """Prefill configuration: one step of `--tokens` tokens through all layers, cold cache then warm."""
+    import torch
+    from paper_2608_16157_b200 import binding as Bd
+    from paper_2608_16157_b200 import workload as W
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    shape = W.QWEN3_30B
+    L, E, k, d, I = args.layers, shape.n_experts, shape.top_k, shape.d, shape.inter
+    S = shape.expert_bytes
+    Ns = W.slots_for_fraction(args.cache_frac, E)
+    T = args.tokens
+    pool = Bd.HostPool(L * E * S)
+    W.fill_pool(pool.tensor, shape, L, SEED, device=dev, chunk=32)
+    common = dict(hidden=d, inter=I, n_experts=E, top_k=k, n_layers=L, slots_per_layer=Ns, max_tokens=T,
+                  host_pool_ptr=pool.ptr.value, host_pool_bytes=pool.n_bytes,
+                  fill_mode=Bd.FT_FILL_SM if args.fill == "sm" else Bd.FT_FILL_COPY_ENGINE,
+                  gemm_min_tokens=args.gemm_min_tokens)
+    moe = Bd.FtMoe(Bd.make_config(**common))
+    cal = moe.calibrate()
+    moe.destroy()
+    moe = Bd.FtMoe(Bd.make_config(bw_fill=max(cal["fill_MBps"], 1), bw_zc=max(cal["zc_MBps"], 1), bw_zc_residual=0,
+                                  bw_hbm=max(cal["hbm_MBps"], 1), **common))
+    stream = torch.cuda.current_stream()
+    xbuf = torch.empty((L, T, d), dtype=torch.bfloat16, device=dev)
+    ybuf = torch.empty((L, T, d), dtype=torch.bfloat16, device=dev)
+    out = {}
+    peak_hbm, peak_kind = peaks()
+    pk = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    tf_burst, tf_sust = FALLBACK_BF16_TFLOPS, 1400.0
+    if os.path.exists(pk):
+        dd = json.load(open(pk))
+        tf_burst, tf_sust = float(dd["bf16_tflops"]), float(dd["bf16_tflops_sustained"])
+    for name, step in (("cold", 0), ("warm", 1)):
+        lg = torch.from_numpy(W.prefill_logits(L, T, E, ALPHA, SEED, step)).to(dev)
+        g = torch.Generator(device=dev)
+        g.manual_seed(W.mix64(SEED, 78, step))
+        noise = torch.randn((L, T, d), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        st0 = {kk: sum(moe.get_stats(l)[kk] for l in range(L)) for kk in Bd.STAT_NAMES}
+        moe.timing_enable(True)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0 = moe.launch_count()
+        e0.record(stream)
+        for l in range(L):
+            if l == 0:
+                x = noise[0]
+            else:
+                x = xbuf[l]
+                torch.add(noise[l], ybuf[l - 1], out=x)
+            moe.layer(l, lg[l], x, ybuf[l], T, stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        tim = moe.timing_read()
+        moe.timing_enable(False)
+        st1 = {kk: sum(moe.get_stats(l)[kk] for l in range(L)) for kk in Bd.STAT_NAMES}
+        dst = {kk: st1[kk] - st0[kk] for kk in st1}
+        flops = 2.0 * 3 * d * I * dst["pairs_gemm"]
+        gemm_us = tim["gemm1"][0] + tim["gemm2"][0]
+        fill_us = tim["fill"][0]
+        out[name] = {"ms": ms, "tok_per_s": T / (ms * 1e-3), "launches": moe.launch_count() - l0 + L - 1,
+                     "fills": dst["fills"], "zero_copy": dst["zc"], "hits": dst["hits"],
+                     "pairs": dst["pairs"], "pairs_gemm": dst["pairs_gemm"],
+                     "gemm_tflops": flops / (gemm_us * 1e-6) / 1e12 if gemm_us > 0 else None,
+                     "gemm1_tflops": (flops * 2 / 3) / (tim["gemm1"][0] * 1e-6) / 1e12 if tim["gemm1"][0] > 0 else None,
+                     "gemm2_tflops": (flops / 3) / (tim["gemm2"][0] * 1e-6) / 1e12 if tim["gemm2"][0] > 0 else None,
+                     "fill_GBps": dst["fills"] * S / (fill_us * 1e-6) / 1e9 if fill_us > 0 else None,
+                     "kernel_ms": {kk: v[0] / 1e3 for kk, v in tim.items()}}
+        log(f"prefill {name}: {out[name]}")
+    w = out["warm"]
+    line = {"metric": "moe_prefill_tok_per_s", "value": out["cold"]["tok_per_s"], "unit": "tok/s", "n_gpus": 1,
+            "steps": 1, "warmup": 0, "ms_per_step": out["cold"]["ms"], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "prefill Qwen3-30B-A3B-shaped MoE stack (config 2), cold cache", "tokens": T,
+                       "layers": L, "hidden": d, "experts": E, "inter": I, "top_k": k, "slots_per_layer": Ns,
+                       "gemm_min_tokens": args.gemm_min_tokens, "fill_mode": args.fill},
+            "cold": out["cold"], "warm": out["warm"],
+            "roofline": {"bound": "tensor", "kernel": "grouped_gemm_kernel<0>+<1> (warm pass)",
+                         "achieved": w["gemm_tflops"], "peak": tf_burst, "unit": "TFLOP/s",
+                         "frac": (w["gemm_tflops"] / tf_burst) if w["gemm_tflops"] else None,
+                         "frac_of_sustained": (w["gemm_tflops"] / tf_sust) if w["gemm_tflops"] else None,
+                         "peak_source": peak_kind, "traffic": None},
+            "fill": {"GBps": out["cold"]["fill_GBps"], "link_GBps_measured": cal["fill_MBps"] / 1e3},
+            "gpu_launches": out["cold"]["launches"]}
+    print(json.dumps(line), flush=True)
+    moe.destroy()
+    pool.free()
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--mode", default="decode", choices=["decode", "prefill"])
+    ap.add_argument("--tokens", type=int, default=4096)
+    ap.add_argument("--gemm-min-tokens", type=int, default=32)
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=256)
     ap.add_argument("--warmup", type=int, default=32)
@@ -414,6 +507,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.mode == "prefill":
+        run_prefill(args)
     else:
         run_ours(args)
 

@@ -116,7 +116,7 @@ typedef struct {
 } ft_moe_plan_t;
 
 enum { FT_STAT_STEPS = 0, FT_STAT_ROUTED, FT_STAT_HITS, FT_STAT_MISSES, FT_STAT_FILLS, FT_STAT_ZC,
-       FT_STAT_EVICTIONS, FT_STAT_PAIRS, FT_STAT_PAIRS_RESIDENT, FT_STAT_COUNT };
+       FT_STAT_EVICTIONS, FT_STAT_PAIRS, FT_STAT_PAIRS_RESIDENT, FT_STAT_PAIRS_GEMM, FT_STAT_COUNT };
 
 /* S, the bytes of one expert record for this configuration (0 if the shape is not supported). */
 size_t ft_moe_expert_bytes(const ft_moe_config_t *cfg);
@@ -195,7 +195,7 @@ ft_status_t ft_moe_last_fill(ft_moe_t *h, float *out_us, uint64_t *out_bytes);
  * returns, per kind FT_TIME_*, the summed microseconds and the number of timed launches since
  * enable.  Timing adds two event records per launch, so throughput is measured with it off. */
 enum { FT_TIME_ROUTE = 0, FT_TIME_PLAN, FT_TIME_FFN_ZC, FT_TIME_FFN_RES, FT_TIME_FINALIZE, FT_TIME_FILL,
-       FT_TIME_COUNT };
+       FT_TIME_GATHER, FT_TIME_GEMM1, FT_TIME_GEMM2, FT_TIME_COMBINE, FT_TIME_COUNT };
 ft_status_t ft_moe_timing_enable(ft_moe_t *h, int on);
 ft_status_t ft_moe_timing_read(ft_moe_t *h, double *out_us, uint64_t *out_launches, int n);
 /* Number of kernels this handle has launched since create. */

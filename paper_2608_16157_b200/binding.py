@@ -17,7 +17,8 @@ FT_ERR_INVALID_ARG, FT_ERR_NOT_PINNED, FT_ERR_OOM, FT_ERR_CUDA = 1, 2, 3, 4
 FT_ERR_STATE, FT_ERR_TIMEOUT, FT_ERR_NONFINITE, FT_ERR_UNSUPPORTED = 5, 6, 7, 8
 FT_W_BF16, FT_W_INT4_G128 = 0, 1
 FT_FILL_COPY_ENGINE, FT_FILL_SM = 0, 1
-STAT_NAMES = ("steps", "routed", "hits", "misses", "fills", "zc", "evictions", "pairs", "pairs_resident")
+STAT_NAMES = ("steps", "routed", "hits", "misses", "fills", "zc", "evictions", "pairs", "pairs_resident",
+              "pairs_gemm")
 
 # every symbol include/ftmoe.h declares
 SYMBOLS = (
@@ -28,7 +29,7 @@ SYMBOLS = (
     "ft_moe_status_string", "ft_moe_timing_enable", "ft_moe_timing_read", "ft_moe_ffn_noalloc",
 )
 NOALLOC_MAX_TOKENS, NOALLOC_MAX_HIDDEN = 64, 2048
-TIME_NAMES = ("route", "plan", "ffn_zc", "ffn_res", "finalize", "fill")
+TIME_NAMES = ("route", "plan", "ffn_zc", "ffn_res", "finalize", "fill", "gather", "gemm1", "gemm2", "combine")
 
 
 class Config(C.Structure):

@@ -11,6 +11,7 @@
 #include "common.cuh"
 #include "ffn_mma.cuh"
 #include "ffn_stream.cuh"
+#include "gemm_tc.cuh"
 #include "fill.cuh"
 #include "route_plan.cuh"
 
@@ -54,6 +55,12 @@ struct ft_moe {
   WorkItem *items_res = nullptr, *items_zc = nullptr, *items_gemm = nullptr;
   int32_t *res_pref = nullptr;
   bool plan_mirrored = false;
+  // prefill (grouped GEMM) path, allocated only when gemm_min_tokens > 0
+  bool gemm = false;
+  int32_t *gemm_pref = nullptr;
+  uint8_t *is_gemm = nullptr;
+  __nv_bfloat16 *xs = nullptr, *hbuf = nullptr, *obuf = nullptr;   // [P][d], [P][I], [P][d]
+  CUtensorMap tm_xs, tm_h, tm_w128, tm_w64;
   uint32_t *status_dev = nullptr;
   uint32_t *seq_dev = nullptr;
   uint32_t *done_dev = nullptr;          // CTA completion counter of the streaming MMA kernel
@@ -214,6 +221,22 @@ void launch_stream_any(ft_moe *h, const FfnParams &fp, int T, cudaStream_t st) {
   }
 }
 
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// 2-D bf16 row-major tensor [rows][cols] with a [box_rows][box_cols] tile, 128-byte swizzle.
+bool make_tensor_map(EncodeTiledFn fn, CUtensorMap *tm, void *base, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                     uint32_t box_cols) {
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols * 2};
+  const cuuint32_t box[2] = {box_cols, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+         CUDA_SUCCESS;
+}
+
 }  // namespace
 
 extern "C" {
@@ -272,6 +295,11 @@ ft_status_t ft_moe_destroy(ft_moe_t *h) {
   cudaFree(h->items_zc);
   cudaFree(h->items_gemm);
   cudaFree(h->res_pref);
+  cudaFree(h->gemm_pref);
+  cudaFree(h->is_gemm);
+  cudaFree(h->xs);
+  cudaFree(h->hbuf);
+  cudaFree(h->obuf);
   cudaFree(h->status_dev);
   cudaFree(h->seq_dev);
   cudaFree(h->done_dev);
@@ -306,7 +334,9 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
     return FT_ERR_INVALID_ARG;
   const size_t S = expert_bytes_of(cfg);
   if (S == 0 || !geometry_ok(c)) return FT_ERR_UNSUPPORTED;
-  if (c.gemm_min_tokens != 0) return FT_ERR_UNSUPPORTED;
+  if (c.gemm_min_tokens != 0 &&
+      (c.wdtype != FT_W_BF16 || c.slots_per_layer == 0 || c.hidden % 256 || c.inter % 128 || c.gemm_min_tokens < 8))
+    return FT_ERR_UNSUPPORTED;
   if (!c.host_pool || c.host_pool_bytes < (size_t)c.n_layers * c.n_experts * S) return FT_ERR_INVALID_ARG;
   if (c.n_shared && !c.shared_weights) return FT_ERR_INVALID_ARG;
   if ((long long)c.max_tokens * c.top_k > (1ll << 30)) return FT_ERR_INVALID_ARG;
@@ -388,6 +418,33 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
   FT_TRY(cudaMalloc(&h->items_gemm, E * sizeof(WorkItem)));
   FT_TRY(cudaMalloc(&h->res_pref, (E + 2) * 4));
   FT_TRY(cudaMemset(h->res_pref, 0, (E + 2) * 4));
+  if (c.gemm_min_tokens > 0) {
+    const size_t Pr = P + 128;   // one spare tile of rows so that full boxes stay inside the tensors
+    FT_TRY(cudaMalloc(&h->gemm_pref, (E + 1) * 4));
+    FT_TRY(cudaMemset(h->gemm_pref, 0, (E + 1) * 4));
+    FT_TRY(cudaMalloc(&h->is_gemm, E));
+    FT_TRY(cudaMemset(h->is_gemm, 0, E));
+    FT_TRY(cudaMalloc(&h->xs, Pr * c.hidden * 2));
+    FT_TRY(cudaMalloc(&h->hbuf, Pr * c.inter * 2));
+    FT_TRY(cudaMalloc(&h->obuf, Pr * c.hidden * 2));
+    FT_TRY(cudaMemset(h->xs, 0, Pr * c.hidden * 2));
+    FT_TRY(cudaMemset(h->hbuf, 0, Pr * c.inter * 2));
+    void *fnp = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    FT_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fnp, cudaEnableDefault, &qres));
+    if (!fnp || qres != cudaDriverEntryPointSuccess) return fail(FT_ERR_CUDA);
+    EncodeTiledFn enc = reinterpret_cast<EncodeTiledFn>(fnp);
+    const uint64_t wrows = (uint64_t)L * Ns * 3 * c.inter;
+    if (!make_tensor_map(enc, &h->tm_xs, h->xs, Pr, c.hidden, 128, 64) ||
+        !make_tensor_map(enc, &h->tm_h, h->hbuf, Pr, c.inter, 128, 64) ||
+        !make_tensor_map(enc, &h->tm_w128, h->slots, wrows, c.hidden, 128, 64) ||
+        !make_tensor_map(enc, &h->tm_w64, h->slots, wrows, c.hidden, 64, 64))
+      return fail(FT_ERR_CUDA);
+    const int gsm = (int)grouped_gemm_smem_bytes();
+    FT_TRY(cudaFuncSetAttribute(grouped_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, gsm));
+    FT_TRY(cudaFuncSetAttribute(grouped_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, gsm));
+    h->gemm = true;
+  }
   FT_TRY(cudaMalloc(&h->status_dev, 4));
   FT_TRY(cudaMemset(h->status_dev, 0, 4));
   FT_TRY(cudaMalloc(&h->seq_dev, 4));
@@ -473,6 +530,9 @@ static PlanParams make_plan_params(ft_moe *h, int layer, bool mirror_to_host) {
   pp.hdr_host = mirror_to_host ? h->plan_host_devptr : nullptr;
   pp.items_res = h->items_res; pp.res_pref = h->res_pref;
   pp.items_zc = h->items_zc; pp.items_gemm = h->items_gemm;
+  pp.gemm_pref = h->gemm_pref; pp.is_gemm = h->is_gemm;
+  // decode-sized calls on a prefill-capable handle keep every expert on the streaming kernels
+  if (L.T < c.gemm_min_tokens) pp.cm.gemm_min_tokens = 0;
   pp.seq = h->seq_dev;
   return pp;
 }
@@ -635,6 +695,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   }
   // resident set after the fills have landed
   if (c.slots_per_layer > 0) FT_CUDA(cudaStreamWaitEvent(st, h->ev_fill, 0));
+  const bool use_gemm = h->gemm && L.T >= c.gemm_min_tokens;
   if (c.wdtype == FT_W_BF16) {
     // resident experts: bulk-copy pipelined tensor-core streaming kernel; its last CTA finalizes y
     FfnMmaParams mp;
@@ -644,7 +705,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     mp.x = fp.x; mp.perm = h->perm; mp.topk_w = h->topk_w; mp.y_acc = h->y_acc;
     mp.y = static_cast<__nv_bfloat16 *>(y_dev);
     mp.done = h->done_dev; mp.status = h->status_dev;
-    mp.d = c.hidden; mp.inter = c.inter; mp.top_k = c.top_k; mp.T = L.T; mp.finalize = 1;
+    mp.d = c.hidden; mp.inter = c.inter; mp.top_k = c.top_k; mp.T = L.T; mp.finalize = use_gemm ? 0 : 1;
     const size_t smem = ffn_mma_smem_bytes(c.hidden);
     {
       TimeScope ts(h, st, FT_TIME_FFN_RES);
@@ -657,6 +718,36 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     }
     h->launches++;
     FT_CUDA(cudaGetLastError());
+    if (use_gemm) {
+      // experts with many tokens: gather x rows into expert order, two grouped tcgen05 GEMMs, fused combine
+      {
+        TimeScope ts(h, st, FT_TIME_GATHER);
+        gather_rows_kernel<<<h->sm_count * 8, 256, 0, st>>>(fp.x, h->perm, c.top_k, c.hidden, h->offset + c.n_experts, h->xs);
+      }
+      GemmParams gp;
+      gp.items = h->items_gemm; gp.n_items = &h->plan_dev->n_gemm_items; gp.mt_pref = h->gemm_pref;
+      gp.inter = c.inter; gp.d = c.hidden;
+      gp.layer_row0 = (long long)layer * c.slots_per_layer * 3 * c.inter;
+      gp.status = h->status_dev;
+      const size_t gsm = grouped_gemm_smem_bytes();
+      gp.K = c.hidden; gp.n_tiles = c.inter / 128; gp.out = h->hbuf;
+      {
+        TimeScope ts(h, st, FT_TIME_GEMM1);
+        grouped_gemm_kernel<0><<<h->sm_count, kGemmThreads, gsm, st>>>(h->tm_xs, h->tm_w128, gp);
+      }
+      gp.K = c.inter; gp.n_tiles = c.hidden / kGemmBN; gp.out = h->obuf;
+      {
+        TimeScope ts(h, st, FT_TIME_GEMM2);
+        grouped_gemm_kernel<1><<<h->sm_count, kGemmThreads, gsm, st>>>(h->tm_h, h->tm_w64, gp);
+      }
+      {
+        TimeScope ts(h, st, FT_TIME_COMBINE);
+        combine_kernel<<<h->sm_count * 8, 256, 0, st>>>(h->obuf, h->ids, h->topk_w, h->inv, h->is_gemm, h->y_acc,
+                                                        static_cast<__nv_bfloat16 *>(y_dev), L.T, c.top_k, c.hidden);
+      }
+      h->launches += 4;
+      FT_CUDA(cudaGetLastError());
+    }
     return FT_OK;
   }
   if (c.slots_per_layer > 0 || c.n_shared) {

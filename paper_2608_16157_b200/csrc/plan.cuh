@@ -35,6 +35,8 @@ struct PlanParams {
   int32_t *res_pref;     // [E+2]  exclusive prefix of the weight passes of items_res
   WorkItem *items_zc;    // [E]    experts evaluated from the mapped host pool
   WorkItem *items_gemm;  // [E]    experts evaluated from slots by the grouped GEMM
+  int32_t *gemm_pref;    // [E+1]  exclusive prefix of the 128-row tiles of items_gemm
+  uint8_t *is_gemm;      // [E]    1 if the expert goes through the grouped GEMM in this step
   uint32_t *seq;         // [1] plan sequence number
 };
 
@@ -209,6 +211,17 @@ __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, uns
   unsigned long long totC;
   const unsigned long long exC =
       block_excl_scan64(((unsigned long long)(resident ? c : 0) << 32) | (unsigned long long)passes, sm.w, totC);
+  if (p.cm.gemm_min_tokens > 0) {   // uniform branch: only prefill-capable handles pay for this scan
+    unsigned long long totD;
+    const unsigned long long exD = block_excl_scan64(
+        use_gemm ? (((unsigned long long)c << 32) | (unsigned long long)((c + 127) / 128)) : 0ull, sm.w, totD);
+    if (use_gemm) p.gemm_pref[unpack(exB, 3)] = (int32_t)(exD & 0xffffffffull);
+    if (tid == 0) {
+      p.gemm_pref[n_gemm] = (int32_t)(totD & 0xffffffffull);
+      p.stats[9] += (unsigned long long)(totD >> 32);   // pairs served by the grouped GEMM
+    }
+    if (tid < E) p.is_gemm[tid] = (uint8_t)use_gemm;
+  }
   if (is_fill) a_fill[unpack(exB, 0)] = tid;
   if (is_zc) a_zc[unpack(exB, 1)] = tid;
   if (tid < E) a_loc[tid] = loc;
