@@ -497,7 +497,7 @@ def main():
     ap.add_argument("--batch", type=int, default=8)
     ap.add_argument("--layers", type=int, default=48)
     ap.add_argument("--cache-frac", type=float, default=0.5)
-    ap.add_argument("--fill", default="ce", choices=["ce", "sm"])
+    ap.add_argument("--fill", default="sm", choices=["ce", "sm"])
     ap.add_argument("--residual", type=int, default=0, help="use the measured residual zero-copy rate in the plan")
     ap.add_argument("--prof-steps", type=int, default=16)
     ap.add_argument("--e2e-steps", type=int, default=32)

@@ -498,6 +498,15 @@ ft_status_t ft_moe_reset(ft_moe_t *h, int layer) {
   return FT_OK;
 }
 
+// Threads of the single-CTA route / plan kernels: one per expert, one warp per token, at least 256.
+static int single_cta_threads(int E, int T) {
+  int n = E > 32 * T ? E : 32 * T;
+  n = ((n + 31) / 32) * 32;
+  if (n < 256) n = 256;
+  if (n > 1024) n = 1024;
+  return n;
+}
+
 static RouteParams make_route_params(ft_moe *h, const float *logits_dev, int T) {
   RouteParams rp;
   rp.logits = logits_dev;
@@ -533,7 +542,7 @@ static PlanParams make_plan_params(ft_moe *h, int layer, bool mirror_to_host) {
   pp.gemm_pref = h->gemm_pref; pp.is_gemm = h->is_gemm;
   // decode-sized calls on a prefill-capable handle keep every expert on the streaming kernels
   if (L.T < c.gemm_min_tokens) pp.cm.gemm_min_tokens = 0;
-  pp.seq = h->seq_dev;
+  pp.seq_value = h->seq_host + 1;
   return pp;
 }
 
@@ -549,7 +558,7 @@ ft_status_t ft_moe_route(ft_moe_t *h, int layer, const float *logits_dev, int T,
   const RouteParams rp = make_route_params(h, logits_dev, T);
   TimeScope ts(h, st, FT_TIME_ROUTE);
   if (T <= kRouteSmallMaxTokens) {
-    route_small_kernel<<<1, 1024, 0, st>>>(rp);
+    route_small_kernel<<<1, single_cta_threads(h->cfg.n_experts, T), 0, st>>>(rp);
     h->launches++;
   } else {
     FT_CUDA(cudaMemsetAsync(h->count, 0, sizeof(int32_t) * rp.E, st));
@@ -782,7 +791,7 @@ ft_status_t ft_moe_layer(ft_moe_t *h, int layer, const float *logits_dev, const 
     const PlanParams pp = make_plan_params(h, layer, mirror);
     {
       TimeScope ts(h, st, FT_TIME_PLAN);
-      route_plan_small_kernel<<<1, 1024, (size_t)c.slots_per_layer * 16, st>>>(rp, pp);
+      route_plan_small_kernel<<<1, single_cta_threads(c.n_experts, T), (size_t)c.slots_per_layer * 16, st>>>(rp, pp);
     }
     h->launches++;
     h->seq_host++;

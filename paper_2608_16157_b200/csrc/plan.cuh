@@ -37,7 +37,7 @@ struct PlanParams {
   WorkItem *items_gemm;  // [E]    experts evaluated from slots by the grouped GEMM
   int32_t *gemm_pref;    // [E+1]  exclusive prefix of the 128-row tiles of items_gemm
   uint8_t *is_gemm;      // [E]    1 if the expert goes through the grouped GEMM in this step
-  uint32_t *seq;         // [1] plan sequence number
+  uint32_t seq_value;    // sequence number of this plan (counted by the host)
 };
 
 // Block-wide exclusive scan of one 64-bit value per thread (several small counters packed into it).
@@ -83,33 +83,47 @@ struct PlanSmem {
   unsigned long long w[33];
   int32_t cnt[kMaxExperts];
   uint8_t elig[kMaxExperts];
+  uint8_t isfill[kMaxExperts];
   int32_t forder[kMaxExperts];
-  int K;
+  int16_t miss[kMaxExperts];
 };
 
 // One plan step.  Thread `tid` < E owns expert `tid`: `c` = its token count, `off` = its offset in the
 // expert-sorted pair order, `n_pairs` = all pairs of the call.  blockDim.x >= E, a multiple of 32.
 // s_dyn: int64 stamp[n_slots]; int32 sexp[n_slots]; int32 victim[n_slots].
+// Issues every global read of the layer's state up front (step counter, this thread's expert_slot, the slot
+// table into shared memory) so their latencies overlap each other and whatever the caller does next.
+// A barrier must separate this from plan_body.
+__device__ __forceinline__ void plan_prefetch(const PlanParams &p, unsigned char *s_dyn, int64_t &t, int &slot) {
+  int64_t *s_stamp = reinterpret_cast<int64_t *>(s_dyn);
+  int32_t *s_sexp = reinterpret_cast<int32_t *>(s_stamp + p.n_slots);
+  const int tid = threadIdx.x;
+  t = *p.step;
+  slot = (tid < p.E) ? p.expert_slot[tid] : -1;
+  for (int s = tid; s < p.n_slots; s += blockDim.x) {
+    s_stamp[s] = p.slot_stamp[s];
+    s_sexp[s] = p.slot_expert[s];
+  }
+}
+
 __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, unsigned char *s_dyn, int c, int off,
-                                          int n_pairs) {
+                                          int n_pairs, const int64_t t, const int slot_in) {
   int64_t *s_stamp = reinterpret_cast<int64_t *>(s_dyn);
   int32_t *s_sexp = reinterpret_cast<int32_t *>(s_stamp + p.n_slots);
   int32_t *s_victim = s_sexp + p.n_slots;
   const int tid = threadIdx.x;
   const int E = p.E;
   if (n_pairs == 0) return;  // nothing routed: the step does not advance
-  const int64_t t = *p.step;
 
   int32_t *a_hit = reinterpret_cast<int32_t *>(p.hdr_dev + 1);
   int32_t *a_miss = a_hit + E, *a_fill = a_miss + E, *a_zc = a_fill + E, *a_forder = a_zc + E;
   int32_t *a_fslot = a_forder + E, *a_fevict = a_fslot + E, *a_loc = a_fevict + E;
 
   // ---- 1/2: classify, refresh recency of hits; 4: which misses are worth a fill
-  int slot = -1, cls = 0, elig = 0;
+  int slot = slot_in, cls = 0, elig = 0;
   if (tid < E) {
-    slot = p.expert_slot[tid];
     cls = (c > 0) ? (slot >= 0 ? 1 : 2) : 0;
-    if (cls == 1) p.slot_stamp[slot] = t;
+    if (cls == 1) { p.slot_stamp[slot] = t; s_stamp[slot] = t; }
     if (cls == 2) {
       const int64_t pz = (c + p.cm.tz - 1) / p.cm.tz, pg = (c + p.cm.tg - 1) / p.cm.tg;
       const int64_t v = pz * p.cm.ns_zc - (p.cm.ns_fill + pg * p.cm.ns_hbm) +
@@ -118,42 +132,48 @@ __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, uns
     }
     sm.cnt[tid] = c;
     sm.elig[tid] = (uint8_t)elig;
+    sm.isfill[tid] = 0;
   }
-  if (tid == 0) sm.K = 0;
   unsigned long long totA;
   const unsigned long long exA = block_excl_scan64(pack4(cls != 0, cls == 1, cls == 2, elig), sm.w, totA);
   const int n_routed = unpack(totA, 0), n_hit = unpack(totA, 1), n_miss = unpack(totA, 2), n_elig = unpack(totA, 3);
   if (cls == 1) a_hit[unpack(exA, 1)] = tid;
-  if (cls == 2) a_miss[unpack(exA, 2)] = tid;
-
-  // ---- 3: victim candidates, ordered in one pass by counting how many candidates precede each
-  // (the scan's barriers make the refreshed stamps visible to the whole block)
-  for (int s = tid; s < p.n_slots; s += blockDim.x) {
-    s_stamp[s] = p.slot_stamp[s];
-    s_sexp[s] = p.slot_expert[s];
+  if (cls == 2) {
+    a_miss[unpack(exA, 2)] = tid;
+    sm.miss[unpack(exA, 2)] = (int16_t)tid;
   }
-  __syncthreads();
-  for (int s = tid; s < p.n_slots; s += blockDim.x) {
+  __syncthreads();   // sm.miss and the refreshed stamps are visible to the whole block from here on
+
+  // ---- 3: victim candidates, ordered in one pass: each warp ranks a few candidates by counting, 32 slots per
+  // ballot, how many candidates precede them (free slots first by index, then (stamp, resident expert id))
+  // (the scan's barriers make the refreshed stamps in shared memory visible to the whole block)
+  const int lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+  int K = 0;
+  for (int base = 0; base < p.n_slots; base += 32) {
+    const int o = base + lane;
+    const bool oc = (o < p.n_slots) && ((s_sexp[o] < 0) || (s_stamp[o] < t));
+    K += __popc(__ballot_sync(0xffffffffu, oc));
+  }
+  for (int s = warp; s < p.n_slots; s += nwarps) {
     const int64_t st = s_stamp[s];
     const int ex = s_sexp[s];
-    const bool cand = (ex < 0) || (st < t);
-    if (!cand) continue;
+    if (!((ex < 0) || (st < t))) continue;      // warp-uniform
     int rank = 0;
-    for (int o = 0; o < p.n_slots; ++o) {
-      const int oex = s_sexp[o];
-      const int64_t ost = s_stamp[o];
-      if (!((oex < 0) || (ost < t)) || o == s) continue;
-      bool before;
-      if (oex < 0) before = (ex >= 0) || (o < s);            // free slots first, by slot index
-      else if (ex < 0) before = false;
-      else before = (ost < st) || (ost == st && oex < ex);   // then (stamp, resident expert id)
-      rank += before ? 1 : 0;
+    for (int base = 0; base < p.n_slots; base += 32) {
+      const int o = base + lane;
+      bool before = false;
+      if (o < p.n_slots && o != s) {
+        const int oex = s_sexp[o];
+        const int64_t ost = s_stamp[o];
+        if ((oex < 0) || (ost < t)) {
+          if (oex < 0) before = (ex >= 0) || (o < s);
+          else if (ex >= 0) before = (ost < st) || (ost == st && oex < ex);
+        }
+      }
+      rank += __popc(__ballot_sync(0xffffffffu, before));
     }
-    s_victim[rank] = s;
-    atomicAdd(&sm.K, 1);  // a count
+    if (lane == 0) s_victim[rank] = s;
   }
-  __syncthreads();
-  const int K = sm.K;
 
   // ---- 5: fill count
   int q = 0;
@@ -166,18 +186,26 @@ __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, uns
     if (q > K) q = K;
   }
 
-  // ---- 6: priority of the eligible misses (tokens descending, id ascending)
-  int is_fill = 0;
-  if (elig) {
+  // ---- 6: priority of the eligible misses (tokens descending, id ascending): each warp ranks a few misses
+  // by ballots over the experts; sm.miss was written before the scan's barriers
+  for (int i = warp; i < n_miss; i += nwarps) {
+    const int e = sm.miss[i];
+    if (!sm.elig[e]) continue;                  // warp-uniform
+    const int ce = sm.cnt[e];
     int rank = 0;
-    for (int o = 0; o < E; ++o) {
-      if (!sm.elig[o] || o == tid) continue;
-      const int oc = sm.cnt[o];
-      rank += (oc > c || (oc == c && o < tid)) ? 1 : 0;
+    for (int base = 0; base < E; base += 32) {
+      const int o = base + lane;
+      bool better = false;
+      if (o < E && o != e && sm.elig[o]) {
+        const int oc = sm.cnt[o];
+        better = (oc > ce) || (oc == ce && o < e);
+      }
+      rank += __popc(__ballot_sync(0xffffffffu, better));
     }
-    if (rank < q) { is_fill = 1; sm.forder[rank] = tid; }
+    if (lane == 0 && rank < q) { sm.forder[rank] = e; sm.isfill[e] = 1; }
   }
   __syncthreads();
+  const int is_fill = (tid < E) ? sm.isfill[tid] : 0;
 
   // ---- 7: the i-th fill takes the i-th candidate slot
   int loc = kLocNotRouted;
@@ -218,7 +246,7 @@ __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, uns
     if (use_gemm) p.gemm_pref[unpack(exB, 3)] = (int32_t)(exD & 0xffffffffull);
     if (tid == 0) {
       p.gemm_pref[n_gemm] = (int32_t)(totD & 0xffffffffull);
-      p.stats[9] += (unsigned long long)(totD >> 32);   // pairs served by the grouped GEMM
+      atomicAdd(&p.stats[9], (unsigned long long)(totD >> 32));   // pairs served by the grouped GEMM
     }
     if (tid < E) p.is_gemm[tid] = (uint8_t)use_gemm;
   }
@@ -269,22 +297,22 @@ __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, uns
     h.step = t;
     h.n_routed = n_routed; h.n_hit = n_hit; h.n_miss = n_miss; h.n_fill = n_fill; h.n_zc = n_zc;
     h.n_res_items = n_res_items; h.n_zc_items = n_zc; h.n_gemm_items = n_gemm;
-    h.seq = *p.seq + 1;
+    h.seq = p.seq_value;
     h.pad[0] = h.pad[1] = h.pad[2] = h.pad[3] = h.pad[4] = 0;
     *p.hdr_dev = h;
-    *p.seq = h.seq;
     *p.step = t + 1;
     int evictions = 0;
     for (int i = 0; i < n_fill; ++i) evictions += (s_sexp[s_victim[i]] >= 0);
-    p.stats[0] += 1;
-    p.stats[1] += n_routed;
-    p.stats[2] += n_hit;
-    p.stats[3] += n_miss;
-    p.stats[4] += n_fill;
-    p.stats[5] += n_zc;
-    p.stats[6] += evictions;
-    p.stats[7] += n_pairs;
-    p.stats[8] += (unsigned long long)(totC >> 32);
+    // fire-and-forget adds: nothing waits for the old values
+    atomicAdd(&p.stats[0], 1ull);
+    atomicAdd(&p.stats[1], (unsigned long long)n_routed);
+    atomicAdd(&p.stats[2], (unsigned long long)n_hit);
+    atomicAdd(&p.stats[3], (unsigned long long)n_miss);
+    atomicAdd(&p.stats[4], (unsigned long long)n_fill);
+    atomicAdd(&p.stats[5], (unsigned long long)n_zc);
+    atomicAdd(&p.stats[6], (unsigned long long)evictions);
+    atomicAdd(&p.stats[7], (unsigned long long)n_pairs);
+    atomicAdd(&p.stats[8], (unsigned long long)(totC >> 32));
   }
   // mirror the record into mapped host memory when the host reads the plan (copy-engine fills)
   if (p.hdr_host != nullptr) {
@@ -301,10 +329,14 @@ __global__ void __launch_bounds__(1024) plan_kernel(PlanParams p) {
   extern __shared__ __align__(16) unsigned char s_dyn[];
   __shared__ PlanSmem sm;
   const int tid = threadIdx.x;
+  int64_t t;
+  int slot;
+  plan_prefetch(p, s_dyn, t, slot);
   const int n_pairs = p.offset[p.E];
   int c = 0, off = 0;
   if (tid < p.E) { c = p.count[tid]; off = p.offset[tid]; }
-  plan_body(p, sm, s_dyn, c, off, n_pairs);
+  __syncthreads();
+  plan_body(p, sm, s_dyn, c, off, n_pairs, t, slot);
 }
 
 }  // namespace ftmoe

@@ -94,14 +94,15 @@ struct RouteSmem {
   int32_t wsum[32];
 };
 
-// Decode-sized calls: one CTA (1024 threads) routes all tokens, counts, scans and permutes.  On
+// Decode-sized calls: one CTA (a warp multiple of at least E threads) routes all tokens, counts, scans and permutes.  On
 // return (after a barrier) s.cnt / s.off hold count[] and offset[] for the caller.
 __device__ __forceinline__ void route_small_body(const RouteParams &p, RouteSmem &s) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int P = p.T * p.k;
   for (int e = tid; e < p.E; e += blockDim.x) s.cnt[e] = 0;
   __syncthreads();
-  for (int t = warp; t < p.T; t += 32) {
+  const int nwarps = blockDim.x >> 5;
+  for (int t = warp; t < p.T; t += nwarps) {
     int id;
     float w;
     route_token_any(p, t, lane, id, w);
@@ -125,7 +126,7 @@ __device__ __forceinline__ void route_small_body(const RouteParams &p, RouteSmem
     if (lane == 31) s.wsum[warp] = incl;
     __syncthreads();
     if (warp == 0) {
-      int ws = s.wsum[lane];
+      int ws = (lane < nwarps) ? s.wsum[lane] : 0;
       int wincl = ws;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
@@ -145,7 +146,7 @@ __device__ __forceinline__ void route_small_body(const RouteParams &p, RouteSmem
   }
   __syncthreads();
   // one warp per expert walks the pairs in index order: rank = number of earlier pairs with this key
-  for (int e = warp; e < p.E; e += 32) {
+  for (int e = warp; e < p.E; e += nwarps) {
     if (s.cnt[e] == 0) continue;
     int run = s.off[e];
     for (int base = 0; base < P; base += 32) {

@@ -9,12 +9,15 @@ __global__ void __launch_bounds__(1024) route_plan_small_kernel(RouteParams rp, 
   extern __shared__ __align__(16) unsigned char s_dyn[];
   __shared__ RouteSmem rs;
   __shared__ PlanSmem ps;
+  int64_t t;
+  int slot;
+  plan_prefetch(pp, s_dyn, t, slot);   // state loads overlap the logits load of the routing below
   route_small_body(rp, rs);
   __syncthreads();
   const int tid = threadIdx.x;
   int c = 0, off = 0;
   if (tid < rp.E) { c = rs.cnt[tid]; off = rs.off[tid]; }
-  plan_body(pp, ps, s_dyn, c, off, rp.T * rp.k);
+  plan_body(pp, ps, s_dyn, c, off, rp.T * rp.k, t, slot);
 }
 
 }  // namespace ftmoe
