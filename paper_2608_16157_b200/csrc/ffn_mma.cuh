@@ -17,7 +17,7 @@
 
 namespace ftmoe {
 
-constexpr int kMmaStages = 3;
+constexpr int kMmaStages = 6;     // one per (matrix, row half): a block of 16 neurons is 6 half tiles
 constexpr int kMmaTileRows = 16;
 constexpr int kMmaConsumers = 256;
 constexpr int kMmaThreads = kMmaConsumers + 32;
@@ -35,6 +35,7 @@ struct FfnMmaParams {
   uint32_t *done;           // CTA completion counter, zero between launches
   uint32_t *status;
   int d, inter, top_k, T, finalize;
+  int max_items;            // capacity of items / pref (entries beyond *n_items are ignored)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -92,22 +93,24 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t add
 }
 
 // Dynamic shared memory layout (bytes): [stages][16 rows x (2d+64)] | red [8][2][16][8] f32 | hs [8][16] bf16
-// | pref [kMaxExperts+2] i32 | mbarriers full[3], empty[3] | abort flag.
+// | pref [kMaxExperts+2] i32 | mbarriers full[], empty[] | abort flag | record pointers [kMaxExperts+1].
 template <int KB>  // KB = d / 256: 32-wide k-blocks per warp in the gate/up phase
 __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p) {
   constexpr int CTW = 2 * KB;  // 16-column tiles per warp in the down phase
   extern __shared__ __align__(128) unsigned char smem[];
   const int d = p.d;
   const uint32_t row_bytes = 2u * d;
-  const uint32_t stride_gu = row_bytes + 64;   // = 64 mod 128: conflict-free 16-byte fragment loads
-  const uint32_t stride_d = row_bytes + 16;    // = 16 mod 128: conflict-free ldmatrix rows
+  const uint32_t half_bytes = row_bytes / 2;   // a stage holds the lower or upper half of 16 rows
+  const uint32_t stride_gu = half_bytes + 64;  // = 64 mod 128: conflict-free 16-byte fragment loads
+  const uint32_t stride_d = half_bytes + 16;   // = 16 mod 128: conflict-free ldmatrix rows
   const uint32_t stage_bytes = kMmaTileRows * stride_gu;
   unsigned char *sp = smem + (size_t)kMmaStages * stage_bytes;
   float *s_red = reinterpret_cast<float *>(sp); sp += 8 * 2 * 16 * 8 * 4;
   __nv_bfloat16 *s_h = reinterpret_cast<__nv_bfloat16 *>(sp); sp += 8 * 16 * 2;
   int32_t *s_pref = reinterpret_cast<int32_t *>(sp); sp += (kMaxExperts + 2) * 4;
   uint64_t *s_bar = reinterpret_cast<uint64_t *>(sp); sp += 2 * kMmaStages * 8;
-  volatile int *s_abort = reinterpret_cast<volatile int *>(sp);
+  volatile int *s_abort = reinterpret_cast<volatile int *>(sp); sp += 16;
+  const uint8_t **s_recs = reinterpret_cast<const uint8_t **>(sp);
   __shared__ int s_last;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -121,55 +124,62 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
   if (tid == 0) {
     for (int s = 0; s < kMmaStages; ++s) {
       mbar_init(full_bar(s), 1);
-      mbar_init(empty_bar(s), 8);
+      mbar_init(empty_bar(s), 4);   // the four warps that own this half
     }
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  // prefix sums of the weight passes per item (8 tokens per pass), written by the plan kernel
-  for (int i = tid; i <= n_items; i += blockDim.x) s_pref[i] = p.pref[i];
+  // prefix sums of the weight passes per item (8 tokens per pass) and the record pointers, written by the
+  // plan kernel; loaded up to the lists' capacity so that these loads do not wait for the item count
+  for (int i = tid; i <= p.max_items; i += blockDim.x) {
+    s_pref[i] = p.pref[i];
+    if (i < p.max_items) s_recs[i] = p.items[i].w;
+  }
   __syncthreads();
   const long long total = (long long)s_pref[n_items] * NBLK;
   long long u = total * blockIdx.x / gridDim.x;
   const long long u1 = total * (blockIdx.x + 1) / gridDim.x;
   int item = 0;
-  uint32_t tile = 0;  // tiles consumed / produced so far by this CTA
+  uint32_t tile = 0;  // 16-neuron blocks consumed / produced so far by this CTA
 
   if (warp == 8) {
     // ------------------------------ producer ------------------------------
-    if (lane == 0) {
-      while (u < u1) {
-        const long long pu = u / NBLK;
-        while (s_pref[item + 1] <= pu) ++item;
-        const int b_begin = (int)(u - pu * NBLK);
-        const long long left = u1 - u;
-        const int b_end = (left < (long long)(NBLK - b_begin)) ? b_begin + (int)left : NBLK;
-        const uint8_t *rec = p.items[item].w;
-        const size_t mat_bytes = (size_t)row_bytes * p.inter;
-        for (int b = b_begin; b < b_end; ++b) {
+    // lane 0 waits for the stage and posts the byte count; lanes 0..15 then issue one row copy each, so the
+    // issue rate of a single thread never limits the stream
+    while (u < u1) {
+      const long long pu = u / NBLK;
+      while (s_pref[item + 1] <= pu) ++item;
+      const int b_begin = (int)(u - pu * NBLK);
+      const long long left = u1 - u;
+      const int b_end = (left < (long long)(NBLK - b_begin)) ? b_begin + (int)left : NBLK;
+      const uint8_t *rec = s_recs[item];
+      const size_t mat_bytes = (size_t)row_bytes * p.inter;
+      for (int b = b_begin; b < b_end; ++b, ++tile) {
+        const uint32_t ph = tile & 1u;     // `tile` counts this CTA's blocks; stage = 2*matrix + half
 #pragma unroll 1
-          for (int which = 0; which < 3; ++which) {
-            const int s = tile % kMmaStages;
-            const uint32_t ph = (tile / kMmaStages) & 1u;
+        for (int s = 0; s < kMmaStages; ++s) {
+          const int which = s >> 1, half = s & 1;
+          if (lane == 0) {
             mbar_wait(empty_bar(s), ph ^ 1u, s_abort, p.status);
-            if (*s_abort) break;
-            mbar_expect_tx(full_bar(s), kMmaTileRows * row_bytes);
-            const uint8_t *src = rec + which * mat_bytes + (size_t)b * kMmaTileRows * row_bytes;
-            const uint32_t dst = smem_base + s * stage_bytes;
+            mbar_expect_tx(full_bar(s), kMmaTileRows * half_bytes);
+          }
+          __syncwarp();
+          if (lane < kMmaTileRows && !*s_abort) {
+            const uint8_t *src = rec + which * mat_bytes + (size_t)(b * kMmaTileRows + lane) * row_bytes + half * half_bytes;
             const uint32_t stride = (which == 2) ? stride_d : stride_gu;
-#pragma unroll 4
-            for (int r = 0; r < kMmaTileRows; ++r) bulk_g2s(dst + r * stride, src + (size_t)r * row_bytes, row_bytes, full_bar(s));
-            ++tile;
+            bulk_g2s(smem_base + s * stage_bytes + lane * stride, src, half_bytes, full_bar(s));
           }
         }
-        u += (b_end - b_begin);
       }
+      u += (b_end - b_begin);
     }
   } else {
     // ------------------------------ consumers ------------------------------
     const int g = lane >> 2, q = lane & 3;
     const int kslice = warp * (d / 8);      // first k of this warp's slice (gate/up) and first column (down)
+    const int half = warp >> 2;             // which half of the rows' bytes this warp reads
+    const int kl = (warp & 3) * (d / 8);    // the same offset inside that half
     while (u < u1) {
       const long long pu = u / NBLK;
       while (s_pref[item + 1] <= pu) ++item;
@@ -207,12 +217,12 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
         float cgu[2][4];
 #pragma unroll
         for (int which = 0; which < 2; ++which) {
-          const int s = tile % kMmaStages;
-          const uint32_t ph = (tile / kMmaStages) & 1u;
+          const int s = 2 * which + half;
+          const uint32_t ph = tile & 1u;
           cgu[which][0] = cgu[which][1] = cgu[which][2] = cgu[which][3] = 0.f;
           const bool ok = mbar_wait(full_bar(s), ph, s_abort, p.status);
           if (ok) {
-            const uint32_t base = smem_base + s * stage_bytes + (uint32_t)(kslice + 8 * q) * 2u;
+            const uint32_t base = smem_base + s * stage_bytes + (uint32_t)(kl + 8 * q) * 2u;
 #pragma unroll
             for (int kb = 0; kb < KB; ++kb) {
               const uint4 lo = lds_v4(base + g * stride_gu + kb * 64);
@@ -223,7 +233,6 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(empty_bar(s));
-          ++tile;
         }
         // cross-warp reduction of the [16 neurons][8 tokens] partial sums
         {
@@ -249,8 +258,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
         asm volatile("bar.sync 1, 256;" ::: "memory");
         // down tile
         {
-          const int s = tile % kMmaStages;
-          const uint32_t ph = (tile / kMmaStages) & 1u;
+          const int s = 4 + half;
+          const uint32_t ph = tile & 1u;
           const bool ok = mbar_wait(full_bar(s), ph, s_abort, p.status);
           if (ok) {
             const uint32_t *h32 = reinterpret_cast<const uint32_t *>(s_h);
@@ -258,7 +267,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
             // ldmatrix.x4.trans: lanes 0-7 / 8-15 / 16-23 / 24-31 address the four 8x8 blocks
             const int mat = lane >> 3, r = lane & 7;
             const uint32_t abase = smem_base + s * stage_bytes + (uint32_t)(r + 8 * (mat >> 1)) * stride_d +
-                                   (uint32_t)(kslice + 8 * (mat & 1)) * 2u;
+                                   (uint32_t)(kl + 8 * (mat & 1)) * 2u;
 #pragma unroll
             for (int c = 0; c < CTW; ++c) {
               uint32_t a[4];
@@ -319,8 +328,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
 }
 
 inline size_t ffn_mma_smem_bytes(int d) {
-  return (size_t)kMmaStages * kMmaTileRows * (2 * (size_t)d + 64) + 8 * 2 * 16 * 8 * 4 + 8 * 16 * 2 +
-         (kMaxExperts + 2) * 4 + 2 * kMmaStages * 8 + 16;
+  return (size_t)kMmaStages * kMmaTileRows * ((size_t)d + 64) + 8 * 2 * 16 * 8 * 4 + 8 * 16 * 2 +
+         (kMaxExperts + 2) * 4 + 2 * kMmaStages * 8 + 16 + (kMaxExperts + 1) * 8;
 }
 
 }  // namespace ftmoe

@@ -711,6 +711,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     mp.items = h->items_res;
     mp.n_items = &h->plan_dev->n_res_items;
     mp.pref = h->res_pref;
+    mp.max_items = c.n_experts + 1;
     mp.x = fp.x; mp.perm = h->perm; mp.topk_w = h->topk_w; mp.y_acc = h->y_acc;
     mp.y = static_cast<__nv_bfloat16 *>(y_dev);
     mp.done = h->done_dev; mp.status = h->status_dev;
