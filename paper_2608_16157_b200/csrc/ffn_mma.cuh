@@ -25,7 +25,8 @@ constexpr int kMmaTokens = 8;  // tokens per weight pass
 
 struct FfnMmaParams {
   const WorkItem *items;
-  const int32_t *n_items;
+  const int32_t *n_items;   // resident items (records in HBM slots)
+  const int32_t *n_zc;      // zero-copy items appended after them (records in the mapped host pool)
   const int32_t *pref;      // [n_items+1] exclusive prefix of the weight passes per item (from the plan)
   const __nv_bfloat16 *x;   // [T][d]
   const int32_t *perm;
@@ -93,7 +94,7 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t add
 }
 
 // Dynamic shared memory layout (bytes): [stages][16 rows x (2d+64)] | red [8][2][16][8] f32 | hs [8][16] bf16
-// | pref [kMaxExperts+2] i32 | mbarriers full[], empty[] | abort flag | record pointers [kMaxExperts+1].
+// | pref [2*kMaxExperts+2] i32 | mbarriers full[], empty[] | abort flag.
 template <int KB>  // KB = d / 256: 32-wide k-blocks per warp in the gate/up phase
 __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p) {
   constexpr int CTW = 2 * KB;  // 16-column tiles per warp in the down phase
@@ -107,10 +108,9 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
   unsigned char *sp = smem + (size_t)kMmaStages * stage_bytes;
   float *s_red = reinterpret_cast<float *>(sp); sp += 8 * 2 * 16 * 8 * 4;
   __nv_bfloat16 *s_h = reinterpret_cast<__nv_bfloat16 *>(sp); sp += 8 * 16 * 2;
-  int32_t *s_pref = reinterpret_cast<int32_t *>(sp); sp += (kMaxExperts + 2) * 4;
+  int32_t *s_pref = reinterpret_cast<int32_t *>(sp); sp += (2 * kMaxExperts + 2) * 4;
   uint64_t *s_bar = reinterpret_cast<uint64_t *>(sp); sp += 2 * kMmaStages * 8;
-  volatile int *s_abort = reinterpret_cast<volatile int *>(sp); sp += 16;
-  const uint8_t **s_recs = reinterpret_cast<const uint8_t **>(sp);
+  volatile int *s_abort = reinterpret_cast<volatile int *>(sp);
   __shared__ int s_last;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -132,14 +132,13 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
   }
   // prefix sums of the weight passes per item (8 tokens per pass) and the record pointers, written by the
   // plan kernel; loaded up to the lists' capacity so that these loads do not wait for the item count
-  for (int i = tid; i <= p.max_items; i += blockDim.x) {
-    s_pref[i] = p.pref[i];
-    if (i < p.max_items) s_recs[i] = p.items[i].w;
-  }
+  const int n_zc = *p.n_zc;
+  for (int i = tid; i <= p.max_items; i += blockDim.x) s_pref[i] = p.pref[i];
   __syncthreads();
-  const long long total = (long long)s_pref[n_items] * NBLK;
-  long long u = total * blockIdx.x / gridDim.x;
-  const long long u1 = total * (blockIdx.x + 1) / gridDim.x;
+  // two work ranges, each split evenly over the CTAs: HBM-resident blocks, then host-resident blocks (the
+  // latter are bound by the host link, so every CTA takes an equal share of them)
+  const long long total_res = (long long)s_pref[n_items] * NBLK;
+  const long long total_all = (long long)s_pref[n_items + n_zc] * NBLK;
   int item = 0;
   uint32_t tile = 0;  // 16-neuron blocks consumed / produced so far by this CTA
 
@@ -147,13 +146,17 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
     // ------------------------------ producer ------------------------------
     // lane 0 waits for the stage and posts the byte count; lanes 0..15 then issue one row copy each, so the
     // issue rate of a single thread never limits the stream
+    for (int range = 0; range < 2; ++range) {
+    const long long r0 = range ? total_res : 0, rn = range ? total_all - total_res : total_res;
+    long long u = r0 + rn * blockIdx.x / gridDim.x;
+    const long long u1 = r0 + rn * (blockIdx.x + 1) / gridDim.x;
     while (u < u1) {
       const long long pu = u / NBLK;
       while (s_pref[item + 1] <= pu) ++item;
       const int b_begin = (int)(u - pu * NBLK);
       const long long left = u1 - u;
       const int b_end = (left < (long long)(NBLK - b_begin)) ? b_begin + (int)left : NBLK;
-      const uint8_t *rec = s_recs[item];
+      const uint8_t *rec = p.items[item].w;
       const size_t mat_bytes = (size_t)row_bytes * p.inter;
       for (int b = b_begin; b < b_end; ++b, ++tile) {
         const uint32_t ph = tile & 1u;     // `tile` counts this CTA's blocks; stage = 2*matrix + half
@@ -174,12 +177,17 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
       }
       u += (b_end - b_begin);
     }
+    }
   } else {
     // ------------------------------ consumers ------------------------------
     const int g = lane >> 2, q = lane & 3;
     const int kslice = warp * (d / 8);      // first k of this warp's slice (gate/up) and first column (down)
     const int half = warp >> 2;             // which half of the rows' bytes this warp reads
     const int kl = (warp & 3) * (d / 8);    // the same offset inside that half
+    for (int range = 0; range < 2; ++range) {
+    const long long r0 = range ? total_res : 0, rn = range ? total_all - total_res : total_res;
+    long long u = r0 + rn * blockIdx.x / gridDim.x;
+    const long long u1 = r0 + rn * (blockIdx.x + 1) / gridDim.x;
     while (u < u1) {
       const long long pu = u / NBLK;
       while (s_pref[item + 1] <= pu) ++item;
@@ -301,6 +309,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
       }
       u += (b_end - b_begin);
     }
+    }
   }
 
   // ---- the last CTA to finish rounds the accumulator to bf16 and clears it ----
@@ -329,7 +338,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
 
 inline size_t ffn_mma_smem_bytes(int d) {
   return (size_t)kMmaStages * kMmaTileRows * ((size_t)d + 64) + 8 * 2 * 16 * 8 * 4 + 8 * 16 * 2 +
-         (kMaxExperts + 2) * 4 + 2 * kMmaStages * 8 + 16 + (kMaxExperts + 1) * 8;
+         (2 * kMaxExperts + 2) * 4 + 2 * kMmaStages * 8 + 16;
 }
 
 }  // namespace ftmoe

@@ -28,6 +28,7 @@ struct NoAllocCtl {
   WorkItem item;       // the one expert: all T tokens, gate weight 1
   int32_t pref[2];     // {0, passes}
   int32_t n_items;     // 1
+  int32_t n_zc;        // 0: no host-resident records here
   uint32_t done;       // CTA completion counter of the kernel
   uint32_t status;     // latched device status of the last call
 };
@@ -53,6 +54,7 @@ __global__ void noalloc_setup_kernel(const uint8_t *record, int T, int hidden) {
     ctl->pref[0] = 0;
     ctl->pref[1] = (T + kMmaTokens - 1) / kMmaTokens;
     ctl->n_items = 1;
+    ctl->n_zc = 0;
     ctl->done = 0u;
     ctl->status = 0u;
   }
@@ -110,6 +112,7 @@ extern "C" ft_status_t ft_moe_ffn_noalloc(int device, const void *record_dev, in
   FfnMmaParams mp;
   mp.items = &ctl->item;
   mp.n_items = &ctl->n_items;
+  mp.n_zc = &ctl->n_zc;
   mp.pref = ctl->pref;
   mp.max_items = 1;
   mp.x = static_cast<const __nv_bfloat16 *>(x_dev);

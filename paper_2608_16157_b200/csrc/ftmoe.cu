@@ -413,11 +413,12 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
   FT_TRY(cudaHostAlloc(&h->plan_host, h->plan_bytes, cudaHostAllocMapped));
   memset(h->plan_host, 0, h->plan_bytes);
   FT_TRY(cudaHostGetDevicePointer(reinterpret_cast<void **>(&h->plan_host_devptr), h->plan_host, 0));
-  FT_TRY(cudaMalloc(&h->items_res, (E + 1) * sizeof(WorkItem)));
+  FT_TRY(cudaMalloc(&h->items_res, (2 * E + 1) * sizeof(WorkItem)));
+  FT_TRY(cudaMemset(h->items_res, 0, (2 * E + 1) * sizeof(WorkItem)));
   FT_TRY(cudaMalloc(&h->items_zc, E * sizeof(WorkItem)));
   FT_TRY(cudaMalloc(&h->items_gemm, E * sizeof(WorkItem)));
-  FT_TRY(cudaMalloc(&h->res_pref, (E + 2) * 4));
-  FT_TRY(cudaMemset(h->res_pref, 0, (E + 2) * 4));
+  FT_TRY(cudaMalloc(&h->res_pref, (2 * E + 2) * 4));
+  FT_TRY(cudaMemset(h->res_pref, 0, (2 * E + 2) * 4));
   if (c.gemm_min_tokens > 0) {
     const size_t Pr = P + 128;   // one spare tile of rows so that full boxes stay inside the tensors
     FT_TRY(cudaMalloc(&h->gemm_pref, (E + 1) * 4));
@@ -695,10 +696,10 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   fp.x = static_cast<const __nv_bfloat16 *>(x_dev);
   fp.perm = h->perm; fp.topk_w = h->topk_w; fp.y_acc = h->y_acc;
   fp.d = c.hidden; fp.inter = c.inter; fp.top_k = c.top_k;
-  // zero-copy set first: it does not depend on the fills and shares the host link with them
-  fp.items = h->items_zc;
-  fp.n_items = &h->plan_dev->n_zc_items;
-  {
+  if (c.wdtype != FT_W_BF16) {
+    // zero-copy set first: it does not depend on the fills and shares the host link with them
+    fp.items = h->items_zc;
+    fp.n_items = &h->plan_dev->n_zc_items;
     TimeScope ts(h, st, FT_TIME_FFN_ZC);
     launch_stream_any(h, fp, L.T, st);
   }
@@ -710,8 +711,9 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     FfnMmaParams mp;
     mp.items = h->items_res;
     mp.n_items = &h->plan_dev->n_res_items;
+    mp.n_zc = &h->plan_dev->n_zc_items;
     mp.pref = h->res_pref;
-    mp.max_items = c.n_experts + 1;
+    mp.max_items = 2 * c.n_experts + 1;
     mp.x = fp.x; mp.perm = h->perm; mp.topk_w = h->topk_w; mp.y_acc = h->y_acc;
     mp.y = static_cast<__nv_bfloat16 *>(y_dev);
     mp.done = h->done_dev; mp.status = h->status_dev;

@@ -31,8 +31,9 @@ struct PlanParams {
   // outputs
   PlanHeader *hdr_dev;   // device plan record (header + 8 arrays of E)
   PlanHeader *hdr_host;  // mapped host mirror, or nullptr when the host does not read the plan
-  WorkItem *items_res;   // [E+1]  experts evaluated from slots by the streaming kernel
-  int32_t *res_pref;     // [E+2]  exclusive prefix of the weight passes of items_res
+  WorkItem *items_res;   // [2E+1] experts evaluated by the streaming kernel: from slots, then the shared
+                         //        expert, then the zero-copy experts (records in the mapped host pool)
+  int32_t *res_pref;     // [2E+2] exclusive prefix of the weight passes of items_res
   WorkItem *items_zc;    // [E]    experts evaluated from the mapped host pool
   WorkItem *items_gemm;  // [E]    experts evaluated from slots by the grouped GEMM
   int32_t *gemm_pref;    // [E+1]  exclusive prefix of the 128-row tiles of items_gemm
@@ -86,11 +87,9 @@ struct PlanSmem {
   uint8_t isfill[kMaxExperts];
   int32_t forder[kMaxExperts];
   int16_t miss[kMaxExperts];
+  int pairs_res;
 };
 
-// One plan step.  Thread `tid` < E owns expert `tid`: `c` = its token count, `off` = its offset in the
-// expert-sorted pair order, `n_pairs` = all pairs of the call.  blockDim.x >= E, a multiple of 32.
-// s_dyn: int64 stamp[n_slots]; int32 sexp[n_slots]; int32 victim[n_slots].
 // Issues every global read of the layer's state up front (step counter, this thread's expert_slot, the slot
 // table into shared memory) so their latencies overlap each other and whatever the caller does next.
 // A barrier must separate this from plan_body.
@@ -106,6 +105,9 @@ __device__ __forceinline__ void plan_prefetch(const PlanParams &p, unsigned char
   }
 }
 
+// One plan step.  Thread `tid` < E owns expert `tid`: `c` = its token count, `off` = its offset in the
+// expert-sorted pair order, `n_pairs` = all pairs of the call.  blockDim.x >= E, a multiple of 32.
+// s_dyn: int64 stamp[n_slots]; int32 sexp[n_slots]; int32 victim[n_slots] (filled by plan_prefetch).
 __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, unsigned char *s_dyn, int c, int off,
                                           int n_pairs, const int64_t t, const int slot_in) {
   int64_t *s_stamp = reinterpret_cast<int64_t *>(s_dyn);
@@ -134,6 +136,7 @@ __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, uns
     sm.elig[tid] = (uint8_t)elig;
     sm.isfill[tid] = 0;
   }
+  if (tid == 0) sm.pairs_res = 0;
   unsigned long long totA;
   const unsigned long long exA = block_excl_scan64(pack4(cls != 0, cls == 1, cls == 2, elig), sm.w, totA);
   const int n_routed = unpack(totA, 0), n_hit = unpack(totA, 1), n_miss = unpack(totA, 2), n_elig = unpack(totA, 3);
@@ -232,13 +235,19 @@ __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, uns
   const int resident = (cls == 1 || is_fill);
   const int use_gemm = resident && p.cm.gemm_min_tokens > 0 && c >= p.cm.gemm_min_tokens;
   const int res_stream = resident && !use_gemm;
+  if (resident) atomicAdd(&sm.pairs_res, c);   // a sum: order-free; read after the scans' barriers
   unsigned long long totB;
   const unsigned long long exB = block_excl_scan64(pack4(is_fill, is_zc, res_stream, use_gemm), sm.w, totB);
   const int n_fill = unpack(totB, 0), n_zc = unpack(totB, 1), n_res = unpack(totB, 2), n_gemm = unpack(totB, 3);
-  const int passes = res_stream ? (c + p.tokens_per_pass - 1) / p.tokens_per_pass : 0;
+  // weight passes (tokens_per_pass tokens each): low word for the resident streaming items, high word for the
+  // zero-copy items, which the streaming kernel finds appended to the same list
+  const int passes = (res_stream || is_zc) ? (c + p.tokens_per_pass - 1) / p.tokens_per_pass : 0;
   unsigned long long totC;
-  const unsigned long long exC =
-      block_excl_scan64(((unsigned long long)(resident ? c : 0) << 32) | (unsigned long long)passes, sm.w, totC);
+  const unsigned long long exC = block_excl_scan64(
+      ((unsigned long long)(is_zc ? passes : 0) << 32) | (unsigned long long)(res_stream ? passes : 0), sm.w, totC);
+  const int n_shared_items = (p.shared_rec != nullptr) ? 1 : 0;
+  const int shared_passes = n_shared_items ? (p.T + p.tokens_per_pass - 1) / p.tokens_per_pass : 0;
+  const int res_pass_total = (int)(totC & 0xffffffffull) + shared_passes;
   if (p.cm.gemm_min_tokens > 0) {   // uniform branch: only prefill-capable handles pay for this scan
     unsigned long long totD;
     const unsigned long long exD = block_excl_scan64(
@@ -275,24 +284,25 @@ __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, uns
     it.off = off;
     it.slot = -1;
     p.items_zc[unpack(exB, 1)] = it;
+    const int zi = n_res + n_shared_items + unpack(exB, 1);   // appended after the resident items
+    p.items_res[zi] = it;
+    p.res_pref[zi] = res_pass_total + (int32_t)(exC >> 32);
   }
 
   if (tid == 0) {
-    int n_res_items = n_res;
-    int pass_total = (int)(totC & 0xffffffffull);
-    if (p.shared_rec != nullptr) {
+    const int n_res_items = n_res + n_shared_items;
+    if (n_shared_items) {
       WorkItem it;
       it.w = p.shared_rec;
       it.expert = -1;
       it.n_tok = p.T;
       it.off = 0;
       it.slot = -1;
-      p.items_res[n_res_items] = it;
-      p.res_pref[n_res_items] = pass_total;
-      pass_total += (p.T + p.tokens_per_pass - 1) / p.tokens_per_pass;
-      ++n_res_items;
+      p.items_res[n_res] = it;
+      p.res_pref[n_res] = (int)(totC & 0xffffffffull);
     }
-    p.res_pref[n_res_items] = pass_total;
+    p.res_pref[n_res_items + n_zc] = res_pass_total + (int)(totC >> 32);
+    if (n_zc == 0) p.res_pref[n_res_items] = res_pass_total;
     PlanHeader h;
     h.step = t;
     h.n_routed = n_routed; h.n_hit = n_hit; h.n_miss = n_miss; h.n_fill = n_fill; h.n_zc = n_zc;
@@ -312,7 +322,7 @@ __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, uns
     atomicAdd(&p.stats[5], (unsigned long long)n_zc);
     atomicAdd(&p.stats[6], (unsigned long long)evictions);
     atomicAdd(&p.stats[7], (unsigned long long)n_pairs);
-    atomicAdd(&p.stats[8], (unsigned long long)(totC >> 32));
+    atomicAdd(&p.stats[8], (unsigned long long)sm.pairs_res);
   }
   // mirror the record into mapped host memory when the host reads the plan (copy-engine fills)
   if (p.hdr_host != nullptr) {
