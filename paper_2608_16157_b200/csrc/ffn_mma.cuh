@@ -196,100 +196,39 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
       const long long left = u1 - u;
       const int b_end = (left < (long long)(NBLK - b_begin)) ? b_begin + (int)left : NBLK;
       const WorkItem it = p.items[item];
-      const int nt = min(kMmaTokens, it.n_tok - kMmaTokens * pass);
-      // token g of this pass: row of x and gate weight
+      // Resident records: one group of up to 8 tokens per weight pass, accumulators live across the CTA's
+      // blocks of this pass.  Host-resident records cross the link once: every group of 8 tokens is served
+      // from the staged block before its stages are released, and the accumulators are flushed per block.
+      const bool host = (range == 1);
+      const int n_groups = host ? (it.n_tok + kMmaTokens - 1) / kMmaTokens : 1;
       int tok_g = -1;
       float gw_g = 0.f;
-      if (g < nt) {
-        if (it.expert >= 0) {
-          const int pr = p.perm[it.off + kMmaTokens * pass + g];
-          tok_g = pr / p.top_k;
-          gw_g = p.topk_w[pr];
-        } else {
-          tok_g = kMmaTokens * pass + g;
-          gw_g = 1.f;
-        }
-      }
       uint32_t xf[KB][4];
-#pragma unroll
-      for (int kb = 0; kb < KB; ++kb) {
-        uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (tok_g >= 0) v = *reinterpret_cast<const uint4 *>(p.x + (size_t)tok_g * d + kslice + 32 * kb + 8 * q);
-        xf[kb][0] = v.x; xf[kb][1] = v.y; xf[kb][2] = v.z; xf[kb][3] = v.w;
-      }
       float dacc[CTW][4];
-#pragma unroll
-      for (int c = 0; c < CTW; ++c) { dacc[c][0] = dacc[c][1] = dacc[c][2] = dacc[c][3] = 0.f; }
-
-      for (int b = b_begin; b < b_end; ++b) {
-        float cgu[2][4];
-#pragma unroll
-        for (int which = 0; which < 2; ++which) {
-          const int s = 2 * which + half;
-          const uint32_t ph = tile & 1u;
-          cgu[which][0] = cgu[which][1] = cgu[which][2] = cgu[which][3] = 0.f;
-          const bool ok = mbar_wait(full_bar(s), ph, s_abort, p.status);
-          if (ok) {
-            const uint32_t base = smem_base + s * stage_bytes + (uint32_t)(kl + 8 * q) * 2u;
-#pragma unroll
-            for (int kb = 0; kb < KB; ++kb) {
-              const uint4 lo = lds_v4(base + g * stride_gu + kb * 64);
-              const uint4 hi = lds_v4(base + (g + 8) * stride_gu + kb * 64);
-              mma_bf16(cgu[which], lo.x, hi.x, lo.y, hi.y, xf[kb][0], xf[kb][1]);
-              mma_bf16(cgu[which], lo.z, hi.z, lo.w, hi.w, xf[kb][2], xf[kb][3]);
-            }
+      auto load_group = [&](int grp) {   // token g of the group: row of x, gate weight, x fragments
+        const int nt = min(kMmaTokens, it.n_tok - kMmaTokens * grp);
+        tok_g = -1;
+        gw_g = 0.f;
+        if (g < nt) {
+          if (it.expert >= 0) {
+            const int pr = p.perm[it.off + kMmaTokens * grp + g];
+            tok_g = pr / p.top_k;
+            gw_g = p.topk_w[pr];
+          } else {
+            tok_g = kMmaTokens * grp + g;
+            gw_g = 1.f;
           }
-          __syncwarp();
-          if (lane == 0) mbar_arrive(empty_bar(s));
         }
-        // cross-warp reduction of the [16 neurons][8 tokens] partial sums
-        {
-          float *r0 = s_red + ((warp * 2 + 0) * 16) * 8;
-          float *r1 = s_red + ((warp * 2 + 1) * 16) * 8;
-          *reinterpret_cast<float2 *>(r0 + g * 8 + 2 * q) = make_float2(cgu[0][0], cgu[0][1]);
-          *reinterpret_cast<float2 *>(r0 + (g + 8) * 8 + 2 * q) = make_float2(cgu[0][2], cgu[0][3]);
-          *reinterpret_cast<float2 *>(r1 + g * 8 + 2 * q) = make_float2(cgu[1][0], cgu[1][1]);
-          *reinterpret_cast<float2 *>(r1 + (g + 8) * 8 + 2 * q) = make_float2(cgu[1][2], cgu[1][3]);
-        }
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        if (tid < 128) {
-          const int n = tid >> 3, t = tid & 7;
-          float a = 0.f, c = 0.f;
 #pragma unroll
-          for (int w = 0; w < 8; ++w) {
-            a += s_red[((w * 2 + 0) * 16 + n) * 8 + t];
-            c += s_red[((w * 2 + 1) * 16 + n) * 8 + t];
-          }
-          const float h = a / (1.f + __expf(-a)) * c;
-          s_h[t * 16 + n] = __float2bfloat16_rn(h);
+        for (int kb = 0; kb < KB; ++kb) {
+          uint4 v = make_uint4(0u, 0u, 0u, 0u);
+          if (tok_g >= 0) v = *reinterpret_cast<const uint4 *>(p.x + (size_t)tok_g * d + kslice + 32 * kb + 8 * q);
+          xf[kb][0] = v.x; xf[kb][1] = v.y; xf[kb][2] = v.z; xf[kb][3] = v.w;
         }
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        // down tile
-        {
-          const int s = 4 + half;
-          const uint32_t ph = tile & 1u;
-          const bool ok = mbar_wait(full_bar(s), ph, s_abort, p.status);
-          if (ok) {
-            const uint32_t *h32 = reinterpret_cast<const uint32_t *>(s_h);
-            const uint32_t b0 = h32[g * 8 + q], b1 = h32[g * 8 + q + 4];
-            // ldmatrix.x4.trans: lanes 0-7 / 8-15 / 16-23 / 24-31 address the four 8x8 blocks
-            const int mat = lane >> 3, r = lane & 7;
-            const uint32_t abase = smem_base + s * stage_bytes + (uint32_t)(r + 8 * (mat >> 1)) * stride_d +
-                                   (uint32_t)(kl + 8 * (mat & 1)) * 2u;
 #pragma unroll
-            for (int c = 0; c < CTW; ++c) {
-              uint32_t a[4];
-              ldmatrix_x4_trans(a, abase + c * 32);
-              mma_bf16(dacc[c], a[0], a[1], a[2], a[3], b0, b1);
-            }
-          }
-          __syncwarp();
-          if (lane == 0) mbar_arrive(empty_bar(s));
-          ++tile;
-        }
-      }
-      // gate-weighted combine: D fragment = [column g / g+8 of the tile][tokens 2q, 2q+1]
-      {
+        for (int c = 0; c < CTW; ++c) { dacc[c][0] = dacc[c][1] = dacc[c][2] = dacc[c][3] = 0.f; }
+      };
+      auto flush = [&]() {   // gate-weighted combine: D fragment = [column g / g+8 of the tile][tokens 2q, 2q+1]
         const int tok_a = __shfl_sync(0xffffffffu, tok_g, (2 * q) * 4);
         const int tok_b = __shfl_sync(0xffffffffu, tok_g, (2 * q + 1) * 4);
         const float gw_a = __shfl_sync(0xffffffffu, gw_g, (2 * q) * 4);
@@ -306,7 +245,80 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
             atomicAdd(p.y_acc + (size_t)tok_b * d + col + 8, gw_b * dacc[c][3]);
           }
         }
+      };
+      if (!host) load_group(pass);
+
+      for (int b = b_begin; b < b_end; ++b, ++tile) {
+        const uint32_t ph = tile & 1u;
+        for (int grp = 0; grp < n_groups; ++grp) {
+          const bool last = (grp == n_groups - 1);
+          if (host) load_group(grp);
+          float cgu[2][4];
+#pragma unroll
+          for (int which = 0; which < 2; ++which) {
+            const int s = 2 * which + half;
+            cgu[which][0] = cgu[which][1] = cgu[which][2] = cgu[which][3] = 0.f;
+            const bool ok = mbar_wait(full_bar(s), ph, s_abort, p.status);
+            if (ok) {
+              const uint32_t base = smem_base + s * stage_bytes + (uint32_t)(kl + 8 * q) * 2u;
+#pragma unroll
+              for (int kb = 0; kb < KB; ++kb) {
+                const uint4 lo = lds_v4(base + g * stride_gu + kb * 64);
+                const uint4 hi = lds_v4(base + (g + 8) * stride_gu + kb * 64);
+                mma_bf16(cgu[which], lo.x, hi.x, lo.y, hi.y, xf[kb][0], xf[kb][1]);
+                mma_bf16(cgu[which], lo.z, hi.z, lo.w, hi.w, xf[kb][2], xf[kb][3]);
+              }
+            }
+            __syncwarp();
+            if (last && lane == 0) mbar_arrive(empty_bar(s));
+          }
+          // cross-warp reduction of the [16 neurons][8 tokens] partial sums
+          {
+            float *r0 = s_red + ((warp * 2 + 0) * 16) * 8;
+            float *r1 = s_red + ((warp * 2 + 1) * 16) * 8;
+            *reinterpret_cast<float2 *>(r0 + g * 8 + 2 * q) = make_float2(cgu[0][0], cgu[0][1]);
+            *reinterpret_cast<float2 *>(r0 + (g + 8) * 8 + 2 * q) = make_float2(cgu[0][2], cgu[0][3]);
+            *reinterpret_cast<float2 *>(r1 + g * 8 + 2 * q) = make_float2(cgu[1][0], cgu[1][1]);
+            *reinterpret_cast<float2 *>(r1 + (g + 8) * 8 + 2 * q) = make_float2(cgu[1][2], cgu[1][3]);
+          }
+          asm volatile("bar.sync 1, 256;" ::: "memory");
+          if (tid < 128) {
+            const int n = tid >> 3, t = tid & 7;
+            float a = 0.f, c = 0.f;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) {
+              a += s_red[((w * 2 + 0) * 16 + n) * 8 + t];
+              c += s_red[((w * 2 + 1) * 16 + n) * 8 + t];
+            }
+            const float h = a / (1.f + __expf(-a)) * c;
+            s_h[t * 16 + n] = __float2bfloat16_rn(h);
+          }
+          asm volatile("bar.sync 1, 256;" ::: "memory");
+          // down tile
+          {
+            const int s = 4 + half;
+            const bool ok = mbar_wait(full_bar(s), ph, s_abort, p.status);
+            if (ok) {
+              const uint32_t *h32 = reinterpret_cast<const uint32_t *>(s_h);
+              const uint32_t b0 = h32[g * 8 + q], b1 = h32[g * 8 + q + 4];
+              // ldmatrix.x4.trans: lanes 0-7 / 8-15 / 16-23 / 24-31 address the four 8x8 blocks
+              const int mat = lane >> 3, r = lane & 7;
+              const uint32_t abase = smem_base + s * stage_bytes + (uint32_t)(r + 8 * (mat >> 1)) * stride_d +
+                                     (uint32_t)(kl + 8 * (mat & 1)) * 2u;
+#pragma unroll
+              for (int c = 0; c < CTW; ++c) {
+                uint32_t a[4];
+                ldmatrix_x4_trans(a, abase + c * 32);
+                mma_bf16(dacc[c], a[0], a[1], a[2], a[3], b0, b1);
+              }
+            }
+            __syncwarp();
+            if (last && lane == 0) mbar_arrive(empty_bar(s));
+          }
+          if (host) flush();
+        }
       }
+      if (!host) flush();
       u += (b_end - b_begin);
     }
     }
