@@ -485,9 +485,81 @@ def run_prefill(args):
     pool.free()
 
 
+def run_sweep(args):
+    """Cache-pressure sweep on the decode shapes: cache fraction x locality rho x batch, `--sweep-steps` steps
+    each from an empty cache.  One JSON line with a record per point."""
+    import torch
+    from paper_2608_16157_b200 import binding as Bd
+    from paper_2608_16157_b200 import workload as W
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    shape = W.QWEN3_30B
+    L, E, k, d = args.layers, shape.n_experts, shape.top_k, shape.d
+    S = shape.expert_bytes
+    steps = args.sweep_steps
+    pool = Bd.HostPool(L * E * S)
+    W.fill_pool(pool.tensor, shape, L, SEED, device=dev, chunk=32)
+    stream = torch.cuda.current_stream()
+    points = []
+    xbuf = torch.empty((L, 64, d), dtype=torch.bfloat16, device=dev)
+    ybuf = torch.empty((L, 64, d), dtype=torch.bfloat16, device=dev)
+    cal = None
+    for frac in (0.10, 0.25, 0.50, 0.75, 1.00):
+        Ns = W.slots_for_fraction(frac, E)
+        common = dict(hidden=d, inter=shape.inter, n_experts=E, top_k=k, n_layers=L, slots_per_layer=Ns,
+                      max_tokens=64, host_pool_ptr=pool.ptr.value, host_pool_bytes=pool.n_bytes,
+                      fill_mode=Bd.FT_FILL_SM if args.fill == "sm" else Bd.FT_FILL_COPY_ENGINE)
+        if cal is None:
+            m0 = Bd.FtMoe(Bd.make_config(**common))
+            cal = m0.calibrate()
+            m0.destroy()
+        moe = Bd.FtMoe(Bd.make_config(bw_fill=max(cal["fill_MBps"], 1), bw_zc=max(cal["zc_MBps"], 1),
+                                      bw_zc_residual=0, bw_hbm=max(cal["hbm_MBps"], 1), **common))
+        for rho in (0.0, 0.5, 0.9):
+            for batch in (1, 16, 64):
+                lg = torch.from_numpy(W.ar1_logits(L, steps, batch, E, rho, ALPHA, SEED)).to(dev)
+                g = torch.Generator(device=dev)
+                g.manual_seed(W.mix64(SEED, 79, batch))
+                noise = torch.randn((steps, L, batch, d), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+                moe.reset()
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                for s_ in range(steps):
+                    for l in range(L):
+                        if l == 0:
+                            x = noise[s_, 0]
+                        else:
+                            x = xbuf[l, :batch]
+                            torch.add(noise[s_, l], ybuf[l - 1, :batch], out=x)
+                        moe.layer(l, lg[s_, l], x, ybuf[l, :batch], batch, stream)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                ms = e0.elapsed_time(e1)
+                st = {kk: sum(moe.get_stats(l)[kk] for l in range(L)) for kk in Bd.STAT_NAMES}
+                pt = {"cache_frac": frac, "slots": Ns, "rho": rho, "batch": batch, "steps": steps,
+                      "tok_per_s": batch * steps / (ms * 1e-3), "ms_per_step": ms / steps,
+                      "hit_rate_unique": st["hits"] / max(st["routed"], 1),
+                      "hit_rate_pairs": st["pairs_resident"] / max(st["pairs"], 1),
+                      "fills": st["fills"], "zero_copies": st["zc"], "evictions": st["evictions"],
+                      "fill_bytes": st["fills"] * S, "zero_copy_bytes": st["zc"] * S,
+                      "routed_unique_per_layer_step": st["routed"] / (steps * L)}
+                points.append(pt)
+                log(f"sweep {pt}")
+        moe.destroy()
+    line = {"metric": "moe_decode_sweep", "unit": "tok/s", "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "cache-pressure sweep on the decode shapes (config 4)", "layers": L,
+                       "hidden": d, "experts": E, "inter": shape.inter, "top_k": k, "fill_mode": args.fill,
+                       "zipf_alpha": ALPHA, "steps_per_point": steps, "cold_start": True},
+            "link_GBps_measured": cal["fill_MBps"] / 1e3, "points": points}
+    print(json.dumps(line), flush=True)
+    pool.free()
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--mode", default="decode", choices=["decode", "prefill"])
+    ap.add_argument("--sweep-steps", type=int, default=128)
+    ap.add_argument("--mode", default="decode", choices=["decode", "prefill", "sweep"])
     ap.add_argument("--tokens", type=int, default=4096)
     ap.add_argument("--gemm-min-tokens", type=int, default=32)
     ap.add_argument("--gpus", type=int, default=1)
@@ -509,6 +581,8 @@ def main():
         run_reference(args)
     elif args.mode == "prefill":
         run_prefill(args)
+    elif args.mode == "sweep":
+        run_sweep(args)
     else:
         run_ours(args)
 

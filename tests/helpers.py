@@ -21,12 +21,15 @@ class Pair:
     """A CUDA handle and per-layer oracles over the same pinned pool."""
 
     def __init__(self, shape: W.LayerShape, n_slots: int, max_tokens: int, n_layers: int = 1, seed: int = 0,
-                 fill_mode: int = B.FT_FILL_COPY_ENGINE, gen_device="cpu", **cost):
+                 fill_mode: int = B.FT_FILL_COPY_ENGINE, gen_device="cpu", pool=None, **cost):
         self.shape, self.n_slots, self.L = shape, n_slots, n_layers
         S = shape.expert_bytes
         self.S = S
-        self.pool = B.HostPool(n_layers * shape.n_experts * S)
-        W.fill_pool(self.pool.tensor, shape, n_layers, seed, device=gen_device)
+        self.owns_pool = pool is None
+        if pool is None:
+            pool = B.HostPool(n_layers * shape.n_experts * S)
+            W.fill_pool(pool.tensor, shape, n_layers, seed, device=gen_device)
+        self.pool = pool
         self.shared = None
         if shape.n_shared:
             self.shared = W.make_shared_records(shape, n_layers, seed, device=gen_device)
@@ -50,7 +53,8 @@ class Pair:
 
     def close(self):
         self.moe.destroy()
-        self.pool.free()
+        if self.owns_pool:
+            self.pool.free()
 
     def step(self, layer: int, logits: np.ndarray, x: torch.Tensor, check_y: bool = True,
              check_slots: bool = False, fused: bool = False):
