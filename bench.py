@@ -181,15 +181,19 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    shape = W.QWEN3_30B
-    L, E, k, d = args.layers, shape.n_experts, shape.top_k, shape.d
+    dsv3 = args.workload == "dsv3"
+    shape = W.DSV3_INT4 if dsv3 else W.QWEN3_30B
+    RHO, ALPHA = (0.9, 1.2) if dsv3 else (0.8, 1.1)
+    L = (4 if args.layers == 48 else args.layers) if dsv3 else args.layers
+    E, k, d = shape.n_experts, shape.top_k, shape.d
     S = shape.expert_bytes
-    Ns = W.slots_for_fraction(args.cache_frac, E)
-    B = args.batch
+    Ns = 64 if dsv3 else W.slots_for_fraction(args.cache_frac, E)
+    B = (4 if args.batch == 8 else args.batch) if dsv3 else args.batch
     Wn, K = args.warmup, args.steps
     t_setup = time.perf_counter()
     pool = Bd.HostPool(L * E * S)
     W.fill_pool(pool.tensor, shape, L, SEED, device=dev, chunk=32)
+    shared = W.make_shared_records(shape, L, SEED, device=dev) if shape.n_shared else None
     log(f"[rank {rank}] pool {L * E * S / 2**30:.1f} GiB pinned+filled in {time.perf_counter() - t_setup:.1f}s")
 
     fill_mode = Bd.FT_FILL_SM if args.fill == "sm" else Bd.FT_FILL_COPY_ENGINE
@@ -197,7 +201,9 @@ def run_ours(args):
     def make(bw):
         cfg = Bd.make_config(hidden=d, inter=shape.inter, n_experts=E, top_k=k, n_layers=L, slots_per_layer=Ns,
                              max_tokens=max(B, 8), host_pool_ptr=pool.ptr.value, host_pool_bytes=pool.n_bytes,
-                             fill_mode=fill_mode, device=local, **bw)
+                             fill_mode=fill_mode, device=local,
+                             wdtype=Bd.FT_W_INT4_G128 if shape.wdtype == "int4" else Bd.FT_W_BF16,
+                             n_shared=shape.n_shared, shared_ptr=None if shared is None else shared.data_ptr(), **bw)
         return Bd.FtMoe(cfg)
 
     # bandwidth profiling at deployment, then frozen into the plan's cost model
@@ -266,7 +272,7 @@ def run_ours(args):
         return tot
 
     results = {}
-    for batch in ([B] if args.only_batch else [B, 1] if B != 1 else [1]):
+    for batch in ([B] if (args.only_batch or dsv3) else [B, 1] if B != 1 else [1]):
         lg, noise = gen_inputs(batch)
         moe.reset()
         for s in range(Wn):
@@ -284,7 +290,8 @@ def run_ours(args):
         tim = moe.timing_read()
         st3 = stats_sum()
         moe.timing_enable(False)
-        res_bytes = (st3["hits"] - st2["hits"] + st3["fills"] - st2["fills"]) * S
+        res_bytes = (st3["hits"] - st2["hits"] + st3["fills"] - st2["fills"] +
+                     shape.n_shared * (st3["steps"] - st2["steps"])) * S
         results[batch] = dict(ms=ms, clocks=clocks, launches=launches, dstats=dst, timing=tim,
                               res_bytes=res_bytes, prof_fill_bytes=(st3["fills"] - st2["fills"]) * S,
                               lg=lg, noise=noise)
@@ -297,6 +304,8 @@ def run_ours(args):
     hbm_peak, peak_kind = peaks()
     tim = main["timing"]
     ffn_us, ffn_n = tim["ffn_res"]
+    if dsv3:   # the int4 path streams a record with two kernels: gate/up (timed in the ffn_zc slot) + down
+        ffn_us += tim["ffn_zc"][0]
     achieved = main["res_bytes"] / (ffn_us * 1e-6) / 1e9 if ffn_us > 0 else 0.0
     fill_us, fill_n = tim["fill"]
 
@@ -356,17 +365,20 @@ def run_ours(args):
         line = {
             "metric": "moe_decode_tok_per_s", "value": value, "unit": "tok/s", "n_gpus": world, "steps": K,
             "warmup": Wn, "ms_per_step": main["ms"] / K, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "decode Qwen3-30B-A3B-shaped MoE stack (config 1)", "batch": B, "layers": L,
+            "vs_baseline": None, "dtype": "int4 weights, bf16 activations, fp32 accumulate" if dsv3 else "bf16",
+            "data": "synthetic",
+            "config": {"workload": ("decode DeepSeek-V3-shaped int4 MoE stack (config 3)" if dsv3 else
+                                    "decode Qwen3-30B-A3B-shaped MoE stack (config 1)"), "batch": B, "layers": L,
                        "hidden": d, "experts": E, "inter": shape.inter, "top_k": k, "slots_per_layer": Ns,
                        "fill_mode": args.fill, "rho": RHO, "zipf_alpha": ALPHA,
-                       "l2": "inputs larger than L2: each step streams >= 3.4 GB of distinct expert records "
-                             "from a 27 GiB slot pool, no L2 flush needed",
+                       "l2": "inputs larger than L2: every step streams GBs of distinct expert records from the slot "
+                             "pool, far beyond the 126 MB L2; no flush needed",
                        "parallelism": "replicas" if world > 1 else "single"},
             "clocks": main["clocks"],
             "e2e": e2e,
             "gpu_launches": main["launches"],
-            "roofline": {"bound": "hbm", "kernel": "ffn_stream_kernel (resident experts)",
+            "roofline": {"bound": "hbm", "kernel": ("q4_gateup_kernel + q4_down_kernel (one pass over each record)" if dsv3
+                                                   else "ffn_mma_kernel (resident experts)"),
                          "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
                          "frac": achieved / hbm_peak if hbm_peak else None, "peak_source": peak_kind,
                          "launches_timed": ffn_n, "avg_launch_us": ffn_us / ffn_n if ffn_n else None,
@@ -559,6 +571,7 @@ def run_sweep(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--sweep-steps", type=int, default=128)
+    ap.add_argument("--workload", default="qwen", choices=["qwen", "dsv3"])
     ap.add_argument("--mode", default="decode", choices=["decode", "prefill", "sweep"])
     ap.add_argument("--tokens", type=int, default=4096)
     ap.add_argument("--gemm-min-tokens", type=int, default=32)

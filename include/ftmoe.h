@@ -201,6 +201,8 @@ ft_status_t ft_moe_timing_read(ft_moe_t *h, double *out_us, uint64_t *out_launch
 /* Number of kernels this handle has launched since create. */
 ft_status_t ft_moe_launch_count(ft_moe_t *h, uint64_t *out);
 const char *ft_moe_status_string(ft_status_t s);
+/* Text of the CUDA runtime error behind the most recent FT_ERR_CUDA / FT_ERR_OOM of this process. */
+const char *ft_moe_last_cuda_error(void);
 
 /* An expert FFN for callers that are not allowed to allocate.  (The paper has no counterpart: this
  * is a convenience of this library.)

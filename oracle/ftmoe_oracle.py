@@ -242,10 +242,13 @@ def unpack_record(rec: np.ndarray, d: int, inter: int, wdtype: str):
 
     bf16 record: three row-major [I][d] bf16 matrices (gate and up stored transposed,
     i.e. one row per intermediate neuron), then nothing.
-    int4 record: the same three [I][d] matrices as 4-bit two's-complement codes, two per
-    byte along d (low nibble = even column), followed by bf16 scales sg[I][d/128],
-    su[I][d/128] (groups along the hidden index) and sd[I/128][d] (groups along the
-    neuron index); weight = scale * code.
+    int4 record: 4-bit two's-complement codes, then bf16 scales sg[I][d/128], su[I][d/128]
+    (groups along the hidden index) and sd[I/128][d] (groups along the neuron index);
+    weight = scale * code.  Gate and up codes are row-major [I][d/2] bytes, two per byte along
+    d (low nibble = even column).  Down codes are stored in fragment order: 16-neuron blocks x
+    16-column tiles x 32 little-endian 32-bit words; in word l = 4g + q of block b, tile ct,
+    nibble j is the code of neuron 16b + NN[j] + q, column 16ct + CC[j] + g, with
+    NN = (0,8,0,8,4,12,4,12) and CC = (0,0,8,8,0,0,8,8).
     """
     rec = np.ascontiguousarray(rec).view(np.uint8).reshape(-1)
     n = inter * d
@@ -256,7 +259,7 @@ def unpack_record(rec: np.ndarray, d: int, inter: int, wdtype: str):
     if wdtype == "int4":
         nb = n // 2
         codes = []
-        for which in range(3):
+        for which in range(2):
             b = rec[which * nb:(which + 1) * nb].reshape(inter, d // 2)
             lo = (b & 0xF).astype(np.int16)
             hi = (b >> 4).astype(np.int16)
@@ -265,6 +268,17 @@ def unpack_record(rec: np.ndarray, d: int, inter: int, wdtype: str):
             q[:, 1::2] = hi
             q = np.where(q >= 8, q - 16, q)
             codes.append(q.astype(np.float64))
+        # down: walk the fragment-order words
+        words = rec[2 * nb:3 * nb].view("<u4").reshape(inter // 16, d // 16, 32)
+        qd = np.zeros((inter, d), dtype=np.int16)
+        NN, CC = (0, 8, 0, 8, 4, 12, 4, 12), (0, 0, 8, 8, 0, 0, 8, 8)
+        for l in range(32):
+            g_, q_ = l // 4, l % 4
+            for j in range(8):
+                nib = ((words[:, :, l] >> np.uint32(4 * j)) & np.uint32(0xF)).astype(np.int16)
+                qd[NN[j] + q_::16, CC[j] + g_::16] = nib
+        qd = np.where(qd >= 8, qd - 16, qd)
+        codes.append(qd.astype(np.float64))
         off = 3 * nb
         ng = inter * (d // GROUP)
         sg = _bf16_bits_to_f64(rec[off:off + 2 * ng].view(np.uint16)).reshape(inter, d // GROUP)

@@ -27,6 +27,7 @@ SYMBOLS = (
     "ft_moe_layer_host", "ft_moe_get_routing", "ft_moe_get_slot_table", "ft_moe_read_slot",
     "ft_moe_get_stats", "ft_moe_reset", "ft_moe_sync_status", "ft_moe_last_fill", "ft_moe_launch_count",
     "ft_moe_status_string", "ft_moe_timing_enable", "ft_moe_timing_read", "ft_moe_ffn_noalloc",
+    "ft_moe_last_cuda_error",
 )
 NOALLOC_MAX_TOKENS, NOALLOC_MAX_HIDDEN = 64, 2048
 TIME_NAMES = ("route", "plan", "ffn_zc", "ffn_res", "finalize", "fill", "gather", "gemm1", "gemm2", "combine")
@@ -58,7 +59,10 @@ class PlanOut(C.Structure):
 class FtMoeError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
-        super().__init__(f"{where}: {status_string(code)} ({code})")
+        detail = ""
+        if code in (FT_ERR_CUDA, FT_ERR_OOM):
+            detail = " [" + load().ft_moe_last_cuda_error().decode() + "]"
+        super().__init__(f"{where}: {status_string(code)} ({code}){detail}")
 
 
 _lib = None
@@ -99,6 +103,7 @@ def load(rebuild: bool = False):
         "ft_moe_timing_enable": (i32, [vp, i32]),
         "ft_moe_timing_read": (i32, [vp, vp, vp, i32]),
         "ft_moe_ffn_noalloc": (i32, [i32, vp, i32, i32, vp, vp, i32, vp]),
+        "ft_moe_last_cuda_error": (C.c_char_p, []),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)

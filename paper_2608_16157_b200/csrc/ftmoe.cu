@@ -10,7 +10,7 @@
 
 #include "common.cuh"
 #include "ffn_mma.cuh"
-#include "ffn_stream.cuh"
+#include "ffn_q4.cuh"
 #include "gemm_tc.cuh"
 #include "fill.cuh"
 #include "route_plan.cuh"
@@ -64,6 +64,7 @@ struct ft_moe {
   uint32_t *status_dev = nullptr;
   uint32_t *seq_dev = nullptr;
   uint32_t *done_dev = nullptr;          // CTA completion counter of the streaming MMA kernel
+  uint2 *q4_hbuf = nullptr;              // int4 path: h of every (pass, 16-neuron block) in fragment order
   uint32_t seq_host = 0;                // plans launched
   float *stage_logits = nullptr;
   __nv_bfloat16 *stage_x = nullptr, *stage_y = nullptr;
@@ -86,10 +87,13 @@ struct ft_moe {
 
 namespace {
 
+cudaError_t g_last_cuda_error = cudaSuccess;   // the CUDA error behind the latest FT_ERR_CUDA / FT_ERR_OOM
+
 #define FT_CUDA(expr)                                                                     \
   do {                                                                                    \
     cudaError_t e_ = (expr);                                                              \
     if (e_ != cudaSuccess) {                                                              \
+      g_last_cuda_error = e_;                                                             \
       if (e_ == cudaErrorMemoryAllocation) { (void)cudaGetLastError(); return FT_ERR_OOM; } \
       return FT_ERR_CUDA;                                                                 \
     }                                                                                     \
@@ -103,26 +107,16 @@ size_t expert_bytes_of(const ft_moe_config_t *c) {
     return 3 * I * d * 2;
   }
   if (c->wdtype == FT_W_INT4_G128) {
-    if (d % 512 || d > 8192 || I % 128) return 0;
+    if (d % 512 || d > 8192 || I % 128) return 0;   // (the kernels further restrict d, see q4_shape_ok)
     return 3 * I * d / 2 + (2 * I * (d / 128) + (I / 128) * d) * 2;
   }
   return 0;
 }
 
-// threads across a row, row groups, threads per CTA of the streaming kernel
-void stream_geometry(const ft_moe_config_t &c, int &CT, int &G) {
-  const int epl = (c.wdtype == FT_W_BF16) ? 8 : 16;
-  CT = c.hidden / epl;
-  G = (CT >= 256) ? 1 : 256 / CT;
-}
-
-bool geometry_ok(const ft_moe_config_t &c) {
-  int CT, G;
-  stream_geometry(c, CT, G);
-  if (CT % 32 || CT > (c.wdtype == FT_W_BF16 ? 256 : 512)) return false;
-  if (CT < 256 && (256 % CT)) return false;
-  if (c.inter % (8 * G)) return false;
-  return true;
+// shapes the int4 kernels are instantiated for
+bool q4_shape_ok(const ft_moe_config_t &c) {
+  const int d = c.hidden;
+  return (d == 512 || d == 1024 || d == 2048 || d == 4096 || d == 7168 || d == 8192) && c.inter % 128 == 0;
 }
 
 ft_status_t drain_status(ft_moe *h) {
@@ -199,28 +193,6 @@ ft_status_t reset_layer(ft_moe *h, int l) {
   return FT_OK;
 }
 
-template <int WD, int TC, int NR>
-void launch_stream(ft_moe *h, const FfnParams &fp, int threads, int grid, cudaStream_t st) {
-  ffn_stream_kernel<WD, TC, NR><<<grid, threads, 0, st>>>(fp);
-  h->launches++;
-}
-
-void launch_stream_any(ft_moe *h, const FfnParams &fp, int T, cudaStream_t st) {
-  int CT, G;
-  stream_geometry(h->cfg, CT, G);
-  const int threads = CT * G;
-  const int grid = h->sm_count * ((threads <= 256) ? 2 : 1);
-  if (h->cfg.wdtype == FT_W_BF16) {
-    if (T <= 1) launch_stream<0, 1, 8>(h, fp, threads, grid, st);
-    else if (T <= 2) launch_stream<0, 2, 4>(h, fp, threads, grid, st);
-    else if (T <= 4) launch_stream<0, 4, 4>(h, fp, threads, grid, st);
-    else launch_stream<0, 8, 2>(h, fp, threads, grid, st);
-  } else {
-    if (T <= 1) launch_stream<1, 1, 8>(h, fp, threads, grid, st);
-    else launch_stream<1, 2, 4>(h, fp, threads, grid, st);
-  }
-}
-
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -242,6 +214,8 @@ bool make_tensor_map(EncodeTiledFn fn, CUtensorMap *tm, void *base, uint64_t row
 extern "C" {
 
 size_t ft_moe_expert_bytes(const ft_moe_config_t *cfg) { return expert_bytes_of(cfg); }
+
+const char *ft_moe_last_cuda_error(void) { return cudaGetErrorString(g_last_cuda_error); }
 
 const char *ft_moe_status_string(ft_status_t s) {
   switch (s) {
@@ -303,6 +277,7 @@ ft_status_t ft_moe_destroy(ft_moe_t *h) {
   cudaFree(h->status_dev);
   cudaFree(h->seq_dev);
   cudaFree(h->done_dev);
+  cudaFree(h->q4_hbuf);
   cudaFree(h->stage_logits);
   cudaFree(h->stage_x);
   cudaFree(h->stage_y);
@@ -333,7 +308,7 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
       c.zc_tokens_per_pass < 1 || c.hbm_tokens_per_pass < 1 || c.gemm_min_tokens < 0)
     return FT_ERR_INVALID_ARG;
   const size_t S = expert_bytes_of(cfg);
-  if (S == 0 || !geometry_ok(c)) return FT_ERR_UNSUPPORTED;
+  if (S == 0 || (c.wdtype == FT_W_INT4_G128 && !q4_shape_ok(c))) return FT_ERR_UNSUPPORTED;
   if (c.gemm_min_tokens != 0 &&
       (c.wdtype != FT_W_BF16 || c.slots_per_layer == 0 || c.hidden % 256 || c.inter % 128 || c.gemm_min_tokens < 8))
     return FT_ERR_UNSUPPORTED;
@@ -457,6 +432,22 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
     FT_TRY(cudaFuncSetAttribute(plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn));
     FT_TRY(cudaFuncSetAttribute(route_plan_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn));
   }
+  if (c.wdtype == FT_W_INT4_G128) {
+    const size_t passes = (P + 7) / 8 + 2 * E + 2;
+    FT_TRY(cudaMalloc(&h->q4_hbuf, passes * (c.inter / 16) * 32 * sizeof(uint2)));
+    const int sa = (int)q4_gateup_smem_bytes(c.hidden), sb = (int)q4_down_smem_bytes(c.hidden);
+    FT_TRY(cudaFuncSetAttribute(q4_gateup_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(q4_gateup_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(q4_gateup_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(q4_gateup_kernel<7>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(q4_gateup_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(q4_down_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
+    FT_TRY(cudaFuncSetAttribute(q4_down_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
+    FT_TRY(cudaFuncSetAttribute(q4_down_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
+    FT_TRY(cudaFuncSetAttribute(q4_down_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
+    FT_TRY(cudaFuncSetAttribute(q4_down_kernel<28>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
+    FT_TRY(cudaFuncSetAttribute(q4_down_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
+  }
   if (c.wdtype == FT_W_BF16) {
     const int smem = (int)ffn_mma_smem_bytes(c.hidden);
     FT_TRY(cudaFuncSetAttribute(ffn_mma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
@@ -536,6 +527,7 @@ static PlanParams make_plan_params(ft_moe *h, int layer, bool mirror_to_host) {
   pp.shared_rec = c.n_shared ? h->shared_dev + (size_t)layer * h->S : nullptr;
   pp.S = h->S; pp.T = L.T;
   pp.tokens_per_pass = kMmaTokens;
+  pp.zc_single_pass = (c.wdtype == FT_W_BF16) ? 1 : 0;
   pp.hdr_dev = h->plan_dev;
   pp.hdr_host = mirror_to_host ? h->plan_host_devptr : nullptr;
   pp.items_res = h->items_res; pp.res_pref = h->res_pref;
@@ -692,17 +684,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   if (!x_dev || !y_dev) return FT_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const ft_moe_config_t &c = h->cfg;
-  FfnParams fp;
-  fp.x = static_cast<const __nv_bfloat16 *>(x_dev);
-  fp.perm = h->perm; fp.topk_w = h->topk_w; fp.y_acc = h->y_acc;
-  fp.d = c.hidden; fp.inter = c.inter; fp.top_k = c.top_k;
-  if (c.wdtype != FT_W_BF16) {
-    // zero-copy set first: it does not depend on the fills and shares the host link with them
-    fp.items = h->items_zc;
-    fp.n_items = &h->plan_dev->n_zc_items;
-    TimeScope ts(h, st, FT_TIME_FFN_ZC);
-    launch_stream_any(h, fp, L.T, st);
-  }
+  const __nv_bfloat16 *x_bf = static_cast<const __nv_bfloat16 *>(x_dev);
   // resident set after the fills have landed
   if (c.slots_per_layer > 0) FT_CUDA(cudaStreamWaitEvent(st, h->ev_fill, 0));
   const bool use_gemm = h->gemm && L.T >= c.gemm_min_tokens;
@@ -714,7 +696,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     mp.n_zc = &h->plan_dev->n_zc_items;
     mp.pref = h->res_pref;
     mp.max_items = 2 * c.n_experts + 1;
-    mp.x = fp.x; mp.perm = h->perm; mp.topk_w = h->topk_w; mp.y_acc = h->y_acc;
+    mp.x = x_bf; mp.perm = h->perm; mp.topk_w = h->topk_w; mp.y_acc = h->y_acc;
     mp.y = static_cast<__nv_bfloat16 *>(y_dev);
     mp.done = h->done_dev; mp.status = h->status_dev;
     mp.d = c.hidden; mp.inter = c.inter; mp.top_k = c.top_k; mp.T = L.T; mp.finalize = use_gemm ? 0 : 1;
@@ -734,7 +716,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
       // experts with many tokens: gather x rows into expert order, two grouped tcgen05 GEMMs, fused combine
       {
         TimeScope ts(h, st, FT_TIME_GATHER);
-        gather_rows_kernel<<<h->sm_count * 8, 256, 0, st>>>(fp.x, h->perm, c.top_k, c.hidden, h->offset + c.n_experts, h->xs);
+        gather_rows_kernel<<<h->sm_count * 8, 256, 0, st>>>(x_bf, h->perm, c.top_k, c.hidden, h->offset + c.n_experts, h->xs);
       }
       GemmParams gp;
       gp.items = h->items_gemm; gp.n_items = &h->plan_dev->n_gemm_items; gp.mt_pref = h->gemm_pref;
@@ -762,18 +744,43 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     }
     return FT_OK;
   }
-  if (c.slots_per_layer > 0 || c.n_shared) {
-    fp.items = h->items_res;
-    fp.n_items = &h->plan_dev->n_res_items;
-    TimeScope ts(h, st, FT_TIME_FFN_RES);
-    launch_stream_any(h, fp, L.T, st);
-  }
-  const long long n4 = (long long)L.T * c.hidden / 4;
+  // int4: gate/up kernel writes h, down kernel accumulates, its last CTA finalizes y
+  Q4Params qp;
+  qp.items = h->items_res;
+  qp.n_items = &h->plan_dev->n_res_items;
+  qp.n_zc = &h->plan_dev->n_zc_items;
+  qp.pref = h->res_pref;
+  qp.max_items = 2 * c.n_experts + 1;
+  qp.x = x_bf; qp.perm = h->perm; qp.topk_w = h->topk_w;
+  qp.hbuf = h->q4_hbuf;
+  qp.y_acc = h->y_acc; qp.y = static_cast<__nv_bfloat16 *>(y_dev);
+  qp.done = h->done_dev; qp.status = h->status_dev;
+  qp.d = c.hidden; qp.inter = c.inter; qp.top_k = c.top_k; qp.T = L.T; qp.finalize = 1;
+  const size_t sa = q4_gateup_smem_bytes(c.hidden), sb = q4_down_smem_bytes(c.hidden);
+  const int grid = h->sm_count & ~1;   // CTA pairs split the columns in the down kernel
   {
-    TimeScope ts(h, st, FT_TIME_FINALIZE);
-    finalize_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(h->y_acc, static_cast<__nv_bfloat16 *>(y_dev), n4);
+    TimeScope ts(h, st, FT_TIME_FFN_ZC);   // (timing slot reused for the gate/up kernel of the int4 path)
+    switch (c.hidden) {
+      case 512: q4_gateup_kernel<1><<<grid, kQ4Threads, sa, st>>>(qp); break;
+      case 1024: q4_gateup_kernel<1><<<grid, kQ4Threads, sa, st>>>(qp); break;
+      case 2048: q4_gateup_kernel<2><<<grid, kQ4Threads, sa, st>>>(qp); break;
+      case 4096: q4_gateup_kernel<4><<<grid, kQ4Threads, sa, st>>>(qp); break;
+      case 7168: q4_gateup_kernel<7><<<grid, kQ4Threads, sa, st>>>(qp); break;
+      default: q4_gateup_kernel<8><<<grid, kQ4Threads, sa, st>>>(qp); break;
+    }
   }
-  h->launches++;
+  {
+    TimeScope ts(h, st, FT_TIME_FFN_RES);
+    switch (c.hidden) {
+      case 512: q4_down_kernel<2><<<grid, kQ4Threads, sb, st>>>(qp); break;
+      case 1024: q4_down_kernel<4><<<grid, kQ4Threads, sb, st>>>(qp); break;
+      case 2048: q4_down_kernel<8><<<grid, kQ4Threads, sb, st>>>(qp); break;
+      case 4096: q4_down_kernel<16><<<grid, kQ4Threads, sb, st>>>(qp); break;
+      case 7168: q4_down_kernel<28><<<grid, kQ4Threads, sb, st>>>(qp); break;
+      default: q4_down_kernel<32><<<grid, kQ4Threads, sb, st>>>(qp); break;
+    }
+  }
+  h->launches += 2;
   FT_CUDA(cudaGetLastError());
   return FT_OK;
 }

@@ -13,12 +13,18 @@ flattened identifier of Sec. 4.2 of the paper):
 ``bf16``  three row-major ``[I][d]`` bf16 matrices, in this order
           ``Wg_t`` (``Wg_t[n][i] = W_gate[i][n]``), ``Wu_t`` (same for W_up),
           ``Wd`` (``Wd[n][c] = W_down[n][c]``).  ``S = 3*I*d*2`` bytes.
-``int4``  the same three ``[I][d]`` matrices as 4-bit two's-complement codes
-          in [-8, 7], two per byte along ``d`` (low nibble = even column), then
-          bf16 scales: ``sg[I][d/128]``, ``su[I][d/128]`` (groups of 128
-          consecutive ``i``: the contraction dimension of gate/up) and
-          ``sd[I/128][d]`` (groups of 128 consecutive ``n``: the contraction
-          dimension of down).  ``S = 3*I*d/2 + (2*I*d/128 + (I/128)*d)*2``.
+``int4``  4-bit two's-complement codes in [-8, 7] for the same three matrices,
+          then bf16 scales.  ``Wg_q`` and ``Wu_q`` are row-major ``[I][d/2]`` bytes,
+          two codes per byte along ``d`` (low nibble = even column).  ``Wd_q`` is
+          stored in tensor-core fragment order: blocks of 16 neurons x tiles of 16
+          columns x 32 little-endian 32-bit words; word ``l = 4*g + q`` of block
+          ``b``, tile ``ct`` holds in nibble ``j`` (bits ``4j..4j+3``) the code of
+          neuron ``16b + NN[j] + q`` and column ``16ct + CC[j] + g`` with
+          ``NN = (0, 8, 0, 8, 4, 12, 4, 12)`` and ``CC = (0, 0, 8, 8, 0, 0, 8, 8)``.
+          Scales: ``sg[I][d/128]``, ``su[I][d/128]`` (groups of 128 consecutive
+          ``i``: the contraction dimension of gate/up) and ``sd[I/128][d]``
+          (groups of 128 consecutive ``n``: the contraction dimension of down).
+          ``S = 3*I*d/2 + (2*I*d/128 + (I/128)*d)*2``.
 
 The routing-logit recipes follow the workload descriptions: a Zipf-style
 popularity bias ``b_e = -alpha * ln(rank_e)`` with ``rank`` a seeded permutation
@@ -125,6 +131,24 @@ def _pack_nibbles(q: torch.Tensor) -> torch.Tensor:
     return u[..., 0::2] | (u[..., 1::2] << 4)
 
 
+WD_NN = (0, 8, 0, 8, 4, 12, 4, 12)   # neuron offset (plus q) of nibble j in a fragment-order word
+WD_CC = (0, 0, 8, 8, 0, 0, 8, 8)     # column offset (plus g) of nibble j
+
+
+def _pack_wd_fragment_order(q: torch.Tensor) -> torch.Tensor:
+    """int8 codes ``[I][d]`` of W_down -> uint8 bytes of the fragment-order layout."""
+    I, d = q.shape
+    blocks = q.reshape(I // 16, 16, d // 16, 16)                     # [b][nn][ct][cc]
+    l = torch.arange(32, device=q.device)
+    g, qq = l // 4, l % 4
+    nn = torch.tensor(WD_NN, device=q.device)[None, :] + qq[:, None]   # [32][8]
+    cc = torch.tensor(WD_CC, device=q.device)[None, :] + g[:, None]    # [32][8]
+    nib = blocks.permute(0, 2, 1, 3)[:, :, nn, cc]                    # [b][ct][32][8]
+    u = (nib.to(torch.int16) & 0xF).to(torch.uint8)
+    by = u[..., 0::2] | (u[..., 1::2] << 4)                            # [b][ct][32][4] bytes, little endian
+    return by.reshape(-1)
+
+
 def make_records(shape: LayerShape, seed: int, layer: int, first: int, count: int,
                  device="cpu", std: float = 0.02) -> torch.Tensor:
     """Records of experts ``first .. first+count-1`` of ``layer`` as uint8 ``[count, S]``.
@@ -144,7 +168,7 @@ def make_records(shape: LayerShape, seed: int, layer: int, first: int, count: in
             qu, su = _quantise_int4(w[1:2], 2)
             qd, sd = _quantise_int4(w[2:3], 1)
             parts = [_pack_nibbles(qg).reshape(-1), _pack_nibbles(qu).reshape(-1),
-                     _pack_nibbles(qd).reshape(-1),
+                     _pack_wd_fragment_order(qd[0]),
                      sg.reshape(-1).view(torch.uint8), su.reshape(-1).view(torch.uint8),
                      sd.reshape(-1).view(torch.uint8)]
             out[j] = torch.cat(parts)

@@ -36,13 +36,24 @@ def test_unpack_bf16_record_orientation():
 
 
 def _record_int4_by_definition(qg, qu, qd, sg, su, sd):
-    """qX: int codes [I][d] in stored orientation; sg/su [I][d/128]; sd [I/128][d] (floats, bf16-exact)."""
+    """qX: int codes [I][d] (row = neuron); sg/su [I][d/128]; sd [I/128][d] (floats, bf16-exact).
+    Gate/up: two codes per byte along d, low nibble = even column.  Down: fragment order, written
+    word by word from the documented nibble table."""
     I, d = qg.shape
     out = bytearray()
-    for q in (qg, qu, qd):
+    for q in (qg, qu):
         for n in range(I):
             for c in range(0, d, 2):
                 out.append((int(q[n, c]) & 0xF) | ((int(q[n, c + 1]) & 0xF) << 4))
+    NN, CC = (0, 8, 0, 8, 4, 12, 4, 12), (0, 0, 8, 8, 0, 0, 8, 8)
+    for b in range(I // 16):
+        for ct in range(d // 16):
+            for l in range(32):
+                g, q_ = divmod(l, 4)
+                word = 0
+                for j in range(8):
+                    word |= (int(qd[16 * b + NN[j] + q_, 16 * ct + CC[j] + g]) & 0xF) << (4 * j)
+                out += word.to_bytes(4, "little")
     for s in (sg, su, sd):
         out += _bf16_bits(s).tobytes()
     return np.frombuffer(bytes(out), dtype=np.uint8)
