@@ -29,15 +29,23 @@
  *   FT_W_BF16     : three row-major [inter][hidden] bf16 matrices, in this order:
  *                     Wg_t  (Wg_t[n][i] = W_gate[i][n]),  Wu_t (Wu_t[n][i] = W_up[i][n]),
  *                     Wd    (Wd[n][c]   = W_down[n][c]).          S = 3*inter*hidden*2 bytes.
- *   FT_W_INT4_G128: the same three [inter][hidden] matrices as 4-bit two's-complement codes in
- *                   [-8,7], two per byte along hidden (low nibble = even column), followed by bf16
- *                   scales sg[inter][hidden/128], su[inter][hidden/128] (groups of 128 consecutive
- *                   hidden indices: the contraction dimension of gate/up) and sd[inter/128][hidden]
- *                   (groups of 128 consecutive neurons: the contraction dimension of down);
+ *   FT_W_INT4_G128: 4-bit two's-complement codes in [-8,7] for the same three matrices, then bf16 scales;
  *                   weight = scale * code.
- *   Shape limits: bf16: hidden in {256, 512, 1024, 2048}, inter % 64 == 0; int4: hidden % 512 == 0,
- *   hidden <= 8192, inter % 128 == 0; n_experts <= 1024; top_k <= min(n_experts, 32);
- *   slots_per_layer <= 2048.
+ *                     Wg_q, Wu_q : row-major [inter][hidden/2] bytes, two codes per byte along hidden
+ *                                  (low nibble = even column).
+ *                     Wd_q       : tensor-core fragment order: blocks of 16 neurons x tiles of 16 columns x
+ *                                  32 little-endian 32-bit words; in word l = 4g + q of block b, tile ct,
+ *                                  nibble j (bits 4j..4j+3) is the code of neuron 16b + NN[j] + q and column
+ *                                  16ct + CC[j] + g, NN = (0,8,0,8,4,12,4,12), CC = (0,0,8,8,0,0,8,8).
+ *                     sg, su     : [inter][hidden/128] bf16 (groups of 128 consecutive hidden indices: the
+ *                                  contraction dimension of gate/up).
+ *                     sd         : [inter/128][hidden] bf16 (groups of 128 consecutive neurons: the
+ *                                  contraction dimension of down).
+ *                   S = 3*inter*hidden/2 + (2*inter*hidden/128 + (inter/128)*hidden)*2 bytes.
+ *   Shape limits: bf16: hidden in {256, 512, 1024, 2048}, inter % 16 == 0; int4: hidden in
+ *   {512, 1024, 2048, 4096, 7168, 8192}, inter % 128 == 0; n_experts <= 1024;
+ *   top_k <= min(n_experts, 32); slots_per_layer <= 2048.  The tensor-core prefill path
+ *   (gemm_min_tokens > 0) needs bf16 weights, slots_per_layer > 0 and inter % 128 == 0.
  */
 #ifndef FTMOE_H_
 #define FTMOE_H_

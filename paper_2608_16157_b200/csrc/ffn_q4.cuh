@@ -43,13 +43,12 @@ struct Q4Params {
   int d, inter, top_k, T, finalize;
 };
 
-// codes (s/4) and (s/4 + 4) of a word -> signed values as bf16x2
-__device__ __forceinline__ uint32_t q4_pair(uint32_t w, int s) {
-  uint32_t t = ((w >> s) & 0x000F000Fu) ^ 0x43084308u;
-  const uint32_t bias = 0x43084308u;  // (136.0, 136.0)
-  __nv_bfloat162 v = __hsub2(*reinterpret_cast<__nv_bfloat162 *>(&t), *reinterpret_cast<const __nv_bfloat162 *>(&bias));
-  return *reinterpret_cast<uint32_t *>(&v);
-}
+// codes (s/4) and (s/4 + 4) of a word -> the bf16x2 pair (136 + code, 136 + code): two instructions per
+// fragment register.  The constant 136 is taken out again in fp32: sum_k (136 + v_k) a_k = 136 sum_k a_k + sum_k v_k a_k.
+constexpr float kQ4Bias = 136.f;
+__device__ __forceinline__ uint32_t q4_pair(uint32_t w, int s) { return ((w >> s) & 0x000F000Fu) ^ 0x43084308u; }
+__device__ __forceinline__ float bf16lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
 
 // token g of a pass: row of x, gate weight
 __device__ __forceinline__ void q4_token(const Q4Params &p, const WorkItem &it, int pass, int g, int &tok, float &gw) {
@@ -156,8 +155,10 @@ __global__ void __launch_bounds__(kQ4Threads, 1) q4_gateup_kernel(Q4Params p) {
         // x fragments: lane (g, q) holds token g, contraction indices [128*(warp*SB+sb) + 32q, +32), each run of 8
         // rearranged as the pairs (0,4) (1,5) (2,6) (3,7) the dequantiser produces
         uint32_t xf[SB][4][4];
+        float xs[SB][2];   // 136 * (sum of x over the group) for tokens 2q and 2q+1: the bias term of the dot products
 #pragma unroll
-        for (int sb = 0; sb < SB; ++sb)
+        for (int sb = 0; sb < SB; ++sb) {
+          float part = 0.f;
 #pragma unroll
           for (int wi = 0; wi < 4; ++wi) {
             uint4 v = make_uint4(0u, 0u, 0u, 0u);
@@ -167,7 +168,14 @@ __global__ void __launch_bounds__(kQ4Threads, 1) q4_gateup_kernel(Q4Params p) {
             xf[sb][wi][1] = __byte_perm(v.x, v.z, 0x7632);
             xf[sb][wi][2] = __byte_perm(v.y, v.w, 0x5410);
             xf[sb][wi][3] = __byte_perm(v.y, v.w, 0x7632);
+            part += (bf16lo(v.x) + bf16hi(v.x)) + (bf16lo(v.y) + bf16hi(v.y)) + (bf16lo(v.z) + bf16hi(v.z)) +
+                    (bf16lo(v.w) + bf16hi(v.w));
           }
+          part += __shfl_xor_sync(0xffffffffu, part, 1);
+          part += __shfl_xor_sync(0xffffffffu, part, 2);    // all four lanes of token g hold its group sum
+          xs[sb][0] = kQ4Bias * __shfl_sync(0xffffffffu, part, (2 * q) * 4);
+          xs[sb][1] = kQ4Bias * __shfl_sync(0xffffffffu, part, (2 * q + 1) * 4);
+        }
         for (int b = b_begin; b < b_end; ++b) {
           float cgu[2][4];
 #pragma unroll
@@ -195,10 +203,10 @@ __global__ void __launch_bounds__(kQ4Threads, 1) q4_gateup_kernel(Q4Params p) {
                 }
                 const float s_lo = __bfloat162float(sc[g * (d / kGroup) + grp]);
                 const float s_hi = __bfloat162float(sc[(g + 8) * (d / kGroup) + grp]);
-                cgu[which][0] = fmaf(s_lo, acc[0], cgu[which][0]);
-                cgu[which][1] = fmaf(s_lo, acc[1], cgu[which][1]);
-                cgu[which][2] = fmaf(s_hi, acc[2], cgu[which][2]);
-                cgu[which][3] = fmaf(s_hi, acc[3], cgu[which][3]);
+                cgu[which][0] = fmaf(s_lo, acc[0] - xs[sb][0], cgu[which][0]);
+                cgu[which][1] = fmaf(s_lo, acc[1] - xs[sb][1], cgu[which][1]);
+                cgu[which][2] = fmaf(s_hi, acc[2] - xs[sb][0], cgu[which][2]);
+                cgu[which][3] = fmaf(s_hi, acc[3] - xs[sb][1], cgu[which][3]);
               }
             }
             __syncwarp();
@@ -304,59 +312,75 @@ __global__ void __launch_bounds__(kQ4Threads, 1) q4_down_kernel(Q4Params p) {
         const __nv_bfloat16 *sd = reinterpret_cast<const __nv_bfloat16 *>(it.w + 3 * mat_bytes + 2 * smat_bytes);
         const int col0 = hf * (d / 2) + warp * CTW * 16;   // first column of this warp
         float dacc[CTW][4];
-        uint32_t sdr[CTW];   // (scale of column g, scale of column g+8) as two bf16
+        float hsum = 0.f;   // sum over the neurons accumulated so far of h[n][token g] (as rounded to bf16)
 #pragma unroll
-        for (int c = 0; c < CTW; ++c) { dacc[c][0] = dacc[c][1] = dacc[c][2] = dacc[c][3] = 0.f; sdr[c] = 0u; }
-        int cur_grp = -1;
+        for (int c = 0; c < CTW; ++c) { dacc[c][0] = dacc[c][1] = dacc[c][2] = dacc[c][3] = 0.f; }
+        const int tok_a = __shfl_sync(0xffffffffu, tok_g, (2 * q) * 4);
+        const int tok_b = __shfl_sync(0xffffffffu, tok_g, (2 * q + 1) * 4);
+        const float gw_a = __shfl_sync(0xffffffffu, gw_g, (2 * q) * 4);
+        const float gw_b = __shfl_sync(0xffffffffu, gw_g, (2 * q + 1) * 4);
+        // The accumulators hold sum_n (136 + code) h; within one quantisation group of 128 neurons the scale is a
+        // per-column constant, so bias and scale are applied when the group (or the CTA's range) ends:
+        //   y += gate * scale[c] * (acc - 136 * sum_n h[n][t]).
+        auto flush = [&](int grp) {
+          float hs = hsum;
+          hs += __shfl_xor_sync(0xffffffffu, hs, 1);
+          hs += __shfl_xor_sync(0xffffffffu, hs, 2);
+          const float ha = kQ4Bias * __shfl_sync(0xffffffffu, hs, (2 * q) * 4);
+          const float hb2 = kQ4Bias * __shfl_sync(0xffffffffu, hs, (2 * q + 1) * 4);
+          uint32_t sdr[CTW];   // all scale loads are issued before the first atomic so their latencies overlap
+#pragma unroll
+          for (int c = 0; c < CTW; ++c) {
+            const __nv_bfloat16 *sp2 = sd + (size_t)grp * d + col0 + 16 * c + g;
+            sdr[c] = (uint32_t)__bfloat16_as_ushort(sp2[0]) | ((uint32_t)__bfloat16_as_ushort(sp2[8]) << 16);
+          }
+#pragma unroll
+          for (int c = 0; c < CTW; ++c) {
+            const int col = col0 + 16 * c + g;
+            const float s_lo = bf16lo(sdr[c]), s_hi = bf16hi(sdr[c]);
+            if (tok_a >= 0) {
+              atomicAdd(p.y_acc + (size_t)tok_a * d + col, gw_a * s_lo * (dacc[c][0] - ha));
+              atomicAdd(p.y_acc + (size_t)tok_a * d + col + 8, gw_a * s_hi * (dacc[c][2] - ha));
+            }
+            if (tok_b >= 0) {
+              atomicAdd(p.y_acc + (size_t)tok_b * d + col, gw_b * s_lo * (dacc[c][1] - hb2));
+              atomicAdd(p.y_acc + (size_t)tok_b * d + col + 8, gw_b * s_hi * (dacc[c][3] - hb2));
+            }
+            dacc[c][0] = dacc[c][1] = dacc[c][2] = dacc[c][3] = 0.f;
+          }
+          hsum = 0.f;
+        };
+        int cur_grp = (b_begin * 16) / kGroup;
+        // h fragments are fetched two blocks ahead (they sit in L2; a block is consumed faster than one L2 round trip)
+        const uint2 *hsrc = p.hbuf + (size_t)pu * NBLK * 32 + lane;
+        uint2 hb0 = hsrc[(size_t)b_begin * 32];
+        uint2 hb1 = (b_begin + 1 < b_end) ? hsrc[(size_t)(b_begin + 1) * 32] : make_uint2(0u, 0u);
         for (int b = b_begin; b < b_end; ++b, ++tile) {
-          const uint2 hb = p.hbuf[((size_t)pu * NBLK + b) * 32 + lane];   // issued before the wait on the stage
+          const uint2 hb = hb0;
+          hb0 = hb1;
+          if (b + 2 < b_end) hb1 = hsrc[(size_t)(b + 2) * 32];
           const int grp = (b * 16) / kGroup;
           if (grp != cur_grp) {
+            flush(cur_grp);
             cur_grp = grp;
-#pragma unroll
-            for (int c = 0; c < CTW; ++c) {
-              const __nv_bfloat16 *sp2 = sd + (size_t)grp * d + col0 + 16 * c + g;
-              sdr[c] = (uint32_t)__bfloat16_as_ushort(sp2[0]) | ((uint32_t)__bfloat16_as_ushort(sp2[8]) << 16);
-            }
           }
           const int s = tile % kQ4StagesB;
           const uint32_t ph = (tile / kQ4StagesB) & 1u;
           const bool ok = mbar_wait(full_bar(s), ph, s_abort, p.status);
           if (ok) {
+            hsum += (bf16lo(hb.x) + bf16hi(hb.x)) + (bf16lo(hb.y) + bf16hi(hb.y));
             const uint32_t base = smem_base + s * stage_bytes + (uint32_t)(warp * CTW) * 128 + 4 * lane;
 #pragma unroll
             for (int c = 0; c < CTW; ++c) {
               uint32_t w;
               asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w) : "r"(base + c * 128));
-              float t4[4] = {0.f, 0.f, 0.f, 0.f};
-              mma_bf16(t4, q4_pair(w, 0), q4_pair(w, 8), q4_pair(w, 4), q4_pair(w, 12), hb.x, hb.y);
-              const float s_lo = __uint_as_float(sdr[c] << 16), s_hi = __uint_as_float(sdr[c] & 0xffff0000u);
-              dacc[c][0] = fmaf(s_lo, t4[0], dacc[c][0]);
-              dacc[c][1] = fmaf(s_lo, t4[1], dacc[c][1]);
-              dacc[c][2] = fmaf(s_hi, t4[2], dacc[c][2]);
-              dacc[c][3] = fmaf(s_hi, t4[3], dacc[c][3]);
+              mma_bf16(dacc[c], q4_pair(w, 0), q4_pair(w, 8), q4_pair(w, 4), q4_pair(w, 12), hb.x, hb.y);
             }
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(empty_bar(s));
         }
-        // gate-weighted combine
-        const int tok_a = __shfl_sync(0xffffffffu, tok_g, (2 * q) * 4);
-        const int tok_b = __shfl_sync(0xffffffffu, tok_g, (2 * q + 1) * 4);
-        const float gw_a = __shfl_sync(0xffffffffu, gw_g, (2 * q) * 4);
-        const float gw_b = __shfl_sync(0xffffffffu, gw_g, (2 * q + 1) * 4);
-#pragma unroll
-        for (int c = 0; c < CTW; ++c) {
-          const int col = col0 + 16 * c + g;
-          if (tok_a >= 0) {
-            atomicAdd(p.y_acc + (size_t)tok_a * d + col, gw_a * dacc[c][0]);
-            atomicAdd(p.y_acc + (size_t)tok_a * d + col + 8, gw_a * dacc[c][2]);
-          }
-          if (tok_b >= 0) {
-            atomicAdd(p.y_acc + (size_t)tok_b * d + col, gw_b * dacc[c][1]);
-            atomicAdd(p.y_acc + (size_t)tok_b * d + col + 8, gw_b * dacc[c][3]);
-          }
-        }
+        flush(cur_grp);
       }
       u += (b_end - b_begin);
     }

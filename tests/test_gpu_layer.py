@@ -217,3 +217,15 @@ def test_qwen3_shaped_decode_two_layers(batch):
     st = pr.moe.get_stats(0)
     assert st["hits"] > 0 and st["fills"] > 0
     pr.close()
+
+
+def test_dsv3_shaped_int4_decode_one_layer():
+    """d=7168, 256 routed experts (int4, group 128) + 1 shared expert, I=2048, top-8, 64 slots, batch 4."""
+    shape = W.DSV3_INT4
+    steps = 3
+    pr = Pair(shape, n_slots=64, max_tokens=8, n_layers=1, seed=0, gen_device="cuda")
+    logits = W.ar1_logits(1, steps, 4, 256, rho=0.9, alpha=1.2, seed=0)
+    for t in range(steps):
+        x = W.noise_x(4, 7168, 0, t, 0)
+        pr.step(0, logits[t, 0], x, check_y=(t != 1), check_slots=(t == 0), fused=(t == 2))
+    pr.close()
