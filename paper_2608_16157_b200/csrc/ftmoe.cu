@@ -416,9 +416,10 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
         !make_tensor_map(enc, &h->tm_w128, h->slots, wrows, c.hidden, 128, 64) ||
         !make_tensor_map(enc, &h->tm_w64, h->slots, wrows, c.hidden, 64, 64))
       return fail(FT_ERR_CUDA);
-    const int gsm = (int)grouped_gemm_smem_bytes();
-    FT_TRY(cudaFuncSetAttribute(grouped_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, gsm));
-    FT_TRY(cudaFuncSetAttribute(grouped_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, gsm));
+    FT_TRY(cudaFuncSetAttribute(grouped_gemm_kernel<0, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)grouped_gemm_smem_bytes<1>()));
+    FT_TRY(cudaFuncSetAttribute(grouped_gemm_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)grouped_gemm_smem_bytes<1>()));
     h->gemm = true;
   }
   FT_TRY(cudaMalloc(&h->status_dev, 4));
@@ -723,16 +724,15 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
       gp.inter = c.inter; gp.d = c.hidden;
       gp.layer_row0 = (long long)layer * c.slots_per_layer * 3 * c.inter;
       gp.status = h->status_dev;
-      const size_t gsm = grouped_gemm_smem_bytes();
       gp.K = c.hidden; gp.n_tiles = c.inter / 128; gp.out = h->hbuf;
       {
         TimeScope ts(h, st, FT_TIME_GEMM1);
-        grouped_gemm_kernel<0><<<h->sm_count, kGemmThreads, gsm, st>>>(h->tm_xs, h->tm_w128, gp);
+        grouped_gemm_kernel<0, 1><<<h->sm_count, kGemmThreads, grouped_gemm_smem_bytes<1>(), st>>>(h->tm_xs, h->tm_w128, gp);
       }
       gp.K = c.inter; gp.n_tiles = c.hidden / kGemmBN; gp.out = h->obuf;
       {
         TimeScope ts(h, st, FT_TIME_GEMM2);
-        grouped_gemm_kernel<1><<<h->sm_count, kGemmThreads, gsm, st>>>(h->tm_h, h->tm_w64, gp);
+        grouped_gemm_kernel<1, 1><<<h->sm_count, kGemmThreads, grouped_gemm_smem_bytes<1>(), st>>>(h->tm_h, h->tm_w64, gp);
       }
       {
         TimeScope ts(h, st, FT_TIME_COMBINE);

@@ -20,8 +20,18 @@
 namespace ftmoe {
 
 constexpr int kGemmThreads = 192;
-constexpr int kGemmBM = 128, kGemmBN = 256, kGemmBK = 64, kGemmStages = 4;
-constexpr int kGemmStageBytes = kGemmBM * kGemmBK * 2 + kGemmBN * kGemmBK * 2;  // 16 KiB + 32 KiB
+constexpr int kGemmBM = 128, kGemmBN = 256, kGemmBK = 64;
+constexpr int kGemmATile = kGemmBM * kGemmBK * 2;   // 16 KiB
+constexpr int kGemmBTile = kGemmBN * kGemmBK * 2;   // 32 KiB
+// MT = 128-row tiles of one expert that share every B tile (1 or 2).  With MT = 2 a stage holds two A tiles and
+// one B tile (64 KiB for 2 x 128 x 256 x 64 MACs instead of 48 KiB for one), which takes the kernel off the
+// L2-to-shared-memory bandwidth limit; the price is that both TMEM accumulators belong to one unit, so the
+// epilogue no longer overlaps the next main loop.
+template <int MT> struct GemmCfg {
+  static constexpr int kStageBytes = MT * kGemmATile + kGemmBTile;
+  static constexpr int kStages = (MT == 1) ? 4 : 3;
+  static constexpr int kBufs = (MT == 1) ? 2 : 1;   // TMEM accumulator sets in flight
+};
 
 struct GemmParams {
   const WorkItem *items;
@@ -78,6 +88,14 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// SiLU(g) * u with one MUFU: sigmoid(g) = 0.5 * tanh(0.5 g) + 0.5 (tanh.approx, rel. error ~2^-11, far below
+// the bf16 rounding of the result).
+__device__ __forceinline__ float swiglu_fast(float g, float u) {
+  float t;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(0.5f * g));
+  return g * fmaf(0.5f, t, 0.5f) * u;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<uint32_t *>(&v);
@@ -85,16 +103,19 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 
 // Dynamic shared memory (1024-byte aligned by the kernel): [stages][A 16 KiB | B 32 KiB] | barriers | tmem base |
 // abort flag | tile prefix.
-template <int MODE>
+template <int MODE, int MT>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  constexpr int kGemmStages = GemmCfg<MT>::kStages, kGemmStageBytes = GemmCfg<MT>::kStageBytes;
+  constexpr int kBufs = GemmCfg<MT>::kBufs;
   unsigned char *sp = smem + kGemmStages * kGemmStageBytes;
   uint64_t *s_bar = reinterpret_cast<uint64_t *>(sp); sp += 16 * 8;
   uint32_t *s_tmem = reinterpret_cast<uint32_t *>(sp); sp += 8;
   volatile int *s_abort = reinterpret_cast<volatile int *>(sp); sp += 8;
-  int32_t *s_pref = reinterpret_cast<int32_t *>(sp);
+  int32_t *s_pref = reinterpret_cast<int32_t *>(sp); sp += (kMaxExperts + 2) * 4;
+  int32_t *s_upref = reinterpret_cast<int32_t *>(sp);   // exclusive prefix of the units (groups of MT row tiles)
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t smem_base = smem_u32(smem);
@@ -121,21 +142,31 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if (tid == 0) {
+    int acc = 0;
+    for (int i = 0; i < n_items; ++i) {
+      s_upref[i] = acc;
+      acc += (s_pref[i + 1] - s_pref[i] + MT - 1) / MT;
+    }
+    s_upref[n_items] = acc;
+  }
+  __syncthreads();
   const uint32_t tmem_base = *s_tmem;
-  const int total_tiles = s_pref[n_items] * p.n_tiles;
+  const int total_tiles = s_upref[n_items] * p.n_tiles;
   const int kblocks = p.K / kGemmBK;
 
-  // tile -> (item, row tile inside the item, n tile)
-  auto locate = [&](int tile, int &item, int &mt_in, int &nt) {
-    const int mt = tile / p.n_tiles;
-    nt = tile - mt * p.n_tiles;
-    int lo = 0, hi = n_items;            // largest item with pref[item] <= mt
+  // work unit -> (item, first row tile inside the item, row tiles in the unit, n tile)
+  auto locate = [&](int tile, int &item, int &mt_in, int &n_mt, int &nt) {
+    const int un = tile / p.n_tiles;
+    nt = tile - un * p.n_tiles;
+    int lo = 0, hi = n_items;            // largest item with upref[item] <= un
     while (hi - lo > 1) {
       const int mid = (lo + hi) >> 1;
-      if (s_pref[mid] <= mt) lo = mid; else hi = mid;
+      if (s_upref[mid] <= un) lo = mid; else hi = mid;
     }
     item = lo;
-    mt_in = mt - s_pref[lo];
+    mt_in = (un - s_upref[lo]) * MT;
+    n_mt = min(MT, s_pref[lo + 1] - s_pref[lo] - mt_in);
   };
 
   if (warp == 0) {
@@ -143,8 +174,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (lane == 0) {
       uint32_t it_k = 0;
       for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-        int item, mt_in, nt;
-        locate(tile, item, mt_in, nt);
+        int item, mt_in, n_mt, nt;
+        locate(tile, item, mt_in, n_mt, nt);
         const WorkItem it = p.items[item];
         const int a_row = it.off + mt_in * kGemmBM;
         const long long rec_row = p.layer_row0 + (long long)it.slot * 3 * p.inter;
@@ -154,9 +185,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           mbar_wait(empty_bar(s), ph ^ 1u, s_abort, p.status);
           if (*s_abort) break;
           const uint32_t sa = smem_base + s * kGemmStageBytes;
-          const uint32_t sb = sa + kGemmBM * kGemmBK * 2;
-          mbar_expect_tx(full_bar(s), kGemmStageBytes);
-          tma_load_2d(sa, &tmA, kb * kGemmBK, a_row, full_bar(s));
+          const uint32_t sb = sa + MT * kGemmATile;
+          mbar_expect_tx(full_bar(s), n_mt * kGemmATile + kGemmBTile);
+          for (int m = 0; m < n_mt; ++m) tma_load_2d(sa + m * kGemmATile, &tmA, kb * kGemmBK, a_row + m * kGemmBM, full_bar(s));
           if (MODE == 0) {
             const int n0 = nt * 128;
             tma_load_2d(sb, &tmB, kb * kGemmBK, (int)(rec_row + n0), full_bar(s));                       // gate rows
@@ -177,10 +208,12 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                              ((uint32_t)(kGemmBN >> 3) << 17) | ((uint32_t)(kGemmBM >> 4) << 24);
       uint32_t it_k = 0, n_tile = 0;
       for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++n_tile) {
-        const int buf = n_tile & 1;
-        mbar_wait(tempty_bar(buf), ((n_tile >> 1) & 1u) ^ 1u, s_abort, p.status);
+        int item, mt_in, n_mt, nt;
+        locate(tile, item, mt_in, n_mt, nt);
+        const int buf = n_tile % kBufs;
+        mbar_wait(tempty_bar(buf), ((n_tile / kBufs) & 1u) ^ 1u, s_abort, p.status);
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)buf * kGemmBN;
+        const uint32_t d_tmem = tmem_base + (uint32_t)buf * kGemmBN;   // (kBufs == 1: accumulator m at column m*256)
         for (int kb = 0; kb < kblocks; ++kb, ++it_k) {
           const int s = it_k % kGemmStages;
           const uint32_t ph = (it_k / kGemmStages) & 1u;
@@ -188,13 +221,15 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           tc_fence_after();
           if (ok) {
             const uint32_t sa = smem_base + s * kGemmStageBytes;
-            const uint32_t sb = sa + kGemmBM * kGemmBK * 2;
+            const uint32_t sb = sa + MT * kGemmATile;
 #pragma unroll
             for (int k16 = 0; k16 < kGemmBK / 16; ++k16) {
-              const uint64_t adesc = umma_desc(sa + k16 * 32, 16, 1024);
               const uint64_t bdesc = (MODE == 0) ? umma_desc(sb + k16 * 32, 16, 1024)
                                                  : umma_desc(sb + k16 * 2048, 8192, 1024);
-              umma_bf16(d_tmem, adesc, bdesc, idesc, (kb | k16) != 0 ? 1u : 0u);
+              for (int m = 0; m < n_mt; ++m) {
+                const uint64_t adesc = umma_desc(sa + m * kGemmATile + k16 * 32, 16, 1024);
+                umma_bf16(d_tmem + (uint32_t)m * kGemmBN, adesc, bdesc, idesc, (kb | k16) != 0 ? 1u : 0u);
+              }
             }
           }
           umma_commit(empty_bar(s));   // the stage is free once these MMAs have read it
@@ -207,16 +242,17 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const int quarter = warp & 3;      // TMEM lanes [32*quarter, 32*quarter+32) are visible to this warp
     uint32_t n_tile = 0;
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++n_tile) {
-      int item, mt_in, nt;
-      locate(tile, item, mt_in, nt);
+      int item, mt_in, n_mt, nt;
+      locate(tile, item, mt_in, n_mt, nt);
       const WorkItem it = p.items[item];
-      const int buf = n_tile & 1;
-      const bool ok = mbar_wait(tfull_bar(buf), (n_tile >> 1) & 1u, s_abort, p.status);
+      const int buf = n_tile % kBufs;
+      const bool ok = mbar_wait(tfull_bar(buf), (n_tile / kBufs) & 1u, s_abort, p.status);
       tc_fence_after();
-      const int row_in = mt_in * kGemmBM + quarter * 32 + lane;
+      for (int m = 0; m < n_mt; ++m) {
+      const int row_in = (mt_in + m) * kGemmBM + quarter * 32 + lane;
       const bool valid = ok && row_in < it.n_tok;
       const size_t row = (size_t)it.off + row_in;
-      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * kGemmBN;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf + m) * kGemmBN;
       if (MODE == 0) {
         __nv_bfloat16 *dst = p.out + row * p.inter + nt * 128;
 #pragma unroll 1
@@ -229,10 +265,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             uint32_t o[16];
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
-              const float g0 = __uint_as_float(g[2 * j]), g1 = __uint_as_float(g[2 * j + 1]);
-              const float h0 = g0 / (1.f + __expf(-g0)) * __uint_as_float(u[2 * j]);
-              const float h1 = g1 / (1.f + __expf(-g1)) * __uint_as_float(u[2 * j + 1]);
-              o[j] = pack_bf16(h0, h1);
+              o[j] = pack_bf16(swiglu_fast(__uint_as_float(g[2 * j]), __uint_as_float(u[2 * j])),
+                               swiglu_fast(__uint_as_float(g[2 * j + 1]), __uint_as_float(u[2 * j + 1])));
             }
             uint4 *d4 = reinterpret_cast<uint4 *>(dst + c);
 #pragma unroll
@@ -257,6 +291,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
         }
       }
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(buf));
@@ -270,8 +305,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   }
 }
 
+template <int MT>
 inline size_t grouped_gemm_smem_bytes() {
-  return 1024 + (size_t)kGemmStages * kGemmStageBytes + 16 * 8 + 16 + (kMaxExperts + 2) * 4;
+  return 1024 + (size_t)GemmCfg<MT>::kStages * GemmCfg<MT>::kStageBytes + 16 * 8 + 16 + 2 * (kMaxExperts + 2) * 4;
 }
 
 // x rows into expert-sorted order: xs[pos] = x[perm[pos] / k]  (16 bytes per thread).
