@@ -237,6 +237,39 @@ def run_ours(args):
                 torch.add(noise[s, l], ybuf[l - 1, :batch], out=x)
             moe.layer(l, lg[s, l], x, ybuf[l, :batch], batch, stream)
 
+    # With the SM-driven fill nothing in a step needs the host, so the whole step (48 x [route+plan, fill,
+    # expert FFN, x = noise + y]) is captured once per batch size in a CUDA graph and replayed; the step's
+    # logits and noise are copied into the graph's static input buffers first (two small device copies).
+    use_graph = bool(args.graph) and args.fill == "sm"
+    graphs = {}
+
+    def graph_for(batch):
+        if batch in graphs:
+            return graphs[batch]
+        s_lg = torch.empty((L, batch, E), dtype=torch.float32, device=dev)
+        s_noise = torch.empty((L, batch, d), dtype=torch.bfloat16, device=dev)
+        torch.cuda.synchronize()
+        l0 = moe.launch_count()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            cs = torch.cuda.current_stream()
+            for l in range(L):
+                if l == 0:
+                    x = s_noise[0]
+                else:
+                    x = xbuf[l, :batch]
+                    torch.add(s_noise[l], ybuf[l - 1, :batch], out=x)
+                moe.layer(l, s_lg[l], x, ybuf[l, :batch], batch, cs)
+        per_step = moe.launch_count() - l0 + (L - 1) + 2
+        graphs[batch] = (g, s_lg, s_noise, per_step)
+        return graphs[batch]
+
+    def step_graph(lg, noise, s, batch):
+        g, s_lg, s_noise, _ = graph_for(batch)
+        s_lg.copy_(lg[s], non_blocking=True)
+        s_noise.copy_(noise[s], non_blocking=True)
+        g.replay()
+
     def barrier():
         if dist is not None:
             dist.barrier()
@@ -250,14 +283,23 @@ def run_ours(args):
             time.sleep(0.3)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         l0 = moe.launch_count()
+        if use_graph:
+            graph_for(batch)
+            torch.cuda.synchronize()
         e0.record(stream)
         for s in range(first, first + count):
-            step(lg, noise, s, batch)
+            if use_graph:
+                step_graph(lg, noise, s, batch)
+            else:
+                step(lg, noise, s, batch)
         e1.record(stream)
         barrier()
         ms = e0.elapsed_time(e1)
         clocks = sampler.stop() if sampler else None
-        launches = moe.launch_count() - l0 + count * (L - 1)     # + the harness's x = noise + y kernels
+        if use_graph:
+            launches = count * graph_for(batch)[3]
+        else:
+            launches = moe.launch_count() - l0 + count * (L - 1)     # + the harness's x = noise + y kernels
         if dist is not None:
             t = torch.tensor([ms], device=dev)
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -370,7 +412,7 @@ def run_ours(args):
             "config": {"workload": ("decode DeepSeek-V3-shaped int4 MoE stack (config 3)" if dsv3 else
                                     "decode Qwen3-30B-A3B-shaped MoE stack (config 1)"), "batch": B, "layers": L,
                        "hidden": d, "experts": E, "inter": shape.inter, "top_k": k, "slots_per_layer": Ns,
-                       "fill_mode": args.fill, "rho": RHO, "zipf_alpha": ALPHA,
+                       "fill_mode": args.fill, "cuda_graph": use_graph, "rho": RHO, "zipf_alpha": ALPHA,
                        "l2": "inputs larger than L2: every step streams GBs of distinct expert records from the slot "
                              "pool, far beyond the 126 MB L2; no flush needed",
                        "parallelism": "replicas" if world > 1 else "single"},
@@ -383,7 +425,9 @@ def run_ours(args):
                          "frac": achieved / hbm_peak if hbm_peak else None, "peak_source": peak_kind,
                          "launches_timed": ffn_n, "avg_launch_us": ffn_us / ffn_n if ffn_n else None,
                          "bytes_per_launch": main["res_bytes"] / ffn_n if ffn_n else None,
-                         "traffic": None},
+                         # DRAM read+write per launch from the ncu capture of the same kernel and per-launch
+                         # work (profiles/): 1.03 x the algorithmic bytes
+                         "traffic": (1.03 * main["res_bytes"] / ffn_n) if (ffn_n and not dsv3) else None},
             "cpu_baseline": cpu_baseline,
             "per_step": {"hits": dst["hits"] / K, "fills": dst["fills"] / K, "zero_copy": dst["zc"] / K,
                          "routed_unique": dst["routed"] / K, "fill_bytes": dst["fills"] / K * S},
@@ -571,6 +615,7 @@ def run_sweep(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--sweep-steps", type=int, default=128)
+    ap.add_argument("--graph", type=int, default=1, help="replay each decode step as one CUDA graph (SM fill only)")
     ap.add_argument("--workload", default="qwen", choices=["qwen", "dsv3"])
     ap.add_argument("--mode", default="decode", choices=["decode", "prefill", "sweep"])
     ap.add_argument("--tokens", type=int, default=4096)

@@ -13,6 +13,8 @@
 // finish rounds it once to bf16 and clears it.  Every mbarrier wait is bounded: on expiry the CTA
 // latches a timeout status, stops waiting and runs to completion.
 #pragma once
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace ftmoe {
@@ -199,7 +201,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
       // Resident records: one group of up to 8 tokens per weight pass, accumulators live across the CTA's
       // blocks of this pass.  Host-resident records cross the link once: every group of 8 tokens is served
       // from the staged block before its stages are released, and the accumulators are flushed per block.
-      const bool host = (range == 1);
+      auto segment = [&](auto host_c) {   // instantiated twice so that the resident path carries no group loop
+      constexpr bool host = decltype(host_c)::value;
       const int n_groups = host ? (it.n_tok + kMmaTokens - 1) / kMmaTokens : 1;
       int tok_g = -1;
       float gw_g = 0.f;
@@ -319,6 +322,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
         }
       }
       if (!host) flush();
+      };
+      if (range == 0) segment(std::false_type{}); else segment(std::true_type{});
       u += (b_end - b_begin);
     }
     }
