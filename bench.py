@@ -191,8 +191,19 @@ def run_ours(args):
     B = (4 if args.batch == 8 else args.batch) if dsv3 else args.batch
     Wn, K = args.warmup, args.steps
     t_setup = time.perf_counter()
-    pool = Bd.HostPool(L * E * S)
-    W.fill_pool(pool.tensor, shape, L, SEED, device=dev, chunk=32)
+    from paper_2608_16157_b200 import multirank as MR
+    shm_name = None
+    if world > 1 and MR.shm_has_room(L * E * S):
+        # one copy of the host pool for all replicas of the node: rank 0 fills a /dev/shm file, every rank
+        # maps it and pins it in place
+        def _fill(arr):
+            W.fill_pool(torch.from_numpy(arr), shape, L, SEED, device=dev, chunk=32)
+        arr, shm_name = MR.open_shared_pool(L * E * S, f"{os.environ.get('MASTER_PORT', '0')}_{args.workload}", rank,
+                                            dist.barrier, fill=_fill)
+        pool = Bd.RegisteredPool(arr)
+    else:
+        pool = Bd.HostPool(L * E * S)
+        W.fill_pool(pool.tensor, shape, L, SEED, device=dev, chunk=32)
     shared = W.make_shared_records(shape, L, SEED, device=dev) if shape.n_shared else None
     log(f"[rank {rank}] pool {L * E * S / 2**30:.1f} GiB pinned+filled in {time.perf_counter() - t_setup:.1f}s")
 
@@ -415,7 +426,8 @@ def run_ours(args):
                        "fill_mode": args.fill, "cuda_graph": use_graph, "rho": RHO, "zipf_alpha": ALPHA,
                        "l2": "inputs larger than L2: every step streams GBs of distinct expert records from the slot "
                              "pool, far beyond the 126 MB L2; no flush needed",
-                       "parallelism": "replicas" if world > 1 else "single"},
+                       "parallelism": "replicas" if world > 1 else "single",
+                       "host_pool": "one /dev/shm copy shared by all ranks" if shm_name else "private pinned pool"},
             "clocks": main["clocks"],
             "e2e": e2e,
             "gpu_launches": main["launches"],
@@ -447,6 +459,8 @@ def run_ours(args):
         print(json.dumps(line), flush=True)
     moe.destroy()
     pool.free()
+    if shm_name is not None:
+        MR.close_shared_pool(pool.array, shm_name, rank, dist.barrier)
     if dist is not None:
         dist.destroy_process_group()
 

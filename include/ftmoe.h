@@ -133,6 +133,12 @@ size_t ft_moe_expert_bytes(const ft_moe_config_t *cfg);
  * out; free with ft_moe_host_free.  Contents are uninitialised. */
 ft_status_t ft_moe_host_alloc(size_t bytes, void **out_host);
 ft_status_t ft_moe_host_free(void *host);
+/* Pins and maps memory the caller already owns (cudaHostRegister, portable | mapped), e.g. a file mapping
+ * of the pool that several processes on the node share, or a pool that was read from disk into ordinary
+ * memory first and is pinned only afterwards (paper Sec. 3.3: pin after the buffers are filled).  HOST
+ * pointer, page aligned; undo with ft_moe_host_unregister before the memory goes away. */
+ft_status_t ft_moe_host_register(void *host, size_t bytes);
+ft_status_t ft_moe_host_unregister(void *host);
 
 /* Validates the configuration, checks that host_pool is pinned and mapped (else FT_ERR_NOT_PINNED),
  * allocates n_layers*slots_per_layer slots (FT_ERR_OOM if HBM cannot hold them) and empty tables

@@ -27,7 +27,7 @@ SYMBOLS = (
     "ft_moe_layer_host", "ft_moe_get_routing", "ft_moe_get_slot_table", "ft_moe_read_slot",
     "ft_moe_get_stats", "ft_moe_reset", "ft_moe_sync_status", "ft_moe_last_fill", "ft_moe_launch_count",
     "ft_moe_status_string", "ft_moe_timing_enable", "ft_moe_timing_read", "ft_moe_ffn_noalloc",
-    "ft_moe_last_cuda_error",
+    "ft_moe_last_cuda_error", "ft_moe_host_register", "ft_moe_host_unregister",
 )
 NOALLOC_MAX_TOKENS, NOALLOC_MAX_HIDDEN = 64, 2048
 TIME_NAMES = ("route", "plan", "ffn_zc", "ffn_res", "finalize", "fill", "gather", "gemm1", "gemm2", "combine")
@@ -82,6 +82,8 @@ def load(rebuild: bool = False):
         "ft_moe_expert_bytes": (sz, [C.POINTER(Config)]),
         "ft_moe_host_alloc": (i32, [sz, C.POINTER(vp)]),
         "ft_moe_host_free": (i32, [vp]),
+        "ft_moe_host_register": (i32, [vp, sz]),
+        "ft_moe_host_unregister": (i32, [vp]),
         "ft_moe_create": (i32, [C.POINTER(Config), C.POINTER(vp)]),
         "ft_moe_destroy": (i32, [vp]),
         "ft_moe_calibrate": (i32, [vp, C.POINTER(C.c_uint32)]),
@@ -172,6 +174,26 @@ class HostPool:
             self.free()
         except Exception:
             pass
+
+
+class RegisteredPool:
+    """Caller-owned host memory (a numpy array, e.g. a shared file mapping) pinned and mapped in place
+    with ``ft_moe_host_register``; same interface as :class:`HostPool`."""
+
+    def __init__(self, array: np.ndarray):
+        import torch
+        assert array.dtype == np.uint8 and array.flags["C_CONTIGUOUS"]
+        self.array = array
+        self.n_bytes = array.size
+        self.ptr = C.c_void_p(array.ctypes.data)
+        _check(load().ft_moe_host_register(self.ptr, self.n_bytes), "ft_moe_host_register")
+        self.tensor = torch.from_numpy(array)
+
+    def free(self):
+        if self.ptr is not None and self.ptr.value:
+            _check(load().ft_moe_host_unregister(self.ptr), "ft_moe_host_unregister")
+            self.ptr = None
+            self.tensor = None
 
 
 def _ptr(t) -> int:

@@ -249,6 +249,23 @@ ft_status_t ft_moe_host_free(void *host) {
   return FT_OK;
 }
 
+ft_status_t ft_moe_host_register(void *host, size_t bytes) {
+  if (!host || bytes == 0) return FT_ERR_INVALID_ARG;
+  cudaError_t e = cudaHostRegister(host, bytes, cudaHostRegisterPortable | cudaHostRegisterMapped);
+  if (e != cudaSuccess) {
+    g_last_cuda_error = e;
+    (void)cudaGetLastError();
+    return e == cudaErrorMemoryAllocation ? FT_ERR_OOM : FT_ERR_CUDA;
+  }
+  return FT_OK;
+}
+
+ft_status_t ft_moe_host_unregister(void *host) {
+  if (!host) return FT_OK;
+  FT_CUDA(cudaHostUnregister(host));
+  return FT_OK;
+}
+
 ft_status_t ft_moe_destroy(ft_moe_t *h) {
   if (!h) return FT_OK;
   cudaSetDevice(h->cfg.device);

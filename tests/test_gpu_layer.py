@@ -229,3 +229,19 @@ def test_dsv3_shaped_int4_decode_one_layer():
         x = W.noise_x(4, 7168, 0, t, 0)
         pr.step(0, logits[t, 0], x, check_y=(t != 1), check_slots=(t == 0), fused=(t == 2))
     pr.close()
+
+
+def test_pool_pinned_in_place_with_host_register():
+    """A pool in ordinary (here: anonymously mapped) memory, pinned afterwards with ft_moe_host_register."""
+    import mmap
+    shape = W.TINY
+    S = shape.expert_bytes
+    buf = mmap.mmap(-1, shape.n_experts * S)
+    arr = np.frombuffer(buf, dtype=np.uint8)
+    W.fill_pool(torch.from_numpy(arr), shape, 1, seed=0)
+    pool = B.RegisteredPool(arr)
+    pr = Pair(shape, n_slots=4, max_tokens=8, pool=pool)
+    for step in range(2):
+        pr.step(0, W.normal_logits(8, 8, 0, step), W.noise_x(8, 256, 0, step, 0), check_slots=True)
+    pr.close()
+    pool.free()
