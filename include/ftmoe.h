@@ -212,6 +212,11 @@ enum { FT_TIME_ROUTE = 0, FT_TIME_PLAN, FT_TIME_FFN_ZC, FT_TIME_FFN_RES, FT_TIME
        FT_TIME_GATHER, FT_TIME_GEMM1, FT_TIME_GEMM2, FT_TIME_COMBINE, FT_TIME_COUNT };
 ft_status_t ft_moe_timing_enable(ft_moe_t *h, int on);
 ft_status_t ft_moe_timing_read(ft_moe_t *h, double *out_us, uint64_t *out_launches, int n);
+/* Per-CTA record of the latest bf16 streaming-kernel launch: out[4*i .. 4*i+3] = global timer (ns) at the
+ * start and at the end of CTA i's streaming work, 16-neuron blocks it streamed, segments (expert, pass) it
+ * touched (for the CTA that finalized y: minus the global timer when it finished).  n_ctas
+ * entries at most (one CTA per SM).  Waits for the device. */
+ft_status_t ft_moe_get_cta_trace(ft_moe_t *h, int64_t *out, int n_ctas);
 /* Number of kernels this handle has launched since create. */
 ft_status_t ft_moe_launch_count(ft_moe_t *h, uint64_t *out);
 const char *ft_moe_status_string(ft_status_t s);

@@ -39,6 +39,8 @@ struct FfnMmaParams {
   uint32_t *status;
   int d, inter, top_k, T, finalize;
   int max_items;            // capacity of items / pref (entries beyond *n_items are ignored)
+  long long *trace;         // optional [gridDim.x][4]: start and end of the CTA's streaming (global timer, ns), blocks
+                            // streamed, segments (the finalizing CTA stores minus its finish time there); or nullptr
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -116,6 +118,9 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
   __shared__ int s_last;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  long long t_start;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_start));
+  int trace_blocks = 0, trace_segments = 0;
   const int n_items = *p.n_items;
   const int NBLK = p.inter / kMmaTileRows;
   const uint32_t smem_base = smem_u32(smem);
@@ -160,6 +165,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
       const int b_end = (left < (long long)(NBLK - b_begin)) ? b_begin + (int)left : NBLK;
       const uint8_t *rec = p.items[item].w;
       const size_t mat_bytes = (size_t)row_bytes * p.inter;
+      trace_blocks += b_end - b_begin;
+      ++trace_segments;
       for (int b = b_begin; b < b_end; ++b, ++tile) {
         const uint32_t ph = tile & 1u;     // `tile` counts this CTA's blocks; stage = 2*matrix + half
 #pragma unroll 1
@@ -329,6 +336,12 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
     }
   }
 
+  if (p.trace != nullptr && tid == 256) {   // lane 0 of the producer warp
+    long long *tr = p.trace + 4 * blockIdx.x;
+    long long t_end;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_end));
+    tr[0] = t_start; tr[1] = t_end; tr[2] = trace_blocks; tr[3] = trace_segments;
+  }
   // ---- the last CTA to finish rounds the accumulator to bf16 and clears it ----
   if (!p.finalize) return;
   __threadfence();
@@ -341,16 +354,35 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
   if (!s_last) return;
   __threadfence();
   const long long n4 = (long long)p.T * d / 4;
-  for (long long i = tid; i < n4; i += blockDim.x) {
-    const float4 v = __ldcg(reinterpret_cast<const float4 *>(p.y_acc) + i);
-    __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
-    uint2 o;
-    o.x = *reinterpret_cast<uint32_t *>(&a);
-    o.y = *reinterpret_cast<uint32_t *>(&b);
-    reinterpret_cast<uint2 *>(p.y)[i] = o;
-    reinterpret_cast<float4 *>(p.y_acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  // eight independent L2 loads in flight per thread: the round trips overlap instead of adding up
+  for (long long i0 = tid; i0 < n4; i0 += 8LL * blockDim.x) {
+    float4 v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const long long i = i0 + (long long)j * blockDim.x;
+      v[j] = (i < n4) ? __ldcg(reinterpret_cast<const float4 *>(p.y_acc) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const long long i = i0 + (long long)j * blockDim.x;
+      if (i < n4) {
+        __nv_bfloat162 a = __floats2bfloat162_rn(v[j].x, v[j].y), b = __floats2bfloat162_rn(v[j].z, v[j].w);
+        uint2 o;
+        o.x = *reinterpret_cast<uint32_t *>(&a);
+        o.y = *reinterpret_cast<uint32_t *>(&b);
+        reinterpret_cast<uint2 *>(p.y)[i] = o;
+        reinterpret_cast<float4 *>(p.y_acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
   }
-  if (tid == 0) *p.done = 0u;
+  if (tid == 0) {
+    *p.done = 0u;
+    if (p.trace != nullptr) {   // the finalizing CTA also notes when the whole kernel was done
+      long long t_fin;
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_fin));
+      p.trace[4 * blockIdx.x + 3] = -t_fin;
+    }
+  }
 }
 
 inline size_t ffn_mma_smem_bytes(int d) {

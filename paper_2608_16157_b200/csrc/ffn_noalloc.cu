@@ -115,6 +115,7 @@ extern "C" ft_status_t ft_moe_ffn_noalloc(int device, const void *record_dev, in
   mp.n_zc = &ctl->n_zc;
   mp.pref = ctl->pref;
   mp.max_items = 1;
+  mp.trace = nullptr;
   mp.x = static_cast<const __nv_bfloat16 *>(x_dev);
   mp.perm = nullptr;       // unused: the item addresses tokens directly
   mp.topk_w = nullptr;

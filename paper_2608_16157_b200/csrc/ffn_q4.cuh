@@ -397,14 +397,26 @@ __global__ void __launch_bounds__(kQ4Threads, 1) q4_down_kernel(Q4Params p) {
   if (!s_last) return;
   __threadfence();
   const long long n4 = (long long)p.T * d / 4;
-  for (long long i = tid; i < n4; i += blockDim.x) {
-    const float4 v = __ldcg(reinterpret_cast<const float4 *>(p.y_acc) + i);
-    __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
-    uint2 o;
-    o.x = *reinterpret_cast<uint32_t *>(&a);
-    o.y = *reinterpret_cast<uint32_t *>(&b);
-    reinterpret_cast<uint2 *>(p.y)[i] = o;
-    reinterpret_cast<float4 *>(p.y_acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  // eight independent L2 loads in flight per thread: the round trips overlap instead of adding up
+  for (long long i0 = tid; i0 < n4; i0 += 8LL * blockDim.x) {
+    float4 v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const long long i = i0 + (long long)j * blockDim.x;
+      v[j] = (i < n4) ? __ldcg(reinterpret_cast<const float4 *>(p.y_acc) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const long long i = i0 + (long long)j * blockDim.x;
+      if (i < n4) {
+        __nv_bfloat162 a = __floats2bfloat162_rn(v[j].x, v[j].y), b = __floats2bfloat162_rn(v[j].z, v[j].w);
+        uint2 o;
+        o.x = *reinterpret_cast<uint32_t *>(&a);
+        o.y = *reinterpret_cast<uint32_t *>(&b);
+        reinterpret_cast<uint2 *>(p.y)[i] = o;
+        reinterpret_cast<float4 *>(p.y_acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
   }
   if (tid == 0) *p.done = 0u;
 }

@@ -64,6 +64,7 @@ struct ft_moe {
   uint32_t *status_dev = nullptr;
   uint32_t *seq_dev = nullptr;
   uint32_t *done_dev = nullptr;          // CTA completion counter of the streaming MMA kernel
+  long long *trace_dev = nullptr;        // per-CTA clocks of the latest streaming-kernel launch
   uint2 *q4_hbuf = nullptr;              // int4 path: h of every (pass, 16-neuron block) in fragment order
   uint32_t seq_host = 0;                // plans launched
   float *stage_logits = nullptr;
@@ -295,6 +296,7 @@ ft_status_t ft_moe_destroy(ft_moe_t *h) {
   cudaFree(h->seq_dev);
   cudaFree(h->done_dev);
   cudaFree(h->q4_hbuf);
+  cudaFree(h->trace_dev);
   cudaFree(h->stage_logits);
   cudaFree(h->stage_x);
   cudaFree(h->stage_y);
@@ -443,6 +445,8 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
   FT_TRY(cudaMemset(h->status_dev, 0, 4));
   FT_TRY(cudaMalloc(&h->seq_dev, 4));
   FT_TRY(cudaMemset(h->seq_dev, 0, 4));
+  FT_TRY(cudaMalloc(&h->trace_dev, (size_t)h->sm_count * 4 * sizeof(long long)));
+  FT_TRY(cudaMemset(h->trace_dev, 0, (size_t)h->sm_count * 4 * sizeof(long long)));
   FT_TRY(cudaMalloc(&h->done_dev, 4));
   FT_TRY(cudaMemset(h->done_dev, 0, 4));
   if ((size_t)c.slots_per_layer * 16 + 36 * 1024 > 48 * 1024) {
@@ -714,6 +718,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     mp.n_zc = &h->plan_dev->n_zc_items;
     mp.pref = h->res_pref;
     mp.max_items = 2 * c.n_experts + 1;
+    mp.trace = h->trace_dev;
     mp.x = x_bf; mp.perm = h->perm; mp.topk_w = h->topk_w; mp.y_acc = h->y_acc;
     mp.y = static_cast<__nv_bfloat16 *>(y_dev);
     mp.done = h->done_dev; mp.status = h->status_dev;
@@ -933,6 +938,15 @@ ft_status_t ft_moe_last_fill(ft_moe_t *h, float *out_us, uint64_t *out_bytes) {
     bytes = (uint64_t)hd.n_fill * h->S;
   }
   if (out_bytes) *out_bytes = bytes;
+  return FT_OK;
+}
+
+ft_status_t ft_moe_get_cta_trace(ft_moe_t *h, int64_t *out, int n_ctas) {
+  if (!h || !out || n_ctas < 0) return FT_ERR_INVALID_ARG;
+  FT_CUDA(cudaSetDevice(h->cfg.device));
+  FT_CUDA(cudaDeviceSynchronize());
+  const int n = n_ctas < h->sm_count ? n_ctas : h->sm_count;
+  FT_CUDA(cudaMemcpy(out, h->trace_dev, (size_t)n * 4 * sizeof(long long), cudaMemcpyDeviceToHost));
   return FT_OK;
 }
 
