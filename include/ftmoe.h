@@ -110,6 +110,10 @@ typedef struct {
   int32_t hbm_tokens_per_pass;  /* T_g >= 1: tokens one resident weight pass serves                 */
   int32_t gemm_min_tokens;      /* experts with at least this many tokens and a slot use the
                                    tensor-core grouped GEMM; 0 = never                              */
+  int32_t split_min_pairs;      /* calls with T*top_k at or above this evaluate the hit experts in a
+                                   launch of their own while the fills are still in flight, the
+                                   filled experts after the fill event; 0 = always one launch after
+                                   the fills (cheaper for a few tokens)                             */
 } ft_moe_config_t;
 
 /* Host-visible plan of one (layer, step).  The caller provides arrays of n_experts int32 each. */

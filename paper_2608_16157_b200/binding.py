@@ -43,7 +43,7 @@ class Config(C.Structure):
         ("host_pool", C.c_void_p), ("host_pool_bytes", C.c_size_t), ("shared_weights", C.c_void_p),
         ("bw_fill_MBps", C.c_uint32), ("bw_zc_MBps", C.c_uint32), ("bw_zc_residual_MBps", C.c_uint32),
         ("bw_hbm_MBps", C.c_uint32), ("reuse_credit", C.c_int32), ("zc_tokens_per_pass", C.c_int32),
-        ("hbm_tokens_per_pass", C.c_int32), ("gemm_min_tokens", C.c_int32),
+        ("hbm_tokens_per_pass", C.c_int32), ("gemm_min_tokens", C.c_int32), ("split_min_pairs", C.c_int32),
     ]
 
 
@@ -130,7 +130,7 @@ def make_config(*, hidden, inter, n_experts, top_k, n_layers=1, slots_per_layer,
                 host_pool_ptr, host_pool_bytes, wdtype=FT_W_BF16, n_shared=0, shared_ptr=None,
                 fill_mode=FT_FILL_COPY_ENGINE, device=0, bw_fill=50000, bw_zc=50000, bw_zc_residual=0,
                 bw_hbm=6000000, reuse_credit=1, zc_tokens_per_pass=64, hbm_tokens_per_pass=128,
-                gemm_min_tokens=0) -> Config:
+                gemm_min_tokens=0, split_min_pairs=32) -> Config:
     c = Config()
     c.struct_size = C.sizeof(Config)
     c.device, c.n_layers, c.hidden, c.inter = device, n_layers, hidden, inter
@@ -140,6 +140,7 @@ def make_config(*, hidden, inter, n_experts, top_k, n_layers=1, slots_per_layer,
     c.bw_fill_MBps, c.bw_zc_MBps, c.bw_zc_residual_MBps, c.bw_hbm_MBps = bw_fill, bw_zc, bw_zc_residual, bw_hbm
     c.reuse_credit, c.zc_tokens_per_pass, c.hbm_tokens_per_pass = reuse_credit, zc_tokens_per_pass, hbm_tokens_per_pass
     c.gemm_min_tokens = gemm_min_tokens
+    c.split_min_pairs = split_min_pairs
     return c
 
 

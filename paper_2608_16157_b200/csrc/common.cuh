@@ -34,9 +34,10 @@ struct __align__(16) WorkItem {
 struct PlanHeader {
   int64_t step;
   int32_t n_routed, n_hit, n_miss, n_fill, n_zc;
-  int32_t n_res_items, n_zc_items, n_gemm_items;
+  int32_t n_res_items, n_zc_items, n_gemm_items;   // streaming list: [hits][shared][fills] = n_res_items, then zc
   uint32_t seq;      // incremented by every plan kernel; lets the host detect a stale record
-  int32_t pad[5];
+  int32_t n_hit_items;   // leading entries of the streaming list that do not depend on this step's fills
+  int32_t pad[4];
 };
 static_assert(sizeof(PlanHeader) == 64, "PlanHeader layout");
 

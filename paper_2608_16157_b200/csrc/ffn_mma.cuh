@@ -27,7 +27,9 @@ constexpr int kMmaTokens = 8;  // tokens per weight pass
 
 struct FfnMmaParams {
   const WorkItem *items;
-  const int32_t *n_items;   // resident items (records in HBM slots)
+  const int32_t *n_items;   // resident items (records in HBM slots): [hits][shared expert][fills]
+  const int32_t *n_hit;     // how many of them lead the list and do not depend on this step's fills
+  int part;                 // 0: everything; 1: hits + zero-copy items; 2: fills only
   const int32_t *n_zc;      // zero-copy items appended after them (records in the mapped host pool)
   const int32_t *pref;      // [n_items+1] exclusive prefix of the weight passes per item (from the plan)
   const __nv_bfloat16 *x;   // [T][d]
@@ -143,9 +145,14 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
   for (int i = tid; i <= p.max_items; i += blockDim.x) s_pref[i] = p.pref[i];
   __syncthreads();
   // two work ranges, each split evenly over the CTAs: HBM-resident blocks, then host-resident blocks (the
-  // latter are bound by the host link, so every CTA takes an equal share of them)
-  const long long total_res = (long long)s_pref[n_items] * NBLK;
-  const long long total_all = (long long)s_pref[n_items + n_zc] * NBLK;
+  // latter are bound by the host link, so every CTA takes an equal share of them).  `part` restricts the launch
+  // to the items that do not depend on the fills (plus the zero-copy items) or to the filled items.
+  const int n_hit = (p.part == 0) ? 0 : *p.n_hit;
+  const int a0 = (p.part == 2) ? n_hit : 0, a1 = (p.part == 1) ? n_hit : n_items;
+  const long long first_res = (long long)s_pref[a0] * NBLK;
+  const long long total_res = (long long)s_pref[a1] * NBLK;
+  const long long zc_begin = (long long)s_pref[n_items] * NBLK;
+  const long long total_all = (p.part == 2) ? zc_begin : (long long)s_pref[n_items + n_zc] * NBLK;
   int item = 0;
   uint32_t tile = 0;  // 16-neuron blocks consumed / produced so far by this CTA
 
@@ -154,7 +161,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
     // lane 0 waits for the stage and posts the byte count; lanes 0..15 then issue one row copy each, so the
     // issue rate of a single thread never limits the stream
     for (int range = 0; range < 2; ++range) {
-    const long long r0 = range ? total_res : 0, rn = range ? total_all - total_res : total_res;
+    const long long r0 = range ? zc_begin : first_res, rn = range ? total_all - zc_begin : total_res - first_res;
     long long u = r0 + rn * blockIdx.x / gridDim.x;
     const long long u1 = r0 + rn * (blockIdx.x + 1) / gridDim.x;
     while (u < u1) {
@@ -194,7 +201,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
     const int half = warp >> 2;             // which half of the rows' bytes this warp reads
     const int kl = (warp & 3) * (d / 8);    // the same offset inside that half
     for (int range = 0; range < 2; ++range) {
-    const long long r0 = range ? total_res : 0, rn = range ? total_all - total_res : total_res;
+    const long long r0 = range ? zc_begin : first_res, rn = range ? total_all - zc_begin : total_res - first_res;
     long long u = r0 + rn * blockIdx.x / gridDim.x;
     const long long u1 = r0 + rn * (blockIdx.x + 1) / gridDim.x;
     while (u < u1) {

@@ -113,6 +113,8 @@ extern "C" ft_status_t ft_moe_ffn_noalloc(int device, const void *record_dev, in
   mp.items = &ctl->item;
   mp.n_items = &ctl->n_items;
   mp.n_zc = &ctl->n_zc;
+  mp.n_hit = &ctl->n_zc;   // unused with part = 0
+  mp.part = 0;
   mp.pref = ctl->pref;
   mp.max_items = 1;
   mp.trace = nullptr;

@@ -324,7 +324,7 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
     return FT_ERR_INVALID_ARG;
   if (c.wdtype != FT_W_BF16 && c.wdtype != FT_W_INT4_G128) return FT_ERR_INVALID_ARG;
   if (c.bw_fill_MBps == 0 || c.bw_zc_MBps == 0 || c.bw_hbm_MBps == 0 || c.reuse_credit < 0 ||
-      c.zc_tokens_per_pass < 1 || c.hbm_tokens_per_pass < 1 || c.gemm_min_tokens < 0)
+      c.zc_tokens_per_pass < 1 || c.hbm_tokens_per_pass < 1 || c.gemm_min_tokens < 0 || c.split_min_pairs < 0)
     return FT_ERR_INVALID_ARG;
   const size_t S = expert_bytes_of(cfg);
   if (S == 0 || (c.wdtype == FT_W_INT4_G128 && !q4_shape_ok(c))) return FT_ERR_UNSUPPORTED;
@@ -454,6 +454,7 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
     FT_TRY(cudaFuncSetAttribute(plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn));
     FT_TRY(cudaFuncSetAttribute(route_plan_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn));
   }
+  FT_TRY(cudaFuncSetAttribute(fill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFillStages * (int)kFillChunk));
   if (c.wdtype == FT_W_INT4_G128) {
     const size_t passes = (P + 7) / 8 + 2 * E + 2;
     FT_TRY(cudaMalloc(&h->q4_hbuf, passes * (c.inter / 16) * 32 * sizeof(uint2)));
@@ -685,7 +686,7 @@ ft_status_t ft_moe_fill(ft_moe_t *h, int layer, void *copy_stream) {
     FT_CUDA(cudaEventRecord(h->ev_fill_t0, cs));
     {
       TimeScope ts(h, cs, FT_TIME_FILL);
-      fill_kernel<<<h->sm_count * 4, 256, 0, cs>>>(fp);
+      fill_kernel<<<kFillCtas, kFillThreads, kFillStages * kFillChunk, cs>>>(fp, h->status_dev);
     }
     h->launches++;
     FT_CUDA(cudaGetLastError());
@@ -707,14 +708,13 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const ft_moe_config_t &c = h->cfg;
   const __nv_bfloat16 *x_bf = static_cast<const __nv_bfloat16 *>(x_dev);
-  // resident set after the fills have landed
-  if (c.slots_per_layer > 0) FT_CUDA(cudaStreamWaitEvent(st, h->ev_fill, 0));
   const bool use_gemm = h->gemm && L.T >= c.gemm_min_tokens;
   if (c.wdtype == FT_W_BF16) {
-    // resident experts: bulk-copy pipelined tensor-core streaming kernel; its last CTA finalizes y
+    // bulk-copy pipelined tensor-core streaming kernel; the last CTA of the last launch finalizes y
     FfnMmaParams mp;
     mp.items = h->items_res;
     mp.n_items = &h->plan_dev->n_res_items;
+    mp.n_hit = &h->plan_dev->n_hit_items;
     mp.n_zc = &h->plan_dev->n_zc_items;
     mp.pref = h->res_pref;
     mp.max_items = 2 * c.n_experts + 1;
@@ -722,18 +722,34 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     mp.x = x_bf; mp.perm = h->perm; mp.topk_w = h->topk_w; mp.y_acc = h->y_acc;
     mp.y = static_cast<__nv_bfloat16 *>(y_dev);
     mp.done = h->done_dev; mp.status = h->status_dev;
-    mp.d = c.hidden; mp.inter = c.inter; mp.top_k = c.top_k; mp.T = L.T; mp.finalize = use_gemm ? 0 : 1;
+    mp.d = c.hidden; mp.inter = c.inter; mp.top_k = c.top_k; mp.T = L.T;
     const size_t smem = ffn_mma_smem_bytes(c.hidden);
-    {
-      TimeScope ts(h, st, FT_TIME_FFN_RES);
+    auto launch = [&](int part, int finalize) {
+      mp.part = part;
+      mp.finalize = finalize;
+      TimeScope ts(h, st, part == 1 ? FT_TIME_FFN_ZC : FT_TIME_FFN_RES);
+      // while the device-driven fill holds kFillCtas SMs, the overlapping launch takes the others
+      const int grid = (part == 1 && c.fill_mode == FT_FILL_SM) ? h->sm_count - kFillCtas : h->sm_count;
       switch (c.hidden / 256) {
-        case 1: ffn_mma_kernel<1><<<h->sm_count, kMmaThreads, smem, st>>>(mp); break;
-        case 2: ffn_mma_kernel<2><<<h->sm_count, kMmaThreads, smem, st>>>(mp); break;
-        case 4: ffn_mma_kernel<4><<<h->sm_count, kMmaThreads, smem, st>>>(mp); break;
-        default: ffn_mma_kernel<8><<<h->sm_count, kMmaThreads, smem, st>>>(mp); break;
+        case 1: ffn_mma_kernel<1><<<grid, kMmaThreads, smem, st>>>(mp); break;
+        case 2: ffn_mma_kernel<2><<<grid, kMmaThreads, smem, st>>>(mp); break;
+        case 4: ffn_mma_kernel<4><<<grid, kMmaThreads, smem, st>>>(mp); break;
+        default: ffn_mma_kernel<8><<<grid, kMmaThreads, smem, st>>>(mp); break;
       }
+      h->launches++;
+    };
+    // With enough tokens in the call the hits (and the zero-copy experts) are worth a launch of their own that
+    // overlaps the fills; the filled experts follow once the fill event has fired.  With few tokens the extra
+    // launch costs more than the overlap buys, so everything goes in one launch after the fills.
+    const bool split = c.slots_per_layer > 0 && (long long)L.T * c.top_k >= c.split_min_pairs && c.split_min_pairs > 0;
+    if (split) {
+      launch(1, 0);
+      FT_CUDA(cudaStreamWaitEvent(st, h->ev_fill, 0));
+      launch(2, use_gemm ? 0 : 1);
+    } else {
+      if (c.slots_per_layer > 0) FT_CUDA(cudaStreamWaitEvent(st, h->ev_fill, 0));
+      launch(0, use_gemm ? 0 : 1);
     }
-    h->launches++;
     FT_CUDA(cudaGetLastError());
     if (use_gemm) {
       // experts with many tokens: gather x rows into expert order, two grouped tcgen05 GEMMs, fused combine
@@ -767,6 +783,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     return FT_OK;
   }
   // int4: gate/up kernel writes h, down kernel accumulates, its last CTA finalizes y
+  if (c.slots_per_layer > 0) FT_CUDA(cudaStreamWaitEvent(st, h->ev_fill, 0));
   Q4Params qp;
   qp.items = h->items_res;
   qp.n_items = &h->plan_dev->n_res_items;

@@ -237,19 +237,26 @@ __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, uns
   const int use_gemm = resident && p.cm.gemm_min_tokens > 0 && c >= p.cm.gemm_min_tokens;
   const int res_stream = resident && !use_gemm;
   if (resident) atomicAdd(&sm.pairs_res, c);   // a sum: order-free; read after the scans' barriers
+  // The streaming kernel's list: [hits][shared expert][fills][zero-copy], so that the hits can be evaluated
+  // while the fills are still in flight.
+  const int hs = res_stream && cls == 1, fs = res_stream && is_fill;
   unsigned long long totB;
-  const unsigned long long exB = block_excl_scan64(pack4(is_fill, is_zc, res_stream, use_gemm), sm.w, totB);
-  const int n_fill = unpack(totB, 0), n_zc = unpack(totB, 1), n_res = unpack(totB, 2), n_gemm = unpack(totB, 3);
-  // weight passes (tokens_per_pass tokens each): low word for the resident streaming items, high word for the
-  // zero-copy items, which the streaming kernel finds appended to the same list
+  const unsigned long long exB = block_excl_scan64(
+      pack4(is_fill, is_zc, hs, use_gemm) | ((unsigned long long)fs << (4 * kPlanField)), sm.w, totB);
+  const int n_fill = unpack(totB, 0), n_zc = unpack(totB, 1), n_hs = unpack(totB, 2), n_gemm = unpack(totB, 3);
+  const int n_fs = unpack(totB, 4);
+  // weight passes (tokens_per_pass tokens each) of the list entries, in list order
   const int passes = (res_stream || (is_zc && !p.zc_single_pass)) ? (c + p.tokens_per_pass - 1) / p.tokens_per_pass
                                                                   : (is_zc ? 1 : 0);
-  unsigned long long totC;
+  unsigned long long totC, totZ;
   const unsigned long long exC = block_excl_scan64(
-      ((unsigned long long)(is_zc ? passes : 0) << 32) | (unsigned long long)(res_stream ? passes : 0), sm.w, totC);
+      ((unsigned long long)(fs ? passes : 0) << 32) | (unsigned long long)(hs ? passes : 0), sm.w, totC);
+  const unsigned long long exZ = block_excl_scan64((unsigned long long)(is_zc ? passes : 0), sm.w, totZ);
   const int n_shared_items = (p.shared_rec != nullptr) ? 1 : 0;
   const int shared_passes = n_shared_items ? (p.T + p.tokens_per_pass - 1) / p.tokens_per_pass : 0;
-  const int res_pass_total = (int)(totC & 0xffffffffull) + shared_passes;
+  const int pass_hits = (int)(totC & 0xffffffffull) + shared_passes;   // passes before the first fill
+  const int pass_res = pass_hits + (int)(totC >> 32);                   // passes before the first zero-copy item
+  const int n_hit_items = n_hs + n_shared_items, n_res_items = n_hit_items + n_fs;
   if (p.cm.gemm_min_tokens > 0) {   // uniform branch: only prefill-capable handles pay for this scan
     unsigned long long totD;
     const unsigned long long exD = block_excl_scan64(
@@ -273,9 +280,12 @@ __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, uns
     it.slot = loc;
     if (use_gemm) {
       p.items_gemm[unpack(exB, 3)] = it;
-    } else {
+    } else if (hs) {
       p.items_res[unpack(exB, 2)] = it;
       p.res_pref[unpack(exB, 2)] = (int32_t)(exC & 0xffffffffull);
+    } else {
+      p.items_res[n_hit_items + unpack(exB, 4)] = it;
+      p.res_pref[n_hit_items + unpack(exB, 4)] = pass_hits + (int32_t)(exC >> 32);
     }
   }
   if (is_zc) {
@@ -286,13 +296,12 @@ __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, uns
     it.off = off;
     it.slot = -1;
     p.items_zc[unpack(exB, 1)] = it;
-    const int zi = n_res + n_shared_items + unpack(exB, 1);   // appended after the resident items
+    const int zi = n_res_items + unpack(exB, 1);   // appended after the resident items
     p.items_res[zi] = it;
-    p.res_pref[zi] = res_pass_total + (int32_t)(exC >> 32);
+    p.res_pref[zi] = pass_res + (int32_t)exZ;
   }
 
   if (tid == 0) {
-    const int n_res_items = n_res + n_shared_items;
     if (n_shared_items) {
       WorkItem it;
       it.w = p.shared_rec;
@@ -300,17 +309,19 @@ __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, uns
       it.n_tok = p.T;
       it.off = 0;
       it.slot = -1;
-      p.items_res[n_res] = it;
-      p.res_pref[n_res] = (int)(totC & 0xffffffffull);
+      p.items_res[n_hs] = it;
+      p.res_pref[n_hs] = (int)(totC & 0xffffffffull);
     }
-    p.res_pref[n_res_items + n_zc] = res_pass_total + (int)(totC >> 32);
-    if (n_zc == 0) p.res_pref[n_res_items] = res_pass_total;
+    if (n_fs == 0) p.res_pref[n_hit_items] = pass_hits;
+    if (n_zc == 0) p.res_pref[n_res_items] = pass_res;
+    p.res_pref[n_res_items + n_zc] = pass_res + (int)totZ;
     PlanHeader h;
     h.step = t;
     h.n_routed = n_routed; h.n_hit = n_hit; h.n_miss = n_miss; h.n_fill = n_fill; h.n_zc = n_zc;
     h.n_res_items = n_res_items; h.n_zc_items = n_zc; h.n_gemm_items = n_gemm;
     h.seq = p.seq_value;
-    h.pad[0] = h.pad[1] = h.pad[2] = h.pad[3] = h.pad[4] = 0;
+    h.n_hit_items = n_hit_items;
+    h.pad[0] = h.pad[1] = h.pad[2] = h.pad[3] = 0;
     *p.hdr_dev = h;
     *p.step = t + 1;
     int evictions = 0;
