@@ -37,12 +37,13 @@ def open_shared_pool(n_bytes: int, tag: str, rank: int, barrier, fill=None, path
 
 def close_shared_pool(arr, name: str, rank: int, barrier) -> None:
     del arr
-    barrier()
+    barrier()                      # nobody uses the mapping any more
     if rank == 0:
         try:
             os.unlink(name)
         except OSError:
             pass
+    barrier()                      # the file is gone when any rank returns
 
 
 def max_over_ranks(value: float, dist=None, device=None) -> float:
