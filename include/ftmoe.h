@@ -45,7 +45,7 @@
  *   Shape limits: bf16: hidden in {256, 512, 1024, 2048}, inter % 16 == 0; int4: hidden in
  *   {512, 1024, 2048, 4096, 7168, 8192}, inter % 128 == 0; n_experts <= 1024;
  *   top_k <= min(n_experts, 32); slots_per_layer <= 2048.  The tensor-core prefill path
- *   (gemm_min_tokens > 0) needs bf16 weights, slots_per_layer > 0 and inter % 128 == 0.
+ *   (gemm_min_tokens > 0) needs bf16 weights, slots_per_layer > 0 and inter % 256 == 0.
  */
 #ifndef FTMOE_H_
 #define FTMOE_H_

@@ -12,6 +12,7 @@
 #include "ffn_mma.cuh"
 #include "ffn_q4.cuh"
 #include "gemm_tc.cuh"
+#include "gemm_tc2.cuh"
 #include "fill.cuh"
 #include "route_plan.cuh"
 
@@ -60,7 +61,7 @@ struct ft_moe {
   int32_t *gemm_pref = nullptr;
   uint8_t *is_gemm = nullptr;
   __nv_bfloat16 *xs = nullptr, *hbuf = nullptr, *obuf = nullptr;   // [P][d], [P][I], [P][d]
-  CUtensorMap tm_xs, tm_h, tm_w128, tm_w64;
+  CUtensorMap tm_xs, tm_h, tm_w128, tm_w64;   // x rows, H rows (128-row boxes), weight rows (128 / 64-row boxes)
   uint32_t *status_dev = nullptr;
   uint32_t *seq_dev = nullptr;
   uint32_t *done_dev = nullptr;          // CTA completion counter of the streaming MMA kernel
@@ -329,7 +330,7 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
   const size_t S = expert_bytes_of(cfg);
   if (S == 0 || (c.wdtype == FT_W_INT4_G128 && !q4_shape_ok(c))) return FT_ERR_UNSUPPORTED;
   if (c.gemm_min_tokens != 0 &&
-      (c.wdtype != FT_W_BF16 || c.slots_per_layer == 0 || c.hidden % 256 || c.inter % 128 || c.gemm_min_tokens < 8))
+      (c.wdtype != FT_W_BF16 || c.slots_per_layer == 0 || c.hidden % 256 || c.inter % 256 || c.gemm_min_tokens < 8))
     return FT_ERR_UNSUPPORTED;
   if (!c.host_pool || c.host_pool_bytes < (size_t)c.n_layers * c.n_experts * S) return FT_ERR_INVALID_ARG;
   if (c.n_shared && !c.shared_weights) return FT_ERR_INVALID_ARG;
@@ -414,7 +415,7 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
   FT_TRY(cudaMalloc(&h->res_pref, (2 * E + 2) * 4));
   FT_TRY(cudaMemset(h->res_pref, 0, (2 * E + 2) * 4));
   if (c.gemm_min_tokens > 0) {
-    const size_t Pr = P + 128;   // one spare tile of rows so that full boxes stay inside the tensors
+    const size_t Pr = P + 256;   // spare rows so that full boxes stay inside the tensors
     FT_TRY(cudaMalloc(&h->gemm_pref, (E + 1) * 4));
     FT_TRY(cudaMemset(h->gemm_pref, 0, (E + 1) * 4));
     FT_TRY(cudaMalloc(&h->is_gemm, E));
@@ -437,8 +438,8 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
       return fail(FT_ERR_CUDA);
     FT_TRY(cudaFuncSetAttribute(grouped_gemm_kernel<0, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)grouped_gemm_smem_bytes<1>()));
-    FT_TRY(cudaFuncSetAttribute(grouped_gemm_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)grouped_gemm_smem_bytes<1>()));
+    FT_TRY(cudaFuncSetAttribute(grouped_gemm2_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)grouped_gemm2_smem_bytes<1>()));
     h->gemm = true;
   }
   FT_TRY(cudaMalloc(&h->status_dev, 4));
@@ -762,15 +763,29 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
       gp.inter = c.inter; gp.d = c.hidden;
       gp.layer_row0 = (long long)layer * c.slots_per_layer * 3 * c.inter;
       gp.status = h->status_dev;
+      // CTA pairs (clusters of two) share every 256x256 tile
+      cudaLaunchConfig_t lc = {};
+      lc.gridDim = dim3((unsigned)(h->sm_count & ~1));
+      lc.blockDim = dim3(kGemmThreads);
+      lc.stream = st;
+      cudaLaunchAttribute la[1];
+      la[0].id = cudaLaunchAttributeClusterDimension;
+      la[0].val.clusterDim.x = 2; la[0].val.clusterDim.y = 1; la[0].val.clusterDim.z = 1;
+      lc.attrs = la;
+      lc.numAttrs = 1;
+      // gate/up + SwiGLU: one CTA per 128 x 256 tile (A = x rows, B = 128 gate + 128 up rows); measured faster
+      // than the CTA-pair form for this GEMM, whose fused epilogue needs gate and up in the same TMEM
       gp.K = c.hidden; gp.n_tiles = c.inter / 128; gp.out = h->hbuf;
       {
         TimeScope ts(h, st, FT_TIME_GEMM1);
         grouped_gemm_kernel<0, 1><<<h->sm_count, kGemmThreads, grouped_gemm_smem_bytes<1>(), st>>>(h->tm_xs, h->tm_w128, gp);
       }
-      gp.K = c.inter; gp.n_tiles = c.hidden / kGemmBN; gp.out = h->obuf;
+      // down: A = Wd[k][column] (box 64 columns x 64 k rows, twice), B = H rows (box 64 x 128 per CTA)
+      gp.K = c.inter; gp.out = h->obuf;
+      lc.dynamicSmemBytes = grouped_gemm2_smem_bytes<1>();
       {
         TimeScope ts(h, st, FT_TIME_GEMM2);
-        grouped_gemm_kernel<1, 1><<<h->sm_count, kGemmThreads, grouped_gemm_smem_bytes<1>(), st>>>(h->tm_h, h->tm_w64, gp);
+        FT_CUDA(cudaLaunchKernelEx(&lc, grouped_gemm2_kernel<1>, h->tm_w64, h->tm_h, gp));
       }
       {
         TimeScope ts(h, st, FT_TIME_COMBINE);
