@@ -153,41 +153,69 @@ __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, uns
   // (the scan's barriers make the refreshed stamps in shared memory visible to the whole block)
   const int lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   int K = 0;
-  for (int base = 0; base < p.n_slots; base += 32) {
-    const int o = base + lane;
-    const bool oc = (o < p.n_slots) && ((s_sexp[o] < 0) || (s_stamp[o] < t));
-    K += __popc(__ballot_sync(0xffffffffu, oc));
-  }
-  for (int s = warp; s < p.n_slots; s += nwarps) {
-    const int64_t st = s_stamp[s];
-    const int ex = s_sexp[s];
-    if (!((ex < 0) || (st < t))) continue;      // warp-uniform
-    int rank = 0;
+  int q = 0;
+  if (n_miss > 0) {    // block-uniform: with no miss there is nothing to evict or fill
     for (int base = 0; base < p.n_slots; base += 32) {
       const int o = base + lane;
-      bool before = false;
-      if (o < p.n_slots && o != s) {
-        const int oex = s_sexp[o];
-        const int64_t ost = s_stamp[o];
-        if ((oex < 0) || (ost < t)) {
-          if (oex < 0) before = (ex >= 0) || (o < s);
-          else if (ex >= 0) before = (ost < st) || (ost == st && oex < ex);
-        }
-      }
-      rank += __popc(__ballot_sync(0xffffffffu, before));
+      const bool oc = (o < p.n_slots) && ((s_sexp[o] < 0) || (s_stamp[o] < t));
+      K += __popc(__ballot_sync(0xffffffffu, oc));
     }
-    if (lane == 0) s_victim[rank] = s;
-  }
-
-  // ---- 5: fill count
-  int q = 0;
-  if (n_miss > 0) {
+    // ---- 5: fill count
     const int64_t bt = p.cm.bw_fill + p.cm.bw_res;
     int64_t qbw = (2 * (int64_t)n_miss * p.cm.bw_fill + bt) / (2 * bt);
     if (qbw < 1) qbw = 1;
     q = (int)qbw;
     if (q > n_elig) q = n_elig;
     if (q > K) q = K;
+    // The order key of a candidate slot: free slots by index, then occupied ones by (stamp, resident expert id);
+    // keys are distinct, non-candidates get the largest value.
+    auto slot_key = [&](int o) -> unsigned long long {
+      if (o >= p.n_slots) return ~0ull;
+      const int oex = s_sexp[o];
+      const int64_t ost = s_stamp[o];
+      if (oex < 0) return (unsigned long long)o;
+      if (ost >= t) return ~0ull;
+      return (1ull << 62) | ((unsigned long long)(ost + 1) << 20) | (unsigned long long)oex;
+    };
+    if (q <= 8 && p.n_slots <= 256) {
+      // few fills (decode): warp 0 extracts the q smallest keys one after the other (q warp-wide minima)
+      if (warp == 0) {
+        unsigned long long key[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) key[i] = slot_key(lane + 32 * i);
+        for (int r = 0; r < q; ++r) {
+          unsigned long long best = key[0];
+          int bslot = lane;
+#pragma unroll
+          for (int i = 1; i < 8; ++i)
+            if (key[i] < best) { best = key[i]; bslot = lane + 32 * i; }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const unsigned long long ob = __shfl_xor_sync(0xffffffffu, best, o);
+            const int os = __shfl_xor_sync(0xffffffffu, bslot, o);
+            if (ob < best) { best = ob; bslot = os; }
+          }
+          if (lane == 0) s_victim[r] = bslot;
+          if ((bslot & 31) == lane) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              if (i == (bslot >> 5)) key[i] = ~0ull;
+          }
+        }
+      }
+    } else {
+      // many fills (prefill): every candidate is ranked in one pass, 32 slots per ballot
+      for (int s = warp; s < p.n_slots; s += nwarps) {
+        const unsigned long long ks = slot_key(s);
+        if (ks == ~0ull) continue;      // warp-uniform
+        int rank = 0;
+        for (int base = 0; base < p.n_slots; base += 32) {
+          const int o = base + lane;
+          rank += __popc(__ballot_sync(0xffffffffu, o != s && slot_key(o) < ks));
+        }
+        if (lane == 0) s_victim[rank] = s;
+      }
+    }
   }
 
   // ---- 6: priority of the eligible misses (tokens descending, id ascending): each warp ranks a few misses

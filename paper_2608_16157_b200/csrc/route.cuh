@@ -43,6 +43,11 @@ __device__ __forceinline__ void route_token(const float *__restrict__ z, int E, 
     v[i] = x;
   }
   if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(status, kStatNonFinite);
+  // order-preserving map float -> uint32 (-0 folded into +0), so that a warp maximum is one redux instruction
+  auto ordered = [](float x) -> uint32_t {
+    const uint32_t u = __float_as_uint(x + 0.f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+  };
   float my_v = 0.f;
   int my_i = 0;
   for (int r = 0; r < k; ++r) {
@@ -53,12 +58,12 @@ __device__ __forceinline__ void route_token(const float *__restrict__ z, int E, 
       const int e = lane + 32 * i;
       if (e < E && route_better(v[i], e, bv, bi)) { bv = v[i]; bi = e; }
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-      if (route_better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
-    }
+    // warp arg-max in the total order (value descending, index ascending): maximum of the values, then the
+    // smallest index among the lanes that hold it
+    const uint32_t mx = __reduce_max_sync(0xffffffffu, ordered(bv));
+    const uint32_t cand = (ordered(bv) == mx) ? (uint32_t)bi : 0xffffffffu;
+    bi = (int)__reduce_min_sync(0xffffffffu, cand);
+    bv = __shfl_sync(0xffffffffu, bv, bi & 31);
     if (bi == 0x7fffffff) bi = 0;  // only reachable with non-finite input (already latched)
     if (lane == r) { my_v = bv; my_i = bi; }
     if ((bi & 31) == lane) {
