@@ -221,6 +221,9 @@ ft_status_t ft_moe_timing_read(ft_moe_t *h, double *out_us, uint64_t *out_launch
  * touched (for the CTA that finalized y: minus the global timer when it finished).  n_ctas
  * entries at most (one CTA per SM).  Waits for the device. */
 ft_status_t ft_moe_get_cta_trace(ft_moe_t *h, int64_t *out, int n_ctas);
+/* Changes split_min_pairs of a live handle (see ft_moe_config_t); takes effect at the next ft_moe_forward.
+ * Used to time the streaming kernel alone (0) or overlapped with the fills. */
+ft_status_t ft_moe_set_split_min_pairs(ft_moe_t *h, int pairs);
 /* Number of kernels this handle has launched since create. */
 ft_status_t ft_moe_launch_count(ft_moe_t *h, uint64_t *out);
 const char *ft_moe_status_string(ft_status_t s);

@@ -28,7 +28,7 @@ SYMBOLS = (
     "ft_moe_get_stats", "ft_moe_reset", "ft_moe_sync_status", "ft_moe_last_fill", "ft_moe_launch_count",
     "ft_moe_status_string", "ft_moe_timing_enable", "ft_moe_timing_read", "ft_moe_ffn_noalloc",
     "ft_moe_last_cuda_error", "ft_moe_host_register", "ft_moe_host_unregister",
-    "ft_moe_get_cta_trace",
+    "ft_moe_get_cta_trace", "ft_moe_set_split_min_pairs",
 )
 NOALLOC_MAX_TOKENS, NOALLOC_MAX_HIDDEN = 64, 2048
 TIME_NAMES = ("route", "plan", "ffn_zc", "ffn_res", "finalize", "fill", "gather", "gemm1", "gemm2", "combine")
@@ -85,6 +85,7 @@ def load(rebuild: bool = False):
         "ft_moe_host_free": (i32, [vp]),
         "ft_moe_host_register": (i32, [vp, sz]),
         "ft_moe_get_cta_trace": (i32, [vp, vp, i32]),
+        "ft_moe_set_split_min_pairs": (i32, [vp, i32]),
         "ft_moe_host_unregister": (i32, [vp]),
         "ft_moe_create": (i32, [C.POINTER(Config), C.POINTER(vp)]),
         "ft_moe_destroy": (i32, [vp]),
@@ -338,6 +339,9 @@ class FtMoe:
         a = np.zeros((n_ctas, 4), dtype=np.int64)
         _check(self._lib.ft_moe_get_cta_trace(self._h, _ptr(a), n_ctas), "ft_moe_get_cta_trace")
         return a
+
+    def set_split_min_pairs(self, pairs):
+        _check(self._lib.ft_moe_set_split_min_pairs(self._h, int(pairs)), "ft_moe_set_split_min_pairs")
 
     def launch_count(self):
         n = C.c_uint64()

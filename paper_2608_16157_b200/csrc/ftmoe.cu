@@ -982,6 +982,12 @@ ft_status_t ft_moe_get_cta_trace(ft_moe_t *h, int64_t *out, int n_ctas) {
   return FT_OK;
 }
 
+ft_status_t ft_moe_set_split_min_pairs(ft_moe_t *h, int pairs) {
+  if (!h || pairs < 0) return FT_ERR_INVALID_ARG;
+  h->cfg.split_min_pairs = pairs;
+  return FT_OK;
+}
+
 ft_status_t ft_moe_launch_count(ft_moe_t *h, uint64_t *out) {
   if (!h || !out) return FT_ERR_INVALID_ARG;
   *out = h->launches;
