@@ -15,14 +15,14 @@ struct FillParams {
   size_t S;                       // multiple of 16
 };
 
-constexpr int kFillCtas = 8;             // the copy needs bytes in flight, not SMs: 8 CTAs x 4 x 32 KiB
+constexpr int kFillCtas = 2;             // the copy needs bytes in flight, not SMs: 2 CTAs x 4 x 32 KiB saturate the link
 constexpr int kFillStages = 4;
 constexpr uint32_t kFillChunk = 32768;   // bytes per bulk copy
 constexpr int kFillThreads = 32;
 
 // A few single-warp CTAs move the records with the bulk-copy engine: host pool -> shared memory
 // (cp.async.bulk, completion on an mbarrier) -> slot (cp.async.bulk shared -> global).  No SM arithmetic, no
-// registers per byte, and only kFillCtas SMs are touched, so the expert kernel keeps the rest of the GPU
+// registers per byte, and only kFillCtas SMs are touched (more CTAs were measured to slow the concurrent expert kernel without raising the link rate), so the expert kernel keeps the rest of the GPU
 // while records stream in over the host link.
 __global__ void __launch_bounds__(kFillThreads) fill_kernel(FillParams p, uint32_t *status) {
   extern __shared__ __align__(128) unsigned char smem[];
