@@ -1,6 +1,7 @@
 // Shared device-side declarations of the expert-cached MoE layer library.
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 

@@ -83,7 +83,7 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t
 }
 __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
-  asm volatile(
+  asm(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
@@ -275,6 +275,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
           for (int which = 0; which < 2; ++which) {
             const int s = 2 * which + half;
             cgu[which][0] = cgu[which][1] = cgu[which][2] = cgu[which][3] = 0.f;
+            float c2[4] = {0.f, 0.f, 0.f, 0.f};   // second accumulator: consecutive MMAs do not wait for each other
             const bool ok = mbar_wait(full_bar(s), ph, s_abort, p.status);
             if (ok) {
               const uint32_t base = smem_base + s * stage_bytes + (uint32_t)(kl + 8 * q) * 2u;
@@ -283,9 +284,11 @@ __global__ void __launch_bounds__(kMmaThreads, 1) ffn_mma_kernel(FfnMmaParams p)
                 const uint4 lo = lds_v4(base + g * stride_gu + kb * 64);
                 const uint4 hi = lds_v4(base + (g + 8) * stride_gu + kb * 64);
                 mma_bf16(cgu[which], lo.x, hi.x, lo.y, hi.y, xf[kb][0], xf[kb][1]);
-                mma_bf16(cgu[which], lo.z, hi.z, lo.w, hi.w, xf[kb][2], xf[kb][3]);
+                mma_bf16(c2, lo.z, hi.z, lo.w, hi.w, xf[kb][2], xf[kb][3]);
               }
             }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) cgu[which][i] += c2[i];
             __syncwarp();
             if (last && lane == 0) mbar_arrive(empty_bar(s));
           }

@@ -465,12 +465,12 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
     FT_TRY(cudaFuncSetAttribute(q4_gateup_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
     FT_TRY(cudaFuncSetAttribute(q4_gateup_kernel<7>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
     FT_TRY(cudaFuncSetAttribute(q4_gateup_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(q4_down_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
     FT_TRY(cudaFuncSetAttribute(q4_down_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
     FT_TRY(cudaFuncSetAttribute(q4_down_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
     FT_TRY(cudaFuncSetAttribute(q4_down_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
+    FT_TRY(cudaFuncSetAttribute(q4_down_kernel<14>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
     FT_TRY(cudaFuncSetAttribute(q4_down_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
-    FT_TRY(cudaFuncSetAttribute(q4_down_kernel<28>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
-    FT_TRY(cudaFuncSetAttribute(q4_down_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
   }
   if (c.wdtype == FT_W_BF16) {
     const int smem = (int)ffn_mma_smem_bytes(c.hidden);
@@ -811,7 +811,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   qp.done = h->done_dev; qp.status = h->status_dev;
   qp.d = c.hidden; qp.inter = c.inter; qp.top_k = c.top_k; qp.T = L.T; qp.finalize = 1;
   const size_t sa = q4_gateup_smem_bytes(c.hidden), sb = q4_down_smem_bytes(c.hidden);
-  const int grid = h->sm_count & ~1;   // CTA pairs split the columns in the down kernel
+  const int grid = h->sm_count & ~3;   // groups of four CTAs split the columns in the down kernel
   {
     TimeScope ts(h, st, FT_TIME_FFN_ZC);   // (timing slot reused for the gate/up kernel of the int4 path)
     switch (c.hidden) {
@@ -826,12 +826,12 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   {
     TimeScope ts(h, st, FT_TIME_FFN_RES);
     switch (c.hidden) {
-      case 512: q4_down_kernel<2><<<grid, kQ4Threads, sb, st>>>(qp); break;
-      case 1024: q4_down_kernel<4><<<grid, kQ4Threads, sb, st>>>(qp); break;
-      case 2048: q4_down_kernel<8><<<grid, kQ4Threads, sb, st>>>(qp); break;
-      case 4096: q4_down_kernel<16><<<grid, kQ4Threads, sb, st>>>(qp); break;
-      case 7168: q4_down_kernel<28><<<grid, kQ4Threads, sb, st>>>(qp); break;
-      default: q4_down_kernel<32><<<grid, kQ4Threads, sb, st>>>(qp); break;
+      case 512: q4_down_kernel<1><<<grid, kQ4Threads, sb, st>>>(qp); break;
+      case 1024: q4_down_kernel<2><<<grid, kQ4Threads, sb, st>>>(qp); break;
+      case 2048: q4_down_kernel<4><<<grid, kQ4Threads, sb, st>>>(qp); break;
+      case 4096: q4_down_kernel<8><<<grid, kQ4Threads, sb, st>>>(qp); break;
+      case 7168: q4_down_kernel<14><<<grid, kQ4Threads, sb, st>>>(qp); break;
+      default: q4_down_kernel<16><<<grid, kQ4Threads, sb, st>>>(qp); break;
     }
   }
   h->launches += 2;
