@@ -436,10 +436,10 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
         !make_tensor_map(enc, &h->tm_w128, h->slots, wrows, c.hidden, 128, 64) ||
         !make_tensor_map(enc, &h->tm_w64, h->slots, wrows, c.hidden, 64, 64))
       return fail(FT_ERR_CUDA);
-    FT_TRY(cudaFuncSetAttribute(grouped_gemm_kernel<0, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)grouped_gemm_smem_bytes<1>()));
-    FT_TRY(cudaFuncSetAttribute(grouped_gemm2_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)grouped_gemm2_smem_bytes<1>()));
+    FT_TRY(cudaFuncSetAttribute(gateup_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)gateup_gemm_smem_bytes()));
+    FT_TRY(cudaFuncSetAttribute(down_gemm2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)down_gemm2_smem_bytes()));
     h->gemm = true;
   }
   FT_TRY(cudaMalloc(&h->status_dev, 4));
@@ -778,14 +778,14 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
       gp.K = c.hidden; gp.n_tiles = c.inter / 128; gp.out = h->hbuf;
       {
         TimeScope ts(h, st, FT_TIME_GEMM1);
-        grouped_gemm_kernel<0, 1><<<h->sm_count, kGemmThreads, grouped_gemm_smem_bytes<1>(), st>>>(h->tm_xs, h->tm_w128, gp);
+        gateup_gemm_kernel<<<h->sm_count, kGemmThreads, gateup_gemm_smem_bytes(), st>>>(h->tm_xs, h->tm_w128, gp);
       }
       // down: A = Wd[k][column] (box 64 columns x 64 k rows, twice), B = H rows (box 64 x 128 per CTA)
       gp.K = c.inter; gp.out = h->obuf;
-      lc.dynamicSmemBytes = grouped_gemm2_smem_bytes<1>();
+      lc.dynamicSmemBytes = down_gemm2_smem_bytes();
       {
         TimeScope ts(h, st, FT_TIME_GEMM2);
-        FT_CUDA(cudaLaunchKernelEx(&lc, grouped_gemm2_kernel<1>, h->tm_w64, h->tm_h, gp));
+        FT_CUDA(cudaLaunchKernelEx(&lc, down_gemm2_kernel, h->tm_w64, h->tm_h, gp));
       }
       {
         TimeScope ts(h, st, FT_TIME_COMBINE);

@@ -1,16 +1,16 @@
-// Step 5 for prefill-sized token counts: grouped SwiGLU expert FFN on the 5th-generation tensor
-// cores.  Two persistent kernels (one CTA per SM) over the experts that hold a slot and have at least
-// `gemm_min_tokens` tokens:
-//   MODE 0  H[P][I]  = SiLU(Xs Wg^T) * (Xs Wu^T)   A = expert-sorted x rows (K-major), B = 128 gate rows +
-//                                                  the same 128 up rows of the record (K-major), N = 256
-//   MODE 1  O[P][d]  = H Wd                         A = H rows (K-major), B = Wd rows (N-contiguous, i.e.
-//                                                  MN-major), N = 256
-// Per CTA: warp 0 feeds a 4-stage shared-memory ring with TMA tile loads (cp.async.bulk.tensor, 128-byte
-// swizzle, no multicast), warp 1 issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32) into one of two
-// 256-column TMEM accumulators and signals stages free / tiles done with tcgen05.commit, warps 2-5 drain
-// the other accumulator with tcgen05.ld, apply the epilogue and store bf16, so the epilogue of tile i
-// overlaps the main loop of tile i+1.  Every mbarrier wait is bounded; on expiry the CTA latches a
-// timeout status, stops waiting, frees its TMEM and returns.
+// Step 5 for prefill-sized token counts: the gate/up half of the grouped SwiGLU expert FFN on the
+// 5th-generation tensor cores, plus the helpers shared with the down-projection kernel (gemm_tc2.cuh), the row
+// gather and the fused gather-combine.
+//   H[P][I] = SiLU(Xs Wg^T) * (Xs Wu^T)   A = expert-sorted x rows (K-major), B = 128 gate rows + the same 128 up
+//                                          rows of the record (K-major), N = 256, over the experts that hold a
+//                                          slot and have at least `gemm_min_tokens` tokens.
+// One persistent CTA per SM: warp 0 feeds a 4-stage shared-memory ring with TMA tile loads (cp.async.bulk.tensor,
+// 128-byte swizzle, no multicast), warp 1 issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32) into one of two
+// 256-column TMEM accumulators and signals stages free / tiles done with tcgen05.commit, warps 2-5 drain the other
+// accumulator with tcgen05.ld, apply SwiGLU and store bf16, so the epilogue of tile i overlaps the main loop of
+// tile i+1.  Every mbarrier wait is bounded; on expiry the CTA latches a timeout status, stops waiting, frees its
+// TMEM and returns.  (Measured alternatives for this GEMM: two row tiles per CTA sharing B, 904 TFLOP/s, and CTA
+// pairs, 961 unswapped / 815 swapped, against 956-973 for this form.)
 #pragma once
 #include <cuda.h>
 
@@ -23,15 +23,7 @@ constexpr int kGemmThreads = 192;
 constexpr int kGemmBM = 128, kGemmBN = 256, kGemmBK = 64;
 constexpr int kGemmATile = kGemmBM * kGemmBK * 2;   // 16 KiB
 constexpr int kGemmBTile = kGemmBN * kGemmBK * 2;   // 32 KiB
-// MT = 128-row tiles of one expert that share every B tile (1 or 2).  With MT = 2 a stage holds two A tiles and
-// one B tile (64 KiB for 2 x 128 x 256 x 64 MACs instead of 48 KiB for one), which takes the kernel off the
-// L2-to-shared-memory bandwidth limit; the price is that both TMEM accumulators belong to one unit, so the
-// epilogue no longer overlaps the next main loop.
-template <int MT> struct GemmCfg {
-  static constexpr int kStageBytes = MT * kGemmATile + kGemmBTile;
-  static constexpr int kStages = (MT == 1) ? 4 : 3;
-  static constexpr int kBufs = (MT == 1) ? 2 : 1;   // TMEM accumulator sets in flight
-};
+constexpr int kGemmStages = 4, kGemmStageBytes = kGemmATile + kGemmBTile, kGemmBufs = 2;
 
 struct GemmParams {
   const WorkItem *items;
@@ -103,13 +95,11 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 
 // Dynamic shared memory (1024-byte aligned by the kernel): [stages][A 16 KiB | B 32 KiB] | barriers | tmem base |
 // abort flag | tile prefix.
-template <int MODE, int MT>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p) {
+gateup_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  constexpr int kGemmStages = GemmCfg<MT>::kStages, kGemmStageBytes = GemmCfg<MT>::kStageBytes;
-  constexpr int kBufs = GemmCfg<MT>::kBufs;
+  constexpr int MODE = 0, MT = 1, kBufs = kGemmBufs;   // one 128-row tile per unit, two accumulator buffers
   unsigned char *sp = smem + kGemmStages * kGemmStageBytes;
   uint64_t *s_bar = reinterpret_cast<uint64_t *>(sp); sp += 16 * 8;
   uint32_t *s_tmem = reinterpret_cast<uint32_t *>(sp); sp += 8;
@@ -305,9 +295,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   }
 }
 
-template <int MT>
-inline size_t grouped_gemm_smem_bytes() {
-  return 1024 + (size_t)GemmCfg<MT>::kStages * GemmCfg<MT>::kStageBytes + 16 * 8 + 16 + 2 * (kMaxExperts + 2) * 4;
+inline size_t gateup_gemm_smem_bytes() {
+  return 1024 + (size_t)kGemmStages * kGemmStageBytes + 16 * 8 + 16 + 2 * (kMaxExperts + 2) * 4;
 }
 
 // x rows into expert-sorted order: xs[pos] = x[perm[pos] / k]  (16 bytes per thread).

@@ -1,5 +1,5 @@
-// Step 5 for prefill-sized token counts, CTA-pair version of the grouped SwiGLU GEMMs (see gemm_tc.cuh for the
-// single-CTA kernel it replaces on the hot path).
+// Step 5 for prefill-sized token counts: the down-projection half of the grouped SwiGLU expert FFN on CTA pairs
+// (gemm_tc.cuh holds the gate/up half and the shared helpers).
 //
 // Two CTAs of a cluster (two SMs) work on one tile with tcgen05.mma.cta_group::2 (M = 256 over the pair): each
 // CTA stages its own 128 rows of A and one half of the rows of B, the leader CTA issues the MMAs for both, and
@@ -57,29 +57,21 @@ __device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
 
 // Swapped operands: the weights are the M side (always full 128-row tiles per CTA, 256 per pair), the tokens
 // are the N side, so a ragged expert is padded to a multiple of 16 tokens instead of 128 rows.
-//   MODE 0  H^T[neuron][token] : A = 128 gate rows and the same 128 up rows of this CTA's neurons (two
-//           accumulators that share the B tile), B = up to 128 expert-sorted x rows (each CTA stages half).
-//   MODE 1  O^T[column][token] : A = Wd[k rows][128 columns] (column-contiguous, i.e. MN-major), B = up to 256
-//           rows of H (each CTA stages half).
-// TMEM lane = neuron / output column, TMEM column = token; the epilogue writes H[token][neuron] / O[token][column].
-template <int MODE> struct Gemm2Cfg;
-template <> struct Gemm2Cfg<0> {
-  static constexpr int kTokTile = 128;                                  // tokens per unit
-  static constexpr int kStageBytes = 2 * kGemmATile + kGemmATile / 2;   // gate 16 KiB + up 16 KiB + 64 token rows 8 KiB
-  static constexpr int kStages = 5;
-};
-template <> struct Gemm2Cfg<1> {
-  static constexpr int kTokTile = 256;
+//   O^T[column][token] : A = Wd[k rows][128 columns] (column-contiguous, i.e. MN-major), B = up to 256 rows of H
+//   (each CTA stages half).  TMEM lane = output column, TMEM column = token; the epilogue writes O[token][column].
+struct Gemm2Cfg {
+  static constexpr int kTokTile = 256;                                  // tokens per unit
   static constexpr int kStageBytes = kGemmATile + kGemmATile;           // Wd tile 16 KiB + 128 token rows 16 KiB
   static constexpr int kStages = 6;
 };
 
 // Dynamic shared memory (1024-byte aligned by the kernel): [stages][A | B half] | barriers | tmem base |
 // abort flag | tile prefix | unit prefix.
-template <int MODE>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p) {
-  using Cfg = Gemm2Cfg<MODE>;
+down_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p) {
+  constexpr int MODE = 1;   // (the gate/up form of this kernel, MODE 0, measured slower than gemm_tc.cuh's and is kept
+                            // only as the constant-folded branches below)
+  using Cfg = Gemm2Cfg;
   constexpr int kStages = Cfg::kStages, kStageBytes = Cfg::kStageBytes, kTok = Cfg::kTokTile;
   extern __shared__ unsigned char smem_raw[];
   unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -285,9 +277,8 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   }
 }
 
-template <int MODE>
-inline size_t grouped_gemm2_smem_bytes() {
-  return 1024 + (size_t)Gemm2Cfg<MODE>::kStages * Gemm2Cfg<MODE>::kStageBytes + 16 * 8 + 16 + 2 * (kMaxExperts + 2) * 4 +
+inline size_t down_gemm2_smem_bytes() {
+  return 1024 + (size_t)Gemm2Cfg::kStages * Gemm2Cfg::kStageBytes + 16 * 8 + 16 + 2 * (kMaxExperts + 2) * 4 +
          16 + 4 * 32 * 32 * 2;
 }
 
