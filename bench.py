@@ -214,7 +214,8 @@ def run_ours(args):
                              max_tokens=max(B, 8), host_pool_ptr=pool.ptr.value, host_pool_bytes=pool.n_bytes,
                              fill_mode=fill_mode, device=local,
                              wdtype=Bd.FT_W_INT4_G128 if shape.wdtype == "int4" else Bd.FT_W_BF16,
-                             n_shared=shape.n_shared, shared_ptr=None if shared is None else shared.data_ptr(), **bw)
+                             n_shared=shape.n_shared, shared_ptr=None if shared is None else shared.data_ptr(),
+                             global_pool=args.global_pool, **bw)
         return Bd.FtMoe(cfg)
 
     # bandwidth profiling at deployment, then frozen into the plan's cost model
@@ -430,7 +431,7 @@ def run_ours(args):
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         lg, noise = main["lg"], main["noise"]
-        n_samp = args.cpu_layers
+        n_samp = min(args.cpu_layers, 2) if dsv3 else args.cpu_layers
         pool_np = pool.tensor.view(L, E, S).numpy()
         lg_np = lg[Wn].cpu().numpy()
         xb = [noise[Wn, l].cpu().view(torch.int16).numpy().view(np.uint16) for l in range(n_samp)]
@@ -451,7 +452,7 @@ def run_ours(args):
             "config": {"workload": ("decode DeepSeek-V3-shaped int4 MoE stack (config 3)" if dsv3 else
                                     "decode Qwen3-30B-A3B-shaped MoE stack (config 1)"), "batch": B, "layers": L,
                        "hidden": d, "experts": E, "inter": shape.inter, "top_k": k, "slots_per_layer": Ns,
-                       "fill_mode": args.fill, "cuda_graph": use_graph, "rho": RHO, "zipf_alpha": ALPHA,
+                       "fill_mode": args.fill, "cuda_graph": use_graph, "global_pool": bool(args.global_pool), "rho": RHO, "zipf_alpha": ALPHA,
                        "l2": "inputs larger than L2: every step streams GBs of distinct expert records from the slot "
                              "pool, far beyond the 126 MB L2; no flush needed",
                        "parallelism": "replicas" if world > 1 else "single",
@@ -663,6 +664,7 @@ def run_sweep(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--sweep-steps", type=int, default=128)
+    ap.add_argument("--global-pool", type=int, default=0, help="1: one slot pool and LRU clock shared by all layers")
     ap.add_argument("--graph", type=int, default=1, help="replay each decode step as one CUDA graph (SM fill only)")
     ap.add_argument("--workload", default="qwen", choices=["qwen", "dsv3"])
     ap.add_argument("--mode", default="decode", choices=["decode", "prefill", "sweep"])

@@ -44,7 +44,7 @@
  *                   S = 3*inter*hidden/2 + (2*inter*hidden/128 + (inter/128)*hidden)*2 bytes.
  *   Shape limits: bf16: hidden in {256, 512, 1024, 2048}, inter % 16 == 0; int4: hidden in
  *   {512, 1024, 2048, 4096, 7168, 8192}, inter % 128 == 0; n_experts <= 1024;
- *   top_k <= min(n_experts, 32); slots_per_layer <= 2048.  The tensor-core prefill path
+ *   top_k <= min(n_experts, 32); slots per table (slots_per_layer, or n_layers*slots_per_layer with global_pool) <= 6144.  The tensor-core prefill path
  *   (gemm_min_tokens > 0) needs bf16 weights, slots_per_layer > 0 and inter % 256 == 0.
  */
 #ifndef FTMOE_H_
@@ -114,6 +114,12 @@ typedef struct {
                                    launch of their own while the fills are still in flight, the
                                    filled experts after the fill event; 0 = always one launch after
                                    the fills (cheaper for a few tokens)                             */
+  int32_t global_pool;          /* 0: every layer owns slots_per_layer slots (an LRU per layer).
+                                   1: one pool of n_layers*slots_per_layer slots and one LRU clock
+                                   shared by all layers, keyed by the flattened id layer*n_experts +
+                                   expert (paper Sec. 3: a single elastic cache shared by all MoE
+                                   layers); slot indices, ft_moe_get_slot_table and fill_evicted then
+                                   refer to the shared pool / flattened ids                         */
 } ft_moe_config_t;
 
 /* Host-visible plan of one (layer, step).  The caller provides arrays of n_experts int32 each. */
@@ -204,6 +210,11 @@ ft_status_t ft_moe_read_slot(ft_moe_t *h, int layer, int slot, void *host_dst /*
 ft_status_t ft_moe_get_stats(ft_moe_t *h, int layer, uint64_t *counters, int n);
 /* Empties the slot table and zeroes step counter and statistics; layer = -1 for all layers. */
 ft_status_t ft_moe_reset(ft_moe_t *h, int layer);
+/* Runtime cache reconfiguration (paper Sec. 3.3): rebuilds the slot pool for a new budget of
+ * slots_per_layer slots per layer (n_layers * slots_per_layer shared slots with global_pool) without touching
+ * the host pool.  Call it at a safe point (no call of this handle in flight; it waits for the device).  The
+ * cache restarts empty, step counters and statistics are kept.  FT_ERR_OOM leaves the handle with zero slots. */
+ft_status_t ft_moe_resize(ft_moe_t *h, int slots_per_layer);
 /* Waits for the device and returns (and clears) the latched device status. */
 ft_status_t ft_moe_sync_status(ft_moe_t *h);
 /* Duration of the most recent ft_moe_fill's copies in microseconds and their bytes (waits for them). */

@@ -28,7 +28,7 @@ SYMBOLS = (
     "ft_moe_get_stats", "ft_moe_reset", "ft_moe_sync_status", "ft_moe_last_fill", "ft_moe_launch_count",
     "ft_moe_status_string", "ft_moe_timing_enable", "ft_moe_timing_read", "ft_moe_ffn_noalloc",
     "ft_moe_last_cuda_error", "ft_moe_host_register", "ft_moe_host_unregister",
-    "ft_moe_get_cta_trace", "ft_moe_set_split_min_pairs",
+    "ft_moe_get_cta_trace", "ft_moe_set_split_min_pairs", "ft_moe_resize",
 )
 NOALLOC_MAX_TOKENS, NOALLOC_MAX_HIDDEN = 64, 2048
 TIME_NAMES = ("route", "plan", "ffn_zc", "ffn_res", "finalize", "fill", "gather", "gemm1", "gemm2", "combine")
@@ -44,6 +44,7 @@ class Config(C.Structure):
         ("bw_fill_MBps", C.c_uint32), ("bw_zc_MBps", C.c_uint32), ("bw_zc_residual_MBps", C.c_uint32),
         ("bw_hbm_MBps", C.c_uint32), ("reuse_credit", C.c_int32), ("zc_tokens_per_pass", C.c_int32),
         ("hbm_tokens_per_pass", C.c_int32), ("gemm_min_tokens", C.c_int32), ("split_min_pairs", C.c_int32),
+        ("global_pool", C.c_int32),
     ]
 
 
@@ -86,6 +87,7 @@ def load(rebuild: bool = False):
         "ft_moe_host_register": (i32, [vp, sz]),
         "ft_moe_get_cta_trace": (i32, [vp, vp, i32]),
         "ft_moe_set_split_min_pairs": (i32, [vp, i32]),
+        "ft_moe_resize": (i32, [vp, i32]),
         "ft_moe_host_unregister": (i32, [vp]),
         "ft_moe_create": (i32, [C.POINTER(Config), C.POINTER(vp)]),
         "ft_moe_destroy": (i32, [vp]),
@@ -131,7 +133,7 @@ def make_config(*, hidden, inter, n_experts, top_k, n_layers=1, slots_per_layer,
                 host_pool_ptr, host_pool_bytes, wdtype=FT_W_BF16, n_shared=0, shared_ptr=None,
                 fill_mode=FT_FILL_COPY_ENGINE, device=0, bw_fill=50000, bw_zc=50000, bw_zc_residual=0,
                 bw_hbm=6000000, reuse_credit=1, zc_tokens_per_pass=64, hbm_tokens_per_pass=128,
-                gemm_min_tokens=0, split_min_pairs=32) -> Config:
+                gemm_min_tokens=0, split_min_pairs=32, global_pool=0) -> Config:
     c = Config()
     c.struct_size = C.sizeof(Config)
     c.device, c.n_layers, c.hidden, c.inter = device, n_layers, hidden, inter
@@ -142,6 +144,7 @@ def make_config(*, hidden, inter, n_experts, top_k, n_layers=1, slots_per_layer,
     c.reuse_credit, c.zc_tokens_per_pass, c.hbm_tokens_per_pass = reuse_credit, zc_tokens_per_pass, hbm_tokens_per_pass
     c.gemm_min_tokens = gemm_min_tokens
     c.split_min_pairs = split_min_pairs
+    c.global_pool = global_pool
     return c
 
 
@@ -226,6 +229,7 @@ class FtMoe:
         self._lib = load()
         self.cfg = cfg
         self.E, self.k, self.Ns = cfg.n_experts, cfg.top_k, cfg.slots_per_layer
+        self.L, self.global_pool = cfg.n_layers, bool(cfg.global_pool)
         self.expert_bytes = ft_moe_expert_bytes(cfg)
         self._h = C.c_void_p()
         _check(self._lib.ft_moe_create(C.byref(cfg), C.byref(self._h)), "ft_moe_create")
@@ -297,11 +301,19 @@ class FtMoe:
         return ids.reshape(T, self.k), w.reshape(T, self.k), count, offset, perm, inv
 
     def get_slot_table(self, layer):
-        se = np.zeros(max(self.Ns, 1), dtype=np.int32)
-        ss = np.zeros(max(self.Ns, 1), dtype=np.int64)
+        """(slot_expert, slot_stamp, expert_slot of `layer`); with a global pool the first two cover the shared
+        pool and hold flattened ids layer*E + expert."""
+        n = self.Ns * self.L if self.global_pool else self.Ns
+        se = np.zeros(max(n, 1), dtype=np.int32)
+        ss = np.zeros(max(n, 1), dtype=np.int64)
         es = np.zeros(self.E, dtype=np.int32)
         _check(self._lib.ft_moe_get_slot_table(self._h, layer, _ptr(se), _ptr(ss), _ptr(es)), "ft_moe_get_slot_table")
-        return se[:self.Ns], ss[:self.Ns], es
+        return se[:n], ss[:n], es
+
+    def resize(self, slots_per_layer):
+        _check(self._lib.ft_moe_resize(self._h, int(slots_per_layer)), "ft_moe_resize")
+        self.Ns = int(slots_per_layer)
+        self.cfg.slots_per_layer = int(slots_per_layer)
 
     def read_slot(self, layer, slot):
         buf = np.empty(self.expert_bytes, dtype=np.uint8)

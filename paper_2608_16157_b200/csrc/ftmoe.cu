@@ -26,7 +26,8 @@ struct LayerState {
   int32_t *slot_expert = nullptr;
   int64_t *slot_stamp = nullptr;
   int32_t *expert_slot = nullptr;
-  int64_t *step = nullptr;
+  int64_t *step = nullptr;     // plan calls of this layer
+  int64_t *clock = nullptr;    // the LRU clock the layer's plans advance (its own step counter, or the shared one)
   unsigned long long *stats = nullptr;
   int phase = PH_IDLE;
   int T = 0;
@@ -42,8 +43,10 @@ struct ft_moe {
   uint8_t *slots = nullptr;         // [L][N_s][S]
   uint8_t *shared_dev = nullptr;    // [L][n_shared][S]
   const uint8_t *pool_dev = nullptr;  // device alias of host_pool
-  uint8_t *tables = nullptr;        // one allocation for all per-layer tables
+  uint8_t *tables = nullptr;        // one allocation for all tables (per layer, or shared by all layers)
   size_t tables_bytes = 0;
+  uint8_t *stats_mem = nullptr;     // per-layer step counters and statistics (survive a resize)
+  int table_slots = 0;              // slots per table: slots_per_layer, or n_layers*slots_per_layer when shared
   std::vector<LayerState> layers;
   // per-handle scratch (layers are stream-ordered, so one set serves all)
   int32_t *ids = nullptr, *count = nullptr, *offset = nullptr, *perm = nullptr, *inv = nullptr;
@@ -180,18 +183,72 @@ struct TimeScope {
   }
 };
 
-ft_status_t reset_layer(ft_moe *h, int l) {
+// Empties the residency tables `l` uses (with a shared pool: everybody's) and, unless keep_counters, the layer's
+// step counter and statistics.
+ft_status_t reset_layer(ft_moe *h, int l, bool keep_counters = false) {
   LayerState &L = h->layers[l];
-  const int Ns = h->cfg.slots_per_layer, E = h->cfg.n_experts;
+  const int Ns = h->table_slots, E = h->cfg.n_experts;
   if (Ns > 0) {
     FT_CUDA(cudaMemset(L.slot_expert, 0xff, sizeof(int32_t) * Ns));
     FT_CUDA(cudaMemset(L.slot_stamp, 0xff, sizeof(int64_t) * Ns));
   }
-  FT_CUDA(cudaMemset(L.expert_slot, 0xff, sizeof(int32_t) * E));
-  FT_CUDA(cudaMemset(L.step, 0, sizeof(int64_t)));
-  FT_CUDA(cudaMemset(L.stats, 0, sizeof(unsigned long long) * FT_STAT_COUNT));
+  FT_CUDA(cudaMemset(h->cfg.global_pool ? L.expert_slot + (size_t)l * E : L.expert_slot, 0xff, sizeof(int32_t) * E));
+  if (!keep_counters) {
+    FT_CUDA(cudaMemset(L.step, 0, sizeof(int64_t)));
+    FT_CUDA(cudaMemset(L.stats, 0, sizeof(unsigned long long) * FT_STAT_COUNT));
+  }
   L.phase = PH_IDLE;
   L.T = 0;
+  return FT_OK;
+}
+
+// (Re)allocates the slot pool and the residency tables for h->cfg.slots_per_layer and empties them.
+ft_status_t alloc_cache(ft_moe *h) {
+  const ft_moe_config_t &c = h->cfg;
+  const size_t E = c.n_experts, Ns = c.slots_per_layer, L = c.n_layers;
+  cudaFree(h->slots); h->slots = nullptr;
+  cudaFree(h->tables); h->tables = nullptr;
+  (void)cudaGetLastError();
+  h->table_slots = c.global_pool ? (int)(L * Ns) : (int)Ns;
+  if (Ns > 0) FT_CUDA(cudaMalloc(&h->slots, L * Ns * h->S));
+  auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+  if (c.global_pool) {
+    // one table for all layers, keyed by the flattened id layer*E + expert; one clock
+    const size_t Nt = L * Ns;
+    h->tables_bytes = up(Nt * 4) + up(Nt * 8) + up(L * E * 4) + up(8);
+    FT_CUDA(cudaMalloc(&h->tables, h->tables_bytes));
+    uint8_t *b = h->tables;
+    int32_t *se = reinterpret_cast<int32_t *>(b); b += up(Nt * 4);
+    int64_t *ss = reinterpret_cast<int64_t *>(b); b += up(Nt * 8);
+    int32_t *es = reinterpret_cast<int32_t *>(b); b += up(L * E * 4);
+    int64_t *clock = reinterpret_cast<int64_t *>(b);
+    FT_CUDA(cudaMemset(clock, 0, 8));
+    for (size_t l = 0; l < L; ++l) {
+      LayerState &ls = h->layers[l];
+      ls.slot_expert = se; ls.slot_stamp = ss; ls.expert_slot = es; ls.clock = clock;
+    }
+  } else {
+    const size_t per_layer = up(Ns * 4) + up(Ns * 8) + up(E * 4);
+    h->tables_bytes = per_layer * L;
+    FT_CUDA(cudaMalloc(&h->tables, h->tables_bytes));
+    for (size_t l = 0; l < L; ++l) {
+      uint8_t *b = h->tables + l * per_layer;
+      LayerState &ls = h->layers[l];
+      ls.slot_expert = reinterpret_cast<int32_t *>(b); b += up(Ns * 4);
+      ls.slot_stamp = reinterpret_cast<int64_t *>(b); b += up(Ns * 8);
+      ls.expert_slot = reinterpret_cast<int32_t *>(b);
+      ls.clock = ls.step;     // the layer's own step counter is its LRU clock
+    }
+  }
+  for (size_t l = 0; l < L; ++l) {
+    ft_status_t rc = reset_layer(h, (int)l, true);
+    if (rc != FT_OK) return rc;
+  }
+  const int dyn = h->table_slots * 16;
+  if ((size_t)dyn + 36 * 1024 > 48 * 1024) {
+    FT_CUDA(cudaFuncSetAttribute(plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn));
+    FT_CUDA(cudaFuncSetAttribute(route_plan_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn));
+  }
   return FT_OK;
 }
 
@@ -275,6 +332,7 @@ ft_status_t ft_moe_destroy(ft_moe_t *h) {
   cudaFree(h->slots);
   cudaFree(h->shared_dev);
   cudaFree(h->tables);
+  cudaFree(h->stats_mem);
   cudaFree(h->ids);
   cudaFree(h->count);
   cudaFree(h->offset);
@@ -319,7 +377,9 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
   if (!cfg || cfg->struct_size != sizeof(ft_moe_config_t)) return FT_ERR_INVALID_ARG;
   const ft_moe_config_t &c = *cfg;
   if (c.n_layers <= 0 || c.n_experts <= 0 || c.n_experts > kMaxExperts || c.top_k <= 0 ||
-      c.top_k > c.n_experts || c.top_k > kMaxTopK || c.slots_per_layer < 0 || c.slots_per_layer > 2048 ||
+      c.top_k > c.n_experts || c.top_k > kMaxTopK || c.slots_per_layer < 0 ||
+      (c.global_pool != 0 && c.global_pool != 1) ||
+      (long long)c.slots_per_layer * (c.global_pool ? c.n_layers : 1) > 6144 ||
       c.max_tokens <= 0 || (c.n_shared != 0 && c.n_shared != 1) || c.device < 0 ||
       (c.fill_mode != FT_FILL_COPY_ENGINE && c.fill_mode != FT_FILL_SM))
     return FT_ERR_INVALID_ARG;
@@ -375,25 +435,22 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
 
   const size_t E = c.n_experts, Ns = c.slots_per_layer, L = c.n_layers;
   const size_t P = (size_t)c.max_tokens * c.top_k;
-  if (Ns > 0) FT_TRY(cudaMalloc(&h->slots, L * Ns * S));
   if (c.n_shared) {
     FT_TRY(cudaMalloc(&h->shared_dev, L * S));
     FT_TRY(cudaMemcpy(h->shared_dev, c.shared_weights, L * S, cudaMemcpyHostToDevice));
   }
-  // per-layer tables, 256-byte aligned pieces
-  auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
-  const size_t per_layer = up(Ns * 4) + up(Ns * 8) + up(E * 4) + up(8) + up(FT_STAT_COUNT * 8);
-  h->tables_bytes = per_layer * L;
-  FT_TRY(cudaMalloc(&h->tables, h->tables_bytes));
-  for (size_t l = 0; l < L; ++l) {
-    uint8_t *b = h->tables + l * per_layer;
-    LayerState &ls = h->layers[l];
-    ls.slot_expert = reinterpret_cast<int32_t *>(b); b += up(Ns * 4);
-    ls.slot_stamp = reinterpret_cast<int64_t *>(b); b += up(Ns * 8);
-    ls.expert_slot = reinterpret_cast<int32_t *>(b); b += up(E * 4);
-    ls.step = reinterpret_cast<int64_t *>(b); b += up(8);
-    ls.stats = reinterpret_cast<unsigned long long *>(b);
+  // per-layer step counters and statistics
+  {
+    const size_t per = 256 + ((FT_STAT_COUNT * 8 + 255) & ~(size_t)255);
+    FT_TRY(cudaMalloc(&h->stats_mem, per * L));
+    FT_TRY(cudaMemset(h->stats_mem, 0, per * L));
+    for (size_t l = 0; l < L; ++l) {
+      h->layers[l].step = reinterpret_cast<int64_t *>(h->stats_mem + l * per);
+      h->layers[l].stats = reinterpret_cast<unsigned long long *>(h->stats_mem + l * per + 256);
+    }
   }
+  rc = alloc_cache(h);
+  if (rc != FT_OK) return fail(rc);
   FT_TRY(cudaMalloc(&h->ids, P * 4 + 16));
   FT_TRY(cudaMalloc(&h->topk_w, P * 4 + 16));
   FT_TRY(cudaMalloc(&h->count, E * 4));
@@ -450,11 +507,6 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
   FT_TRY(cudaMemset(h->trace_dev, 0, (size_t)h->sm_count * 4 * sizeof(long long)));
   FT_TRY(cudaMalloc(&h->done_dev, 4));
   FT_TRY(cudaMemset(h->done_dev, 0, 4));
-  if ((size_t)c.slots_per_layer * 16 + 36 * 1024 > 48 * 1024) {
-    const int dyn = c.slots_per_layer * 16;
-    FT_TRY(cudaFuncSetAttribute(plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn));
-    FT_TRY(cudaFuncSetAttribute(route_plan_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn));
-  }
   FT_TRY(cudaFuncSetAttribute(fill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFillStages * (int)kFillChunk));
   if (c.wdtype == FT_W_INT4_G128) {
     const size_t passes = (P + 7) / 8 + 2 * E + 2;
@@ -504,11 +556,13 @@ ft_status_t ft_moe_reset(ft_moe_t *h, int layer) {
   if (!h || layer < -1 || layer >= h->cfg.n_layers) return FT_ERR_INVALID_ARG;
   FT_CUDA(cudaSetDevice(h->cfg.device));
   FT_CUDA(cudaDeviceSynchronize());
+  if (h->cfg.global_pool && layer >= 0) return FT_ERR_UNSUPPORTED;   // the shared pool has no per-layer part
   for (int l = 0; l < h->cfg.n_layers; ++l)
     if (layer < 0 || l == layer) {
       ft_status_t rc = reset_layer(h, l);
       if (rc != FT_OK) return rc;
     }
+  if (h->cfg.global_pool) FT_CUDA(cudaMemset(h->layers[0].clock, 0, 8));
   FT_CUDA(cudaMemset(h->y_acc, 0, (size_t)h->cfg.max_tokens * h->cfg.hidden * 4));
   FT_CUDA(cudaDeviceSynchronize());
   return FT_OK;
@@ -537,7 +591,8 @@ static PlanParams make_plan_params(ft_moe *h, int layer, bool mirror_to_host) {
   LayerState &L = h->layers[layer];
   PlanParams pp;
   pp.count = h->count; pp.offset = h->offset;
-  pp.E = c.n_experts; pp.n_slots = c.slots_per_layer;
+  pp.E = c.n_experts; pp.n_slots = h->table_slots;
+  pp.id_base = c.global_pool ? layer * c.n_experts : 0;
   pp.cm.ns_fill = (int64_t)(h->S * 1000 / c.bw_fill_MBps);
   pp.cm.ns_zc = (int64_t)(h->S * 1000 / c.bw_zc_MBps);
   pp.cm.ns_hbm = (int64_t)(h->S * 1000 / c.bw_hbm_MBps);
@@ -545,9 +600,9 @@ static PlanParams make_plan_params(ft_moe *h, int layer, bool mirror_to_host) {
   pp.cm.reuse_credit = c.reuse_credit; pp.cm.tz = c.zc_tokens_per_pass; pp.cm.tg = c.hbm_tokens_per_pass;
   pp.cm.gemm_min_tokens = c.gemm_min_tokens;
   pp.slot_expert = L.slot_expert; pp.slot_stamp = L.slot_stamp; pp.expert_slot = L.expert_slot;
-  pp.step = L.step; pp.stats = L.stats;
+  pp.step = L.clock; pp.layer_steps = L.step; pp.stats = L.stats;
   pp.pool_layer_dev = h->pool_dev + (size_t)layer * c.n_experts * h->S;
-  pp.slots_layer = h->slots ? h->slots + (size_t)layer * c.slots_per_layer * h->S : nullptr;
+  pp.slots_layer = h->slots ? h->slots + (c.global_pool ? 0 : (size_t)layer * c.slots_per_layer * h->S) : nullptr;
   pp.shared_rec = c.n_shared ? h->shared_dev + (size_t)layer * h->S : nullptr;
   pp.S = h->S; pp.T = L.T;
   pp.tokens_per_pass = kMmaTokens;
@@ -596,7 +651,7 @@ ft_status_t ft_moe_plan(ft_moe_t *h, int layer, ft_moe_plan_t *out, void *stream
   if (L.T > 0) {
     const bool mirror = (out != nullptr) || c.fill_mode == FT_FILL_COPY_ENGINE;
     const PlanParams pp = make_plan_params(h, layer, mirror);
-    const size_t smem = (size_t)c.slots_per_layer * 16;
+    const size_t smem = (size_t)h->table_slots * 16;
     int threads = ((c.n_experts + 31) / 32) * 32;
     if (threads < 128) threads = 128;
     {
@@ -648,7 +703,7 @@ ft_status_t ft_moe_fill(ft_moe_t *h, int layer, void *copy_stream) {
   if (L.T == 0 || h->cfg.slots_per_layer == 0) return FT_OK;
   cudaStream_t cs = static_cast<cudaStream_t>(copy_stream);
   const ft_moe_config_t &c = h->cfg;
-  uint8_t *slots_layer = h->slots + (size_t)layer * c.slots_per_layer * h->S;
+  uint8_t *slots_layer = h->slots + (c.global_pool ? 0 : (size_t)layer * c.slots_per_layer * h->S);
   if (c.fill_mode == FT_FILL_COPY_ENGINE) {
     // the host needs the fill list: wait for the plan record (one host round trip per layer)
     FT_CUDA(cudaEventSynchronize(h->ev_plan));
@@ -664,7 +719,7 @@ ft_status_t ft_moe_fill(ft_moe_t *h, int layer, void *copy_stream) {
       {
         TimeScope ts(h, cs, FT_TIME_FILL);
         for (int i = 0; i < hd.n_fill; ++i) {
-          if (forder[i] < 0 || forder[i] >= E || fslot[i] < 0 || fslot[i] >= c.slots_per_layer) return FT_ERR_CUDA;
+          if (forder[i] < 0 || forder[i] >= E || fslot[i] < 0 || fslot[i] >= h->table_slots) return FT_ERR_CUDA;
           FT_CUDA(cudaMemcpyAsync(slots_layer + (size_t)fslot[i] * h->S, pool_layer + (size_t)forder[i] * h->S,
                                   h->S, cudaMemcpyHostToDevice, cs));
         }
@@ -761,7 +816,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
       GemmParams gp;
       gp.items = h->items_gemm; gp.n_items = &h->plan_dev->n_gemm_items; gp.mt_pref = h->gemm_pref;
       gp.inter = c.inter; gp.d = c.hidden;
-      gp.layer_row0 = (long long)layer * c.slots_per_layer * 3 * c.inter;
+      gp.layer_row0 = c.global_pool ? 0 : (long long)layer * c.slots_per_layer * 3 * c.inter;
       gp.status = h->status_dev;
       // CTA pairs (clusters of two) share every 256x256 tile
       cudaLaunchConfig_t lc = {};
@@ -855,7 +910,7 @@ ft_status_t ft_moe_layer(ft_moe_t *h, int layer, const float *logits_dev, const 
     const PlanParams pp = make_plan_params(h, layer, mirror);
     {
       TimeScope ts(h, st, FT_TIME_PLAN);
-      route_plan_small_kernel<<<1, single_cta_threads(c.n_experts, T), (size_t)c.slots_per_layer * 16, st>>>(rp, pp);
+      route_plan_small_kernel<<<1, single_cta_threads(c.n_experts, T), (size_t)h->table_slots * 16, st>>>(rp, pp);
     }
     h->launches++;
     h->seq_host++;
@@ -920,19 +975,21 @@ ft_status_t ft_moe_get_slot_table(ft_moe_t *h, int layer, int32_t *slot_expert, 
   FT_CUDA(cudaSetDevice(h->cfg.device));
   FT_CUDA(cudaDeviceSynchronize());
   const LayerState &L = h->layers[layer];
-  const size_t Ns = h->cfg.slots_per_layer;
+  const size_t Ns = h->table_slots;
   if (slot_expert && Ns) FT_CUDA(cudaMemcpy(slot_expert, L.slot_expert, Ns * 4, cudaMemcpyDeviceToHost));
   if (slot_stamp && Ns) FT_CUDA(cudaMemcpy(slot_stamp, L.slot_stamp, Ns * 8, cudaMemcpyDeviceToHost));
-  if (expert_slot) FT_CUDA(cudaMemcpy(expert_slot, L.expert_slot, (size_t)h->cfg.n_experts * 4, cudaMemcpyDeviceToHost));
+  if (expert_slot)
+    FT_CUDA(cudaMemcpy(expert_slot, L.expert_slot + (h->cfg.global_pool ? (size_t)layer * h->cfg.n_experts : 0),
+                       (size_t)h->cfg.n_experts * 4, cudaMemcpyDeviceToHost));
   return FT_OK;
 }
 
 ft_status_t ft_moe_read_slot(ft_moe_t *h, int layer, int slot, void *host_dst) {
-  if (!h || layer < 0 || layer >= h->cfg.n_layers || slot < 0 || slot >= h->cfg.slots_per_layer || !host_dst)
+  if (!h || layer < 0 || layer >= h->cfg.n_layers || slot < 0 || slot >= h->table_slots || !host_dst)
     return FT_ERR_INVALID_ARG;
   FT_CUDA(cudaSetDevice(h->cfg.device));
   FT_CUDA(cudaDeviceSynchronize());
-  FT_CUDA(cudaMemcpy(host_dst, h->slots + ((size_t)layer * h->cfg.slots_per_layer + slot) * h->S, h->S,
+  FT_CUDA(cudaMemcpy(host_dst, h->slots + ((h->cfg.global_pool ? 0 : (size_t)layer * h->cfg.slots_per_layer) + slot) * h->S, h->S,
                      cudaMemcpyDeviceToHost));
   return FT_OK;
 }
@@ -979,6 +1036,24 @@ ft_status_t ft_moe_get_cta_trace(ft_moe_t *h, int64_t *out, int n_ctas) {
   FT_CUDA(cudaDeviceSynchronize());
   const int n = n_ctas < h->sm_count ? n_ctas : h->sm_count;
   FT_CUDA(cudaMemcpy(out, h->trace_dev, (size_t)n * 4 * sizeof(long long), cudaMemcpyDeviceToHost));
+  return FT_OK;
+}
+
+ft_status_t ft_moe_resize(ft_moe_t *h, int slots_per_layer) {
+  if (!h || slots_per_layer < 0) return FT_ERR_INVALID_ARG;
+  if ((long long)slots_per_layer * (h->cfg.global_pool ? h->cfg.n_layers : 1) > 6144) return FT_ERR_INVALID_ARG;
+  if (h->gemm) return FT_ERR_UNSUPPORTED;   // the tensor maps of the prefill path are bound to the slot pool
+  FT_CUDA(cudaSetDevice(h->cfg.device));
+  FT_CUDA(cudaDeviceSynchronize());
+  for (auto &L : h->layers) L.phase = PH_IDLE;
+  h->cfg.slots_per_layer = slots_per_layer;
+  ft_status_t rc = alloc_cache(h);
+  if (rc != FT_OK) {
+    h->cfg.slots_per_layer = 0;
+    (void)alloc_cache(h);
+    return rc;
+  }
+  FT_CUDA(cudaDeviceSynchronize());
   return FT_OK;
 }
 

@@ -13,13 +13,15 @@ struct PlanParams {
   // inputs
   const int32_t *count;   // [E]
   const int32_t *offset;  // [E+1]
-  int E, n_slots;
+  int E, n_slots;        // experts of this layer; slots of the table (per layer, or the shared pool)
+  int id_base;           // flattened id of this layer's expert 0 in the tables (layer*E with a shared pool, else 0)
   CostModelDev cm;
   // per-layer state
   int32_t *slot_expert;  // [n_slots]
   int64_t *slot_stamp;   // [n_slots]
   int32_t *expert_slot;  // [E]
-  int64_t *step;         // [1]
+  int64_t *step;         // [1] the LRU clock: stamps come from it and it advances by one per plan
+  int64_t *layer_steps;  // [1] plan calls of this layer (the same counter unless the pool is shared)
   unsigned long long *stats;  // [FT_STAT_COUNT]
   // where records live
   const uint8_t *pool_layer_dev;  // device alias of the host pool, first record of this layer
@@ -71,6 +73,7 @@ __device__ __forceinline__ unsigned long long block_excl_scan64(unsigned long lo
   return incl - v + s_w[warp];
 }
 
+constexpr int64_t kSlotTaken = 0x7fffffffffffffffll;   // stamp marker of a slot already chosen as a victim
 constexpr int kPlanField = 11;  // bits per packed counter (values <= 1024)
 __device__ __forceinline__ unsigned long long pack4(int a, int b, int c, int d) {
   return (unsigned long long)a | ((unsigned long long)b << kPlanField) | ((unsigned long long)c << (2 * kPlanField)) |
@@ -99,7 +102,7 @@ __device__ __forceinline__ void plan_prefetch(const PlanParams &p, unsigned char
   int32_t *s_sexp = reinterpret_cast<int32_t *>(s_stamp + p.n_slots);
   const int tid = threadIdx.x;
   t = *p.step;
-  slot = (tid < p.E) ? p.expert_slot[tid] : -1;
+  slot = (tid < p.E) ? p.expert_slot[p.id_base + tid] : -1;
   for (int s = tid; s < p.n_slots; s += blockDim.x) {
     s_stamp[s] = p.slot_stamp[s];
     s_sexp[s] = p.slot_expert[s];
@@ -173,11 +176,47 @@ __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, uns
       if (o >= p.n_slots) return ~0ull;
       const int oex = s_sexp[o];
       const int64_t ost = s_stamp[o];
+      if (ost == kSlotTaken) return ~0ull;
       if (oex < 0) return (unsigned long long)o;
       if (ost >= t) return ~0ull;
       return (1ull << 62) | ((unsigned long long)(ost + 1) << 20) | (unsigned long long)oex;
     };
-    if (q <= 8 && p.n_slots <= 256) {
+    if (q <= 16 && p.n_slots > 256) {
+      // few fills out of a large (shared) pool: q block-wide minima; a chosen slot is marked as touched
+      unsigned long long *s_wmin = reinterpret_cast<unsigned long long *>(sm.forder);   // [32] keys (forder is free here)
+      int *s_wslot = reinterpret_cast<int *>(s_wmin + 32);                               // [32] slots
+      for (int r = 0; r < q; ++r) {
+        unsigned long long best = ~0ull;
+        int bslot = -1;
+        for (int o = tid; o < p.n_slots; o += blockDim.x) {
+          const unsigned long long ko = slot_key(o);
+          if (ko < best) { best = ko; bslot = o; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const unsigned long long ob = __shfl_xor_sync(0xffffffffu, best, o);
+          const int os = __shfl_xor_sync(0xffffffffu, bslot, o);
+          if (ob < best) { best = ob; bslot = os; }
+        }
+        if (lane == 0) { s_wmin[warp] = best; s_wslot[warp] = bslot; }
+        __syncthreads();
+        if (warp == 0) {
+          best = (lane < nwarps) ? s_wmin[lane] : ~0ull;
+          bslot = (lane < nwarps) ? s_wslot[lane] : -1;
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const unsigned long long ob = __shfl_xor_sync(0xffffffffu, best, o);
+            const int os = __shfl_xor_sync(0xffffffffu, bslot, o);
+            if (ob < best) { best = ob; bslot = os; }
+          }
+          if (lane == 0) {
+            s_victim[r] = bslot;
+            s_stamp[bslot] = kSlotTaken;   // no longer a candidate (the shared-memory copy is not used afterwards)
+          }
+        }
+        __syncthreads();
+      }
+    } else if (q <= 8 && p.n_slots <= 256) {
       // few fills (decode): warp 0 extracts the q smallest keys one after the other (q warp-wide minima)
       if (warp == 0) {
         unsigned long long key[8];
@@ -246,9 +285,9 @@ __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, uns
     const int e = sm.forder[tid];
     const int s = s_victim[tid];
     const int old = s_sexp[s];
-    if (old >= 0) p.expert_slot[old] = -1;
-    p.slot_expert[s] = e;
-    p.expert_slot[e] = s;
+    if (old >= 0) p.expert_slot[old] = -1;      // `old` is a flattened id: it may belong to another layer
+    p.slot_expert[s] = p.id_base + e;
+    p.expert_slot[p.id_base + e] = s;
     p.slot_stamp[s] = t;
     a_forder[tid] = e;
     a_fslot[tid] = s;
@@ -352,6 +391,7 @@ __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, uns
     h.pad[0] = h.pad[1] = h.pad[2] = h.pad[3] = 0;
     *p.hdr_dev = h;
     *p.step = t + 1;
+    if (p.layer_steps != p.step) *p.layer_steps += 1;
     int evictions = 0;
     for (int i = 0; i < n_fill; ++i) evictions += (s_sexp[s_victim[i]] >= 0);
     // fire-and-forget adds: nothing waits for the old values

@@ -26,8 +26,8 @@ def test_library_builds_loads_and_exports_every_declared_symbol():
 
 
 def test_config_struct_matches_header_size_and_expert_bytes():
-    # 12 int32 + (ptr, size_t, ptr) + 4 uint32 + 5 int32 (+ 4 bytes of tail padding) on LP64
-    assert ctypes.sizeof(B.Config) == 12 * 4 + 3 * 8 + 9 * 4 + 4
+    # 12 int32 + (ptr, size_t, ptr) + 4 uint32 + 6 int32 on LP64
+    assert ctypes.sizeof(B.Config) == 12 * 4 + 3 * 8 + 10 * 4
     cfg = B.make_config(hidden=2048, inter=768, n_experts=128, top_k=8, slots_per_layer=64, max_tokens=8,
                         host_pool_ptr=None, host_pool_bytes=0)
     assert B.ft_moe_expert_bytes(cfg) == 9437184
