@@ -10,9 +10,14 @@ Expert record formats (one contiguous record per (layer, expert); the pool is
 ``n_layers * n_experts`` records back to back, record index ``l * E + e``, the
 flattened identifier of Sec. 4.2 of the paper):
 
-``bf16``  three row-major ``[I][d]`` bf16 matrices, in this order
-          ``Wg_t`` (``Wg_t[n][i] = W_gate[i][n]``), ``Wu_t`` (same for W_up),
-          ``Wd`` (``Wd[n][c] = W_down[n][c]``).  ``S = 3*I*d*2`` bytes.
+``bf16``  ``I/16`` units of 16 neurons, each ``96*d`` bytes: a gate part, an up part and a
+          down part of ``32*d`` bytes each, all in 8 x 8 blocks of bf16 (8 rows of 16 bytes).
+          Gate/up part: tiles of 16 neurons x 32 hidden indices (1 KiB), tile ``i // 32``;
+          inside a tile the block of neuron half ``(n % 16) // 8`` and hidden quarter
+          ``(i % 32) // 8`` starts at ``512*half + 128*quarter``, row ``n % 8``, element ``i % 8``.
+          Down part: tiles of 16 output columns x the unit's 16 neurons (512 bytes), tile
+          ``c // 16``; block of column half ``(c % 16) // 8`` and neuron half ``(n % 16) // 8`` at
+          ``256*chalf + 128*nhalf``, row ``c % 8``, element ``n % 8``.  ``S = 3*I*d*2`` bytes.
 ``int4``  4-bit two's-complement codes in [-8, 7] for the same three matrices,
           then bf16 scales.  ``Wg_q`` and ``Wu_q`` are row-major ``[I][d/2]`` bytes,
           two codes per byte along ``d`` (low nibble = even column).  ``Wd_q`` is
@@ -149,6 +154,17 @@ def _pack_wd_fragment_order(q: torch.Tensor) -> torch.Tensor:
     return by.reshape(-1)
 
 
+def _pack_bf16_tiles(w: torch.Tensor) -> torch.Tensor:
+    """bf16 ``[3][I][d]`` (gate and up one row per neuron, down ``[n][c]``) -> the tiled record, flat."""
+    _, I, d = w.shape
+    U = I // 16
+    # gate / up: [unit][neuron half][row][tile][quarter][element] -> [unit][tile][half][quarter][row][element]
+    gu = w[0:2].reshape(2, U, 2, 8, d // 32, 4, 8).permute(0, 1, 4, 2, 5, 3, 6).reshape(2, U, 16 * d)
+    # down: [unit][neuron half][element][tile][column half][row] -> [unit][tile][chalf][nhalf][row][element]
+    dn = w[2].reshape(U, 2, 8, d // 16, 2, 8).permute(0, 3, 4, 1, 5, 2).reshape(U, 16 * d)
+    return torch.cat([gu[0], gu[1], dn], dim=1).contiguous().reshape(-1)
+
+
 def make_records(shape: LayerShape, seed: int, layer: int, first: int, count: int,
                  device="cpu", std: float = 0.02) -> torch.Tensor:
     """Records of experts ``first .. first+count-1`` of ``layer`` as uint8 ``[count, S]``.
@@ -162,7 +178,7 @@ def make_records(shape: LayerShape, seed: int, layer: int, first: int, count: in
         g = _gen(device, mix64(seed, _TAG_W, layer, first + j))
         w = torch.randn((3, I, d), generator=g, device=device, dtype=torch.float32) * std
         if shape.wdtype == "bf16":
-            out[j] = w.to(torch.bfloat16).reshape(-1).view(torch.uint8)
+            out[j] = _pack_bf16_tiles(w.to(torch.bfloat16)).view(torch.uint8)
         else:
             qg, sg = _quantise_int4(w[0:1], 2)
             qu, su = _quantise_int4(w[1:2], 2)

@@ -18,18 +18,26 @@ def _record_bf16_by_definition(wg, wu, wd):
     d, I = wg.shape
     rec = np.zeros(3 * I * d, dtype=np.uint16)
     gb, ub, db = _bf16_bits(wg), _bf16_bits(wu), _bf16_bits(wd)
+    unit_el = 48 * d                      # 16 neurons: gate part, up part, down part of 16*d elements each
     for n in range(I):
+        unit, nhalf, nrow = n // 16, (n % 16) // 8, n % 8
         for i in range(d):
-            rec[0 * I * d + n * d + i] = gb[i, n]
-            rec[1 * I * d + n * d + i] = ub[i, n]
-            rec[2 * I * d + n * d + i] = db[n, i]
+            # gate / up: 1 KiB tiles of 16 neurons x 32 hidden indices, 8 x 8 blocks inside
+            tile, quarter, e = i // 32, (i % 32) // 8, i % 8
+            at = unit * unit_el + tile * 512 + nhalf * 256 + quarter * 64 + nrow * 8 + e
+            rec[at] = gb[i, n]
+            rec[at + 16 * d] = ub[i, n]
+            # down (i is the output column here): 512-byte tiles of 16 columns x the unit's 16 neurons
+            ctile, chalf, crow = i // 16, (i % 16) // 8, i % 8
+            rec[unit * unit_el + 32 * d + ctile * 256 + chalf * 128 + nhalf * 64 + crow * 8 + nrow] = db[n, i]
     return rec.view(np.uint8)
 
 
 def test_unpack_bf16_record_orientation():
-    d, I = 16, 8
-    wg = np.arange(d * I, dtype=np.float32).reshape(d, I) / 4.0        # all exactly representable
-    wu = -np.arange(d * I, dtype=np.float32).reshape(d, I) / 8.0
+    d, I = 64, 32
+    # all exactly representable in bf16; the periods (251, 127, 31) are coprime to every stride of the layout
+    wg = ((np.arange(d * I, dtype=np.float32).reshape(d, I) % 251) - 125.0) / 4.0
+    wu = -((np.arange(d * I, dtype=np.float32).reshape(d, I) % 127) - 63.0) / 8.0
     wd = (np.arange(I * d, dtype=np.float32).reshape(I, d) % 31) - 15.0
     g, u, dn = O.unpack_record(_record_bf16_by_definition(wg, wu, wd), d, I, "bf16")
     assert np.array_equal(g, wg) and np.array_equal(u, wu) and np.array_equal(dn, wd)
