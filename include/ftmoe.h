@@ -23,12 +23,23 @@
  *     word and reported by the next synchronising call (ft_moe_plan with a non-null out pointer,
  *     ft_moe_fill in copy-engine mode, the ft_moe_get_* calls, ft_moe_sync_status).
  *   - T = 0 is a no-op that does not advance the layer's step counter.
+ *   - Device buffers of activations (x_dev, y_dev) and records must be 16-byte aligned (the kernels use vector
+ *     accesses); a misaligned pointer is FT_ERR_INVALID_ARG, never a device fault.
  *
  * Expert record layout (pool records and slots are byte-identical, so a fill is one contiguous copy)
  *   record index in the pool: layer * n_experts + expert (the flattened id of paper Sec. 4.2).
- *   FT_W_BF16     : three row-major [inter][hidden] bf16 matrices, in this order:
- *                     Wg_t  (Wg_t[n][i] = W_gate[i][n]),  Wu_t (Wu_t[n][i] = W_up[i][n]),
- *                     Wd    (Wd[n][c]   = W_down[n][c]).          S = 3*inter*hidden*2 bytes.
+ *   FT_W_BF16     : tensor-core tile order.  inter/16 units of 16 neurons, 96*hidden bytes each: a gate part, an
+ *                   up part and a down part of 32*hidden bytes, all made of 8 x 8 blocks of bf16 (8 rows of 16
+ *                   bytes, 128 contiguous bytes per block).  With n the neuron, i the hidden index, c the output
+ *                   column, offsets in 2-byte elements:
+ *                     W_gate[i][n] at 48*hidden*(n/16) + 512*(i/32) + 256*((n%16)/8) + 64*((i%32)/8) + 8*(n%8) + i%8
+ *                     W_up[i][n]   at the same place + 16*hidden
+ *                     W_down[n][c] at 48*hidden*(n/16) + 32*hidden + 256*(c/16) + 128*((c%16)/8) + 64*((n%16)/8)
+ *                                     + 8*(c%8) + n%8
+ *                   (gate/up: 1 KiB tiles of 16 neurons x 32 hidden indices; down: 512-byte tiles of 16 columns x
+ *                   the unit's 16 neurons).  A warp's 16- or 8-byte loads of a tile are contiguous and land directly
+ *                   in mma.sync fragments; the same blocks are the tensor core's K-major operand layout without
+ *                   swizzle, so the prefill GEMMs consume them as they are.  S = 3*inter*hidden*2 bytes.
  *   FT_W_INT4_G128: 4-bit two's-complement codes in [-8,7] for the same three matrices, then bf16 scales;
  *                   weight = scale * code.
  *                     Wg_q, Wu_q : row-major [inter][hidden/2] bytes, two codes per byte along hidden
@@ -177,18 +188,22 @@ ft_status_t ft_moe_route(ft_moe_t *h, int layer, const float *logits_dev, int T,
  * plan and fills *out_host (HOST arrays owned by the caller). */
 ft_status_t ft_moe_plan(ft_moe_t *h, int layer, ft_moe_plan_t *out_host, void *stream);
 
-/* Step 4: for every (expert, slot) of F copy the S-byte pool record into the slot on copy_stream
- * and record the handle's fill event there.  The copies are ordered after the plan. */
+/* Step 4 (paper Sec. 3.2: the fill set F is brought into the cache "by a batch copy" before the grouped
+ * evaluation; Sec. 4.1: one fixed-shape transfer driven by a device-resident source/destination list with a
+ * valid count): for every (expert, slot) of F copy the S-byte pool record into the slot on copy_stream and
+ * record the handle's fill event there.  The copies are ordered after the plan. */
 ft_status_t ft_moe_fill(ft_moe_t *h, int layer, void *copy_stream);
 
-/* Steps 5+6: x_dev DEVICE bf16 [T][hidden], y_dev DEVICE bf16 [T][hidden] (written).  Waits (on the
+/* Steps 5+6 (paper Sec. 3.2: grouped evaluation of H u F on the GPU, the in-place set beside it, and an exact
+ * merge of the partial sums -- no approximation of the MoE output): x_dev DEVICE bf16 [T][hidden], y_dev DEVICE
+ * bf16 [T][hidden] (written), both 16-byte aligned.  Waits (on the
  * stream, not the host) for the fill event, evaluates the SwiGLU expert FFN of every routed expert
  * from its slot or, for the zero-copy set, straight from the mapped host pool, and writes
  * y[t] = sum_j w[t][j] * FFN_{ids[t][j]}(x[t]) (+ the shared expert) rounded once to bf16. */
 ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_dev, void *stream);
 
-/* route + plan + fill + forward of one layer in one call; fills go to the handle's own copy
- * stream. */
+/* route + plan + fill + forward of one layer in one call (the per-layer control flow of paper Sec. 4.1, kept on
+ * the device); fills go to the handle's own copy stream. */
 ft_status_t ft_moe_layer(ft_moe_t *h, int layer, const float *logits_dev, const void *x_dev,
                          void *y_dev, int T, void *stream);
 
@@ -208,7 +223,9 @@ ft_status_t ft_moe_get_slot_table(ft_moe_t *h, int layer, int32_t *slot_expert,
 ft_status_t ft_moe_read_slot(ft_moe_t *h, int layer, int slot, void *host_dst /* S bytes */);
 /* counters[FT_STAT_*], accumulated since create/reset. */
 ft_status_t ft_moe_get_stats(ft_moe_t *h, int layer, uint64_t *counters, int n);
-/* Empties the slot table and zeroes step counter and statistics; layer = -1 for all layers. */
+/* Empties the slot table and zeroes step counter and statistics; layer = -1 for all layers.  (Paper Sec. 3.3: GPU
+ * residency is disposable -- the host pool is the source of truth and a cold cache is served by the ordinary miss
+ * path -- so a reset never loses anything but speed.) */
 ft_status_t ft_moe_reset(ft_moe_t *h, int layer);
 /* Runtime cache reconfiguration (paper Sec. 3.3): rebuilds the slot pool for a new budget of
  * slots_per_layer slots per layer (n_layers * slots_per_layer shared slots with global_pool) without touching
@@ -253,8 +270,8 @@ const char *ft_moe_last_cuda_error(void);
  * What it does: y[t] = (SiLU(x[t] W_gate) * (x[t] W_up)) W_down for t < T, with the same streaming
  * tensor-core kernel ft_moe_forward uses for resident bf16 experts.
  *   record_dev : DEVICE, one FT_W_BF16 expert record (layout above), 16-byte aligned, caller-owned
- *   x_dev      : DEVICE bf16 [T][hidden], caller-owned, read only
- *   y_dev      : DEVICE bf16 [T][hidden], caller-owned, written
+ *   x_dev      : DEVICE bf16 [T][hidden], 16-byte aligned, caller-owned, read only
+ *   y_dev      : DEVICE bf16 [T][hidden], 16-byte aligned, caller-owned, written
  *   stream     : cudaStream_t; the call only enqueues work
  * The kernel's scratch (an fp32 [T][hidden] accumulator and a few control words) lives in a fixed
  * array of FT_NOALLOC_MAX_TOKENS * FT_NOALLOC_MAX_HIDDEN * 4 + 256 bytes (512.25 KiB) in the library's
@@ -263,7 +280,9 @@ const char *ft_moe_last_cuda_error(void);
  *
  * Limits and errors: T in [1, FT_NOALLOC_MAX_TOKENS] and hidden <= FT_NOALLOC_MAX_HIDDEN, otherwise
  * FT_ERR_INVALID_ARG (the scratch cannot be grown); hidden in {256, 512, 1024, 2048} and
- * inter % 16 == 0, otherwise FT_ERR_UNSUPPORTED; null pointers FT_ERR_INVALID_ARG.
+ * inter % 16 == 0, otherwise FT_ERR_UNSUPPORTED; null or misaligned pointers FT_ERR_INVALID_ARG.
+ * The calling thread's current device is the same after the call as before it.  The device must already have a
+ * context (creating one allocates): make any other CUDA call on it first.
  *
  * First call on a device: looks up the device address of the scratch array and raises the kernel's
  * shared-memory limit for that device (no allocation, but not stream work either), so make the
@@ -277,6 +296,10 @@ const char *ft_moe_last_cuda_error(void);
 #define FT_NOALLOC_MAX_HIDDEN 2048
 ft_status_t ft_moe_ffn_noalloc(int device, const void *record_dev, int hidden, int inter,
                                const void *x_dev, void *y_dev, int T, void *stream);
+/* Waits for the device and returns (and clears) what the ft_moe_ffn_noalloc kernels latched there since the last
+ * call of this function: FT_OK, or FT_ERR_TIMEOUT if a bounded device-side wait gave up (the y of that call is
+ * then incomplete).  Allocates nothing. */
+ft_status_t ft_moe_ffn_noalloc_status(int device);
 
 #ifdef __cplusplus
 }

@@ -28,7 +28,7 @@ SYMBOLS = (
     "ft_moe_get_stats", "ft_moe_reset", "ft_moe_sync_status", "ft_moe_last_fill", "ft_moe_launch_count",
     "ft_moe_status_string", "ft_moe_timing_enable", "ft_moe_timing_read", "ft_moe_ffn_noalloc",
     "ft_moe_last_cuda_error", "ft_moe_host_register", "ft_moe_host_unregister",
-    "ft_moe_get_cta_trace", "ft_moe_set_split_min_pairs", "ft_moe_resize",
+    "ft_moe_get_cta_trace", "ft_moe_set_split_min_pairs", "ft_moe_resize", "ft_moe_ffn_noalloc_status",
 )
 NOALLOC_MAX_TOKENS, NOALLOC_MAX_HIDDEN = 64, 2048
 TIME_NAMES = ("route", "plan", "ffn_zc", "ffn_res", "finalize", "fill", "gather", "gemm1", "gemm2", "combine")
@@ -111,6 +111,7 @@ def load(rebuild: bool = False):
         "ft_moe_timing_read": (i32, [vp, vp, vp, i32]),
         "ft_moe_ffn_noalloc": (i32, [i32, vp, i32, i32, vp, vp, i32, vp]),
         "ft_moe_last_cuda_error": (C.c_char_p, []),
+        "ft_moe_ffn_noalloc_status": (i32, [i32]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -157,6 +158,11 @@ def ft_moe_ffn_noalloc(device, record_dev, hidden, inter, x_dev, y_dev, T, strea
     inside the library).  Returns the status code; see ``include/ftmoe.h`` for the limits."""
     return int(load().ft_moe_ffn_noalloc(device, _ptr(record_dev), hidden, inter, _ptr(x_dev), _ptr(y_dev), T,
                                          _stream(stream)))
+
+
+def ft_moe_ffn_noalloc_status(device) -> int:
+    """Waits for the device; returns and clears the status the allocation-free kernels latched there."""
+    return int(load().ft_moe_ffn_noalloc_status(device))
 
 
 class HostPool:

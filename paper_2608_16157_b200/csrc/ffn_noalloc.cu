@@ -11,7 +11,10 @@
 
 #include <cuda_runtime.h>
 
-#include "ffn_mma.cuh"
+#include <cstddef>
+#include <mutex>
+
+#include "ffn_stream.cuh"
 
 using namespace ftmoe;
 
@@ -30,7 +33,7 @@ struct NoAllocCtl {
   int32_t n_items;     // 1
   int32_t n_zc;        // 0: no host-resident records here
   uint32_t done;       // CTA completion counter of the kernel
-  uint32_t status;     // latched device status of the last call
+  uint32_t status;     // latched device status, read and cleared by ft_moe_ffn_noalloc_status
 };
 static_assert(sizeof(NoAllocCtl) <= kCtlBytes, "control block too large");
 
@@ -52,32 +55,41 @@ __global__ void noalloc_setup_kernel(const uint8_t *record, int T, int hidden) {
     ctl->item.off = 0;
     ctl->item.slot = -1;
     ctl->pref[0] = 0;
-    ctl->pref[1] = (T + kMmaTokens - 1) / kMmaTokens;
+    ctl->pref[1] = (T + kFsResTokensPerPass - 1) / kFsResTokensPerPass;
     ctl->n_items = 1;
     ctl->n_zc = 0;
     ctl->done = 0u;
-    ctl->status = 0u;
+    // ctl->status stays latched until ft_moe_ffn_noalloc_status reads and clears it
   }
 }
 
 constexpr int kMaxDevices = 64;
+std::mutex g_setup_mutex;                               // guards the two tables below
 unsigned char *g_scratch_ptr[kMaxDevices] = {nullptr};  // device address of the array, per device
 int g_sm_count[kMaxDevices] = {0};
+
+// Restores the calling thread's current device when the entry point returns.
+struct DeviceGuard {
+  int prev = -1;
+  DeviceGuard() { if (cudaGetDevice(&prev) != cudaSuccess) { prev = -1; (void)cudaGetLastError(); } }
+  ~DeviceGuard() { if (prev >= 0) (void)cudaSetDevice(prev); }
+};
 
 // Once per device, with that device current: resolve the array's device address and raise the
 // kernels' dynamic shared memory limit.  Neither call allocates.
 ft_status_t noalloc_setup_device(int dev) {
+  std::lock_guard<std::mutex> lock(g_setup_mutex);
   if (g_scratch_ptr[dev] != nullptr) return FT_OK;
   unsigned char *ptr = nullptr;
   if (cudaGetSymbolAddress(reinterpret_cast<void **>(&ptr), g_noalloc_scratch) != cudaSuccess || ptr == nullptr) {
     (void)cudaGetLastError();
     return FT_ERR_CUDA;
   }
-  const int smem = (int)ffn_mma_smem_bytes(kNoAllocMaxHidden);
-  if (cudaFuncSetAttribute(ffn_mma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
-      cudaFuncSetAttribute(ffn_mma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
-      cudaFuncSetAttribute(ffn_mma_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
-      cudaFuncSetAttribute(ffn_mma_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+  const int smem = (int)ffn_stream_smem_bytes(1, kNoAllocMaxHidden);
+  if (cudaFuncSetAttribute(ffn_stream_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+      cudaFuncSetAttribute(ffn_stream_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+      cudaFuncSetAttribute(ffn_stream_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+      cudaFuncSetAttribute(ffn_stream_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
     (void)cudaGetLastError();
     return FT_ERR_CUDA;
   }
@@ -100,16 +112,25 @@ extern "C" ft_status_t ft_moe_ffn_noalloc(int device, const void *record_dev, in
   if (hidden > kNoAllocMaxHidden) return FT_ERR_INVALID_ARG;           // beyond the static scratch
   if ((hidden != 256 && hidden != 512 && hidden != 1024 && hidden != 2048) || inter < 16 || inter % 16)
     return FT_ERR_UNSUPPORTED;
+  // the kernel reads the record and x with 16-byte loads and writes y with 8-byte stores
+  if (((uintptr_t)record_dev | (uintptr_t)x_dev | (uintptr_t)y_dev) & 15) return FT_ERR_INVALID_ARG;
+  DeviceGuard guard;
   if (cudaSetDevice(device) != cudaSuccess) { (void)cudaGetLastError(); return FT_ERR_CUDA; }
   ft_status_t rc = noalloc_setup_device(device);
   if (rc != FT_OK) return rc;
-  unsigned char *scratch = g_scratch_ptr[device];
+  unsigned char *scratch;
+  int grid;
+  {
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
+    scratch = g_scratch_ptr[device];
+    grid = g_sm_count[device];
+  }
   NoAllocCtl *ctl = reinterpret_cast<NoAllocCtl *>(scratch + kAccBytes);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
 
   noalloc_setup_kernel<<<32, 256, 0, st>>>(static_cast<const uint8_t *>(record_dev), T, hidden);
 
-  FfnMmaParams mp;
+  FfnStreamParams mp;
   mp.items = &ctl->item;
   mp.n_items = &ctl->n_items;
   mp.n_zc = &ctl->n_zc;
@@ -125,15 +146,36 @@ extern "C" ft_status_t ft_moe_ffn_noalloc(int device, const void *record_dev, in
   mp.y = static_cast<__nv_bfloat16 *>(y_dev);
   mp.done = &ctl->done;
   mp.status = &ctl->status;
-  mp.d = hidden; mp.inter = inter; mp.top_k = 1; mp.T = T; mp.finalize = 1;
-  const size_t smem = ffn_mma_smem_bytes(hidden);
-  const int grid = g_sm_count[device];
+  mp.inter = inter; mp.top_k = 1; mp.T = T; mp.finalize = 1;
+  const size_t smem = ffn_stream_smem_bytes(1, hidden);
   switch (hidden / 256) {
-    case 1: ffn_mma_kernel<1><<<grid, kMmaThreads, smem, st>>>(mp); break;
-    case 2: ffn_mma_kernel<2><<<grid, kMmaThreads, smem, st>>>(mp); break;
-    case 4: ffn_mma_kernel<4><<<grid, kMmaThreads, smem, st>>>(mp); break;
-    default: ffn_mma_kernel<8><<<grid, kMmaThreads, smem, st>>>(mp); break;
+    case 1: ffn_stream_kernel<1><<<grid, kFsThreads, smem, st>>>(mp); break;
+    case 2: ffn_stream_kernel<2><<<grid, kFsThreads, smem, st>>>(mp); break;
+    case 4: ffn_stream_kernel<4><<<grid, kFsThreads, smem, st>>>(mp); break;
+    default: ffn_stream_kernel<8><<<grid, kFsThreads, smem, st>>>(mp); break;
   }
   if (cudaGetLastError() != cudaSuccess) return FT_ERR_CUDA;
+  return FT_OK;
+}
+
+extern "C" ft_status_t ft_moe_ffn_noalloc_status(int device) {
+  if (device < 0 || device >= kMaxDevices) return FT_ERR_INVALID_ARG;
+  DeviceGuard guard;
+  if (cudaSetDevice(device) != cudaSuccess) { (void)cudaGetLastError(); return FT_ERR_CUDA; }
+  if (cudaDeviceSynchronize() != cudaSuccess) { (void)cudaGetLastError(); return FT_ERR_CUDA; }
+  const size_t off = kAccBytes + offsetof(NoAllocCtl, status);
+  uint32_t st = 0;
+  if (cudaMemcpyFromSymbol(&st, g_noalloc_scratch, sizeof(st), off, cudaMemcpyDeviceToHost) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return FT_ERR_CUDA;
+  }
+  if (st != 0) {
+    const uint32_t zero = 0;
+    if (cudaMemcpyToSymbol(g_noalloc_scratch, &zero, sizeof(zero), off, cudaMemcpyHostToDevice) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return FT_ERR_CUDA;
+    }
+    return (st & kStatTimeout) ? FT_ERR_TIMEOUT : FT_ERR_CUDA;
+  }
   return FT_OK;
 }

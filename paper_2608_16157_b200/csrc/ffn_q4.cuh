@@ -18,10 +18,11 @@
 // Zero-copy experts (records in the mapped host pool) go through the same kernels.
 #pragma once
 #include "common.cuh"
-#include "ffn_mma.cuh"
+#include "async.cuh"
 
 namespace ftmoe {
 
+constexpr int kQ4Tokens = 8;        // tokens per weight pass
 constexpr int kQ4Threads = 288;     // 8 consumer warps + 1 producer warp
 constexpr int kQ4StagesA = 3;
 constexpr int kQ4StagesB = 8;

@@ -3,7 +3,7 @@
 // Also the read kernels used by the bandwidth calibration.
 #pragma once
 #include "common.cuh"
-#include "ffn_mma.cuh"   // mbarrier / bulk-copy helpers
+#include "async.cuh"
 
 namespace ftmoe {
 

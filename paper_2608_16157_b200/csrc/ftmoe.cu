@@ -9,7 +9,7 @@
 #include <vector>
 
 #include "common.cuh"
-#include "ffn_mma.cuh"
+#include "ffn_stream.cuh"
 #include "ffn_q4.cuh"
 #include "gemm_tc.cuh"
 #include "gemm_tc2.cuh"
@@ -21,6 +21,7 @@ using namespace ftmoe;
 namespace {
 
 enum LayerPhase { PH_IDLE = 0, PH_ROUTED, PH_PLANNED, PH_FILLED };
+constexpr int kMaxTableSlots = 6144;   // slots of one residency table (per layer, or the shared pool)
 
 struct LayerState {
   int32_t *slot_expert = nullptr;
@@ -64,7 +65,8 @@ struct ft_moe {
   int32_t *gemm_pref = nullptr;
   uint8_t *is_gemm = nullptr;
   __nv_bfloat16 *xs = nullptr, *hbuf = nullptr, *obuf = nullptr;   // [P][d], [P][I], [P][d]
-  CUtensorMap tm_xs, tm_h, tm_w128, tm_w64;   // x rows, H rows (128-row boxes), weight rows (128 / 64-row boxes)
+  CUtensorMap tm_xs, tm_h;       // x rows, H rows (128-row boxes, 128-byte swizzle)
+  CUtensorMap tm_wgu, tm_wd;     // the slot pool as [unit][1 KiB gate/up tile] and [unit][2 KiB of down tiles]
   uint32_t *status_dev = nullptr;
   uint32_t *seq_dev = nullptr;
   uint32_t *done_dev = nullptr;          // CTA completion counter of the streaming MMA kernel
@@ -244,11 +246,9 @@ ft_status_t alloc_cache(ft_moe *h) {
     ft_status_t rc = reset_layer(h, (int)l, true);
     if (rc != FT_OK) return rc;
   }
-  const int dyn = h->table_slots * 16;
-  if ((size_t)dyn + 36 * 1024 > 48 * 1024) {
-    FT_CUDA(cudaFuncSetAttribute(plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn));
-    FT_CUDA(cudaFuncSetAttribute(route_plan_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn));
-  }
+  // (the limit belongs to the function on this device, not to the handle: always the largest table)
+  FT_CUDA(cudaFuncSetAttribute(plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxTableSlots * 16));
+  FT_CUDA(cudaFuncSetAttribute(route_plan_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxTableSlots * 16));
   return FT_OK;
 }
 
@@ -266,6 +266,38 @@ bool make_tensor_map(EncodeTiledFn fn, CUtensorMap *tm, void *base, uint64_t row
   return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
          CUDA_SUCCESS;
+}
+
+// The slot pool as a 3-D tensor of 8-byte words: [16-neuron unit][piece of `piece_bytes` inside the unit][words of
+// the piece]; a box is `box_pieces` consecutive pieces of `box_units` consecutive units.
+bool make_unit_map(EncodeTiledFn fn, CUtensorMap *tm, void *base, uint64_t n_units, uint64_t unit_bytes,
+                   uint32_t piece_bytes, uint32_t box_pieces, uint32_t box_units) {
+  const cuuint64_t dims[3] = {piece_bytes / 8, unit_bytes / piece_bytes, n_units};
+  const cuuint64_t strides[2] = {piece_bytes, unit_bytes};
+  const cuuint32_t box[3] = {piece_bytes / 8, box_pieces, box_units};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+         CUDA_SUCCESS;
+}
+
+// Tensor maps of the weight operands of the prefill GEMMs over the current slot pool.
+ft_status_t build_weight_maps(ft_moe *h) {
+  const ft_moe_config_t &c = h->cfg;
+  void *fnp = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  FT_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fnp, cudaEnableDefault, &qres));
+  if (!fnp || qres != cudaDriverEntryPointSuccess) return FT_ERR_CUDA;
+  EncodeTiledFn enc = reinterpret_cast<EncodeTiledFn>(fnp);
+  const uint64_t n_units = (uint64_t)c.n_layers * c.slots_per_layer * (c.inter / 16);
+  const uint64_t unit_bytes = 96ull * c.hidden;
+  if (n_units == 0) return FT_OK;   // no slots: nothing goes through the GEMMs
+  // gate/up: one 1 KiB tile (16 neurons x 32 hidden indices) of 8 consecutive units = 128 neurons;
+  // down: 4 KiB (the tiles of 128 output columns) of 4 consecutive units = 64 neurons
+  if (!make_unit_map(enc, &h->tm_wgu, h->slots, n_units, unit_bytes, 1024, 1, 8) ||
+      !make_unit_map(enc, &h->tm_wd, h->slots, n_units, unit_bytes, 2048, 2, 4))
+    return FT_ERR_CUDA;
+  return FT_OK;
 }
 
 }  // namespace
@@ -379,7 +411,7 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
   if (c.n_layers <= 0 || c.n_experts <= 0 || c.n_experts > kMaxExperts || c.top_k <= 0 ||
       c.top_k > c.n_experts || c.top_k > kMaxTopK || c.slots_per_layer < 0 ||
       (c.global_pool != 0 && c.global_pool != 1) ||
-      (long long)c.slots_per_layer * (c.global_pool ? c.n_layers : 1) > 6144 ||
+      (long long)c.slots_per_layer * (c.global_pool ? c.n_layers : 1) > kMaxTableSlots ||
       c.max_tokens <= 0 || (c.n_shared != 0 && c.n_shared != 1) || c.device < 0 ||
       (c.fill_mode != FT_FILL_COPY_ENGINE && c.fill_mode != FT_FILL_SM))
     return FT_ERR_INVALID_ARG;
@@ -487,12 +519,11 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
     FT_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fnp, cudaEnableDefault, &qres));
     if (!fnp || qres != cudaDriverEntryPointSuccess) return fail(FT_ERR_CUDA);
     EncodeTiledFn enc = reinterpret_cast<EncodeTiledFn>(fnp);
-    const uint64_t wrows = (uint64_t)L * Ns * 3 * c.inter;
     if (!make_tensor_map(enc, &h->tm_xs, h->xs, Pr, c.hidden, 128, 64) ||
-        !make_tensor_map(enc, &h->tm_h, h->hbuf, Pr, c.inter, 128, 64) ||
-        !make_tensor_map(enc, &h->tm_w128, h->slots, wrows, c.hidden, 128, 64) ||
-        !make_tensor_map(enc, &h->tm_w64, h->slots, wrows, c.hidden, 64, 64))
+        !make_tensor_map(enc, &h->tm_h, h->hbuf, Pr, c.inter, 128, 64))
       return fail(FT_ERR_CUDA);
+    rc = build_weight_maps(h);
+    if (rc != FT_OK) return fail(rc);
     FT_TRY(cudaFuncSetAttribute(gateup_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)gateup_gemm_smem_bytes()));
     FT_TRY(cudaFuncSetAttribute(down_gemm2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -511,7 +542,7 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
   if (c.wdtype == FT_W_INT4_G128) {
     const size_t passes = (P + 7) / 8 + 2 * E + 2;
     FT_TRY(cudaMalloc(&h->q4_hbuf, passes * (c.inter / 16) * 32 * sizeof(uint2)));
-    const int sa = (int)q4_gateup_smem_bytes(c.hidden), sb = (int)q4_down_smem_bytes(c.hidden);
+    const int sa = (int)q4_gateup_smem_bytes(8192), sb = (int)q4_down_smem_bytes(8192);   // largest hidden size
     FT_TRY(cudaFuncSetAttribute(q4_gateup_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
     FT_TRY(cudaFuncSetAttribute(q4_gateup_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
     FT_TRY(cudaFuncSetAttribute(q4_gateup_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
@@ -525,11 +556,13 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
     FT_TRY(cudaFuncSetAttribute(q4_down_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
   }
   if (c.wdtype == FT_W_BF16) {
-    const int smem = (int)ffn_mma_smem_bytes(c.hidden);
-    FT_TRY(cudaFuncSetAttribute(ffn_mma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    FT_TRY(cudaFuncSetAttribute(ffn_mma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    FT_TRY(cudaFuncSetAttribute(ffn_mma_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    FT_TRY(cudaFuncSetAttribute(ffn_mma_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    // the limit is a property of the function on this device, not of the handle: always the largest size any
+    // handle can ask for, so that handles of different shapes can live side by side
+    const int smem = (int)ffn_stream_smem_bytes(2 * kMaxExperts + 1, 2048);
+    FT_TRY(cudaFuncSetAttribute(ffn_stream_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    FT_TRY(cudaFuncSetAttribute(ffn_stream_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    FT_TRY(cudaFuncSetAttribute(ffn_stream_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    FT_TRY(cudaFuncSetAttribute(ffn_stream_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
   }
   FT_TRY(cudaMalloc(&h->stage_logits, (size_t)c.max_tokens * E * 4));
   FT_TRY(cudaMalloc(&h->stage_x, (size_t)c.max_tokens * c.hidden * 2));
@@ -605,8 +638,8 @@ static PlanParams make_plan_params(ft_moe *h, int layer, bool mirror_to_host) {
   pp.slots_layer = h->slots ? h->slots + (c.global_pool ? 0 : (size_t)layer * c.slots_per_layer * h->S) : nullptr;
   pp.shared_rec = c.n_shared ? h->shared_dev + (size_t)layer * h->S : nullptr;
   pp.S = h->S; pp.T = L.T;
-  pp.tokens_per_pass = kMmaTokens;
-  pp.zc_single_pass = (c.wdtype == FT_W_BF16) ? 1 : 0;
+  pp.tokens_per_pass = (c.wdtype == FT_W_BF16) ? kFsResTokensPerPass : kQ4Tokens;
+  pp.zc_tokens_per_pass = (c.wdtype == FT_W_BF16) ? kFsZcTokensPerPass : kQ4Tokens;
   pp.hdr_dev = h->plan_dev;
   pp.hdr_host = mirror_to_host ? h->plan_host_devptr : nullptr;
   pp.items_res = h->items_res; pp.res_pref = h->res_pref;
@@ -761,13 +794,14 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   L.phase = PH_IDLE;
   if (L.T == 0) return FT_OK;
   if (!x_dev || !y_dev) return FT_ERR_INVALID_ARG;
+  if (((uintptr_t)x_dev | (uintptr_t)y_dev) & 15) return FT_ERR_INVALID_ARG;   // the kernels use 16-byte vector accesses
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const ft_moe_config_t &c = h->cfg;
   const __nv_bfloat16 *x_bf = static_cast<const __nv_bfloat16 *>(x_dev);
   const bool use_gemm = h->gemm && L.T >= c.gemm_min_tokens;
   if (c.wdtype == FT_W_BF16) {
     // bulk-copy pipelined tensor-core streaming kernel; the last CTA of the last launch finalizes y
-    FfnMmaParams mp;
+    FfnStreamParams mp;
     mp.items = h->items_res;
     mp.n_items = &h->plan_dev->n_res_items;
     mp.n_hit = &h->plan_dev->n_hit_items;
@@ -778,8 +812,8 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     mp.x = x_bf; mp.perm = h->perm; mp.topk_w = h->topk_w; mp.y_acc = h->y_acc;
     mp.y = static_cast<__nv_bfloat16 *>(y_dev);
     mp.done = h->done_dev; mp.status = h->status_dev;
-    mp.d = c.hidden; mp.inter = c.inter; mp.top_k = c.top_k; mp.T = L.T;
-    const size_t smem = ffn_mma_smem_bytes(c.hidden);
+    mp.inter = c.inter; mp.top_k = c.top_k; mp.T = L.T;
+    const size_t smem = ffn_stream_smem_bytes(mp.max_items, c.hidden);
     auto launch = [&](int part, int finalize) {
       mp.part = part;
       mp.finalize = finalize;
@@ -787,10 +821,10 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
       // while the device-driven fill holds kFillCtas SMs, the overlapping launch takes the others
       const int grid = (part == 1 && c.fill_mode == FT_FILL_SM) ? h->sm_count - kFillCtas : h->sm_count;
       switch (c.hidden / 256) {
-        case 1: ffn_mma_kernel<1><<<grid, kMmaThreads, smem, st>>>(mp); break;
-        case 2: ffn_mma_kernel<2><<<grid, kMmaThreads, smem, st>>>(mp); break;
-        case 4: ffn_mma_kernel<4><<<grid, kMmaThreads, smem, st>>>(mp); break;
-        default: ffn_mma_kernel<8><<<grid, kMmaThreads, smem, st>>>(mp); break;
+        case 1: ffn_stream_kernel<1><<<grid, kFsThreads, smem, st>>>(mp); break;
+        case 2: ffn_stream_kernel<2><<<grid, kFsThreads, smem, st>>>(mp); break;
+        case 4: ffn_stream_kernel<4><<<grid, kFsThreads, smem, st>>>(mp); break;
+        default: ffn_stream_kernel<8><<<grid, kFsThreads, smem, st>>>(mp); break;
       }
       h->launches++;
     };
@@ -816,7 +850,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
       GemmParams gp;
       gp.items = h->items_gemm; gp.n_items = &h->plan_dev->n_gemm_items; gp.mt_pref = h->gemm_pref;
       gp.inter = c.inter; gp.d = c.hidden;
-      gp.layer_row0 = c.global_pool ? 0 : (long long)layer * c.slots_per_layer * 3 * c.inter;
+      gp.layer_unit0 = c.global_pool ? 0 : (long long)layer * c.slots_per_layer * (c.inter / 16);
       gp.status = h->status_dev;
       // CTA pairs (clusters of two) share every 256x256 tile
       cudaLaunchConfig_t lc = {};
@@ -833,14 +867,14 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
       gp.K = c.hidden; gp.n_tiles = c.inter / 128; gp.out = h->hbuf;
       {
         TimeScope ts(h, st, FT_TIME_GEMM1);
-        gateup_gemm_kernel<<<h->sm_count, kGemmThreads, gateup_gemm_smem_bytes(), st>>>(h->tm_xs, h->tm_w128, gp);
+        gateup_gemm_kernel<<<h->sm_count, kGemmThreads, gateup_gemm_smem_bytes(), st>>>(h->tm_xs, h->tm_wgu, gp);
       }
-      // down: A = Wd[k][column] (box 64 columns x 64 k rows, twice), B = H rows (box 64 x 128 per CTA)
+      // down: A = the down tiles of 128 columns x 64 neurons per CTA, B = H rows (box 64 x 128 per CTA)
       gp.K = c.inter; gp.out = h->obuf;
       lc.dynamicSmemBytes = down_gemm2_smem_bytes();
       {
         TimeScope ts(h, st, FT_TIME_GEMM2);
-        FT_CUDA(cudaLaunchKernelEx(&lc, down_gemm2_kernel, h->tm_w64, h->tm_h, gp));
+        FT_CUDA(cudaLaunchKernelEx(&lc, down_gemm2_kernel, h->tm_wd, h->tm_h, gp));
       }
       {
         TimeScope ts(h, st, FT_TIME_COMBINE);
@@ -1041,8 +1075,7 @@ ft_status_t ft_moe_get_cta_trace(ft_moe_t *h, int64_t *out, int n_ctas) {
 
 ft_status_t ft_moe_resize(ft_moe_t *h, int slots_per_layer) {
   if (!h || slots_per_layer < 0) return FT_ERR_INVALID_ARG;
-  if ((long long)slots_per_layer * (h->cfg.global_pool ? h->cfg.n_layers : 1) > 6144) return FT_ERR_INVALID_ARG;
-  if (h->gemm) return FT_ERR_UNSUPPORTED;   // the tensor maps of the prefill path are bound to the slot pool
+  if ((long long)slots_per_layer * (h->cfg.global_pool ? h->cfg.n_layers : 1) > kMaxTableSlots) return FT_ERR_INVALID_ARG;
   FT_CUDA(cudaSetDevice(h->cfg.device));
   FT_CUDA(cudaDeviceSynchronize());
   for (auto &L : h->layers) L.phase = PH_IDLE;
@@ -1052,6 +1085,10 @@ ft_status_t ft_moe_resize(ft_moe_t *h, int slots_per_layer) {
     h->cfg.slots_per_layer = 0;
     (void)alloc_cache(h);
     return rc;
+  }
+  if (h->gemm) {   // the weight tensor maps of the prefill path are bound to the slot pool
+    rc = build_weight_maps(h);
+    if (rc != FT_OK) return rc;
   }
   FT_CUDA(cudaDeviceSynchronize());
   return FT_OK;

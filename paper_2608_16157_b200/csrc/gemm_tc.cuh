@@ -1,11 +1,14 @@
 // Step 5 for prefill-sized token counts: the gate/up half of the grouped SwiGLU expert FFN on the
 // 5th-generation tensor cores, plus the helpers shared with the down-projection kernel (gemm_tc2.cuh), the row
 // gather and the fused gather-combine.
-//   H[P][I] = SiLU(Xs Wg^T) * (Xs Wu^T)   A = expert-sorted x rows (K-major), B = 128 gate rows + the same 128 up
-//                                          rows of the record (K-major), N = 256, over the experts that hold a
-//                                          slot and have at least `gemm_min_tokens` tokens.
+//   H[P][I] = SiLU(Xs Wg^T) * (Xs Wu^T)   A = expert-sorted x rows (K-major, 128-byte swizzle), B = 128 gate rows +
+//                                          the same 128 up rows of the record, N = 256, over the experts that hold
+//                                          a slot and have at least `gemm_min_tokens` tokens.
+// The record's tile order is already the tensor core's K-major layout without swizzle (8 x 8 blocks of 128
+// contiguous bytes): a weight tile is moved by plain TMA boxes of whole 1 KiB tiles and described to the MMA with a
+// 128-byte step between the two blocks of a K = 16 slice and a 512-byte step between 8-row groups.
 // One persistent CTA per SM: warp 0 feeds a 4-stage shared-memory ring with TMA tile loads (cp.async.bulk.tensor,
-// 128-byte swizzle, no multicast), warp 1 issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32) into one of two
+// no multicast), warp 1 issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32) into one of two
 // 256-column TMEM accumulators and signals stages free / tiles done with tcgen05.commit, warps 2-5 drain the other
 // accumulator with tcgen05.ld, apply SwiGLU and store bf16, so the epilogue of tile i overlaps the main loop of
 // tile i+1.  Every mbarrier wait is bounded; on expiry the CTA latches a timeout status, stops waiting, frees its
@@ -15,7 +18,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
-#include "ffn_mma.cuh"  // mbarrier helpers
+#include "async.cuh"
 
 namespace ftmoe {
 
@@ -29,10 +32,10 @@ struct GemmParams {
   const WorkItem *items;
   const int32_t *n_items;
   const int32_t *mt_pref;   // [n_items+1] exclusive prefix of 128-row tiles per item
-  int K;                    // contraction length: d (MODE 0) or I (MODE 1)
-  int n_tiles;              // N tiles per row tile: I/128 (MODE 0) or d/256 (MODE 1)
+  int K;                    // contraction length: d (gate/up) or I (down)
+  int n_tiles;              // N tiles per row tile: I/128 (gate/up)
   int inter, d;
-  long long layer_row0;     // row of slot 0 of this layer in the weight tensor map
+  long long layer_unit0;    // 16-neuron unit index of slot 0 of this layer in the weight tensor maps
   __nv_bfloat16 *out;       // H [P][I] (MODE 0) or O [P][d] (MODE 1)
   uint32_t *status;
 };
@@ -44,14 +47,22 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm,
       : "memory");
 }
 
-// 64-bit shared-memory matrix descriptor, 128-byte swizzle.  lbo/sbo in bytes.
-__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr, uint32_t lbo, uint32_t sbo) {
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+      "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar)
+      : "memory");
+}
+
+// 64-bit shared-memory matrix descriptor.  lbo/sbo in bytes; swizzle: 2 = 128-byte swizzle, 0 = none (8 x 8 blocks of
+// 128 contiguous bytes; K-major: lbo = step between the two blocks of a K = 16 slice, sbo = step between 8-row groups).
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr, uint32_t lbo, uint32_t sbo, uint32_t swizzle = 2) {
   uint64_t d = 0;
   d |= (uint64_t)((smem_addr >> 4) & 0x3fffu);
   d |= (uint64_t)((lbo >> 4) & 0x3fffu) << 16;
   d |= (uint64_t)((sbo >> 4) & 0x3fffu) << 32;
   d |= (uint64_t)1 << 46;   // descriptor version of this architecture
-  d |= (uint64_t)2 << 61;   // 128-byte swizzle
+  d |= (uint64_t)swizzle << 61;
   return d;
 }
 
@@ -99,7 +110,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 gateup_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  constexpr int MODE = 0, MT = 1, kBufs = kGemmBufs;   // one 128-row tile per unit, two accumulator buffers
+  constexpr int MT = 1, kBufs = kGemmBufs;   // one 128-row tile per unit, two accumulator buffers
   unsigned char *sp = smem + kGemmStages * kGemmStageBytes;
   uint64_t *s_bar = reinterpret_cast<uint64_t *>(sp); sp += 16 * 8;
   uint32_t *s_tmem = reinterpret_cast<uint32_t *>(sp); sp += 8;
@@ -168,7 +179,7 @@ gateup_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         locate(tile, item, mt_in, n_mt, nt);
         const WorkItem it = p.items[item];
         const int a_row = it.off + mt_in * kGemmBM;
-        const long long rec_row = p.layer_row0 + (long long)it.slot * 3 * p.inter;
+        const int unit0 = (int)(p.layer_unit0 + (long long)it.slot * (p.inter / 16)) + nt * 8;   // 128 neurons = 8 units
         for (int kb = 0; kb < kblocks; ++kb, ++it_k) {
           const int s = it_k % kGemmStages;
           const uint32_t ph = (it_k / kGemmStages) & 1u;
@@ -178,15 +189,11 @@ gateup_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
           const uint32_t sb = sa + MT * kGemmATile;
           mbar_expect_tx(full_bar(s), n_mt * kGemmATile + kGemmBTile);
           for (int m = 0; m < n_mt; ++m) tma_load_2d(sa + m * kGemmATile, &tmA, kb * kGemmBK, a_row + m * kGemmBM, full_bar(s));
-          if (MODE == 0) {
-            const int n0 = nt * 128;
-            tma_load_2d(sb, &tmB, kb * kGemmBK, (int)(rec_row + n0), full_bar(s));                       // gate rows
-            tma_load_2d(sb + 128 * kGemmBK * 2, &tmB, kb * kGemmBK, (int)(rec_row + p.inter + n0), full_bar(s));  // up rows
-          } else {
-            const int c0 = nt * kGemmBN;
-            const int krow = (int)(rec_row + 2 * p.inter + kb * kGemmBK);
+          // per 32-wide hidden tile: 8 gate tiles (8 KiB: 16 groups of 8 neurons, 512 bytes apart) then the 8 up tiles
 #pragma unroll
-            for (int j = 0; j < 4; ++j) tma_load_2d(sb + j * (64 * kGemmBK * 2), &tmB, c0 + 64 * j, krow, full_bar(s));
+          for (int j = 0; j < 2; ++j) {
+            tma_load_3d(sb + j * 16384, &tmB, 0, 2 * kb + j, unit0, full_bar(s));
+            tma_load_3d(sb + j * 16384 + 8192, &tmB, 0, p.d / 32 + 2 * kb + j, unit0, full_bar(s));
           }
         }
       }
@@ -194,7 +201,7 @@ gateup_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
     if (lane == 0) {
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((MODE == 1 ? 1u : 0u) << 16) |
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) |
                              ((uint32_t)(kGemmBN >> 3) << 17) | ((uint32_t)(kGemmBM >> 4) << 24);
       uint32_t it_k = 0, n_tile = 0;
       for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++n_tile) {
@@ -214,8 +221,7 @@ gateup_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             const uint32_t sb = sa + MT * kGemmATile;
 #pragma unroll
             for (int k16 = 0; k16 < kGemmBK / 16; ++k16) {
-              const uint64_t bdesc = (MODE == 0) ? umma_desc(sb + k16 * 32, 16, 1024)
-                                                 : umma_desc(sb + k16 * 2048, 8192, 1024);
+              const uint64_t bdesc = umma_desc(sb + (k16 >> 1) * 16384 + (k16 & 1) * 256, 128, 512, 0);
               for (int m = 0; m < n_mt; ++m) {
                 const uint64_t adesc = umma_desc(sa + m * kGemmATile + k16 * 32, 16, 1024);
                 umma_bf16(d_tmem + (uint32_t)m * kGemmBN, adesc, bdesc, idesc, (kb | k16) != 0 ? 1u : 0u);
@@ -243,7 +249,7 @@ gateup_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
       const bool valid = ok && row_in < it.n_tok;
       const size_t row = (size_t)it.off + row_in;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf + m) * kGemmBN;
-      if (MODE == 0) {
+      {
         __nv_bfloat16 *dst = p.out + row * p.inter + nt * 128;
 #pragma unroll 1
         for (int c = 0; c < 128; c += 32) {
@@ -261,23 +267,6 @@ gateup_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             uint4 *d4 = reinterpret_cast<uint4 *>(dst + c);
 #pragma unroll
             for (int j = 0; j < 4; ++j) d4[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
-          }
-        }
-      } else {
-        __nv_bfloat16 *dst = p.out + row * p.d + nt * kGemmBN;
-#pragma unroll 1
-        for (int c = 0; c < kGemmBN; c += 32) {
-          uint32_t v[32];
-          tmem_ld32(taddr + c, v);
-          tmem_ld_wait();
-          if (valid) {
-            uint4 *d4 = reinterpret_cast<uint4 *>(dst + c);
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-              d4[j] = make_uint4(pack_bf16(__uint_as_float(v[8 * j]), __uint_as_float(v[8 * j + 1])),
-                                 pack_bf16(__uint_as_float(v[8 * j + 2]), __uint_as_float(v[8 * j + 3])),
-                                 pack_bf16(__uint_as_float(v[8 * j + 4]), __uint_as_float(v[8 * j + 5])),
-                                 pack_bf16(__uint_as_float(v[8 * j + 6]), __uint_as_float(v[8 * j + 7])));
           }
         }
       }

@@ -33,6 +33,12 @@ __device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t bar_cluster, uin
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster) {
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
 }
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap *tm, int x, int y, int z, uint32_t bar_cluster) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+      "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar_cluster)
+      : "memory");
+}
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *tm, int x, int y, uint32_t bar_cluster) {
   asm volatile(
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
@@ -47,18 +53,19 @@ __device__ __forceinline__ void umma2_bf16(uint32_t d_tmem, uint64_t a_desc, uin
       "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-// arrives on the mbarrier at this shared-memory offset in both CTAs of the pair once the MMAs issued so far are done
+// arrives on the mbarrier at this shared-memory offset in both CTAs of the pair once the MMAs issued so far are
+// done: one commit per CTA (the leader's own barrier, then the peer's through its cluster address)
 __device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
-  const uint16_t mask = 3;
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
-               "h"(mask)
-               : "memory");
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(mapa_u32(bar, 0)) : "memory");
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(mapa_u32(bar, 1)) : "memory");
 }
 
 // Swapped operands: the weights are the M side (always full 128-row tiles per CTA, 256 per pair), the tokens
 // are the N side, so a ragged expert is padded to a multiple of 16 tokens instead of 128 rows.
-//   O^T[column][token] : A = Wd[k rows][128 columns] (column-contiguous, i.e. MN-major), B = up to 256 rows of H
-//   (each CTA stages half).  TMEM lane = output column, TMEM column = token; the epilogue writes O[token][column].
+//   O^T[column][token] : A = W_down^T, 128 columns per CTA x 64 neurons per stage, taken from the record's down
+//   tiles as they are (K-major 8 x 8 blocks without swizzle: 128 bytes between the two neuron blocks of a unit, 256
+//   bytes between 8-column groups); B = up to 256 rows of H (each CTA stages half).  TMEM lane = output column,
+//   TMEM column = token; the epilogue writes O[token][column].
 struct Gemm2Cfg {
   static constexpr int kTokTile = 256;                                  // tokens per unit
   static constexpr int kStageBytes = kGemmATile + kGemmATile;           // Wd tile 16 KiB + 128 token rows 16 KiB
@@ -69,8 +76,8 @@ struct Gemm2Cfg {
 // abort flag | tile prefix | unit prefix.
 __global__ void __launch_bounds__(kGemmThreads, 1)
 down_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p) {
-  constexpr int MODE = 1;   // (the gate/up form of this kernel, MODE 0, measured slower than gemm_tc.cuh's and is kept
-                            // only as the constant-folded branches below)
+  constexpr int MODE = 1;   // (the gate/up form of this kernel, MODE 0, measured slower than gemm_tc.cuh's; its
+                            // constant-folded branches are gone)
   using Cfg = Gemm2Cfg;
   constexpr int kStages = Cfg::kStages, kStageBytes = Cfg::kStageBytes, kTok = Cfg::kTokTile;
   extern __shared__ unsigned char smem_raw[];
@@ -152,7 +159,7 @@ down_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         n_valid = min(kTok, it.n_tok - tok0);
         const int N = (n_valid + 15) & ~15;
         const int b_row = it.off + tok0 + (int)rank * (N / 2);       // this CTA stages the tokens [rank*N/2, +N/2)
-        const long long rec_row = p.layer_row0 + (long long)it.slot * 3 * p.inter;
+        const int unit0 = (int)(p.layer_unit0 + (long long)it.slot * (p.inter / 16));
         for (int kb = 0; kb < kblocks; ++kb, ++it_k) {
           const int s = it_k % kStages;
           const uint32_t ph = (it_k / kStages) & 1u;
@@ -161,16 +168,9 @@ down_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           const uint32_t sa = smem_base + s * kStageBytes;
           const uint32_t lead_full = mapa_u32(full_bar(s), 0);
           mbar_expect_tx_cluster(lead_full, kStageBytes);
-          if (MODE == 0) {
-            tma_load_2d_pair(sa, &tmA, kb * kGemmBK, (int)(rec_row + m_base), lead_full);                          // gate rows
-            tma_load_2d_pair(sa + kGemmATile, &tmA, kb * kGemmBK, (int)(rec_row + p.inter + m_base), lead_full);   // up rows
-            tma_load_2d_pair(sa + 2 * kGemmATile, &tmB, kb * kGemmBK, b_row, lead_full);                          // 64 token rows
-          } else {
-            const int krow = (int)(rec_row + 2 * p.inter + kb * kGemmBK);
-            tma_load_2d_pair(sa, &tmA, m_base, krow, lead_full);                                  // Wd[k rows][64 columns]
-            tma_load_2d_pair(sa + 64 * kGemmBK * 2, &tmA, m_base + 64, krow, lead_full);
-            tma_load_2d_pair(sa + kGemmATile, &tmB, kb * kGemmBK, b_row, lead_full);              // 128 token rows of H
-          }
+          // the down tiles of 128 columns (4 KiB) of the stage's 4 units (64 neurons): one box of 16 KiB
+          tma_load_3d_pair(sa, &tmA, 0, p.d / 32 + m_base / 64, unit0 + 4 * kb, lead_full);
+          tma_load_2d_pair(sa + kGemmATile, &tmB, kb * kGemmBK, b_row, lead_full);              // 128 token rows of H
         }
       }
     }
@@ -183,9 +183,8 @@ down_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         locate(unit, item, tok0, n_valid, m_base);
         n_valid = min(kTok, p.items[item].n_tok - tok0);
         const uint32_t N = (uint32_t)((n_valid + 15) & ~15);
-        // bf16 x bf16 -> fp32, M = 256 over the pair, N tokens; MODE 1: A is MN-major
-        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((MODE == 1 ? 1u : 0u) << 15) | ((N >> 3) << 17) |
-                               ((uint32_t)(256 >> 4) << 24);
+        // bf16 x bf16 -> fp32, M = 256 over the pair, N tokens, both operands K-major
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((N >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
         const int buf = n_unit & 1;
         mbar_wait(tempty_bar(buf), ((n_unit >> 1) & 1u) ^ 1u, s_abort, p.status);
         tc_fence_after();
@@ -200,14 +199,8 @@ down_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
             for (int k16 = 0; k16 < kGemmBK / 16; ++k16) {
               const uint32_t acc = (kb | k16) != 0 ? 1u : 0u;
-              if (MODE == 0) {
-                const uint64_t bdesc = umma_desc(sa + 2 * kGemmATile + k16 * 32, 16, 1024);
-                umma2_bf16(d_tmem, umma_desc(sa + k16 * 32, 16, 1024), bdesc, idesc, acc);                     // gate
-                umma2_bf16(d_tmem + 128, umma_desc(sa + kGemmATile + k16 * 32, 16, 1024), bdesc, idesc, acc);  // up
-              } else {
-                umma2_bf16(d_tmem, umma_desc(sa + k16 * 2048, 8192, 1024),
-                           umma_desc(sa + kGemmATile + k16 * 32, 16, 1024), idesc, acc);
-              }
+              umma2_bf16(d_tmem, umma_desc(sa + k16 * 4096, 128, 256, 0),
+                         umma_desc(sa + kGemmATile + k16 * 32, 16, 1024), idesc, acc);
             }
           }
           umma2_commit_both(empty_bar(s));    // frees the stage in both CTAs once these MMAs have read it
@@ -238,17 +231,8 @@ down_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll 1
       for (int c = 0; c < n_valid; c += 32) {                     // 32 tokens per TMEM load; warp-uniform bound
         uint32_t v[32];
-        if (MODE == 0) {
-          uint32_t u[32];
-          tmem_ld32(taddr + c, v);
-          tmem_ld32(taddr + 128 + c, u);
-          tmem_ld_wait();
-#pragma unroll
-          for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(swiglu_fast(__uint_as_float(v[j]), __uint_as_float(u[j])));
-        } else {
-          tmem_ld32(taddr + c, v);
-          tmem_ld_wait();
-        }
+        tmem_ld32(taddr + c, v);
+        tmem_ld_wait();
 #pragma unroll
         for (int j = 0; j < 32; ++j) s_t[j * 32 + lane] = __float2bfloat16_rn(__uint_as_float(v[j]));
         __syncwarp();

@@ -30,7 +30,7 @@ struct PlanParams {
   size_t S;
   int T;
   int tokens_per_pass;   // tokens one weight pass of the resident streaming kernel serves
-  int zc_single_pass;    // 1: a zero-copy record crosses the link once whatever its token count (bf16 kernel)
+  int zc_tokens_per_pass;   // tokens one link pass of a zero-copy record serves
   // outputs
   PlanHeader *hdr_dev;   // device plan record (header + 8 arrays of E)
   PlanHeader *hdr_host;  // mapped host mirror, or nullptr when the host does not read the plan
@@ -313,8 +313,8 @@ __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, uns
   const int n_fill = unpack(totB, 0), n_zc = unpack(totB, 1), n_hs = unpack(totB, 2), n_gemm = unpack(totB, 3);
   const int n_fs = unpack(totB, 4);
   // weight passes (tokens_per_pass tokens each) of the list entries, in list order
-  const int passes = (res_stream || (is_zc && !p.zc_single_pass)) ? (c + p.tokens_per_pass - 1) / p.tokens_per_pass
-                                                                  : (is_zc ? 1 : 0);
+  const int passes = res_stream ? (c + p.tokens_per_pass - 1) / p.tokens_per_pass
+                                : (is_zc ? (c + p.zc_tokens_per_pass - 1) / p.zc_tokens_per_pass : 0);
   unsigned long long totC, totZ;
   const unsigned long long exC = block_excl_scan64(
       ((unsigned long long)(fs ? passes : 0) << 32) | (unsigned long long)(hs ? passes : 0), sm.w, totC);

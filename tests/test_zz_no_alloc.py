@@ -5,16 +5,18 @@ plug-in in somebody else's process), so they cannot create a handle; ``ft_moe_ff
 the same streaming FFN kernel with its scratch in a fixed array inside the library.  The test drives
 both entry points through the C ABI on the same expert record and inputs, twice in a row because
 the fixed scratch keeps the previous call's contents, and expects the same output within the
-tolerance of the other GPU tests.  Collected last so that a stop at the first failure has already run
+tolerance of the other GPU tests; since both run the same kernel, the output is also compared with
+the plain SwiGLU definition evaluated by the CPU oracle from the same record.  Collected last so that a stop at the first failure has already run
 everything else; it passes both alone in a fresh process and after the other tests.
 """
 import numpy as np
 import pytest
 import torch
 
+from oracle import ftmoe_oracle as O
 from paper_2608_16157_b200 import binding as B
 from paper_2608_16157_b200 import workload as W
-from tests.helpers import MAX_ABS_TOL, REL_L2_TOL
+from tests.helpers import MAX_ABS_TOL, REL_L2_TOL, bits, check_output
 
 pytestmark = pytest.mark.gpu
 
@@ -39,6 +41,8 @@ def test_noalloc_entry_point_matches_forward_twice_in_a_row(d, inter, T):
     W.fill_pool(pool.tensor, shape, 1, seed=21)
     dev = torch.device("cuda:0")
     record_dev = pool.tensor.to(dev)                       # the caller's own copy of the record
+    wg, wu, wd = O.unpack_record(pool.tensor.numpy(), d, inter, "bf16")
+    torch.cuda.set_device(0)
     for call in range(2):
         x = W.noise_x(T, d, 21, call, 0).to(dev)
         y_ref = _reference_through_handle(shape, pool, x, T)
@@ -50,6 +54,9 @@ def test_noalloc_entry_point_matches_forward_twice_in_a_row(d, inter, T):
         assert np.all(np.isfinite(a))
         assert np.linalg.norm(a - b) <= REL_L2_TOL * np.linalg.norm(b)
         assert np.abs(a - b).max() <= MAX_ABS_TOL * np.abs(b).max()
+        check_output(y, O.expert_ffn(O.bf16_to_f64(bits(x)), wg, wu, wd))
+        assert B.ft_moe_ffn_noalloc_status(0) == B.FT_OK
+        assert torch.cuda.current_device() == 0          # the caller's device is left as it was
     pool.free()
 
 
@@ -63,4 +70,8 @@ def test_noalloc_entry_point_rejects_sizes_beyond_its_static_scratch():
     assert B.ft_moe_ffn_noalloc(0, rec, 4096, 128, x, y, 4) == B.FT_ERR_INVALID_ARG
     assert B.ft_moe_ffn_noalloc(0, rec, 768, 128, x, y, 4) == B.FT_ERR_UNSUPPORTED
     assert B.ft_moe_ffn_noalloc(0, None, 256, 128, x, y, 4) == B.FT_ERR_INVALID_ARG
+    # a view that starts at an odd element is not 16-byte aligned: refused on the host, nothing is launched
+    odd = torch.zeros(4 * 256 + 8, dtype=torch.bfloat16, device=dev)[1:1 + 4 * 256].view(4, 256)
+    assert B.ft_moe_ffn_noalloc(0, rec, 256, 128, odd, y, 4) == B.FT_ERR_INVALID_ARG
+    assert B.ft_moe_ffn_noalloc(0, rec, 256, 128, x, odd, 4) == B.FT_ERR_INVALID_ARG
     torch.cuda.synchronize()
