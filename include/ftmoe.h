@@ -29,17 +29,21 @@
  * Expert record layout (pool records and slots are byte-identical, so a fill is one contiguous copy)
  *   record index in the pool: layer * n_experts + expert (the flattened id of paper Sec. 4.2).
  *   FT_W_BF16     : tensor-core tile order.  inter/16 units of 16 neurons, 96*hidden bytes each: a gate part, an
- *                   up part and a down part of 32*hidden bytes, all made of 8 x 8 blocks of bf16 (8 rows of 16
- *                   bytes, 128 contiguous bytes per block).  With n the neuron, i the hidden index, c the output
- *                   column, offsets in 2-byte elements:
- *                     W_gate[i][n] at 48*hidden*(n/16) + 512*(i/32) + 256*((n%16)/8) + 64*((i%32)/8) + 8*(n%8) + i%8
+ *                   up part and a down part of 32*hidden bytes.  Gate/up part: 1 KiB tiles of 16 neurons x 32
+ *                   hidden indices = two groups of 8 neuron rows of 64 bytes; down part: 512-byte tiles of 16 output
+ *                   columns x the unit's 16 neurons = two groups of 8 column rows of 32 bytes.  The 16-byte chunks of
+ *                   a row are stored swizzled (the tensor core's 64-byte / 32-byte swizzle of a K-major operand).
+ *                   With n the neuron, i the hidden index, c the output column, offsets in 2-byte elements,
+ *                   r = n%8 for gate/up and r = c%8 for down:
+ *                     W_gate[i][n] at 48*hidden*(n/16) + 512*(i/32) + 256*((n%16)/8) + 32*r
+ *                                     + 8*(((i%32)/8) ^ (r>>1)) + i%8
  *                     W_up[i][n]   at the same place + 16*hidden
- *                     W_down[n][c] at 48*hidden*(n/16) + 32*hidden + 256*(c/16) + 128*((c%16)/8) + 64*((n%16)/8)
- *                                     + 8*(c%8) + n%8
- *                   (gate/up: 1 KiB tiles of 16 neurons x 32 hidden indices; down: 512-byte tiles of 16 columns x
- *                   the unit's 16 neurons).  A warp's 16- or 8-byte loads of a tile are contiguous and land directly
- *                   in mma.sync fragments; the same blocks are the tensor core's K-major operand layout without
- *                   swizzle, so the prefill GEMMs consume them as they are.  S = 3*inter*hidden*2 bytes.
+ *                     W_down[n][c] at 48*hidden*(n/16) + 32*hidden + 256*(c/16) + 128*((c%16)/8) + 16*r
+ *                                     + 8*(((n%16)/8) ^ (r>>2)) + n%8
+ *                   A warp's 16-byte (gate/up) or 8-byte (down) loads of a tile cover whole 128-byte lines in lane
+ *                   order and land directly in mma.sync fragments; a bulk copy of the same bytes into shared memory
+ *                   is a valid swizzled K-major tcgen05 operand, so the prefill GEMMs consume the tiles as they are.
+ *                   S = 3*inter*hidden*2 bytes.
  *   FT_W_INT4_G128: 4-bit two's-complement codes in [-8,7] for the same three matrices, then bf16 scales;
  *                   weight = scale * code.
  *                     Wg_q, Wu_q : row-major [inter][hidden/2] bytes, two codes per byte along hidden
@@ -213,7 +217,8 @@ ft_status_t ft_moe_layer_host(ft_moe_t *h, int layer, const float *logits_host, 
                               void *y_host, int T, void *stream);
 
 /* ---- introspection (tests, reports); each synchronises the device ---- */
-/* Results of the latest ft_moe_route on this handle, which must have been for `layer`.  HOST arrays:
+/* Results of the latest ft_moe_route of `layer` (every layer keeps its own routing arrays, plan record and work
+ * lists, so route/plan/fill of several layers may be issued before their forward calls).  HOST arrays:
  * ids[T*k], w[T*k], count[E], offset[E+1], perm[T*k], inv[T*k]; any may be NULL. */
 ft_status_t ft_moe_get_routing(ft_moe_t *h, int layer, int32_t *ids, float *w, int32_t *count,
                                int32_t *offset, int32_t *perm, int32_t *inv);
@@ -252,6 +257,14 @@ ft_status_t ft_moe_get_cta_trace(ft_moe_t *h, int64_t *out, int n_ctas);
 /* Changes split_min_pairs of a live handle (see ft_moe_config_t); takes effect at the next ft_moe_forward.
  * Used to time the streaming kernel alone (0) or overlapped with the fills. */
 ft_status_t ft_moe_set_split_min_pairs(ft_moe_t *h, int pairs);
+/* How ft_moe_forward launches the bf16 streaming kernel.  0 (default): a plain launch.  1: a programmatic
+ * dependent launch -- the grid may be scheduled while the preceding kernel of the stream is still running, and
+ * waits for that kernel's completion before it reads anything; results are the same as with 0, only the launch
+ * latency is hidden.  2: as 1, but the grid waits only before its first write to the output accumulator, so its
+ * weight streaming overlaps the tail of the preceding kernel; the caller asserts that x_dev, the slots and the plan
+ * of this layer are not produced by that preceding kernel (e.g. forward calls of several already planned layers
+ * issued back to back).  Takes effect at the next ft_moe_forward. */
+ft_status_t ft_moe_set_launch_overlap(ft_moe_t *h, int mode);
 /* Number of kernels this handle has launched since create. */
 ft_status_t ft_moe_launch_count(ft_moe_t *h, uint64_t *out);
 const char *ft_moe_status_string(ft_status_t s);

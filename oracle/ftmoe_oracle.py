@@ -241,10 +241,12 @@ def unpack_record(rec: np.ndarray, d: int, inter: int, wdtype: str):
     """Record bytes -> (W_gate [d, I], W_up [d, I], W_down [I, d]) in float64.
 
     bf16 record: I/16 units of 16 neurons, 96*d bytes each = gate part, up part, down part
-    (32*d bytes each), built from 8 x 8 blocks of bf16 (8 rows of 16 bytes).  In 2-byte elements:
-      W_gate[i][n] at 48*d*(n//16) + 512*(i//32) + 256*((n%16)//8) + 64*((i%32)//8) + 8*(n%8) + i%8
+    (32*d bytes each).  Rows of 64 bytes (gate/up: a neuron's 32 hidden indices) or 32 bytes (down: a
+    column's 16 neurons) in groups of 8 rows; the 16-byte chunks of a row are stored swizzled.  In
+    2-byte elements, with r = n%8 (gate/up) or c%8 (down):
+      W_gate[i][n] at 48*d*(n//16) + 512*(i//32) + 256*((n%16)//8) + 32*r + 8*(((i%32)//8) ^ (r>>1)) + i%8
       W_up[i][n]   at the same place + 16*d
-      W_down[n][c] at 48*d*(n//16) + 32*d + 256*(c//16) + 128*((c%16)//8) + 64*((n%16)//8) + 8*(c%8) + n%8
+      W_down[n][c] at 48*d*(n//16) + 32*d + 256*(c//16) + 128*((c%16)//8) + 16*r + 8*(((n%16)//8) ^ (r>>2)) + n%8
     int4 record: 4-bit two's-complement codes, then bf16 scales sg[I][d/128], su[I][d/128]
     (groups along the hidden index) and sd[I/128][d] (groups along the neuron index);
     weight = scale * code.  Gate and up codes are row-major [I][d/2] bytes, two per byte along
@@ -260,12 +262,12 @@ def unpack_record(rec: np.ndarray, d: int, inter: int, wdtype: str):
         el = _bf16_bits_to_f64(rec.view(np.uint16))
         i = np.arange(d, dtype=np.int64)[:, None]        # hidden index (gate/up) along axis 0
         nn = np.arange(inter, dtype=np.int64)[None, :]   # neuron along axis 1
-        at_gate = 48 * d * (nn // 16) + 512 * (i // 32) + 256 * ((nn % 16) // 8) + 64 * ((i % 32) // 8) \
-            + 8 * (nn % 8) + i % 8
+        at_gate = 48 * d * (nn // 16) + 512 * (i // 32) + 256 * ((nn % 16) // 8) + 32 * (nn % 8) \
+            + 8 * (((i % 32) // 8) ^ ((nn % 8) >> 1)) + i % 8
         n = np.arange(inter, dtype=np.int64)[:, None]    # neuron along axis 0 (down)
         c = np.arange(d, dtype=np.int64)[None, :]        # output column along axis 1
-        at_down = 48 * d * (n // 16) + 32 * d + 256 * (c // 16) + 128 * ((c % 16) // 8) + 64 * ((n % 16) // 8) \
-            + 8 * (c % 8) + n % 8
+        at_down = 48 * d * (n // 16) + 32 * d + 256 * (c // 16) + 128 * ((c % 16) // 8) + 16 * (c % 8) \
+            + 8 * (((n % 16) // 8) ^ ((c % 8) >> 2)) + n % 8
         return el[at_gate], el[at_gate + 16 * d], el[at_down]
     if wdtype == "int4":
         nb = n // 2

@@ -146,7 +146,7 @@ extern "C" ft_status_t ft_moe_ffn_noalloc(int device, const void *record_dev, in
   mp.y = static_cast<__nv_bfloat16 *>(y_dev);
   mp.done = &ctl->done;
   mp.status = &ctl->status;
-  mp.inter = inter; mp.top_k = 1; mp.T = T; mp.finalize = 1;
+  mp.inter = inter; mp.top_k = 1; mp.T = T; mp.finalize = 1; mp.overlap = 0;
   const size_t smem = ffn_stream_smem_bytes(1, hidden);
   switch (hidden / 256) {
     case 1: ffn_stream_kernel<1><<<grid, kFsThreads, smem, st>>>(mp); break;

@@ -1,24 +1,24 @@
 // Steps 5+6 for bf16 experts at decode-sized token counts: an HBM-streaming SwiGLU FFN whose weight loads go
 // straight from global memory into tensor-core fragments.
 //
-// The record is stored in tile order (include/ftmoe.h): a warp's 16-byte (gate/up) or 8-byte (down) loads of one
-// tile are contiguous 512 / 256 bytes and the loaded registers ARE the A fragments of mma.sync.m16n8k16, so there
-// is no shared-memory staging, no ldmatrix and no producer warp.  One persistent CTA of 16 warps per SM walks a
-// contiguous range of 16-neuron units (96*d bytes each: gate part, up part, down part):
+// The record is stored in tile order (include/ftmoe.h): a warp's 16-byte (gate/up) or 8-byte (down) accesses of one
+// tile cover 512 / 256 contiguous bytes, every quarter warp one whole 128-byte line, and the loaded words ARE the A
+// fragments of mma.sync.m16n8k16, so there is no ldmatrix, no transposition and no producer warp.  One persistent
+// CTA of 16 warps per SM walks a contiguous range of 16-neuron units (96*d bytes each: gate, up, down part):
 //   gate/up : warp w owns the hidden slice [w*d/16, (w+1)*d/16); [16 neurons x 8 tokens] partial sums are reduced
 //             across warps through shared memory, then h = SiLU(g) * u (rounded to bf16).
 //   down    : warp w owns the output columns [w*d/16, (w+1)*d/16); A = the unit's 16 x 16 tiles of W_down^T,
 //             B = h; fp32 accumulators persist across the CTA's units of one (expert, pass).
 // Tokens sit in the N dimension of the MMA (8 per group), so the arithmetic does not grow with the token count.
-// The loads are software-pipelined over two register buffers in the order gate, up, down: while one part is being
-// consumed the next one (of this unit or the next) is in flight, also across the barriers of the reduction.
+// Every part has a buffer of its own that is refilled with the next unit's part as soon as it has been consumed:
+// gate and up parts go straight into registers (two buffers of 16-byte loads), the down part is copied by
+// cp.async into shared memory, each warp its own 16-column tiles.  So ~190 KB per SM are in flight and every load
+// has about one unit's time to arrive, also across the barriers of the reduction.
 // The gate-weighted combine is a red.global.add into the fp32 [T][d] accumulator; the last CTA to finish rounds
 // it once to bf16 and clears it.  Records in the mapped host pool (zero-copy experts) stream through the same
-// loads; since they must cross the host link only once, all token groups of such an expert are served from the
-// registers of one pass (up to kFsMaxGroups groups) and the partial outputs are flushed per unit.
+// loads; since they must cross the host link only once, all token groups of such an expert are served from one
+// pass (up to kFsMaxGroups groups) and the partial outputs are flushed per unit.
 #pragma once
-#include <type_traits>
-
 #include "async.cuh"
 #include "common.cuh"
 
@@ -27,9 +27,9 @@ namespace ftmoe {
 constexpr int kFsThreads = 512;
 constexpr int kFsWarps = 16;
 constexpr int kFsTokens = 8;       // tokens per group = N of the MMA
-constexpr int kFsMaxGroups = 4;    // token groups one pass can serve from the registers
+constexpr int kFsMaxGroups = 2;    // token groups one pass can serve
 constexpr int kFsResTokensPerPass = kFsTokens;                 // HBM-resident records: accumulators stay in registers
-constexpr int kFsZcTokensPerPass = kFsTokens * kFsMaxGroups;   // host-resident records: one link pass for 32 tokens
+constexpr int kFsZcTokensPerPass = kFsTokens * kFsMaxGroups;   // host-resident records: one link pass for 16 tokens
 
 struct FfnStreamParams {
   const WorkItem *items;
@@ -47,15 +47,23 @@ struct FfnStreamParams {
   uint32_t *status;
   int inter, top_k, T, finalize;
   int max_items;            // capacity of items / pref (entries beyond the counts are ignored)
-  long long *trace;         // optional [gridDim.x][4]: start and end of the CTA's streaming (global timer, ns), units
-                            // streamed, 0 (the finalizing CTA stores minus its finish time there); or nullptr
+  int overlap;              // programmatic dependent launch: 0 = plain launch; 1 = the grid may be scheduled while the
+                            // preceding kernel of the stream still runs and waits for it before reading anything;
+                            // 2 = it waits only before its first write to y_acc (inputs must already be final)
+  long long *trace;         // optional [gridDim.x][4]: start and end of the CTA's streaming (global timer, ns), 0, 0
+                            // (the finalizing CTA stores minus its finish time in the last field); or nullptr
 };
 
-// Dynamic shared memory: red [groups][16 warps][2][16 x 8] f32 | h [groups][8][16] bf16 | tok [32] | gw [32] |
-// x [8][d + 32] bf16 | items [max_items] | pref [max_items + 1].
+// Dynamic shared memory: red [groups][16 warps][2][16 x 8] f32 | h [groups][8][16] bf16 | tok, gw [16] |
+// x [8][d + 32] bf16 | down part of the current unit [32 d bytes] | items [max_items] | pref [max_items + 1].
 inline size_t ffn_stream_smem_bytes(int max_items, int d) {
   return (size_t)kFsMaxGroups * kFsWarps * 2 * 128 * 4 + kFsMaxGroups * 128 * 2 + kFsZcTokensPerPass * 8 +
-         (size_t)kFsTokens * (2 * d + 64) + (size_t)max_items * sizeof(WorkItem) + ((size_t)max_items + 1) * 4 + 16;
+         (size_t)kFsTokens * (2 * d + 64) + 32 * (size_t)d + (size_t)max_items * sizeof(WorkItem) +
+         ((size_t)max_items + 1) * 4 + 16;
+}
+
+__device__ __forceinline__ void red_add_f32(float *addr, float v) {
+  asm volatile("red.global.add.f32 [%0], %1;" ::"l"(addr), "f"(v) : "memory");
 }
 
 template <int DB>  // DB = d / 256
@@ -63,7 +71,6 @@ __global__ void __launch_bounds__(kFsThreads, 1) ffn_stream_kernel(FfnStreamPara
   constexpr int KT = (DB >= 2) ? DB / 2 : 1;   // 16 x 32 gate/up tiles per active warp
   constexpr int NWK = (DB * 8) / KT;           // warps that take part in gate/up (all 16 unless d = 256)
   constexpr int CTW = DB;                      // 16-column down tiles per warp
-  constexpr int NB = (2 * KT > CTW) ? 2 * KT : CTW;   // 16-byte registers of one buffer
   constexpr int d = 256 * DB;
   constexpr uint32_t kPart = 32u * d, kUnit = 96u * d;
   constexpr uint32_t kXStride = 2u * d + 64u;   // = 64 mod 128: conflict-free 16-byte fragment loads
@@ -73,7 +80,8 @@ __global__ void __launch_bounds__(kFsThreads, 1) ffn_stream_kernel(FfnStreamPara
   int32_t *s_tok = reinterpret_cast<int32_t *>(s_h + kFsMaxGroups * 128);
   float *s_gw = reinterpret_cast<float *>(s_tok + kFsZcTokensPerPass);
   unsigned char *s_x = reinterpret_cast<unsigned char *>(s_gw + kFsZcTokensPerPass);
-  WorkItem *s_items = reinterpret_cast<WorkItem *>(s_x + kFsTokens * kXStride);
+  unsigned char *s_d = s_x + kFsTokens * kXStride;   // the current unit's down part, byte for byte
+  WorkItem *s_items = reinterpret_cast<WorkItem *>(s_d + kPart);
   int32_t *s_pref = reinterpret_cast<int32_t *>(s_items + p.max_items);
   __shared__ int s_last;
 
@@ -84,9 +92,11 @@ __global__ void __launch_bounds__(kFsThreads, 1) ffn_stream_kernel(FfnStreamPara
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_start));
     p.trace[4 * blockIdx.x] = t_start;
   }
-  int trace_units = 0;
+  if (p.overlap == 1) asm volatile("griddepcontrol.wait;" ::: "memory");
+  bool dep_waited = p.overlap != 2;
   const int n_items = *p.n_items;
   const int n_zc = *p.n_zc;
+  const int n_hit = (p.part == 0) ? 0 : *p.n_hit;
   const bool dense = p.T <= kFsTokens;   // MMA column j is token j: the x rows are staged once per CTA
   // x rows of the MMA columns into shared memory (16 bytes per thread and step); zeros for absent columns
   auto stage_x = [&](auto tok_of_column) {
@@ -98,7 +108,6 @@ __global__ void __launch_bounds__(kFsThreads, 1) ffn_stream_kernel(FfnStreamPara
       *reinterpret_cast<uint4 *>(s_x + j * kXStride + 16 * c8) = v;
     }
   };
-  if (dense) stage_x([&](int j) { return j < p.T ? j : -1; });
   // the work list and the prefix of its weight passes, up to the lists' capacity so that these loads do not wait
   // for the counts
   for (int i = tid; i <= p.max_items; i += kFsThreads) s_pref[i] = p.pref[i];
@@ -109,87 +118,177 @@ __global__ void __launch_bounds__(kFsThreads, 1) ffn_stream_kernel(FfnStreamPara
     for (int i = tid; i < 2 * p.max_items; i += kFsThreads) dst[i] = src[i];
   }
   __syncthreads();
-  const int NBLK = p.inter / 16;
-  // two work ranges, each split evenly over the CTAs: HBM-resident units, then host-resident units (the latter
-  // are bound by the host link, so every CTA takes an equal share of them).  `part` restricts the launch to the
-  // items that do not depend on the fills (plus the zero-copy items) or to the filled items.
-  const int n_hit = (p.part == 0) ? 0 : *p.n_hit;
-  const int a0 = (p.part == 2) ? n_hit : 0, a1 = (p.part == 1) ? n_hit : n_items;
-  long long rb0, rb1;   // first unit of this CTA in the two ranges
-  int rn0, rn1;         // and how many
-  {
-    const long long first_res = (long long)s_pref[a0] * NBLK, total_res = (long long)s_pref[a1] * NBLK;
-    const long long zc_begin = (long long)s_pref[n_items] * NBLK;
-    const long long total_all = (p.part == 2) ? zc_begin : (long long)s_pref[n_items + n_zc] * NBLK;
-    rb0 = first_res + (total_res - first_res) * blockIdx.x / gridDim.x;
-    rn0 = (int)(first_res + (total_res - first_res) * (blockIdx.x + 1) / gridDim.x - rb0);
-    rb1 = zc_begin + (total_all - zc_begin) * blockIdx.x / gridDim.x;
-    rn1 = (int)(zc_begin + (total_all - zc_begin) * (blockIdx.x + 1) / gridDim.x - rb1);
-  }
-  // A cursor over this CTA's units: (range, flattened pass index, unit inside the pass, item).
-  struct Cur { int range, b, item, pu, left; };
-  auto cur_enter = [&](Cur &c) {   // positions at the start of range c.range, skipping empty ranges
-    while (c.range < 2) {
-      const long long u = c.range ? rb1 : rb0;
-      c.left = c.range ? rn1 : rn0;
-      if (c.left > 0) {
-        c.pu = (int)(u / NBLK);
-        c.b = (int)(u - (long long)c.pu * NBLK);
-        while (s_pref[c.item + 1] <= c.pu) ++c.item;
-        return;
-      }
-      ++c.range;
-    }
-  };
-  auto cur_next = [&](Cur &c) {
-    if (--c.left > 0) {
-      if (++c.b == NBLK) {
-        c.b = 0;
-        ++c.pu;
-        while (s_pref[c.item + 1] <= c.pu) ++c.item;
-      }
-    } else {
-      ++c.range;
-      cur_enter(c);
-    }
-  };
-  auto unit_ptr = [&](const Cur &c) { return s_items[c.item].w + (size_t)c.b * kUnit; };
+  const uint32_t NBLK = (uint32_t)p.inter / 16u;
 
-  // ---- loads: one part of a unit into one register buffer ----
-  auto load_gu = [&](uint4 (&buf)[NB], const uint8_t *part) {
-    if (NWK == kFsWarps || warp < NWK) {
-      const uint8_t *a = part + (size_t)(warp * KT) * 1024 + q * 128 + g * 16;
+  // ---- per-lane constants of the loads ----
+  // gate/up: tile kb = warp*KT + t; row g, chunk q of the 64-byte row (stored at position q ^ (g >> 1))
+  const uint32_t gu_off = (uint32_t)(warp * KT) * 1024u + g * 64u + ((q ^ (g >> 1)) * 16u);
+  // down: this warp's CTW tiles of 512 bytes are copied as they are into the same place of s_d ...
+  const uint32_t d_off = (uint32_t)(warp * CTW) * 512u + lane * 16u;
+  const uint32_t my_d = smem_u32(s_d) + d_off;
+  // ... and read back as A fragments: column row g (and g + 8), neurons 4q..4q+3 = half (q & 1) of chunk (q >> 1)
+  const uint32_t my_dfrag =
+      smem_u32(s_d) + (uint32_t)(warp * CTW) * 512u + g * 32u + (((q >> 1) ^ (g >> 2)) * 16u) + (q & 1) * 8u;
+  const uint32_t my_x = smem_u32(s_x) + g * kXStride + (uint32_t)(warp * KT) * 64u + 16u * q;
+  const bool gu_warp = (NWK == kFsWarps) || warp < NWK;
+
+  uint4 bufg[2 * KT], bufu[2 * KT];
+  auto load_gu = [&](uint4 (&buf)[2 * KT], const uint8_t *part) {
+    if (gu_warp) {
 #pragma unroll
       for (int t = 0; t < KT; ++t) {
-        buf[2 * t] = ld_stream_16(a + t * 1024);
-        buf[2 * t + 1] = ld_stream_16(a + t * 1024 + 512);
+        buf[2 * t] = ld_stream_16(part + gu_off + t * 1024);
+        buf[2 * t + 1] = ld_stream_16(part + gu_off + t * 1024 + 512);
       }
     }
   };
-  auto load_d = [&](uint4 (&buf)[NB], const uint8_t *part) {
-    const uint8_t *a = part + (size_t)(warp * CTW) * 512 + (q >> 1) * 128 + g * 16 + (q & 1) * 8;
+  auto load_d = [&](const uint8_t *part) {   // only this warp reads the region: warp-level synchronisation suffices
 #pragma unroll
-    for (int c = 0; c < CTW; ++c) {
-      const uint2 lo = ld_stream_8(a + c * 512), hi = ld_stream_8(a + c * 512 + 256);
-      buf[c] = make_uint4(lo.x, lo.y, hi.x, hi.y);
-    }
+    for (int c = 0; c < CTW; ++c)
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(my_d + c * 512), "l"(part + d_off + c * 512) : "memory");
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  auto load_unit = [&](const uint8_t *unit) {
+    load_gu(bufg, unit);
+    load_gu(bufu, unit + kPart);
+    load_d(unit + 2 * kPart);
   };
 
-  // ---- per-segment state (a segment = this CTA's units of one (item, pass)) ----
+  // partial [16 neurons x 8 tokens] sums of one part over this warp's hidden slice -> shared memory
+  // (x fragments of MMA column g: from the staged rows, or -- tok != -2 -- straight from global memory, zeros if tok < 0)
+  auto gu_part = [&](const uint4 (&buf)[2 * KT], float *r, int tok) {
+    if (gu_warp) {
+      float c1[4] = {0.f, 0.f, 0.f, 0.f}, c2[4] = {0.f, 0.f, 0.f, 0.f};   // two chains: consecutive MMAs do not wait
+#pragma unroll
+      for (int t = 0; t < KT; ++t) {
+        uint4 xv = make_uint4(0u, 0u, 0u, 0u);
+        if (tok == -2) xv = lds_v4(my_x + 64u * t);
+        else if (tok >= 0) xv = *reinterpret_cast<const uint4 *>(p.x + (size_t)tok * d + 32 * (warp * KT + t) + 8 * q);
+        mma_bf16(c1, buf[2 * t].x, buf[2 * t + 1].x, buf[2 * t].y, buf[2 * t + 1].y, xv.x, xv.y);
+        mma_bf16(c2, buf[2 * t].z, buf[2 * t + 1].z, buf[2 * t].w, buf[2 * t + 1].w, xv.z, xv.w);
+      }
+      *reinterpret_cast<float2 *>(r + g * 8 + 2 * q) = make_float2(c1[0] + c2[0], c1[1] + c2[1]);
+      *reinterpret_cast<float2 *>(r + (g + 8) * 8 + 2 * q) = make_float2(c1[2] + c2[2], c1[3] + c2[3]);
+    }
+  };
+  // h = SiLU(sum gate) * (sum up), bf16, [group][token][neuron]: four threads per value, each sums a quarter of the
+  // warps' partial sums
+  auto reduce_h = [&](int ngroups) {
+    const int r = tid >> 2, qu = tid & 3;   // r = neuron * 8 + token
+    for (int grp = 0; grp < ngroups; ++grp) {
+      const float *base = s_red + (size_t)grp * kFsWarps * 2 * 128 + r;
+      float a = 0.f, c = 0.f;
+#pragma unroll
+      for (int w = 0; w < NWK / 4; ++w) {
+        a += base[((qu * (NWK / 4) + w) * 2 + 0) * 128];
+        c += base[((qu * (NWK / 4) + w) * 2 + 1) * 128];
+      }
+      a += __shfl_xor_sync(0xffffffffu, a, 1);
+      c += __shfl_xor_sync(0xffffffffu, c, 1);
+      a += __shfl_xor_sync(0xffffffffu, a, 2);
+      c += __shfl_xor_sync(0xffffffffu, c, 2);
+      if (qu == 0) s_h[grp * 128 + (r & 7) * 16 + (r >> 3)] = __float2bfloat16_rn(__fdividef(a, 1.f + __expf(-a)) * c);
+    }
+  };
   float dacc[CTW][4];
-  int my_tok = -1;      // lane i < ntok: token and gate weight of the pass's i-th pair
-  float my_w = 0.f;
-  int ntok = 0, ngroups = 1;
+  auto down_part = [&](int grp) {
+    const uint2 hb = *reinterpret_cast<const uint2 *>(s_h + grp * 128 + g * 16 + 4 * q);
+#pragma unroll
+    for (int cc = 0; cc < CTW; ++cc) {
+      uint2 lo, hi;
+      asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(lo.x), "=r"(lo.y) : "r"(my_dfrag + cc * 512));
+      asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(hi.x), "=r"(hi.y) : "r"(my_dfrag + cc * 512 + 256));
+      mma_bf16(dacc[cc], lo.x, hi.x, lo.y, hi.y, hb.x, hb.y);
+    }
+  };
+  // gate-weighted combine of the accumulators: D fragment = [column g / g+8 of the tile][MMA columns 2q, 2q+1]
+  auto flush = [&](int tok_a, float gw_a, int tok_b, float gw_b) {
+    if (!dep_waited) {   // the preceding kernel's last writes to y_acc (its finalize) are ordered before ours
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      dep_waited = true;
+    }
+    float *ya = p.y_acc + (size_t)(tok_a < 0 ? 0 : tok_a) * d + 16 * (warp * CTW) + g;
+    float *yb = p.y_acc + (size_t)(tok_b < 0 ? 0 : tok_b) * d + 16 * (warp * CTW) + g;
+#pragma unroll
+    for (int cc = 0; cc < CTW; ++cc) {
+      if (tok_a >= 0) {
+        red_add_f32(ya + 16 * cc, gw_a * dacc[cc][0]);
+        red_add_f32(ya + 16 * cc + 8, gw_a * dacc[cc][2]);
+      }
+      if (tok_b >= 0) {
+        red_add_f32(yb + 16 * cc, gw_b * dacc[cc][1]);
+        red_add_f32(yb + 16 * cc + 8, gw_b * dacc[cc][3]);
+      }
+    }
+  };
+  auto zero_dacc = [&]() {
+#pragma unroll
+    for (int cc = 0; cc < CTW; ++cc) { dacc[cc][0] = dacc[cc][1] = dacc[cc][2] = dacc[cc][3] = 0.f; }
+  };
 
-  auto begin_segment = [&](const Cur &c) {
-    const WorkItem &it = s_items[c.item];
-    const int tpp = c.range ? kFsZcTokensPerPass : kFsResTokensPerPass;
-    const int tok0 = (int)(c.pu - s_pref[c.item]) * tpp;
-    ntok = min(tpp, it.n_tok - tok0);
-    ngroups = (ntok + kFsTokens - 1) / kFsTokens;
-    if (ngroups == 1) {
-      my_tok = -1;
-      my_w = 0.f;
+  // ---- this CTA's share of the two work ranges ----
+  // HBM-resident units, then host-resident units (bound by the host link, so every CTA takes an equal share of
+  // them), each split evenly over the CTAs.  `part` restricts the launch to the items that do not depend on the
+  // fills (plus the zero-copy items) or to the filled items.
+  auto share = [&](uint32_t total, uint32_t &first, uint32_t &count) {   // CTA i: total/grid units, the first total%grid CTAs one more
+    const uint32_t per = total / gridDim.x, rem = total - per * gridDim.x;
+    first = blockIdx.x * per + min((uint32_t)blockIdx.x, rem);
+    count = per + (blockIdx.x < rem ? 1u : 0u);
+  };
+  const int a0 = (p.part == 2) ? n_hit : 0, a1 = (p.part == 1) ? n_hit : n_items;
+  uint32_t rfirst0, rcount0, rfirst1, rcount1;
+  share((uint32_t)(s_pref[a1] - s_pref[a0]) * NBLK, rfirst0, rcount0);
+  rfirst0 += (uint32_t)s_pref[a0] * NBLK;
+  share((p.part == 2) ? 0u : (uint32_t)(s_pref[n_items + n_zc] - s_pref[n_items]) * NBLK, rfirst1, rcount1);
+  rfirst1 += (uint32_t)s_pref[n_items] * NBLK;
+
+  // Segments (this CTA's units of one (item, pass)) in order; the loads of a segment's first unit are issued by
+  // the previous segment's last step (or right here for the very first one).
+  struct Seg { const uint8_t *unit0; int item, pass, n_units, zc; };
+  int range = 0, item = 0;
+  uint32_t pu = 0, b = 0, left = 0;
+  auto next_segment = [&](Seg &s) -> bool {   // false when the CTA's work is exhausted
+    while (left == 0) {
+      if (range == 2) return false;
+      left = range ? rcount1 : rcount0;
+      if (left > 0) {
+        const uint32_t first = range ? rfirst1 : rfirst0;
+        pu = first / NBLK;
+        b = first - pu * NBLK;
+      }
+      ++range;
+    }
+    while ((uint32_t)s_pref[item + 1] <= pu) ++item;
+    s.item = item;
+    s.pass = (int)(pu - (uint32_t)s_pref[item]);
+    s.n_units = (int)min(left, NBLK - b);
+    s.unit0 = s_items[item].w + (size_t)b * kUnit;
+    s.zc = range - 1;
+    left -= s.n_units;
+    ++pu;
+    b = 0;
+    return true;
+  };
+
+  Seg sg, nsg;
+  bool more = next_segment(sg);
+  if (more) load_unit(sg.unit0);
+  if (dense) {   // staged while the first unit's loads are in flight
+    stage_x([&](int j) { return j < p.T ? j : -1; });
+    __syncthreads();
+  }
+
+  while (more) {
+    more = next_segment(nsg);
+    const uint8_t *after = more ? nsg.unit0 : nullptr;   // the unit that follows this segment's last one
+    const WorkItem &it = s_items[sg.item];
+    const int tpp = sg.zc ? kFsZcTokensPerPass : kFsResTokensPerPass;
+    const int tok0 = sg.pass * tpp;
+    const int ntok = min(tpp, it.n_tok - tok0);
+    if (ntok <= kFsTokens) {
+      // ---------------- one token group: accumulators persist over the segment ----------------
+      int my_tok = -1;      // lane i < ntok: token and gate weight of the pass's i-th pair
+      float my_w = 0.f;
       if (lane < ntok) {
         if (it.expert >= 0) {
           const int pr = p.perm[it.off + tok0 + lane];
@@ -200,18 +299,53 @@ __global__ void __launch_bounds__(kFsThreads, 1) ffn_stream_kernel(FfnStreamPara
           my_w = 1.f;
         }
       }
-      if (!dense) {
+      if (!dense) {   // MMA column j is the pass's j-th pair: stage those tokens' rows
         // (the previous segment's readers of s_x are past the barriers of their last unit)
-        const int tok0_ = tok0, off_ = it.off, expert_ = it.expert, ntok_ = ntok;
+        const int off_ = it.off + tok0, expert_ = it.expert;
         stage_x([&](int j) {
-          if (j >= ntok_) return -1;
-          return expert_ >= 0 ? p.perm[off_ + tok0_ + j] / p.top_k : tok0_ + j;
+          if (j >= ntok) return -1;
+          return expert_ >= 0 ? p.perm[off_ + j] / p.top_k : tok0 + j;
         });
         __syncthreads();
       }
-#pragma unroll
-      for (int cc = 0; cc < CTW; ++cc) { dacc[cc][0] = dacc[cc][1] = dacc[cc][2] = dacc[cc][3] = 0.f; }
+      zero_dacc();
+      const uint8_t *unit = sg.unit0;
+      for (int k = 0; k < sg.n_units; ++k, unit += kUnit) {
+        const uint8_t *nunit = (k + 1 < sg.n_units) ? unit + kUnit : after;
+        gu_part(bufg, s_red + (warp * 2 + 0) * 128, -2);
+        if (nunit) load_gu(bufg, nunit);
+        gu_part(bufu, s_red + (warp * 2 + 1) * 128, -2);
+        if (nunit) load_gu(bufu, nunit + kPart);
+        __syncthreads();
+        reduce_h(1);
+        asm volatile("cp.async.wait_group 0;" ::: "memory");   // this lane's copies of the down part have landed
+        __syncthreads();                                        // h is complete (and so are the other lanes' copies)
+        down_part(0);
+        __syncwarp();   // every lane has read its fragments: the region may be overwritten
+        if (nunit) load_d(nunit + 2 * kPart);
+      }
+      // combine
+      int tok_a, tok_b;
+      float gw_a, gw_b;
+      if (dense) {   // MMA column j is token j: find the pairs (if any) of tokens 2q and 2q+1
+        tok_a = tok_b = -1;
+        gw_a = gw_b = 0.f;
+        for (int i = 0; i < ntok; ++i) {
+          const int ti = __shfl_sync(0xffffffffu, my_tok, i);
+          const float wi = __shfl_sync(0xffffffffu, my_w, i);
+          if (ti == 2 * q) { tok_a = ti; gw_a = wi; }
+          if (ti == 2 * q + 1) { tok_b = ti; gw_b = wi; }
+        }
+      } else {
+        tok_a = __shfl_sync(0xffffffffu, my_tok, 2 * q);
+        tok_b = __shfl_sync(0xffffffffu, my_tok, 2 * q + 1);
+        gw_a = __shfl_sync(0xffffffffu, my_w, 2 * q);
+        gw_b = __shfl_sync(0xffffffffu, my_w, 2 * q + 1);
+      }
+      flush(tok_a, gw_a, tok_b, gw_b);
     } else {
+      // ---------------- several token groups from one pass over the record: flush per unit ----------------
+      const int ngroups = (ntok + kFsTokens - 1) / kFsTokens;
       __syncthreads();   // the previous segment's readers of s_tok / s_gw are done
       if (tid < kFsZcTokensPerPass) {
         int tk = -1;
@@ -230,148 +364,42 @@ __global__ void __launch_bounds__(kFsThreads, 1) ffn_stream_kernel(FfnStreamPara
         s_gw[tid] = w;
       }
       __syncthreads();
-    }
-  };
-  // gate-weighted combine of the accumulators: D fragment = [column g / g+8 of the tile][MMA columns 2q, 2q+1]
-  auto flush = [&](int tok_a, float gw_a, int tok_b, float gw_b) {
-#pragma unroll
-    for (int cc = 0; cc < CTW; ++cc) {
-      const int col = 16 * (warp * CTW + cc) + g;
-      if (tok_a >= 0) {
-        atomicAdd(p.y_acc + (size_t)tok_a * d + col, gw_a * dacc[cc][0]);
-        atomicAdd(p.y_acc + (size_t)tok_a * d + col + 8, gw_a * dacc[cc][2]);
-      }
-      if (tok_b >= 0) {
-        atomicAdd(p.y_acc + (size_t)tok_b * d + col, gw_b * dacc[cc][1]);
-        atomicAdd(p.y_acc + (size_t)tok_b * d + col + 8, gw_b * dacc[cc][3]);
-      }
-    }
-  };
-  auto end_segment = [&]() {   // single-group segments only: the other kind flushes per unit
-    int tok_a = -1, tok_b = -1;
-    float gw_a = 0.f, gw_b = 0.f;
-    if (dense) {   // MMA column j is token j: find the pairs (if any) of tokens 2q and 2q+1
-      for (int i = 0; i < ntok; ++i) {
-        const int ti = __shfl_sync(0xffffffffu, my_tok, i);
-        const float wi = __shfl_sync(0xffffffffu, my_w, i);
-        if (ti == 2 * q) { tok_a = ti; gw_a = wi; }
-        if (ti == 2 * q + 1) { tok_b = ti; gw_b = wi; }
-      }
-    } else {       // MMA column j is the pass's j-th pair
-      tok_a = __shfl_sync(0xffffffffu, my_tok, 2 * q);
-      tok_b = __shfl_sync(0xffffffffu, my_tok, 2 * q + 1);
-      gw_a = __shfl_sync(0xffffffffu, my_w, 2 * q);
-      gw_b = __shfl_sync(0xffffffffu, my_w, 2 * q + 1);
-    }
-    flush(tok_a, gw_a, tok_b, gw_b);
-  };
-  // partial [16 neurons x 8 tokens] sums of one part over this warp's hidden slice -> shared memory
-  // (x fragments: from the staged rows, or for multi-group passes straight from global memory, tok = the token of
-  // MMA column g)
-  auto gu_part = [&](const uint4 (&buf)[NB], int grp, int which, bool staged, int tok) {
-    if (NWK == kFsWarps || warp < NWK) {
-      float c1[4] = {0.f, 0.f, 0.f, 0.f}, c2[4] = {0.f, 0.f, 0.f, 0.f};   // two chains: consecutive MMAs do not wait
-      const uint32_t xs = smem_u32(s_x) + g * kXStride + (uint32_t)(warp * KT) * 64u + 16u * q;
-#pragma unroll
-      for (int t = 0; t < KT; ++t) {
-        uint4 xv = make_uint4(0u, 0u, 0u, 0u);
-        if (staged) xv = lds_v4(xs + 64u * t);
-        else if (tok >= 0) xv = *reinterpret_cast<const uint4 *>(p.x + (size_t)tok * d + 32 * (warp * KT + t) + 8 * q);
-        mma_bf16(c1, buf[2 * t].x, buf[2 * t + 1].x, buf[2 * t].y, buf[2 * t + 1].y, xv.x, xv.y);
-        mma_bf16(c2, buf[2 * t].z, buf[2 * t + 1].z, buf[2 * t].w, buf[2 * t + 1].w, xv.z, xv.w);
-      }
-      float *r = s_red + (((size_t)grp * kFsWarps + warp) * 2 + which) * 128;
-      *reinterpret_cast<float2 *>(r + g * 8 + 2 * q) = make_float2(c1[0] + c2[0], c1[1] + c2[1]);
-      *reinterpret_cast<float2 *>(r + (g + 8) * 8 + 2 * q) = make_float2(c1[2] + c2[2], c1[3] + c2[3]);
-    }
-  };
-  auto consume_gu = [&](const uint4 (&buf)[NB], int which) {
-    if (ngroups == 1) {
-      gu_part(buf, 0, which, true, 0);
-    } else {
-      for (int grp = 0; grp < ngroups; ++grp) gu_part(buf, grp, which, false, s_tok[grp * kFsTokens + g]);
-    }
-  };
-  auto reduce_h = [&]() {   // h = SiLU(sum gate) * (sum up), bf16, [group][token][neuron]
-    for (int idx = tid; idx < 128 * ngroups; idx += kFsThreads) {
-      const int grp = idx >> 7, r = idx & 127, n = r >> 3, t = r & 7;
-      const float *base = s_red + (size_t)grp * kFsWarps * 2 * 128 + r;
-      float a = 0.f, c = 0.f;
-#pragma unroll
-      for (int w = 0; w < NWK; ++w) {
-        a += base[(w * 2 + 0) * 128];
-        c += base[(w * 2 + 1) * 128];
-      }
-      s_h[grp * 128 + t * 16 + n] = __float2bfloat16_rn(a / (1.f + __expf(-a)) * c);
-    }
-  };
-  auto down_part = [&](const uint4 (&buf)[NB], int grp) {
-    const uint2 hb = *reinterpret_cast<const uint2 *>(s_h + grp * 128 + g * 16 + 4 * q);
-#pragma unroll
-    for (int cc = 0; cc < CTW; ++cc) mma_bf16(dacc[cc], buf[cc].x, buf[cc].z, buf[cc].y, buf[cc].w, hb.x, hb.y);
-  };
-  auto consume_d = [&](const uint4 (&buf)[NB]) {
-    if (ngroups == 1) {
-      down_part(buf, 0);
-    } else {
-      for (int grp = 0; grp < ngroups; ++grp) {
-#pragma unroll
-        for (int cc = 0; cc < CTW; ++cc) { dacc[cc][0] = dacc[cc][1] = dacc[cc][2] = dacc[cc][3] = 0.f; }
-        down_part(buf, grp);
-        const int ia = grp * kFsTokens + 2 * q;
-        flush(s_tok[ia], s_gw[ia], s_tok[ia + 1], s_gw[ia + 1]);
+      const uint8_t *unit = sg.unit0;
+      for (int k = 0; k < sg.n_units; ++k, unit += kUnit) {
+        const uint8_t *nunit = (k + 1 < sg.n_units) ? unit + kUnit : after;
+        for (int which = 0; which < 2; ++which) {
+          for (int grp = 0; grp < ngroups; ++grp) {
+            const int tok = s_tok[grp * kFsTokens + g];   // x fragments straight from global memory
+            float *r = s_red + (((size_t)grp * kFsWarps + warp) * 2 + which) * 128;
+            if (which == 0) gu_part(bufg, r, tok); else gu_part(bufu, r, tok);
+          }
+          if (nunit) { if (which == 0) load_gu(bufg, nunit); else load_gu(bufu, nunit + kPart); }
+        }
+        __syncthreads();
+        reduce_h(ngroups);
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncthreads();
+        for (int grp = 0; grp < ngroups; ++grp) {
+          zero_dacc();
+          down_part(grp);
+          const int ia = grp * kFsTokens + 2 * q;
+          flush(s_tok[ia], s_gw[ia], s_tok[ia + 1], s_gw[ia + 1]);
+        }
+        __syncwarp();
+        if (nunit) load_d(nunit + 2 * kPart);
       }
     }
-  };
-
-  // ---- the stream: gate -> buffer par, up -> buffer par^1, down -> buffer par; the next unit swaps the roles ----
-  uint4 buf[2][NB];
-  Cur cu;
-  cu.range = 0; cu.item = 0; cu.b = 0; cu.pu = 0; cu.left = 0;
-  cur_enter(cu);
-  if (cu.range < 2) {
-    Cur nx = cu;
-    {
-      const uint8_t *u0 = unit_ptr(cu);
-      load_gu(buf[0], u0);
-      load_gu(buf[1], u0 + kPart);
-    }
-    cur_next(nx);
-    bool seg_first = true;
-    auto step = [&](auto parc) -> bool {
-      constexpr int par = decltype(parc)::value;
-      if (seg_first) begin_segment(cu);
-      const uint8_t *unit = unit_ptr(cu);
-      const bool has_next = nx.range < 2;
-      const uint8_t *nunit = has_next ? unit_ptr(nx) : unit;
-      ++trace_units;
-      consume_gu(buf[par], 0);
-      load_d(buf[par], unit + 2 * kPart);
-      consume_gu(buf[par ^ 1], 1);
-      if (has_next) load_gu(buf[par ^ 1], nunit);
-      __syncthreads();
-      reduce_h();
-      __syncthreads();
-      consume_d(buf[par]);
-      if (has_next) load_gu(buf[par], nunit + kPart);
-      const bool seg_last = !(has_next && nx.pu == cu.pu && nx.range == cu.range);
-      if (seg_last && ngroups == 1) end_segment();
-      seg_first = seg_last;
-      cu = nx;
-      if (has_next) cur_next(nx);
-      return has_next;
-    };
-    while (true) {
-      if (!step(std::integral_constant<int, 0>{})) break;
-      if (!step(std::integral_constant<int, 1>{})) break;
-    }
+    sg = nsg;
   }
 
+  // the next kernel of the stream, if it was launched as a programmatic dependent, may be scheduled from here on
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (!dep_waited) asm volatile("griddepcontrol.wait;" ::: "memory");   // (a CTA without work still orders its exit)
   if (p.trace != nullptr && tid == 0) {
     long long *tr = p.trace + 4 * blockIdx.x;
     long long t_end;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_end));
-    tr[1] = t_end; tr[2] = trace_units; tr[3] = 0;
+    tr[1] = t_end; tr[2] = 0; tr[3] = 0;
   }
   // ---- the last CTA to finish rounds the accumulator to bf16 and clears it ----
   if (!p.finalize) return;
@@ -384,23 +412,23 @@ __global__ void __launch_bounds__(kFsThreads, 1) ffn_stream_kernel(FfnStreamPara
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  const long long n4 = (long long)p.T * d / 4;
+  const int n4 = p.T * (d / 4);
   // several independent L2 loads in flight per thread: the round trips overlap instead of adding up
-  for (long long i0 = tid; i0 < n4; i0 += 8LL * kFsThreads) {
+  for (int i0 = tid; i0 < n4; i0 += 8 * kFsThreads) {
     float4 v[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      const long long i = i0 + (long long)j * kFsThreads;
+      const int i = i0 + j * kFsThreads;
       v[j] = (i < n4) ? __ldcg(reinterpret_cast<const float4 *>(p.y_acc) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      const long long i = i0 + (long long)j * kFsThreads;
+      const int i = i0 + j * kFsThreads;
       if (i < n4) {
-        __nv_bfloat162 a = __floats2bfloat162_rn(v[j].x, v[j].y), b = __floats2bfloat162_rn(v[j].z, v[j].w);
+        __nv_bfloat162 a = __floats2bfloat162_rn(v[j].x, v[j].y), b2 = __floats2bfloat162_rn(v[j].z, v[j].w);
         uint2 o;
         o.x = *reinterpret_cast<uint32_t *>(&a);
-        o.y = *reinterpret_cast<uint32_t *>(&b);
+        o.y = *reinterpret_cast<uint32_t *>(&b2);
         reinterpret_cast<uint2 *>(p.y)[i] = o;
         reinterpret_cast<float4 *>(p.y_acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
       }

@@ -32,6 +32,18 @@ struct LayerState {
   unsigned long long *stats = nullptr;
   int phase = PH_IDLE;
   int T = 0;
+  uint32_t seq = 0;            // plans launched for this layer (stale-record check of the host mirror)
+};
+
+// Per-layer scratch: the routing arrays, the plan record and the work lists of the layer's latest step.  Every
+// layer has its own set, so route/plan/fill of several layers may be issued before their forward calls.
+struct Scratch {
+  int32_t *ids, *count, *offset, *perm, *inv;
+  float *topk_w;
+  PlanHeader *plan_dev, *plan_host, *plan_host_devptr;
+  WorkItem *items_res, *items_zc, *items_gemm;
+  int32_t *res_pref, *gemm_pref;
+  uint8_t *is_gemm;
 };
 
 }  // namespace
@@ -49,7 +61,8 @@ struct ft_moe {
   uint8_t *stats_mem = nullptr;     // per-layer step counters and statistics (survive a resize)
   int table_slots = 0;              // slots per table: slots_per_layer, or n_layers*slots_per_layer when shared
   std::vector<LayerState> layers;
-  // per-handle scratch (layers are stream-ordered, so one set serves all)
+  // scratch: one set per layer (see Scratch), allocated as [L] x stride arrays
+  size_t pair_stride = 0, plan_stride = 0;   // bytes per layer of the pair arrays / the plan record
   int32_t *ids = nullptr, *count = nullptr, *offset = nullptr, *perm = nullptr, *inv = nullptr;
   float *topk_w = nullptr;
   float *y_acc = nullptr;
@@ -72,7 +85,8 @@ struct ft_moe {
   uint32_t *done_dev = nullptr;          // CTA completion counter of the streaming MMA kernel
   long long *trace_dev = nullptr;        // per-CTA clocks of the latest streaming-kernel launch
   uint2 *q4_hbuf = nullptr;              // int4 path: h of every (pass, 16-neuron block) in fragment order
-  uint32_t seq_host = 0;                // plans launched
+  int last_fill_layer = -1;
+  int overlap = 0;                      // launch mode of the streaming kernel (see FfnStreamParams::overlap)
   float *stage_logits = nullptr;
   __nv_bfloat16 *stage_x = nullptr, *stage_y = nullptr;
   // streams / events
@@ -81,7 +95,6 @@ struct ft_moe {
   cudaEvent_t ev_fill_t0 = nullptr, ev_fill_t1 = nullptr;
   uint64_t last_fill_bytes = 0;
   bool fill_timed = false;
-  int last_routed_layer = -1;
   uint64_t launches = 0;
   // optional per-kernel timing (CUDA events on the launching stream)
   bool timing = false;
@@ -105,6 +118,28 @@ cudaError_t g_last_cuda_error = cudaSuccess;   // the CUDA error behind the late
       return FT_ERR_CUDA;                                                                 \
     }                                                                                     \
   } while (0)
+
+Scratch scratch_of(const ft_moe *h, int layer) {
+  const size_t E = h->cfg.n_experts, l = (size_t)layer;
+  auto at = [&](auto *base, size_t bytes_per_layer) {
+    using T = decltype(base);
+    return base ? reinterpret_cast<T>(reinterpret_cast<uint8_t *>(base) + l * bytes_per_layer) : base;
+  };
+  Scratch s;
+  s.ids = at(h->ids, h->pair_stride); s.perm = at(h->perm, h->pair_stride); s.inv = at(h->inv, h->pair_stride);
+  s.topk_w = at(h->topk_w, h->pair_stride);
+  s.count = at(h->count, E * 4); s.offset = at(h->offset, (E + 1) * 4);
+  s.plan_dev = at(h->plan_dev, h->plan_stride);
+  s.plan_host = at(h->plan_host, h->plan_stride);
+  s.plan_host_devptr = at(h->plan_host_devptr, h->plan_stride);
+  s.items_res = at(h->items_res, (2 * E + 1) * sizeof(WorkItem));
+  s.items_zc = at(h->items_zc, E * sizeof(WorkItem));
+  s.items_gemm = at(h->items_gemm, E * sizeof(WorkItem));
+  s.res_pref = at(h->res_pref, (2 * E + 2) * 4);
+  s.gemm_pref = at(h->gemm_pref, (E + 1) * 4);
+  s.is_gemm = at(h->is_gemm, E);
+  return s;
+}
 
 size_t expert_bytes_of(const ft_moe_config_t *c) {
   if (!c || c->hidden <= 0 || c->inter <= 0) return 0;
@@ -483,32 +518,34 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
   }
   rc = alloc_cache(h);
   if (rc != FT_OK) return fail(rc);
-  FT_TRY(cudaMalloc(&h->ids, P * 4 + 16));
-  FT_TRY(cudaMalloc(&h->topk_w, P * 4 + 16));
-  FT_TRY(cudaMalloc(&h->count, E * 4));
-  FT_TRY(cudaMalloc(&h->offset, (E + 1) * 4));
-  FT_TRY(cudaMalloc(&h->perm, P * 4 + 16));
-  FT_TRY(cudaMalloc(&h->inv, P * 4 + 16));
+  h->pair_stride = (P * 4 + 16 + 15) & ~(size_t)15;
+  FT_TRY(cudaMalloc(&h->ids, L * h->pair_stride));
+  FT_TRY(cudaMalloc(&h->topk_w, L * h->pair_stride));
+  FT_TRY(cudaMalloc(&h->count, L * E * 4));
+  FT_TRY(cudaMalloc(&h->offset, L * (E + 1) * 4));
+  FT_TRY(cudaMalloc(&h->perm, L * h->pair_stride));
+  FT_TRY(cudaMalloc(&h->inv, L * h->pair_stride));
   FT_TRY(cudaMalloc(&h->y_acc, (size_t)c.max_tokens * c.hidden * 4));
   FT_TRY(cudaMemset(h->y_acc, 0, (size_t)c.max_tokens * c.hidden * 4));
   h->plan_bytes = sizeof(PlanHeader) + 8 * E * 4;
-  FT_TRY(cudaMalloc(&h->plan_dev, h->plan_bytes));
-  FT_TRY(cudaMemset(h->plan_dev, 0, h->plan_bytes));
-  FT_TRY(cudaHostAlloc(&h->plan_host, h->plan_bytes, cudaHostAllocMapped));
-  memset(h->plan_host, 0, h->plan_bytes);
+  h->plan_stride = (h->plan_bytes + 63) & ~(size_t)63;
+  FT_TRY(cudaMalloc(&h->plan_dev, L * h->plan_stride));
+  FT_TRY(cudaMemset(h->plan_dev, 0, L * h->plan_stride));
+  FT_TRY(cudaHostAlloc(&h->plan_host, L * h->plan_stride, cudaHostAllocMapped));
+  memset(h->plan_host, 0, L * h->plan_stride);
   FT_TRY(cudaHostGetDevicePointer(reinterpret_cast<void **>(&h->plan_host_devptr), h->plan_host, 0));
-  FT_TRY(cudaMalloc(&h->items_res, (2 * E + 1) * sizeof(WorkItem)));
-  FT_TRY(cudaMemset(h->items_res, 0, (2 * E + 1) * sizeof(WorkItem)));
-  FT_TRY(cudaMalloc(&h->items_zc, E * sizeof(WorkItem)));
-  FT_TRY(cudaMalloc(&h->items_gemm, E * sizeof(WorkItem)));
-  FT_TRY(cudaMalloc(&h->res_pref, (2 * E + 2) * 4));
-  FT_TRY(cudaMemset(h->res_pref, 0, (2 * E + 2) * 4));
+  FT_TRY(cudaMalloc(&h->items_res, L * (2 * E + 1) * sizeof(WorkItem)));
+  FT_TRY(cudaMemset(h->items_res, 0, L * (2 * E + 1) * sizeof(WorkItem)));
+  FT_TRY(cudaMalloc(&h->items_zc, L * E * sizeof(WorkItem)));
+  FT_TRY(cudaMalloc(&h->items_gemm, L * E * sizeof(WorkItem)));
+  FT_TRY(cudaMalloc(&h->res_pref, L * (2 * E + 2) * 4));
+  FT_TRY(cudaMemset(h->res_pref, 0, L * (2 * E + 2) * 4));
   if (c.gemm_min_tokens > 0) {
     const size_t Pr = P + 256;   // spare rows so that full boxes stay inside the tensors
-    FT_TRY(cudaMalloc(&h->gemm_pref, (E + 1) * 4));
-    FT_TRY(cudaMemset(h->gemm_pref, 0, (E + 1) * 4));
-    FT_TRY(cudaMalloc(&h->is_gemm, E));
-    FT_TRY(cudaMemset(h->is_gemm, 0, E));
+    FT_TRY(cudaMalloc(&h->gemm_pref, L * (E + 1) * 4));
+    FT_TRY(cudaMemset(h->gemm_pref, 0, L * (E + 1) * 4));
+    FT_TRY(cudaMalloc(&h->is_gemm, L * E));
+    FT_TRY(cudaMemset(h->is_gemm, 0, L * E));
     FT_TRY(cudaMalloc(&h->xs, Pr * c.hidden * 2));
     FT_TRY(cudaMalloc(&h->hbuf, Pr * c.inter * 2));
     FT_TRY(cudaMalloc(&h->obuf, Pr * c.hidden * 2));
@@ -610,20 +647,22 @@ static int single_cta_threads(int E, int T) {
   return n;
 }
 
-static RouteParams make_route_params(ft_moe *h, const float *logits_dev, int T) {
+static RouteParams make_route_params(ft_moe *h, int layer, const float *logits_dev, int T) {
+  const Scratch sc = scratch_of(h, layer);
   RouteParams rp;
   rp.logits = logits_dev;
   rp.T = T; rp.E = h->cfg.n_experts; rp.k = h->cfg.top_k;
-  rp.ids = h->ids; rp.w = h->topk_w; rp.count = h->count; rp.offset = h->offset;
-  rp.perm = h->perm; rp.inv = h->inv; rp.status = h->status_dev;
+  rp.ids = sc.ids; rp.w = sc.topk_w; rp.count = sc.count; rp.offset = sc.offset;
+  rp.perm = sc.perm; rp.inv = sc.inv; rp.status = h->status_dev;
   return rp;
 }
 
 static PlanParams make_plan_params(ft_moe *h, int layer, bool mirror_to_host) {
   const ft_moe_config_t &c = h->cfg;
   LayerState &L = h->layers[layer];
+  const Scratch sc = scratch_of(h, layer);
   PlanParams pp;
-  pp.count = h->count; pp.offset = h->offset;
+  pp.count = sc.count; pp.offset = sc.offset;
   pp.E = c.n_experts; pp.n_slots = h->table_slots;
   pp.id_base = c.global_pool ? layer * c.n_experts : 0;
   pp.cm.ns_fill = (int64_t)(h->S * 1000 / c.bw_fill_MBps);
@@ -640,14 +679,14 @@ static PlanParams make_plan_params(ft_moe *h, int layer, bool mirror_to_host) {
   pp.S = h->S; pp.T = L.T;
   pp.tokens_per_pass = (c.wdtype == FT_W_BF16) ? kFsResTokensPerPass : kQ4Tokens;
   pp.zc_tokens_per_pass = (c.wdtype == FT_W_BF16) ? kFsZcTokensPerPass : kQ4Tokens;
-  pp.hdr_dev = h->plan_dev;
-  pp.hdr_host = mirror_to_host ? h->plan_host_devptr : nullptr;
-  pp.items_res = h->items_res; pp.res_pref = h->res_pref;
-  pp.items_zc = h->items_zc; pp.items_gemm = h->items_gemm;
-  pp.gemm_pref = h->gemm_pref; pp.is_gemm = h->is_gemm;
+  pp.hdr_dev = sc.plan_dev;
+  pp.hdr_host = mirror_to_host ? sc.plan_host_devptr : nullptr;
+  pp.items_res = sc.items_res; pp.res_pref = sc.res_pref;
+  pp.items_zc = sc.items_zc; pp.items_gemm = sc.items_gemm;
+  pp.gemm_pref = sc.gemm_pref; pp.is_gemm = sc.is_gemm;
   // decode-sized calls on a prefill-capable handle keep every expert on the streaming kernels
   if (L.T < c.gemm_min_tokens) pp.cm.gemm_min_tokens = 0;
-  pp.seq_value = h->seq_host + 1;
+  pp.seq_value = L.seq + 1;
   return pp;
 }
 
@@ -657,16 +696,15 @@ ft_status_t ft_moe_route(ft_moe_t *h, int layer, const float *logits_dev, int T,
   LayerState &L = h->layers[layer];
   L.phase = PH_ROUTED;
   L.T = T;
-  h->last_routed_layer = layer;
   if (T == 0) return FT_OK;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const RouteParams rp = make_route_params(h, logits_dev, T);
+  const RouteParams rp = make_route_params(h, layer, logits_dev, T);
   TimeScope ts(h, st, FT_TIME_ROUTE);
   if (T <= kRouteSmallMaxTokens) {
     route_small_kernel<<<1, single_cta_threads(h->cfg.n_experts, T), 0, st>>>(rp);
     h->launches++;
   } else {
-    FT_CUDA(cudaMemsetAsync(h->count, 0, sizeof(int32_t) * rp.E, st));
+    FT_CUDA(cudaMemsetAsync(rp.count, 0, sizeof(int32_t) * rp.E, st));
     route_topk_kernel<<<(T + 7) / 8, 256, 0, st>>>(rp);
     permute_kernel<<<(rp.E + 7) / 8, 256, 0, st>>>(rp);
     h->launches += 2;
@@ -678,7 +716,7 @@ ft_status_t ft_moe_route(ft_moe_t *h, int layer, const float *logits_dev, int T,
 ft_status_t ft_moe_plan(ft_moe_t *h, int layer, ft_moe_plan_t *out, void *stream) {
   if (!h || layer < 0 || layer >= h->cfg.n_layers) return FT_ERR_INVALID_ARG;
   LayerState &L = h->layers[layer];
-  if (L.phase != PH_ROUTED || h->last_routed_layer != layer) return FT_ERR_STATE;
+  if (L.phase != PH_ROUTED) return FT_ERR_STATE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const ft_moe_config_t &c = h->cfg;
   if (L.T > 0) {
@@ -692,13 +730,14 @@ ft_status_t ft_moe_plan(ft_moe_t *h, int layer, ft_moe_plan_t *out, void *stream
       plan_kernel<<<1, threads, smem, st>>>(pp);
     }
     h->launches++;
-    h->seq_host++;
+    L.seq++;
     h->plan_mirrored = mirror;
     FT_CUDA(cudaGetLastError());
     FT_CUDA(cudaEventRecord(h->ev_plan, st));
   }
   L.phase = PH_PLANNED;
   if (out) {
+    const Scratch sc = scratch_of(h, layer);
     const int E = c.n_experts;
     if (L.T == 0) {
       out->step = -1;
@@ -707,9 +746,9 @@ ft_status_t ft_moe_plan(ft_moe_t *h, int layer, ft_moe_plan_t *out, void *stream
       return FT_OK;
     }
     FT_CUDA(cudaEventSynchronize(h->ev_plan));
-    const PlanHeader hd = *h->plan_host;
-    if (hd.seq != h->seq_host) return FT_ERR_CUDA;
-    const int32_t *a = reinterpret_cast<const int32_t *>(h->plan_host + 1);
+    const PlanHeader hd = *sc.plan_host;
+    if (hd.seq != L.seq) return FT_ERR_CUDA;
+    const int32_t *a = reinterpret_cast<const int32_t *>(sc.plan_host + 1);
     out->step = hd.step;
     out->n_routed = hd.n_routed; out->n_hit = hd.n_hit; out->n_miss = hd.n_miss;
     out->n_fill = hd.n_fill; out->n_zc = hd.n_zc;
@@ -733,6 +772,8 @@ ft_status_t ft_moe_fill(ft_moe_t *h, int layer, void *copy_stream) {
   L.phase = PH_FILLED;
   h->fill_timed = false;
   h->last_fill_bytes = 0;
+  h->last_fill_layer = layer;
+  const Scratch sc = scratch_of(h, layer);
   if (L.T == 0 || h->cfg.slots_per_layer == 0) return FT_OK;
   cudaStream_t cs = static_cast<cudaStream_t>(copy_stream);
   const ft_moe_config_t &c = h->cfg;
@@ -740,11 +781,11 @@ ft_status_t ft_moe_fill(ft_moe_t *h, int layer, void *copy_stream) {
   if (c.fill_mode == FT_FILL_COPY_ENGINE) {
     // the host needs the fill list: wait for the plan record (one host round trip per layer)
     FT_CUDA(cudaEventSynchronize(h->ev_plan));
-    const PlanHeader hd = *h->plan_host;
-    if (hd.seq != h->seq_host) return FT_ERR_CUDA;
+    const PlanHeader hd = *sc.plan_host;
+    if (hd.seq != L.seq) return FT_ERR_CUDA;
     if (hd.n_fill > 0) {
       const int E = c.n_experts;
-      const int32_t *a = reinterpret_cast<const int32_t *>(h->plan_host + 1);
+      const int32_t *a = reinterpret_cast<const int32_t *>(sc.plan_host + 1);
       const int32_t *forder = a + 4 * E, *fslot = a + 5 * E;
       const uint8_t *pool_layer = static_cast<const uint8_t *>(c.host_pool) + (size_t)layer * E * h->S;
       FT_CUDA(cudaStreamWaitEvent(cs, h->ev_plan, 0));
@@ -768,7 +809,7 @@ ft_status_t ft_moe_fill(ft_moe_t *h, int layer, void *copy_stream) {
     }
   } else {
     FillParams fp;
-    fp.hdr = h->plan_dev; fp.E = c.n_experts;
+    fp.hdr = sc.plan_dev; fp.E = c.n_experts;
     fp.pool_layer_dev = h->pool_dev + (size_t)layer * c.n_experts * h->S;
     fp.slots_layer = slots_layer; fp.S = h->S;
     FT_CUDA(cudaStreamWaitEvent(cs, h->ev_plan, 0));
@@ -799,33 +840,48 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   const ft_moe_config_t &c = h->cfg;
   const __nv_bfloat16 *x_bf = static_cast<const __nv_bfloat16 *>(x_dev);
   const bool use_gemm = h->gemm && L.T >= c.gemm_min_tokens;
+  const Scratch sc = scratch_of(h, layer);
   if (c.wdtype == FT_W_BF16) {
     // bulk-copy pipelined tensor-core streaming kernel; the last CTA of the last launch finalizes y
     FfnStreamParams mp;
-    mp.items = h->items_res;
-    mp.n_items = &h->plan_dev->n_res_items;
-    mp.n_hit = &h->plan_dev->n_hit_items;
-    mp.n_zc = &h->plan_dev->n_zc_items;
-    mp.pref = h->res_pref;
+    mp.items = sc.items_res;
+    mp.n_items = &sc.plan_dev->n_res_items;
+    mp.n_hit = &sc.plan_dev->n_hit_items;
+    mp.n_zc = &sc.plan_dev->n_zc_items;
+    mp.pref = sc.res_pref;
     mp.max_items = 2 * c.n_experts + 1;
     mp.trace = h->trace_dev;
-    mp.x = x_bf; mp.perm = h->perm; mp.topk_w = h->topk_w; mp.y_acc = h->y_acc;
+    mp.x = x_bf; mp.perm = sc.perm; mp.topk_w = sc.topk_w; mp.y_acc = h->y_acc;
     mp.y = static_cast<__nv_bfloat16 *>(y_dev);
     mp.done = h->done_dev; mp.status = h->status_dev;
     mp.inter = c.inter; mp.top_k = c.top_k; mp.T = L.T;
     const size_t smem = ffn_stream_smem_bytes(mp.max_items, c.hidden);
+    cudaError_t launch_err = cudaSuccess;
     auto launch = [&](int part, int finalize) {
       mp.part = part;
       mp.finalize = finalize;
+      mp.overlap = h->overlap;
       TimeScope ts(h, st, part == 1 ? FT_TIME_FFN_ZC : FT_TIME_FFN_RES);
       // while the device-driven fill holds kFillCtas SMs, the overlapping launch takes the others
       const int grid = (part == 1 && c.fill_mode == FT_FILL_SM) ? h->sm_count - kFillCtas : h->sm_count;
+      cudaLaunchConfig_t lc = {};
+      lc.gridDim = dim3((unsigned)grid);
+      lc.blockDim = dim3(kFsThreads);
+      lc.dynamicSmemBytes = smem;
+      lc.stream = st;
+      cudaLaunchAttribute la[1];
+      la[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      la[0].val.programmaticStreamSerializationAllowed = 1;
+      lc.attrs = la;
+      lc.numAttrs = h->overlap ? 1 : 0;
+      cudaError_t e;
       switch (c.hidden / 256) {
-        case 1: ffn_stream_kernel<1><<<grid, kFsThreads, smem, st>>>(mp); break;
-        case 2: ffn_stream_kernel<2><<<grid, kFsThreads, smem, st>>>(mp); break;
-        case 4: ffn_stream_kernel<4><<<grid, kFsThreads, smem, st>>>(mp); break;
-        default: ffn_stream_kernel<8><<<grid, kFsThreads, smem, st>>>(mp); break;
+        case 1: e = cudaLaunchKernelEx(&lc, ffn_stream_kernel<1>, mp); break;
+        case 2: e = cudaLaunchKernelEx(&lc, ffn_stream_kernel<2>, mp); break;
+        case 4: e = cudaLaunchKernelEx(&lc, ffn_stream_kernel<4>, mp); break;
+        default: e = cudaLaunchKernelEx(&lc, ffn_stream_kernel<8>, mp); break;
       }
+      if (e != cudaSuccess) launch_err = e;
       h->launches++;
     };
     // With enough tokens in the call the hits (and the zero-copy experts) are worth a launch of their own that
@@ -840,15 +896,16 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
       if (c.slots_per_layer > 0) FT_CUDA(cudaStreamWaitEvent(st, h->ev_fill, 0));
       launch(0, use_gemm ? 0 : 1);
     }
+    FT_CUDA(launch_err);
     FT_CUDA(cudaGetLastError());
     if (use_gemm) {
       // experts with many tokens: gather x rows into expert order, two grouped tcgen05 GEMMs, fused combine
       {
         TimeScope ts(h, st, FT_TIME_GATHER);
-        gather_rows_kernel<<<h->sm_count * 8, 256, 0, st>>>(x_bf, h->perm, c.top_k, c.hidden, h->offset + c.n_experts, h->xs);
+        gather_rows_kernel<<<h->sm_count * 8, 256, 0, st>>>(x_bf, sc.perm, c.top_k, c.hidden, sc.offset + c.n_experts, h->xs);
       }
       GemmParams gp;
-      gp.items = h->items_gemm; gp.n_items = &h->plan_dev->n_gemm_items; gp.mt_pref = h->gemm_pref;
+      gp.items = sc.items_gemm; gp.n_items = &sc.plan_dev->n_gemm_items; gp.mt_pref = sc.gemm_pref;
       gp.inter = c.inter; gp.d = c.hidden;
       gp.layer_unit0 = c.global_pool ? 0 : (long long)layer * c.slots_per_layer * (c.inter / 16);
       gp.status = h->status_dev;
@@ -878,7 +935,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
       }
       {
         TimeScope ts(h, st, FT_TIME_COMBINE);
-        combine_kernel<<<h->sm_count * 8, 256, 0, st>>>(h->obuf, h->ids, h->topk_w, h->inv, h->is_gemm, h->y_acc,
+        combine_kernel<<<h->sm_count * 8, 256, 0, st>>>(h->obuf, sc.ids, sc.topk_w, sc.inv, sc.is_gemm, h->y_acc,
                                                         static_cast<__nv_bfloat16 *>(y_dev), L.T, c.top_k, c.hidden);
       }
       h->launches += 4;
@@ -889,12 +946,12 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   // int4: gate/up kernel writes h, down kernel accumulates, its last CTA finalizes y
   if (c.slots_per_layer > 0) FT_CUDA(cudaStreamWaitEvent(st, h->ev_fill, 0));
   Q4Params qp;
-  qp.items = h->items_res;
-  qp.n_items = &h->plan_dev->n_res_items;
-  qp.n_zc = &h->plan_dev->n_zc_items;
-  qp.pref = h->res_pref;
+  qp.items = sc.items_res;
+  qp.n_items = &sc.plan_dev->n_res_items;
+  qp.n_zc = &sc.plan_dev->n_zc_items;
+  qp.pref = sc.res_pref;
   qp.max_items = 2 * c.n_experts + 1;
-  qp.x = x_bf; qp.perm = h->perm; qp.topk_w = h->topk_w;
+  qp.x = x_bf; qp.perm = sc.perm; qp.topk_w = sc.topk_w;
   qp.hbuf = h->q4_hbuf;
   qp.y_acc = h->y_acc; qp.y = static_cast<__nv_bfloat16 *>(y_dev);
   qp.done = h->done_dev; qp.status = h->status_dev;
@@ -938,16 +995,15 @@ ft_status_t ft_moe_layer(ft_moe_t *h, int layer, const float *logits_dev, const 
     const ft_moe_config_t &c = h->cfg;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     L.T = T;
-    h->last_routed_layer = layer;
     const bool mirror = c.fill_mode == FT_FILL_COPY_ENGINE;
-    const RouteParams rp = make_route_params(h, logits_dev, T);
+    const RouteParams rp = make_route_params(h, layer, logits_dev, T);
     const PlanParams pp = make_plan_params(h, layer, mirror);
     {
       TimeScope ts(h, st, FT_TIME_PLAN);
       route_plan_small_kernel<<<1, single_cta_threads(c.n_experts, T), (size_t)h->table_slots * 16, st>>>(rp, pp);
     }
     h->launches++;
-    h->seq_host++;
+    L.seq++;
     h->plan_mirrored = mirror;
     FT_CUDA(cudaGetLastError());
     FT_CUDA(cudaEventRecord(h->ev_plan, st));
@@ -985,21 +1041,21 @@ ft_status_t ft_moe_layer_host(ft_moe_t *h, int layer, const float *logits_host, 
 ft_status_t ft_moe_get_routing(ft_moe_t *h, int layer, int32_t *ids, float *w, int32_t *count,
                                int32_t *offset, int32_t *perm, int32_t *inv) {
   if (!h || layer < 0 || layer >= h->cfg.n_layers) return FT_ERR_INVALID_ARG;
-  if (h->last_routed_layer != layer) return FT_ERR_STATE;
   FT_CUDA(cudaSetDevice(h->cfg.device));
   FT_CUDA(cudaDeviceSynchronize());
+  const Scratch sc = scratch_of(h, layer);
   const size_t P = (size_t)h->layers[layer].T * h->cfg.top_k, E = h->cfg.n_experts;
   if (P == 0) {
     if (count) memset(count, 0, E * 4);
     if (offset) memset(offset, 0, (E + 1) * 4);
     return FT_OK;
   }
-  if (ids) FT_CUDA(cudaMemcpy(ids, h->ids, P * 4, cudaMemcpyDeviceToHost));
-  if (w) FT_CUDA(cudaMemcpy(w, h->topk_w, P * 4, cudaMemcpyDeviceToHost));
-  if (count) FT_CUDA(cudaMemcpy(count, h->count, E * 4, cudaMemcpyDeviceToHost));
-  if (offset) FT_CUDA(cudaMemcpy(offset, h->offset, (E + 1) * 4, cudaMemcpyDeviceToHost));
-  if (perm) FT_CUDA(cudaMemcpy(perm, h->perm, P * 4, cudaMemcpyDeviceToHost));
-  if (inv) FT_CUDA(cudaMemcpy(inv, h->inv, P * 4, cudaMemcpyDeviceToHost));
+  if (ids) FT_CUDA(cudaMemcpy(ids, sc.ids, P * 4, cudaMemcpyDeviceToHost));
+  if (w) FT_CUDA(cudaMemcpy(w, sc.topk_w, P * 4, cudaMemcpyDeviceToHost));
+  if (count) FT_CUDA(cudaMemcpy(count, sc.count, E * 4, cudaMemcpyDeviceToHost));
+  if (offset) FT_CUDA(cudaMemcpy(offset, sc.offset, (E + 1) * 4, cudaMemcpyDeviceToHost));
+  if (perm) FT_CUDA(cudaMemcpy(perm, sc.perm, P * 4, cudaMemcpyDeviceToHost));
+  if (inv) FT_CUDA(cudaMemcpy(inv, sc.inv, P * 4, cudaMemcpyDeviceToHost));
   return drain_status(h);
 }
 
@@ -1057,7 +1113,8 @@ ft_status_t ft_moe_last_fill(ft_moe_t *h, float *out_us, uint64_t *out_bytes) {
   uint64_t bytes = h->last_fill_bytes;
   if (bytes == ~0ull) {
     PlanHeader hd;
-    FT_CUDA(cudaMemcpy(&hd, h->plan_dev, sizeof(hd), cudaMemcpyDeviceToHost));
+    FT_CUDA(cudaMemcpy(&hd, scratch_of(h, h->last_fill_layer < 0 ? 0 : h->last_fill_layer).plan_dev, sizeof(hd),
+                       cudaMemcpyDeviceToHost));
     bytes = (uint64_t)hd.n_fill * h->S;
   }
   if (out_bytes) *out_bytes = bytes;
@@ -1097,6 +1154,12 @@ ft_status_t ft_moe_resize(ft_moe_t *h, int slots_per_layer) {
 ft_status_t ft_moe_set_split_min_pairs(ft_moe_t *h, int pairs) {
   if (!h || pairs < 0) return FT_ERR_INVALID_ARG;
   h->cfg.split_min_pairs = pairs;
+  return FT_OK;
+}
+
+ft_status_t ft_moe_set_launch_overlap(ft_moe_t *h, int mode) {
+  if (!h || mode < 0 || mode > 2) return FT_ERR_INVALID_ARG;
+  h->overlap = mode;
   return FT_OK;
 }
 

@@ -4,9 +4,9 @@
 //   H[P][I] = SiLU(Xs Wg^T) * (Xs Wu^T)   A = expert-sorted x rows (K-major, 128-byte swizzle), B = 128 gate rows +
 //                                          the same 128 up rows of the record, N = 256, over the experts that hold
 //                                          a slot and have at least `gemm_min_tokens` tokens.
-// The record's tile order is already the tensor core's K-major layout without swizzle (8 x 8 blocks of 128
-// contiguous bytes): a weight tile is moved by plain TMA boxes of whole 1 KiB tiles and described to the MMA with a
-// 128-byte step between the two blocks of a K = 16 slice and a 512-byte step between 8-row groups.
+// The record's tile order is already the tensor core's K-major layout with 64-byte swizzle (groups of 8 rows of
+// 64 bytes): a weight tile is moved by plain TMA boxes of whole 1 KiB tiles and described to the MMA with a
+// 512-byte step between 8-row groups; the two K = 16 slices of a tile are 32 bytes apart.
 // One persistent CTA per SM: warp 0 feeds a 4-stage shared-memory ring with TMA tile loads (cp.async.bulk.tensor,
 // no multicast), warp 1 issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32) into one of two
 // 256-column TMEM accumulators and signals stages free / tiles done with tcgen05.commit, warps 2-5 drain the other
@@ -54,8 +54,8 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm,
       : "memory");
 }
 
-// 64-bit shared-memory matrix descriptor.  lbo/sbo in bytes; swizzle: 2 = 128-byte swizzle, 0 = none (8 x 8 blocks of
-// 128 contiguous bytes; K-major: lbo = step between the two blocks of a K = 16 slice, sbo = step between 8-row groups).
+// 64-bit shared-memory matrix descriptor.  lbo/sbo in bytes (K-major: sbo = step between 8-row groups);
+// swizzle: 2 = 128-byte, 4 = 64-byte, 6 = 32-byte rows.
 __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr, uint32_t lbo, uint32_t sbo, uint32_t swizzle = 2) {
   uint64_t d = 0;
   d |= (uint64_t)((smem_addr >> 4) & 0x3fffu);
@@ -221,7 +221,7 @@ gateup_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             const uint32_t sb = sa + MT * kGemmATile;
 #pragma unroll
             for (int k16 = 0; k16 < kGemmBK / 16; ++k16) {
-              const uint64_t bdesc = umma_desc(sb + (k16 >> 1) * 16384 + (k16 & 1) * 256, 128, 512, 0);
+              const uint64_t bdesc = umma_desc(sb + (k16 >> 1) * 16384 + (k16 & 1) * 32, 16, 512, 4);
               for (int m = 0; m < n_mt; ++m) {
                 const uint64_t adesc = umma_desc(sa + m * kGemmATile + k16 * 32, 16, 1024);
                 umma_bf16(d_tmem + (uint32_t)m * kGemmBN, adesc, bdesc, idesc, (kb | k16) != 0 ? 1u : 0u);

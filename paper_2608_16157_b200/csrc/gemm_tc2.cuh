@@ -63,8 +63,8 @@ __device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
 // Swapped operands: the weights are the M side (always full 128-row tiles per CTA, 256 per pair), the tokens
 // are the N side, so a ragged expert is padded to a multiple of 16 tokens instead of 128 rows.
 //   O^T[column][token] : A = W_down^T, 128 columns per CTA x 64 neurons per stage, taken from the record's down
-//   tiles as they are (K-major 8 x 8 blocks without swizzle: 128 bytes between the two neuron blocks of a unit, 256
-//   bytes between 8-column groups); B = up to 256 rows of H (each CTA stages half).  TMEM lane = output column,
+//   tiles as they are (K-major rows of 32 bytes with 32-byte swizzle, 256 bytes between 8-column groups); B = up
+//   to 256 rows of H (each CTA stages half).  TMEM lane = output column,
 //   TMEM column = token; the epilogue writes O[token][column].
 struct Gemm2Cfg {
   static constexpr int kTokTile = 256;                                  // tokens per unit
@@ -199,7 +199,7 @@ down_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
             for (int k16 = 0; k16 < kGemmBK / 16; ++k16) {
               const uint32_t acc = (kb | k16) != 0 ? 1u : 0u;
-              umma2_bf16(d_tmem, umma_desc(sa + k16 * 4096, 128, 256, 0),
+              umma2_bf16(d_tmem, umma_desc(sa + k16 * 4096, 16, 256, 6),
                          umma_desc(sa + kGemmATile + k16 * 32, 16, 1024), idesc, acc);
             }
           }

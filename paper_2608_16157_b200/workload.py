@@ -11,13 +11,14 @@ Expert record formats (one contiguous record per (layer, expert); the pool is
 flattened identifier of Sec. 4.2 of the paper):
 
 ``bf16``  ``I/16`` units of 16 neurons, each ``96*d`` bytes: a gate part, an up part and a
-          down part of ``32*d`` bytes each, all in 8 x 8 blocks of bf16 (8 rows of 16 bytes).
-          Gate/up part: tiles of 16 neurons x 32 hidden indices (1 KiB), tile ``i // 32``;
-          inside a tile the block of neuron half ``(n % 16) // 8`` and hidden quarter
-          ``(i % 32) // 8`` starts at ``512*half + 128*quarter``, row ``n % 8``, element ``i % 8``.
+          down part of ``32*d`` bytes each.  Gate/up part: tiles of 16 neurons x 32 hidden
+          indices (1 KiB), tile ``i // 32``; a tile is two groups of 8 neuron rows of 64 bytes
+          (group ``(n % 16) // 8``, row ``r = n % 8``); the four 16-byte chunks of a row are
+          stored swizzled: chunk ``(i % 32) // 8`` sits at position ``chunk ^ (r >> 1)``.
           Down part: tiles of 16 output columns x the unit's 16 neurons (512 bytes), tile
-          ``c // 16``; block of column half ``(c % 16) // 8`` and neuron half ``(n % 16) // 8`` at
-          ``256*chalf + 128*nhalf``, row ``c % 8``, element ``n % 8``.  ``S = 3*I*d*2`` bytes.
+          ``c // 16``; two groups of 8 column rows of 32 bytes (group ``(c % 16) // 8``,
+          row ``r = c % 8``); the two 16-byte chunks of a row are stored at position
+          ``((n % 16) // 8) ^ (r >> 2)``.  ``S = 3*I*d*2`` bytes.
 ``int4``  4-bit two's-complement codes in [-8, 7] for the same three matrices,
           then bf16 scales.  ``Wg_q`` and ``Wu_q`` are row-major ``[I][d/2]`` bytes,
           two codes per byte along ``d`` (low nibble = even column).  ``Wd_q`` is
@@ -158,10 +159,17 @@ def _pack_bf16_tiles(w: torch.Tensor) -> torch.Tensor:
     """bf16 ``[3][I][d]`` (gate and up one row per neuron, down ``[n][c]``) -> the tiled record, flat."""
     _, I, d = w.shape
     U = I // 16
-    # gate / up: [unit][neuron half][row][tile][quarter][element] -> [unit][tile][half][quarter][row][element]
-    gu = w[0:2].reshape(2, U, 2, 8, d // 32, 4, 8).permute(0, 1, 4, 2, 5, 3, 6).reshape(2, U, 16 * d)
-    # down: [unit][neuron half][element][tile][column half][row] -> [unit][tile][chalf][nhalf][row][element]
-    dn = w[2].reshape(U, 2, 8, d // 16, 2, 8).permute(0, 3, 4, 1, 5, 2).reshape(U, 16 * d)
+    # gate / up: [unit][group][row][tile][chunk][element] -> [unit][tile][group][row][position][element]
+    gu = w[0:2].reshape(2, U, 2, 8, d // 32, 4, 8).permute(0, 1, 4, 2, 3, 5, 6)
+    row = torch.arange(8, device=w.device)
+    pos = torch.arange(4, device=w.device)
+    src = pos[None, :] ^ (row[:, None] >> 1)                    # chunk stored at position pos of row r
+    gu = gu[:, :, :, :, row[:, None], src, :].reshape(2, U, 16 * d)
+    # down: [unit][chunk][element][tile][group][row] -> [unit][tile][group][row][position][element]
+    dn = w[2].reshape(U, 2, 8, d // 16, 2, 8).permute(0, 3, 4, 5, 1, 2)
+    pos2 = torch.arange(2, device=w.device)
+    src2 = pos2[None, :] ^ (row[:, None] >> 2)
+    dn = dn[:, :, :, row[:, None], src2, :].reshape(U, 16 * d)
     return torch.cat([gu[0], gu[1], dn], dim=1).contiguous().reshape(-1)
 
 

@@ -22,14 +22,17 @@ def _record_bf16_by_definition(wg, wu, wd):
     for n in range(I):
         unit, nhalf, nrow = n // 16, (n % 16) // 8, n % 8
         for i in range(d):
-            # gate / up: 1 KiB tiles of 16 neurons x 32 hidden indices, 8 x 8 blocks inside
-            tile, quarter, e = i // 32, (i % 32) // 8, i % 8
-            at = unit * unit_el + tile * 512 + nhalf * 256 + quarter * 64 + nrow * 8 + e
+            # gate / up: 1 KiB tiles of 16 neurons x 32 hidden indices: two groups of 8 rows of 64 bytes (32
+            # elements); chunk (8 elements) number `chunk` of row r is stored at position chunk ^ (r >> 1)
+            tile, chunk, e = i // 32, (i % 32) // 8, i % 8
+            position = chunk ^ (nrow >> 1)
+            at = unit * unit_el + tile * 512 + nhalf * 256 + nrow * 32 + position * 8 + e
             rec[at] = gb[i, n]
             rec[at + 16 * d] = ub[i, n]
-            # down (i is the output column here): 512-byte tiles of 16 columns x the unit's 16 neurons
+            # down (i is the output column here): 512-byte tiles of 16 columns x the unit's 16 neurons: two
+            # groups of 8 column rows of 32 bytes; the chunk of neuron half nhalf is stored at nhalf ^ (r >> 2)
             ctile, chalf, crow = i // 16, (i % 16) // 8, i % 8
-            rec[unit * unit_el + 32 * d + ctile * 256 + chalf * 128 + nhalf * 64 + crow * 8 + nrow] = db[n, i]
+            rec[unit * unit_el + 32 * d + ctile * 256 + chalf * 128 + crow * 16 + (nhalf ^ (crow >> 2)) * 8 + nrow] = db[n, i]
     return rec.view(np.uint8)
 
 
