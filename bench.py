@@ -226,6 +226,8 @@ def run_ours(args):
     bw = dict(bw_fill=max(cal["fill_MBps"], 1), bw_zc=max(cal["zc_MBps"], 1),
               bw_zc_residual=cal["zc_residual_MBps"] if args.residual else 0, bw_hbm=max(cal["hbm_MBps"], 1))
     moe = make(bw)
+    if not dsv3:
+        moe.set_launch_overlap(args.overlap)
 
     stream = torch.cuda.current_stream()
     moe_sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
@@ -684,6 +686,8 @@ def main():
     ap.add_argument("--cpu-layers", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--only-batch", action="store_true")
+    ap.add_argument("--overlap", type=int, default=0,
+                    help="launch mode of the streaming kernel in the timed region (ft_moe_set_launch_overlap)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -265,6 +265,18 @@ ft_status_t ft_moe_set_split_min_pairs(ft_moe_t *h, int pairs);
  * of this layer are not produced by that preceding kernel (e.g. forward calls of several already planned layers
  * issued back to back).  Takes effect at the next ft_moe_forward. */
 ft_status_t ft_moe_set_launch_overlap(ft_moe_t *h, int mode);
+/* Test hook for the failure path of the bounded device-side waits (every wait of a kernel on an mbarrier gives up
+ * after a limited number of polls, latches FT_ERR_TIMEOUT in the device status word, lets the copies already in
+ * flight land and runs to completion: nothing traps, faults or hangs).  withhold_mask: FT_DEBUG_WITHHOLD_* bits;
+ * the named kernel's producer then leaves out one copy of its first stage, so the consumer's wait can never be
+ * satisfied.  wait_polls: the poll limit of every wait from now on (0 = the default, 2^22).  The setting is per
+ * process and device and stays until changed; call with (0, 0) to restore normal operation.  The output of a
+ * call that timed out is unspecified; ft_moe_sync_status reports FT_ERR_TIMEOUT once, and after ft_moe_reset
+ * the handle works as before.  Waits for the device. */
+enum { FT_DEBUG_WITHHOLD_FILL = 1,      /* device-driven fill kernel (FT_FILL_SM) */
+       FT_DEBUG_WITHHOLD_Q4 = 2,        /* int4 gate/up streaming kernel */
+       FT_DEBUG_WITHHOLD_GEMM = 4 };    /* prefill gate/up grouped GEMM */
+ft_status_t ft_moe_debug_inject(ft_moe_t *h, uint32_t withhold_mask, uint32_t wait_polls);
 /* Number of kernels this handle has launched since create. */
 ft_status_t ft_moe_launch_count(ft_moe_t *h, uint64_t *out);
 const char *ft_moe_status_string(ft_status_t s);

@@ -29,7 +29,7 @@ SYMBOLS = (
     "ft_moe_status_string", "ft_moe_timing_enable", "ft_moe_timing_read", "ft_moe_ffn_noalloc",
     "ft_moe_last_cuda_error", "ft_moe_host_register", "ft_moe_host_unregister",
     "ft_moe_get_cta_trace", "ft_moe_set_split_min_pairs", "ft_moe_resize", "ft_moe_ffn_noalloc_status",
-    "ft_moe_set_launch_overlap",
+    "ft_moe_set_launch_overlap", "ft_moe_debug_inject",
 )
 NOALLOC_MAX_TOKENS, NOALLOC_MAX_HIDDEN = 64, 2048
 TIME_NAMES = ("route", "plan", "ffn_zc", "ffn_res", "finalize", "fill", "gather", "gemm1", "gemm2", "combine")
@@ -114,6 +114,7 @@ def load(rebuild: bool = False):
         "ft_moe_last_cuda_error": (C.c_char_p, []),
         "ft_moe_ffn_noalloc_status": (i32, [i32]),
         "ft_moe_set_launch_overlap": (i32, [vp, i32]),
+        "ft_moe_debug_inject": (i32, [vp, C.c_uint32, C.c_uint32]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -365,6 +366,9 @@ class FtMoe:
 
     def set_launch_overlap(self, mode):
         _check(self._lib.ft_moe_set_launch_overlap(self._h, int(mode)), "ft_moe_set_launch_overlap")
+
+    def debug_inject(self, withhold_mask, wait_polls):
+        _check(self._lib.ft_moe_debug_inject(self._h, int(withhold_mask), int(wait_polls)), "ft_moe_debug_inject")
 
     def launch_count(self):
         n = C.c_uint64()

@@ -8,6 +8,19 @@ namespace ftmoe {
 // and runs to completion.  (A per-module variable so that a test can shorten it; the default is far beyond any
 // legitimate wait.)
 static __device__ uint32_t g_wait_polls = 1u << 22;
+constexpr uint32_t kDefaultWaitPolls = 1u << 22;
+
+// Test hook (ft_moe_debug_inject): bits that make one producer withhold a single copy, so that the consumer's
+// bounded wait runs out and the error path can be exercised without faulting, trapping or hanging anything.
+static __device__ uint32_t g_debug_withhold = 0;
+constexpr uint32_t kWithholdFill = 1u, kWithholdQ4 = 2u, kWithholdGemm = 4u;
+
+// After a bounded wait has given up: give the copies this CTA has already issued time to land before its shared
+// memory is released (bounded: about 50 us).
+__device__ __forceinline__ void abort_drain(volatile int *abort_flag) {
+  if (*abort_flag)
+    for (int i = 0; i < 50; ++i) __nanosleep(1000);
+}
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 

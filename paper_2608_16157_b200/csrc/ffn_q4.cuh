@@ -167,7 +167,8 @@ __global__ void __launch_bounds__(kQ4Threads, 1) q4_gateup_kernel(Q4Params p) {
               mbar_expect_tx(full_bar(s), 16 * row_bytes + 16 * scale_row);
             }
             __syncwarp();
-            if (!*s_abort) {
+            const bool withhold = (g_debug_withhold & kWithholdQ4) && tile == 0;   // test hook
+            if (!*s_abort && !withhold) {
               const uint32_t dst = smem_base + s * stage_bytes;
               if (lane < 16)
                 bulk_g2s(dst + lane * stride, it.w + which * mat_bytes + (size_t)(b * 16 + lane) * row_bytes, row_bytes,
@@ -278,6 +279,7 @@ __global__ void __launch_bounds__(kQ4Threads, 1) q4_gateup_kernel(Q4Params p) {
       u += (b_end - b_begin);
     }
   }
+  abort_drain(s_abort);
 }
 
 // CTW = 16-column tiles per warp; four CTAs (blockIdx.x & 3) share a range of blocks and split the columns in
@@ -440,6 +442,7 @@ __global__ void __launch_bounds__(kQ4Threads, 1) q4_down_kernel(Q4Params p) {
       u += (b_end - b_begin);
     }
   }
+  abort_drain(s_abort);
 
   if (!p.finalize) return;
   __threadfence();

@@ -92,6 +92,10 @@ __global__ void __launch_bounds__(kFsThreads, 1) ffn_stream_kernel(FfnStreamPara
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_start));
     p.trace[4 * blockIdx.x] = t_start;
   }
+  // The next kernel of the stream, if it was launched as a programmatic dependent, may be scheduled as soon as an SM
+  // has room for one of its CTAs, i.e. when one of this grid's CTAs has finished (what it may touch before this
+  // grid has completed is its own business: see `overlap`).
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (p.overlap == 1) asm volatile("griddepcontrol.wait;" ::: "memory");
   bool dep_waited = p.overlap != 2;
   const int n_items = *p.n_items;
@@ -392,8 +396,6 @@ __global__ void __launch_bounds__(kFsThreads, 1) ffn_stream_kernel(FfnStreamPara
     sg = nsg;
   }
 
-  // the next kernel of the stream, if it was launched as a programmatic dependent, may be scheduled from here on
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (!dep_waited) asm volatile("griddepcontrol.wait;" ::: "memory");   // (a CTA without work still orders its exit)
   if (p.trace != nullptr && tid == 0) {
     long long *tr = p.trace + 4 * blockIdx.x;

@@ -27,7 +27,7 @@ constexpr int kFillThreads = 32;
 __global__ void __launch_bounds__(kFillThreads) fill_kernel(FillParams p, uint32_t *status) {
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ uint64_t s_bar[kFillStages];
-  __shared__ int s_abort;
+  __shared__ volatile int s_abort;
   const int n_fill = p.hdr->n_fill;
   if (n_fill == 0 || threadIdx.x != 0) return;
   const int32_t *forder = reinterpret_cast<const int32_t *>(p.hdr + 1) + 4 * p.E;
@@ -54,6 +54,7 @@ __global__ void __launch_bounds__(kFillThreads) fill_kernel(FillParams p, uint32
     locate(i, src, dst, bytes);
     const int s = (int)(i % kFillStages);
     mbar_expect_tx(bar_base + 8 * s, bytes);
+    if ((g_debug_withhold & kWithholdFill) && i == 0) return;   // test hook: this copy never arrives
     bulk_g2s(smem_base + s * kFillChunk, src, bytes, bar_base + 8 * s);
   };
   for (long long i = 0; i < mine && i < kFillStages; ++i) issue_load(i);
@@ -72,6 +73,7 @@ __global__ void __launch_bounds__(kFillThreads) fill_kernel(FillParams p, uint32
     }
   }
   asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  abort_drain(&s_abort);
 }
 
 // Reads `bytes` (multiple of 16) and folds them into one word so the loads cannot be elided.

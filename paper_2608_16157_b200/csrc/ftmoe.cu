@@ -1163,6 +1163,17 @@ ft_status_t ft_moe_set_launch_overlap(ft_moe_t *h, int mode) {
   return FT_OK;
 }
 
+ft_status_t ft_moe_debug_inject(ft_moe_t *h, uint32_t withhold_mask, uint32_t wait_polls) {
+  if (!h || (withhold_mask & ~7u)) return FT_ERR_INVALID_ARG;
+  FT_CUDA(cudaSetDevice(h->cfg.device));
+  FT_CUDA(cudaDeviceSynchronize());
+  const uint32_t polls = wait_polls ? wait_polls : kDefaultWaitPolls;
+  FT_CUDA(cudaMemcpyToSymbol(g_debug_withhold, &withhold_mask, sizeof(uint32_t)));
+  FT_CUDA(cudaMemcpyToSymbol(g_wait_polls, &polls, sizeof(uint32_t)));
+  FT_CUDA(cudaDeviceSynchronize());
+  return FT_OK;
+}
+
 ft_status_t ft_moe_launch_count(ft_moe_t *h, uint64_t *out) {
   if (!h || !out) return FT_ERR_INVALID_ARG;
   *out = h->launches;

@@ -188,6 +188,7 @@ gateup_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
           const uint32_t sa = smem_base + s * kGemmStageBytes;
           const uint32_t sb = sa + MT * kGemmATile;
           mbar_expect_tx(full_bar(s), n_mt * kGemmATile + kGemmBTile);
+          if ((g_debug_withhold & kWithholdGemm) && it_k == 0) continue;   // test hook: stage never fills
           for (int m = 0; m < n_mt; ++m) tma_load_2d(sa + m * kGemmATile, &tmA, kb * kGemmBK, a_row + m * kGemmBM, full_bar(s));
           // per 32-wide hidden tile: 8 gate tiles (8 KiB: 16 groups of 8 neurons, 512 bytes apart) then the 8 up tiles
 #pragma unroll
@@ -276,6 +277,7 @@ gateup_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
       if (lane == 0) mbar_arrive(tempty_bar(buf));
     }
   }
+  abort_drain(s_abort);   // (after a bounded wait gave up: let the copies in flight land before the CTA goes away)
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {

@@ -252,6 +252,7 @@ down_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       if (lane == 0) mbar_arrive_cluster(mapa_u32(tempty_bar(buf), 0));   // the leader's MMA thread waits for both CTAs
     }
   }
+  abort_drain(s_abort);
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();                   // neither CTA leaves while the other may still touch its memory or barriers

@@ -418,6 +418,9 @@ __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, uns
 // Stand-alone plan kernel: blockDim.x = E rounded up to a warp multiple (at least 128).
 __global__ void __launch_bounds__(1024) plan_kernel(PlanParams p) {
   extern __shared__ __align__(16) unsigned char s_dyn[];
+  // a streaming kernel launched as a programmatic dependent may be scheduled now; it waits for this grid to
+  // complete before it reads the plan
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   __shared__ PlanSmem sm;
   const int tid = threadIdx.x;
   int64_t t;

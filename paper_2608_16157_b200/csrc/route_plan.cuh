@@ -7,6 +7,9 @@ namespace ftmoe {
 
 __global__ void __launch_bounds__(1024) route_plan_small_kernel(RouteParams rp, PlanParams pp) {
   extern __shared__ __align__(16) unsigned char s_dyn[];
+  // a streaming kernel launched as a programmatic dependent may be scheduled now; it waits for this grid to
+  // complete before it reads the plan
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   __shared__ RouteSmem rs;
   __shared__ PlanSmem ps;
   int64_t t;

@@ -65,3 +65,18 @@ def test_create_rejects_bad_arguments_without_a_gpu_call():
     cfg.hidden = 256
     assert lib.ft_moe_create(ctypes.byref(cfg), ctypes.byref(h)) == B.FT_ERR_INVALID_ARG   # null pool
     assert not h.value
+
+
+def test_noalloc_entry_point_checks_its_arguments_before_any_device_work():
+    """Size limits and pointer alignment are checked on the host: a view with an odd element offset is refused with
+    FT_ERR_INVALID_ARG instead of faulting on the device (no GPU needed: nothing is launched)."""
+    lib = B.load()
+    base = 0x7f0000001000                    # never dereferenced
+    f = lib.ft_moe_ffn_noalloc
+    assert f(0, base + 2, 256, 128, base, base, 4, None) == B.FT_ERR_INVALID_ARG
+    assert f(0, base, 256, 128, base + 6, base, 4, None) == B.FT_ERR_INVALID_ARG
+    assert f(0, base, 256, 128, base, base + 8, 4, None) == B.FT_ERR_INVALID_ARG
+    assert f(0, base, 256, 128, base, base, 0, None) == B.FT_ERR_INVALID_ARG
+    assert f(0, base, 256, 128, base, base, B.NOALLOC_MAX_TOKENS + 1, None) == B.FT_ERR_INVALID_ARG
+    assert f(0, None, 256, 128, base, base, 4, None) == B.FT_ERR_INVALID_ARG
+    assert f(0, base, 300, 128, base, base, 4, None) == B.FT_ERR_UNSUPPORTED

@@ -26,7 +26,7 @@ def _make(shape, L, n_slots, max_tokens, pool, **kw):
 def test_decode_config1_full_stack_graph_replay():
     """48 layers x 128 experts (54 GiB pinned pool, 27 GiB of slots), batch 8, the step replayed as one CUDA graph."""
     shape = W.QWEN3_30B
-    L, E, k, d, Bt, steps = 48, 128, 8, 2048, 8, 3
+    L, E, k, d, Bt, steps = 48, 128, 8, 2048, 8, 4
     S = shape.expert_bytes
     dev = torch.device("cuda:0")
     pool = B.HostPool(L * E * S)
@@ -35,6 +35,13 @@ def test_decode_config1_full_stack_graph_replay():
     recs = pool.tensor.view(L, E, S).numpy()
     oracles = [O.OracleLayer(d, shape.inter, E, k, 64, "bf16", recs[l], cm) for l in range(L)]
     logits = W.ar1_logits(L, steps, Bt, E, 0.8, 1.1, 0)
+    # step 0 routes the 64 pairs of every layer to 64 different experts, so all 64 slots are taken at once and
+    # the following steps have to evict
+    for l in range(L):
+        z = np.full((Bt, E), -20.0, dtype=np.float32)
+        for t in range(Bt):
+            z[t, (5 * l + 8 * t + np.arange(8)) % E] = np.linspace(2.0, 1.0, 8)
+        logits[0, l] = z
     lg_all = torch.from_numpy(logits).to(dev)
     s_lg = torch.empty((L, Bt, E), dtype=torch.float32, device=dev)
     s_noise = torch.empty((L, Bt, d), dtype=torch.bfloat16, device=dev)
@@ -68,6 +75,7 @@ def test_decode_config1_full_stack_graph_replay():
                 check_output(ybuf[l], r.y)
         st = moe.get_stats(17)
         assert st["steps"] == t + 1 and st["routed"] == st["hits"] + st["fills"] + st["zc"]
+    assert sum(moe.get_stats(l)["evictions"] for l in range(L)) > L      # the LRU was exercised at full size
     moe.destroy()
     pool.free()
 

@@ -118,6 +118,31 @@ def test_int4_group_dequant_and_shared_expert(n_shared, T):
     pr.close()
 
 
+@pytest.mark.parametrize("T", [9, 24, 40])
+def test_int4_resident_experts_with_many_tokens_and_shared_expert(T):
+    """More than 8 tokens per slot-resident int4 expert (several weight passes) and the shared expert at T > 8."""
+    shape = W.LayerShape(d=512, inter=256, n_experts=4, top_k=2, wdtype="int4", n_shared=1)
+    pr = Pair(shape, n_slots=4, max_tokens=40, seed=6)
+    for step in range(3):
+        _, r = pr.step(0, W.normal_logits(T, 4, 6, step), W.noise_x(T, 512, 6, step, 0))
+        if step > 0:
+            assert r.plan.zc == []                       # every routed expert is resident ...
+            assert T < 24 or max(r.count) >= 9           # ... some with more than 8 tokens (at T = 9 the shared one)
+    pr.close()
+
+
+@pytest.mark.parametrize("scale_log2", [-2, 2])
+def test_int4_activation_range(scale_log2):
+    """The int4 kernels convert activations to fp16 internally; inputs scaled by 2^-10 and 2^10 still meet the
+    tolerance (the output scales by the square: the FFN is bilinear in x)."""
+    shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2, wdtype="int4", n_shared=1)
+    pr = Pair(shape, n_slots=4, max_tokens=8, seed=8)
+    for step in range(2):
+        x = (W.noise_x(6, 512, 8, step, 0).float() * (2.0 ** scale_log2)).to(torch.bfloat16)
+        pr.step(0, W.normal_logits(6, 8, 8, step), x)
+    pr.close()
+
+
 def test_plan_and_permutation_are_deterministic():
     shape = W.LayerShape(d=256, inter=64, n_experts=32, top_k=4)
     runs = []
