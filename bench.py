@@ -34,6 +34,10 @@ if ROOT not in sys.path:
 SEED = 0
 RHO, ALPHA = 0.8, 1.1
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
+# DRAM bytes (read + write) of one ffn_stream_kernel launch over its algorithmic bytes, from the ncu capture
+# summarised in profiles/ (same kernel, batch 8, 24 resident experts per launch)
+NCU_TRAFFIC_RATIO = 1.03
+NCU_TRAFFIC_SOURCE = "profiles/ffn_stream_kernel_decode_qwen3_b8.md"
 
 
 def log(*a):
@@ -230,8 +234,8 @@ def run_ours(args):
         moe.set_launch_overlap(args.overlap)
 
     stream = torch.cuda.current_stream()
-    moe_sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
-    n_total = Wn + K + args.prof_steps + 12
+    CW = args.cache_warm_steps
+    n_total = CW + Wn + K + args.prof_steps + 12
 
     def gen_inputs(batch):
         lg = torch.from_numpy(W.ar1_logits(L, n_total, batch, E, RHO, ALPHA, SEED)).to(dev)
@@ -328,59 +332,98 @@ def run_ours(args):
                 tot[kk] = tot.get(kk, 0) + v
         return tot
 
+    def kernel_alone(lg, noise, batch, first, count, overlap):
+        """The expert-FFN kernel(s) timed alone: route, plan and fill every layer of a step first (untimed), then
+        the forward calls of all L layers back to back between two CUDA events.  Returns (us per layer, record
+        bytes streamed from HBM per layer)."""
+        moe.set_launch_overlap(overlap)
+        us, nbytes = [], []
+        for s in range(first, first + count):
+            st0 = stats_sum()
+            for l in range(L):
+                moe.route(l, lg[s, l], batch, stream)
+                moe.plan(l, stream, want=False)
+                moe.fill(l, None)
+            torch.cuda.synchronize()
+            st1 = stats_sum()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for l in range(L):
+                moe.forward(l, noise[s, l], ybuf[l, :batch], stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            us.append(e0.elapsed_time(e1) * 1e3 / L)
+            nbytes.append((st1["hits"] - st0["hits"] + st1["fills"] - st0["fills"] +
+                           shape.n_shared * (st1["steps"] - st0["steps"])) * S / L)
+        moe.set_launch_overlap(0)
+        return statistics.median(us), sum(nbytes) / len(nbytes)
+
     results = {}
     for batch in ([B] if (args.only_batch or dsv3) else [B, 1] if B != 1 else [1]):
         lg, noise = gen_inputs(batch)
         moe.reset()
-        for s in range(Wn):
+        moe.set_launch_overlap(args.overlap if not dsv3 else 0)
+        # cache pre-warm: a fixed number of untimed steps from the empty cache, whatever --warmup is, so that the
+        # timed region is the steady state; the first K of them are timed separately as the cold-start figure
+        torch.cuda.synchronize()
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_cold = min(K, CW)
+        c0.record(stream)
+        for s in range(CW):
             step(lg, noise, s, batch)
+            if s == n_cold - 1:
+                c1.record(stream)
+        torch.cuda.synchronize()
+        cold_ms = c0.elapsed_time(c1) if n_cold > 0 else None
+        for s in range(CW, CW + Wn):
+            if use_graph:
+                step_graph(lg, noise, s, batch)
+            else:
+                step(lg, noise, s, batch)
         torch.cuda.synchronize()
         st0 = stats_sum()
-        ms, clocks, launches = timed(lg, noise, batch, Wn, K, sample_clocks=(batch == B))
+        ms, clocks, launches = timed(lg, noise, batch, CW + Wn, K, sample_clocks=(batch == B))
         st1 = stats_sum()
         dst = {kk: st1[kk] - st0[kk] for kk in st1}
-        # per-kernel durations with CUDA events on the launching stream (separate pass: events perturb).  The
-        # roofline kernel is timed alone: one launch per layer after the fills, not overlapped with them.
+        # ---- the roofline kernel, timed alone (one launch per layer: no split into hit / fill parts) ----
         split_saved = moe.cfg.split_min_pairs
         moe.set_split_min_pairs(0)
+        p0 = CW + Wn + K
+        n_alone = max(2, args.prof_steps // 4)
+        alone = {}
+        if not dsv3:
+            for name, ov in (("overlapped", 2), ("plain", 0)):
+                kernel_alone(lg, noise, batch, p0, 1, ov)                       # warm-up of the pass itself
+                alone[name] = kernel_alone(lg, noise, batch, p0 + 1, n_alone, ov)
+        else:
+            kernel_alone(lg, noise, batch, p0, 1, 0)
+            alone["plain"] = kernel_alone(lg, noise, batch, p0 + 1, n_alone, 0)
+        # ---- per-kernel durations inside the step, each launch bracketed by two events (separate pass) ----
         moe.timing_enable(True)
         st2 = stats_sum()
-        for s in range(Wn + K, Wn + K + args.prof_steps):
+        for s in range(p0 + 1 + n_alone, p0 + 1 + n_alone + max(2, args.prof_steps // 2)):
             step(lg, noise, s, batch)
         tim = moe.timing_read()
         st3 = stats_sum()
         moe.timing_enable(False)
         res_bytes = (st3["hits"] - st2["hits"] + st3["fills"] - st2["fills"] +
                      shape.n_shared * (st3["steps"] - st2["steps"])) * S
-        # device-timer view of the same kernel (no event bracketing): first CTA start -> y finalized, per launch
-        dev_us, dev_bytes = 0.0, 0
-        if not dsv3:
-            s_ = Wn + K + args.prof_steps
-            for l in range(L):
-                h0 = moe.get_stats(l)
-                x = noise[s_, 0] if l == 0 else torch.add(noise[s_, l], ybuf[l - 1, :batch], out=xbuf[l, :batch])
-                moe.layer(l, lg[s_, l], x, ybuf[l, :batch], batch, stream)
-                tr = moe.cta_trace(moe_sm_count)
-                h1 = moe.get_stats(l)
-                fin = -int(tr[:, 3].min())
-                if fin > 0:
-                    dev_us += (fin - int(tr[:, 0].min())) * 1e-3
-                    dev_bytes += (h1["hits"] - h0["hits"] + h1["fills"] - h0["fills"]) * S
         moe.set_split_min_pairs(split_saved)
         # the same steps with the hits overlapping the fills, as in the timed region
         tim_ov = None
         if split_saved > 0 and batch * k >= split_saved and not dsv3:
             moe.timing_enable(True)
-            for s in range(Wn + K + args.prof_steps + 1, Wn + K + args.prof_steps + 5):
+            for s in range(n_total - 6, n_total - 2):
                 step(lg, noise, s, batch)
             tim_ov = moe.timing_read()
             moe.timing_enable(False)
         results[batch] = dict(ms=ms, clocks=clocks, launches=launches, dstats=dst, timing=tim, timing_overlapped=tim_ov,
-                              dev_us=dev_us, dev_bytes=dev_bytes,
+                              alone=alone, cold_ms=cold_ms, n_cold=n_cold,
                               res_bytes=res_bytes, prof_fill_bytes=(st3["fills"] - st2["fills"]) * S,
                               lg=lg, noise=noise)
         log(f"[rank {rank}] batch {batch}: {ms / K:.3f} ms/step, {batch * K * world / (ms * 1e-3):.1f} tok/s, "
-            f"per step: hits {dst['hits'] / K:.1f} fills {dst['fills'] / K:.2f} zc {dst['zc'] / K:.2f}")
+            f"per step: hits {dst['hits'] / K:.1f} fills {dst['fills'] / K:.2f} zc {dst['zc'] / K:.2f}; "
+            f"kernel alone (us/launch, bytes/launch): {alone}")
         log(f"[rank {rank}]   kernel timing (us total, launches): {tim}")
 
     main = results[B]
@@ -390,8 +433,10 @@ def run_ours(args):
     ffn_us, ffn_n = tim["ffn_res"]
     if dsv3:   # the int4 path streams a record with two kernels: gate/up (timed in the ffn_zc slot) + down
         ffn_us += tim["ffn_zc"][0]
-    achieved = main["res_bytes"] / (ffn_us * 1e-6) / 1e9 if ffn_us > 0 else 0.0
+    in_step = main["res_bytes"] / (ffn_us * 1e-6) / 1e9 if ffn_us > 0 else 0.0
     fill_us, fill_n = tim["fill"]
+    best = main["alone"].get("overlapped") or main["alone"]["plain"]
+    achieved = best[1] / (best[0] * 1e-6) / 1e9
 
     # end to end through the host-buffer entry point
     e2e = None
@@ -412,12 +457,12 @@ def run_ours(args):
                     torch.add(noise_h[s, l], yh[l - 1], out=x)
                 moe.layer_host(l, lg_h[s, l], x, yh[l], B, stream)
 
-        for s in range(Wn + K, Wn + K + 3):
+        for s in range(CW + Wn + K, CW + Wn + K + 3):
             step_host(s)
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
-        for s in range(Wn, Wn + Ke):
+        for s in range(CW + Wn, CW + Wn + Ke):
             step_host(s)
         e1.record(stream)
         barrier()
@@ -435,8 +480,8 @@ def run_ours(args):
         lg, noise = main["lg"], main["noise"]
         n_samp = min(args.cpu_layers, 2) if dsv3 else args.cpu_layers
         pool_np = pool.tensor.view(L, E, S).numpy()
-        lg_np = lg[Wn].cpu().numpy()
-        xb = [noise[Wn, l].cpu().view(torch.int16).numpy().view(np.uint16) for l in range(n_samp)]
+        lg_np = lg[CW + Wn].cpu().numpy()
+        xb = [noise[CW + Wn, l].cpu().view(torch.int16).numpy().view(np.uint16) for l in range(n_samp)]
         cm_args = (S, bw["bw_fill"], bw["bw_zc_residual"], bw["bw_zc"], bw["bw_hbm"], 1, 64, 128)
         sec = oracle_sample_seconds(pool_np, shape, Ns, cm_args, lg_np, xb, range(n_samp))
         cpu_baseline = {"value": B / (sec * L / n_samp), "unit": "tok/s", "cores": len(os.sched_getaffinity(0)),
@@ -457,25 +502,42 @@ def run_ours(args):
                        "fill_mode": args.fill, "cuda_graph": use_graph, "global_pool": bool(args.global_pool), "rho": RHO, "zipf_alpha": ALPHA,
                        "l2": "inputs larger than L2: every step streams GBs of distinct expert records from the slot "
                              "pool, far beyond the 126 MB L2; no flush needed",
+                       "cache_warm_steps": CW, "launch_overlap_in_step": args.overlap,
                        "parallelism": "replicas" if world > 1 else "single",
                        "host_pool": "one /dev/shm copy shared by all ranks" if shm_name else "private pinned pool"},
             "clocks": main["clocks"],
             "e2e": e2e,
             "gpu_launches": main["launches"],
-            "roofline": {"bound": "hbm", "kernel": ("q4_gateup_kernel + q4_down_kernel (one pass over each record)" if dsv3
-                                                   else "ffn_mma_kernel (resident experts)"),
-                         "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
-                         "frac": achieved / hbm_peak if hbm_peak else None, "peak_source": peak_kind,
-                         "launches_timed": ffn_n, "avg_launch_us": ffn_us / ffn_n if ffn_n else None,
-                         "bytes_per_launch": main["res_bytes"] / ffn_n if ffn_n else None,
-                         # DRAM read+write per launch from the ncu capture of the same kernel and per-launch
-                         # work (profiles/): 1.03 x the algorithmic bytes
-                         "traffic": (1.03 * main["res_bytes"] / ffn_n) if (ffn_n and not dsv3) else None,
-                         # the same launches timed by the kernel's own global-timer trace (first CTA start to
-                         # y finalized): excludes the ~5 us that bracketing a launch with two events adds
-                         "achieved_device_timer": (main["dev_bytes"] / (main["dev_us"] * 1e-6) / 1e9) if main["dev_us"] else None,
-                         "frac_device_timer": (main["dev_bytes"] / (main["dev_us"] * 1e-6) / 1e9 / hbm_peak) if main["dev_us"] else None},
+            "roofline": {
+                "bound": "hbm",
+                "kernel": ("q4_gateup_kernel + q4_down_kernel (one pass over each record)" if dsv3
+                           else "ffn_stream_kernel (expert FFN over the HBM-resident records of a layer)"),
+                "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
+                "frac": achieved / hbm_peak if hbm_peak else None, "peak_source": peak_kind + " (burst: kernel timed alone)",
+                "how": (f"kernel timed alone: route, plan and fill of all {L} layers of a step issued first (untimed), "
+                        f"then the {L} forward launches back to back on the stream between two CUDA events, "
+                        "launched as programmatic dependents (ft_moe_set_launch_overlap 2: a launch streams its "
+                        "weights while the previous one drains and orders only its output accumulation after it); "
+                        "duration = elapsed / launches, median over steps; bytes = resident experts x record bytes"
+                        if "overlapped" in main["alone"] else
+                        f"kernel timed alone: the {L} forward launches of a planned step back to back between two events"),
+                "avg_launch_us": best[0], "bytes_per_launch": best[1], "launches_timed": L * max(2, args.prof_steps // 4),
+                # DRAM read+write per launch from the ncu capture of the same kernel (profiles/): ratio to the
+                # algorithmic bytes, scaled to this run's bytes per launch
+                "traffic": (NCU_TRAFFIC_RATIO * best[1]) if not dsv3 else None,
+                "traffic_source": (NCU_TRAFFIC_SOURCE if not dsv3 else None),
+                # the same launches as plain back-to-back launches (no dependent-launch overlap)
+                "plain_back_to_back": {"avg_launch_us": main["alone"]["plain"][0],
+                                       "achieved": main["alone"]["plain"][1] / (main["alone"]["plain"][0] * 1e-6) / 1e9,
+                                       "frac": main["alone"]["plain"][1] / (main["alone"]["plain"][0] * 1e-6) / 1e9 / hbm_peak},
+                # and inside the step, every launch bracketed by its own pair of events (adds ~5 us per launch)
+                "in_step_bracketed": {"avg_launch_us": ffn_us / ffn_n if ffn_n else None, "achieved": in_step,
+                                      "frac": in_step / hbm_peak if hbm_peak else None,
+                                      "bytes_per_launch": main["res_bytes"] / ffn_n if ffn_n else None}},
             "cpu_baseline": cpu_baseline,
+            "cold_start": {"value": B * main["n_cold"] * world / (main["cold_ms"] * 1e-3) if main["cold_ms"] else None,
+                           "unit": "tok/s", "steps": main["n_cold"],
+                           "what": "the first steps from an empty cache (untimed part of the run, before the pre-warm ends)"},
             "per_step": {"hits": dst["hits"] / K, "fills": dst["fills"] / K, "zero_copy": dst["zc"] / K,
                          "routed_unique": dst["routed"] / K, "fill_bytes": dst["fills"] / K * S},
             "fill": {"GBps": (main["prof_fill_bytes"] / (fill_us * 1e-6) / 1e9) if fill_us > 0 else None,
@@ -489,28 +551,54 @@ def run_ours(args):
         if 1 in results and B != 1:
             r1 = results[1]
             t1 = r1["timing"]
-            a1 = r1["res_bytes"] / (t1["ffn_res"][0] * 1e-6) / 1e9 if t1["ffn_res"][0] > 0 else 0.0
+            b1 = r1["alone"].get("overlapped") or r1["alone"]["plain"]
+            a1 = b1[1] / (b1[0] * 1e-6) / 1e9
+            a1p = r1["alone"]["plain"][1] / (r1["alone"]["plain"][0] * 1e-6) / 1e9
+            a1s = r1["res_bytes"] / (t1["ffn_res"][0] * 1e-6) / 1e9 if t1["ffn_res"][0] > 0 else 0.0
             line["batch1"] = {"value": K * world / (r1["ms"] * 1e-3), "unit": "tok/s", "ms_per_step": r1["ms"] / K,
-                              "ffn_res_GBps": a1, "ffn_res_frac": a1 / hbm_peak,
-                              "fills_per_step": r1["dstats"]["fills"] / K}
-        print(json.dumps(line), flush=True)
+                              "ffn_res_GBps": a1, "ffn_res_frac": a1 / hbm_peak, "avg_launch_us": b1[0],
+                              "bytes_per_launch": b1[1],
+                              "plain_back_to_back_frac": a1p / hbm_peak, "in_step_bracketed_frac": a1s / hbm_peak,
+                              "fills_per_step": r1["dstats"]["fills"] / K,
+                              "cold_start_tok_per_s": (r1["n_cold"] * world / (r1["cold_ms"] * 1e-3)) if r1["cold_ms"] else None}
     moe.destroy()
     pool.free()
+    results.clear()
+    del xbuf, ybuf
+    torch.cuda.empty_cache()
+    if rank == 0:
+        if world == 1 and not dsv3 and args.layers == 48:
+            # bounded sub-records of the other single-GPU configurations (a few layers each)
+            for name in [n for n in args.sub.split(",") if n]:
+                t_sub = time.perf_counter()
+                try:
+                    line[name] = SUBRECORDS[name](args, dev, cal)
+                except Exception as exc:      # a sub-record never takes the headline down with it
+                    line[name] = {"error": f"{type(exc).__name__}: {exc}"}
+                log(f"[rank 0] sub-record {name}: {time.perf_counter() - t_sub:.1f}s {line[name]}")
+        print(json.dumps(line), flush=True)
     if shm_name is not None:
         MR.close_shared_pool(pool.array, shm_name, rank, dist.barrier)
     if dist is not None:
         dist.destroy_process_group()
 
 
-def run_prefill(args):
-    """Prefill configuration: one step of `--tokens` tokens through all layers, cold cache then warm."""
+def tensor_peaks():
+    pk = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(pk):
+        dd = json.load(open(pk))
+        return float(dd["bf16_tflops"]), float(dd["bf16_tflops_sustained"]), "measured"
+    return FALLBACK_BF16_TFLOPS, 1400.0, "fallback"
+
+
+def prefill_passes(args, dev, L, cal=None):
+    """Config 2 on L layers: one 4096-token step from a cold cache, then one on the cache it left behind.  Returns
+    (per-pass records, calibration, layer constants)."""
     import torch
     from paper_2608_16157_b200 import binding as Bd
     from paper_2608_16157_b200 import workload as W
-    torch.cuda.set_device(0)
-    dev = torch.device("cuda", 0)
     shape = W.QWEN3_30B
-    L, E, k, d, I = args.layers, shape.n_experts, shape.top_k, shape.d, shape.inter
+    E, k, d, I = shape.n_experts, shape.top_k, shape.d, shape.inter
     S = shape.expert_bytes
     Ns = W.slots_for_fraction(args.cache_frac, E)
     T = args.tokens
@@ -520,21 +608,16 @@ def run_prefill(args):
                   host_pool_ptr=pool.ptr.value, host_pool_bytes=pool.n_bytes,
                   fill_mode=Bd.FT_FILL_SM if args.fill == "sm" else Bd.FT_FILL_COPY_ENGINE,
                   gemm_min_tokens=args.gemm_min_tokens)
-    moe = Bd.FtMoe(Bd.make_config(**common))
-    cal = moe.calibrate()
-    moe.destroy()
+    if cal is None:
+        moe = Bd.FtMoe(Bd.make_config(**common))
+        cal = moe.calibrate()
+        moe.destroy()
     moe = Bd.FtMoe(Bd.make_config(bw_fill=max(cal["fill_MBps"], 1), bw_zc=max(cal["zc_MBps"], 1), bw_zc_residual=0,
                                   bw_hbm=max(cal["hbm_MBps"], 1), **common))
     stream = torch.cuda.current_stream()
     xbuf = torch.empty((L, T, d), dtype=torch.bfloat16, device=dev)
     ybuf = torch.empty((L, T, d), dtype=torch.bfloat16, device=dev)
     out = {}
-    peak_hbm, peak_kind = peaks()
-    pk = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    tf_burst, tf_sust = FALLBACK_BF16_TFLOPS, 1400.0
-    if os.path.exists(pk):
-        dd = json.load(open(pk))
-        tf_burst, tf_sust = float(dd["bf16_tflops"]), float(dd["bf16_tflops_sustained"])
     for name, step in (("cold", 0), ("warm", 1)):
         lg = torch.from_numpy(W.prefill_logits(L, T, E, ALPHA, SEED, step)).to(dev)
         g = torch.Generator(device=dev)
@@ -563,6 +646,7 @@ def run_prefill(args):
         flops = 2.0 * 3 * d * I * dst["pairs_gemm"]
         gemm_us = tim["gemm1"][0] + tim["gemm2"][0]
         fill_us = tim["fill"][0]
+        route_us = tim["route"][0] + tim["plan"][0]
         out[name] = {"ms": ms, "tok_per_s": T / (ms * 1e-3), "launches": moe.launch_count() - l0 + L - 1,
                      "fills": dst["fills"], "zero_copy": dst["zc"], "hits": dst["hits"],
                      "pairs": dst["pairs"], "pairs_gemm": dst["pairs_gemm"],
@@ -570,17 +654,33 @@ def run_prefill(args):
                      "gemm1_tflops": (flops * 2 / 3) / (tim["gemm1"][0] * 1e-6) / 1e12 if tim["gemm1"][0] > 0 else None,
                      "gemm2_tflops": (flops / 3) / (tim["gemm2"][0] * 1e-6) / 1e12 if tim["gemm2"][0] > 0 else None,
                      "fill_GBps": dst["fills"] * S / (fill_us * 1e-6) / 1e9 if fill_us > 0 else None,
+                     "route_plan_us_per_layer": route_us / L,
                      "kernel_ms": {kk: v[0] / 1e3 for kk, v in tim.items()}}
         log(f"prefill {name}: {out[name]}")
+    moe.destroy()
+    pool.free()
+    del xbuf, ybuf
+    torch.cuda.empty_cache()
+    return out, cal, dict(T=T, L=L, d=d, E=E, I=I, k=k, Ns=Ns)
+
+
+def run_prefill(args):
+    """One prefill step of `--tokens` tokens through the stack, cold cache then warm (second step on the state
+    the first left behind).  One JSON line; the roofline object is the tensor-core grouped GEMM."""
+    import torch
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    out, cal, c = prefill_passes(args, dev, args.layers)
+    tf_burst, tf_sust, peak_kind = tensor_peaks()
     w = out["warm"]
     line = {"metric": "moe_prefill_tok_per_s", "value": out["cold"]["tok_per_s"], "unit": "tok/s", "n_gpus": 1,
             "steps": 1, "warmup": 0, "ms_per_step": out["cold"]["ms"], "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "prefill Qwen3-30B-A3B-shaped MoE stack (config 2), cold cache", "tokens": T,
-                       "layers": L, "hidden": d, "experts": E, "inter": I, "top_k": k, "slots_per_layer": Ns,
-                       "gemm_min_tokens": args.gemm_min_tokens, "fill_mode": args.fill},
+            "config": {"workload": "prefill Qwen3-30B-A3B-shaped MoE stack (config 2), cold cache", "tokens": c["T"],
+                       "layers": c["L"], "hidden": c["d"], "experts": c["E"], "inter": c["I"], "top_k": c["k"],
+                       "slots_per_layer": c["Ns"], "gemm_min_tokens": args.gemm_min_tokens, "fill_mode": args.fill},
             "cold": out["cold"], "warm": out["warm"],
-            "roofline": {"bound": "tensor", "kernel": "grouped_gemm_kernel<0>+<1> (warm pass)",
+            "roofline": {"bound": "tensor", "kernel": "gateup_gemm_kernel + down_gemm2_kernel (warm pass)",
                          "achieved": w["gemm_tflops"], "peak": tf_burst, "unit": "TFLOP/s",
                          "frac": (w["gemm_tflops"] / tf_burst) if w["gemm_tflops"] else None,
                          "frac_of_sustained": (w["gemm_tflops"] / tf_sust) if w["gemm_tflops"] else None,
@@ -588,8 +688,115 @@ def run_prefill(args):
             "fill": {"GBps": out["cold"]["fill_GBps"], "link_GBps_measured": cal["fill_MBps"] / 1e3},
             "gpu_launches": out["cold"]["launches"]}
     print(json.dumps(line), flush=True)
+
+
+def sub_prefill(args, dev, cal):
+    """Sub-record of the decode line: config 2 (4096-token prefill) on 4 of the 48 layers."""
+    L = 4
+    out, cal, c = prefill_passes(args, dev, L, cal)
+    tf_burst, tf_sust, peak_kind = tensor_peaks()
+    w, cd = out["warm"], out["cold"]
+    return {"config": f"prefill, config 2 shapes, {c['T']} tokens, {L} of 48 layers, {c['Ns']} slots per layer, "
+                      f"experts with >= {args.gemm_min_tokens} tokens and a slot on the tcgen05 grouped GEMMs",
+            "cold_ms": cd["ms"], "warm_ms": w["ms"], "cold_ms_scaled_to_48_layers": cd["ms"] * 48 / L,
+            "warm_ms_scaled_to_48_layers": w["ms"] * 48 / L,
+            "useful_tflops": w["gemm_tflops"], "gateup_tflops": w["gemm1_tflops"], "down_tflops": w["gemm2_tflops"],
+            "frac": (w["gemm_tflops"] / tf_burst) if w["gemm_tflops"] else None,
+            "frac_of_sustained": (w["gemm_tflops"] / tf_sust) if w["gemm_tflops"] else None,
+            "peak_burst_tflops": tf_burst, "peak_sustained_tflops": tf_sust, "peak_source": peak_kind,
+            "how": "useful (unpadded) flops of the pairs served by the GEMMs / summed CUDA-event durations of the "
+                   "two GEMM kernels, warm pass",
+            "fill_GBps_cold": cd["fill_GBps"], "route_plan_us_per_layer": w["route_plan_us_per_layer"],
+            "pairs_on_gemm_frac": w["pairs_gemm"] / max(w["pairs"], 1), "zero_copy_experts_cold": cd["zero_copy"]}
+
+
+def sub_int4(args, dev, cal):
+    """Sub-record of the decode line: config 3 (DeepSeek-V3-shaped int4 decode, 4 layers, batch 4, 64 slots)."""
+    import torch
+    from paper_2608_16157_b200 import binding as Bd
+    from paper_2608_16157_b200 import workload as W
+    shape = W.DSV3_INT4
+    L, E, k, d, B, Ns = 4, shape.n_experts, shape.top_k, shape.d, 4, 64
+    S = shape.expert_bytes
+    warm, K = 48, 16
+    pool = Bd.HostPool(L * E * S)
+    W.fill_pool(pool.tensor, shape, L, SEED, device=dev, chunk=16)
+    shared = W.make_shared_records(shape, L, SEED, device=dev)
+    moe = Bd.FtMoe(Bd.make_config(hidden=d, inter=shape.inter, n_experts=E, top_k=k, n_layers=L, slots_per_layer=Ns,
+                                  max_tokens=8, host_pool_ptr=pool.ptr.value, host_pool_bytes=pool.n_bytes,
+                                  fill_mode=Bd.FT_FILL_SM, wdtype=Bd.FT_W_INT4_G128, n_shared=1,
+                                  shared_ptr=shared.data_ptr(), bw_fill=max(cal["fill_MBps"], 1),
+                                  bw_zc=max(cal["zc_MBps"], 1), bw_zc_residual=0, bw_hbm=max(cal["hbm_MBps"], 1)))
+    stream = torch.cuda.current_stream()
+    n_total = warm + K + 12
+    lg = torch.from_numpy(W.ar1_logits(L, n_total, B, E, 0.9, 1.2, SEED)).to(dev)
+    g = torch.Generator(device=dev)
+    g.manual_seed(W.mix64(SEED, 80, B))
+    noise = torch.randn((n_total, L, B, d), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    xbuf = torch.empty((L, B, d), dtype=torch.bfloat16, device=dev)
+    ybuf = torch.empty((L, B, d), dtype=torch.bfloat16, device=dev)
+
+    def step(s):
+        for l in range(L):
+            x = noise[s, 0] if l == 0 else torch.add(noise[s, l], ybuf[l - 1], out=xbuf[l])
+            moe.layer(l, lg[s, l], x, ybuf[l], B, stream)
+
+    def stats_sum():
+        tot = {}
+        for l in range(L):
+            for kk, v in moe.get_stats(l).items():
+                tot[kk] = tot.get(kk, 0) + v
+        return tot
+
+    for s in range(warm):
+        step(s)
+    torch.cuda.synchronize()
+    st0 = stats_sum()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for s in range(warm, warm + K):
+        step(s)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    st1 = stats_sum()
+    # the two int4 kernels (gate/up, down) timed alone: all layers planned and filled first, then the forward
+    # calls back to back between two events
+    us, nbytes = [], []
+    for s in range(warm + K, warm + K + 8):
+        a = stats_sum()
+        for l in range(L):
+            moe.route(l, lg[s, l], B, stream)
+            moe.plan(l, stream, want=False)
+            moe.fill(l, None)
+        torch.cuda.synchronize()
+        b = stats_sum()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(stream)
+        for l in range(L):
+            moe.forward(l, noise[s, l], ybuf[l], stream)
+        f1.record(stream)
+        torch.cuda.synchronize()
+        us.append(f0.elapsed_time(f1) * 1e3 / L)
+        nbytes.append((b["hits"] - a["hits"] + b["fills"] - a["fills"] + (b["steps"] - a["steps"])) * S / L)
+    assert moe.sync_status() == 0
     moe.destroy()
     pool.free()
+    hbm_peak, peak_kind = peaks()
+    t_us, nb = statistics.median(us[2:]), sum(nbytes[2:]) / len(nbytes[2:])
+    gbps = nb / (t_us * 1e-6) / 1e9
+    return {"config": "decode, config 3: d=7168, 256 int4-g128 experts + 1 shared, I=2048, top-8, 4 layers, 64 slots "
+                      "per layer, batch 4, rho 0.9, alpha 1.2",
+            "tok_per_s": B * K / (ms * 1e-3), "ms_per_step": ms / K,
+            "fills_per_step": (st1["fills"] - st0["fills"]) / K, "cache_warm_steps": warm,
+            "GBps": gbps, "frac": gbps / hbm_peak, "peak": hbm_peak, "peak_source": peak_kind,
+            "avg_us_per_layer": t_us, "bytes_per_layer": nb,
+            "how": "gate/up + down kernels of a layer timed alone: the 4 layers of a step planned and filled first, "
+                   "then their forward calls back to back between two CUDA events; bytes = (resident routed experts "
+                   "+ the shared expert) x record bytes"}
+
+
+SUBRECORDS = {"int4": sub_int4, "prefill": sub_prefill}
 
 
 def run_sweep(args):
@@ -686,6 +893,9 @@ def main():
     ap.add_argument("--cpu-layers", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--only-batch", action="store_true")
+    ap.add_argument("--cache-warm-steps", type=int, default=64,
+                    help="untimed steps from the empty cache before warm-up and timing (steady-state headline)")
+    ap.add_argument("--sub", default="int4,prefill", help="bounded sub-records added to the decode line (N=1 only)")
     ap.add_argument("--overlap", type=int, default=0,
                     help="launch mode of the streaming kernel in the timed region (ft_moe_set_launch_overlap)")
     args = ap.parse_args()
