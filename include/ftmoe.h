@@ -198,6 +198,19 @@ ft_status_t ft_moe_plan(ft_moe_t *h, int layer, ft_moe_plan_t *out_host, void *s
  * record the handle's fill event there.  The copies are ordered after the plan. */
 ft_status_t ft_moe_fill(ft_moe_t *h, int layer, void *copy_stream);
 
+/* Full-layer prefetch for prefill (paper Sec. 3.1: while layer l is being computed, a transfer stream loads the
+ * complete expert set of layer l+1, before its routing is known, into the second of two full-layer buffers taken
+ * from the same slot pool; the survivors seed the decode cache).  Admits every expert of `layer` that is not yet
+ * resident through the ordinary residency machinery -- one plan over "all experts routed once" on `stream`, then
+ * the fills on copy_stream (NULL = the handle's own copy stream) -- so the victims are the least recently used
+ * slots, i.e. those of layers already computed.  Nothing is evaluated and no step of the layer is counted; the
+ * layer's later route/plan finds hits.  The handle's fill event is recorded: the next ft_moe_forward waits for
+ * it.  Needs room for two full-layer buffers: with global_pool a shared pool of at least 2*n_experts slots,
+ * otherwise slots_per_layer >= n_experts; else FT_ERR_UNSUPPORTED and the caller falls back to on-demand fills
+ * (paper: "if the memory budget cannot support two full-layer buffers, prefill falls back to on-demand
+ * loading").  The layer must be idle (no route/plan/fill of it pending). */
+ft_status_t ft_moe_prefetch_layer(ft_moe_t *h, int layer, void *stream, void *copy_stream);
+
 /* Steps 5+6 (paper Sec. 3.2: grouped evaluation of H u F on the GPU, the in-place set beside it, and an exact
  * merge of the partial sums -- no approximation of the MoE output): x_dev DEVICE bf16 [T][hidden], y_dev DEVICE
  * bf16 [T][hidden] (written), both 16-byte aligned.  Waits (on the

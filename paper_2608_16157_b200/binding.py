@@ -29,7 +29,7 @@ SYMBOLS = (
     "ft_moe_status_string", "ft_moe_timing_enable", "ft_moe_timing_read", "ft_moe_ffn_noalloc",
     "ft_moe_last_cuda_error", "ft_moe_host_register", "ft_moe_host_unregister",
     "ft_moe_get_cta_trace", "ft_moe_set_split_min_pairs", "ft_moe_resize", "ft_moe_ffn_noalloc_status",
-    "ft_moe_set_launch_overlap", "ft_moe_debug_inject",
+    "ft_moe_set_launch_overlap", "ft_moe_debug_inject", "ft_moe_prefetch_layer",
 )
 NOALLOC_MAX_TOKENS, NOALLOC_MAX_HIDDEN = 64, 2048
 TIME_NAMES = ("route", "plan", "ffn_zc", "ffn_res", "finalize", "fill", "gather", "gemm1", "gemm2", "combine")
@@ -115,6 +115,7 @@ def load(rebuild: bool = False):
         "ft_moe_ffn_noalloc_status": (i32, [i32]),
         "ft_moe_set_launch_overlap": (i32, [vp, i32]),
         "ft_moe_debug_inject": (i32, [vp, C.c_uint32, C.c_uint32]),
+        "ft_moe_prefetch_layer": (i32, [vp, i32, vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -279,6 +280,10 @@ class FtMoe:
 
     def fill(self, layer, copy_stream=None):
         _check(self._lib.ft_moe_fill(self._h, layer, _stream(copy_stream)), "ft_moe_fill")
+
+    def prefetch_layer(self, layer, stream=None, copy_stream=None):
+        _check(self._lib.ft_moe_prefetch_layer(self._h, layer, _stream(stream), _stream(copy_stream)),
+               "ft_moe_prefetch_layer")
 
     def forward(self, layer, x_dev, y_dev, stream=None):
         _check(self._lib.ft_moe_forward(self._h, layer, _ptr(x_dev), _ptr(y_dev), _stream(stream)), "ft_moe_forward")

@@ -33,6 +33,8 @@ struct LayerState {
   int phase = PH_IDLE;
   int T = 0;
   uint32_t seq = 0;            // plans launched for this layer (stale-record check of the host mirror)
+  cudaEvent_t ev_fill = nullptr;   // recorded on the copy stream after the layer's latest fills (or whole-layer prefetch)
+  bool fill_recorded = false;
 };
 
 // Per-layer scratch: the routing arrays, the plan record and the work lists of the layer's latest step.  Every
@@ -65,6 +67,7 @@ struct ft_moe {
   size_t pair_stride = 0, plan_stride = 0;   // bytes per layer of the pair arrays / the plan record
   int32_t *ids = nullptr, *count = nullptr, *offset = nullptr, *perm = nullptr, *inv = nullptr;
   float *topk_w = nullptr;
+  int32_t *route_hist = nullptr;        // [blocks of 128 tokens][E] histograms of the blocked route / permute kernels
   float *y_acc = nullptr;
   PlanHeader *plan_dev = nullptr;
   PlanHeader *plan_host = nullptr;      // pinned, mapped
@@ -406,6 +409,7 @@ ft_status_t ft_moe_destroy(ft_moe_t *h) {
   cudaFree(h->perm);
   cudaFree(h->inv);
   cudaFree(h->topk_w);
+  cudaFree(h->route_hist);
   cudaFree(h->y_acc);
   cudaFree(h->plan_dev);
   if (h->plan_host) cudaFreeHost(h->plan_host);
@@ -431,6 +435,8 @@ ft_status_t ft_moe_destroy(ft_moe_t *h) {
   cudaEvent_t evs[] = {h->ev_plan, h->ev_fill, h->ev_fork, h->ev_join, h->ev_fill_t0, h->ev_fill_t1};
   for (cudaEvent_t e : evs)
     if (e) cudaEventDestroy(e);
+  for (auto &ls : h->layers)
+    if (ls.ev_fill) cudaEventDestroy(ls.ev_fill);
   for (auto &p : h->pending) { cudaEventDestroy(p.e0); cudaEventDestroy(p.e1); }
   for (cudaEvent_t e : h->free_events) cudaEventDestroy(e);
   (void)cudaGetLastError();
@@ -525,6 +531,7 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
   FT_TRY(cudaMalloc(&h->offset, L * (E + 1) * 4));
   FT_TRY(cudaMalloc(&h->perm, L * h->pair_stride));
   FT_TRY(cudaMalloc(&h->inv, L * h->pair_stride));
+  FT_TRY(cudaMalloc(&h->route_hist, ((size_t)c.max_tokens / kRouteBlockTokens + 1) * E * 4));
   FT_TRY(cudaMalloc(&h->y_acc, (size_t)c.max_tokens * c.hidden * 4));
   FT_TRY(cudaMemset(h->y_acc, 0, (size_t)c.max_tokens * c.hidden * 4));
   h->plan_bytes = sizeof(PlanHeader) + 8 * E * 4;
@@ -608,6 +615,7 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
   FT_TRY(cudaStreamCreateWithFlags(&h->aux_stream, cudaStreamNonBlocking));
   FT_TRY(cudaEventCreateWithFlags(&h->ev_plan, cudaEventDisableTiming));
   FT_TRY(cudaEventCreateWithFlags(&h->ev_fill, cudaEventDisableTiming));
+  for (auto &ls : h->layers) FT_TRY(cudaEventCreateWithFlags(&ls.ev_fill, cudaEventDisableTiming));
   FT_TRY(cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming));
   FT_TRY(cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming));
   FT_TRY(cudaEventCreate(&h->ev_fill_t0));
@@ -687,6 +695,7 @@ static PlanParams make_plan_params(ft_moe *h, int layer, bool mirror_to_host) {
   // decode-sized calls on a prefill-capable handle keep every expert on the streaming kernels
   if (L.T < c.gemm_min_tokens) pp.cm.gemm_min_tokens = 0;
   pp.seq_value = L.seq + 1;
+  pp.prefetch = 0;
   return pp;
 }
 
@@ -704,10 +713,12 @@ ft_status_t ft_moe_route(ft_moe_t *h, int layer, const float *logits_dev, int T,
     route_small_kernel<<<1, single_cta_threads(h->cfg.n_experts, T), 0, st>>>(rp);
     h->launches++;
   } else {
-    FT_CUDA(cudaMemsetAsync(rp.count, 0, sizeof(int32_t) * rp.E, st));
-    route_topk_kernel<<<(T + 7) / 8, 256, 0, st>>>(rp);
-    permute_kernel<<<(rp.E + 7) / 8, 256, 0, st>>>(rp);
-    h->launches += 2;
+    const int n_blocks = (T + kRouteBlockTokens - 1) / kRouteBlockTokens;
+    int scan_threads = ((rp.E + 31) / 32) * 32;
+    route_block_kernel<<<n_blocks, 1024, 0, st>>>(rp, h->route_hist);
+    route_scan_kernel<<<1, scan_threads, 0, st>>>(rp, h->route_hist, n_blocks);
+    permute_block_kernel<<<n_blocks, 256, 0, st>>>(rp, h->route_hist);
+    h->launches += 3;
   }
   FT_CUDA(cudaGetLastError());
   return FT_OK;
@@ -765,6 +776,36 @@ ft_status_t ft_moe_plan(ft_moe_t *h, int layer, ft_moe_plan_t *out, void *stream
   return FT_OK;
 }
 
+ft_status_t ft_moe_prefetch_layer(ft_moe_t *h, int layer, void *stream, void *copy_stream) {
+  if (!h || layer < 0 || layer >= h->cfg.n_layers) return FT_ERR_INVALID_ARG;
+  const ft_moe_config_t &c = h->cfg;
+  LayerState &L = h->layers[layer];
+  if (L.phase != PH_IDLE) return FT_ERR_STATE;
+  // two full-layer buffers must fit: the layer being computed and the one being loaded
+  if (c.global_pool ? (h->table_slots < 2 * c.n_experts) : (c.slots_per_layer < c.n_experts)) return FT_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const Scratch sc = scratch_of(h, layer);
+  all_experts_kernel<<<1, 256, 0, st>>>(sc.count, sc.offset, c.n_experts);
+  L.T = c.n_experts <= c.max_tokens ? c.n_experts : c.max_tokens;   // (only sizes the shared expert's passes: unused here)
+  const bool mirror = c.fill_mode == FT_FILL_COPY_ENGINE;
+  PlanParams pp = make_plan_params(h, layer, mirror);
+  pp.prefetch = 1;
+  pp.cm.gemm_min_tokens = 0;
+  int threads = ((c.n_experts + 31) / 32) * 32;
+  if (threads < 128) threads = 128;
+  plan_kernel<<<1, threads, (size_t)h->table_slots * 16, st>>>(pp);
+  h->launches += 2;
+  L.seq++;
+  h->plan_mirrored = mirror;
+  FT_CUDA(cudaGetLastError());
+  FT_CUDA(cudaEventRecord(h->ev_plan, st));
+  L.phase = PH_PLANNED;
+  ft_status_t rc = ft_moe_fill(h, layer, copy_stream ? copy_stream : h->copy_stream);
+  L.phase = PH_IDLE;
+  L.T = 0;
+  return rc;
+}
+
 ft_status_t ft_moe_fill(ft_moe_t *h, int layer, void *copy_stream) {
   if (!h || layer < 0 || layer >= h->cfg.n_layers) return FT_ERR_INVALID_ARG;
   LayerState &L = h->layers[layer];
@@ -799,13 +840,15 @@ ft_status_t ft_moe_fill(ft_moe_t *h, int layer, void *copy_stream) {
         }
       }
       FT_CUDA(cudaEventRecord(h->ev_fill_t1, cs));
-      FT_CUDA(cudaEventRecord(h->ev_fill, cs));
+      FT_CUDA(cudaEventRecord(L.ev_fill, cs));
+      L.fill_recorded = true;
       h->fill_timed = true;
       h->last_fill_bytes = (uint64_t)hd.n_fill * h->S;
     } else {
       // nothing to copy: the fill event of an earlier layer must not be waited on needlessly
       FT_CUDA(cudaStreamWaitEvent(cs, h->ev_plan, 0));
-      FT_CUDA(cudaEventRecord(h->ev_fill, cs));
+      FT_CUDA(cudaEventRecord(L.ev_fill, cs));
+      L.fill_recorded = true;
     }
   } else {
     FillParams fp;
@@ -821,7 +864,8 @@ ft_status_t ft_moe_fill(ft_moe_t *h, int layer, void *copy_stream) {
     h->launches++;
     FT_CUDA(cudaGetLastError());
     FT_CUDA(cudaEventRecord(h->ev_fill_t1, cs));
-    FT_CUDA(cudaEventRecord(h->ev_fill, cs));
+    FT_CUDA(cudaEventRecord(L.ev_fill, cs));
+    L.fill_recorded = true;
     h->fill_timed = true;
     h->last_fill_bytes = ~0ull;  // resolved from the plan record when asked
   }
@@ -890,10 +934,10 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     const bool split = c.slots_per_layer > 0 && (long long)L.T * c.top_k >= c.split_min_pairs && c.split_min_pairs > 0;
     if (split) {
       launch(1, 0);
-      FT_CUDA(cudaStreamWaitEvent(st, h->ev_fill, 0));
+      if (L.fill_recorded) FT_CUDA(cudaStreamWaitEvent(st, L.ev_fill, 0));
       launch(2, use_gemm ? 0 : 1);
     } else {
-      if (c.slots_per_layer > 0) FT_CUDA(cudaStreamWaitEvent(st, h->ev_fill, 0));
+      if (c.slots_per_layer > 0 && L.fill_recorded) FT_CUDA(cudaStreamWaitEvent(st, L.ev_fill, 0));
       launch(0, use_gemm ? 0 : 1);
     }
     FT_CUDA(launch_err);
@@ -944,7 +988,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     return FT_OK;
   }
   // int4: gate/up kernel writes h, down kernel accumulates, its last CTA finalizes y
-  if (c.slots_per_layer > 0) FT_CUDA(cudaStreamWaitEvent(st, h->ev_fill, 0));
+  if (c.slots_per_layer > 0 && L.fill_recorded) FT_CUDA(cudaStreamWaitEvent(st, L.ev_fill, 0));
   Q4Params qp;
   qp.items = sc.items_res;
   qp.n_items = &sc.plan_dev->n_res_items;

@@ -42,6 +42,7 @@ struct PlanParams {
   int32_t *gemm_pref;    // [E+1]  exclusive prefix of the 128-row tiles of items_gemm
   uint8_t *is_gemm;      // [E]    1 if the expert goes through the grouped GEMM in this step
   uint32_t seq_value;    // sequence number of this plan (counted by the host)
+  int prefetch;          // 1: admission of a whole layer ahead of its routing (no step of the layer is counted)
 };
 
 // Block-wide exclusive scan of one 64-bit value per thread (several small counters packed into it).
@@ -391,19 +392,21 @@ __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, uns
     h.pad[0] = h.pad[1] = h.pad[2] = h.pad[3] = 0;
     *p.hdr_dev = h;
     *p.step = t + 1;
-    if (p.layer_steps != p.step) *p.layer_steps += 1;
+    if (p.layer_steps != p.step && !p.prefetch) *p.layer_steps += 1;
     int evictions = 0;
     for (int i = 0; i < n_fill; ++i) evictions += (s_sexp[s_victim[i]] >= 0);
     // fire-and-forget adds: nothing waits for the old values
-    atomicAdd(&p.stats[0], 1ull);
-    atomicAdd(&p.stats[1], (unsigned long long)n_routed);
-    atomicAdd(&p.stats[2], (unsigned long long)n_hit);
-    atomicAdd(&p.stats[3], (unsigned long long)n_miss);
     atomicAdd(&p.stats[4], (unsigned long long)n_fill);
-    atomicAdd(&p.stats[5], (unsigned long long)n_zc);
     atomicAdd(&p.stats[6], (unsigned long long)evictions);
-    atomicAdd(&p.stats[7], (unsigned long long)n_pairs);
-    atomicAdd(&p.stats[8], (unsigned long long)sm.pairs_res);
+    if (!p.prefetch) {
+      atomicAdd(&p.stats[0], 1ull);
+      atomicAdd(&p.stats[1], (unsigned long long)n_routed);
+      atomicAdd(&p.stats[2], (unsigned long long)n_hit);
+      atomicAdd(&p.stats[3], (unsigned long long)n_miss);
+      atomicAdd(&p.stats[5], (unsigned long long)n_zc);
+      atomicAdd(&p.stats[7], (unsigned long long)n_pairs);
+      atomicAdd(&p.stats[8], (unsigned long long)sm.pairs_res);
+    }
   }
   // mirror the record into mapped host memory when the host reads the plan (copy-engine fills)
   if (p.hdr_host != nullptr) {
@@ -412,6 +415,14 @@ __device__ __forceinline__ void plan_body(const PlanParams &p, PlanSmem &sm, uns
     const uint32_t *src = reinterpret_cast<const uint32_t *>(p.hdr_dev);
     volatile uint32_t *dst = reinterpret_cast<volatile uint32_t *>(p.hdr_host);
     for (int i = tid; i < n_words; i += blockDim.x) dst[i] = src[i];
+  }
+}
+
+// Counts of a layer whose every expert is "routed" once: the input of a whole-layer admission.
+__global__ void __launch_bounds__(1024) all_experts_kernel(int32_t *count, int32_t *offset, int E) {
+  for (int e = threadIdx.x; e <= E; e += blockDim.x) {
+    if (e < E) count[e] = 1;
+    offset[e] = e;
   }
 }
 

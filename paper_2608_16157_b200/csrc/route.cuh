@@ -173,64 +173,117 @@ __global__ void __launch_bounds__(1024) route_small_kernel(RouteParams p) {
   route_small_body(p, s);
 }
 
-// Prefill-sized calls, kernel 1: one warp per token; counts by integer atomics (order-free result).
-__global__ void __launch_bounds__(256) route_topk_kernel(RouteParams p) {
-  const int lane = threadIdx.x & 31;
-  const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (t >= p.T) return;
-  int id;
-  float w;
-  route_token_any(p, t, lane, id, w);
-  if (lane < p.k) {
-    p.ids[t * p.k + lane] = id;
-    p.w[t * p.k + lane] = w;
-    atomicAdd(&p.count[id], 1);
+// ---- prefill-sized calls: three launches over blocks of kRouteBlockTokens tokens ----
+constexpr int kRouteBlockTokens = 128;
+
+// Kernel 1: block b routes its tokens (one warp per token at a time), writes ids / w and the block's histogram
+// hist[b][E] (integer atomics in shared memory: the counts do not depend on the order of the adds).
+__global__ void __launch_bounds__(1024) route_block_kernel(RouteParams p, int32_t *hist) {
+  __shared__ int32_t s_cnt[kMaxExperts];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int e = tid; e < p.E; e += blockDim.x) s_cnt[e] = 0;
+  __syncthreads();
+  const int t0 = blockIdx.x * kRouteBlockTokens;
+  const int t1 = min(p.T, t0 + kRouteBlockTokens);
+  for (int t = t0 + warp; t < t1; t += (blockDim.x >> 5)) {
+    int id;
+    float w;
+    route_token_any(p, t, lane, id, w);
+    if (lane < p.k) {
+      p.ids[t * p.k + lane] = id;
+      p.w[t * p.k + lane] = w;
+      atomicAdd(&s_cnt[id], 1);
+    }
+  }
+  __syncthreads();
+  for (int e = tid; e < p.E; e += blockDim.x) hist[(size_t)blockIdx.x * p.E + e] = s_cnt[e];
+}
+
+// Kernel 2: one CTA, one thread per expert: count[e], the exclusive prefix of the block histograms over the blocks
+// (written back into hist) and offset[] by a block scan of the counts.  blockDim.x >= E, a multiple of 32.
+__global__ void __launch_bounds__(1024) route_scan_kernel(RouteParams p, int32_t *hist, int n_blocks) {
+  __shared__ int32_t s_wsum[32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+  int c = 0;
+  if (tid < p.E) {
+    for (int b = 0; b < n_blocks; ++b) {
+      const int v = hist[(size_t)b * p.E + tid];
+      hist[(size_t)b * p.E + tid] = c;
+      c += v;
+    }
+  }
+  int incl = c;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int n = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += n;
+  }
+  if (lane == 31) s_wsum[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    const int ws = (lane < nwarps) ? s_wsum[lane] : 0;
+    int wincl = ws;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int n = __shfl_up_sync(0xffffffffu, wincl, o);
+      if (lane >= o) wincl += n;
+    }
+    s_wsum[lane] = wincl - ws;
+  }
+  __syncthreads();
+  const int excl = incl - c + s_wsum[warp];
+  if (tid < p.E) {
+    p.count[tid] = c;
+    p.offset[tid] = excl;
+    if (tid == p.E - 1) p.offset[p.E] = excl + c;
   }
 }
 
-// Prefill-sized calls, kernel 2: one warp per expert; offset = sum of the counts before it, then a
-// walk over all pair keys (four per lane and iteration) ranks this expert's pairs in index order.
-__global__ void __launch_bounds__(256) permute_kernel(RouteParams p) {
-  const int lane = threadIdx.x & 31;
-  const int e = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (e >= p.E) return;
-  int before = 0;
-  for (int i = lane; i < e; i += 32) before += p.count[i];
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
-  const int c = p.count[e];
-  if (lane == 0) {
-    p.offset[e] = before;
-    if (e == p.E - 1) p.offset[p.E] = before + c;
-  }
-  if (c == 0) return;
+// Kernel 3: block b ranks its pairs.  pos(p) = offset[e] + pairs of expert e in earlier blocks + pairs of e earlier
+// in this block, which keeps the order stable in the pair index.  Each warp owns a contiguous part of the block's
+// pairs and walks it 32 pairs at a time; lanes with equal keys find each other with match.any.
+__global__ void __launch_bounds__(256) permute_block_kernel(RouteParams p, const int32_t *hist) {
+  __shared__ int32_t s_base[8][kMaxExperts];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int P = p.T * p.k;
-  int run = before;
-  const int end = before + c;
-  for (int base = 0; base < P && run < end; base += 128) {
-    const int q0 = base + lane * 4;
-    int4 kk = make_int4(-1, -1, -1, -1);
-    if (q0 + 3 < P) {
-      kk = *reinterpret_cast<const int4 *>(p.ids + q0);
-    } else {
-      if (q0 < P) kk.x = p.ids[q0];
-      if (q0 + 1 < P) kk.y = p.ids[q0 + 1];
-      if (q0 + 2 < P) kk.z = p.ids[q0 + 2];
-    }
-    const int n_mine = (kk.x == e) + (kk.y == e) + (kk.z == e) + (kk.w == e);
-    // exclusive prefix of n_mine over the lanes (pairs of lower lanes come first)
-    int incl = n_mine;
+  const int q0 = blockIdx.x * kRouteBlockTokens * p.k;
+  const int q1 = min(P, q0 + kRouteBlockTokens * p.k);
+  const int per_warp = (((q1 - q0 + 7) / 8) + 31) & ~31;    // a multiple of 32 pairs
+  const int w0 = q0 + warp * per_warp, w1 = min(q1, w0 + per_warp);
+  for (int e = tid; e < p.E; e += blockDim.x)
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int n = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += n;
+    for (int w = 0; w < 8; ++w) s_base[w][e] = 0;
+  __syncthreads();
+  const unsigned lt = (1u << lane) - 1u;
+  for (int q = w0 + lane; q - lane < w1; q += 32) {         // this warp's histogram
+    const int key = (q < w1) ? p.ids[q] : -1;
+    const unsigned m = __match_any_sync(0xffffffffu, key);
+    if (key >= 0 && (m & lt) == 0) s_base[warp][key] += __popc(m);   // one leader per key: no conflict
+    __syncwarp();
+  }
+  __syncthreads();
+  for (int e = tid; e < p.E; e += blockDim.x) {             // where each warp's pairs of expert e begin
+    int base = p.offset[e] + hist[(size_t)blockIdx.x * p.E + e];
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+      const int n = s_base[w][e];
+      s_base[w][e] = base;
+      base += n;
     }
-    int pos = run + incl - n_mine;
-    if (kk.x == e) { p.perm[pos] = q0; p.inv[q0] = pos; ++pos; }
-    if (kk.y == e) { p.perm[pos] = q0 + 1; p.inv[q0 + 1] = pos; ++pos; }
-    if (kk.z == e) { p.perm[pos] = q0 + 2; p.inv[q0 + 2] = pos; ++pos; }
-    if (kk.w == e) { p.perm[pos] = q0 + 3; p.inv[q0 + 3] = pos; ++pos; }
-    run += __shfl_sync(0xffffffffu, incl, 31);
+  }
+  __syncthreads();
+  for (int q = w0 + lane; q - lane < w1; q += 32) {
+    const int key = (q < w1) ? p.ids[q] : -1;
+    const unsigned m = __match_any_sync(0xffffffffu, key);
+    int pos = 0;
+    if (key >= 0) pos = s_base[warp][key] + __popc(m & lt);
+    __syncwarp();
+    if (key >= 0 && (m & lt) == 0) s_base[warp][key] += __popc(m);
+    __syncwarp();
+    if (key >= 0) {
+      p.perm[pos] = q;
+      p.inv[q] = pos;
+    }
   }
 }
 

@@ -79,6 +79,69 @@ def _run(shape, L, slots_per_layer, steps, T, seed, fused_every=2):
     return cross_layer_evictions
 
 
+@pytest.mark.parametrize("fill_mode", [B.FT_FILL_COPY_ENGINE, B.FT_FILL_SM])
+def test_full_layer_prefetch_ahead_of_routing(fill_mode):
+    """Double-buffered prefill: while layer l is evaluated the whole expert set of layer l+1 is admitted into the
+    shared pool (its routing still unknown); the layer's own plan then finds only hits, the victims are the least
+    recently used slots (layers already computed), and the outputs are unchanged."""
+    shape = W.LayerShape(d=256, inter=64, n_experts=8, top_k=2)
+    L, E, S, T = 4, 8, shape.expert_bytes, 12
+    pool = B.HostPool(L * E * S)
+    W.fill_pool(pool.tensor, shape, L, 61)
+    cfg = B.make_config(hidden=shape.d, inter=shape.inter, n_experts=E, top_k=2, n_layers=L, slots_per_layer=5,
+                        max_tokens=T, host_pool_ptr=pool.ptr.value, host_pool_bytes=pool.n_bytes,
+                        fill_mode=fill_mode, global_pool=1)          # 20 shared slots >= two layers of 8
+    moe = B.FtMoe(cfg)
+    cm = O.CostModel(S, cfg.bw_fill_MBps, cfg.bw_zc_residual_MBps, cfg.bw_zc_MBps, cfg.bw_hbm_MBps,
+                     cfg.reuse_credit, cfg.zc_tokens_per_pass, cfg.hbm_tokens_per_pass)
+    recs = pool.tensor.view(L, E, S).numpy()
+    ora = SharedPoolOracle(shape, L, 20, recs, cm)
+    dev = torch.device("cuda:0")
+
+    def prefetch(l):
+        flat = np.zeros(L * E, dtype=np.int32)
+        flat[l * E:(l + 1) * E] = 1                       # every expert of the layer "routed" once
+        p = O.plan(ora.state, flat, cm)
+        moe.prefetch_layer(l)
+        return p
+
+    for t in range(3):
+        p0 = prefetch(0)
+        assert t > 0 or len(p0.fill) == E
+        for l in range(L):
+            logits = W.normal_logits(T, E, 61 + l, t)
+            x = W.noise_x(T, shape.d, 61, t, l)
+            ids, w, count, offset, perm, inv, p, y_ref = ora.step(l, logits, bits(x), compute_y=True)
+            assert p.miss == []                           # everything was brought in ahead of the routing
+            lg, xd = torch.from_numpy(logits).to(dev), x.to(dev)
+            y = torch.empty_like(xd)
+            moe.route(l, lg, T)
+            plan = moe.plan(l)
+            moe.fill(l, None)
+            if l + 1 < L:
+                pn = prefetch(l + 1)                      # loads while layer l is evaluated
+                assert all(g < 0 or g // E != l for g in pn.fill_evicted)     # never the layer in use
+            moe.forward(l, xd, y)
+            assert moe.sync_status() == 0
+            assert plan["miss"] == [] and plan["hit"] == [g - l * E for g in p.hit]
+            se, ss, es = moe.get_slot_table(l)
+            assert np.array_equal(se, ora.state.slot_expert) and np.array_equal(ss, ora.state.slot_stamp)
+            check_output(y, y_ref)
+            for s_ in range(20):
+                g = int(ora.state.slot_expert[s_])
+                if g >= 0 and g // E == min(l + 1, L - 1):
+                    assert np.array_equal(moe.read_slot(0, s_), recs[g // E][g % E])
+        st = moe.get_stats(1)
+        assert st["steps"] == t + 1                       # a prefetch is not a step of the layer
+    # a pool that cannot hold two full layers refuses: the caller falls back to on-demand fills
+    moe.resize(3)
+    with pytest.raises(B.FtMoeError) as ei:
+        moe.prefetch_layer(0)
+    assert ei.value.code == B.FT_ERR_UNSUPPORTED
+    moe.destroy()
+    pool.free()
+
+
 def test_shared_pool_small_table_paths():
     """3 layers sharing 9 slots: layers evict each other's experts by the common clock."""
     ev = _run(W.LayerShape(d=256, inter=64, n_experts=8, top_k=2), L=3, slots_per_layer=3, steps=6, T=4, seed=51)
