@@ -873,7 +873,10 @@ def run_sweep(args):
     xbuf = torch.empty((L, 64, d), dtype=torch.bfloat16, device=dev)
     ybuf = torch.empty((L, 64, d), dtype=torch.bfloat16, device=dev)
     cal = None
-    for frac in (0.10, 0.25, 0.50, 0.75, 1.00):
+    fracs = [float(v) for v in args.sweep_fracs.split(",")]
+    rhos = [float(v) for v in args.sweep_rhos.split(",")]
+    batches = [int(v) for v in args.sweep_batches.split(",")]
+    for frac in fracs:
         Ns = W.slots_for_fraction(frac, E)
         common = dict(hidden=d, inter=shape.inter, n_experts=E, top_k=k, n_layers=L, slots_per_layer=Ns,
                       max_tokens=64, host_pool_ptr=pool.ptr.value, host_pool_bytes=pool.n_bytes,
@@ -884,8 +887,8 @@ def run_sweep(args):
             m0.destroy()
         moe = Bd.FtMoe(Bd.make_config(bw_fill=max(cal["fill_MBps"], 1), bw_zc=max(cal["zc_MBps"], 1),
                                       bw_zc_residual=0, bw_hbm=max(cal["hbm_MBps"], 1), **common))
-        for rho in (0.0, 0.5, 0.9):
-            for batch in (1, 16, 64):
+        for rho in rhos:
+            for batch in batches:
                 lg = torch.from_numpy(W.ar1_logits(L, steps, batch, E, rho, ALPHA, SEED)).to(dev)
                 g = torch.Generator(device=dev)
                 g.manual_seed(W.mix64(SEED, 79, batch))
@@ -912,7 +915,8 @@ def run_sweep(args):
                       "hit_rate_pairs": st["pairs_resident"] / max(st["pairs"], 1),
                       "fills": st["fills"], "zero_copies": st["zc"], "evictions": st["evictions"],
                       "fill_bytes": st["fills"] * S, "zero_copy_bytes": st["zc"] * S,
-                      "routed_unique_per_layer_step": st["routed"] / (steps * L)}
+                      "routed_unique_per_layer_step": st["routed"] / (steps * L),
+                      "resident_record_GBps": (st["hits"] + st["fills"]) * S / (ms * 1e-3) / 1e9}
                 points.append(pt)
                 log(f"sweep {pt}")
         moe.destroy()
@@ -928,6 +932,9 @@ def run_sweep(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--sweep-steps", type=int, default=128)
+    ap.add_argument("--sweep-fracs", default="0.10,0.25,0.50,0.75,1.00")
+    ap.add_argument("--sweep-rhos", default="0,0.5,0.9")
+    ap.add_argument("--sweep-batches", default="1,16,64")
     ap.add_argument("--global-pool", type=int, default=0, help="1: one slot pool and LRU clock shared by all layers")
     ap.add_argument("--graph", type=int, default=1, help="replay each decode step as one CUDA graph (SM fill only)")
     ap.add_argument("--workload", default="qwen", choices=["qwen", "dsv3"])

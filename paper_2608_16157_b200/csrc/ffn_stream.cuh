@@ -66,6 +66,20 @@ __device__ __forceinline__ void red_add_f32(float *addr, float v) {
   asm volatile("red.global.add.f32 [%0], %1;" ::"l"(addr), "f"(v) : "memory");
 }
 
+// y = bf16(y_acc), y_acc = 0 over the whole grid: the output rounding of calls with many tokens, where one CTA (the
+// last one of the streaming kernel) would take longer than a launch of its own.
+static __global__ void __launch_bounds__(256) finalize_kernel(float *y_acc, __nv_bfloat16 *y, int n4) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += gridDim.x * blockDim.x) {
+    const float4 v = __ldcg(reinterpret_cast<const float4 *>(y_acc) + i);
+    __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+    uint2 o;
+    o.x = *reinterpret_cast<uint32_t *>(&a);
+    o.y = *reinterpret_cast<uint32_t *>(&b);
+    reinterpret_cast<uint2 *>(y)[i] = o;
+    reinterpret_cast<float4 *>(y_acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+}
+
 template <int DB>  // DB = d / 256
 __global__ void __launch_bounds__(kFsThreads, 1) ffn_stream_kernel(FfnStreamParams p) {
   constexpr int KT = (DB >= 2) ? DB / 2 : 1;   // 16 x 32 gate/up tiles per active warp

@@ -21,6 +21,7 @@ using namespace ftmoe;
 namespace {
 
 enum LayerPhase { PH_IDLE = 0, PH_ROUTED, PH_PLANNED, PH_FILLED };
+constexpr int kFinalizeInKernelMaxTokens = 16;
 constexpr int kMaxTableSlots = 6144;   // slots of one residency table (per layer, or the shared pool)
 
 struct LayerState {
@@ -932,13 +933,25 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     // overlaps the fills; the filled experts follow once the fill event has fired.  With few tokens the extra
     // launch costs more than the overlap buys, so everything goes in one launch after the fills.
     const bool split = c.slots_per_layer > 0 && (long long)L.T * c.top_k >= c.split_min_pairs && c.split_min_pairs > 0;
+    // the last CTA of the last launch rounds y itself unless the call has so many tokens that a launch of its own,
+    // spread over the whole GPU, is quicker (or the GEMM path's combine does it)
+    const bool own_finalize = !use_gemm && L.T > kFinalizeInKernelMaxTokens;
+    const int fin = (use_gemm || own_finalize) ? 0 : 1;
     if (split) {
       launch(1, 0);
       if (L.fill_recorded) FT_CUDA(cudaStreamWaitEvent(st, L.ev_fill, 0));
-      launch(2, use_gemm ? 0 : 1);
+      launch(2, fin);
     } else {
       if (c.slots_per_layer > 0 && L.fill_recorded) FT_CUDA(cudaStreamWaitEvent(st, L.ev_fill, 0));
-      launch(0, use_gemm ? 0 : 1);
+      launch(0, fin);
+    }
+    if (own_finalize) {
+      TimeScope ts(h, st, FT_TIME_FINALIZE);
+      const int n4 = L.T * (c.hidden / 4);
+      int grid = (n4 + 255) / 256;
+      if (grid > h->sm_count * 4) grid = h->sm_count * 4;
+      finalize_kernel<<<grid, 256, 0, st>>>(h->y_acc, static_cast<__nv_bfloat16 *>(y_dev), n4);
+      h->launches++;
     }
     FT_CUDA(launch_err);
     FT_CUDA(cudaGetLastError());
