@@ -247,13 +247,18 @@ def unpack_record(rec: np.ndarray, d: int, inter: int, wdtype: str):
       W_gate[i][n] at 48*d*(n//16) + 512*(i//32) + 256*((n%16)//8) + 32*r + 8*(((i%32)//8) ^ (r>>1)) + i%8
       W_up[i][n]   at the same place + 16*d
       W_down[n][c] at 48*d*(n//16) + 32*d + 256*(c//16) + 128*((c%16)//8) + 16*r + 8*(((n%16)//8) ^ (r>>2)) + n%8
-    int4 record: 4-bit two's-complement codes, then bf16 scales sg[I][d/128], su[I][d/128]
-    (groups along the hidden index) and sd[I/128][d] (groups along the neuron index);
-    weight = scale * code.  Gate and up codes are row-major [I][d/2] bytes, two per byte along
-    d (low nibble = even column).  Down codes are stored in fragment order: 16-neuron blocks x
-    16-column tiles x 32 little-endian 32-bit words; in word l = 4g + q of block b, tile ct,
-    nibble j is the code of neuron 16b + NN[j] + q, column 16ct + CC[j] + g, with
-    NN = (0,8,0,8,4,12,4,12) and CC = (0,0,8,8,0,0,8,8).
+    int4 record: 4-bit two's-complement codes and bf16 scales, weight = scale * code, groups of 128 along the
+    contraction dimension; G = d/128, NG = I/128, UA = 2112*G bytes per 16-neuron unit of section A,
+    NWD = min(16, d/64), CBW = 64*NWD, CB = d/CBW.  Byte addresses (the code is the low nibble when `lo`):
+      gate code of (neuron n, hidden i): UA*(n//16) + 1024*(i//128) + 64*(n%16) + 16*((i%32)//8) + 4*((i%128)//32)
+                                         + (i%8)//2,  lo = i even;      up: the same + 1024*G
+      gate scale of (n, group i//128):   UA*(n//16) + 2048*G + 32*(i//128) + 4*(n%8) + 2*((n%16)//8);  up: + 32*G
+      down code of (neuron n, column c): with ng = n//128, uu = (n%128)//16, q = (n%16)//4, r = n%4, g = c%8,
+                                         half = (c%16)//8, cb = c//CBW, t = (c%CBW)//16, w = t//4, j = t%4,
+                                         e = half + 2*(r//2) + 4*(r%2):
+                                         UA*I/16 + ((((cb*NG + ng)*8 + uu)*NWD + w)*32 + 4*g + q)*16 + 4*j + e//2,
+                                         lo = e even
+      down scale of (group ng, column c): UA*I/16 + I*d/2 + ((ng*CB + cb)*NWD + w)*128 + 16*g + 4*j + 2*half
     """
     rec = np.ascontiguousarray(rec).view(np.uint8).reshape(-1)
     n = inter * d
@@ -270,42 +275,39 @@ def unpack_record(rec: np.ndarray, d: int, inter: int, wdtype: str):
             + 8 * (((n % 16) // 8) ^ ((c % 8) >> 2)) + n % 8
         return el[at_gate], el[at_gate + 16 * d], el[at_down]
     if wdtype == "int4":
-        nb = n // 2
-        codes = []
-        for which in range(2):
-            b = rec[which * nb:(which + 1) * nb].reshape(inter, d // 2)
-            lo = (b & 0xF).astype(np.int16)
-            hi = (b >> 4).astype(np.int16)
-            q = np.empty((inter, d), dtype=np.int16)
-            q[:, 0::2] = lo
-            q[:, 1::2] = hi
-            q = np.where(q >= 8, q - 16, q)
-            codes.append(q.astype(np.float64))
-        # down: walk the fragment-order words
-        words = rec[2 * nb:3 * nb].view("<u4").reshape(inter // 16, d // 16, 32)
-        qd = np.zeros((inter, d), dtype=np.int16)
-        NN, CC = (0, 8, 0, 8, 4, 12, 4, 12), (0, 0, 8, 8, 0, 0, 8, 8)
-        for l in range(32):
-            g_, q_ = l // 4, l % 4
-            for j in range(8):
-                nib = ((words[:, :, l] >> np.uint32(4 * j)) & np.uint32(0xF)).astype(np.int16)
-                qd[NN[j] + q_::16, CC[j] + g_::16] = nib
-        qd = np.where(qd >= 8, qd - 16, qd)
-        codes.append(qd.astype(np.float64))
-        off = 3 * nb
-        ng = inter * (d // GROUP)
-        sg = _bf16_bits_to_f64(rec[off:off + 2 * ng].view(np.uint16)).reshape(inter, d // GROUP)
-        off += 2 * ng
-        su = _bf16_bits_to_f64(rec[off:off + 2 * ng].view(np.uint16)).reshape(inter, d // GROUP)
-        off += 2 * ng
-        nd = (inter // GROUP) * d
-        sd = _bf16_bits_to_f64(rec[off:off + 2 * nd].view(np.uint16)).reshape(inter // GROUP, d)
-        off += 2 * nd
-        assert off == rec.size
-        wg = codes[0] * np.repeat(sg, GROUP, axis=1)
-        wu = codes[1] * np.repeat(su, GROUP, axis=1)
-        wd = codes[2] * np.repeat(sd, GROUP, axis=0)
-        return wg.T.copy(), wu.T.copy(), wd
+        G, NG, U = d // GROUP, inter // GROUP, inter // 16
+        UA = 2112 * G
+        nwd = min(16, d // 64)
+        cbw = 64 * nwd
+        CB = d // cbw
+        assert rec.size == U * UA + inter * d // 2 + NG * d * 2
+
+        def codes(addr, lo):
+            b = rec[addr].astype(np.int16)
+            q = np.where(lo, b & 0xF, b >> 4)
+            return np.where(q >= 8, q - 16, q).astype(np.float64)
+
+        def bf16_at(addr):
+            return _bf16_bits_to_f64(rec[addr].astype(np.uint16) | (rec[addr + 1].astype(np.uint16) << 8))
+
+        i = np.arange(d, dtype=np.int64)[:, None]          # hidden index along axis 0 (gate/up are returned [d, I])
+        nn = np.arange(inter, dtype=np.int64)[None, :]
+        a_gate = UA * (nn // 16) + 1024 * (i // 128) + 64 * (nn % 16) + 16 * ((i % 32) // 8) + 4 * ((i % 128) // 32) \
+            + (i % 8) // 2
+        s_gate = UA * (nn // 16) + 2048 * G + 32 * (i // 128) + 4 * (nn % 8) + 2 * ((nn % 16) // 8)
+        lo = (i % 2 == 0) & (nn >= 0)
+        wg = codes(a_gate, lo) * bf16_at(s_gate)
+        wu = codes(a_gate + 1024 * G, lo) * bf16_at(s_gate + 32 * G)
+        n = np.arange(inter, dtype=np.int64)[:, None]      # down is returned [I, d]
+        c = np.arange(d, dtype=np.int64)[None, :]
+        ng, uu, q, r = n // 128, (n % 128) // 16, (n % 16) // 4, n % 4
+        g, half, cb, t = c % 8, (c % 16) // 8, c // cbw, (c % cbw) // 16
+        w, j = t // 4, t % 4
+        e = half + 2 * (r // 2) + 4 * (r % 2)
+        a_down = UA * U + ((((cb * NG + ng) * 8 + uu) * nwd + w) * 32 + 4 * g + q) * 16 + 4 * j + e // 2
+        s_down = UA * U + inter * d // 2 + ((ng * CB + cb) * nwd + w) * 128 + 16 * g + 4 * j + 2 * half
+        wd = codes(a_down, e % 2 == 0) * bf16_at(s_down + 0 * n)
+        return wg, wu, wd
     raise ValueError(wdtype)
 
 

@@ -19,17 +19,20 @@ flattened identifier of Sec. 4.2 of the paper):
           ``c // 16``; two groups of 8 column rows of 32 bytes (group ``(c % 16) // 8``,
           row ``r = c % 8``); the two 16-byte chunks of a row are stored at position
           ``((n % 16) // 8) ^ (r >> 2)``.  ``S = 3*I*d*2`` bytes.
-``int4``  4-bit two's-complement codes in [-8, 7] for the same three matrices,
-          then bf16 scales.  ``Wg_q`` and ``Wu_q`` are row-major ``[I][d/2]`` bytes,
-          two codes per byte along ``d`` (low nibble = even column).  ``Wd_q`` is
-          stored in tensor-core fragment order: blocks of 16 neurons x tiles of 16
-          columns x 32 little-endian 32-bit words; word ``l = 4*g + q`` of block
-          ``b``, tile ``ct`` holds in nibble ``j`` (bits ``4j..4j+3``) the code of
-          neuron ``16b + NN[j] + q`` and column ``16ct + CC[j] + g`` with
-          ``NN = (0, 8, 0, 8, 4, 12, 4, 12)`` and ``CC = (0, 0, 8, 8, 0, 0, 8, 8)``.
-          Scales: ``sg[I][d/128]``, ``su[I][d/128]`` (groups of 128 consecutive
-          ``i``: the contraction dimension of gate/up) and ``sd[I/128][d]``
-          (groups of 128 consecutive ``n``: the contraction dimension of down).
+``int4``  4-bit two's-complement codes in [-8, 7] and bf16 scales, weight = scale * code, groups of
+          128 along the contraction dimension (``G = d/128`` hidden groups for gate/up, ``NG = I/128``
+          neuron groups for down), in tensor-core tile order.  Three sections:
+          A. ``I/16`` units of 16 neurons, ``2112*G`` bytes each: gate tiles, up tiles, gate scales, up
+             scales.  A tile is 16 neuron rows x 128 hidden indices = 16 rows of 64 bytes; in a row the
+             code of hidden index ``128*grp + 32*j + 8*q + e`` is nibble ``e`` (low nibble = even ``e``) of
+             the little-endian 32-bit word ``j`` of the 16-byte chunk ``q``.  The scales of a tile are 8
+             pairs ``(row r, row r+8)`` of bf16.
+          B. down codes: for each column block ``cb`` (``CBW = 64*min(16, d/64)`` columns), neuron group
+             ``ng`` and 16-neuron step ``uu`` of the group: ``CBW/64`` x 512 bytes; in each 512 bytes lane
+             ``l = 4g + q`` owns 16 bytes = 4 words, word ``j`` belongs to the 16-column tile ``4w + j`` of the
+             block; its nibble ``e`` is the code of column ``g + 8*(e & 1)`` of the tile and neuron
+             ``4q + NU[e]`` of the step, ``NU = (0, 0, 2, 2, 1, 1, 3, 3)``.
+          C. down scales ``sd[ng][column]`` in the order (ng, cb, w, g, j, half): 8 pairs per tile again.
           ``S = 3*I*d/2 + (2*I*d/128 + (I/128)*d)*2``.
 
 The routing-logit recipes follow the workload descriptions: a Zipf-style
@@ -132,27 +135,43 @@ def _quantise_int4(w: torch.Tensor, group_axis: int) -> tuple[torch.Tensor, torc
 
 
 def _pack_nibbles(q: torch.Tensor) -> torch.Tensor:
-    """int8 codes ``[..., d]`` -> uint8 ``[..., d/2]``, low nibble = even column."""
+    """int8 codes ``[..., n]`` -> uint8 ``[..., n/2]``, low nibble = even index."""
     u = (q.to(torch.int16) & 0xF).to(torch.uint8)
     return u[..., 0::2] | (u[..., 1::2] << 4)
 
 
-WD_NN = (0, 8, 0, 8, 4, 12, 4, 12)   # neuron offset (plus q) of nibble j in a fragment-order word
-WD_CC = (0, 0, 8, 8, 0, 0, 8, 8)     # column offset (plus g) of nibble j
+WD_NU = (0, 0, 2, 2, 1, 1, 3, 3)     # neuron offset (plus 4q) of nibble e in a word of the down section
 
 
-def _pack_wd_fragment_order(q: torch.Tensor) -> torch.Tensor:
-    """int8 codes ``[I][d]`` of W_down -> uint8 bytes of the fragment-order layout."""
-    I, d = q.shape
-    blocks = q.reshape(I // 16, 16, d // 16, 16)                     # [b][nn][ct][cc]
-    l = torch.arange(32, device=q.device)
-    g, qq = l // 4, l % 4
-    nn = torch.tensor(WD_NN, device=q.device)[None, :] + qq[:, None]   # [32][8]
-    cc = torch.tensor(WD_CC, device=q.device)[None, :] + g[:, None]    # [32][8]
-    nib = blocks.permute(0, 2, 1, 3)[:, :, nn, cc]                    # [b][ct][32][8]
-    u = (nib.to(torch.int16) & 0xF).to(torch.uint8)
-    by = u[..., 0::2] | (u[..., 1::2] << 4)                            # [b][ct][32][4] bytes, little endian
-    return by.reshape(-1)
+def _pack_int4_record(qg, qu, qd, sg, su, sd) -> torch.Tensor:
+    """Codes int8 ``[I][d]`` (gate/up: one row per neuron; down: ``[n][c]``), scales bf16 ``sg, su [I][d/128]``,
+    ``sd [I/128][d]`` -> the tiled record, uint8 flat."""
+    I, d = qg.shape
+    dev = qg.device
+    U, G, NG = I // 16, d // GROUP, I // GROUP
+    nwd = min(16, d // 64)
+    cbw = 64 * nwd
+    CB = d // cbw
+
+    def gu_tiles(q):      # [U][16 rows][G][j][q][e] -> [U][G][row][q][j][e], nibbles packed along e
+        t = q.reshape(U, 16, G, 4, 4, 8).permute(0, 2, 1, 4, 3, 5)
+        return _pack_nibbles(t).reshape(U, G * 1024)
+
+    def gu_scales(s_):    # [U][half][r][G] -> [U][G][r][half]
+        t = s_.reshape(U, 2, 8, G).permute(0, 3, 2, 1).contiguous()
+        return t.view(torch.uint8).reshape(U, G * 32)
+
+    sec_a = torch.cat([gu_tiles(qg), gu_tiles(qu), gu_scales(sg), gu_scales(su)], dim=1).reshape(-1)
+    # section B: gather the code of every nibble position
+    ar = lambda n: torch.arange(n, device=dev)
+    cb, ng, uu, w, g, q, j, e = torch.meshgrid(ar(CB), ar(NG), ar(8), ar(nwd), ar(8), ar(4), ar(4), ar(8), indexing="ij")
+    nu = torch.tensor(WD_NU, device=dev)[e]
+    n_idx = 128 * ng + 16 * uu + 4 * q + nu
+    c_idx = cb * cbw + (4 * w + j) * 16 + g + 8 * (e & 1)
+    sec_b = _pack_nibbles(qd[n_idx, c_idx]).reshape(-1)
+    ng2, cb2, w2, g2, j2, half = torch.meshgrid(ar(NG), ar(CB), ar(nwd), ar(8), ar(4), ar(2), indexing="ij")
+    sec_c = sd[ng2, cb2 * cbw + (4 * w2 + j2) * 16 + g2 + 8 * half].contiguous().view(torch.uint8).reshape(-1)
+    return torch.cat([sec_a, sec_b, sec_c])
 
 
 def _pack_bf16_tiles(w: torch.Tensor) -> torch.Tensor:
@@ -191,11 +210,7 @@ def make_records(shape: LayerShape, seed: int, layer: int, first: int, count: in
             qg, sg = _quantise_int4(w[0:1], 2)
             qu, su = _quantise_int4(w[1:2], 2)
             qd, sd = _quantise_int4(w[2:3], 1)
-            parts = [_pack_nibbles(qg).reshape(-1), _pack_nibbles(qu).reshape(-1),
-                     _pack_wd_fragment_order(qd[0]),
-                     sg.reshape(-1).view(torch.uint8), su.reshape(-1).view(torch.uint8),
-                     sd.reshape(-1).view(torch.uint8)]
-            out[j] = torch.cat(parts)
+            out[j] = _pack_int4_record(qg[0], qu[0], qd[0], sg[0], su[0], sd[0])
     return out
 
 

@@ -47,26 +47,49 @@ def test_unpack_bf16_record_orientation():
 
 
 def _record_int4_by_definition(qg, qu, qd, sg, su, sd):
-    """qX: int codes [I][d] (row = neuron); sg/su [I][d/128]; sd [I/128][d] (floats, bf16-exact).
-    Gate/up: two codes per byte along d, low nibble = even column.  Down: fragment order, written
-    word by word from the documented nibble table."""
+    """qX: int codes [I][d] (row = neuron); sg/su [I][d/128]; sd [I/128][d] (floats, bf16-exact).  Written section
+    by section, word by word, from the documented tile order."""
     I, d = qg.shape
+    G, NG, U = d // 128, I // 128, I // 16
+    nwd = min(16, d // 64)
+    cbw, CB = 64 * nwd, d // (64 * nwd)
+    NU = (0, 0, 2, 2, 1, 1, 3, 3)
     out = bytearray()
-    for q in (qg, qu):
-        for n in range(I):
-            for c in range(0, d, 2):
-                out.append((int(q[n, c]) & 0xF) | ((int(q[n, c + 1]) & 0xF) << 4))
-    NN, CC = (0, 8, 0, 8, 4, 12, 4, 12), (0, 0, 8, 8, 0, 0, 8, 8)
-    for b in range(I // 16):
-        for ct in range(d // 16):
-            for l in range(32):
-                g, q_ = divmod(l, 4)
-                word = 0
-                for j in range(8):
-                    word |= (int(qd[16 * b + NN[j] + q_, 16 * ct + CC[j] + g]) & 0xF) << (4 * j)
-                out += word.to_bytes(4, "little")
-    for s in (sg, su, sd):
-        out += _bf16_bits(s).tobytes()
+
+    def word(nibbles):
+        v = 0
+        for e, c in enumerate(nibbles):
+            v |= (int(c) & 0xF) << (4 * e)
+        return v.to_bytes(4, "little")
+
+    for u in range(U):                                   # section A: units of 16 neurons
+        for q_ in (qg, qu):
+            for grp in range(G):                          # a tile: 16 rows of 64 bytes = 4 chunks of 4 words
+                for row in range(16):
+                    for chunk in range(4):
+                        for j in range(4):
+                            i0 = 128 * grp + 32 * j + 8 * chunk
+                            out += word(q_[16 * u + row, i0:i0 + 8])
+        for s_ in (sg, su):
+            for grp in range(G):
+                for r in range(8):                        # pairs (row r, row r + 8)
+                    out += _bf16_bits(np.array([s_[16 * u + r, grp], s_[16 * u + r + 8, grp]])).tobytes()
+    for cb in range(CB):                                  # section B: down codes
+        for ng in range(NG):
+            for uu in range(8):
+                for w in range(nwd):
+                    for lane in range(32):
+                        g, q = divmod(lane, 4)
+                        for j in range(4):
+                            col0 = cb * cbw + (4 * w + j) * 16
+                            out += word([qd[128 * ng + 16 * uu + 4 * q + NU[e], col0 + g + 8 * (e & 1)] for e in range(8)])
+    for ng in range(NG):                                  # section C: down scales
+        for cb in range(CB):
+            for w in range(nwd):
+                for g in range(8):
+                    for j in range(4):
+                        col0 = cb * cbw + (4 * w + j) * 16
+                        out += _bf16_bits(np.array([sd[ng, col0 + g], sd[ng, col0 + g + 8]])).tobytes()
     return np.frombuffer(bytes(out), dtype=np.uint8)
 
 
@@ -80,11 +103,9 @@ def test_unpack_int4_record_by_definition():
     rec = _record_int4_by_definition(qg, qu, qd, sg, su, sd)
     assert rec.size == W.LayerShape(d, I, 1, 1, "int4").expert_bytes
     wg, wu, wd = O.unpack_record(rec, d, I, "int4")
-    for n in (0, 5, 127):
-        for i in (0, 1, 127, 128, 255):
-            assert wg[i, n] == qg[n, i] * sg[n, i // 128]
-            assert wu[i, n] == qu[n, i] * su[n, i // 128]
-            assert wd[n, i] == qd[n, i] * sd[n // 128, i]
+    assert np.array_equal(wg, (qg * np.repeat(sg, 128, axis=1)).T)
+    assert np.array_equal(wu, (qu * np.repeat(su, 128, axis=1)).T)
+    assert np.array_equal(wd, qd * np.repeat(sd, 128, axis=0))
     # all-zero codes give zero weights; code 1 with scale 1 gives column sums of x
     z = np.zeros((I, d), dtype=np.int64)
     one = np.ones((I, d), dtype=np.int64)
