@@ -287,8 +287,8 @@ ft_status_t ft_moe_set_launch_overlap(ft_moe_t *h, int mode);
  * call that timed out is unspecified; ft_moe_sync_status reports FT_ERR_TIMEOUT once, and after ft_moe_reset
  * the handle works as before.  Waits for the device. */
 enum { FT_DEBUG_WITHHOLD_FILL = 1,      /* device-driven fill kernel (FT_FILL_SM) */
-       FT_DEBUG_WITHHOLD_Q4 = 2,        /* int4 gate/up streaming kernel */
        FT_DEBUG_WITHHOLD_GEMM = 4 };    /* prefill gate/up grouped GEMM */
+/* (The bf16 and int4 streaming kernels load weights straight into registers and contain no waits.) */
 ft_status_t ft_moe_debug_inject(ft_moe_t *h, uint32_t withhold_mask, uint32_t wait_polls);
 /* Number of kernels this handle has launched since create. */
 ft_status_t ft_moe_launch_count(ft_moe_t *h, uint64_t *out);

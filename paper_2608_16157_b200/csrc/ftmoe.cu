@@ -10,7 +10,7 @@
 
 #include "common.cuh"
 #include "ffn_stream.cuh"
-#include "ffn_q4.cuh"
+#include "ffn_w4.cuh"
 #include "gemm_tc.cuh"
 #include "gemm_tc2.cuh"
 #include "fill.cuh"
@@ -88,7 +88,7 @@ struct ft_moe {
   uint32_t *seq_dev = nullptr;
   uint32_t *done_dev = nullptr;          // CTA completion counter of the streaming MMA kernel
   long long *trace_dev = nullptr;        // per-CTA clocks of the latest streaming-kernel launch
-  uint2 *q4_hbuf = nullptr;              // int4 path: h of every (pass, 16-neuron block) in fragment order
+  __nv_bfloat16 *w4_hbuf = nullptr;      // int4 path: h as [pass][16-neuron unit][token 8][neuron 16]
   int last_fill_layer = -1;
   int overlap = 0;                      // launch mode of the streaming kernel (see FfnStreamParams::overlap)
   float *stage_logits = nullptr;
@@ -153,14 +153,14 @@ size_t expert_bytes_of(const ft_moe_config_t *c) {
     return 3 * I * d * 2;
   }
   if (c->wdtype == FT_W_INT4_G128) {
-    if (d % 512 || d > 8192 || I % 128) return 0;   // (the kernels further restrict d, see q4_shape_ok)
+    if (d % 512 || d > 8192 || I % 128) return 0;   // (the kernels further restrict d, see w4_shape_ok)
     return 3 * I * d / 2 + (2 * I * (d / 128) + (I / 128) * d) * 2;
   }
   return 0;
 }
 
 // shapes the int4 kernels are instantiated for
-bool q4_shape_ok(const ft_moe_config_t &c) {
+bool w4_shape_ok(const ft_moe_config_t &c) {
   const int d = c.hidden;
   return (d == 512 || d == 1024 || d == 2048 || d == 4096 || d == 7168 || d == 8192) && c.inter % 128 == 0;
 }
@@ -426,7 +426,7 @@ ft_status_t ft_moe_destroy(ft_moe_t *h) {
   cudaFree(h->status_dev);
   cudaFree(h->seq_dev);
   cudaFree(h->done_dev);
-  cudaFree(h->q4_hbuf);
+  cudaFree(h->w4_hbuf);
   cudaFree(h->trace_dev);
   cudaFree(h->stage_logits);
   cudaFree(h->stage_x);
@@ -462,7 +462,7 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
       c.zc_tokens_per_pass < 1 || c.hbm_tokens_per_pass < 1 || c.gemm_min_tokens < 0 || c.split_min_pairs < 0)
     return FT_ERR_INVALID_ARG;
   const size_t S = expert_bytes_of(cfg);
-  if (S == 0 || (c.wdtype == FT_W_INT4_G128 && !q4_shape_ok(c))) return FT_ERR_UNSUPPORTED;
+  if (S == 0 || (c.wdtype == FT_W_INT4_G128 && !w4_shape_ok(c))) return FT_ERR_UNSUPPORTED;
   if (c.gemm_min_tokens != 0 &&
       (c.wdtype != FT_W_BF16 || c.slots_per_layer == 0 || c.hidden % 256 || c.inter % 256 || c.gemm_min_tokens < 8))
     return FT_ERR_UNSUPPORTED;
@@ -586,19 +586,19 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
   FT_TRY(cudaFuncSetAttribute(fill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFillStages * (int)kFillChunk));
   if (c.wdtype == FT_W_INT4_G128) {
     const size_t passes = (P + 7) / 8 + 2 * E + 2;
-    FT_TRY(cudaMalloc(&h->q4_hbuf, passes * (c.inter / 16) * 32 * sizeof(uint2)));
-    const int sa = (int)q4_gateup_smem_bytes(8192), sb = (int)q4_down_smem_bytes(8192);   // largest hidden size
-    FT_TRY(cudaFuncSetAttribute(q4_gateup_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
-    FT_TRY(cudaFuncSetAttribute(q4_gateup_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
-    FT_TRY(cudaFuncSetAttribute(q4_gateup_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
-    FT_TRY(cudaFuncSetAttribute(q4_gateup_kernel<7>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
-    FT_TRY(cudaFuncSetAttribute(q4_gateup_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
-    FT_TRY(cudaFuncSetAttribute(q4_down_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
-    FT_TRY(cudaFuncSetAttribute(q4_down_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
-    FT_TRY(cudaFuncSetAttribute(q4_down_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
-    FT_TRY(cudaFuncSetAttribute(q4_down_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
-    FT_TRY(cudaFuncSetAttribute(q4_down_kernel<14>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
-    FT_TRY(cudaFuncSetAttribute(q4_down_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
+    FT_TRY(cudaMalloc(&h->w4_hbuf, passes * (c.inter / 16) * 256));
+    // (limits are per function and device, not per handle: always the largest a CTA can have, and the handle's own
+    // need is checked against it)
+    const int sa = 232448, sb = (int)w4_down_smem_bytes(2 * kMaxExperts + 1);
+    if (w4_gateup_smem_bytes(2 * c.n_experts + 1, c.hidden) > (size_t)sa) return fail(FT_ERR_UNSUPPORTED);
+    FT_TRY(cudaFuncSetAttribute(w4_gateup_kernel<1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(w4_gateup_kernel<1, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(w4_gateup_kernel<1, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(w4_gateup_kernel<2, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(w4_gateup_kernel<4, 14>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(w4_gateup_kernel<4, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(w4_down_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
+    FT_TRY(cudaFuncSetAttribute(w4_down_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
   }
   if (c.wdtype == FT_W_BF16) {
     // the limit is a property of the function on this device, not of the handle: always the largest size any
@@ -1002,39 +1002,40 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   }
   // int4: gate/up kernel writes h, down kernel accumulates, its last CTA finalizes y
   if (c.slots_per_layer > 0 && L.fill_recorded) FT_CUDA(cudaStreamWaitEvent(st, L.ev_fill, 0));
-  Q4Params qp;
+  W4Params qp;
   qp.items = sc.items_res;
   qp.n_items = &sc.plan_dev->n_res_items;
   qp.n_zc = &sc.plan_dev->n_zc_items;
   qp.pref = sc.res_pref;
   qp.max_items = 2 * c.n_experts + 1;
   qp.x = x_bf; qp.perm = sc.perm; qp.topk_w = sc.topk_w;
-  qp.hbuf = h->q4_hbuf;
+  qp.hbuf = h->w4_hbuf;
   qp.y_acc = h->y_acc; qp.y = static_cast<__nv_bfloat16 *>(y_dev);
   qp.done = h->done_dev; qp.status = h->status_dev;
-  qp.d = c.hidden; qp.inter = c.inter; qp.top_k = c.top_k; qp.T = L.T; qp.finalize = 1;
-  const size_t sa = q4_gateup_smem_bytes(c.hidden), sb = q4_down_smem_bytes(c.hidden);
-  const int grid = h->sm_count & ~3;   // groups of four CTAs split the columns in the down kernel
+  qp.inter = c.inter; qp.top_k = c.top_k; qp.T = L.T;
+  const bool own_finalize = L.T > kFinalizeInKernelMaxTokens;
+  qp.finalize = own_finalize ? 0 : 1;
+  const size_t sa = w4_gateup_smem_bytes(qp.max_items, c.hidden), sb = w4_down_smem_bytes(qp.max_items);
+  const int grid = h->sm_count;
   {
     TimeScope ts(h, st, FT_TIME_FFN_ZC);   // (timing slot reused for the gate/up kernel of the int4 path)
     switch (c.hidden) {
-      case 512: q4_gateup_kernel<1><<<grid, kQ4Threads, sa, st>>>(qp); break;
-      case 1024: q4_gateup_kernel<1><<<grid, kQ4Threads, sa, st>>>(qp); break;
-      case 2048: q4_gateup_kernel<2><<<grid, kQ4Threads, sa, st>>>(qp); break;
-      case 4096: q4_gateup_kernel<4><<<grid, kQ4Threads, sa, st>>>(qp); break;
-      case 7168: q4_gateup_kernel<7><<<grid, kQ4Threads, sa, st>>>(qp); break;
-      default: q4_gateup_kernel<8><<<grid, kQ4Threads, sa, st>>>(qp); break;
+      case 512: w4_gateup_kernel<1, 4><<<grid, kW4Threads, sa, st>>>(qp); break;
+      case 1024: w4_gateup_kernel<1, 8><<<grid, kW4Threads, sa, st>>>(qp); break;
+      case 2048: w4_gateup_kernel<1, 16><<<grid, kW4Threads, sa, st>>>(qp); break;
+      case 4096: w4_gateup_kernel<2, 16><<<grid, kW4Threads, sa, st>>>(qp); break;
+      case 7168: w4_gateup_kernel<4, 14><<<grid, kW4Threads, sa, st>>>(qp); break;
+      default: w4_gateup_kernel<4, 16><<<grid, kW4Threads, sa, st>>>(qp); break;
     }
   }
   {
     TimeScope ts(h, st, FT_TIME_FFN_RES);
-    switch (c.hidden) {
-      case 512: q4_down_kernel<1><<<grid, kQ4Threads, sb, st>>>(qp); break;
-      case 1024: q4_down_kernel<2><<<grid, kQ4Threads, sb, st>>>(qp); break;
-      case 2048: q4_down_kernel<4><<<grid, kQ4Threads, sb, st>>>(qp); break;
-      case 4096: q4_down_kernel<8><<<grid, kQ4Threads, sb, st>>>(qp); break;
-      case 7168: q4_down_kernel<14><<<grid, kQ4Threads, sb, st>>>(qp); break;
-      default: q4_down_kernel<16><<<grid, kQ4Threads, sb, st>>>(qp); break;
+    if (c.hidden == 512) w4_down_kernel<8><<<grid, kW4Threads, sb, st>>>(qp, c.hidden);
+    else w4_down_kernel<16><<<grid, kW4Threads, sb, st>>>(qp, c.hidden);
+    if (own_finalize) {
+      const int n4 = L.T * (c.hidden / 4);
+      finalize_kernel<<<std::min((n4 + 255) / 256, h->sm_count * 8), 256, 0, st>>>(h->y_acc, qp.y, n4);
+      h->launches++;
     }
   }
   h->launches += 2;

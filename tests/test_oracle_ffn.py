@@ -93,9 +93,9 @@ def _record_int4_by_definition(qg, qu, qd, sg, su, sd):
     return np.frombuffer(bytes(out), dtype=np.uint8)
 
 
-def test_unpack_int4_record_by_definition():
+@pytest.mark.parametrize("d,I", [(256, 128), (2048, 256)])      # one / two column blocks, one / two neuron groups
+def test_unpack_int4_record_by_definition(d, I):
     rng = np.random.default_rng(0)
-    d, I = 256, 128
     qg, qu, qd = (rng.integers(-8, 8, size=(I, d)) for _ in range(3))
     sg = rng.integers(1, 9, size=(I, d // 128)).astype(np.float32) / 64.0
     su = rng.integers(1, 9, size=(I, d // 128)).astype(np.float32) / 32.0
