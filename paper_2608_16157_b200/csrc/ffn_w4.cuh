@@ -8,18 +8,20 @@
 // instructions.  The constant is removed in fp32: sum (136 + c) a = 136 sum a + sum c a, with the sums of the
 // activations over a group computed once; the group scale multiplies the fp32 partial sum once per group.  Weights
 // and activations are bf16 operands, so the activation range is that of bf16.
-//   w4_gateup_kernel : one persistent CTA of 16 warps per SM walks 16-neuron units (gate tiles, up tiles and their
-//                      scales, contiguous).  Warp w owns GW quantisation groups of the hidden dimension; a lane's two
-//                      16-byte loads per group are rows g and g+8 of the group's tile.  Partial [16 x 8] sums are
-//                      reduced across warps through (double-buffered) shared memory: one barrier per unit.
-//                      h = SiLU(g) * u goes to a small global buffer, bf16 [pass][unit][token][neuron].
+//   w4_gateup_kernel : 16 warps per SM, every warp streams whole 16-neuron units (gate tiles, up tiles and their
+//                      scales: contiguous) by itself: no partial sums to exchange, no block-level synchronisation
+//                      while a call has at most 8 tokens.  A lane's two 16-byte loads per quantisation group are rows
+//                      g and g+8 of the group's tile; a rolling buffer of 16 such loads per lane is refilled as soon
+//                      as a pair has been consumed, so about 128 KiB per SM stay in flight.  h = SiLU(g) * u goes
+//                      to a small global buffer, bf16 [pass][unit][token][neuron].
 //   w4_down_kernel   : walks chunks (expert pass, block of 64*NWD output columns, group of 128 neurons) = 8 steps
 //                      of 16 neurons x 512 bytes per warp.  Every warp owns four 16-column tiles: its 16-byte load
-//                      per step is their four A fragments.  No block-level synchronisation at all: a warp stages
-//                      the chunk's h fragments for itself with cp.async.  Scale and bias are folded when the
-//                      chunk (= one neuron group) ends; the scaled totals persist while consecutive chunks belong
-//                      to the same pass and column block.  The gate-weighted combine is a red.global.add into the
-//                      fp32 accumulator; the last CTA rounds it once to bf16.
+//                      per step is their four A fragments; the same rolling buffer, two chunks deep.  No block-level
+//                      synchronisation: a warp stages the chunk's h fragments and scales for itself with cp.async.
+//                      Scale and bias are folded when the chunk (= one neuron group) ends; the scaled totals persist
+//                      while consecutive chunks belong to the same pass and column block.  The gate-weighted combine
+//                      is a red.global.add into the fp32 accumulator; the last CTA rounds it once to bf16.  Launched
+//                      as a programmatic dependent of the gate/up kernel: its set-up overlaps that kernel's tail.
 // Zero-copy experts (records in the mapped host pool) go through the same kernels.
 #pragma once
 #include "async.cuh"
@@ -30,7 +32,11 @@ namespace ftmoe {
 
 constexpr int kQ4Tokens = 8;         // tokens per weight pass
 constexpr int kW4Threads = 512;
-constexpr float kW4Bias = 136.f;     // the dequantised operand is 136 + code
+constexpr int kW4Warps = kW4Threads / 32;
+constexpr float kW4Bias = 136.f;
+#ifndef W4_BLOCK_PAIRS
+#define W4_BLOCK_PAIRS 4
+#endif     // the dequantised operand is 136 + code
 
 struct W4Params {
   const WorkItem *items;
@@ -42,58 +48,83 @@ struct W4Params {
   const int32_t *perm;
   const float *topk_w;
   __nv_bfloat16 *hbuf;      // [pass][16-neuron unit][token 8][neuron 16]
+  float *hbias;             // [pass][16-neuron unit][token 8]: 136 x the sum of the unit's 16 (rounded) h values
   float *y_acc;             // [T][d]
   __nv_bfloat16 *y;
   uint32_t *done;
   uint32_t *status;
   int inter, top_k, T, finalize;
+  uint32_t mask, magic;     // 0x000F000F, 0x43084308 (see w4_unpack)
 };
 
 // 8 codes of one word -> four bf16x2 registers holding 136 + code: pairs (0,4) (1,5) (2,6) (3,7).
 struct W4Frag { uint32_t p04, p15, p26, p37; };
-__device__ __forceinline__ W4Frag w4_unpack(uint32_t w) {
+// mask = 0x000F000F and magic = 0x43084308 arrive as kernel arguments: as literals the compiler encodes both as
+// immediates and needs two logic instructions per register (an instruction carries one immediate); as values it
+// cannot see through they live in registers and (x & mask) ^ magic is a single three-input logic instruction.
+struct W4Const { uint32_t mask, magic; };
+__device__ __forceinline__ W4Frag w4_unpack(uint32_t w, const W4Const &k) {
   W4Frag f;
-  f.p04 = (w & 0x000F000Fu) ^ 0x43084308u;
-  f.p15 = ((w >> 4) & 0x000F000Fu) ^ 0x43084308u;
-  f.p26 = ((w >> 8) & 0x000F000Fu) ^ 0x43084308u;
-  f.p37 = ((w >> 12) & 0x000F000Fu) ^ 0x43084308u;
+  f.p04 = (w & k.mask) ^ k.magic;
+  f.p15 = ((w >> 4) & k.mask) ^ k.magic;
+  f.p26 = ((w >> 8) & k.mask) ^ k.magic;
+  f.p37 = ((w >> 12) & k.mask) ^ k.magic;
   return f;
+}
+// d = a * b (no accumulator to clear first)
+__device__ __forceinline__ void mma_bf16_first(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
 }
 __device__ __forceinline__ float bf16lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
 
-// This CTA's share of `total` work items: total/grid each, the first total%grid CTAs one more.
-__device__ __forceinline__ void w4_share(uint32_t total, uint32_t &first, uint32_t &count) {
-  const uint32_t per = total / gridDim.x, rem = total - per * gridDim.x;
-  first = blockIdx.x * per + min((uint32_t)blockIdx.x, rem);
-  count = per + (blockIdx.x < rem ? 1u : 0u);
+// Share number `who` of `total` work items split over `n`: total/n each, the first total%n one more.
+__device__ __forceinline__ uint32_t w4_first(uint32_t total, uint32_t n, uint32_t who) {
+  const uint32_t per = total / n, rem = total - per * n;
+  return who * per + min(who, rem);
+}
+// Largest i in [0, n) with pref[i] <= v  (pref is non-decreasing, pref[0] = 0).
+__device__ __forceinline__ int w4_find_item(const int32_t *pref, int n, uint32_t v) {
+  int lo = 0, hi = n - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if ((uint32_t)pref[mid] <= v) lo = mid; else hi = mid - 1;
+  }
+  return lo;
 }
 
-// Dynamic shared memory of the gate/up kernel: red [2][16 warps][2][16 x 8] f32 | x [8][2d + 64] bytes (every run of 8
-// elements stored as 0,4,1,5,2,6,3,7) | xsum [8][G] f32 | items [max_items] | pref [max_items + 1].
+// Dynamic shared memory of the gate/up kernel: x [8][2d + 64] bytes (every run of 8 elements stored as
+// 0,4,1,5,2,6,3,7) | xbias [8][G] f32 (136 x the sum of x over a group) | items [max_items] | pref [max_items + 1].
 inline size_t w4_gateup_smem_bytes(int max_items, int d) {
-  return (size_t)2 * 16 * 2 * 128 * 4 + (size_t)8 * (2 * d + 64) + (size_t)8 * (d / kGroup) * 4 +
-         (size_t)max_items * sizeof(WorkItem) + ((size_t)max_items + 1) * 4 + 16;
+  return (size_t)8 * (2 * d + 64) + (size_t)8 * (d / kGroup) * 4 + (size_t)max_items * sizeof(WorkItem) +
+         ((size_t)max_items + 1) * 4 + 16;
 }
-// ... of the down kernel: h [16 warps][2][8 units x 8 tokens x 16 neurons] bf16 | items | pref.
+// ... of the down kernel: per warp 3 slots of (h [8 units x 8 tokens x 16 neurons] bf16 | 128 bytes of scales |
+// h bias [8 units][8 tokens] f32) | items | pref.
+constexpr uint32_t kW4DownSlot = 2048 + 128 + 256;
 inline size_t w4_down_smem_bytes(int max_items) {
-  return (size_t)16 * 2 * 2048 + (size_t)max_items * sizeof(WorkItem) + ((size_t)max_items + 1) * 4 + 16;
+  return (size_t)kW4Warps * 3 * kW4DownSlot + (size_t)max_items * sizeof(WorkItem) + ((size_t)max_items + 1) * 4 + 16;
 }
 
-template <int GW, int NW>   // GW quantisation groups per warp, NW warps take part: d = 128 * GW * NW
+template <int G>   // quantisation groups of the hidden dimension: d = 128 G, G a multiple of 4
 __global__ void __launch_bounds__(kW4Threads, 1) w4_gateup_kernel(W4Params p) {
-  constexpr int G = GW * NW, d = kGroup * G;
+  constexpr int d = kGroup * G;
+  constexpr int kPairs = 2 * G;                     // (row g, row g+8) load pairs of a unit: G gate groups, G up groups
   constexpr uint32_t kUA = 2112u * G;               // bytes of a unit: gate tiles, up tiles, gate scales, up scales
   constexpr uint32_t kXStride = 2u * d + 64u;
+  static_assert(G % 4 == 0, "the rolling buffer holds 8 pairs");
   extern __shared__ __align__(128) unsigned char smem[];
-  float *s_red = reinterpret_cast<float *>(smem);                         // [2][16][2][128]
-  unsigned char *s_x = smem + 2 * 16 * 2 * 128 * 4;
-  float *s_xsum = reinterpret_cast<float *>(s_x + 8 * kXStride);          // [8][G]
-  WorkItem *s_items = reinterpret_cast<WorkItem *>(s_xsum + 8 * G);
+  unsigned char *s_x = smem;
+  float *s_xbias = reinterpret_cast<float *>(s_x + 8 * kXStride);          // [8][G]
+  WorkItem *s_items = reinterpret_cast<WorkItem *>(s_xbias + 8 * G);
   int32_t *s_pref = reinterpret_cast<int32_t *>(s_items + p.max_items);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, q = lane & 3;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the down kernel may set itself up meanwhile
   const int n_items = *p.n_items, n_zc = *p.n_zc;
   for (int i = tid; i <= p.max_items; i += kW4Threads) s_pref[i] = p.pref[i];
   {
@@ -104,10 +135,9 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_gateup_kernel(W4Params p) {
   __syncthreads();
   const uint32_t NBLK = (uint32_t)p.inter / 16u;
   const bool dense = p.T <= kQ4Tokens;
-  const bool k_warp = (NW == 16) || warp < NW;
 
   // x rows of the MMA columns into shared memory, every run of 8 stored as 0,4,1,5,2,6,3,7 (the order in which the
-  // dequantiser produces the codes of a word), and their sums over each quantisation group
+  // dequantiser produces the codes of a word), and 136 x their sums over each quantisation group
   auto stage_x = [&](auto tok_of_column) {
     for (int i = tid; i < 8 * (d / 8); i += kW4Threads) {
       const int j = i / (d / 8), c8 = i - j * (d / 8);
@@ -124,155 +154,151 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_gateup_kernel(W4Params p) {
                   bf16hi(v.w);
 #pragma unroll
       for (int o2 = 1; o2 < 16; o2 <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o2);   // 16 chunks = one group
-      if ((lane & 15) == 0) s_xsum[j * G + c8 / 16] = sum;
+      if ((lane & 15) == 0) s_xbias[j * G + c8 / 16] = kW4Bias * sum;
     }
   };
 
-  // ---- per-lane constants ----
-  const uint32_t t_off = (uint32_t)(warp * GW) * 1024u + g * 64u + q * 16u;      // row g, chunk q of the warp's first tile
-  const uint32_t s_off = 2048u * G + (uint32_t)(warp * GW) * 32u + g * 4u;       // (scale of row g, of row g + 8)
-  const uint32_t my_x = smem_u32(s_x) + g * kXStride + (uint32_t)(warp * GW) * 256u + 16u * q;
+  const uint32_t my_x = smem_u32(s_x) + g * kXStride + 16u * q;
+  const float *my_b0 = s_xbias + (2 * q) * G, *my_b1 = s_xbias + (2 * q + 1) * G;
 
-  uint4 bufg[2 * GW], bufu[2 * GW];
-  uint32_t scg[GW], scu[GW];
-  auto load_part = [&](uint4 (&buf)[2 * GW], uint32_t (&sc)[GW], const uint8_t *unit, uint32_t which) {
-    if (k_warp) {
-      const uint8_t *t = unit + which * (1024u * G) + t_off;
-#pragma unroll
-      for (int gw = 0; gw < GW; ++gw) {
-        buf[2 * gw] = ld_stream_16(t + gw * 1024);
-        buf[2 * gw + 1] = ld_stream_16(t + gw * 1024 + 512);
+  const W4Const ks = {p.mask, p.magic};
+  // One warp streams `n_units` consecutive units starting at `base`; their h goes to rows hrow0.. of the h buffer.
+  // Work proceeds in blocks of 8 (row g, row g+8) load pairs = 8 quantisation groups of the gate or the up part.
+  constexpr int kBP = W4_BLOCK_PAIRS;               // pairs of a block = depth of the rolling register buffer
+  constexpr int kBlocks = kPairs / kBP;             // blocks of a unit
+  static_assert(G % kBP == 0, "a block lies in the gate or in the up part");
+  auto run = [&](const uint8_t *base, int n_units, uint32_t hrow0) {
+    uint4 buf[2 * kBP];
+    uint32_t sc[kBP];   // and the two rows' scales
+    const uint8_t *nptr = base + g * 64 + q * 16;              // next block to request
+    const uint8_t *nsc = base + 2048u * G + g * 4;
+    int nblk = 0, blocks_left = n_units * kBlocks;             // its index in its unit; blocks not yet requested
+    auto advance = [&]() {
+      nptr += kBP * 1024;
+      nsc += kBP * 32;
+      --blocks_left;
+      if (++nblk == kBlocks) {   // on to the next unit: skip this unit's scales / the next unit's tiles
+        nblk = 0;
+        nptr += 64 * G;
+        nsc += 2048u * G;
       }
-      const uint8_t *s = unit + which * (32u * G) + s_off;
+    };
 #pragma unroll
-      for (int gw = 0; gw < GW; ++gw)
-        asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(sc[gw]) : "l"(s + gw * 32));
+    for (int pi = 0; pi < kBP; ++pi) {
+      buf[2 * pi] = ld_stream_16(nptr + pi * 1024);
+      buf[2 * pi + 1] = ld_stream_16(nptr + pi * 1024 + 512);
+      asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(sc[pi]) : "l"(nsc + pi * 32));
     }
-  };
-  // scaled partial sums of one part over this warp's groups -> shared memory
-  auto part_sums = [&](const uint4 (&buf)[2 * GW], const uint32_t (&sc)[GW], float *r) {
-    if (k_warp) {
-      float tot[4] = {0.f, 0.f, 0.f, 0.f};
+    advance();
+    for (int u = 0; u < n_units; ++u) {
+      float tot[4] = {0.f, 0.f, 0.f, 0.f}, tg[4] = {0.f, 0.f, 0.f, 0.f};
+      int xg = 0;                                    // first group of the block
+      for (int blk = 0; blk < kBlocks; ++blk) {
+        const bool more = blocks_left > 0;
+        const uint8_t *rp = nptr, *rs = nsc;         // the block that refills this one's registers
+        if (more) advance();
+        const uint32_t xa = my_x + xg * 256u;
+        const float *b0p = my_b0 + xg, *b1p = my_b1 + xg;
 #pragma unroll
-      for (int gw = 0; gw < GW; ++gw) {
-        float a1[4] = {0.f, 0.f, 0.f, 0.f}, a2[4] = {0.f, 0.f, 0.f, 0.f};
-        const uint32_t lo[4] = {buf[2 * gw].x, buf[2 * gw].y, buf[2 * gw].z, buf[2 * gw].w};
-        const uint32_t hi[4] = {buf[2 * gw + 1].x, buf[2 * gw + 1].y, buf[2 * gw + 1].z, buf[2 * gw + 1].w};
+        for (int pi = 0; pi < kBP; ++pi) {
+          float a1[4], a2[4];
+          const uint32_t lo[4] = {buf[2 * pi].x, buf[2 * pi].y, buf[2 * pi].z, buf[2 * pi].w};
+          const uint32_t hi[4] = {buf[2 * pi + 1].x, buf[2 * pi + 1].y, buf[2 * pi + 1].z, buf[2 * pi + 1].w};
+          const uint32_t scale = sc[pi];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {   // word j: hidden indices 32j + 8q + 0..7 of the group
-          const W4Frag fl = w4_unpack(lo[j]), fh = w4_unpack(hi[j]);
-          const uint4 xv = lds_v4(my_x + gw * 256u + j * 64u);
-          mma_bf16(a1, fl.p04, fh.p04, fl.p15, fh.p15, xv.x, xv.y);
-          mma_bf16(a2, fl.p26, fh.p26, fl.p37, fh.p37, xv.z, xv.w);
+          for (int j = 0; j < 4; ++j) {   // word j: hidden indices 32j + 8q + 0..7 of the group
+            const W4Frag fl = w4_unpack(lo[j], ks), fh = w4_unpack(hi[j], ks);
+            const uint4 xv = lds_v4(xa + pi * 256u + j * 64u);
+            if (j == 0) {
+              mma_bf16_first(a1, fl.p04, fh.p04, fl.p15, fh.p15, xv.x, xv.y);
+              mma_bf16_first(a2, fl.p26, fh.p26, fl.p37, fh.p37, xv.z, xv.w);
+            } else {
+              mma_bf16(a1, fl.p04, fh.p04, fl.p15, fh.p15, xv.x, xv.y);
+              mma_bf16(a2, fl.p26, fh.p26, fl.p37, fh.p37, xv.z, xv.w);
+            }
+          }
+          if (more) {   // refill the pair just consumed
+            buf[2 * pi] = ld_stream_16(rp + pi * 1024);
+            buf[2 * pi + 1] = ld_stream_16(rp + pi * 1024 + 512);
+            asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(sc[pi]) : "l"(rs + pi * 32));
+          }
+          const float s_lo = bf16lo(scale), s_hi = bf16hi(scale);
+          const float b0 = b0p[pi], b1 = b1p[pi];
+          tot[0] += s_lo * (a1[0] + a2[0] - b0);
+          tot[1] += s_lo * (a1[1] + a2[1] - b1);
+          tot[2] += s_hi * (a1[2] + a2[2] - b0);
+          tot[3] += s_hi * (a1[3] + a2[3] - b1);
         }
-        const float s_lo = bf16lo(sc[gw]), s_hi = bf16hi(sc[gw]);
-        const int grp = warp * GW + gw;
-        const float b0 = kW4Bias * s_xsum[(2 * q) * G + grp], b1 = kW4Bias * s_xsum[(2 * q + 1) * G + grp];
-        tot[0] += s_lo * (a1[0] + a2[0] - b0);
-        tot[1] += s_lo * (a1[1] + a2[1] - b1);
-        tot[2] += s_hi * (a1[2] + a2[2] - b0);
-        tot[3] += s_hi * (a1[3] + a2[3] - b1);
+        xg += kBP;
+        if (xg == G) {
+          xg = 0;
+          if (blk < kBlocks - 1) {   // the gate sums are complete: the up groups follow
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { tg[i] = tot[i]; tot[i] = 0.f; }
+          }
+        }
       }
-      *reinterpret_cast<float2 *>(r + g * 8 + 2 * q) = make_float2(tot[0], tot[1]);
-      *reinterpret_cast<float2 *>(r + (g + 8) * 8 + 2 * q) = make_float2(tot[2], tot[3]);
+      // h = SiLU(gate) * up of neurons g, g+8 and tokens 2q, 2q+1, rounded to bf16; and 136 x its sums over the
+      // unit's 16 neurons, which the down kernel subtracts
+      __nv_bfloat16 *hrow = p.hbuf + ((size_t)hrow0 + u) * 128;
+      float hr[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float a = tg[i];
+        const __nv_bfloat16 hv = __float2bfloat16_rn(__fdividef(a, 1.f + __expf(-a)) * tot[i]);
+        hrow[(2 * q + (i & 1)) * 16 + g + 8 * (i >> 1)] = hv;
+        hr[i] = __bfloat162float(hv);
+      }
+      float s0 = hr[0] + hr[2], s1 = hr[1] + hr[3];
+#pragma unroll
+      for (int o = 4; o < 32; o <<= 1) {
+        s0 += __shfl_xor_sync(0xffffffffu, s0, o);
+        s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+      }
+      if (g == 0) *reinterpret_cast<float2 *>(p.hbias + ((size_t)hrow0 + u) * 8 + 2 * q) = make_float2(kW4Bias * s0, kW4Bias * s1);
     }
   };
 
-  // ---- this CTA's share of the units: resident range, then host-resident range ----
-  uint32_t rfirst0, rcount0, rfirst1, rcount1;
-  w4_share((uint32_t)s_pref[n_items] * NBLK, rfirst0, rcount0);
-  w4_share((uint32_t)(s_pref[n_items + n_zc] - s_pref[n_items]) * NBLK, rfirst1, rcount1);
-  rfirst1 += (uint32_t)s_pref[n_items] * NBLK;
-  struct Seg { const uint8_t *unit0; int item, pass, n_units; uint32_t hrow; };
-  int range = 0, item = 0;
-  uint32_t pu = 0, b = 0, left = 0;
-  auto next_segment = [&](Seg &s) -> bool {
-    while (left == 0) {
-      if (range == 2) return false;
-      left = range ? rcount1 : rcount0;
-      if (left > 0) {
-        const uint32_t first = range ? rfirst1 : rfirst0;
-        pu = first / NBLK;
-        b = first - pu * NBLK;
-      }
-      ++range;
-    }
-    while ((uint32_t)s_pref[item + 1] <= pu) ++item;
-    s.item = item;
-    s.pass = (int)(pu - (uint32_t)s_pref[item]);
-    s.n_units = (int)min(left, NBLK - b);
-    s.unit0 = s_items[item].w + (size_t)b * kUA;
-    s.hrow = pu * NBLK + b;
-    left -= s.n_units;
-    ++pu;
-    b = 0;
-    return true;
-  };
-
-  Seg sg, nsg;
-  bool more = next_segment(sg);
-  if (more) {
-    load_part(bufg, scg, sg.unit0, 0);
-    load_part(bufu, scu, sg.unit0, 1);
-  }
   if (dense) {
     stage_x([&](int j) { return j < p.T ? j : -1; });
     __syncthreads();
   }
-  uint32_t par = 0;
-  while (more) {
-    more = next_segment(nsg);
-    const uint8_t *after = more ? nsg.unit0 : nullptr;
-    if (!dense) {   // MMA column j is the pass's j-th pair: stage those tokens' rows
-      const WorkItem &it = s_items[sg.item];
-      const int tok0 = sg.pass * kQ4Tokens, nt = min(kQ4Tokens, it.n_tok - tok0);
-      const int off_ = it.off + tok0, expert_ = it.expert;
-      __syncthreads();   // the previous segment's readers of s_x / s_xsum are done
-      stage_x([&](int j) {
-        if (j >= nt) return -1;
-        return expert_ >= 0 ? p.perm[off_ + j] / p.top_k : tok0 + j;
-      });
-      __syncthreads();
-    }
-    const uint8_t *unit = sg.unit0;
-    for (int k = 0; k < sg.n_units; ++k, unit += kUA) {
-      const uint8_t *nunit = (k + 1 < sg.n_units) ? unit + kUA : after;
-      float *red = s_red + par * (16 * 2 * 128);
-      part_sums(bufg, scg, red + (warp * 2 + 0) * 128);
-      if (nunit) load_part(bufg, scg, nunit, 0);
-      part_sums(bufu, scu, red + (warp * 2 + 1) * 128);
-      if (nunit) load_part(bufu, scu, nunit, 1);
-      __syncthreads();
-      {   // h = SiLU(sum gate) * (sum up): four threads per value, each sums a quarter of the warps' partial sums
-        const int r = tid >> 2, qu = tid & 3;   // r = neuron * 8 + token
-        float a = 0.f, c = 0.f;
-#pragma unroll
-        for (int w = 0; w < NW / 4; ++w) {
-          a += red[((qu * (NW / 4) + w) * 2 + 0) * 128 + r];
-          c += red[((qu * (NW / 4) + w) * 2 + 1) * 128 + r];
-        }
-        if (NW % 4 != 0 && qu < NW % 4) {   // (NW = 14: two warps left over)
-          a += red[(((NW / 4) * 4 + qu) * 2 + 0) * 128 + r];
-          c += red[(((NW / 4) * 4 + qu) * 2 + 1) * 128 + r];
-        }
-        a += __shfl_xor_sync(0xffffffffu, a, 1);
-        c += __shfl_xor_sync(0xffffffffu, c, 1);
-        a += __shfl_xor_sync(0xffffffffu, a, 2);
-        c += __shfl_xor_sync(0xffffffffu, c, 2);
-        if (qu == 0)
-          p.hbuf[((size_t)sg.hrow + k) * 128 + (r & 7) * 16 + (r >> 3)] = __float2bfloat16_rn(__fdividef(a, 1.f + __expf(-a)) * c);
+  // Units (pass, 16-neuron block) in one flat order, split evenly over all warps of the grid: the slot-resident
+  // range first, then the host-resident range.
+  const uint32_t n_warps = gridDim.x * kW4Warps, wi = blockIdx.x * kW4Warps + warp;
+  for (int range = 0; range < 2; ++range) {
+    const uint32_t pass0 = range ? (uint32_t)s_pref[n_items] : 0u;
+    const uint32_t pass1 = range ? (uint32_t)s_pref[n_items + n_zc] : (uint32_t)s_pref[n_items];
+    const uint32_t total = (pass1 - pass0) * NBLK, ubase = pass0 * NBLK;
+    if (total == 0) continue;
+    const uint32_t wf = ubase + w4_first(total, n_warps, wi), we = ubase + w4_first(total, n_warps, wi + 1);
+    const uint32_t cf = ubase + w4_first(total, n_warps, blockIdx.x * kW4Warps);
+    const uint32_t ce = ubase + w4_first(total, n_warps, (blockIdx.x + 1) * kW4Warps);
+    if (cf >= ce) continue;
+    for (uint32_t pu = cf / NBLK; pu * NBLK < ce; ++pu) {   // the passes this CTA's warps touch
+      const int item = w4_find_item(s_pref, n_items + n_zc, pu);
+      const WorkItem &it = s_items[item];
+      if (!dense) {   // MMA column j is the pass's j-th pair: stage those tokens' rows
+        const int tok0 = (int)(pu - (uint32_t)s_pref[item]) * kQ4Tokens, nt = min(kQ4Tokens, it.n_tok - tok0);
+        const int off_ = it.off + tok0, expert_ = it.expert;
+        __syncthreads();   // the previous pass's readers are done
+        stage_x([&](int j) {
+          if (j >= nt) return -1;
+          return expert_ >= 0 ? p.perm[off_ + j] / p.top_k : tok0 + j;
+        });
+        __syncthreads();
       }
-      par ^= 1u;   // the next unit writes the other buffer: one barrier per unit is enough
+      const uint32_t lo = max(wf, pu * NBLK), hi = min(we, (pu + 1) * NBLK);
+      if (lo < hi) run(it.w + (size_t)(lo - pu * NBLK) * kUA, (int)(hi - lo), lo);
     }
-    sg = nsg;
   }
 }
 
 template <int NWD>   // warps that own output columns: a column block is 64 * NWD columns
 __global__ void __launch_bounds__(kW4Threads, 1) w4_down_kernel(W4Params p, int d) {
   extern __shared__ __align__(128) unsigned char smem[];
-  unsigned char *s_h = smem;                                                // [16 warps][2][2048 bytes]
-  WorkItem *s_items = reinterpret_cast<WorkItem *>(smem + 16 * 2 * 2048);
+  unsigned char *s_h = smem;                                                // [16 warps][3][h 2048 | scales 128]
+  WorkItem *s_items = reinterpret_cast<WorkItem *>(smem + kW4Warps * 3 * kW4DownSlot);
   int32_t *s_pref = reinterpret_cast<int32_t *>(s_items + p.max_items);
   __shared__ int s_last;
 
@@ -291,13 +317,17 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_down_kernel(W4Params p, int 
   const size_t sec_b = (size_t)NBLK * 2112u * G, sec_c = sec_b + (size_t)p.inter * d / 2;
   const uint32_t per_pass = CB * NG;                // chunks of one pass, neuron group fastest
   const bool dense = p.T <= kQ4Tokens;
+  // everything above reads only what was ready before the gate/up kernel; from here on its h is needed
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   if (warp < NWD) {
-    uint32_t rfirst0, rcount0, rfirst1, rcount1;
-    w4_share((uint32_t)s_pref[n_items] * per_pass, rfirst0, rcount0);
-    w4_share((uint32_t)(s_pref[n_items + n_zc] - s_pref[n_items]) * per_pass, rfirst1, rcount1);
-    rfirst1 += (uint32_t)s_pref[n_items] * per_pass;
-    const uint32_t my_h = smem_u32(s_h) + (uint32_t)warp * 4096u;
+    const uint32_t t0 = (uint32_t)s_pref[n_items] * per_pass;
+    const uint32_t t1 = (uint32_t)(s_pref[n_items + n_zc] - s_pref[n_items]) * per_pass;
+    const uint32_t rfirst0 = w4_first(t0, gridDim.x, blockIdx.x), rcount0 = w4_first(t0, gridDim.x, blockIdx.x + 1) - rfirst0;
+    const uint32_t rfirst1 = t0 + w4_first(t1, gridDim.x, blockIdx.x);
+    const uint32_t rcount1 = t0 + w4_first(t1, gridDim.x, blockIdx.x + 1) - rfirst1;
+    const uint32_t my_h = smem_u32(s_h) + (uint32_t)warp * 3u * kW4DownSlot;
+    const W4Const ks = {p.mask, p.magic};
 
     // chunk cursor: (pass pu, column block cb, neuron group ng)
     struct Ck { const uint8_t *rec; uint32_t pu, cb, ng; int item; };
@@ -321,21 +351,25 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_down_kernel(W4Params p, int 
       --left;
       return true;
     };
-    uint4 bufa[8], bufb[8];   // this chunk's / the next chunk's eight steps
-    uint4 sca, scb;           // and their scales: (column g, column g + 8) of the warp's four tiles
-    auto load_chunk = [&](uint4 (&buf)[8], uint4 &sc, const Ck &c, int hslot) {
-      const uint8_t *t = c.rec + sec_b + ((size_t)(c.cb * NG + c.ng) * 8u * NWD + warp) * 512u + lane * 16u;
-#pragma unroll
-      for (int uu = 0; uu < 8; ++uu) buf[uu] = ld_stream_16(t + (size_t)uu * NWD * 512u);
-      sc = ld_stream_16(c.rec + sec_c + ((size_t)(c.ng * CB + c.cb) * NWD + warp) * 128u + g * 16u);
-      // h of the chunk's 8 units (2 KiB, contiguous) for this warp alone
+    // h of the chunk's 8 units (2 KiB, contiguous) and the chunk's scales for this warp alone
+    auto stage = [&](const Ck &c, uint32_t slot) {
       const unsigned char *hsrc = reinterpret_cast<const unsigned char *>(p.hbuf) + ((size_t)c.pu * NBLK + c.ng * 8u) * 256u;
+      const uint32_t dst = my_h + slot * kW4DownSlot;
 #pragma unroll
       for (int i = 0; i < 4; ++i)
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(my_h + hslot * 2048u + (i * 32 + lane) * 16u),
-                     "l"(hsrc + (i * 32 + lane) * 16)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (i * 32 + lane) * 16u), "l"(hsrc + (i * 32 + lane) * 16)
                      : "memory");
-      asm volatile("cp.async.commit_group;" ::: "memory");
+      if (lane < 8)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 2048u + lane * 16u),
+                     "l"(c.rec + sec_c + ((size_t)(c.ng * CB + c.cb) * NWD + warp) * 128u + lane * 16u)
+                     : "memory");
+      else if (lane < 24)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 2176u + (lane - 8) * 16u),
+                     "l"(reinterpret_cast<const unsigned char *>(p.hbias) + ((size_t)c.pu * NBLK + c.ng * 8u) * 32u + (lane - 8) * 16)
+                     : "memory");
+    };
+    auto weights_of = [&](const Ck &c) -> const uint8_t * {
+      return c.rec + sec_b + ((size_t)(c.cb * NG + c.ng) * 8u * NWD + warp) * 512u + lane * 16u;
     };
 
     float dtot[4][4];
@@ -394,31 +428,36 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_down_kernel(W4Params p, int 
         }
       }
     };
-    // one chunk: 8 steps of 16 neurons for the warp's four column tiles, then scale and bias
-    auto consume = [&](const uint4 (&buf)[8], const uint4 &sc, int hslot) {
-      asm volatile("cp.async.wait_group 1;" ::: "memory");   // this chunk's h has landed (the next one's may be in flight)
+    // one chunk: 8 steps of 16 neurons for the warp's four column tiles, then scale and bias; every step's
+    // register is refilled with the same step of the chunk two ahead as soon as it has been consumed
+    auto consume = [&](uint4 (&buf)[8], uint32_t slot, const uint8_t *refill) {
+      asm volatile("cp.async.wait_group 2;" ::: "memory");   // this chunk's h, scales and biases have landed
       __syncwarp();
+      const uint32_t hs_base = my_h + slot * kW4DownSlot;
       float acc[4][4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) { acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f; }
-      float hs = 0.f;
 #pragma unroll
       for (int uu = 0; uu < 8; ++uu) {
         uint2 hb;   // h of token g, neurons 4q..4q+3 of the step
-        asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(hb.x), "=r"(hb.y) : "r"(my_h + hslot * 2048u + uu * 256u + g * 32u + q * 8u));
-        hs += bf16lo(hb.x) + bf16hi(hb.x) + bf16lo(hb.y) + bf16hi(hb.y);
+        asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(hb.x), "=r"(hb.y) : "r"(hs_base + uu * 256u + g * 32u + q * 8u));
         const uint32_t wv[4] = {buf[uu].x, buf[uu].y, buf[uu].z, buf[uu].w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          const W4Frag f = w4_unpack(wv[j]);
-          mma_bf16(acc[j], f.p04, f.p15, f.p26, f.p37, hb.x, hb.y);
+          const W4Frag f = w4_unpack(wv[j], ks);
+          if (uu == 0) mma_bf16_first(acc[j], f.p04, f.p15, f.p26, f.p37, hb.x, hb.y);
+          else mma_bf16(acc[j], f.p04, f.p15, f.p26, f.p37, hb.x, hb.y);
         }
+        if (refill) buf[uu] = ld_stream_16(refill + (size_t)uu * NWD * 512u);
       }
-      __syncwarp();   // every lane has read the slot: it may be overwritten by the chunk after the next
-      hs += __shfl_xor_sync(0xffffffffu, hs, 1);      // sum over the four lanes of token g: its 128 neurons
-      hs += __shfl_xor_sync(0xffffffffu, hs, 2);
-      const float b0 = kW4Bias * __shfl_sync(0xffffffffu, hs, (2 * q) * 4);
-      const float b1 = kW4Bias * __shfl_sync(0xffffffffu, hs, (2 * q + 1) * 4);
+      const uint4 sc = lds_v4(hs_base + 2048u + g * 16u);   // (column g, column g + 8) of the warp's four tiles
+      float b0 = 0.f, b1 = 0.f;                             // 136 x the sums of h over the chunk's 128 neurons
+#pragma unroll
+      for (int uu = 0; uu < 8; ++uu) {
+        float2 hb2;
+        asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(hb2.x), "=f"(hb2.y) : "r"(hs_base + 2176u + uu * 32u + q * 8u));
+        b0 += hb2.x;
+        b1 += hb2.y;
+      }
+      __syncwarp();   // every lane has read the slot: it may be overwritten
       const uint32_t sw[4] = {sc.x, sc.y, sc.z, sc.w};
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
@@ -430,32 +469,43 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_down_kernel(W4Params p, int 
       }
     };
 
-    Ck ck, nk;
-    bool have = next_chunk(ck);
-    if (have) {
-      load_chunk(bufa, sca, ck, 0);
-      begin_pass(ck);
+    uint4 bufa[8], bufb[8];   // even / odd chunks of this CTA's sequence
+    Ck c0, c1, c2;            // the chunk being consumed and the two after it
+    bool h0 = next_chunk(c0), h1 = h0 && next_chunk(c1), h2 = h1 && next_chunk(c2);
+    if (h0) {
+      stage(c0, 0);
+      const uint8_t *w = weights_of(c0);
+#pragma unroll
+      for (int uu = 0; uu < 8; ++uu) bufa[uu] = ld_stream_16(w + (size_t)uu * NWD * 512u);
+      begin_pass(c0);
       zero_tot();
     }
-    int slot = 0;
-    while (have) {
-      const bool more = next_chunk(nk);
-      // even steps: current chunk in bufa; odd steps: in bufb
-      if (slot == 0) {
-        if (more) load_chunk(bufb, scb, nk, 1); else asm volatile("cp.async.commit_group;" ::: "memory");
-        consume(bufa, sca, 0);
-      } else {
-        if (more) load_chunk(bufa, sca, nk, 0); else asm volatile("cp.async.commit_group;" ::: "memory");
-        consume(bufb, scb, 1);
-      }
-      if (!more || nk.pu != ck.pu || nk.cb != ck.cb) {
-        flush(ck.cb);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    if (h1) {
+      stage(c1, 1);
+      const uint8_t *w = weights_of(c1);
+#pragma unroll
+      for (int uu = 0; uu < 8; ++uu) bufb[uu] = ld_stream_16(w + (size_t)uu * NWD * 512u);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    uint32_t slot = 0;
+    int half = 0;
+    while (h0) {
+      const uint32_t slot2 = slot >= 1 ? slot - 1 : 2;   // (slot + 2) % 3
+      if (h2) stage(c2, slot2);
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      const uint8_t *refill = h2 ? weights_of(c2) : nullptr;
+      if (half == 0) consume(bufa, slot, refill); else consume(bufb, slot, refill);
+      if (!h1 || c1.pu != c0.pu || c1.cb != c0.cb) {
+        flush(c0.cb);
         zero_tot();
-        if (more && nk.pu != ck.pu) begin_pass(nk);
+        if (h1 && c1.pu != c0.pu) begin_pass(c1);
       }
-      ck = nk;
-      have = more;
-      slot ^= 1;
+      c0 = c1; c1 = c2;
+      h0 = h1; h1 = h2;
+      h2 = h1 && next_chunk(c2);
+      slot = slot == 2 ? 0 : slot + 1;
+      half ^= 1;
     }
   }
 

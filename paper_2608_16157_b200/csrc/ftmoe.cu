@@ -88,6 +88,7 @@ struct ft_moe {
   uint32_t *seq_dev = nullptr;
   uint32_t *done_dev = nullptr;          // CTA completion counter of the streaming MMA kernel
   long long *trace_dev = nullptr;        // per-CTA clocks of the latest streaming-kernel launch
+  float *w4_hbias = nullptr;             // int4 path: 136 x the sums of h over each unit, [pass][unit][token 8]
   __nv_bfloat16 *w4_hbuf = nullptr;      // int4 path: h as [pass][16-neuron unit][token 8][neuron 16]
   int last_fill_layer = -1;
   int overlap = 0;                      // launch mode of the streaming kernel (see FfnStreamParams::overlap)
@@ -427,6 +428,7 @@ ft_status_t ft_moe_destroy(ft_moe_t *h) {
   cudaFree(h->seq_dev);
   cudaFree(h->done_dev);
   cudaFree(h->w4_hbuf);
+  cudaFree(h->w4_hbias);
   cudaFree(h->trace_dev);
   cudaFree(h->stage_logits);
   cudaFree(h->stage_x);
@@ -587,16 +589,17 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
   if (c.wdtype == FT_W_INT4_G128) {
     const size_t passes = (P + 7) / 8 + 2 * E + 2;
     FT_TRY(cudaMalloc(&h->w4_hbuf, passes * (c.inter / 16) * 256));
+    FT_TRY(cudaMalloc(&h->w4_hbias, passes * (c.inter / 16) * 32));
     // (limits are per function and device, not per handle: always the largest a CTA can have, and the handle's own
     // need is checked against it)
     const int sa = 232448, sb = (int)w4_down_smem_bytes(2 * kMaxExperts + 1);
     if (w4_gateup_smem_bytes(2 * c.n_experts + 1, c.hidden) > (size_t)sa) return fail(FT_ERR_UNSUPPORTED);
-    FT_TRY(cudaFuncSetAttribute(w4_gateup_kernel<1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
-    FT_TRY(cudaFuncSetAttribute(w4_gateup_kernel<1, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
-    FT_TRY(cudaFuncSetAttribute(w4_gateup_kernel<1, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
-    FT_TRY(cudaFuncSetAttribute(w4_gateup_kernel<2, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
-    FT_TRY(cudaFuncSetAttribute(w4_gateup_kernel<4, 14>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
-    FT_TRY(cudaFuncSetAttribute(w4_gateup_kernel<4, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(w4_gateup_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(w4_gateup_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(w4_gateup_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(w4_gateup_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(w4_gateup_kernel<56>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(w4_gateup_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
     FT_TRY(cudaFuncSetAttribute(w4_down_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
     FT_TRY(cudaFuncSetAttribute(w4_down_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
   }
@@ -1009,7 +1012,8 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   qp.pref = sc.res_pref;
   qp.max_items = 2 * c.n_experts + 1;
   qp.x = x_bf; qp.perm = sc.perm; qp.topk_w = sc.topk_w;
-  qp.hbuf = h->w4_hbuf;
+  qp.hbuf = h->w4_hbuf; qp.hbias = h->w4_hbias;
+  qp.mask = 0x000F000Fu; qp.magic = 0x43084308u;
   qp.y_acc = h->y_acc; qp.y = static_cast<__nv_bfloat16 *>(y_dev);
   qp.done = h->done_dev; qp.status = h->status_dev;
   qp.inter = c.inter; qp.top_k = c.top_k; qp.T = L.T;
@@ -1020,18 +1024,26 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   {
     TimeScope ts(h, st, FT_TIME_FFN_ZC);   // (timing slot reused for the gate/up kernel of the int4 path)
     switch (c.hidden) {
-      case 512: w4_gateup_kernel<1, 4><<<grid, kW4Threads, sa, st>>>(qp); break;
-      case 1024: w4_gateup_kernel<1, 8><<<grid, kW4Threads, sa, st>>>(qp); break;
-      case 2048: w4_gateup_kernel<1, 16><<<grid, kW4Threads, sa, st>>>(qp); break;
-      case 4096: w4_gateup_kernel<2, 16><<<grid, kW4Threads, sa, st>>>(qp); break;
-      case 7168: w4_gateup_kernel<4, 14><<<grid, kW4Threads, sa, st>>>(qp); break;
-      default: w4_gateup_kernel<4, 16><<<grid, kW4Threads, sa, st>>>(qp); break;
+      case 512: w4_gateup_kernel<4><<<grid, kW4Threads, sa, st>>>(qp); break;
+      case 1024: w4_gateup_kernel<8><<<grid, kW4Threads, sa, st>>>(qp); break;
+      case 2048: w4_gateup_kernel<16><<<grid, kW4Threads, sa, st>>>(qp); break;
+      case 4096: w4_gateup_kernel<32><<<grid, kW4Threads, sa, st>>>(qp); break;
+      case 7168: w4_gateup_kernel<56><<<grid, kW4Threads, sa, st>>>(qp); break;
+      default: w4_gateup_kernel<64><<<grid, kW4Threads, sa, st>>>(qp); break;
     }
   }
   {
     TimeScope ts(h, st, FT_TIME_FFN_RES);
-    if (c.hidden == 512) w4_down_kernel<8><<<grid, kW4Threads, sb, st>>>(qp, c.hidden);
-    else w4_down_kernel<16><<<grid, kW4Threads, sb, st>>>(qp, c.hidden);
+    // a programmatic dependent of the gate/up kernel: its blocks set themselves up while that kernel drains and
+    // wait for its completion before they read h
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(grid); lc.blockDim = dim3(kW4Threads); lc.dynamicSmemBytes = sb; lc.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = at; lc.numAttrs = 1;
+    if (c.hidden == 512) FT_CUDA(cudaLaunchKernelEx(&lc, w4_down_kernel<8>, qp, c.hidden));
+    else FT_CUDA(cudaLaunchKernelEx(&lc, w4_down_kernel<16>, qp, c.hidden));
     if (own_finalize) {
       const int n4 = L.T * (c.hidden / 4);
       finalize_kernel<<<std::min((n4 + 255) / 256, h->sm_count * 8), 256, 0, st>>>(h->y_acc, qp.y, n4);
