@@ -44,18 +44,22 @@
  *                   order and land directly in mma.sync fragments; a bulk copy of the same bytes into shared memory
  *                   is a valid swizzled K-major tcgen05 operand, so the prefill GEMMs consume the tiles as they are.
  *                   S = 3*inter*hidden*2 bytes.
- *   FT_W_INT4_G128: 4-bit two's-complement codes in [-8,7] for the same three matrices, then bf16 scales;
- *                   weight = scale * code.
- *                     Wg_q, Wu_q : row-major [inter][hidden/2] bytes, two codes per byte along hidden
- *                                  (low nibble = even column).
- *                     Wd_q       : tensor-core fragment order: blocks of 16 neurons x tiles of 16 columns x
- *                                  32 little-endian 32-bit words; in word l = 4g + q of block b, tile ct,
- *                                  nibble j (bits 4j..4j+3) is the code of neuron 16b + NN[j] + q and column
- *                                  16ct + CC[j] + g, NN = (0,8,0,8,4,12,4,12), CC = (0,0,8,8,0,0,8,8).
- *                     sg, su     : [inter][hidden/128] bf16 (groups of 128 consecutive hidden indices: the
- *                                  contraction dimension of gate/up).
- *                     sd         : [inter/128][hidden] bf16 (groups of 128 consecutive neurons: the
- *                                  contraction dimension of down).
+ *   FT_W_INT4_G128: 4-bit two's-complement codes in [-8,7] and bf16 scales, weight = scale * code, groups of 128
+ *                   along the contraction dimension (G = hidden/128 hidden groups for gate/up, NG = inter/128 neuron
+ *                   groups for down), in tensor-core tile order.  Three sections:
+ *                   A. inter/16 units of 16 neurons, 2112*G bytes each: G gate tiles, G up tiles (1 KiB each), gate
+ *                      scales, up scales (32*G bytes each).  A tile is 16 neuron rows x 128 hidden indices = 16
+ *                      rows of 64 bytes; in a row the code of hidden index 128*grp + 32*j + 8*q + e is nibble e
+ *                      (bits 4e..4e+3) of the little-endian 32-bit word j of the 16-byte chunk q.  The scales of a
+ *                      tile are 8 pairs (row r, row r+8) of bf16.
+ *                   B. down codes: for each column block cb (CBW = 64*min(16, hidden/64) columns), neuron group ng
+ *                      and 16-neuron step uu of the group: CBW/64 x 512 bytes; in each 512 bytes lane l = 4g + q
+ *                      owns 16 bytes = 4 words, word j belongs to the 16-column tile 4w + j of the block; its nibble
+ *                      e is the code of column g + 8*(e & 1) of the tile and neuron 4q + e/2 of the step.
+ *                   C. down scales sd[ng][column] in the order (ng, cb, w, g, j, half): 8 pairs per tile again.
+ *                   In both code sections (w & 0x0F0F0F0F) ^ 0x08080808 of a word w and of w >> 4 are operand
+ *                   registers of the int8 tensor-core instruction as they are (bytes code + 8; the kernels subtract
+ *                   8 x the activation sums).
  *                   S = 3*inter*hidden/2 + (2*inter*hidden/128 + (inter/128)*hidden)*2 bytes.
  *   Shape limits: bf16: hidden in {256, 512, 1024, 2048}, inter % 16 == 0; int4: hidden in
  *   {512, 1024, 2048, 4096, 7168, 8192}, inter % 128 == 0; n_experts <= 1024;

@@ -255,7 +255,7 @@ def unpack_record(rec: np.ndarray, d: int, inter: int, wdtype: str):
       gate scale of (n, group i//128):   UA*(n//16) + 2048*G + 32*(i//128) + 4*(n%8) + 2*((n%16)//8);  up: + 32*G
       down code of (neuron n, column c): with ng = n//128, uu = (n%128)//16, q = (n%16)//4, r = n%4, g = c%8,
                                          half = (c%16)//8, cb = c//CBW, t = (c%CBW)//16, w = t//4, j = t%4,
-                                         e = half + 2*(r//2) + 4*(r%2):
+                                         e = half + 2*r:
                                          UA*I/16 + ((((cb*NG + ng)*8 + uu)*NWD + w)*32 + 4*g + q)*16 + 4*j + e//2,
                                          lo = e even
       down scale of (group ng, column c): UA*I/16 + I*d/2 + ((ng*CB + cb)*NWD + w)*128 + 16*g + 4*j + 2*half
@@ -303,7 +303,7 @@ def unpack_record(rec: np.ndarray, d: int, inter: int, wdtype: str):
         ng, uu, q, r = n // 128, (n % 128) // 16, (n % 16) // 4, n % 4
         g, half, cb, t = c % 8, (c % 16) // 8, c // cbw, (c % cbw) // 16
         w, j = t // 4, t % 4
-        e = half + 2 * (r // 2) + 4 * (r % 2)
+        e = half + 2 * r
         a_down = UA * U + ((((cb * NG + ng) * 8 + uu) * nwd + w) * 32 + 4 * g + q) * 16 + 4 * j + e // 2
         s_down = UA * U + inter * d // 2 + ((ng * CB + cb) * nwd + w) * 128 + 16 * g + 4 * j + 2 * half
         wd = codes(a_down, e % 2 == 0) * bf16_at(s_down + 0 * n)

@@ -1,27 +1,30 @@
 // Steps 5+6 for int4 (group 128, bf16 scales) experts at decode-sized token counts: two HBM-streaming kernels whose
-// weight loads go straight from global memory into registers, with the group dequantisation done there, so the
-// path stays bound by the bytes it streams.
-//
-// The record is stored in tile order (include/ftmoe.h).  A 32-bit word holds 8 codes; (w >> 4k) & 0x000F000F puts
-// codes k and k+4 into the two halves of a register and XOR 0x43084308 turns them into the bf16 numbers 136 + code
-// (exact: 128..143 have one-unit spacing in bf16), i.e. one A-fragment register of mma.sync.m16n8k16 per two
-// instructions.  The constant is removed in fp32: sum (136 + c) a = 136 sum a + sum c a, with the sums of the
-// activations over a group computed once; the group scale multiplies the fp32 partial sum once per group.  Weights
-// and activations are bf16 operands, so the activation range is that of bf16.
+// weight loads go straight from global memory into registers.  At 4 bits per weight the bound next to HBM is the
+// integer/logic pipe that unpacks the codes, so the arithmetic is arranged for the cheapest unpacking there is:
+//   * a 32-bit word holds 8 two's-complement codes; (w & 0x0F0F0F0F) ^ 0x08080808 and the same of w >> 4 are two
+//     A-fragment registers of the int8 tensor-core instruction mma.sync.m16n8k32 (three logic instructions per 8
+//     weights), holding code + 8;
+//   * the bf16 activations of a (token, 128-element quantisation group) are re-expressed exactly once as 15-bit
+//     fixed point against the group's largest magnitude m:  a ~ (m / 16256) * (128 hi + lo),  hi in [-127, 127],
+//     lo in [0, 127]; hi and lo are the int8 B operands of two MMAs whose int32 sums are exact.  The representation
+//     error is at most m / 32512 per element, i.e. below the rounding of the largest element to bf16 (m / 512);
+//   * per group and output:  scale_w * ( (m / 16256) * (128 S_hi + S_lo) - 8 (m / 16256) sum(128 hi + lo) )  in fp32
+//     (the second term removes the + 8 of the codes).
 //   w4_gateup_kernel : 16 warps per SM, every warp streams whole 16-neuron units (gate tiles, up tiles and their
 //                      scales: contiguous) by itself: no partial sums to exchange, no block-level synchronisation
 //                      while a call has at most 8 tokens.  A lane's two 16-byte loads per quantisation group are rows
-//                      g and g+8 of the group's tile; a rolling buffer of 16 such loads per lane is refilled as soon
-//                      as a pair has been consumed, so about 128 KiB per SM stay in flight.  h = SiLU(g) * u goes
-//                      to a small global buffer, bf16 [pass][unit][token][neuron].
+//                      g and g+8 of the group's tile; a rolling register buffer is refilled as soon as a pair has
+//                      been consumed.  h = SiLU(g) * u goes to global memory as fp32; the warp that completes a
+//                      group of 128 neurons of a pass (an arrival counter per group; nobody waits) converts that
+//                      group to the fixed-point form above for the down kernel.
 //   w4_down_kernel   : walks chunks (expert pass, block of 64*NWD output columns, group of 128 neurons) = 8 steps
 //                      of 16 neurons x 512 bytes per warp.  Every warp owns four 16-column tiles: its 16-byte load
-//                      per step is their four A fragments; the same rolling buffer, two chunks deep.  No block-level
-//                      synchronisation: a warp stages the chunk's h fragments and scales for itself with cp.async.
-//                      Scale and bias are folded when the chunk (= one neuron group) ends; the scaled totals persist
-//                      while consecutive chunks belong to the same pass and column block.  The gate-weighted combine
-//                      is a red.global.add into the fp32 accumulator; the last CTA rounds it once to bf16.  Launched
-//                      as a programmatic dependent of the gate/up kernel: its set-up overlaps that kernel's tail.
+//                      per step is their A fragments.  No block-level synchronisation: a warp stages the chunk's h
+//                      operands and scales for itself with cp.async.  The fold to fp32 happens when the chunk (= one
+//                      neuron group) ends; the totals persist while consecutive chunks belong to the same pass and
+//                      column block.  The gate-weighted combine is a red.global.add into the fp32 accumulator; the
+//                      last CTA rounds it once to bf16.  Launched as a programmatic dependent of the gate/up
+//                      kernel: its set-up overlaps that kernel's tail.
 // Zero-copy experts (records in the mapped host pool) go through the same kernels.
 #pragma once
 #include "async.cuh"
@@ -33,10 +36,11 @@ namespace ftmoe {
 constexpr int kQ4Tokens = 8;         // tokens per weight pass
 constexpr int kW4Threads = 512;
 constexpr int kW4Warps = kW4Threads / 32;
-constexpr float kW4Bias = 136.f;
-#ifndef W4_BLOCK_PAIRS
-#define W4_BLOCK_PAIRS 4
-#endif     // the dequantised operand is 136 + code
+constexpr float kW4Levels = 16256.f; // 127 * 128: |fixed-point activation| <= this
+#ifndef W4_BS
+#define W4_BS 2
+#endif
+constexpr int kW4BlockSteps = W4_BS;     // depth of the gate/up kernel's rolling register buffer, in quantisation groups
 
 struct W4Params {
   const WorkItem *items;
@@ -47,39 +51,67 @@ struct W4Params {
   const __nv_bfloat16 *x;   // [T][d]
   const int32_t *perm;
   const float *topk_w;
-  __nv_bfloat16 *hbuf;      // [pass][16-neuron unit][token 8][neuron 16]
-  float *hbias;             // [pass][16-neuron unit][token 8]: 136 x the sum of the unit's 16 (rounded) h values
+  float *hraw;              // [pass][16-neuron unit][token 8][neuron 16] fp32
+  int32_t *hcount;          // [pass][128-neuron group]: units of the group written so far (self-resetting)
+  uint8_t *hq;              // [pass][group][unit pair 4][token 8][q 4][hi u0, hi u1, lo u0, lo u1 : 4 neurons each]
+  float2 *hs;               // [pass][group][token 8]: (m / 16256, 8 (m / 16256) sum of the fixed-point values)
   float *y_acc;             // [T][d]
   __nv_bfloat16 *y;
   uint32_t *done;
   uint32_t *status;
   int inter, top_k, T, finalize;
-  uint32_t mask, magic;     // 0x000F000F, 0x43084308 (see w4_unpack)
+  // 0x0F0F0F0F and 0x08080808, passed as data: as literals the compiler encodes both as immediates and needs two
+  // logic instructions per register (an instruction carries one immediate); as values it cannot see through they
+  // live in registers and (x & mask) ^ flip is a single three-input logic instruction
+  uint32_t mask, flip;
 };
 
-// 8 codes of one word -> four bf16x2 registers holding 136 + code: pairs (0,4) (1,5) (2,6) (3,7).
-struct W4Frag { uint32_t p04, p15, p26, p37; };
-// mask = 0x000F000F and magic = 0x43084308 arrive as kernel arguments: as literals the compiler encodes both as
-// immediates and needs two logic instructions per register (an instruction carries one immediate); as values it
-// cannot see through they live in registers and (x & mask) ^ magic is a single three-input logic instruction.
-struct W4Const { uint32_t mask, magic; };
-__device__ __forceinline__ W4Frag w4_unpack(uint32_t w, const W4Const &k) {
-  W4Frag f;
-  f.p04 = (w & k.mask) ^ k.magic;
-  f.p15 = ((w >> 4) & k.mask) ^ k.magic;
-  f.p26 = ((w >> 8) & k.mask) ^ k.magic;
-  f.p37 = ((w >> 12) & k.mask) ^ k.magic;
-  return f;
-}
-// d = a * b (no accumulator to clear first)
-__device__ __forceinline__ void mma_bf16_first(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                               uint32_t b0, uint32_t b1) {
-  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
-      : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
-}
 __device__ __forceinline__ float bf16lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
+
+__device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                       uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// d = a * b (no accumulator to clear first)
+__device__ __forceinline__ void mma_s8_first(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                             uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=r"(c[0]), "=r"(c[1]), "=r"(c[2]), "=r"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(0));
+}
+
+// 8 values of one (token, group) -> fixed point against the group's largest magnitude `m` (already reduced over the
+// group): hi/lo bytes of elements (0,2,4,6) and (1,3,5,7) -- the order in which w & 0x0F0F0F0F and (w >> 4) & ...
+// deliver the codes of a word -- and the sum of the 8 fixed-point values.
+struct W4Fixed { uint32_t hi_even, hi_odd, lo_even, lo_odd; int sum; };
+__device__ __forceinline__ W4Fixed w4_to_fixed(const float (&f)[8], float inv) {
+  int v[8];
+  W4Fixed r;
+  r.sum = 0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    v[i] = __float2int_rn(f[i] * inv);
+    r.sum += v[i];
+  }
+  auto pack = [](int a, int b, int c, int d_) {
+    return (uint32_t)(a & 0xff) | ((uint32_t)(b & 0xff) << 8) | ((uint32_t)(c & 0xff) << 16) | ((uint32_t)(d_ & 0xff) << 24);
+  };
+  r.hi_even = pack(v[0] >> 7, v[2] >> 7, v[4] >> 7, v[6] >> 7);
+  r.hi_odd = pack(v[1] >> 7, v[3] >> 7, v[5] >> 7, v[7] >> 7);
+  r.lo_even = pack(v[0] & 127, v[2] & 127, v[4] & 127, v[6] & 127);
+  r.lo_odd = pack(v[1] & 127, v[3] & 127, v[5] & 127, v[7] & 127);
+  return r;
+}
+// Scale of a group with largest magnitude m (non-finite inputs flagged by `bad`): value = scale * fixed, fixed =
+// rint(value * inv).  A non-finite input makes the scale NaN, so that it reaches the output as it would in bf16.
+__device__ __forceinline__ void w4_group_scale(float m, bool bad, float &scale, float &inv) {
+  if (bad) { scale = __int_as_float(0x7fc00000); inv = 0.f; }
+  else if (m < 1e-30f) { scale = 0.f; inv = 0.f; }
+  else { scale = m * (1.f / kW4Levels); inv = kW4Levels / m; }
+}
 
 // Share number `who` of `total` work items split over `n`: total/n each, the first total%n one more.
 __device__ __forceinline__ uint32_t w4_first(uint32_t total, uint32_t n, uint32_t who) {
@@ -96,30 +128,33 @@ __device__ __forceinline__ int w4_find_item(const int32_t *pref, int n, uint32_t
   return lo;
 }
 
-// Dynamic shared memory of the gate/up kernel: x [8][2d + 64] bytes (every run of 8 elements stored as
-// 0,4,1,5,2,6,3,7) | xbias [8][G] f32 (136 x the sum of x over a group) | items [max_items] | pref [max_items + 1].
+// Dynamic shared memory of the gate/up kernel: x [8][2d + 64] bytes (per run of 8 elements: hi bytes of elements
+// 0,2,4,6 | hi of 1,3,5,7 | lo of 0,2,4,6 | lo of 1,3,5,7) | per (token, group): scale [8][G], bias [8][G] f32 |
+// items [max_items] | pref [max_items + 1].
 inline size_t w4_gateup_smem_bytes(int max_items, int d) {
-  return (size_t)8 * (2 * d + 64) + (size_t)8 * (d / kGroup) * 4 + (size_t)max_items * sizeof(WorkItem) +
+  return (size_t)8 * (2 * d + 64) + (size_t)2 * 8 * (d / kGroup) * 4 + (size_t)max_items * sizeof(WorkItem) +
          ((size_t)max_items + 1) * 4 + 16;
 }
-// ... of the down kernel: per warp 3 slots of (h [8 units x 8 tokens x 16 neurons] bf16 | 128 bytes of scales |
-// h bias [8 units][8 tokens] f32) | items | pref.
-constexpr uint32_t kW4DownSlot = 2048 + 128 + 256;
+// ... of the down kernel: per warp 2 slots of (h operands 2048 | 128 bytes of weight scales | 64 bytes of
+// (scale, bias) per token) | items | pref.
+constexpr uint32_t kW4DownSlot = 2048 + 128 + 64;
 inline size_t w4_down_smem_bytes(int max_items) {
-  return (size_t)kW4Warps * 3 * kW4DownSlot + (size_t)max_items * sizeof(WorkItem) + ((size_t)max_items + 1) * 4 + 16;
+  return (size_t)kW4Warps * 2 * kW4DownSlot + (size_t)max_items * sizeof(WorkItem) + ((size_t)max_items + 1) * 4 + 16;
 }
 
 template <int G>   // quantisation groups of the hidden dimension: d = 128 G, G a multiple of 4
 __global__ void __launch_bounds__(kW4Threads, 1) w4_gateup_kernel(W4Params p) {
   constexpr int d = kGroup * G;
-  constexpr int kPairs = 2 * G;                     // (row g, row g+8) load pairs of a unit: G gate groups, G up groups
   constexpr uint32_t kUA = 2112u * G;               // bytes of a unit: gate tiles, up tiles, gate scales, up scales
   constexpr uint32_t kXStride = 2u * d + 64u;
-  static_assert(G % 4 == 0, "the rolling buffer holds 8 pairs");
+  constexpr int kBS = kW4BlockSteps;                // steps of a block = depth of the rolling register buffer
+  constexpr int kBlocks = G / kBS;                  // blocks of a unit
+  static_assert(G % kBS == 0, "whole blocks");
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char *s_x = smem;
-  float *s_xbias = reinterpret_cast<float *>(s_x + 8 * kXStride);          // [8][G]
-  WorkItem *s_items = reinterpret_cast<WorkItem *>(s_xbias + 8 * G);
+  float *s_sx = reinterpret_cast<float *>(s_x + 8 * kXStride);             // [8][G] m / 16256
+  float *s_xb = s_sx + 8 * G;                                              // [8][G] 8 (m / 16256) sum(fixed)
+  WorkItem *s_items = reinterpret_cast<WorkItem *>(s_xb + 8 * G);
   int32_t *s_pref = reinterpret_cast<int32_t *>(s_items + p.max_items);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -136,126 +171,203 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_gateup_kernel(W4Params p) {
   const uint32_t NBLK = (uint32_t)p.inter / 16u;
   const bool dense = p.T <= kQ4Tokens;
 
-  // x rows of the MMA columns into shared memory, every run of 8 stored as 0,4,1,5,2,6,3,7 (the order in which the
-  // dequantiser produces the codes of a word), and 136 x their sums over each quantisation group
+  // x rows of the MMA columns into shared memory as fixed point per (token, quantisation group)
   auto stage_x = [&](auto tok_of_column) {
     for (int i = tid; i < 8 * (d / 8); i += kW4Threads) {
       const int j = i / (d / 8), c8 = i - j * (d / 8);
       const int tok = tok_of_column(j);
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
       if (tok >= 0) v = *reinterpret_cast<const uint4 *>(p.x + (size_t)tok * d + 8 * c8);
-      uint4 o;
-      o.x = __byte_perm(v.x, v.z, 0x5410);   // (x0, x4)
-      o.y = __byte_perm(v.x, v.z, 0x7632);   // (x1, x5)
-      o.z = __byte_perm(v.y, v.w, 0x5410);   // (x2, x6)
-      o.w = __byte_perm(v.y, v.w, 0x7632);   // (x3, x7)
-      *reinterpret_cast<uint4 *>(s_x + j * kXStride + 16 * c8) = o;
-      float sum = bf16lo(v.x) + bf16hi(v.x) + bf16lo(v.y) + bf16hi(v.y) + bf16lo(v.z) + bf16hi(v.z) + bf16lo(v.w) +
-                  bf16hi(v.w);
+      const float f[8] = {bf16lo(v.x), bf16hi(v.x), bf16lo(v.y), bf16hi(v.y), bf16lo(v.z), bf16hi(v.z), bf16lo(v.w), bf16hi(v.w)};
+      float m = 0.f;
+      bool bad = false;
 #pragma unroll
-      for (int o2 = 1; o2 < 16; o2 <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o2);   // 16 chunks = one group
-      if ((lane & 15) == 0) s_xbias[j * G + c8 / 16] = kW4Bias * sum;
+      for (int e = 0; e < 8; ++e) {
+        m = fmaxf(m, fabsf(f[e]));
+        bad |= !(fabsf(f[e]) <= 3.0e38f);
+      }
+#pragma unroll
+      for (int o2 = 1; o2 < 16; o2 <<= 1) {   // 16 chunks = one group
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o2));
+        bad |= __shfl_xor_sync(0xffffffffu, (int)bad, o2) != 0;
+      }
+      float scale, inv;
+      w4_group_scale(m, bad, scale, inv);
+      const W4Fixed fx = w4_to_fixed(f, inv);
+      *reinterpret_cast<uint4 *>(s_x + j * kXStride + 16 * c8) = make_uint4(fx.hi_even, fx.hi_odd, fx.lo_even, fx.lo_odd);
+      int sum = fx.sum;
+#pragma unroll
+      for (int o2 = 1; o2 < 16; o2 <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o2);
+      if ((lane & 15) == 0) {
+        s_sx[j * G + c8 / 16] = scale;
+        s_xb[j * G + c8 / 16] = 8.f * (float)sum * scale;
+      }
     }
   };
 
   const uint32_t my_x = smem_u32(s_x) + g * kXStride + 16u * q;
-  const float *my_b0 = s_xbias + (2 * q) * G, *my_b1 = s_xbias + (2 * q + 1) * G;
+  const uint32_t km = p.mask, kf = p.flip;
+  const float *my_s0 = s_sx + (2 * q) * G, *my_s1 = s_sx + (2 * q + 1) * G;
+  const float *my_b0 = s_xb + (2 * q) * G, *my_b1 = s_xb + (2 * q + 1) * G;
 
-  const W4Const ks = {p.mask, p.magic};
+  // The warp that completes a group of 128 neurons of a pass converts it to fixed point for the down kernel:
+  // lane = (token, quarter): the quarter's two units of 16 neurons.
+  auto convert_group = [&](uint32_t grp) {
+    const int tok = lane >> 2, qt = lane & 3;
+    const float *src = p.hraw + ((size_t)grp * 8 + 2 * qt) * 128 + tok * 16;
+    float v[2][16];
+#pragma unroll
+    for (int u = 0; u < 2; ++u)
+#pragma unroll
+      for (int k4 = 0; k4 < 4; ++k4) {
+        const float4 t = __ldcg(reinterpret_cast<const float4 *>(src + u * 128) + k4);
+        v[u][4 * k4] = t.x; v[u][4 * k4 + 1] = t.y; v[u][4 * k4 + 2] = t.z; v[u][4 * k4 + 3] = t.w;
+      }
+    float m = 0.f;
+    bool bad = false;
+#pragma unroll
+    for (int u = 0; u < 2; ++u)
+#pragma unroll
+      for (int k = 0; k < 16; ++k) {
+        m = fmaxf(m, fabsf(v[u][k]));
+        bad |= !(fabsf(v[u][k]) <= 3.0e38f);
+      }
+#pragma unroll
+    for (int o = 1; o < 4; o <<= 1) {   // the token's four quarters
+      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      bad |= __shfl_xor_sync(0xffffffffu, (int)bad, o) != 0;
+    }
+    float scale, inv;
+    w4_group_scale(m, bad, scale, inv);
+    int sum = 0;
+    uint8_t *dst = p.hq + (size_t)grp * 2048 + qt * 512 + tok * 64;
+#pragma unroll
+    for (int qq = 0; qq < 4; ++qq) {   // neurons 4qq..4qq+3 of both units: (hi u0, hi u1, lo u0, lo u1)
+      int w[8];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        w[k] = __float2int_rn(v[0][4 * qq + k] * inv);
+        w[4 + k] = __float2int_rn(v[1][4 * qq + k] * inv);
+      }
+      uint32_t o[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        sum += w[k] + w[4 + k];
+        o[0] |= (uint32_t)((w[k] >> 7) & 0xff) << (8 * k);
+        o[1] |= (uint32_t)((w[4 + k] >> 7) & 0xff) << (8 * k);
+        o[2] |= (uint32_t)(w[k] & 127) << (8 * k);
+        o[3] |= (uint32_t)(w[4 + k] & 127) << (8 * k);
+      }
+      *reinterpret_cast<uint4 *>(dst + qq * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+    sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+    sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+    if (qt == 0) p.hs[(size_t)grp * 8 + tok] = make_float2(scale, 8.f * (float)sum * scale);
+  };
+
   // One warp streams `n_units` consecutive units starting at `base`; their h goes to rows hrow0.. of the h buffer.
-  // Work proceeds in blocks of 8 (row g, row g+8) load pairs = 8 quantisation groups of the gate or the up part.
-  constexpr int kBP = W4_BLOCK_PAIRS;               // pairs of a block = depth of the rolling register buffer
-  constexpr int kBlocks = kPairs / kBP;             // blocks of a unit
-  static_assert(G % kBP == 0, "a block lies in the gate or in the up part");
+  // A step is one quantisation group of the hidden dimension: the gate tile and the up tile of that group, which
+  // share their activation fragments.  Registers hold kBS steps; a step's registers are refilled with the step
+  // kBS further on as soon as it has been consumed.
   auto run = [&](const uint8_t *base, int n_units, uint32_t hrow0) {
-    uint4 buf[2 * kBP];
-    uint32_t sc[kBP];   // and the two rows' scales
-    const uint8_t *nptr = base + g * 64 + q * 16;              // next block to request
+    uint4 buf[4 * kBS];     // per step: gate rows g, g+8; up rows g, g+8
+    uint32_t sc[2 * kBS];   // and their scales
+    const uint8_t *nptr = base + g * 64 + q * 16;              // next block to request (its gate tiles)
     const uint8_t *nsc = base + 2048u * G + g * 4;
     int nblk = 0, blocks_left = n_units * kBlocks;             // its index in its unit; blocks not yet requested
     auto advance = [&]() {
-      nptr += kBP * 1024;
-      nsc += kBP * 32;
+      nptr += kBS * 1024;
+      nsc += kBS * 32;
       --blocks_left;
-      if (++nblk == kBlocks) {   // on to the next unit: skip this unit's scales / the next unit's tiles
+      if (++nblk == kBlocks) {   // on to the next unit
         nblk = 0;
-        nptr += 64 * G;
-        nsc += 2048u * G;
+        nptr += kUA - 1024u * G;
+        nsc += kUA - 32u * G;
       }
     };
+    auto request = [&](int si, const uint8_t *tp, const uint8_t *sp) {
+      buf[4 * si] = ld_stream_16(tp + si * 1024);
+      buf[4 * si + 1] = ld_stream_16(tp + si * 1024 + 512);
+      buf[4 * si + 2] = ld_stream_16(tp + si * 1024 + 1024 * G);
+      buf[4 * si + 3] = ld_stream_16(tp + si * 1024 + 1024 * G + 512);
+      asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(sc[2 * si]) : "l"(sp + si * 32));
+      asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(sc[2 * si + 1]) : "l"(sp + si * 32 + 32 * G));
+    };
 #pragma unroll
-    for (int pi = 0; pi < kBP; ++pi) {
-      buf[2 * pi] = ld_stream_16(nptr + pi * 1024);
-      buf[2 * pi + 1] = ld_stream_16(nptr + pi * 1024 + 512);
-      asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(sc[pi]) : "l"(nsc + pi * 32));
-    }
+    for (int si = 0; si < kBS; ++si) request(si, nptr, nsc);
     advance();
     for (int u = 0; u < n_units; ++u) {
-      float tot[4] = {0.f, 0.f, 0.f, 0.f}, tg[4] = {0.f, 0.f, 0.f, 0.f};
-      int xg = 0;                                    // first group of the block
+      float tg[4] = {0.f, 0.f, 0.f, 0.f}, tot[4] = {0.f, 0.f, 0.f, 0.f};   // gate sums, up sums
       for (int blk = 0; blk < kBlocks; ++blk) {
         const bool more = blocks_left > 0;
         const uint8_t *rp = nptr, *rs = nsc;         // the block that refills this one's registers
         if (more) advance();
+        const int xg = blk * kBS;                    // first group of the block
         const uint32_t xa = my_x + xg * 256u;
-        const float *b0p = my_b0 + xg, *b1p = my_b1 + xg;
 #pragma unroll
-        for (int pi = 0; pi < kBP; ++pi) {
-          float a1[4], a2[4];
-          const uint32_t lo[4] = {buf[2 * pi].x, buf[2 * pi].y, buf[2 * pi].z, buf[2 * pi].w};
-          const uint32_t hi[4] = {buf[2 * pi + 1].x, buf[2 * pi + 1].y, buf[2 * pi + 1].z, buf[2 * pi + 1].w};
-          const uint32_t scale = sc[pi];
+        for (int si = 0; si < kBS; ++si) {
+          int gh[4], gl[4], uh[4], ul[4];
+          const uint32_t glo[4] = {buf[4 * si].x, buf[4 * si].y, buf[4 * si].z, buf[4 * si].w};
+          const uint32_t ghi[4] = {buf[4 * si + 1].x, buf[4 * si + 1].y, buf[4 * si + 1].z, buf[4 * si + 1].w};
+          const uint32_t ulo[4] = {buf[4 * si + 2].x, buf[4 * si + 2].y, buf[4 * si + 2].z, buf[4 * si + 2].w};
+          const uint32_t uhi[4] = {buf[4 * si + 3].x, buf[4 * si + 3].y, buf[4 * si + 3].z, buf[4 * si + 3].w};
+          const uint32_t gscale = sc[2 * si], uscale = sc[2 * si + 1];
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {   // word j: hidden indices 32j + 8q + 0..7 of the group
-            const W4Frag fl = w4_unpack(lo[j], ks), fh = w4_unpack(hi[j], ks);
-            const uint4 xv = lds_v4(xa + pi * 256u + j * 64u);
+          for (int j = 0; j < 4; ++j) {   // word j: hidden indices 32j + 8q + 0..7 of the group, rows g and g+8
+            const uint4 xv = lds_v4(xa + si * 256u + j * 64u);
+            const uint32_t a0 = (glo[j] & km) ^ kf, a1 = (ghi[j] & km) ^ kf;
+            const uint32_t a2 = ((glo[j] >> 4) & km) ^ kf, a3 = ((ghi[j] >> 4) & km) ^ kf;
+            const uint32_t c0 = (ulo[j] & km) ^ kf, c1 = (uhi[j] & km) ^ kf;
+            const uint32_t c2 = ((ulo[j] >> 4) & km) ^ kf, c3 = ((uhi[j] >> 4) & km) ^ kf;
             if (j == 0) {
-              mma_bf16_first(a1, fl.p04, fh.p04, fl.p15, fh.p15, xv.x, xv.y);
-              mma_bf16_first(a2, fl.p26, fh.p26, fl.p37, fh.p37, xv.z, xv.w);
+              mma_s8_first(gh, a0, a1, a2, a3, xv.x, xv.y);
+              mma_s8_first(gl, a0, a1, a2, a3, xv.z, xv.w);
+              mma_s8_first(uh, c0, c1, c2, c3, xv.x, xv.y);
+              mma_s8_first(ul, c0, c1, c2, c3, xv.z, xv.w);
             } else {
-              mma_bf16(a1, fl.p04, fh.p04, fl.p15, fh.p15, xv.x, xv.y);
-              mma_bf16(a2, fl.p26, fh.p26, fl.p37, fh.p37, xv.z, xv.w);
+              mma_s8(gh, a0, a1, a2, a3, xv.x, xv.y);
+              mma_s8(gl, a0, a1, a2, a3, xv.z, xv.w);
+              mma_s8(uh, c0, c1, c2, c3, xv.x, xv.y);
+              mma_s8(ul, c0, c1, c2, c3, xv.z, xv.w);
             }
           }
-          if (more) {   // refill the pair just consumed
-            buf[2 * pi] = ld_stream_16(rp + pi * 1024);
-            buf[2 * pi + 1] = ld_stream_16(rp + pi * 1024 + 512);
-            asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(sc[pi]) : "l"(rs + pi * 32));
+          if (more) request(si, rp, rs);   // refill the step just consumed
+          const float sx0 = my_s0[xg + si], sx1 = my_s1[xg + si], b0 = my_b0[xg + si], b1 = my_b1[xg + si];
+          {
+            const float s_lo = bf16lo(gscale), s_hi = bf16hi(gscale);
+            tg[0] += s_lo * ((float)(gh[0] * 128 + gl[0]) * sx0 - b0);
+            tg[1] += s_lo * ((float)(gh[1] * 128 + gl[1]) * sx1 - b1);
+            tg[2] += s_hi * ((float)(gh[2] * 128 + gl[2]) * sx0 - b0);
+            tg[3] += s_hi * ((float)(gh[3] * 128 + gl[3]) * sx1 - b1);
           }
-          const float s_lo = bf16lo(scale), s_hi = bf16hi(scale);
-          const float b0 = b0p[pi], b1 = b1p[pi];
-          tot[0] += s_lo * (a1[0] + a2[0] - b0);
-          tot[1] += s_lo * (a1[1] + a2[1] - b1);
-          tot[2] += s_hi * (a1[2] + a2[2] - b0);
-          tot[3] += s_hi * (a1[3] + a2[3] - b1);
-        }
-        xg += kBP;
-        if (xg == G) {
-          xg = 0;
-          if (blk < kBlocks - 1) {   // the gate sums are complete: the up groups follow
-#pragma unroll
-            for (int i = 0; i < 4; ++i) { tg[i] = tot[i]; tot[i] = 0.f; }
+          {
+            const float s_lo = bf16lo(uscale), s_hi = bf16hi(uscale);
+            tot[0] += s_lo * ((float)(uh[0] * 128 + ul[0]) * sx0 - b0);
+            tot[1] += s_lo * ((float)(uh[1] * 128 + ul[1]) * sx1 - b1);
+            tot[2] += s_hi * ((float)(uh[2] * 128 + ul[2]) * sx0 - b0);
+            tot[3] += s_hi * ((float)(uh[3] * 128 + ul[3]) * sx1 - b1);
           }
         }
       }
-      // h = SiLU(gate) * up of neurons g, g+8 and tokens 2q, 2q+1, rounded to bf16; and 136 x its sums over the
-      // unit's 16 neurons, which the down kernel subtracts
-      __nv_bfloat16 *hrow = p.hbuf + ((size_t)hrow0 + u) * 128;
-      float hr[4];
+      // h = SiLU(gate) * up of neurons g, g+8 and tokens 2q, 2q+1
+      const uint32_t hrow_i = hrow0 + u;
+      float *hrow = p.hraw + (size_t)hrow_i * 128;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const float a = tg[i];
-        const __nv_bfloat16 hv = __float2bfloat16_rn(__fdividef(a, 1.f + __expf(-a)) * tot[i]);
-        hrow[(2 * q + (i & 1)) * 16 + g + 8 * (i >> 1)] = hv;
-        hr[i] = __bfloat162float(hv);
+        hrow[(2 * q + (i & 1)) * 16 + g + 8 * (i >> 1)] = __fdividef(a, 1.f + __expf(-a)) * tot[i];
       }
-      float s0 = hr[0] + hr[2], s1 = hr[1] + hr[3];
-#pragma unroll
-      for (int o = 4; o < 32; o <<= 1) {
-        s0 += __shfl_xor_sync(0xffffffffu, s0, o);
-        s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+      // the 8th unit of a 128-neuron group to arrive converts the group (units of a group are consecutive rows)
+      __threadfence();
+      __syncwarp();
+      int old = 0;
+      if (lane == 0) old = atomicAdd(p.hcount + (hrow_i >> 3), 1);
+      old = __shfl_sync(0xffffffffu, old, 0);
+      if (old == 7) {
+        __threadfence();
+        convert_group(hrow_i >> 3);
+        if (lane == 0) p.hcount[hrow_i >> 3] = 0;
       }
-      if (g == 0) *reinterpret_cast<float2 *>(p.hbias + ((size_t)hrow0 + u) * 8 + 2 * q) = make_float2(kW4Bias * s0, kW4Bias * s1);
     }
   };
 
@@ -297,8 +409,8 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_gateup_kernel(W4Params p) {
 template <int NWD>   // warps that own output columns: a column block is 64 * NWD columns
 __global__ void __launch_bounds__(kW4Threads, 1) w4_down_kernel(W4Params p, int d) {
   extern __shared__ __align__(128) unsigned char smem[];
-  unsigned char *s_h = smem;                                                // [16 warps][3][h 2048 | scales 128]
-  WorkItem *s_items = reinterpret_cast<WorkItem *>(smem + kW4Warps * 3 * kW4DownSlot);
+  unsigned char *s_h = smem;                                                // [16 warps][2 slots]
+  WorkItem *s_items = reinterpret_cast<WorkItem *>(smem + kW4Warps * 2 * kW4DownSlot);
   int32_t *s_pref = reinterpret_cast<int32_t *>(s_items + p.max_items);
   __shared__ int s_last;
 
@@ -326,34 +438,44 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_down_kernel(W4Params p, int 
     const uint32_t rfirst0 = w4_first(t0, gridDim.x, blockIdx.x), rcount0 = w4_first(t0, gridDim.x, blockIdx.x + 1) - rfirst0;
     const uint32_t rfirst1 = t0 + w4_first(t1, gridDim.x, blockIdx.x);
     const uint32_t rcount1 = t0 + w4_first(t1, gridDim.x, blockIdx.x + 1) - rfirst1;
-    const uint32_t my_h = smem_u32(s_h) + (uint32_t)warp * 3u * kW4DownSlot;
-    const W4Const ks = {p.mask, p.magic};
+    const uint32_t my_h = smem_u32(s_h) + (uint32_t)warp * 2u * kW4DownSlot;
+    const uint32_t km = p.mask, kf = p.flip;
 
-    // chunk cursor: (pass pu, column block cb, neuron group ng)
+    // chunk cursor: (pass pu, column block cb, neuron group ng), advanced without divisions
     struct Ck { const uint8_t *rec; uint32_t pu, cb, ng; int item; };
     int range = 0, item = 0;
-    uint32_t cur = 0, left = 0;
+    uint32_t left = 0;
+    Ck cur;
+    cur.pu = cur.cb = cur.ng = 0; cur.item = 0; cur.rec = nullptr;
     auto next_chunk = [&](Ck &c) -> bool {
-      while (left == 0) {
-        if (range == 2) return false;
-        left = range ? rcount1 : rcount0;
-        cur = range ? rfirst1 : rfirst0;
-        ++range;
+      if (left == 0) {
+        while (left == 0) {
+          if (range == 2) return false;
+          left = range ? rcount1 : rcount0;
+          const uint32_t first = range ? rfirst1 : rfirst0;
+          ++range;
+          if (left) {
+            cur.pu = first / per_pass;
+            const uint32_t r = first - cur.pu * per_pass;
+            cur.cb = r / NG;
+            cur.ng = r - cur.cb * NG;
+          }
+        }
+      } else if (++cur.ng == NG) {
+        cur.ng = 0;
+        if (++cur.cb == CB) { cur.cb = 0; ++cur.pu; }
       }
-      c.pu = cur / per_pass;
-      const uint32_t r = cur - c.pu * per_pass;
-      c.cb = r / NG;
-      c.ng = r - c.cb * NG;
-      while ((uint32_t)s_pref[item + 1] <= c.pu) ++item;
-      c.item = item;
-      c.rec = s_items[item].w;
-      ++cur;
+      while ((uint32_t)s_pref[item + 1] <= cur.pu) ++item;
+      cur.item = item;
+      cur.rec = s_items[item].w;
+      c = cur;
       --left;
       return true;
     };
-    // h of the chunk's 8 units (2 KiB, contiguous) and the chunk's scales for this warp alone
+    // the chunk's h operands (2 KiB, contiguous), its weight scales and the per-token (scale, bias) for this warp alone
     auto stage = [&](const Ck &c, uint32_t slot) {
-      const unsigned char *hsrc = reinterpret_cast<const unsigned char *>(p.hbuf) + ((size_t)c.pu * NBLK + c.ng * 8u) * 256u;
+      const size_t grp = (size_t)c.pu * NG + c.ng;
+      const uint8_t *hsrc = p.hq + grp * 2048;
       const uint32_t dst = my_h + slot * kW4DownSlot;
 #pragma unroll
       for (int i = 0; i < 4; ++i)
@@ -363,9 +485,9 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_down_kernel(W4Params p, int 
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 2048u + lane * 16u),
                      "l"(c.rec + sec_c + ((size_t)(c.ng * CB + c.cb) * NWD + warp) * 128u + lane * 16u)
                      : "memory");
-      else if (lane < 24)
+      else if (lane < 12)
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 2176u + (lane - 8) * 16u),
-                     "l"(reinterpret_cast<const unsigned char *>(p.hbias) + ((size_t)c.pu * NBLK + c.ng * 8u) * 32u + (lane - 8) * 16)
+                     "l"(reinterpret_cast<const uint8_t *>(p.hs + grp * 8) + (lane - 8) * 16)
                      : "memory");
     };
     auto weights_of = [&](const Ck &c) -> const uint8_t * {
@@ -428,84 +550,73 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_down_kernel(W4Params p, int 
         }
       }
     };
-    // one chunk: 8 steps of 16 neurons for the warp's four column tiles, then scale and bias; every step's
-    // register is refilled with the same step of the chunk two ahead as soon as it has been consumed
-    auto consume = [&](uint4 (&buf)[8], uint32_t slot, const uint8_t *refill) {
-      asm volatile("cp.async.wait_group 2;" ::: "memory");   // this chunk's h, scales and biases have landed
-      __syncwarp();
-      const uint32_t hs_base = my_h + slot * kW4DownSlot;
-      float acc[4][4];
-#pragma unroll
-      for (int uu = 0; uu < 8; ++uu) {
-        uint2 hb;   // h of token g, neurons 4q..4q+3 of the step
-        asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(hb.x), "=r"(hb.y) : "r"(hs_base + uu * 256u + g * 32u + q * 8u));
-        const uint32_t wv[4] = {buf[uu].x, buf[uu].y, buf[uu].z, buf[uu].w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const W4Frag f = w4_unpack(wv[j], ks);
-          if (uu == 0) mma_bf16_first(acc[j], f.p04, f.p15, f.p26, f.p37, hb.x, hb.y);
-          else mma_bf16(acc[j], f.p04, f.p15, f.p26, f.p37, hb.x, hb.y);
-        }
-        if (refill) buf[uu] = ld_stream_16(refill + (size_t)uu * NWD * 512u);
-      }
-      const uint4 sc = lds_v4(hs_base + 2048u + g * 16u);   // (column g, column g + 8) of the warp's four tiles
-      float b0 = 0.f, b1 = 0.f;                             // 136 x the sums of h over the chunk's 128 neurons
-#pragma unroll
-      for (int uu = 0; uu < 8; ++uu) {
-        float2 hb2;
-        asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(hb2.x), "=f"(hb2.y) : "r"(hs_base + 2176u + uu * 32u + q * 8u));
-        b0 += hb2.x;
-        b1 += hb2.y;
-      }
-      __syncwarp();   // every lane has read the slot: it may be overwritten
-      const uint32_t sw[4] = {sc.x, sc.y, sc.z, sc.w};
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const float s_lo = bf16lo(sw[j]), s_hi = bf16hi(sw[j]);
-        dtot[j][0] += s_lo * (acc[j][0] - b0);
-        dtot[j][1] += s_lo * (acc[j][1] - b1);
-        dtot[j][2] += s_hi * (acc[j][2] - b0);
-        dtot[j][3] += s_hi * (acc[j][3] - b1);
-      }
-    };
 
-    uint4 bufa[8], bufb[8];   // even / odd chunks of this CTA's sequence
-    Ck c0, c1, c2;            // the chunk being consumed and the two after it
-    bool h0 = next_chunk(c0), h1 = h0 && next_chunk(c1), h2 = h1 && next_chunk(c2);
+    uint4 buf[8];             // the chunk's eight steps; a step's register is refilled with the same step of the
+                              // next chunk as soon as it has been consumed
+    Ck c0, c1;                // the chunk being consumed and the one after it
+    bool h0 = next_chunk(c0), h1 = h0 && next_chunk(c1);
     if (h0) {
       stage(c0, 0);
       const uint8_t *w = weights_of(c0);
 #pragma unroll
-      for (int uu = 0; uu < 8; ++uu) bufa[uu] = ld_stream_16(w + (size_t)uu * NWD * 512u);
+      for (int uu = 0; uu < 8; ++uu) buf[uu] = ld_stream_16(w + (size_t)uu * NWD * 512u);
       begin_pass(c0);
       zero_tot();
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
-    if (h1) {
-      stage(c1, 1);
-      const uint8_t *w = weights_of(c1);
-#pragma unroll
-      for (int uu = 0; uu < 8; ++uu) bufb[uu] = ld_stream_16(w + (size_t)uu * NWD * 512u);
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
     uint32_t slot = 0;
-    int half = 0;
     while (h0) {
-      const uint32_t slot2 = slot >= 1 ? slot - 1 : 2;   // (slot + 2) % 3
-      if (h2) stage(c2, slot2);
+      if (h1) stage(c1, slot ^ 1u);
       asm volatile("cp.async.commit_group;" ::: "memory");
-      const uint8_t *refill = h2 ? weights_of(c2) : nullptr;
-      if (half == 0) consume(bufa, slot, refill); else consume(bufb, slot, refill);
+      const uint8_t *refill = h1 ? weights_of(c1) : nullptr;
+      asm volatile("cp.async.wait_group 1;" ::: "memory");   // this chunk's staged data have landed
+      __syncwarp();
+      const uint32_t hs_base = my_h + slot * kW4DownSlot;
+      int ah[4][4], al[4][4];
+#pragma unroll
+      for (int m = 0; m < 4; ++m) {   // unit pair m: neurons 32m .. 32m+31 of the group
+        const uint4 hv = lds_v4(hs_base + m * 512u + g * 64u + q * 16u);   // token g: (hi u0, hi u1, lo u0, lo u1)
+        const uint32_t w0[4] = {buf[2 * m].x, buf[2 * m].y, buf[2 * m].z, buf[2 * m].w};
+        const uint32_t w1[4] = {buf[2 * m + 1].x, buf[2 * m + 1].y, buf[2 * m + 1].z, buf[2 * m + 1].w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {   // tile j: columns g (even codes) and g+8 (odd codes)
+          const uint32_t a0 = (w0[j] & km) ^ kf, a1 = ((w0[j] >> 4) & km) ^ kf;
+          const uint32_t a2 = (w1[j] & km) ^ kf, a3 = ((w1[j] >> 4) & km) ^ kf;
+          if (m == 0) {
+            mma_s8_first(ah[j], a0, a1, a2, a3, hv.x, hv.y);
+            mma_s8_first(al[j], a0, a1, a2, a3, hv.z, hv.w);
+          } else {
+            mma_s8(ah[j], a0, a1, a2, a3, hv.x, hv.y);
+            mma_s8(al[j], a0, a1, a2, a3, hv.z, hv.w);
+          }
+        }
+        if (refill) {
+          buf[2 * m] = ld_stream_16(refill + (size_t)(2 * m) * NWD * 512u);
+          buf[2 * m + 1] = ld_stream_16(refill + (size_t)(2 * m + 1) * NWD * 512u);
+        }
+      }
+      const uint4 sc = lds_v4(hs_base + 2048u + g * 16u);   // (column g, column g + 8) of the warp's four tiles
+      const uint4 tb = lds_v4(hs_base + 2176u + q * 16u);   // tokens 2q, 2q+1: (scale, bias) each
+      __syncwarp();   // every lane has read the slot: it may be overwritten
+      const float sh0 = __uint_as_float(tb.x), b0 = __uint_as_float(tb.y), sh1 = __uint_as_float(tb.z), b1 = __uint_as_float(tb.w);
+      const uint32_t sw[4] = {sc.x, sc.y, sc.z, sc.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float s_lo = bf16lo(sw[j]), s_hi = bf16hi(sw[j]);
+        dtot[j][0] += s_lo * ((float)(ah[j][0] * 128 + al[j][0]) * sh0 - b0);
+        dtot[j][1] += s_lo * ((float)(ah[j][1] * 128 + al[j][1]) * sh1 - b1);
+        dtot[j][2] += s_hi * ((float)(ah[j][2] * 128 + al[j][2]) * sh0 - b0);
+        dtot[j][3] += s_hi * ((float)(ah[j][3] * 128 + al[j][3]) * sh1 - b1);
+      }
       if (!h1 || c1.pu != c0.pu || c1.cb != c0.cb) {
         flush(c0.cb);
         zero_tot();
         if (h1 && c1.pu != c0.pu) begin_pass(c1);
       }
-      c0 = c1; c1 = c2;
-      h0 = h1; h1 = h2;
-      h2 = h1 && next_chunk(c2);
-      slot = slot == 2 ? 0 : slot + 1;
-      half ^= 1;
+      c0 = c1;
+      h0 = h1;
+      h1 = h0 && next_chunk(c1);
+      slot ^= 1u;
     }
   }
 

@@ -88,8 +88,12 @@ struct ft_moe {
   uint32_t *seq_dev = nullptr;
   uint32_t *done_dev = nullptr;          // CTA completion counter of the streaming MMA kernel
   long long *trace_dev = nullptr;        // per-CTA clocks of the latest streaming-kernel launch
-  float *w4_hbias = nullptr;             // int4 path: 136 x the sums of h over each unit, [pass][unit][token 8]
-  __nv_bfloat16 *w4_hbuf = nullptr;      // int4 path: h as [pass][16-neuron unit][token 8][neuron 16]
+  // int4 path: h as fp32 [pass][16-neuron unit][token 8][neuron 16]; arrival counters, fixed-point h and its
+  // (scale, bias) per (pass, 128-neuron group)
+  float *w4_hraw = nullptr;
+  int32_t *w4_hcount = nullptr;
+  uint8_t *w4_hq = nullptr;
+  float2 *w4_hs = nullptr;
   int last_fill_layer = -1;
   int overlap = 0;                      // launch mode of the streaming kernel (see FfnStreamParams::overlap)
   float *stage_logits = nullptr;
@@ -427,8 +431,10 @@ ft_status_t ft_moe_destroy(ft_moe_t *h) {
   cudaFree(h->status_dev);
   cudaFree(h->seq_dev);
   cudaFree(h->done_dev);
-  cudaFree(h->w4_hbuf);
-  cudaFree(h->w4_hbias);
+  cudaFree(h->w4_hraw);
+  cudaFree(h->w4_hcount);
+  cudaFree(h->w4_hq);
+  cudaFree(h->w4_hs);
   cudaFree(h->trace_dev);
   cudaFree(h->stage_logits);
   cudaFree(h->stage_x);
@@ -588,8 +594,11 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
   FT_TRY(cudaFuncSetAttribute(fill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFillStages * (int)kFillChunk));
   if (c.wdtype == FT_W_INT4_G128) {
     const size_t passes = (P + 7) / 8 + 2 * E + 2;
-    FT_TRY(cudaMalloc(&h->w4_hbuf, passes * (c.inter / 16) * 256));
-    FT_TRY(cudaMalloc(&h->w4_hbias, passes * (c.inter / 16) * 32));
+    FT_TRY(cudaMalloc(&h->w4_hraw, passes * (c.inter / 16) * 512));
+    FT_TRY(cudaMalloc(&h->w4_hcount, passes * (c.inter / 128) * 4));
+    FT_TRY(cudaMemset(h->w4_hcount, 0, passes * (c.inter / 128) * 4));
+    FT_TRY(cudaMalloc(&h->w4_hq, passes * (c.inter / 128) * 2048));
+    FT_TRY(cudaMalloc(&h->w4_hs, passes * (c.inter / 128) * 64));
     // (limits are per function and device, not per handle: always the largest a CTA can have, and the handle's own
     // need is checked against it)
     const int sa = 232448, sb = (int)w4_down_smem_bytes(2 * kMaxExperts + 1);
@@ -1012,8 +1021,8 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   qp.pref = sc.res_pref;
   qp.max_items = 2 * c.n_experts + 1;
   qp.x = x_bf; qp.perm = sc.perm; qp.topk_w = sc.topk_w;
-  qp.hbuf = h->w4_hbuf; qp.hbias = h->w4_hbias;
-  qp.mask = 0x000F000Fu; qp.magic = 0x43084308u;
+  qp.mask = 0x0F0F0F0Fu; qp.flip = 0x08080808u;
+  qp.hraw = h->w4_hraw; qp.hcount = h->w4_hcount; qp.hq = h->w4_hq; qp.hs = h->w4_hs;
   qp.y_acc = h->y_acc; qp.y = static_cast<__nv_bfloat16 *>(y_dev);
   qp.done = h->done_dev; qp.status = h->status_dev;
   qp.inter = c.inter; qp.top_k = c.top_k; qp.T = L.T;

@@ -31,7 +31,7 @@ flattened identifier of Sec. 4.2 of the paper):
              ``ng`` and 16-neuron step ``uu`` of the group: ``CBW/64`` x 512 bytes; in each 512 bytes lane
              ``l = 4g + q`` owns 16 bytes = 4 words, word ``j`` belongs to the 16-column tile ``4w + j`` of the
              block; its nibble ``e`` is the code of column ``g + 8*(e & 1)`` of the tile and neuron
-             ``4q + NU[e]`` of the step, ``NU = (0, 0, 2, 2, 1, 1, 3, 3)``.
+             ``4q + e // 2`` of the step.
           C. down scales ``sd[ng][column]`` in the order (ng, cb, w, g, j, half): 8 pairs per tile again.
           ``S = 3*I*d/2 + (2*I*d/128 + (I/128)*d)*2``.
 
@@ -140,7 +140,7 @@ def _pack_nibbles(q: torch.Tensor) -> torch.Tensor:
     return u[..., 0::2] | (u[..., 1::2] << 4)
 
 
-WD_NU = (0, 0, 2, 2, 1, 1, 3, 3)     # neuron offset (plus 4q) of nibble e in a word of the down section
+WD_NU = (0, 0, 1, 1, 2, 2, 3, 3)     # neuron offset (plus 4q) of nibble e in a word of the down section
 
 
 def _pack_int4_record(qg, qu, qd, sg, su, sd) -> torch.Tensor:

@@ -53,7 +53,7 @@ def _record_int4_by_definition(qg, qu, qd, sg, su, sd):
     G, NG, U = d // 128, I // 128, I // 16
     nwd = min(16, d // 64)
     cbw, CB = 64 * nwd, d // (64 * nwd)
-    NU = (0, 0, 2, 2, 1, 1, 3, 3)
+    NU = (0, 0, 1, 1, 2, 2, 3, 3)                         # nibble e: neuron 4q + e//2, column g + 8*(e%2)
     out = bytearray()
 
     def word(nibbles):
