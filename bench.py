@@ -510,7 +510,7 @@ def run_ours(args):
             "gpu_launches": main["launches"],
             "roofline": {
                 "bound": "hbm",
-                "kernel": ("q4_gateup_kernel + q4_down_kernel (one pass over each record)" if dsv3
+                "kernel": ("w4_gateup_kernel + w4_down_kernel (one pass over each record)" if dsv3
                            else "ffn_stream_kernel (expert FFN over the HBM-resident records of a layer)"),
                 "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
                 "frac": achieved / hbm_peak if hbm_peak else None, "peak_source": peak_kind + " (burst: kernel timed alone)",
@@ -569,7 +569,7 @@ def run_ours(args):
     if rank == 0:
         if world == 1 and not dsv3 and args.layers == 48:
             # bounded sub-records of the other single-GPU configurations (a few layers each)
-            for name in [n for n in args.sub.split(",") if n]:
+            for name in [n for n in args.sub.split(",") if n and n != "none"]:
                 t_sub = time.perf_counter()
                 try:
                     line[name] = SUBRECORDS[name](args, dev, cal)
@@ -886,7 +886,8 @@ def run_sweep(args):
             cal = m0.calibrate()
             m0.destroy()
         moe = Bd.FtMoe(Bd.make_config(bw_fill=max(cal["fill_MBps"], 1), bw_zc=max(cal["zc_MBps"], 1),
-                                      bw_zc_residual=0, bw_hbm=max(cal["hbm_MBps"], 1), **common))
+                                      bw_zc_residual=cal["zc_residual_MBps"] if args.residual else 0,
+                                      bw_hbm=max(cal["hbm_MBps"], 1), **common))
         for rho in rhos:
             for batch in batches:
                 lg = torch.from_numpy(W.ar1_logits(L, steps, batch, E, rho, ALPHA, SEED)).to(dev)
@@ -923,7 +924,8 @@ def run_sweep(args):
     line = {"metric": "moe_decode_sweep", "unit": "tok/s", "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": "cache-pressure sweep on the decode shapes (config 4)", "layers": L,
                        "hidden": d, "experts": E, "inter": shape.inter, "top_k": k, "fill_mode": args.fill,
-                       "zipf_alpha": ALPHA, "steps_per_point": steps, "cold_start": True},
+                       "zipf_alpha": ALPHA, "steps_per_point": steps, "cold_start": True,
+                       "plan_uses_residual_zero_copy_rate": bool(args.residual)},
             "link_GBps_measured": cal["fill_MBps"] / 1e3, "points": points}
     print(json.dumps(line), flush=True)
     pool.free()

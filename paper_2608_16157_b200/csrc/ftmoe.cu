@@ -68,7 +68,7 @@ struct ft_moe {
   size_t pair_stride = 0, plan_stride = 0;   // bytes per layer of the pair arrays / the plan record
   int32_t *ids = nullptr, *count = nullptr, *offset = nullptr, *perm = nullptr, *inv = nullptr;
   float *topk_w = nullptr;
-  int32_t *route_hist = nullptr;        // [blocks of 128 tokens][E] histograms of the blocked route / permute kernels
+  int32_t *route_hist = nullptr;        // [blocks of tokens][E] histograms of the blocked route / permute kernels
   float *y_acc = nullptr;
   PlanHeader *plan_dev = nullptr;
   PlanHeader *plan_host = nullptr;      // pinned, mapped
@@ -727,11 +727,9 @@ ft_status_t ft_moe_route(ft_moe_t *h, int layer, const float *logits_dev, int T,
     h->launches++;
   } else {
     const int n_blocks = (T + kRouteBlockTokens - 1) / kRouteBlockTokens;
-    int scan_threads = ((rp.E + 31) / 32) * 32;
     route_block_kernel<<<n_blocks, 1024, 0, st>>>(rp, h->route_hist);
-    route_scan_kernel<<<1, scan_threads, 0, st>>>(rp, h->route_hist, n_blocks);
-    permute_block_kernel<<<n_blocks, 256, 0, st>>>(rp, h->route_hist);
-    h->launches += 3;
+    permute_block_kernel<<<n_blocks, 1024, 0, st>>>(rp, h->route_hist, n_blocks);
+    h->launches += 2;
   }
   FT_CUDA(cudaGetLastError());
   return FT_OK;

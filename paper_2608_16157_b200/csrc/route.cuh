@@ -173,11 +173,11 @@ __global__ void __launch_bounds__(1024) route_small_kernel(RouteParams p) {
   route_small_body(p, s);
 }
 
-// ---- prefill-sized calls: three launches over blocks of kRouteBlockTokens tokens ----
-constexpr int kRouteBlockTokens = 128;
+// ---- prefill-sized calls: two launches over blocks of kRouteBlockTokens tokens ----
+constexpr int kRouteBlockTokens = 32;   // one token per warp of a 1024-thread block: 4096 tokens fill 128 SMs
 
-// Kernel 1: block b routes its tokens (one warp per token at a time), writes ids / w and the block's histogram
-// hist[b][E] (integer atomics in shared memory: the counts do not depend on the order of the adds).
+// Kernel 1: block b routes its tokens (one warp per token), writes ids / w and the block's histogram hist[b][E]
+// (integer atomics in shared memory: the counts do not depend on the order of the adds).
 __global__ void __launch_bounds__(1024) route_block_kernel(RouteParams p, int32_t *hist) {
   __shared__ int32_t s_cnt[kMaxExperts];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -199,58 +199,65 @@ __global__ void __launch_bounds__(1024) route_block_kernel(RouteParams p, int32_
   for (int e = tid; e < p.E; e += blockDim.x) hist[(size_t)blockIdx.x * p.E + e] = s_cnt[e];
 }
 
-// Kernel 2: one CTA, one thread per expert: count[e], the exclusive prefix of the block histograms over the blocks
-// (written back into hist) and offset[] by a block scan of the counts.  blockDim.x >= E, a multiple of 32.
-__global__ void __launch_bounds__(1024) route_scan_kernel(RouteParams p, int32_t *hist, int n_blocks) {
+// Kernel 2: block b ranks its pairs.  pos(p) = offset[e] + pairs of expert e in earlier blocks + pairs of e earlier
+// in this block, which keeps the order stable in the pair index.  Every block sums the (small, L2-resident)
+// histograms itself -- count[e] over all blocks, the part before block b -- and scans the counts into offset[];
+// block 0 publishes count[] and offset[].  Each warp owns a contiguous part of the block's pairs and walks it 32
+// pairs at a time; lanes with equal keys find each other with match.any.  blockDim.x = 1024 >= E.
+__global__ void __launch_bounds__(1024) permute_block_kernel(RouteParams p, const int32_t *hist, int n_blocks) {
+  __shared__ int32_t s_base[8][kMaxExperts];
+  __shared__ int32_t s_start[kMaxExperts];   // offset[e] + pairs of e in earlier blocks
   __shared__ int32_t s_wsum[32];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
-  int c = 0;
-  if (tid < p.E) {
-    for (int b = 0; b < n_blocks; ++b) {
-      const int v = hist[(size_t)b * p.E + tid];
-      hist[(size_t)b * p.E + tid] = c;
-      c += v;
+  const int P = p.T * p.k;
+  {
+    int c = 0, before = 0;
+    if (tid < p.E) {
+      for (int b = 0; b < n_blocks; ++b) {
+        const int v = hist[(size_t)b * p.E + tid];
+        if (b < (int)blockIdx.x) before += v;
+        c += v;
+      }
     }
-  }
-  int incl = c;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int n = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += n;
-  }
-  if (lane == 31) s_wsum[warp] = incl;
-  __syncthreads();
-  if (warp == 0) {
-    const int ws = (lane < nwarps) ? s_wsum[lane] : 0;
-    int wincl = ws;
+    int incl = c;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const int n = __shfl_up_sync(0xffffffffu, wincl, o);
-      if (lane >= o) wincl += n;
+      const int n = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += n;
     }
-    s_wsum[lane] = wincl - ws;
+    if (lane == 31) s_wsum[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      const int ws = (lane < nwarps) ? s_wsum[lane] : 0;
+      int wincl = ws;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, wincl, o);
+        if (lane >= o) wincl += n;
+      }
+      s_wsum[lane] = wincl - ws;
+    }
+    __syncthreads();
+    const int excl = incl - c + s_wsum[warp];
+    if (tid < p.E) {
+      s_start[tid] = excl + before;
+      if (blockIdx.x == 0) {
+        p.count[tid] = c;
+        p.offset[tid] = excl;
+        if (tid == p.E - 1) p.offset[p.E] = excl + c;
+      }
+    }
   }
-  __syncthreads();
-  const int excl = incl - c + s_wsum[warp];
-  if (tid < p.E) {
-    p.count[tid] = c;
-    p.offset[tid] = excl;
-    if (tid == p.E - 1) p.offset[p.E] = excl + c;
+  if (warp >= 8) {   // the ranking below is done by 8 warps
+    __syncthreads();
+    __syncthreads();
+    return;
   }
-}
-
-// Kernel 3: block b ranks its pairs.  pos(p) = offset[e] + pairs of expert e in earlier blocks + pairs of e earlier
-// in this block, which keeps the order stable in the pair index.  Each warp owns a contiguous part of the block's
-// pairs and walks it 32 pairs at a time; lanes with equal keys find each other with match.any.
-__global__ void __launch_bounds__(256) permute_block_kernel(RouteParams p, const int32_t *hist) {
-  __shared__ int32_t s_base[8][kMaxExperts];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int P = p.T * p.k;
   const int q0 = blockIdx.x * kRouteBlockTokens * p.k;
   const int q1 = min(P, q0 + kRouteBlockTokens * p.k);
   const int per_warp = (((q1 - q0 + 7) / 8) + 31) & ~31;    // a multiple of 32 pairs
   const int w0 = q0 + warp * per_warp, w1 = min(q1, w0 + per_warp);
-  for (int e = tid; e < p.E; e += blockDim.x)
+  for (int e = tid; e < p.E; e += 256)
 #pragma unroll
     for (int w = 0; w < 8; ++w) s_base[w][e] = 0;
   __syncthreads();
@@ -262,8 +269,9 @@ __global__ void __launch_bounds__(256) permute_block_kernel(RouteParams p, const
     __syncwarp();
   }
   __syncthreads();
-  for (int e = tid; e < p.E; e += blockDim.x) {             // where each warp's pairs of expert e begin
-    int base = p.offset[e] + hist[(size_t)blockIdx.x * p.E + e];
+  // (the barriers from here on are among the 8 ranking warps only)
+  for (int e = tid; e < p.E; e += 256) {                    // where each warp's pairs of expert e begin
+    int base = s_start[e];
 #pragma unroll
     for (int w = 0; w < 8; ++w) {
       const int n = s_base[w][e];
@@ -271,7 +279,7 @@ __global__ void __launch_bounds__(256) permute_block_kernel(RouteParams p, const
       base += n;
     }
   }
-  __syncthreads();
+  asm volatile("bar.sync 1, 256;" ::: "memory");
   for (int q = w0 + lane; q - lane < w1; q += 32) {
     const int key = (q < w1) ? p.ids[q] : -1;
     const unsigned m = __match_any_sync(0xffffffffu, key);

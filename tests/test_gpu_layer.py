@@ -143,6 +143,19 @@ def test_int4_activation_range(scale_log2):
     pr.close()
 
 
+def test_int4_activation_outlier_in_a_group():
+    """One element 1000 x larger than the rest of its quantisation group: the fixed-point form of the group (15 bits
+    against the group's largest magnitude) keeps the result within the tolerance."""
+    shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2, wdtype="int4", n_shared=1)
+    pr = Pair(shape, n_slots=4, max_tokens=8, seed=12)
+    for step in range(2):
+        x = W.noise_x(6, 512, 12, step, 0).float()
+        x[:, 5::128] *= 1000.0                       # one outlier per group of 128, every token
+        x[2, :] = 0.0                                # and an all-zero token
+        pr.step(0, W.normal_logits(6, 8, 12, step), x.to(torch.bfloat16))
+    pr.close()
+
+
 def test_plan_and_permutation_are_deterministic():
     shape = W.LayerShape(d=256, inter=64, n_experts=32, top_k=4)
     runs = []
