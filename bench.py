@@ -896,9 +896,15 @@ def run_sweep(args):
                 noise = torch.randn((steps, L, batch, d), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
                 moe.reset()
                 torch.cuda.synchronize()
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0, e1, em = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+                tail = max(1, steps // 4)            # the last quarter of the point: the cache has settled
+                st_mid = None
                 e0.record(stream)
                 for s_ in range(steps):
+                    if s_ == steps - tail:
+                        torch.cuda.synchronize()
+                        st_mid = {kk: sum(moe.get_stats(l)[kk] for l in range(L)) for kk in Bd.STAT_NAMES}
+                        em.record(stream)
                     for l in range(L):
                         if l == 0:
                             x = noise[s_, 0]
@@ -909,6 +915,7 @@ def run_sweep(args):
                 e1.record(stream)
                 torch.cuda.synchronize()
                 ms = e0.elapsed_time(e1)
+                ms_tail = em.elapsed_time(e1)
                 st = {kk: sum(moe.get_stats(l)[kk] for l in range(L)) for kk in Bd.STAT_NAMES}
                 pt = {"cache_frac": frac, "slots": Ns, "rho": rho, "batch": batch, "steps": steps,
                       "tok_per_s": batch * steps / (ms * 1e-3), "ms_per_step": ms / steps,
@@ -917,7 +924,12 @@ def run_sweep(args):
                       "fills": st["fills"], "zero_copies": st["zc"], "evictions": st["evictions"],
                       "fill_bytes": st["fills"] * S, "zero_copy_bytes": st["zc"] * S,
                       "routed_unique_per_layer_step": st["routed"] / (steps * L),
-                      "resident_record_GBps": (st["hits"] + st["fills"]) * S / (ms * 1e-3) / 1e9}
+                      "resident_record_GBps": (st["hits"] + st["fills"]) * S / (ms * 1e-3) / 1e9,
+                      "settled": {"steps": tail, "tok_per_s": batch * tail / (ms_tail * 1e-3),
+                                  "ms_per_step": ms_tail / tail,
+                                  "fills_per_step": (st["fills"] - st_mid["fills"]) / tail,
+                                  "resident_record_GBps": (st["hits"] - st_mid["hits"] + st["fills"] - st_mid["fills"])
+                                  * S / (ms_tail * 1e-3) / 1e9}}
                 points.append(pt)
                 log(f"sweep {pt}")
         moe.destroy()
