@@ -259,6 +259,13 @@ def unpack_record(rec: np.ndarray, d: int, inter: int, wdtype: str):
                                          UA*I/16 + ((((cb*NG + ng)*8 + uu)*NWD + w)*32 + 4*g + q)*16 + 4*j + e//2,
                                          lo = e even
       down scale of (group ng, column c): UA*I/16 + I*d/2 + ((ng*CB + cb)*NWD + w)*128 + 16*g + 4*j + 2*half
+    mxfp4 record: 4-bit codes, bit 3 = sign, bits 2..0 index the magnitudes (0, 0.5, 1, 1.5, 2, 3, 4, 6); one scale
+    byte b per 32 consecutive elements of the contraction dimension, weight = (+-magnitude) * 2**(b - 127).  The
+    codes sit where the int4 codes sit with UA = 2176*G; scale bytes (same letters as above):
+      gate scale of (neuron n, block i//32): UA*(n//16) + 2048*G + 64*(i//128) + 8*(n%8) + 4*((n%16)//8) + (i%128)//32
+                                             up: the same + 64*G
+      down scale of (block n//32, column c): UA*I/16 + I*d/2 + ((ng*CB + cb)*NWD + w)*256 + 32*g + 8*j + 4*half
+                                             + (n%128)//32
     """
     rec = np.ascontiguousarray(rec).view(np.uint8).reshape(-1)
     n = inter * d
@@ -307,6 +314,41 @@ def unpack_record(rec: np.ndarray, d: int, inter: int, wdtype: str):
         a_down = UA * U + ((((cb * NG + ng) * 8 + uu) * nwd + w) * 32 + 4 * g + q) * 16 + 4 * j + e // 2
         s_down = UA * U + inter * d // 2 + ((ng * CB + cb) * nwd + w) * 128 + 16 * g + 4 * j + 2 * half
         wd = codes(a_down, e % 2 == 0) * bf16_at(s_down + 0 * n)
+        return wg, wu, wd
+    if wdtype == "mxfp4":
+        G, NG, U = d // GROUP, inter // GROUP, inter // 16
+        UA = 2176 * G
+        nwd = min(16, d // 64)
+        cbw = 64 * nwd
+        CB = d // cbw
+        assert rec.size == U * UA + inter * d // 2 + inter * d // 32
+        magnitude = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
+
+        def fp4(addr, lo):
+            b = rec[addr].astype(np.int64)
+            c = np.where(lo, b & 0xF, b >> 4)
+            return np.where(c & 8, -1.0, 1.0) * magnitude[c & 7]
+
+        def pow2(addr):
+            return np.exp2(rec[addr].astype(np.float64) - 127.0)
+
+        i = np.arange(d, dtype=np.int64)[:, None]
+        nn = np.arange(inter, dtype=np.int64)[None, :]
+        a_gate = UA * (nn // 16) + 1024 * (i // 128) + 64 * (nn % 16) + 16 * ((i % 32) // 8) + 4 * ((i % 128) // 32) \
+            + (i % 8) // 2
+        s_gate = UA * (nn // 16) + 2048 * G + 64 * (i // 128) + 8 * (nn % 8) + 4 * ((nn % 16) // 8) + (i % 128) // 32
+        lo = (i % 2 == 0) & (nn >= 0)
+        wg = fp4(a_gate, lo) * pow2(s_gate)
+        wu = fp4(a_gate + 1024 * G, lo) * pow2(s_gate + 64 * G)
+        n = np.arange(inter, dtype=np.int64)[:, None]
+        c = np.arange(d, dtype=np.int64)[None, :]
+        ng, uu, q, r = n // 128, (n % 128) // 16, (n % 16) // 4, n % 4
+        g, half, cb, t = c % 8, (c % 16) // 8, c // cbw, (c % cbw) // 16
+        w, j = t // 4, t % 4
+        e = half + 2 * r
+        a_down = UA * U + ((((cb * NG + ng) * 8 + uu) * nwd + w) * 32 + 4 * g + q) * 16 + 4 * j + e // 2
+        s_down = UA * U + inter * d // 2 + ((ng * CB + cb) * nwd + w) * 256 + 32 * g + 8 * j + 4 * half + (n % 128) // 32
+        wd = fp4(a_down, e % 2 == 0) * pow2(s_down)
         return wg, wu, wd
     raise ValueError(wdtype)
 

@@ -34,6 +34,14 @@ flattened identifier of Sec. 4.2 of the paper):
              ``4q + e // 2`` of the step.
           C. down scales ``sd[ng][column]`` in the order (ng, cb, w, g, j, half): 8 pairs per tile again.
           ``S = 3*I*d/2 + (2*I*d/128 + (I/128)*d)*2``.
+``mxfp4`` 4-bit e2m1 codes (bit 3 sign; bits 2..0 index 0, 0.5, 1, 1.5, 2, 3, 4, 6) with one power-of-two scale byte
+          ``b`` (value ``2**(b - 127)``) per block of 32 consecutive elements along the contraction dimension
+          (the OCP microscaling FP4 element and scale formats).  The code sections are those of ``int4``; the scales:
+          A. per tile 64 bytes after the tiles of a unit (``2176*G`` bytes per unit): for ``r`` in 0..7 the four block
+             scales (``j`` = 0..3) of row ``r``, then those of row ``r+8``.
+          C. order (ng, cb, w, g, j, half, m): per lane ``g`` 32 bytes = for each tile ``j`` and column half the four
+             32-neuron blocks ``m`` of the 128-neuron group.
+          ``S = 3*I*d/2 + 3*I*d/32``.
 
 The routing-logit recipes follow the workload descriptions: a Zipf-style
 popularity bias ``b_e = -alpha * ln(rank_e)`` with ``rank`` a seeded permutation
@@ -49,6 +57,7 @@ import numpy as np
 import torch
 
 GROUP = 128  # int4 quantisation group length along the contraction dimension
+MX_BLOCK = 32  # elements that share one scale byte in the mxfp4 records
 
 
 @dataclasses.dataclass(frozen=True)
@@ -57,7 +66,7 @@ class LayerShape:
     inter: int        # expert intermediate size I
     n_experts: int    # routed experts E
     top_k: int
-    wdtype: str = "bf16"   # "bf16" | "int4"
+    wdtype: str = "bf16"   # "bf16" | "int4" | "mxfp4"
     n_shared: int = 0      # always-resident shared experts (0 or 1)
 
     @property
@@ -68,6 +77,8 @@ class LayerShape:
             payload = 3 * self.inter * self.d // 2
             scales = (2 * self.inter * (self.d // GROUP) + (self.inter // GROUP) * self.d) * 2
             return payload + scales
+        if self.wdtype == "mxfp4":
+            return 3 * self.inter * self.d // 2 + 3 * self.inter * self.d // MX_BLOCK
         raise ValueError(self.wdtype)
 
 
@@ -75,6 +86,7 @@ class LayerShape:
 TINY = LayerShape(d=256, inter=128, n_experts=8, top_k=2)
 QWEN3_30B = LayerShape(d=2048, inter=768, n_experts=128, top_k=8)
 DSV3_INT4 = LayerShape(d=7168, inter=2048, n_experts=256, top_k=8, wdtype="int4", n_shared=1)
+DSV3_MXFP4 = LayerShape(d=7168, inter=2048, n_experts=256, top_k=8, wdtype="mxfp4", n_shared=1)
 
 
 def mix64(*vals: int) -> int:
@@ -138,6 +150,57 @@ def _pack_nibbles(q: torch.Tensor) -> torch.Tensor:
     """int8 codes ``[..., n]`` -> uint8 ``[..., n/2]``, low nibble = even index."""
     u = (q.to(torch.int16) & 0xF).to(torch.uint8)
     return u[..., 0::2] | (u[..., 1::2] << 4)
+
+
+def _quantise_mxfp4(w: torch.Tensor, block_axis: int) -> tuple[torch.Tensor, torch.Tensor]:
+    """Microscaling FP4 quantiser used to *produce* the synthetic pool.
+
+    ``w``: fp32 ``[I, d]``; blocks of 32 along ``block_axis`` (0 or 1).  Returns (codes uint8 in 0..15 with w's
+    shape, scale bytes uint8 with the block axis reduced by 32).  Shared exponent = floor(log2(amax)) - 2 (2 = the
+    exponent of the largest e2m1 magnitude), elements rounded to the nearest e2m1 value (ties to the even code),
+    saturating at 6.
+    """
+    I, d = w.shape
+    wb = w.reshape(I, d // MX_BLOCK, MX_BLOCK) if block_axis == 1 else w.reshape(I // MX_BLOCK, MX_BLOCK, d)
+    ax = 2 if block_axis == 1 else 1
+    amax = wb.abs().amax(dim=ax, keepdim=True)
+    e = torch.floor(torch.log2(torch.where(amax > 0, amax, torch.ones_like(amax)))) - 2
+    b = torch.clamp(e + 127, 0, 254)
+    v = wb / torch.exp2(b - 127)
+    a = v.abs().clamp(max=6.0)
+    bounds = torch.tensor([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0], device=w.device, dtype=torch.float32)
+    lo_ = torch.bucketize(a, bounds, right=False)     # bounds strictly below a
+    hi_ = torch.bucketize(a, bounds, right=True)      # bounds at or below a
+    idx = torch.where(lo_ != hi_, torch.where(lo_ % 2 == 0, lo_, hi_), lo_)   # a tie goes to the even code
+    code = (idx | torch.where(v < 0, 8, 0)).to(torch.uint8)
+    return code.reshape(I, d), b.squeeze(ax).to(torch.uint8)
+
+
+def _pack_mxfp4_record(cg, cu, cd, bg, bu, bd) -> torch.Tensor:
+    """Codes uint8 ``[I][d]`` (gate/up: one row per neuron; down: ``[n][c]``), scale bytes ``bg, bu [I][d/32]``,
+    ``bd [I/32][d]`` -> the tiled record, uint8 flat."""
+    I, d = cg.shape
+    dev = cg.device
+    U, G, NG = I // 16, d // GROUP, I // GROUP
+    nwd = min(16, d // 64)
+    cbw = 64 * nwd
+    CB = d // cbw
+
+    def gu_tiles(c):      # [U][16 rows][G][j][q][e] -> [U][G][row][q][j][e], nibbles packed along e
+        t = c.reshape(U, 16, G, 4, 4, 8).permute(0, 2, 1, 4, 3, 5)
+        return (t[..., 0::2] | (t[..., 1::2] << 4)).reshape(U, G * 1024)
+
+    def gu_scales(b_):    # [U][half][r][G][j] -> [U][G][r][half][j]
+        return b_.reshape(U, 2, 8, G, 4).permute(0, 3, 2, 1, 4).reshape(U, G * 64)
+
+    sec_a = torch.cat([gu_tiles(cg), gu_tiles(cu), gu_scales(bg), gu_scales(bu)], dim=1).reshape(-1)
+    ar = lambda n: torch.arange(n, device=dev)
+    cb, ng, uu, w, g, q, j, e = torch.meshgrid(ar(CB), ar(NG), ar(8), ar(nwd), ar(8), ar(4), ar(4), ar(8), indexing="ij")
+    t = cd[128 * ng + 16 * uu + 4 * q + e // 2, cb * cbw + (4 * w + j) * 16 + g + 8 * (e & 1)]
+    sec_b = (t[..., 0::2] | (t[..., 1::2] << 4)).reshape(-1)
+    ng2, cb2, w2, g2, j2, half, m = torch.meshgrid(ar(NG), ar(CB), ar(nwd), ar(8), ar(4), ar(2), ar(4), indexing="ij")
+    sec_c = bd[4 * ng2 + m, cb2 * cbw + (4 * w2 + j2) * 16 + g2 + 8 * half].reshape(-1)
+    return torch.cat([sec_a, sec_b, sec_c])
 
 
 WD_NU = (0, 0, 1, 1, 2, 2, 3, 3)     # neuron offset (plus 4q) of nibble e in a word of the down section
@@ -206,6 +269,11 @@ def make_records(shape: LayerShape, seed: int, layer: int, first: int, count: in
         w = torch.randn((3, I, d), generator=g, device=device, dtype=torch.float32) * std
         if shape.wdtype == "bf16":
             out[j] = _pack_bf16_tiles(w.to(torch.bfloat16)).view(torch.uint8)
+        elif shape.wdtype == "mxfp4":
+            cg, bg = _quantise_mxfp4(w[0], 1)
+            cu, bu = _quantise_mxfp4(w[1], 1)
+            cd, bd = _quantise_mxfp4(w[2], 0)
+            out[j] = _pack_mxfp4_record(cg, cu, cd, bg, bu, bd)
         else:
             qg, sg = _quantise_int4(w[0:1], 2)
             qu, su = _quantise_int4(w[1:2], 2)

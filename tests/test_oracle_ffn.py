@@ -118,6 +118,101 @@ def test_unpack_int4_record_by_definition(d, I):
     np.testing.assert_allclose(x @ wg1, np.repeat(x.sum(axis=1, keepdims=True), I, axis=1), rtol=1e-12)
 
 
+FP4_VALUES = (0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0)     # the e2m1 magnitudes, by code & 7
+
+
+def _record_mxfp4_by_definition(cg, cu, cd, bg, bu, bd):
+    """cX: codes 0..15 [I][d] (row = neuron); bg/bu [I][d/32], bd [I/32][d] scale bytes.  Written section by section
+    from the documented tile order."""
+    I, d = cg.shape
+    G, NG, U = d // 128, I // 128, I // 16
+    nwd = min(16, d // 64)
+    cbw, CB = 64 * nwd, d // (64 * nwd)
+    out = bytearray()
+
+    def word(nibbles):
+        v = 0
+        for e, c in enumerate(nibbles):
+            v |= (int(c) & 0xF) << (4 * e)
+        return v.to_bytes(4, "little")
+
+    for u in range(U):
+        for c_ in (cg, cu):
+            for grp in range(G):
+                for row in range(16):
+                    for chunk in range(4):
+                        for j in range(4):
+                            i0 = 128 * grp + 32 * j + 8 * chunk
+                            out += word(c_[16 * u + row, i0:i0 + 8])
+        for b_ in (bg, bu):
+            for grp in range(G):
+                for r in range(8):
+                    out += bytes(int(b_[16 * u + r, 4 * grp + j]) for j in range(4))
+                    out += bytes(int(b_[16 * u + r + 8, 4 * grp + j]) for j in range(4))
+    for cb in range(CB):
+        for ng in range(NG):
+            for uu in range(8):
+                for w in range(nwd):
+                    for lane in range(32):
+                        g, q = divmod(lane, 4)
+                        for j in range(4):
+                            col0 = cb * cbw + (4 * w + j) * 16
+                            out += word([cd[128 * ng + 16 * uu + 4 * q + e // 2, col0 + g + 8 * (e & 1)] for e in range(8)])
+    for ng in range(NG):
+        for cb in range(CB):
+            for w in range(nwd):
+                for g in range(8):
+                    for j in range(4):
+                        for half in range(2):
+                            col = cb * cbw + (4 * w + j) * 16 + g + 8 * half
+                            out += bytes(int(bd[4 * ng + m, col]) for m in range(4))
+    return np.frombuffer(bytes(out), dtype=np.uint8)
+
+
+@pytest.mark.parametrize("d,I", [(256, 128), (1024, 256)])
+def test_unpack_mxfp4_record_by_definition(d, I):
+    rng = np.random.default_rng(3)
+    cg, cu, cd = (rng.integers(0, 16, size=(I, d)) for _ in range(3))
+    bg = rng.integers(120, 131, size=(I, d // 32))
+    bu = rng.integers(110, 127, size=(I, d // 32))
+    bd = rng.integers(125, 135, size=(I // 32, d))
+    rec = _record_mxfp4_by_definition(cg, cu, cd, bg, bu, bd)
+    assert rec.size == W.LayerShape(d, I, 1, 1, "mxfp4").expert_bytes
+    wg, wu, wd = O.unpack_record(rec, d, I, "mxfp4")
+    val = np.array(FP4_VALUES)
+
+    def deq(c, b, axis):
+        return np.where(c & 8, -1.0, 1.0) * val[c & 7] * np.repeat(np.exp2(b.astype(np.float64) - 127), 32, axis=axis)
+
+    assert np.array_equal(wg, deq(cg, bg, 1).T)
+    assert np.array_equal(wu, deq(cu, bu, 1).T)
+    assert np.array_equal(wd, deq(cd, bd, 0))
+    # code 2 (= 1.0) everywhere with scale byte 127 (= 2**0) gives column sums of x; code 10 their negatives
+    ones = np.full((I, d), 2)
+    b0g, b0d = np.full((I, d // 32), 127), np.full((I // 32, d), 127)
+    wg1, _, wd1 = O.unpack_record(_record_mxfp4_by_definition(ones, ones, ones | 8, b0g, b0g, b0d), d, I, "mxfp4")
+    x = rng.standard_normal((3, d))
+    np.testing.assert_allclose(x @ wg1, np.repeat(x.sum(axis=1, keepdims=True), I, axis=1), rtol=1e-12)
+    assert np.array_equal(wd1, -np.ones((I, d)))
+
+
+def test_generated_mxfp4_pool_quantiser_error_bound():
+    """The generator's records, read back by the oracle, are within half a grid step of the fp32 draws: the e2m1 grid
+    step is at most 2 (between 4 and 6) times the block scale 2**(floor(log2(amax)) - 2), i.e. |w - deq| <= amax / 4."""
+    shape = W.LayerShape(d=256, inter=128, n_experts=2, top_k=1, wdtype="mxfp4")
+    rec = W.make_records(shape, seed=0, layer=0, first=0, count=1)[0].numpy()
+    wg, wu, wd = O.unpack_record(rec, 256, 128, "mxfp4")
+    g = torch.Generator().manual_seed(W.mix64(0, 1, 0, 0))
+    w = (torch.randn((3, 128, 256), generator=g) * 0.02).double().numpy()
+    for got, ref, axis in ((wg.T, w[0], 1), (wu.T, w[1], 1), (wd, w[2], 0)):
+        blocks = np.abs(ref).reshape((128, 8, 32) if axis == 1 else (4, 32, 256))
+        amax = np.repeat(blocks.max(axis=2 if axis == 1 else 1), 32, axis=axis)
+        assert np.all(np.abs(got - ref) <= amax / 4 + 1e-15)
+        assert np.all(np.abs(got) <= 1.5 * amax + 1e-15)          # the largest element maps to 4 or 6 times the scale
+    # and the records are not trivially zero
+    assert np.count_nonzero(wg) > wg.size // 2
+
+
 def test_generated_int4_pool_quantiser_error_bound():
     shape = W.LayerShape(d=256, inter=128, n_experts=2, top_k=1, wdtype="int4")
     rec = W.make_records(shape, seed=0, layer=0, first=0, count=1)[0].numpy()
