@@ -61,7 +61,16 @@
  *                   registers of the int8 tensor-core instruction as they are (bytes code + 8; the kernels subtract
  *                   8 x the activation sums).
  *                   S = 3*inter*hidden/2 + (2*inter*hidden/128 + (inter/128)*hidden)*2 bytes.
- *   Shape limits: bf16: hidden in {256, 512, 1024, 2048}, inter % 16 == 0; int4: hidden in
+ *   FT_W_MXFP4    : microscaling FP4 (paper Sec. 5.1 serves MXFP4 experts): 4-bit e2m1 codes (bit 3 sign, bits 2..0
+ *                   index the magnitudes 0, 0.5, 1, 1.5, 2, 3, 4, 6) and one scale byte b per 32 consecutive elements
+ *                   of the contraction dimension, weight = (+-magnitude) * 2^(b-127).  The code sections are those of
+ *                   FT_W_INT4_G128; a unit of section A is 2176*G bytes: its tiles, then per gate tile and per up
+ *                   tile 64 scale bytes = for r in 0..7 the four block scales (j = 0..3) of row r, then those of row
+ *                   r+8.  Section C: order (ng, cb, w, g, j, half, m), i.e. per lane g 32 bytes = for each tile j and
+ *                   column half the scales of the four 32-neuron blocks m of the 128-neuron group.
+ *                   S = 3*inter*hidden/2 + 3*inter*hidden/32 bytes.  Decode-sized calls only (no tensor-core prefill
+ *                   path); shapes as for int4.
+ *   Shape limits: bf16: hidden in {256, 512, 1024, 2048}, inter % 16 == 0; int4 and mxfp4: hidden in
  *   {512, 1024, 2048, 4096, 7168, 8192}, inter % 128 == 0; n_experts <= 1024;
  *   top_k <= min(n_experts, 32); slots per table (slots_per_layer, or n_layers*slots_per_layer with global_pool) <= 6144.  The tensor-core prefill path
  *   (gemm_min_tokens > 0) needs bf16 weights, slots_per_layer > 0 and inter % 256 == 0.
@@ -90,7 +99,7 @@ typedef enum {
   FT_ERR_UNSUPPORTED = 8
 } ft_status_t;
 
-typedef enum { FT_W_BF16 = 0, FT_W_INT4_G128 = 1 } ft_wdtype_t;
+typedef enum { FT_W_BF16 = 0, FT_W_INT4_G128 = 1, FT_W_MXFP4 = 2 } ft_wdtype_t;
 
 /* How ft_moe_fill moves records.  Both give byte-identical slots. */
 typedef enum {

@@ -10,6 +10,7 @@
 
 #include "common.cuh"
 #include "ffn_stream.cuh"
+#include "ffn_mx4.cuh"
 #include "ffn_w4.cuh"
 #include "gemm_tc.cuh"
 #include "gemm_tc2.cuh"
@@ -156,6 +157,10 @@ size_t expert_bytes_of(const ft_moe_config_t *c) {
   if (c->wdtype == FT_W_BF16) {
     if ((d != 256 && d != 512 && d != 1024 && d != 2048) || I % 16) return 0;
     return 3 * I * d * 2;
+  }
+  if (c->wdtype == FT_W_MXFP4) {
+    if (d % 512 || d > 8192 || I % 128) return 0;   // (same shapes as int4)
+    return 3 * I * d / 2 + 3 * I * d / 32;
   }
   if (c->wdtype == FT_W_INT4_G128) {
     if (d % 512 || d > 8192 || I % 128) return 0;   // (the kernels further restrict d, see w4_shape_ok)
@@ -465,12 +470,12 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
       c.max_tokens <= 0 || (c.n_shared != 0 && c.n_shared != 1) || c.device < 0 ||
       (c.fill_mode != FT_FILL_COPY_ENGINE && c.fill_mode != FT_FILL_SM))
     return FT_ERR_INVALID_ARG;
-  if (c.wdtype != FT_W_BF16 && c.wdtype != FT_W_INT4_G128) return FT_ERR_INVALID_ARG;
+  if (c.wdtype != FT_W_BF16 && c.wdtype != FT_W_INT4_G128 && c.wdtype != FT_W_MXFP4) return FT_ERR_INVALID_ARG;
   if (c.bw_fill_MBps == 0 || c.bw_zc_MBps == 0 || c.bw_hbm_MBps == 0 || c.reuse_credit < 0 ||
       c.zc_tokens_per_pass < 1 || c.hbm_tokens_per_pass < 1 || c.gemm_min_tokens < 0 || c.split_min_pairs < 0)
     return FT_ERR_INVALID_ARG;
   const size_t S = expert_bytes_of(cfg);
-  if (S == 0 || (c.wdtype == FT_W_INT4_G128 && !w4_shape_ok(c))) return FT_ERR_UNSUPPORTED;
+  if (S == 0 || (c.wdtype != FT_W_BF16 && !w4_shape_ok(c))) return FT_ERR_UNSUPPORTED;
   if (c.gemm_min_tokens != 0 &&
       (c.wdtype != FT_W_BF16 || c.slots_per_layer == 0 || c.hidden % 256 || c.inter % 256 || c.gemm_min_tokens < 8))
     return FT_ERR_UNSUPPORTED;
@@ -592,7 +597,7 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
   FT_TRY(cudaMalloc(&h->done_dev, 4));
   FT_TRY(cudaMemset(h->done_dev, 0, 4));
   FT_TRY(cudaFuncSetAttribute(fill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFillStages * (int)kFillChunk));
-  if (c.wdtype == FT_W_INT4_G128) {
+  if (c.wdtype == FT_W_INT4_G128 || c.wdtype == FT_W_MXFP4) {
     const size_t passes = (P + 7) / 8 + 2 * E + 2;
     FT_TRY(cudaMalloc(&h->w4_hraw, passes * (c.inter / 16) * 512));
     FT_TRY(cudaMalloc(&h->w4_hcount, passes * (c.inter / 128) * 4));
@@ -611,6 +616,15 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
     FT_TRY(cudaFuncSetAttribute(w4_gateup_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
     FT_TRY(cudaFuncSetAttribute(w4_down_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
     FT_TRY(cudaFuncSetAttribute(w4_down_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
+    const int sbm = (int)mx4_down_smem_bytes(2 * kMaxExperts + 1);
+    FT_TRY(cudaFuncSetAttribute(mx4_gateup_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(mx4_gateup_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(mx4_gateup_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(mx4_gateup_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(mx4_gateup_kernel<56>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(mx4_gateup_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(mx4_down_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sbm));
+    FT_TRY(cudaFuncSetAttribute(mx4_down_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sbm));
   }
   if (c.wdtype == FT_W_BF16) {
     // the limit is a property of the function on this device, not of the handle: always the largest size any
@@ -1010,7 +1024,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     }
     return FT_OK;
   }
-  // int4: gate/up kernel writes h, down kernel accumulates, its last CTA finalizes y
+  // int4 / mxfp4: gate/up kernel writes h, down kernel accumulates, its last CTA finalizes y
   if (c.slots_per_layer > 0 && L.fill_recorded) FT_CUDA(cudaStreamWaitEvent(st, L.ev_fill, 0));
   W4Params qp;
   qp.items = sc.items_res;
@@ -1019,24 +1033,38 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   qp.pref = sc.res_pref;
   qp.max_items = 2 * c.n_experts + 1;
   qp.x = x_bf; qp.perm = sc.perm; qp.topk_w = sc.topk_w;
-  qp.mask = 0x0F0F0F0Fu; qp.flip = 0x08080808u;
+  const bool mx = c.wdtype == FT_W_MXFP4;
+  if (mx) { qp.mask = 0x1C1C1C1Cu; qp.flip = 0x80808080u; }   // (see ffn_mx4.cuh)
+  else { qp.mask = 0x0F0F0F0Fu; qp.flip = 0x08080808u; }
   qp.hraw = h->w4_hraw; qp.hcount = h->w4_hcount; qp.hq = h->w4_hq; qp.hs = h->w4_hs;
   qp.y_acc = h->y_acc; qp.y = static_cast<__nv_bfloat16 *>(y_dev);
   qp.done = h->done_dev; qp.status = h->status_dev;
   qp.inter = c.inter; qp.top_k = c.top_k; qp.T = L.T;
   const bool own_finalize = L.T > kFinalizeInKernelMaxTokens;
   qp.finalize = own_finalize ? 0 : 1;
-  const size_t sa = w4_gateup_smem_bytes(qp.max_items, c.hidden), sb = w4_down_smem_bytes(qp.max_items);
+  const size_t sa = mx ? mx4_gateup_smem_bytes(qp.max_items, c.hidden) : w4_gateup_smem_bytes(qp.max_items, c.hidden);
+  const size_t sb = mx ? mx4_down_smem_bytes(qp.max_items) : w4_down_smem_bytes(qp.max_items);
   const int grid = h->sm_count;
   {
-    TimeScope ts(h, st, FT_TIME_FFN_ZC);   // (timing slot reused for the gate/up kernel of the int4 path)
-    switch (c.hidden) {
-      case 512: w4_gateup_kernel<4><<<grid, kW4Threads, sa, st>>>(qp); break;
-      case 1024: w4_gateup_kernel<8><<<grid, kW4Threads, sa, st>>>(qp); break;
-      case 2048: w4_gateup_kernel<16><<<grid, kW4Threads, sa, st>>>(qp); break;
-      case 4096: w4_gateup_kernel<32><<<grid, kW4Threads, sa, st>>>(qp); break;
-      case 7168: w4_gateup_kernel<56><<<grid, kW4Threads, sa, st>>>(qp); break;
-      default: w4_gateup_kernel<64><<<grid, kW4Threads, sa, st>>>(qp); break;
+    TimeScope ts(h, st, FT_TIME_FFN_ZC);   // (timing slot reused for the gate/up kernel of the 4-bit paths)
+    if (mx) {
+      switch (c.hidden) {
+        case 512: mx4_gateup_kernel<4><<<grid, kW4Threads, sa, st>>>(qp); break;
+        case 1024: mx4_gateup_kernel<8><<<grid, kW4Threads, sa, st>>>(qp); break;
+        case 2048: mx4_gateup_kernel<16><<<grid, kW4Threads, sa, st>>>(qp); break;
+        case 4096: mx4_gateup_kernel<32><<<grid, kW4Threads, sa, st>>>(qp); break;
+        case 7168: mx4_gateup_kernel<56><<<grid, kW4Threads, sa, st>>>(qp); break;
+        default: mx4_gateup_kernel<64><<<grid, kW4Threads, sa, st>>>(qp); break;
+      }
+    } else {
+      switch (c.hidden) {
+        case 512: w4_gateup_kernel<4><<<grid, kW4Threads, sa, st>>>(qp); break;
+        case 1024: w4_gateup_kernel<8><<<grid, kW4Threads, sa, st>>>(qp); break;
+        case 2048: w4_gateup_kernel<16><<<grid, kW4Threads, sa, st>>>(qp); break;
+        case 4096: w4_gateup_kernel<32><<<grid, kW4Threads, sa, st>>>(qp); break;
+        case 7168: w4_gateup_kernel<56><<<grid, kW4Threads, sa, st>>>(qp); break;
+        default: w4_gateup_kernel<64><<<grid, kW4Threads, sa, st>>>(qp); break;
+      }
     }
   }
   {
@@ -1049,8 +1077,13 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = at; lc.numAttrs = 1;
-    if (c.hidden == 512) FT_CUDA(cudaLaunchKernelEx(&lc, w4_down_kernel<8>, qp, c.hidden));
-    else FT_CUDA(cudaLaunchKernelEx(&lc, w4_down_kernel<16>, qp, c.hidden));
+    if (mx) {
+      if (c.hidden == 512) FT_CUDA(cudaLaunchKernelEx(&lc, mx4_down_kernel<8>, qp, c.hidden));
+      else FT_CUDA(cudaLaunchKernelEx(&lc, mx4_down_kernel<16>, qp, c.hidden));
+    } else {
+      if (c.hidden == 512) FT_CUDA(cudaLaunchKernelEx(&lc, w4_down_kernel<8>, qp, c.hidden));
+      else FT_CUDA(cudaLaunchKernelEx(&lc, w4_down_kernel<16>, qp, c.hidden));
+    }
     if (own_finalize) {
       const int n4 = L.T * (c.hidden / 4);
       finalize_kernel<<<std::min((n4 + 255) / 256, h->sm_count * 8), 256, 0, st>>>(h->y_acc, qp.y, n4);

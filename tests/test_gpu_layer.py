@@ -108,20 +108,22 @@ def test_results_do_not_depend_on_residency():
     assert torch.equal(ys["fill"], ys["hit"]) or (ys["fill"] - ys["hit"]).abs().max() <= 1e-2 * scale
 
 
+@pytest.mark.parametrize("wdtype", ["int4", "mxfp4"])
 @pytest.mark.parametrize("n_shared", [0, 1])
 @pytest.mark.parametrize("T", [1, 4, 7])
-def test_int4_group_dequant_and_shared_expert(n_shared, T):
-    shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2, wdtype="int4", n_shared=n_shared)
+def test_int4_group_dequant_and_shared_expert(n_shared, T, wdtype):
+    shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2, wdtype=wdtype, n_shared=n_shared)
     pr = Pair(shape, n_slots=4, max_tokens=8, seed=5)
     for step in range(3):
         pr.step(0, W.normal_logits(T, 8, 5, step), W.noise_x(T, 512, 5, step, 0), check_slots=True)
     pr.close()
 
 
+@pytest.mark.parametrize("wdtype", ["int4", "mxfp4"])
 @pytest.mark.parametrize("T", [9, 24, 40])
-def test_int4_resident_experts_with_many_tokens_and_shared_expert(T):
-    """More than 8 tokens per slot-resident int4 expert (several weight passes) and the shared expert at T > 8."""
-    shape = W.LayerShape(d=512, inter=256, n_experts=4, top_k=2, wdtype="int4", n_shared=1)
+def test_int4_resident_experts_with_many_tokens_and_shared_expert(T, wdtype):
+    """More than 8 tokens per slot-resident 4-bit expert (several weight passes) and the shared expert at T > 8."""
+    shape = W.LayerShape(d=512, inter=256, n_experts=4, top_k=2, wdtype=wdtype, n_shared=1)
     pr = Pair(shape, n_slots=4, max_tokens=40, seed=6)
     for step in range(3):
         _, r = pr.step(0, W.normal_logits(T, 4, 6, step), W.noise_x(T, 512, 6, step, 0))
@@ -131,11 +133,13 @@ def test_int4_resident_experts_with_many_tokens_and_shared_expert(T):
     pr.close()
 
 
+@pytest.mark.parametrize("wdtype", ["int4", "mxfp4"])
 @pytest.mark.parametrize("scale_log2", [-10, 10])
-def test_int4_activation_range(scale_log2):
-    """The int4 kernels keep activations and h in bf16 (fp32 accumulation), so their range is that of bf16: inputs
-    scaled by 2^-10 and 2^10 still meet the tolerance (the output scales roughly by the square)."""
-    shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2, wdtype="int4", n_shared=1)
+def test_int4_activation_range(scale_log2, wdtype):
+    """The 4-bit kernels re-express activations and h per (token, group of 128) against the group's largest magnitude,
+    so their range is that of fp32: inputs scaled by 2^-10 and 2^10 still meet the tolerance (the output scales
+    roughly by the square)."""
+    shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2, wdtype=wdtype, n_shared=1)
     pr = Pair(shape, n_slots=4, max_tokens=8, seed=8)
     for step in range(2):
         x = (W.noise_x(6, 512, 8, step, 0).float() * (2.0 ** scale_log2)).to(torch.bfloat16)
@@ -143,10 +147,11 @@ def test_int4_activation_range(scale_log2):
     pr.close()
 
 
-def test_int4_activation_outlier_in_a_group():
-    """One element 1000 x larger than the rest of its quantisation group: the fixed-point form of the group (15 bits
-    against the group's largest magnitude) keeps the result within the tolerance."""
-    shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2, wdtype="int4", n_shared=1)
+@pytest.mark.parametrize("wdtype", ["int4", "mxfp4"])
+def test_int4_activation_outlier_in_a_group(wdtype):
+    """One element 1000 x larger than the rest of its quantisation group: the group's re-expressed form (15-bit fixed
+    point, or two fp8 numbers, against the group's largest magnitude) keeps the result within the tolerance."""
+    shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2, wdtype=wdtype, n_shared=1)
     pr = Pair(shape, n_slots=4, max_tokens=8, seed=12)
     for step in range(2):
         x = W.noise_x(6, 512, 12, step, 0).float()
@@ -257,9 +262,9 @@ def test_qwen3_shaped_decode_two_layers(batch):
     pr.close()
 
 
-def test_dsv3_shaped_int4_decode_one_layer():
-    """d=7168, 256 routed experts (int4, group 128) + 1 shared expert, I=2048, top-8, 64 slots, batch 4."""
-    shape = W.DSV3_INT4
+@pytest.mark.parametrize("shape", [W.DSV3_INT4, W.DSV3_MXFP4], ids=["int4", "mxfp4"])
+def test_dsv3_shaped_int4_decode_one_layer(shape):
+    """d=7168, 256 routed experts (int4 group 128, or mxfp4) + 1 shared expert, I=2048, top-8, 64 slots, batch 4."""
     steps = 3
     pr = Pair(shape, n_slots=64, max_tokens=8, n_layers=1, seed=0, gen_device="cuda")
     logits = W.ar1_logits(1, steps, 4, 256, rho=0.9, alpha=1.2, seed=0)
