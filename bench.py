@@ -765,12 +765,13 @@ def sub_prefill(args, dev, cal):
             "pairs_on_gemm_frac": w["pairs_gemm"] / max(w["pairs"], 1), "zero_copy_experts_cold": cd["zero_copy"]}
 
 
-def sub_int4(args, dev, cal):
-    """Sub-record of the decode line: config 3 (DeepSeek-V3-shaped int4 decode, 4 layers, batch 4, 64 slots)."""
+def sub_int4(args, dev, cal, wdtype="int4"):
+    """Sub-record of the decode line: config 3 (DeepSeek-V3-shaped 4-bit decode, 4 layers, batch 4, 64 slots), with
+    int4-g128 experts or (the format the paper serves) MXFP4 experts."""
     import torch
     from paper_2608_16157_b200 import binding as Bd
     from paper_2608_16157_b200 import workload as W
-    shape = W.DSV3_INT4
+    shape = W.DSV3_INT4 if wdtype == "int4" else W.DSV3_MXFP4
     L, E, k, d, B, Ns = 4, shape.n_experts, shape.top_k, shape.d, 4, 64
     S = shape.expert_bytes
     warm, K = 48, 16
@@ -779,7 +780,8 @@ def sub_int4(args, dev, cal):
     shared = W.make_shared_records(shape, L, SEED, device=dev)
     moe = Bd.FtMoe(Bd.make_config(hidden=d, inter=shape.inter, n_experts=E, top_k=k, n_layers=L, slots_per_layer=Ns,
                                   max_tokens=8, host_pool_ptr=pool.ptr.value, host_pool_bytes=pool.n_bytes,
-                                  fill_mode=Bd.FT_FILL_SM, wdtype=Bd.FT_W_INT4_G128, n_shared=1,
+                                  fill_mode=Bd.FT_FILL_SM,
+                                  wdtype=Bd.FT_W_INT4_G128 if wdtype == "int4" else Bd.FT_W_MXFP4, n_shared=1,
                                   shared_ptr=shared.data_ptr(), bw_fill=max(cal["fill_MBps"], 1),
                                   bw_zc=max(cal["zc_MBps"], 1), bw_zc_residual=0, bw_hbm=max(cal["hbm_MBps"], 1)))
     stream = torch.cuda.current_stream()
@@ -840,8 +842,11 @@ def sub_int4(args, dev, cal):
     hbm_peak, peak_kind = peaks()
     t_us, nb = statistics.median(us[2:]), sum(nbytes[2:]) / len(nbytes[2:])
     gbps = nb / (t_us * 1e-6) / 1e9
-    return {"config": "decode, config 3: d=7168, 256 int4-g128 experts + 1 shared, I=2048, top-8, 4 layers, 64 slots "
-                      "per layer, batch 4, rho 0.9, alpha 1.2",
+    return {"config": "decode, config 3: d=7168, 256 %s experts + 1 shared, I=2048, top-8, 4 layers, 64 slots "
+                      "per layer, batch 4, rho 0.9, alpha 1.2" % ("int4-g128" if wdtype == "int4" else "mxfp4"),
+            "kernels": "w4_gateup_kernel + w4_down_kernel" if wdtype == "int4" else "mx4_gateup_kernel + mx4_down_kernel",
+            "bound": "hbm" if wdtype == "int4" else "alu (logic pipe: 7 instructions per 8 weights plus a scale per MMA); "
+                     "reported against the HBM peak",
             "tok_per_s": B * K / (ms * 1e-3), "ms_per_step": ms / K,
             "fills_per_step": (st1["fills"] - st0["fills"]) / K, "cache_warm_steps": warm,
             "GBps": gbps, "frac": gbps / hbm_peak, "peak": hbm_peak, "peak_source": peak_kind,
@@ -851,7 +856,11 @@ def sub_int4(args, dev, cal):
                    "+ the shared expert) x record bytes"}
 
 
-SUBRECORDS = {"int4": sub_int4, "prefill": sub_prefill}
+def sub_mxfp4(args, dev, cal):
+    return sub_int4(args, dev, cal, "mxfp4")
+
+
+SUBRECORDS = {"int4": sub_int4, "mxfp4": sub_mxfp4, "prefill": sub_prefill}
 
 
 def run_sweep(args):
@@ -971,7 +980,7 @@ def main():
     ap.add_argument("--only-batch", action="store_true")
     ap.add_argument("--cache-warm-steps", type=int, default=64,
                     help="untimed steps from the empty cache before warm-up and timing (steady-state headline)")
-    ap.add_argument("--sub", default="int4,prefill", help="bounded sub-records added to the decode line (N=1 only)")
+    ap.add_argument("--sub", default="int4,mxfp4,prefill", help="bounded sub-records added to the decode line (N=1 only)")
     ap.add_argument("--overlap", type=int, default=0,
                     help="launch mode of the streaming kernel in the timed region (ft_moe_set_launch_overlap)")
     args = ap.parse_args()
