@@ -185,8 +185,9 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    dsv3 = args.workload == "dsv3"
-    shape = W.DSV3_INT4 if dsv3 else W.QWEN3_30B
+    dsv3 = args.workload in ("dsv3", "dsv3_mxfp4")
+    mxfp4 = args.workload == "dsv3_mxfp4"
+    shape = (W.DSV3_MXFP4 if mxfp4 else W.DSV3_INT4) if dsv3 else W.QWEN3_30B
     RHO, ALPHA = (0.9, 1.2) if dsv3 else (0.8, 1.1)
     L = (4 if args.layers == 48 else args.layers) if dsv3 else args.layers
     E, k, d = shape.n_experts, shape.top_k, shape.d
@@ -217,7 +218,7 @@ def run_ours(args):
         cfg = Bd.make_config(hidden=d, inter=shape.inter, n_experts=E, top_k=k, n_layers=L, slots_per_layer=Ns,
                              max_tokens=max(B, 8), host_pool_ptr=pool.ptr.value, host_pool_bytes=pool.n_bytes,
                              fill_mode=fill_mode, device=local,
-                             wdtype=Bd.FT_W_INT4_G128 if shape.wdtype == "int4" else Bd.FT_W_BF16,
+                             wdtype={"int4": Bd.FT_W_INT4_G128, "mxfp4": Bd.FT_W_MXFP4, "bf16": Bd.FT_W_BF16}[shape.wdtype],
                              n_shared=shape.n_shared, shared_ptr=None if shared is None else shared.data_ptr(),
                              global_pool=args.global_pool, **bw)
         return Bd.FtMoe(cfg)
@@ -494,9 +495,11 @@ def run_ours(args):
         line = {
             "metric": "moe_decode_tok_per_s", "value": value, "unit": "tok/s", "n_gpus": world, "steps": K,
             "warmup": Wn, "ms_per_step": main["ms"] / K, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "int4 weights, bf16 activations, fp32 accumulate" if dsv3 else "bf16",
+            "vs_baseline": None, "dtype": ("mxfp4 weights, bf16 activations, fp32 accumulate" if mxfp4 else
+                                         "int4 weights, bf16 activations, fp32 accumulate") if dsv3 else "bf16",
             "data": "synthetic",
-            "config": {"workload": ("decode DeepSeek-V3-shaped int4 MoE stack (config 3)" if dsv3 else
+            "config": {"workload": ("decode DeepSeek-V3-shaped mxfp4 MoE stack (config 3 shapes)" if mxfp4 else
+                                    "decode DeepSeek-V3-shaped int4 MoE stack (config 3)" if dsv3 else
                                     "decode Qwen3-30B-A3B-shaped MoE stack (config 1)"), "batch": B, "layers": L,
                        "hidden": d, "experts": E, "inter": shape.inter, "top_k": k, "slots_per_layer": Ns,
                        "fill_mode": args.fill, "cuda_graph": use_graph, "global_pool": bool(args.global_pool), "rho": RHO, "zipf_alpha": ALPHA,
@@ -510,7 +513,8 @@ def run_ours(args):
             "gpu_launches": main["launches"],
             "roofline": {
                 "bound": "hbm",
-                "kernel": ("w4_gateup_kernel + w4_down_kernel (one pass over each record)" if dsv3
+                "kernel": ("mx4_gateup_kernel + mx4_down_kernel (one pass over each record)" if mxfp4 else
+                           "w4_gateup_kernel + w4_down_kernel (one pass over each record)" if dsv3
                            else "ffn_stream_kernel (expert FFN over the HBM-resident records of a layer)"),
                 "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
                 "frac": achieved / hbm_peak if hbm_peak else None, "peak_source": peak_kind + " (burst: kernel timed alone)",
@@ -960,7 +964,7 @@ def main():
     ap.add_argument("--sweep-batches", default="1,16,64")
     ap.add_argument("--global-pool", type=int, default=0, help="1: one slot pool and LRU clock shared by all layers")
     ap.add_argument("--graph", type=int, default=1, help="replay each decode step as one CUDA graph (SM fill only)")
-    ap.add_argument("--workload", default="qwen", choices=["qwen", "dsv3"])
+    ap.add_argument("--workload", default="qwen", choices=["qwen", "dsv3", "dsv3_mxfp4"])
     ap.add_argument("--mode", default="decode", choices=["decode", "prefill", "sweep"])
     ap.add_argument("--tokens", type=int, default=4096)
     ap.add_argument("--gemm-min-tokens", type=int, default=32)
