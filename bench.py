@@ -823,8 +823,10 @@ def sub_int4(args, dev, cal, wdtype="int4"):
     st1 = stats_sum()
     # the two int4 kernels (gate/up, down) timed alone: all layers planned and filled first, then the forward
     # calls back to back between two events
-    us, nbytes = [], []
-    for s in range(warm + K, warm + K + 8):
+    us, nbytes = {2: [], 0: []}, {2: [], 0: []}
+    for s in range(warm + K, warm + K + 12):
+        ov = 2 if s < warm + K + 6 else 0     # six steps with the launches overlapped, six plain
+        moe.set_launch_overlap(ov)
         a = stats_sum()
         for l in range(L):
             moe.route(l, lg[s, l], B, stream)
@@ -838,14 +840,17 @@ def sub_int4(args, dev, cal, wdtype="int4"):
             moe.forward(l, noise[s, l], ybuf[l], stream)
         f1.record(stream)
         torch.cuda.synchronize()
-        us.append(f0.elapsed_time(f1) * 1e3 / L)
-        nbytes.append((b["hits"] - a["hits"] + b["fills"] - a["fills"] + (b["steps"] - a["steps"])) * S / L)
+        us[ov].append(f0.elapsed_time(f1) * 1e3 / L)
+        nbytes[ov].append((b["hits"] - a["hits"] + b["fills"] - a["fills"] + (b["steps"] - a["steps"])) * S / L)
+    moe.set_launch_overlap(0)
     assert moe.sync_status() == 0
     moe.destroy()
     pool.free()
     hbm_peak, peak_kind = peaks()
-    t_us, nb = statistics.median(us[2:]), sum(nbytes[2:]) / len(nbytes[2:])
+    t_us, nb = statistics.median(us[2][1:]), sum(nbytes[2][1:]) / len(nbytes[2][1:])
     gbps = nb / (t_us * 1e-6) / 1e9
+    t0_us, nb0 = statistics.median(us[0][1:]), sum(nbytes[0][1:]) / len(nbytes[0][1:])
+    gbps0 = nb0 / (t0_us * 1e-6) / 1e9
     return {"config": "decode, config 3: d=7168, 256 %s experts + 1 shared, I=2048, top-8, 4 layers, 64 slots "
                       "per layer, batch 4, rho 0.9, alpha 1.2" % ("int4-g128" if wdtype == "int4" else "mxfp4"),
             "kernels": "w4_gateup_kernel + w4_down_kernel" if wdtype == "int4" else "mx4_gateup_kernel + mx4_down_kernel",
@@ -855,9 +860,12 @@ def sub_int4(args, dev, cal, wdtype="int4"):
             "fills_per_step": (st1["fills"] - st0["fills"]) / K, "cache_warm_steps": warm,
             "GBps": gbps, "frac": gbps / hbm_peak, "peak": hbm_peak, "peak_source": peak_kind,
             "avg_us_per_layer": t_us, "bytes_per_layer": nb,
+            "plain_back_to_back": {"avg_us_per_layer": t0_us, "GBps": gbps0, "frac": gbps0 / hbm_peak},
             "how": "gate/up + down kernels of a layer timed alone: the 4 layers of a step planned and filled first, "
-                   "then their forward calls back to back between two CUDA events; bytes = (resident routed experts "
-                   "+ the shared expert) x record bytes"}
+                   "then their forward calls back to back between two CUDA events, the gate/up kernels launched as "
+                   "programmatic dependents (ft_moe_set_launch_overlap 2: a layer's set-up overlaps the previous "
+                   "layer's tail); plain_back_to_back = the same with plain launches; bytes = (resident routed "
+                   "experts + the shared expert) x record bytes"}
 
 
 def sub_mxfp4(args, dev, cal):

@@ -108,6 +108,7 @@ __global__ void __launch_bounds__(kW4Threads, 1) mx4_gateup_kernel(W4Params p) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, q = lane & 3;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (p.overlap == 1) asm volatile("griddepcontrol.wait;" ::: "memory");
   const int n_items = *p.n_items, n_zc = *p.n_zc;
   for (int i = tid; i <= p.max_items; i += kW4Threads) s_pref[i] = p.pref[i];
   {
@@ -294,6 +295,9 @@ __global__ void __launch_bounds__(kW4Threads, 1) mx4_gateup_kernel(W4Params p) {
     stage_x([&](int j) { return j < p.T ? j : -1; });
     __syncthreads();
   }
+  // launched as a programmatic dependent with the caller's word that x and the plan are not produced by the
+  // preceding kernel: only from here on (the h buffers, shared with that kernel) must it have completed
+  if (p.overlap == 2) asm volatile("griddepcontrol.wait;" ::: "memory");
   const uint32_t n_warps = gridDim.x * kW4Warps, wi = blockIdx.x * kW4Warps + warp;
   for (int range = 0; range < 2; ++range) {
     const uint32_t pass0 = range ? (uint32_t)s_pref[n_items] : 0u;

@@ -60,6 +60,7 @@ struct W4Params {
   uint32_t *done;
   uint32_t *status;
   int inter, top_k, T, finalize;
+  int overlap;              // launch mode of the gate/up kernel, as FfnStreamParams::overlap (0 plain, 1, 2)
   // 0x0F0F0F0F and 0x08080808, passed as data: as literals the compiler encodes both as immediates and needs two
   // logic instructions per register (an instruction carries one immediate); as values it cannot see through they
   // live in registers and (x & mask) ^ flip is a single three-input logic instruction
@@ -160,6 +161,7 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_gateup_kernel(W4Params p) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, q = lane & 3;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the down kernel may set itself up meanwhile
+  if (p.overlap == 1) asm volatile("griddepcontrol.wait;" ::: "memory");
   const int n_items = *p.n_items, n_zc = *p.n_zc;
   for (int i = tid; i <= p.max_items; i += kW4Threads) s_pref[i] = p.pref[i];
   {
@@ -375,6 +377,9 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_gateup_kernel(W4Params p) {
     stage_x([&](int j) { return j < p.T ? j : -1; });
     __syncthreads();
   }
+  // launched as a programmatic dependent with the caller's word that x and the plan are not produced by the
+  // preceding kernel: only from here on (the h buffers, shared with that kernel) must it have completed
+  if (p.overlap == 2) asm volatile("griddepcontrol.wait;" ::: "memory");
   // Units (pass, 16-neuron block) in one flat order, split evenly over all warps of the grid: the slot-resident
   // range first, then the host-resident range.
   const uint32_t n_warps = gridDim.x * kW4Warps, wi = blockIdx.x * kW4Warps + warp;

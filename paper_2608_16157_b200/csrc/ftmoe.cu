@@ -1034,6 +1034,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   qp.max_items = 2 * c.n_experts + 1;
   qp.x = x_bf; qp.perm = sc.perm; qp.topk_w = sc.topk_w;
   const bool mx = c.wdtype == FT_W_MXFP4;
+  qp.overlap = h->overlap;
   if (mx) { qp.mask = 0x1C1C1C1Cu; qp.flip = 0x80808080u; }   // (see ffn_mx4.cuh)
   else { qp.mask = 0x0F0F0F0Fu; qp.flip = 0x08080808u; }
   qp.hraw = h->w4_hraw; qp.hcount = h->w4_hcount; qp.hq = h->w4_hq; qp.hs = h->w4_hs;
@@ -1047,25 +1048,33 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   const int grid = h->sm_count;
   {
     TimeScope ts(h, st, FT_TIME_FFN_ZC);   // (timing slot reused for the gate/up kernel of the 4-bit paths)
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(grid); lc.blockDim = dim3(kW4Threads); lc.dynamicSmemBytes = sa; lc.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = at; lc.numAttrs = h->overlap ? 1 : 0;
+    cudaError_t le;
     if (mx) {
       switch (c.hidden) {
-        case 512: mx4_gateup_kernel<4><<<grid, kW4Threads, sa, st>>>(qp); break;
-        case 1024: mx4_gateup_kernel<8><<<grid, kW4Threads, sa, st>>>(qp); break;
-        case 2048: mx4_gateup_kernel<16><<<grid, kW4Threads, sa, st>>>(qp); break;
-        case 4096: mx4_gateup_kernel<32><<<grid, kW4Threads, sa, st>>>(qp); break;
-        case 7168: mx4_gateup_kernel<56><<<grid, kW4Threads, sa, st>>>(qp); break;
-        default: mx4_gateup_kernel<64><<<grid, kW4Threads, sa, st>>>(qp); break;
+        case 512: le = cudaLaunchKernelEx(&lc, mx4_gateup_kernel<4>, qp); break;
+        case 1024: le = cudaLaunchKernelEx(&lc, mx4_gateup_kernel<8>, qp); break;
+        case 2048: le = cudaLaunchKernelEx(&lc, mx4_gateup_kernel<16>, qp); break;
+        case 4096: le = cudaLaunchKernelEx(&lc, mx4_gateup_kernel<32>, qp); break;
+        case 7168: le = cudaLaunchKernelEx(&lc, mx4_gateup_kernel<56>, qp); break;
+        default: le = cudaLaunchKernelEx(&lc, mx4_gateup_kernel<64>, qp); break;
       }
     } else {
       switch (c.hidden) {
-        case 512: w4_gateup_kernel<4><<<grid, kW4Threads, sa, st>>>(qp); break;
-        case 1024: w4_gateup_kernel<8><<<grid, kW4Threads, sa, st>>>(qp); break;
-        case 2048: w4_gateup_kernel<16><<<grid, kW4Threads, sa, st>>>(qp); break;
-        case 4096: w4_gateup_kernel<32><<<grid, kW4Threads, sa, st>>>(qp); break;
-        case 7168: w4_gateup_kernel<56><<<grid, kW4Threads, sa, st>>>(qp); break;
-        default: w4_gateup_kernel<64><<<grid, kW4Threads, sa, st>>>(qp); break;
+        case 512: le = cudaLaunchKernelEx(&lc, w4_gateup_kernel<4>, qp); break;
+        case 1024: le = cudaLaunchKernelEx(&lc, w4_gateup_kernel<8>, qp); break;
+        case 2048: le = cudaLaunchKernelEx(&lc, w4_gateup_kernel<16>, qp); break;
+        case 4096: le = cudaLaunchKernelEx(&lc, w4_gateup_kernel<32>, qp); break;
+        case 7168: le = cudaLaunchKernelEx(&lc, w4_gateup_kernel<56>, qp); break;
+        default: le = cudaLaunchKernelEx(&lc, w4_gateup_kernel<64>, qp); break;
       }
     }
+    FT_CUDA(le);
   }
   {
     TimeScope ts(h, st, FT_TIME_FFN_RES);
