@@ -127,8 +127,8 @@ typedef struct {
   const void *shared_weights; /* HOST, n_layers*n_shared records, copied to HBM at create; may be
                                  NULL when n_shared == 0 */
   /* Frozen integer constants of the plan's cost model, MB/s (1e6 bytes/s); all must be > 0 except
-   * bw_zc_residual_MBps which may be 0 (then every miss that can get a slot is filled: the paper's
-   * degenerate "pure on-demand cache fill", text after Eq. 4). */
+   * bw_zc_residual_MBps which may be 0 (then every miss that can get a slot is filled: the limit
+   * of Eq. 4 in which the split degenerates to on-demand fills only, see the text after Eq. 4). */
   uint32_t bw_fill_MBps;        /* B_f: copy-engine fill rate            (the paper's B_PCIe)      */
   uint32_t bw_zc_MBps;          /* B_z: zero-copy read rate alone                                   */
   uint32_t bw_zc_residual_MBps; /* B_r: zero-copy rate while fills saturate the link (Eq. 2)        */
@@ -184,8 +184,8 @@ ft_status_t ft_moe_host_unregister(void *host);
 ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out);
 ft_status_t ft_moe_destroy(ft_moe_t *h);
 
-/* Bandwidth profiling at deployment (paper Sec. 3.2, "empirically profiled on the target
- * hardware"): out_MBps = { fill (pinned H2D copy of records), zero-copy alone, zero-copy while the
+/* Bandwidth profiling at deployment (paper Sec. 3.2: the two bandwidths of Eq. 2 are measured on the machine that
+ * serves): out_MBps = { fill (pinned H2D copy of records), zero-copy alone, zero-copy while the
  * copy engine is saturated, HBM streaming }.  Measures only; plans keep using the frozen constants
  * given at create.  Synchronises the device. */
 ft_status_t ft_moe_calibrate(ft_moe_t *h, uint32_t out_MBps[4]);
@@ -196,7 +196,7 @@ ft_status_t ft_moe_calibrate(ft_moe_t *h, uint32_t out_MBps[4]);
  * permutation perm[P] / inv[P] of the P = T*k pairs p = t*k + j. */
 ft_status_t ft_moe_route(ft_moe_t *h, int layer, const float *logits_dev, int T, void *stream);
 
-/* Step 3 (paper Sec. 3.2 Eq. 1-4 and Sec. 4.1 "device-side cache control"): one device kernel
+/* Step 3 (paper Sec. 3.2 Eq. 1-4; Sec. 4.1: the cache is controlled on the device): one device kernel
  * deduplicates the routed experts, classifies them against the slot table, refreshes the stamps of
  * hits, orders the evictable slots (free first, then least recently used, ties to the lower
  * resident expert id), sizes the fill set q = min(max(1, round(m*B_f/(B_f+B_r))), eligible, K),
@@ -205,7 +205,7 @@ ft_status_t ft_moe_route(ft_moe_t *h, int layer, const float *logits_dev, int T,
  * plan and fills *out_host (HOST arrays owned by the caller). */
 ft_status_t ft_moe_plan(ft_moe_t *h, int layer, ft_moe_plan_t *out_host, void *stream);
 
-/* Step 4 (paper Sec. 3.2: the fill set F is brought into the cache "by a batch copy" before the grouped
+/* Step 4 (paper Sec. 3.2: the fill set F is copied into the cache as one batch before the grouped
  * evaluation; Sec. 4.1: one fixed-shape transfer driven by a device-resident source/destination list with a
  * valid count): for every (expert, slot) of F copy the S-byte pool record into the slot on copy_stream and
  * record the handle's fill event there.  The copies are ordered after the plan. */
@@ -220,8 +220,7 @@ ft_status_t ft_moe_fill(ft_moe_t *h, int layer, void *copy_stream);
  * layer's later route/plan finds hits.  The handle's fill event is recorded: the next ft_moe_forward waits for
  * it.  Needs room for two full-layer buffers: with global_pool a shared pool of at least 2*n_experts slots,
  * otherwise slots_per_layer >= n_experts; else FT_ERR_UNSUPPORTED and the caller falls back to on-demand fills
- * (paper: "if the memory budget cannot support two full-layer buffers, prefill falls back to on-demand
- * loading").  The layer must be idle (no route/plan/fill of it pending). */
+ * (Sec. 3.1 names the same fallback for budgets without room for two full-layer buffers).  The layer must be idle (no route/plan/fill of it pending). */
 ft_status_t ft_moe_prefetch_layer(ft_moe_t *h, int layer, void *stream, void *copy_stream);
 
 /* Steps 5+6 (paper Sec. 3.2: grouped evaluation of H u F on the GPU, the in-place set beside it, and an exact

@@ -4,7 +4,7 @@ A plain, slow, obviously-correct numpy/fp64 statement of what the layer
 computes, written from the paper's description of the method (Sec. 3 intro:
 host expert pool = source of truth, HBM slots = cache; Sec. 3.2: hit set,
 miss partition Eq. 1, residual bandwidth Eq. 2, branch times Eq. 3, fill count
-q* Eq. 4, "always retains at least one fill", LRU residency; Sec. 4.1: one
+q* Eq. 4 with at least one miss always filled, LRU residency; Sec. 4.1: one
 pass yields the K least-recently-used candidate slots).  It shares no code
 with the CUDA library and must never be imported by the product path: only
 tests, the smoke check and the benchmark's CPU-baseline leg use it.
@@ -44,7 +44,7 @@ LOC_ZERO_COPY = -2
 
 
 # ---------------------------------------------------------------------------
-# Step 1: routing (Sec. 3.2: "the router and cache lookup run on the GPU")
+# Step 1: routing (Sec. 3.2: router and cache lookup both run on the GPU)
 # ---------------------------------------------------------------------------
 
 def route(logits: np.ndarray, k: int) -> tuple[np.ndarray, np.ndarray]:
@@ -75,7 +75,7 @@ def route(logits: np.ndarray, k: int) -> tuple[np.ndarray, np.ndarray]:
 
 
 # ---------------------------------------------------------------------------
-# Step 2: permutation of (token, choice) pairs by expert ("grouped evaluation")
+# Step 2: permutation of (token, choice) pairs by expert (experts are evaluated as groups of tokens, Sec. 3.2)
 # ---------------------------------------------------------------------------
 
 def permute(ids: np.ndarray, n_experts: int):

@@ -45,7 +45,7 @@ def test_q_is_rounded_m_bp_over_bh_on_table1():
         for m in range(0, 40):
             exact = Fraction(m * bp, bh)                      # Eq. 4
             rounded = int(exact + Fraction(1, 2))             # half up
-            want = 0 if m == 0 else max(1, rounded)           # "always retains at least one fill"
+            want = 0 if m == 0 else max(1, rounded)           # at least one miss is always filled (Eq. 4)
             assert O.fill_count_bw(m, bp, bh - bp) == want
 
 
