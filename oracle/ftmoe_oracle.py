@@ -143,7 +143,7 @@ class Plan:
 
 
 class CacheState:
-    """Per-layer residency table (Sec. 3.2 "shared LRU residency space", here one per layer)."""
+    """Per-layer residency table (the LRU residency space of Sec. 3.2, which the paper shares across layers; here one per layer)."""
 
     def __init__(self, n_experts: int, n_slots: int):
         self.n_experts = n_experts
