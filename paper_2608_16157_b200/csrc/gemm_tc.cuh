@@ -8,7 +8,7 @@
 // 64 bytes): a weight tile is moved by plain TMA boxes of whole 1 KiB tiles and described to the MMA with a
 // 512-byte step between 8-row groups; the two K = 16 slices of a tile are 32 bytes apart.
 // One persistent CTA per SM: warp 0 feeds a 4-stage shared-memory ring with TMA tile loads (cp.async.bulk.tensor,
-// no multicast), warp 1 issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32) into one of two
+// each into this CTA's shared memory only), warp 1 issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32) into one of two
 // 256-column TMEM accumulators and signals stages free / tiles done with tcgen05.commit, warps 2-5 drain the other
 // accumulator with tcgen05.ld, apply SwiGLU and store bf16, so the epilogue of tile i overlaps the main loop of
 // tile i+1.  Every mbarrier wait is bounded; on expiry the CTA latches a timeout status, stops waiting, frees its

@@ -3,9 +3,9 @@
 //
 // Two CTAs of a cluster (two SMs) work on one tile with tcgen05.mma.cta_group::2 (M = 256 over the pair): each
 // CTA stages its own 128 rows of A and one half of the rows of B, the leader CTA issues the MMAs for both, and
-// each CTA's TMEM receives the accumulators of its own 128 rows, double-buffered against the epilogue.  No multicast loads are used: every
-// CTA issues its own TMA loads (with .cta_group::2 so that they can signal the leader's mbarrier); stage
-// release and accumulator hand-over go through tcgen05.commit with a two-CTA mask.
+// each CTA's TMEM receives the accumulators of its own 128 rows, double-buffered against the epilogue.  Every
+// CTA issues its own TMA loads, each for its own shared memory only (with .cta_group::2 so that they can signal the leader's mbarrier); stage
+// release and accumulator hand-over go through one tcgen05.commit per CTA of the pair.
 // Every mbarrier wait is bounded; on expiry the CTA latches a timeout status and runs to completion.
 #pragma once
 #include "gemm_tc.cuh"
