@@ -36,7 +36,7 @@ RHO, ALPHA = 0.8, 1.1
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
 # DRAM bytes (read + write) of one ffn_stream_kernel launch over its algorithmic bytes, from the ncu capture
 # summarised in profiles/ (same kernel, batch 8, 24 resident experts per launch)
-NCU_TRAFFIC_RATIO = 1.03
+NCU_TRAFFIC_RATIO = 1.025
 NCU_TRAFFIC_SOURCE = "profiles/ffn_stream_kernel_decode_qwen3_b8.md"
 
 
