@@ -68,12 +68,13 @@
  *                   tile 64 scale bytes = for r in 0..7 the four block scales (j = 0..3) of row r, then those of row
  *                   r+8.  Section C: order (ng, cb, w, g, j, half, m), i.e. per lane g 32 bytes = for each tile j and
  *                   column half the scales of the four 32-neuron blocks m of the 128-neuron group.
- *                   S = 3*inter*hidden/2 + 3*inter*hidden/32 bytes.  Decode-sized calls only (no tensor-core prefill
- *                   path); shapes as for int4.
+ *                   S = 3*inter*hidden/2 + 3*inter*hidden/32 bytes.  Shapes as for int4.
  *   Shape limits: bf16: hidden in {256, 512, 1024, 2048}, inter % 16 == 0; int4 and mxfp4: hidden in
  *   {512, 1024, 2048, 4096, 7168, 8192}, inter % 128 == 0; n_experts <= 1024;
- *   top_k <= min(n_experts, 32); slots per table (slots_per_layer, or n_layers*slots_per_layer with global_pool) <= 6144.  The tensor-core prefill path
- *   (gemm_min_tokens > 0) needs bf16 weights, slots_per_layer > 0 and inter % 256 == 0.
+ *   top_k <= min(n_experts, 32); slots per table (slots_per_layer, or n_layers*slots_per_layer with global_pool)
+ *   <= 6144.  The tensor-core prefill path (gemm_min_tokens > 0) needs slots_per_layer > 0, hidden % 256 == 0 and
+ *   inter % 256 == 0; int4 and mxfp4 experts on that path are first expanded, once per call, to bf16 records in a
+ *   scratch pool of slots_per_layer x 3*inter*hidden*2 bytes owned by the handle (not with global_pool).
  */
 #ifndef FTMOE_H_
 #define FTMOE_H_

@@ -1,0 +1,96 @@
+// Many-token calls on 4-bit experts: the experts that go through the tensor-core GEMMs are first expanded, once per
+// call, from their slot into a bf16 record in tile order (the layout the GEMMs' tensor maps read, see
+// include/ftmoe.h) in a per-layer scratch pool.  With hundreds of tokens per expert the expansion (one pass over
+// the record) is small beside the GEMMs, and the GEMMs then run on exact bf16 activations: int4 weights are rounded
+// to bf16 after the multiplication by their scale (11-12 significant bits -> 8), MXFP4 weights are exact in bf16.
+// One thread produces one 16-byte chunk of the destination (8 weights), in destination order, so that the writes
+// are coalesced; the 4-byte source words come from L2.
+#pragma once
+#include "common.cuh"
+#include "ffn_w4.cuh"
+#include "gemm_tc.cuh"   // pack_bf16
+
+namespace ftmoe {
+
+struct DequantParams {
+  const WorkItem *items;    // the GEMM work list: record pointer (slot) and slot index per expert
+  const int32_t *n_items;
+  uint8_t *scratch;         // [slots_per_layer][3 * inter * d * 2] bf16 records in tile order
+  int d, inter;
+};
+
+__device__ __forceinline__ float w4_code_value(uint32_t nib, bool mx) {
+  if (!mx) return (float)((int)(nib ^ 8u) - 8);                 // two's-complement nibble
+  const uint32_t e = (nib >> 1) & 3u, m = nib & 1u;             // e2m1: 0, 0.5 | (1 + m/2) * 2^(e-1)
+  const float mag = e == 0 ? 0.5f * (float)m : __uint_as_float(((e + 126u) << 23) | (m << 22));
+  return (nib & 8u) ? -mag : mag;
+}
+
+template <bool MX>
+__global__ void __launch_bounds__(256) dequant_w4_kernel(DequantParams p) {
+  const int d = p.d, I = p.inter;
+  const uint32_t G = (uint32_t)d / 128u, NG = (uint32_t)I / 128u, NBLK = (uint32_t)I / 16u;
+  const uint32_t NWD = min(16u, (uint32_t)d / 64u), CBW = 64u * NWD, CB = (uint32_t)d / CBW;
+  const size_t UA = (size_t)(MX ? 2176u : 2112u) * G;
+  const size_t sec_b = (size_t)NBLK * UA, sec_c = sec_b + (size_t)I * d / 2;
+  const size_t S16 = (size_t)3 * I * d * 2;
+  const uint32_t chunks_unit = 6u * (uint32_t)d;                // 16-byte chunks of a 96*d-byte destination unit
+  const size_t chunks_rec = (size_t)NBLK * chunks_unit;
+  const int n_items = *p.n_items;
+  const size_t total = (size_t)n_items * chunks_rec;
+  for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
+    const int item = (int)(idx / chunks_rec);
+    const size_t in_rec = idx - (size_t)item * chunks_rec;
+    const uint32_t u = (uint32_t)(in_rec / chunks_unit), k = (uint32_t)(in_rec - (size_t)u * chunks_unit);
+    const uint8_t *rec = p.items[item].w;
+    uint8_t *dst = p.scratch + (size_t)p.items[item].slot * S16 + (size_t)u * 96u * d + (size_t)k * 16u;
+    float v[8];
+    if (k < 4u * (uint32_t)d) {
+      // ---- gate (k < 2d) or up part: tile t of 16 neurons x 32 hidden indices, rows of 64 bytes, swizzled ----
+      const uint32_t mm = k / (2u * d), kk = k - mm * 2u * d;
+      const uint32_t t = kk >> 6, r = (kk >> 2) & 15u, pos = kk & 3u;
+      const uint32_t q = pos ^ ((r & 7u) >> 1);                 // chunk q of the row is stored at position pos
+      const uint32_t grp = t >> 2, j = t & 3u;                  // hidden indices 128 grp + 32 j + 8 q + 0..7
+      const uint8_t *unit = rec + (size_t)u * UA;
+      const uint32_t w = *reinterpret_cast<const uint32_t *>(unit + (size_t)mm * 1024u * G + grp * 1024u + r * 64u + q * 16u + j * 4u);
+      float scale;
+      if (MX) {
+        const uint32_t b = unit[2048u * G + mm * 64u * G + grp * 64u + (r & 7u) * 8u + (r >> 3) * 4u + j];
+        scale = __uint_as_float(b << 23);
+      } else {
+        const uint16_t s = *reinterpret_cast<const uint16_t *>(unit + 2048u * G + mm * 32u * G + grp * 32u + (r & 7u) * 4u + (r >> 3) * 2u);
+        scale = __uint_as_float((uint32_t)s << 16);
+      }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] = scale * w4_code_value((w >> (4 * e)) & 15u, MX);
+    } else {
+      // ---- down part: tile ct of 16 columns x the unit's 16 neurons, rows of 32 bytes, swizzled ----
+      const uint32_t kk = k - 4u * d;
+      const uint32_t ct = kk >> 5, cg = (kk >> 4) & 1u, rr = (kk >> 1) & 7u, pos = kk & 1u;
+      const uint32_t nhalf = pos ^ (rr >> 2);                   // neurons 8 nhalf .. 8 nhalf + 7 of the unit
+      const uint32_t c = 16u * ct + 8u * cg + rr;               // output column
+      const uint32_t ng = u >> 3, uu = u & 7u;
+      const uint32_t cb = c / CBW, tt = (c - cb * CBW) >> 4, wq = tt >> 2, j = tt & 3u;
+      const uint8_t *src = rec + sec_b + ((((size_t)(cb * NG + ng) * 8u + uu) * NWD + wq) * 32u + 4u * rr + 2u * nhalf) * 16u + 4u * j;
+      const uint32_t w0 = *reinterpret_cast<const uint32_t *>(src), w1 = *reinterpret_cast<const uint32_t *>(src + 16);
+      float scale;
+      if (MX) {
+        const uint32_t b = rec[sec_c + ((size_t)(ng * CB + cb) * NWD + wq) * 256u + 32u * rr + 8u * j + 4u * cg + (uu >> 1)];
+        scale = __uint_as_float(b << 23);
+      } else {
+        const uint16_t s = *reinterpret_cast<const uint16_t *>(rec + sec_c + ((size_t)(ng * CB + cb) * NWD + wq) * 128u + 16u * rr + 4u * j + 2u * cg);
+        scale = __uint_as_float((uint32_t)s << 16);
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {   // neuron 8 nhalf + i: word i / 4, nibble 2 (i % 4) + column half
+        const uint32_t w = i < 4 ? w0 : w1;
+        v[i] = scale * w4_code_value((w >> (4 * (2 * (i & 3) + (int)cg))) & 15u, MX);
+      }
+    }
+    uint4 o;
+    o.x = pack_bf16(v[0], v[1]); o.y = pack_bf16(v[2], v[3]); o.z = pack_bf16(v[4], v[5]); o.w = pack_bf16(v[6], v[7]);
+    *reinterpret_cast<uint4 *>(dst) = o;
+  }
+}
+
+}  // namespace ftmoe

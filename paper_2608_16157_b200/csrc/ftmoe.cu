@@ -10,6 +10,7 @@
 
 #include "common.cuh"
 #include "ffn_stream.cuh"
+#include "dequant_w4.cuh"
 #include "ffn_mx4.cuh"
 #include "ffn_w4.cuh"
 #include "gemm_tc.cuh"
@@ -85,6 +86,7 @@ struct ft_moe {
   __nv_bfloat16 *xs = nullptr, *hbuf = nullptr, *obuf = nullptr;   // [P][d], [P][I], [P][d]
   CUtensorMap tm_xs, tm_h;       // x rows, H rows (128-row boxes, 128-byte swizzle)
   CUtensorMap tm_wgu, tm_wd;     // the slot pool as [unit][1 KiB gate/up tile] and [unit][2 KiB of down tiles]
+  uint8_t *wq_scratch = nullptr; // 4-bit experts on the GEMM path: [slots_per_layer] bf16 records (tile order) of the call's layer
   uint32_t *status_dev = nullptr;
   uint32_t *seq_dev = nullptr;
   uint32_t *done_dev = nullptr;          // CTA completion counter of the streaming MMA kernel
@@ -338,14 +340,66 @@ ft_status_t build_weight_maps(ft_moe *h) {
   FT_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fnp, cudaEnableDefault, &qres));
   if (!fnp || qres != cudaDriverEntryPointSuccess) return FT_ERR_CUDA;
   EncodeTiledFn enc = reinterpret_cast<EncodeTiledFn>(fnp);
-  const uint64_t n_units = (uint64_t)c.n_layers * c.slots_per_layer * (c.inter / 16);
+  // bf16 experts are read from their slots; 4-bit experts from the bf16 scratch records of the call's layer
+  const bool scratch = c.wdtype != FT_W_BF16;
+  const uint64_t n_units = (uint64_t)(scratch ? 1 : c.n_layers) * c.slots_per_layer * (c.inter / 16);
   const uint64_t unit_bytes = 96ull * c.hidden;
+  uint8_t *base = scratch ? h->wq_scratch : h->slots;
   if (n_units == 0) return FT_OK;   // no slots: nothing goes through the GEMMs
   // gate/up: one 1 KiB tile (16 neurons x 32 hidden indices) of 8 consecutive units = 128 neurons;
   // down: 4 KiB (the tiles of 128 output columns) of 4 consecutive units = 64 neurons
-  if (!make_unit_map(enc, &h->tm_wgu, h->slots, n_units, unit_bytes, 1024, 1, 8) ||
-      !make_unit_map(enc, &h->tm_wd, h->slots, n_units, unit_bytes, 2048, 2, 4))
+  if (!make_unit_map(enc, &h->tm_wgu, base, n_units, unit_bytes, 1024, 1, 8) ||
+      !make_unit_map(enc, &h->tm_wd, base, n_units, unit_bytes, 2048, 2, 4))
     return FT_ERR_CUDA;
+  return FT_OK;
+}
+
+// The experts with many tokens (the plan's GEMM list): gather x rows into expert order, two grouped tcgen05 GEMMs
+// over the weight tensor maps, fused gather-combine that also rounds y.
+ft_status_t launch_gemm_path(ft_moe *h, int layer, const LayerState &L, const Scratch &sc, const __nv_bfloat16 *x_bf,
+                             void *y_dev, cudaStream_t st) {
+  const ft_moe_config_t &c = h->cfg;
+    // experts with many tokens: gather x rows into expert order, two grouped tcgen05 GEMMs, fused combine
+    {
+      TimeScope ts(h, st, FT_TIME_GATHER);
+      gather_rows_kernel<<<h->sm_count * 8, 256, 0, st>>>(x_bf, sc.perm, c.top_k, c.hidden, sc.offset + c.n_experts, h->xs);
+    }
+    GemmParams gp;
+    gp.items = sc.items_gemm; gp.n_items = &sc.plan_dev->n_gemm_items; gp.mt_pref = sc.gemm_pref;
+    gp.inter = c.inter; gp.d = c.hidden;
+    gp.layer_unit0 = (c.global_pool || c.wdtype != FT_W_BF16) ? 0 : (long long)layer * c.slots_per_layer * (c.inter / 16);
+    gp.status = h->status_dev;
+    // CTA pairs (clusters of two) share every 256x256 tile
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3((unsigned)(h->sm_count & ~1));
+    lc.blockDim = dim3(kGemmThreads);
+    lc.stream = st;
+    cudaLaunchAttribute la[1];
+    la[0].id = cudaLaunchAttributeClusterDimension;
+    la[0].val.clusterDim.x = 2; la[0].val.clusterDim.y = 1; la[0].val.clusterDim.z = 1;
+    lc.attrs = la;
+    lc.numAttrs = 1;
+    // gate/up + SwiGLU: one CTA per 128 x 256 tile (A = x rows, B = 128 gate + 128 up rows); measured faster
+    // than the CTA-pair form for this GEMM, whose fused epilogue needs gate and up in the same TMEM
+    gp.K = c.hidden; gp.n_tiles = c.inter / 128; gp.out = h->hbuf;
+    {
+      TimeScope ts(h, st, FT_TIME_GEMM1);
+      gateup_gemm_kernel<<<h->sm_count, kGemmThreads, gateup_gemm_smem_bytes(), st>>>(h->tm_xs, h->tm_wgu, gp);
+    }
+    // down: A = the down tiles of 128 columns x 64 neurons per CTA, B = H rows (box 64 x 128 per CTA)
+    gp.K = c.inter; gp.out = h->obuf;
+    lc.dynamicSmemBytes = down_gemm2_smem_bytes();
+    {
+      TimeScope ts(h, st, FT_TIME_GEMM2);
+      FT_CUDA(cudaLaunchKernelEx(&lc, down_gemm2_kernel, h->tm_wd, h->tm_h, gp));
+    }
+    {
+      TimeScope ts(h, st, FT_TIME_COMBINE);
+      combine_kernel<<<h->sm_count * 8, 256, 0, st>>>(h->obuf, sc.ids, sc.topk_w, sc.inv, sc.is_gemm, h->y_acc,
+                                                      static_cast<__nv_bfloat16 *>(y_dev), L.T, c.top_k, c.hidden);
+    }
+    h->launches += 4;
+    FT_CUDA(cudaGetLastError());
   return FT_OK;
 }
 
@@ -431,6 +485,7 @@ ft_status_t ft_moe_destroy(ft_moe_t *h) {
   cudaFree(h->gemm_pref);
   cudaFree(h->is_gemm);
   cudaFree(h->xs);
+  cudaFree(h->wq_scratch);
   cudaFree(h->hbuf);
   cudaFree(h->obuf);
   cudaFree(h->status_dev);
@@ -477,7 +532,8 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
   const size_t S = expert_bytes_of(cfg);
   if (S == 0 || (c.wdtype != FT_W_BF16 && !w4_shape_ok(c))) return FT_ERR_UNSUPPORTED;
   if (c.gemm_min_tokens != 0 &&
-      (c.wdtype != FT_W_BF16 || c.slots_per_layer == 0 || c.hidden % 256 || c.inter % 256 || c.gemm_min_tokens < 8))
+      (c.slots_per_layer == 0 || c.hidden % 256 || c.inter % 256 || c.gemm_min_tokens < 8 ||
+       (c.wdtype != FT_W_BF16 && c.global_pool)))   // (4-bit: the bf16 scratch mirrors one layer's slots)
     return FT_ERR_UNSUPPORTED;
   if (!c.host_pool || c.host_pool_bytes < (size_t)c.n_layers * c.n_experts * S) return FT_ERR_INVALID_ARG;
   if (c.n_shared && !c.shared_weights) return FT_ERR_INVALID_ARG;
@@ -580,6 +636,8 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
     if (!make_tensor_map(enc, &h->tm_xs, h->xs, Pr, c.hidden, 128, 64) ||
         !make_tensor_map(enc, &h->tm_h, h->hbuf, Pr, c.inter, 128, 64))
       return fail(FT_ERR_CUDA);
+    if (c.wdtype != FT_W_BF16)
+      FT_TRY(cudaMalloc(&h->wq_scratch, (size_t)c.slots_per_layer * 3 * c.inter * c.hidden * 2));
     rc = build_weight_maps(h);
     if (rc != FT_OK) return fail(rc);
     FT_TRY(cudaFuncSetAttribute(gateup_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -979,49 +1037,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     }
     FT_CUDA(launch_err);
     FT_CUDA(cudaGetLastError());
-    if (use_gemm) {
-      // experts with many tokens: gather x rows into expert order, two grouped tcgen05 GEMMs, fused combine
-      {
-        TimeScope ts(h, st, FT_TIME_GATHER);
-        gather_rows_kernel<<<h->sm_count * 8, 256, 0, st>>>(x_bf, sc.perm, c.top_k, c.hidden, sc.offset + c.n_experts, h->xs);
-      }
-      GemmParams gp;
-      gp.items = sc.items_gemm; gp.n_items = &sc.plan_dev->n_gemm_items; gp.mt_pref = sc.gemm_pref;
-      gp.inter = c.inter; gp.d = c.hidden;
-      gp.layer_unit0 = c.global_pool ? 0 : (long long)layer * c.slots_per_layer * (c.inter / 16);
-      gp.status = h->status_dev;
-      // CTA pairs (clusters of two) share every 256x256 tile
-      cudaLaunchConfig_t lc = {};
-      lc.gridDim = dim3((unsigned)(h->sm_count & ~1));
-      lc.blockDim = dim3(kGemmThreads);
-      lc.stream = st;
-      cudaLaunchAttribute la[1];
-      la[0].id = cudaLaunchAttributeClusterDimension;
-      la[0].val.clusterDim.x = 2; la[0].val.clusterDim.y = 1; la[0].val.clusterDim.z = 1;
-      lc.attrs = la;
-      lc.numAttrs = 1;
-      // gate/up + SwiGLU: one CTA per 128 x 256 tile (A = x rows, B = 128 gate + 128 up rows); measured faster
-      // than the CTA-pair form for this GEMM, whose fused epilogue needs gate and up in the same TMEM
-      gp.K = c.hidden; gp.n_tiles = c.inter / 128; gp.out = h->hbuf;
-      {
-        TimeScope ts(h, st, FT_TIME_GEMM1);
-        gateup_gemm_kernel<<<h->sm_count, kGemmThreads, gateup_gemm_smem_bytes(), st>>>(h->tm_xs, h->tm_wgu, gp);
-      }
-      // down: A = the down tiles of 128 columns x 64 neurons per CTA, B = H rows (box 64 x 128 per CTA)
-      gp.K = c.inter; gp.out = h->obuf;
-      lc.dynamicSmemBytes = down_gemm2_smem_bytes();
-      {
-        TimeScope ts(h, st, FT_TIME_GEMM2);
-        FT_CUDA(cudaLaunchKernelEx(&lc, down_gemm2_kernel, h->tm_wd, h->tm_h, gp));
-      }
-      {
-        TimeScope ts(h, st, FT_TIME_COMBINE);
-        combine_kernel<<<h->sm_count * 8, 256, 0, st>>>(h->obuf, sc.ids, sc.topk_w, sc.inv, sc.is_gemm, h->y_acc,
-                                                        static_cast<__nv_bfloat16 *>(y_dev), L.T, c.top_k, c.hidden);
-      }
-      h->launches += 4;
-      FT_CUDA(cudaGetLastError());
-    }
+    if (use_gemm) return launch_gemm_path(h, layer, L, sc, x_bf, y_dev, st);
     return FT_OK;
   }
   // int4 / mxfp4: gate/up kernel writes h, down kernel accumulates, its last CTA finalizes y
@@ -1041,8 +1057,8 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   qp.y_acc = h->y_acc; qp.y = static_cast<__nv_bfloat16 *>(y_dev);
   qp.done = h->done_dev; qp.status = h->status_dev;
   qp.inter = c.inter; qp.top_k = c.top_k; qp.T = L.T;
-  const bool own_finalize = L.T > kFinalizeInKernelMaxTokens;
-  qp.finalize = own_finalize ? 0 : 1;
+  const bool own_finalize = !use_gemm && L.T > kFinalizeInKernelMaxTokens;
+  qp.finalize = (use_gemm || own_finalize) ? 0 : 1;   // (the GEMM path's combine rounds y)
   const size_t sa = mx ? mx4_gateup_smem_bytes(qp.max_items, c.hidden) : w4_gateup_smem_bytes(qp.max_items, c.hidden);
   const size_t sb = mx ? mx4_down_smem_bytes(qp.max_items) : w4_down_smem_bytes(qp.max_items);
   const int grid = h->sm_count;
@@ -1101,6 +1117,19 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   }
   h->launches += 2;
   FT_CUDA(cudaGetLastError());
+  if (use_gemm) {
+    // the experts of the GEMM list are expanded to bf16 records in the layer's scratch pool first
+    DequantParams dp;
+    dp.items = sc.items_gemm; dp.n_items = &sc.plan_dev->n_gemm_items; dp.scratch = h->wq_scratch;
+    dp.d = c.hidden; dp.inter = c.inter;
+    {
+      TimeScope ts(h, st, FT_TIME_GATHER);
+      if (mx) dequant_w4_kernel<true><<<h->sm_count * 8, 256, 0, st>>>(dp);
+      else dequant_w4_kernel<false><<<h->sm_count * 8, 256, 0, st>>>(dp);
+    }
+    h->launches++;
+    return launch_gemm_path(h, layer, L, sc, x_bf, y_dev, st);
+  }
   return FT_OK;
 }
 

@@ -16,11 +16,13 @@ def _zipf_logits(T, E, seed, step, alpha=1.1):
     return (rng.standard_normal((T, E)) + b).astype(np.float32)
 
 
+@pytest.mark.parametrize("wdtype", ["bf16", "int4", "mxfp4"])
 @pytest.mark.parametrize("T,n_slots", [(300, 8), (1000, 6), (129, 3)])
-def test_prefill_grouped_gemm_matches_oracle(T, n_slots):
-    """Experts with >= 32 tokens and a slot go through the tensor-core GEMMs, the rest through the
-    streaming kernels (slots or zero-copy); row tiles are ragged (token counts are Zipf-skewed)."""
-    shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2)
+def test_prefill_grouped_gemm_matches_oracle(T, n_slots, wdtype):
+    """Experts with >= 32 tokens and a slot go through the tensor-core GEMMs (4-bit experts after their expansion to
+    bf16 records in the scratch pool), the rest through the streaming kernels (slots or zero-copy); row tiles are
+    ragged (token counts are Zipf-skewed)."""
+    shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2, wdtype=wdtype)
     pr = Pair(shape, n_slots=n_slots, max_tokens=1000, seed=31, gemm_min_tokens=32)
     for step in range(2):
         logits = _zipf_logits(T, 8, 31, step)
@@ -28,11 +30,25 @@ def test_prefill_grouped_gemm_matches_oracle(T, n_slots):
         _, r = pr.step(0, logits, x, check_slots=(step == 0))
         if T >= 300:
             assert max(r.count) >= 128      # at least one expert spans more than one 128-row tile
+    assert pr.moe.get_stats(0)["pairs_gemm"] > 0   # the tensor-core path was taken
     pr.close()
 
 
-def test_prefill_then_decode_on_the_same_handle():
-    shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2)
+@pytest.mark.parametrize("wdtype", ["int4", "mxfp4"])
+def test_prefill_4bit_wide_hidden_size(wdtype):
+    """d=7168, I=2048 (the 4-bit decode configuration's layer shape), 8 experts, 256 tokens: K = 7168 in the gate/up
+    GEMM, 56 column tiles in the down GEMM, weights from the bf16 scratch records."""
+    shape = W.LayerShape(d=7168, inter=2048, n_experts=8, top_k=2, wdtype=wdtype)
+    pr = Pair(shape, n_slots=8, max_tokens=256, n_layers=1, seed=35, gen_device="cuda", gemm_min_tokens=32)
+    for step in range(2):
+        pr.step(0, _zipf_logits(256, 8, 35, step), W.noise_x(256, 7168, 35, step, 0), check_slots=(step == 0))
+    assert pr.moe.get_stats(0)["pairs_gemm"] > 0
+    pr.close()
+
+
+@pytest.mark.parametrize("wdtype", ["bf16", "mxfp4"])
+def test_prefill_then_decode_on_the_same_handle(wdtype):
+    shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2, wdtype=wdtype)
     pr = Pair(shape, n_slots=8, max_tokens=512, seed=33, gemm_min_tokens=32)
     pr.step(0, _zipf_logits(512, 8, 33, 0), W.noise_x(512, 512, 33, 0, 0))
     for step in range(1, 4):
