@@ -595,23 +595,27 @@ def tensor_peaks():
     return FALLBACK_BF16_TFLOPS, 1400.0, "fallback"
 
 
-def prefill_passes(args, dev, L, cal=None):
-    """Config 2 on L layers: one 4096-token step from a cold cache, then one on the cache it left behind.  Returns
-    (per-pass records, calibration, layer constants)."""
+def prefill_passes(args, dev, L, cal=None, shape=None, Ns=None):
+    """Config 2 (or another layer shape) on L layers: one 4096-token step from a cold cache, then one on the cache it
+    left behind.  Returns (per-pass records, calibration, layer constants)."""
     import torch
     from paper_2608_16157_b200 import binding as Bd
     from paper_2608_16157_b200 import workload as W
-    shape = W.QWEN3_30B
+    shape = shape or W.QWEN3_30B
     E, k, d, I = shape.n_experts, shape.top_k, shape.d, shape.inter
     S = shape.expert_bytes
-    Ns = W.slots_for_fraction(args.cache_frac, E)
+    Ns = Ns or W.slots_for_fraction(args.cache_frac, E)
     T = args.tokens
     pool = Bd.HostPool(L * E * S)
-    W.fill_pool(pool.tensor, shape, L, SEED, device=dev, chunk=32)
+    W.fill_pool(pool.tensor, shape, L, SEED, device=dev, chunk=32 if shape.wdtype == "bf16" else 16)
     common = dict(hidden=d, inter=I, n_experts=E, top_k=k, n_layers=L, slots_per_layer=Ns, max_tokens=T,
                   host_pool_ptr=pool.ptr.value, host_pool_bytes=pool.n_bytes,
                   fill_mode=Bd.FT_FILL_SM if args.fill == "sm" else Bd.FT_FILL_COPY_ENGINE,
+                  wdtype={"int4": Bd.FT_W_INT4_G128, "mxfp4": Bd.FT_W_MXFP4, "bf16": Bd.FT_W_BF16}[shape.wdtype],
                   gemm_min_tokens=args.gemm_min_tokens)
+    if shape.n_shared:
+        shared = W.make_shared_records(shape, L, SEED, device=dev)
+        common.update(n_shared=1, shared_ptr=shared.data_ptr())
     if cal is None:
         moe = Bd.FtMoe(Bd.make_config(**common))
         cal = moe.calibrate()
@@ -649,12 +653,14 @@ def prefill_passes(args, dev, L, cal=None):
         dst = {kk: st1[kk] - st0[kk] for kk in st1}
         flops = 2.0 * 3 * d * I * dst["pairs_gemm"]
         gemm_us = tim["gemm1"][0] + tim["gemm2"][0]
+        gather_us = tim["gather"][0]          # (4-bit experts: includes their expansion to bf16 records)
         fill_us = tim["fill"][0]
         route_us = tim["route"][0] + tim["plan"][0]
         out[name] = {"ms": ms, "tok_per_s": T / (ms * 1e-3), "launches": moe.launch_count() - l0 + L - 1,
                      "fills": dst["fills"], "zero_copy": dst["zc"], "hits": dst["hits"],
                      "pairs": dst["pairs"], "pairs_gemm": dst["pairs_gemm"],
                      "gemm_tflops": flops / (gemm_us * 1e-6) / 1e12 if gemm_us > 0 else None,
+                     "gemm_with_gather_tflops": flops / ((gemm_us + gather_us) * 1e-6) / 1e12 if gemm_us > 0 else None,
                      "gemm1_tflops": (flops * 2 / 3) / (tim["gemm1"][0] * 1e-6) / 1e12 if tim["gemm1"][0] > 0 else None,
                      "gemm2_tflops": (flops / 3) / (tim["gemm2"][0] * 1e-6) / 1e12 if tim["gemm2"][0] > 0 else None,
                      "fill_GBps": dst["fills"] * S / (fill_us * 1e-6) / 1e9 if fill_us > 0 else None,
@@ -769,6 +775,25 @@ def sub_prefill(args, dev, cal):
             "pairs_on_gemm_frac": w["pairs_gemm"] / max(w["pairs"], 1), "zero_copy_experts_cold": cd["zero_copy"]}
 
 
+def sub_prefill_mxfp4(args, dev, cal):
+    """Sub-record: a 4096-token call on one layer of config 3's shape with MXFP4 experts and 64 slots: the slot-
+    resident experts with >= gemm_min_tokens tokens are expanded to bf16 records and run on the tcgen05 GEMMs."""
+    from paper_2608_16157_b200 import workload as W
+    out, cal, c = prefill_passes(args, dev, 1, cal, shape=W.DSV3_MXFP4, Ns=64)
+    tf_burst, tf_sust, peak_kind = tensor_peaks()
+    w, cd = out["warm"], out["cold"]
+    return {"config": f"prefill, config 3 layer shape (d=7168, 256 mxfp4 experts + 1 shared, I=2048, top-8), "
+                      f"{c['T']} tokens, 1 layer, 64 slots",
+            "cold_ms": cd["ms"], "warm_ms": w["ms"],
+            "useful_tflops_gemms": w["gemm_tflops"], "useful_tflops_with_expansion": w["gemm_with_gather_tflops"],
+            "frac": (w["gemm_with_gather_tflops"] / tf_burst) if w["gemm_with_gather_tflops"] else None,
+            "peak_burst_tflops": tf_burst, "peak_source": peak_kind,
+            "how": "useful (unpadded) flops of the pairs served by the GEMMs / CUDA-event durations of the expansion "
+                   "of the GEMM-list experts to bf16 records + row gather + the two GEMM kernels, warm pass",
+            "pairs_on_gemm_frac": w["pairs_gemm"] / max(w["pairs"], 1), "kernel_ms": w["kernel_ms"],
+            "zero_copy_experts_warm": w["zero_copy"], "hits_warm": w["hits"]}
+
+
 def sub_int4(args, dev, cal, wdtype="int4"):
     """Sub-record of the decode line: config 3 (DeepSeek-V3-shaped 4-bit decode, 4 layers, batch 4, 64 slots), with
     int4-g128 experts or (the format the paper serves) MXFP4 experts."""
@@ -872,7 +897,7 @@ def sub_mxfp4(args, dev, cal):
     return sub_int4(args, dev, cal, "mxfp4")
 
 
-SUBRECORDS = {"int4": sub_int4, "mxfp4": sub_mxfp4, "prefill": sub_prefill}
+SUBRECORDS = {"int4": sub_int4, "mxfp4": sub_mxfp4, "prefill": sub_prefill, "prefill_mxfp4": sub_prefill_mxfp4}
 
 
 def run_sweep(args):
@@ -992,7 +1017,7 @@ def main():
     ap.add_argument("--only-batch", action="store_true")
     ap.add_argument("--cache-warm-steps", type=int, default=64,
                     help="untimed steps from the empty cache before warm-up and timing (steady-state headline)")
-    ap.add_argument("--sub", default="int4,mxfp4,prefill", help="bounded sub-records added to the decode line (N=1 only)")
+    ap.add_argument("--sub", default="int4,mxfp4,prefill,prefill_mxfp4", help="bounded sub-records added to the decode line (N=1 only)")
     ap.add_argument("--overlap", type=int, default=0,
                     help="launch mode of the streaming kernel in the timed region (ft_moe_set_launch_overlap)")
     args = ap.parse_args()
