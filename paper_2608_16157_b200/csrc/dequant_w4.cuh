@@ -35,19 +35,19 @@ __global__ void __launch_bounds__(256) dequant_w4_kernel(DequantParams p) {
   const size_t sec_b = (size_t)NBLK * UA, sec_c = sec_b + (size_t)I * d / 2;
   const size_t S16 = (size_t)3 * I * d * 2;
   const uint32_t chunks_unit = 6u * (uint32_t)d;                // 16-byte chunks of a 96*d-byte destination unit
-  const size_t chunks_rec = (size_t)NBLK * chunks_unit;
-  const int n_items = *p.n_items;
-  const size_t total = (size_t)n_items * chunks_rec;
-  for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
-    const int item = (int)(idx / chunks_rec);
-    const size_t in_rec = idx - (size_t)item * chunks_rec;
-    const uint32_t u = (uint32_t)(in_rec / chunks_unit), k = (uint32_t)(in_rec - (size_t)u * chunks_unit);
-    const uint8_t *rec = p.items[item].w;
-    uint8_t *dst = p.scratch + (size_t)p.items[item].slot * S16 + (size_t)u * 96u * d + (size_t)k * 16u;
+  const uint32_t cbw_shift = 31u - (uint32_t)__clz((int)CBW);   // CBW is 512 or 1024
+  // one block per (16-neuron unit, expert of the GEMM list); the list's length is known on the device only
+  const int item = blockIdx.y;
+  if (item >= *p.n_items) return;
+  const uint32_t u = blockIdx.x;
+  const uint8_t *rec = p.items[item].w;
+  uint8_t *dst_unit = p.scratch + (size_t)p.items[item].slot * S16 + (size_t)u * 96u * d;
+  for (uint32_t k = threadIdx.x; k < chunks_unit; k += blockDim.x) {
+    uint8_t *dst = dst_unit + (size_t)k * 16u;
     float v[8];
     if (k < 4u * (uint32_t)d) {
       // ---- gate (k < 2d) or up part: tile t of 16 neurons x 32 hidden indices, rows of 64 bytes, swizzled ----
-      const uint32_t mm = k / (2u * d), kk = k - mm * 2u * d;
+      const uint32_t mm = k >= 2u * (uint32_t)d ? 1u : 0u, kk = k - mm * 2u * d;
       const uint32_t t = kk >> 6, r = (kk >> 2) & 15u, pos = kk & 3u;
       const uint32_t q = pos ^ ((r & 7u) >> 1);                 // chunk q of the row is stored at position pos
       const uint32_t grp = t >> 2, j = t & 3u;                  // hidden indices 128 grp + 32 j + 8 q + 0..7
@@ -70,7 +70,7 @@ __global__ void __launch_bounds__(256) dequant_w4_kernel(DequantParams p) {
       const uint32_t nhalf = pos ^ (rr >> 2);                   // neurons 8 nhalf .. 8 nhalf + 7 of the unit
       const uint32_t c = 16u * ct + 8u * cg + rr;               // output column
       const uint32_t ng = u >> 3, uu = u & 7u;
-      const uint32_t cb = c / CBW, tt = (c - cb * CBW) >> 4, wq = tt >> 2, j = tt & 3u;
+      const uint32_t cb = c >> cbw_shift, tt = (c - (cb << cbw_shift)) >> 4, wq = tt >> 2, j = tt & 3u;
       const uint8_t *src = rec + sec_b + ((((size_t)(cb * NG + ng) * 8u + uu) * NWD + wq) * 32u + 4u * rr + 2u * nhalf) * 16u + 4u * j;
       const uint32_t w0 = *reinterpret_cast<const uint32_t *>(src), w1 = *reinterpret_cast<const uint32_t *>(src + 16);
       float scale;

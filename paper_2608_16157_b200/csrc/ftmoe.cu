@@ -1124,8 +1124,9 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     dp.d = c.hidden; dp.inter = c.inter;
     {
       TimeScope ts(h, st, FT_TIME_GATHER);
-      if (mx) dequant_w4_kernel<true><<<h->sm_count * 8, 256, 0, st>>>(dp);
-      else dequant_w4_kernel<false><<<h->sm_count * 8, 256, 0, st>>>(dp);
+      const dim3 dg((unsigned)(c.inter / 16), (unsigned)std::min(c.n_experts, c.slots_per_layer));
+      if (mx) dequant_w4_kernel<true><<<dg, 256, 0, st>>>(dp);
+      else dequant_w4_kernel<false><<<dg, 256, 0, st>>>(dp);
     }
     h->launches++;
     return launch_gemm_path(h, layer, L, sc, x_bf, y_dev, st);
