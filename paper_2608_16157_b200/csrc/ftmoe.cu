@@ -13,6 +13,7 @@
 #include "dequant_w4.cuh"
 #include "ffn_mx4.cuh"
 #include "ffn_w4.cuh"
+#include "ffn_w4_half.cuh"
 #include "gemm_tc.cuh"
 #include "gemm_tc2.cuh"
 #include "fill.cuh"
@@ -674,6 +675,14 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
     FT_TRY(cudaFuncSetAttribute(w4_gateup_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
     FT_TRY(cudaFuncSetAttribute(w4_down_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
     FT_TRY(cudaFuncSetAttribute(w4_down_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
+    FT_TRY(cudaFuncSetAttribute(w4_gateup_half_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(w4_gateup_half_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(w4_gateup_half_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(w4_gateup_half_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(w4_gateup_half_kernel<56>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(w4_gateup_half_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_TRY(cudaFuncSetAttribute(w4_down_half_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
+    FT_TRY(cudaFuncSetAttribute(w4_down_half_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
     const int sbm = (int)mx4_down_smem_bytes(2 * kMaxExperts + 1);
     FT_TRY(cudaFuncSetAttribute(mx4_gateup_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
     FT_TRY(cudaFuncSetAttribute(mx4_gateup_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
@@ -1059,8 +1068,11 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   qp.inter = c.inter; qp.top_k = c.top_k; qp.T = L.T;
   const bool own_finalize = !use_gemm && L.T > kFinalizeInKernelMaxTokens;
   qp.finalize = (use_gemm || own_finalize) ? 0 : 1;   // (the GEMM path's combine rounds y)
-  const size_t sa = mx ? mx4_gateup_smem_bytes(qp.max_items, c.hidden) : w4_gateup_smem_bytes(qp.max_items, c.hidden);
-  const size_t sb = mx ? mx4_down_smem_bytes(qp.max_items) : w4_down_smem_bytes(qp.max_items);
+  const bool half = !mx && L.T <= kW4HalfTokens;   // int4 with at most 4 tokens: one MMA per pair of weight words
+  const size_t sa = mx ? mx4_gateup_smem_bytes(qp.max_items, c.hidden)
+                       : half ? w4_gateup_half_smem_bytes(qp.max_items, c.hidden) : w4_gateup_smem_bytes(qp.max_items, c.hidden);
+  const size_t sb = mx ? mx4_down_smem_bytes(qp.max_items)
+                       : half ? w4_down_half_smem_bytes(qp.max_items) : w4_down_smem_bytes(qp.max_items);
   const int grid = h->sm_count;
   {
     TimeScope ts(h, st, FT_TIME_FFN_ZC);   // (timing slot reused for the gate/up kernel of the 4-bit paths)
@@ -1079,6 +1091,15 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
         case 4096: le = cudaLaunchKernelEx(&lc, mx4_gateup_kernel<32>, qp); break;
         case 7168: le = cudaLaunchKernelEx(&lc, mx4_gateup_kernel<56>, qp); break;
         default: le = cudaLaunchKernelEx(&lc, mx4_gateup_kernel<64>, qp); break;
+      }
+    } else if (half) {
+      switch (c.hidden) {
+        case 512: le = cudaLaunchKernelEx(&lc, w4_gateup_half_kernel<4>, qp); break;
+        case 1024: le = cudaLaunchKernelEx(&lc, w4_gateup_half_kernel<8>, qp); break;
+        case 2048: le = cudaLaunchKernelEx(&lc, w4_gateup_half_kernel<16>, qp); break;
+        case 4096: le = cudaLaunchKernelEx(&lc, w4_gateup_half_kernel<32>, qp); break;
+        case 7168: le = cudaLaunchKernelEx(&lc, w4_gateup_half_kernel<56>, qp); break;
+        default: le = cudaLaunchKernelEx(&lc, w4_gateup_half_kernel<64>, qp); break;
       }
     } else {
       switch (c.hidden) {
@@ -1105,6 +1126,9 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     if (mx) {
       if (c.hidden == 512) FT_CUDA(cudaLaunchKernelEx(&lc, mx4_down_kernel<8>, qp, c.hidden));
       else FT_CUDA(cudaLaunchKernelEx(&lc, mx4_down_kernel<16>, qp, c.hidden));
+    } else if (half) {
+      if (c.hidden == 512) FT_CUDA(cudaLaunchKernelEx(&lc, w4_down_half_kernel<8>, qp, c.hidden));
+      else FT_CUDA(cudaLaunchKernelEx(&lc, w4_down_half_kernel<16>, qp, c.hidden));
     } else {
       if (c.hidden == 512) FT_CUDA(cudaLaunchKernelEx(&lc, w4_down_kernel<8>, qp, c.hidden));
       else FT_CUDA(cudaLaunchKernelEx(&lc, w4_down_kernel<16>, qp, c.hidden));
