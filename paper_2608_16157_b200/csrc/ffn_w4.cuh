@@ -40,6 +40,7 @@ constexpr float kW4Levels = 16256.f; // 127 * 128: |fixed-point activation| <= t
 #ifndef W4_BS
 #define W4_BS 2
 #endif
+constexpr int kW4KSplit = 2;             // a unit's hidden dimension is split into this many pieces of work
 constexpr int kW4BlockSteps = W4_BS;     // depth of the gate/up kernel's rolling register buffer, in quantisation groups
 
 struct W4Params {
@@ -51,8 +52,8 @@ struct W4Params {
   const __nv_bfloat16 *x;   // [T][d]
   const int32_t *perm;
   const float *topk_w;
-  float *hraw;              // [pass][16-neuron unit][token 8][neuron 16] fp32
-  int32_t *hcount;          // [pass][128-neuron group]: units of the group written so far (self-resetting)
+  float *hraw;              // [pass][16-neuron unit][gate sums | up sums][token 8][neuron 16] fp32, zero between calls
+  int32_t *hcount;          // [pass][128-neuron group]: pieces of the group added so far (self-resetting)
   uint8_t *hq;              // [pass][group][unit pair 4][token 8][q 4][hi u0, hi u1, lo u0, lo u1 : 4 neurons each]
   float2 *hs;               // [pass][group][token 8]: (m / 16256, 8 (m / 16256) sum of the fixed-point values)
   float *y_acc;             // [T][d]
@@ -150,7 +151,8 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_gateup_kernel(W4Params p) {
   constexpr uint32_t kXStride = 2u * d + 64u;
   constexpr int kBS = kW4BlockSteps;                // steps of a block = depth of the rolling register buffer
   constexpr int kBlocks = G / kBS;                  // blocks of a unit
-  static_assert(G % kBS == 0, "whole blocks");
+  constexpr int kKS = kW4KSplit, kBlocksP = kBlocks / kKS;   // blocks of a piece
+  static_assert(G % kBS == 0 && kBlocks % kKS == 0, "whole blocks, whole pieces");
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char *s_x = smem;
   float *s_sx = reinterpret_cast<float *>(s_x + 8 * kXStride);             // [8][G] m / 16256
@@ -216,14 +218,20 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_gateup_kernel(W4Params p) {
   // lane = (token, quarter): the quarter's two units of 16 neurons.
   auto convert_group = [&](uint32_t grp) {
     const int tok = lane >> 2, qt = lane & 3;
-    const float *src = p.hraw + ((size_t)grp * 8 + 2 * qt) * 128 + tok * 16;
+    float *src = p.hraw + ((size_t)grp * 8 + 2 * qt) * 256 + tok * 16;   // per unit: gate sums [8][16], up sums [8][16]
     float v[2][16];
 #pragma unroll
     for (int u = 0; u < 2; ++u)
 #pragma unroll
       for (int k4 = 0; k4 < 4; ++k4) {
-        const float4 t = __ldcg(reinterpret_cast<const float4 *>(src + u * 128) + k4);
-        v[u][4 * k4] = t.x; v[u][4 * k4 + 1] = t.y; v[u][4 * k4 + 2] = t.z; v[u][4 * k4 + 3] = t.w;
+        float4 *pg = reinterpret_cast<float4 *>(src + u * 256) + k4, *pu_ = reinterpret_cast<float4 *>(src + u * 256 + 128) + k4;
+        const float4 a = __ldcg(pg), b = __ldcg(pu_);
+        __stcg(pg, make_float4(0.f, 0.f, 0.f, 0.f));   // the sums start from zero in the next call
+        __stcg(pu_, make_float4(0.f, 0.f, 0.f, 0.f));
+        v[u][4 * k4] = __fdividef(a.x, 1.f + __expf(-a.x)) * b.x;
+        v[u][4 * k4 + 1] = __fdividef(a.y, 1.f + __expf(-a.y)) * b.y;
+        v[u][4 * k4 + 2] = __fdividef(a.z, 1.f + __expf(-a.z)) * b.z;
+        v[u][4 * k4 + 3] = __fdividef(a.w, 1.f + __expf(-a.w)) * b.w;
       }
     float m = 0.f;
     bool bad = false;
@@ -267,16 +275,17 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_gateup_kernel(W4Params p) {
     if (qt == 0) p.hs[(size_t)grp * 8 + tok] = make_float2(scale, 8.f * (float)sum * scale);
   };
 
-  // One warp streams `n_units` consecutive units starting at `base`; their h goes to rows hrow0.. of the h buffer.
+  // One warp streams `n_pieces` consecutive pieces (a unit's hidden dimension in kKS parts), starting with part ks0
+  // of the unit at `base`; the pieces' partial gate / up sums are added into rows hrow0.. of the h buffer.
   // A step is one quantisation group of the hidden dimension: the gate tile and the up tile of that group, which
   // share their activation fragments.  Registers hold kBS steps; a step's registers are refilled with the step
   // kBS further on as soon as it has been consumed.
-  auto run = [&](const uint8_t *base, int n_units, uint32_t hrow0) {
+  auto run = [&](const uint8_t *base, int ks0, int n_pieces, uint32_t hrow0) {
     uint4 buf[4 * kBS];     // per step: gate rows g, g+8; up rows g, g+8
     uint32_t sc[2 * kBS];   // and their scales
-    const uint8_t *nptr = base + g * 64 + q * 16;              // next block to request (its gate tiles)
-    const uint8_t *nsc = base + 2048u * G + g * 4;
-    int nblk = 0, blocks_left = n_units * kBlocks;             // its index in its unit; blocks not yet requested
+    const uint8_t *nptr = base + ks0 * (G / kKS) * 1024 + g * 64 + q * 16;   // next block to request (its gate tiles)
+    const uint8_t *nsc = base + 2048u * G + ks0 * (G / kKS) * 32 + g * 4;
+    int nblk = ks0 * kBlocksP, blocks_left = n_pieces * kBlocksP;   // its index in its unit; blocks not yet requested
     auto advance = [&]() {
       nptr += kBS * 1024;
       nsc += kBS * 32;
@@ -298,13 +307,15 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_gateup_kernel(W4Params p) {
 #pragma unroll
     for (int si = 0; si < kBS; ++si) request(si, nptr, nsc);
     advance();
-    for (int u = 0; u < n_units; ++u) {
+    int ks = ks0;
+    uint32_t hrow_i = hrow0;
+    for (int piece = 0; piece < n_pieces; ++piece) {
       float tg[4] = {0.f, 0.f, 0.f, 0.f}, tot[4] = {0.f, 0.f, 0.f, 0.f};   // gate sums, up sums
-      for (int blk = 0; blk < kBlocks; ++blk) {
+      for (int blk = 0; blk < kBlocksP; ++blk) {
         const bool more = blocks_left > 0;
         const uint8_t *rp = nptr, *rs = nsc;         // the block that refills this one's registers
         if (more) advance();
-        const int xg = blk * kBS;                    // first group of the block
+        const int xg = ks * (G / kKS) + blk * kBS;   // first group of the block
         const uint32_t xa = my_x + xg * 256u;
 #pragma unroll
         for (int si = 0; si < kBS; ++si) {
@@ -351,25 +362,26 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_gateup_kernel(W4Params p) {
           }
         }
       }
-      // h = SiLU(gate) * up of neurons g, g+8 and tokens 2q, 2q+1
-      const uint32_t hrow_i = hrow0 + u;
-      float *hrow = p.hraw + (size_t)hrow_i * 128;
+      // the piece's gate and up sums of neurons g, g+8 and tokens 2q, 2q+1 join the unit's sums
+      float *hacc = p.hraw + (size_t)hrow_i * 256;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const float a = tg[i];
-        hrow[(2 * q + (i & 1)) * 16 + g + 8 * (i >> 1)] = __fdividef(a, 1.f + __expf(-a)) * tot[i];
+        const int at = (2 * q + (i & 1)) * 16 + g + 8 * (i >> 1);
+        red_add_f32(hacc + at, tg[i]);
+        red_add_f32(hacc + 128 + at, tot[i]);
       }
-      // the 8th unit of a 128-neuron group to arrive converts the group (units of a group are consecutive rows)
+      // the last piece of a 128-neuron group (8 units x kKS pieces) to arrive converts the group
       __threadfence();
       __syncwarp();
       int old = 0;
       if (lane == 0) old = atomicAdd(p.hcount + (hrow_i >> 3), 1);
       old = __shfl_sync(0xffffffffu, old, 0);
-      if (old == 7) {
+      if (old == 8 * kKS - 1) {
         __threadfence();
         convert_group(hrow_i >> 3);
         if (lane == 0) p.hcount[hrow_i >> 3] = 0;
       }
+      if (++ks == kKS) { ks = 0; ++hrow_i; }
     }
   };
 
@@ -380,19 +392,20 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_gateup_kernel(W4Params p) {
   // launched as a programmatic dependent with the caller's word that x and the plan are not produced by the
   // preceding kernel: only from here on (the h buffers, shared with that kernel) must it have completed
   if (p.overlap == 2) asm volatile("griddepcontrol.wait;" ::: "memory");
-  // Units (pass, 16-neuron block) in one flat order, split evenly over all warps of the grid: the slot-resident
-  // range first, then the host-resident range.
+  // Pieces (pass, 16-neuron unit, part of the hidden dimension) in one flat order, split evenly over all warps of
+  // the grid: the slot-resident range first, then the host-resident range.
   const uint32_t n_warps = gridDim.x * kW4Warps, wi = blockIdx.x * kW4Warps + warp;
   for (int range = 0; range < 2; ++range) {
     const uint32_t pass0 = range ? (uint32_t)s_pref[n_items] : 0u;
     const uint32_t pass1 = range ? (uint32_t)s_pref[n_items + n_zc] : (uint32_t)s_pref[n_items];
-    const uint32_t total = (pass1 - pass0) * NBLK, ubase = pass0 * NBLK;
+    const uint32_t PP = NBLK * kKS;                  // pieces of a pass
+    const uint32_t total = (pass1 - pass0) * PP, ubase = pass0 * PP;
     if (total == 0) continue;
     const uint32_t wf = ubase + w4_first(total, n_warps, wi), we = ubase + w4_first(total, n_warps, wi + 1);
     const uint32_t cf = ubase + w4_first(total, n_warps, blockIdx.x * kW4Warps);
     const uint32_t ce = ubase + w4_first(total, n_warps, (blockIdx.x + 1) * kW4Warps);
     if (cf >= ce) continue;
-    for (uint32_t pu = cf / NBLK; pu * NBLK < ce; ++pu) {   // the passes this CTA's warps touch
+    for (uint32_t pu = cf / PP; pu * PP < ce; ++pu) {   // the passes this CTA's warps touch
       const int item = w4_find_item(s_pref, n_items + n_zc, pu);
       const WorkItem &it = s_items[item];
       if (!dense) {   // MMA column j is the pass's j-th pair: stage those tokens' rows
@@ -405,8 +418,11 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_gateup_kernel(W4Params p) {
         });
         __syncthreads();
       }
-      const uint32_t lo = max(wf, pu * NBLK), hi = min(we, (pu + 1) * NBLK);
-      if (lo < hi) run(it.w + (size_t)(lo - pu * NBLK) * kUA, (int)(hi - lo), lo);
+      const uint32_t lo = max(wf, pu * PP), hi = min(we, (pu + 1) * PP);
+      if (lo < hi) {
+        const uint32_t rel = lo - pu * PP;
+        run(it.w + (size_t)(rel / kKS) * kUA, (int)(rel % kKS), (int)(hi - lo), pu * NBLK + rel / kKS);
+      }
     }
   }
 }

@@ -41,7 +41,8 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_gateup_half_kernel(W4Params 
   constexpr uint32_t kXStride = (uint32_t)d + 32u;   // = 32 mod 128: conflict-free 8-byte fragment loads
   constexpr int kBS = kW4HalfBlockSteps;
   constexpr int kBlocks = G / kBS;
-  static_assert(G % kBS == 0, "whole blocks");
+  constexpr int kKS = kW4KSplit, kBlocksP = kBlocks / kKS;   // blocks of a piece
+  static_assert(G % kBS == 0 && kBlocks % kKS == 0, "whole blocks, whole pieces");
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char *s_x = smem;
   float *s_sx = reinterpret_cast<float *>(s_x + 8 * kXStride);             // [4][G] m / 16256
@@ -102,14 +103,22 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_gateup_half_kernel(W4Params 
   auto convert_group = [&](uint32_t grp) {
     const int tok = lane >> 2, qt = lane & 3;
     const bool live = tok < kW4HalfTokens;
-    const float *src = p.hraw + ((size_t)grp * 8 + 2 * qt) * 128 + (live ? tok : 0) * 16;
+    float *src = p.hraw + ((size_t)grp * 8 + 2 * qt) * 256 + (live ? tok : 0) * 16;   // per unit: gate sums | up sums
     float v[2][16];
 #pragma unroll
     for (int u = 0; u < 2; ++u)
 #pragma unroll
       for (int k4 = 0; k4 < 4; ++k4) {
-        const float4 t = __ldcg(reinterpret_cast<const float4 *>(src + u * 128) + k4);
-        v[u][4 * k4] = t.x; v[u][4 * k4 + 1] = t.y; v[u][4 * k4 + 2] = t.z; v[u][4 * k4 + 3] = t.w;
+        float4 *pg = reinterpret_cast<float4 *>(src + u * 256) + k4, *pu_ = reinterpret_cast<float4 *>(src + u * 256 + 128) + k4;
+        const float4 a = __ldcg(pg), b = __ldcg(pu_);
+        if (live) {   // the sums start from zero in the next call
+          __stcg(pg, make_float4(0.f, 0.f, 0.f, 0.f));
+          __stcg(pu_, make_float4(0.f, 0.f, 0.f, 0.f));
+        }
+        v[u][4 * k4] = __fdividef(a.x, 1.f + __expf(-a.x)) * b.x;
+        v[u][4 * k4 + 1] = __fdividef(a.y, 1.f + __expf(-a.y)) * b.y;
+        v[u][4 * k4 + 2] = __fdividef(a.z, 1.f + __expf(-a.z)) * b.z;
+        v[u][4 * k4 + 3] = __fdividef(a.w, 1.f + __expf(-a.w)) * b.w;
       }
     float m = 0.f;
     bool bad = false;
@@ -157,12 +166,12 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_gateup_half_kernel(W4Params 
     if (qt == 0 && live) p.hs[(size_t)grp * 8 + tok] = make_float2(scale, 8.f * (float)sum * scale);
   };
 
-  auto run = [&](const uint8_t *base, int n_units, uint32_t hrow0) {
+  auto run = [&](const uint8_t *base, int ks0, int n_pieces, uint32_t hrow0) {
     uint4 buf[4 * kBS];     // per step: gate rows g, g+8; up rows g, g+8
     uint32_t sc[2 * kBS];
-    const uint8_t *nptr = base + g * 64 + q * 16;
-    const uint8_t *nsc = base + 2048u * G + g * 4;
-    int nblk = 0, blocks_left = n_units * kBlocks;
+    const uint8_t *nptr = base + ks0 * (G / kKS) * 1024 + g * 64 + q * 16;
+    const uint8_t *nsc = base + 2048u * G + ks0 * (G / kKS) * 32 + g * 4;
+    int nblk = ks0 * kBlocksP, blocks_left = n_pieces * kBlocksP;
     auto advance = [&]() {
       nptr += kBS * 1024;
       nsc += kBS * 32;
@@ -184,13 +193,15 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_gateup_half_kernel(W4Params 
 #pragma unroll
     for (int si = 0; si < kBS; ++si) request(si, nptr, nsc);
     advance();
-    for (int u = 0; u < n_units; ++u) {
+    int ks = ks0;
+    uint32_t hrow_i = hrow0;
+    for (int piece = 0; piece < n_pieces; ++piece) {
       float tg[2] = {0.f, 0.f}, tot[2] = {0.f, 0.f};   // gate / up sums of neurons g, g+8 for token q
-      for (int blk = 0; blk < kBlocks; ++blk) {
+      for (int blk = 0; blk < kBlocksP; ++blk) {
         const bool more = blocks_left > 0;
         const uint8_t *rp = nptr, *rs = nsc;
         if (more) advance();
-        const int xg = blk * kBS;
+        const int xg = ks * (G / kKS) + blk * kBS;
         const uint32_t xa = my_x + xg * 128u;
 #pragma unroll
         for (int si = 0; si < kBS; ++si) {
@@ -223,21 +234,23 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_gateup_half_kernel(W4Params 
           tot[1] += bf16hi(uscale) * ((float)(ua[2] * 128 + ua[3]) * sx - xb);
         }
       }
-      // h = SiLU(gate) * up of neurons g, g+8 and token q
-      const uint32_t hrow_i = hrow0 + u;
-      float *hrow = p.hraw + (size_t)hrow_i * 128 + q * 16;
-      hrow[g] = __fdividef(tg[0], 1.f + __expf(-tg[0])) * tot[0];
-      hrow[g + 8] = __fdividef(tg[1], 1.f + __expf(-tg[1])) * tot[1];
+      // the piece's gate and up sums of neurons g, g+8 and token q join the unit's sums
+      float *hacc = p.hraw + (size_t)hrow_i * 256 + q * 16;
+      red_add_f32(hacc + g, tg[0]);
+      red_add_f32(hacc + g + 8, tg[1]);
+      red_add_f32(hacc + 128 + g, tot[0]);
+      red_add_f32(hacc + 128 + g + 8, tot[1]);
       __threadfence();
       __syncwarp();
       int old = 0;
       if (lane == 0) old = atomicAdd(p.hcount + (hrow_i >> 3), 1);
       old = __shfl_sync(0xffffffffu, old, 0);
-      if (old == 7) {
+      if (old == 8 * kKS - 1) {
         __threadfence();
         convert_group(hrow_i >> 3);
         if (lane == 0) p.hcount[hrow_i >> 3] = 0;
       }
+      if (++ks == kKS) { ks = 0; ++hrow_i; }
     }
   };
 
@@ -245,13 +258,17 @@ __global__ void __launch_bounds__(kW4Threads, 1) w4_gateup_half_kernel(W4Params 
   for (int range = 0; range < 2; ++range) {
     const uint32_t pass0 = range ? (uint32_t)s_pref[n_items] : 0u;
     const uint32_t pass1 = range ? (uint32_t)s_pref[n_items + n_zc] : (uint32_t)s_pref[n_items];
-    const uint32_t total = (pass1 - pass0) * NBLK, ubase = pass0 * NBLK;
+    const uint32_t PP = NBLK * kKS;                  // pieces of a pass
+    const uint32_t total = (pass1 - pass0) * PP, ubase = pass0 * PP;
     if (total == 0) continue;
     const uint32_t wf = ubase + w4_first(total, n_warps, wi), we = ubase + w4_first(total, n_warps, wi + 1);
-    for (uint32_t pu = wf / NBLK; pu * NBLK < we; ++pu) {   // the passes (= experts) this warp touches
+    for (uint32_t pu = wf / PP; pu * PP < we; ++pu) {   // the passes (= experts) this warp touches
       const WorkItem &it = s_items[w4_find_item(s_pref, n_items + n_zc, pu)];
-      const uint32_t lo = max(wf, pu * NBLK), hi = min(we, (pu + 1) * NBLK);
-      if (lo < hi) run(it.w + (size_t)(lo - pu * NBLK) * kUA, (int)(hi - lo), lo);
+      const uint32_t lo = max(wf, pu * PP), hi = min(we, (pu + 1) * PP);
+      if (lo < hi) {
+        const uint32_t rel = lo - pu * PP;
+        run(it.w + (size_t)(rel / kKS) * kUA, (int)(rel % kKS), (int)(hi - lo), pu * NBLK + rel / kKS);
+      }
     }
   }
 }

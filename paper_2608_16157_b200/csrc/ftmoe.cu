@@ -658,7 +658,8 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
   FT_TRY(cudaFuncSetAttribute(fill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFillStages * (int)kFillChunk));
   if (c.wdtype == FT_W_INT4_G128 || c.wdtype == FT_W_MXFP4) {
     const size_t passes = (P + 7) / 8 + 2 * E + 2;
-    FT_TRY(cudaMalloc(&h->w4_hraw, passes * (c.inter / 16) * 512));
+    FT_TRY(cudaMalloc(&h->w4_hraw, passes * (c.inter / 16) * 1024));
+    FT_TRY(cudaMemset(h->w4_hraw, 0, passes * (c.inter / 16) * 1024));
     FT_TRY(cudaMalloc(&h->w4_hcount, passes * (c.inter / 128) * 4));
     FT_TRY(cudaMemset(h->w4_hcount, 0, passes * (c.inter / 128) * 4));
     FT_TRY(cudaMalloc(&h->w4_hq, passes * (c.inter / 128) * 2048));
