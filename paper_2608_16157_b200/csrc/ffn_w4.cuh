@@ -10,13 +10,15 @@
 //     error is at most m / 32512 per element, i.e. below the rounding of the largest element to bf16 (m / 512);
 //   * per group and output:  scale_w * ( (m / 16256) * (128 S_hi + S_lo) - 8 (m / 16256) sum(128 hi + lo) )  in fp32
 //     (the second term removes the + 8 of the codes).
-//   w4_gateup_kernel : 16 warps per SM, every warp streams whole 16-neuron units (gate tiles, up tiles and their
-//                      scales: contiguous) by itself: no partial sums to exchange, no block-level synchronisation
-//                      while a call has at most 8 tokens.  A lane's two 16-byte loads per quantisation group are rows
-//                      g and g+8 of the group's tile; a rolling register buffer is refilled as soon as a pair has
-//                      been consumed.  h = SiLU(g) * u goes to global memory as fp32; the warp that completes a
-//                      group of 128 neurons of a pass (an arrival counter per group; nobody waits) converts that
-//                      group to the fixed-point form above for the down kernel.
+//   w4_gateup_kernel : 16 warps per SM; the work is cut into pieces = (16-neuron unit, half of the hidden dimension)
+//                      and every warp streams its share of consecutive pieces by itself (gate tiles, up tiles and
+//                      their scales of a unit are contiguous): no block-level synchronisation while a call has at
+//                      most 8 tokens, and an even share per warp at every batch size.  A lane's two 16-byte loads
+//                      per quantisation group are rows g and g+8 of the group's tile; a rolling register buffer is
+//                      refilled as soon as a step has been consumed.  A piece's partial gate and up sums are added
+//                      (red.global.add) into the unit's fp32 accumulators; the warp that completes a group of 128
+//                      neurons of a pass (an arrival counter per group; nobody waits) applies SiLU(g) * u, converts
+//                      the group to the fixed-point form above for the down kernel and clears the accumulators.
 //   w4_down_kernel   : walks chunks (expert pass, block of 64*NWD output columns, group of 128 neurons) = 8 steps
 //                      of 16 neurons x 512 bytes per warp.  Every warp owns four 16-column tiles: its 16-byte load
 //                      per step is their A fragments.  No block-level synchronisation: a warp stages the chunk's h
