@@ -1,6 +1,6 @@
 // Steps 5+6 for MXFP4 experts (e2m1 codes, one power-of-two scale byte per 32 elements of the contraction
 // dimension) at decode-sized token counts.  Same structure, work distribution and buffers as the int4 kernels of
-// ffn_w4.cuh (every warp of the gate/up kernel streams whole 16-neuron units; the down kernel walks chunks of 128
+// ffn_w4.cuh (every warp of the gate/up kernel streams its share of half-unit pieces; the down kernel walks chunks of 128
 // neurons x 1024 columns; weights go from global memory straight into registers); what differs is the arithmetic:
 //   * an e2m1 code is a 4-bit float, and placing its bits (s, e1 e0, m) at bits (7, 4 3, 2) of a byte gives the fp8
 //     e4m3 number code * 2^-6 exactly, subnormals included.  ((w << 4) & 0x80808080) | ((w << 2) & 0x1C1C1C1C) does
