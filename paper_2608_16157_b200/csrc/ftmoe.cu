@@ -1317,7 +1317,16 @@ ft_status_t ft_moe_resize(ft_moe_t *h, int slots_per_layer) {
     (void)alloc_cache(h);
     return rc;
   }
-  if (h->gemm) {   // the weight tensor maps of the prefill path are bound to the slot pool
+  if (h->gemm) {   // the weight tensor maps of the prefill path are bound to the slot pool (bf16) or to the
+                   // scratch pool of one layer's slots (4-bit), which follows the new slot count
+    if (h->cfg.wdtype != FT_W_BF16) {
+      cudaFree(h->wq_scratch);
+      h->wq_scratch = nullptr;
+      if (slots_per_layer > 0) {
+        const cudaError_t e = cudaMalloc(&h->wq_scratch, (size_t)slots_per_layer * 3 * h->cfg.inter * h->cfg.hidden * 2);
+        if (e != cudaSuccess) { (void)cudaGetLastError(); return FT_ERR_OOM; }
+      }
+    }
     rc = build_weight_maps(h);
     if (rc != FT_OK) return rc;
   }

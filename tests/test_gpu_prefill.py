@@ -57,6 +57,29 @@ def test_prefill_then_decode_on_the_same_handle(wdtype):
     pr.close()
 
 
+@pytest.mark.parametrize("wdtype", ["int4", "mxfp4"])
+def test_prefill_4bit_after_resize(wdtype):
+    """The bf16 scratch pool the GEMMs read 4-bit experts from holds one record per slot of a layer, so a resize to
+    more slots must grow it (and rebind the weight tensor maps): 3 slots -> 8 slots -> 2 slots."""
+    from oracle import ftmoe_oracle as O
+    shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2, wdtype=wdtype)
+    pr = Pair(shape, n_slots=3, max_tokens=512, seed=37, gemm_min_tokens=32)
+    step = 0
+    for new_slots in (None, 8, 2):
+        if new_slots is not None:
+            pr.moe.resize(new_slots)
+            ora = pr.oracles[0]
+            step_now = ora.state.step
+            ora.state = O.CacheState(8, new_slots)
+            ora.state.step = step_now
+            ora.slots = [None] * new_slots
+        for _ in range(2):
+            pr.step(0, _zipf_logits(400, 8, 37, step), W.noise_x(400, 512, 37, step, 0), check_slots=True)
+            step += 1
+    assert pr.moe.get_stats(0)["pairs_gemm"] > 0
+    pr.close()
+
+
 def test_prefill_qwen3_shape_one_layer():
     """d=2048, 128 experts, I=768, top-8, 64 slots, 1024 tokens, cold then warm."""
     shape = W.QWEN3_30B
