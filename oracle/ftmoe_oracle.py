@@ -266,6 +266,18 @@ def unpack_record(rec: np.ndarray, d: int, inter: int, wdtype: str):
                                              up: the same + 64*G
       down scale of (block n//32, column c): UA*I/16 + I*d/2 + ((ng*CB + cb)*NWD + w)*256 + 32*g + 8*j + 4*half
                                              + (n%128)//32
+    nvfp4 record: the same 4-bit codes; one scale byte b per 16 consecutive elements of the contraction dimension,
+    read as an unsigned e4m3 number (E = b >> 3, M = b & 7: 2**(E-7) * (1 + M/8) for E >= 1, 2**-6 * M/8 for E = 0;
+    b <= 0x7E), and one float32 scale per matrix: weight = (+-magnitude) * block scale * matrix scale.  UA = 2304*G.
+      gate code of (neuron n, hidden i): with o = i%32: UA*(n//16) + 1024*(i//128) + 64*(n%16) + 16*((o%16)//4)
+                                         + 4*((i%128)//32) + (o%4),  lo = o < 16;      up: the same + 1024*G
+      gate scale of (n, block i//16):    UA*(n//16) + 2048*G + 128*(i//128) + 16*(n%8) + 8*((n%16)//8) + (i%128)//16
+                                         up: the same + 128*G
+      down code of (neuron n, column c): as in the int4 record
+      down scale of (block n//16, column c): UA*I/16 + I*d/2 + ((ng*CB + cb)*NWD + w)*512 + 64*g + 16*j + 8*half
+                                             + (n%128)//16
+      matrix scales (gate, up, down): three little-endian float32 at UA*I/16 + I*d/2 + I*d/16, then zeros up to
+                                      256 bytes.
     """
     rec = np.ascontiguousarray(rec).view(np.uint8).reshape(-1)
     n = inter * d
@@ -349,6 +361,47 @@ def unpack_record(rec: np.ndarray, d: int, inter: int, wdtype: str):
         a_down = UA * U + ((((cb * NG + ng) * 8 + uu) * nwd + w) * 32 + 4 * g + q) * 16 + 4 * j + e // 2
         s_down = UA * U + inter * d // 2 + ((ng * CB + cb) * nwd + w) * 256 + 32 * g + 8 * j + 4 * half + (n % 128) // 32
         wd = fp4(a_down, e % 2 == 0) * pow2(s_down)
+        return wg, wu, wd
+    if wdtype == "nvfp4":
+        G, NG, U = d // GROUP, inter // GROUP, inter // 16
+        UA = 2304 * G
+        nwd = min(16, d // 64)
+        cbw = 64 * nwd
+        CB = d // cbw
+        sec_c = U * UA + inter * d // 2
+        tail = sec_c + inter * d // 16
+        assert rec.size == tail + 256
+        magnitude = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
+
+        def fp4(addr, lo):
+            b = rec[addr].astype(np.int64)
+            c = np.where(lo, b & 0xF, b >> 4)
+            return np.where(c & 8, -1.0, 1.0) * magnitude[c & 7]
+
+        def ue4m3(addr):
+            b = rec[addr].astype(np.int64)
+            assert np.all(b <= 0x7E)
+            ex, man = b >> 3, (b & 7).astype(np.float64)
+            return np.where(ex >= 1, np.exp2(ex.astype(np.float64) - 7.0) * (1.0 + man / 8.0), 2.0 ** -6 * man / 8.0)
+
+        sg, su, sd = (float(v) for v in rec[tail:tail + 12].view("<f4").astype(np.float64))
+        i = np.arange(d, dtype=np.int64)[:, None]
+        nn = np.arange(inter, dtype=np.int64)[None, :]
+        o = i % 32
+        a_gate = UA * (nn // 16) + 1024 * (i // 128) + 64 * (nn % 16) + 16 * ((o % 16) // 4) + 4 * ((i % 128) // 32) + o % 4
+        s_gate = UA * (nn // 16) + 2048 * G + 128 * (i // 128) + 16 * (nn % 8) + 8 * ((nn % 16) // 8) + (i % 128) // 16
+        lo = (o < 16) & (nn >= 0)
+        wg = fp4(a_gate, lo) * ue4m3(s_gate) * sg
+        wu = fp4(a_gate + 1024 * G, lo) * ue4m3(s_gate + 128 * G) * su
+        n = np.arange(inter, dtype=np.int64)[:, None]
+        c = np.arange(d, dtype=np.int64)[None, :]
+        ng, uu, q, r = n // 128, (n % 128) // 16, (n % 16) // 4, n % 4
+        g, half, cb, t = c % 8, (c % 16) // 8, c // cbw, (c % cbw) // 16
+        w, j = t // 4, t % 4
+        e = half + 2 * r
+        a_down = UA * U + ((((cb * NG + ng) * 8 + uu) * nwd + w) * 32 + 4 * g + q) * 16 + 4 * j + e // 2
+        s_down = sec_c + ((ng * CB + cb) * nwd + w) * 512 + 64 * g + 16 * j + 8 * half + (n % 128) // 16
+        wd = fp4(a_down, e % 2 == 0) * ue4m3(s_down) * sd
         return wg, wu, wd
     raise ValueError(wdtype)
 

@@ -42,6 +42,16 @@ flattened identifier of Sec. 4.2 of the paper):
           C. order (ng, cb, w, g, j, half, m): per lane ``g`` 32 bytes = for each tile ``j`` and column half the four
              32-neuron blocks ``m`` of the 128-neuron group.
           ``S = 3*I*d/2 + 3*I*d/32``.
+``nvfp4`` the same e2m1 codes with one unsigned e4m3 scale byte per block of 16 consecutive elements along the
+          contraction dimension and one float32 scale per matrix.  Differences from ``mxfp4``:
+          A. ``2304*G`` bytes per unit; in a gate/up tile row the code of hidden index ``128*grp + 32*j + 16*(e & 1)
+             + 4*q + e // 2`` is nibble ``e`` of word ``j`` of chunk ``q`` (so that the even nibbles of a word row
+             are one scale block and the odd nibbles the next); per tile 128 scale bytes: for ``r`` in 0..7 the
+             eight block scales of row ``r``, then those of row ``r+8``.
+          C. order (ng, cb, w, g, j, half, unit): per lane ``g`` 64 bytes = for each tile ``j`` and column half the
+             eight 16-neuron blocks of the 128-neuron group.
+          Then the three matrix scales (gate, up, down) as float32, zero-padded to 256 bytes.
+          ``S = 3*I*d/2 + 3*I*d/16 + 256``.
 
 The routing-logit recipes follow the workload descriptions: a Zipf-style
 popularity bias ``b_e = -alpha * ln(rank_e)`` with ``rank`` a seeded permutation
@@ -58,6 +68,8 @@ import torch
 
 GROUP = 128  # int4 quantisation group length along the contraction dimension
 MX_BLOCK = 32  # elements that share one scale byte in the mxfp4 records
+NV_BLOCK = 16  # elements that share one e4m3 scale byte in the nvfp4 records
+NV_TAIL = 256  # bytes of the record's tail holding the three float32 matrix scales
 
 
 @dataclasses.dataclass(frozen=True)
@@ -66,7 +78,7 @@ class LayerShape:
     inter: int        # expert intermediate size I
     n_experts: int    # routed experts E
     top_k: int
-    wdtype: str = "bf16"   # "bf16" | "int4" | "mxfp4"
+    wdtype: str = "bf16"   # "bf16" | "int4" | "mxfp4" | "nvfp4"
     n_shared: int = 0      # always-resident shared experts (0 or 1)
 
     @property
@@ -79,6 +91,8 @@ class LayerShape:
             return payload + scales
         if self.wdtype == "mxfp4":
             return 3 * self.inter * self.d // 2 + 3 * self.inter * self.d // MX_BLOCK
+        if self.wdtype == "nvfp4":
+            return 3 * self.inter * self.d // 2 + 3 * self.inter * self.d // NV_BLOCK + NV_TAIL
         raise ValueError(self.wdtype)
 
 
@@ -87,6 +101,7 @@ TINY = LayerShape(d=256, inter=128, n_experts=8, top_k=2)
 QWEN3_30B = LayerShape(d=2048, inter=768, n_experts=128, top_k=8)
 DSV3_INT4 = LayerShape(d=7168, inter=2048, n_experts=256, top_k=8, wdtype="int4", n_shared=1)
 DSV3_MXFP4 = LayerShape(d=7168, inter=2048, n_experts=256, top_k=8, wdtype="mxfp4", n_shared=1)
+DSV3_NVFP4 = LayerShape(d=7168, inter=2048, n_experts=256, top_k=8, wdtype="nvfp4", n_shared=1)
 
 
 def mix64(*vals: int) -> int:
@@ -203,6 +218,64 @@ def _pack_mxfp4_record(cg, cu, cd, bg, bu, bd) -> torch.Tensor:
     return torch.cat([sec_a, sec_b, sec_c])
 
 
+def _e2m1_codes(v: torch.Tensor) -> torch.Tensor:
+    """Scaled values -> e2m1 codes (uint8 0..15): nearest magnitude, ties to the even code, saturating at 6."""
+    a = v.abs().clamp(max=6.0)
+    bounds = torch.tensor([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0], device=v.device, dtype=torch.float32)
+    lo_ = torch.bucketize(a, bounds, right=False)
+    hi_ = torch.bucketize(a, bounds, right=True)
+    idx = torch.where(lo_ != hi_, torch.where(lo_ % 2 == 0, lo_, hi_), lo_)
+    return (idx | torch.where(v < 0, 8, 0)).to(torch.uint8)
+
+
+def _quantise_nvfp4(w: torch.Tensor, block_axis: int) -> tuple[torch.Tensor, torch.Tensor, float]:
+    """Two-level FP4 quantiser used to *produce* the synthetic pool: blocks of 16 along ``block_axis``.
+
+    Matrix scale = amax / (6 * 448) (the largest block scale is the largest e4m3 number); block scale = block amax /
+    (6 * matrix scale) rounded to e4m3; elements rounded to the nearest e2m1 value of w / (block scale * matrix
+    scale).  Returns (codes uint8 with w's shape, scale bytes uint8 with the block axis reduced by 16, matrix scale).
+    """
+    I, d = w.shape
+    wb = w.reshape(I, d // NV_BLOCK, NV_BLOCK) if block_axis == 1 else w.reshape(I // NV_BLOCK, NV_BLOCK, d)
+    ax = 2 if block_axis == 1 else 1
+    top = w.abs().max().to(torch.float32)
+    ms = torch.where(top > 0, top / (6.0 * 448.0), torch.ones_like(top))
+    amax = wb.abs().amax(dim=ax, keepdim=True)
+    s8 = (amax / (6.0 * ms)).clamp(max=448.0).to(torch.float8_e4m3fn)
+    sb = s8.to(torch.float32)
+    v = torch.where(sb > 0, wb / (torch.where(sb > 0, sb, torch.ones_like(sb)) * ms), torch.zeros_like(wb))
+    return _e2m1_codes(v).reshape(I, d), s8.view(torch.uint8).squeeze(ax), float(ms)
+
+
+def _pack_nvfp4_record(cg, cu, cd, bg, bu, bd, scales) -> torch.Tensor:
+    """Codes uint8 ``[I][d]`` (gate/up: one row per neuron; down: ``[n][c]``), scale bytes ``bg, bu [I][d/16]``,
+    ``bd [I/16][d]``, the three matrix scales -> the tiled record, uint8 flat."""
+    I, d = cg.shape
+    dev = cg.device
+    U, G, NG = I // 16, d // GROUP, I // GROUP
+    nwd = min(16, d // 64)
+    cbw = 64 * nwd
+    CB = d // cbw
+
+    def gu_tiles(c):      # [U][16 rows][G][j][half][q][r] -> [U][G][row][q][j][r][half], nibble e = 2 r + half
+        t = c.reshape(U, 16, G, 4, 2, 4, 4).permute(0, 2, 1, 5, 3, 6, 4)
+        return (t[..., 0] | (t[..., 1] << 4)).reshape(U, G * 1024)
+
+    def gu_scales(b_):    # [U][half][r][G][k] -> [U][G][r][half][k]
+        return b_.reshape(U, 2, 8, G, 8).permute(0, 3, 2, 1, 4).reshape(U, G * 128)
+
+    sec_a = torch.cat([gu_tiles(cg), gu_tiles(cu), gu_scales(bg), gu_scales(bu)], dim=1).reshape(-1)
+    ar = lambda n: torch.arange(n, device=dev)
+    cb, ng, uu, w, g, q, j, e = torch.meshgrid(ar(CB), ar(NG), ar(8), ar(nwd), ar(8), ar(4), ar(4), ar(8), indexing="ij")
+    t = cd[128 * ng + 16 * uu + 4 * q + e // 2, cb * cbw + (4 * w + j) * 16 + g + 8 * (e & 1)]
+    sec_b = (t[..., 0::2] | (t[..., 1::2] << 4)).reshape(-1)
+    ng2, cb2, w2, g2, j2, half, m = torch.meshgrid(ar(NG), ar(CB), ar(nwd), ar(8), ar(4), ar(2), ar(8), indexing="ij")
+    sec_c = bd[8 * ng2 + m, cb2 * cbw + (4 * w2 + j2) * 16 + g2 + 8 * half].reshape(-1)
+    tail = torch.zeros(NV_TAIL, dtype=torch.uint8, device=dev)
+    tail[:12] = torch.tensor(scales, dtype=torch.float32).view(torch.uint8).to(dev)
+    return torch.cat([sec_a, sec_b, sec_c, tail])
+
+
 WD_NU = (0, 0, 1, 1, 2, 2, 3, 3)     # neuron offset (plus 4q) of nibble e in a word of the down section
 
 
@@ -274,6 +347,11 @@ def make_records(shape: LayerShape, seed: int, layer: int, first: int, count: in
             cu, bu = _quantise_mxfp4(w[1], 1)
             cd, bd = _quantise_mxfp4(w[2], 0)
             out[j] = _pack_mxfp4_record(cg, cu, cd, bg, bu, bd)
+        elif shape.wdtype == "nvfp4":
+            cg, bg, mg = _quantise_nvfp4(w[0], 1)
+            cu, bu, mu = _quantise_nvfp4(w[1], 1)
+            cd, bd, md = _quantise_nvfp4(w[2], 0)
+            out[j] = _pack_nvfp4_record(cg, cu, cd, bg, bu, bd, (mg, mu, md))
         else:
             qg, sg = _quantise_int4(w[0:1], 2)
             qu, su = _quantise_int4(w[1:2], 2)

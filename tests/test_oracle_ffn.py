@@ -196,6 +196,119 @@ def test_unpack_mxfp4_record_by_definition(d, I):
     assert np.array_equal(wd1, -np.ones((I, d)))
 
 
+def _record_nvfp4_by_definition(cg, cu, cd, bg, bu, bd, scales):
+    """cX: codes 0..15 [I][d] (row = neuron); bg/bu [I][d/16], bd [I/16][d] e4m3 scale bytes; scales: three floats.
+    Written section by section from the documented tile order."""
+    I, d = cg.shape
+    G, NG, U = d // 128, I // 128, I // 16
+    nwd = min(16, d // 64)
+    cbw, CB = 64 * nwd, d // (64 * nwd)
+    out = bytearray()
+
+    def word(nibbles):
+        v = 0
+        for e, c in enumerate(nibbles):
+            v |= (int(c) & 0xF) << (4 * e)
+        return v.to_bytes(4, "little")
+
+    for u in range(U):
+        for c_ in (cg, cu):
+            for grp in range(G):
+                for row in range(16):
+                    for chunk in range(4):
+                        for j in range(4):
+                            i0 = 128 * grp + 32 * j + 4 * chunk      # nibble e: hidden i0 + 16 (e & 1) + e // 2
+                            out += word([c_[16 * u + row, i0 + 16 * (e & 1) + e // 2] for e in range(8)])
+        for b_ in (bg, bu):
+            for grp in range(G):
+                for r in range(8):
+                    out += bytes(int(b_[16 * u + r, 8 * grp + k]) for k in range(8))
+                    out += bytes(int(b_[16 * u + r + 8, 8 * grp + k]) for k in range(8))
+    for cb in range(CB):
+        for ng in range(NG):
+            for uu in range(8):
+                for w in range(nwd):
+                    for lane in range(32):
+                        g, q = divmod(lane, 4)
+                        for j in range(4):
+                            col0 = cb * cbw + (4 * w + j) * 16
+                            out += word([cd[128 * ng + 16 * uu + 4 * q + e // 2, col0 + g + 8 * (e & 1)] for e in range(8)])
+    for ng in range(NG):
+        for cb in range(CB):
+            for w in range(nwd):
+                for g in range(8):
+                    for j in range(4):
+                        for half in range(2):
+                            col = cb * cbw + (4 * w + j) * 16 + g + 8 * half
+                            out += bytes(int(bd[8 * ng + m, col]) for m in range(8))
+    out += np.asarray(scales, dtype="<f4").tobytes()
+    out += bytes(256 - 12)
+    return np.frombuffer(bytes(out), dtype=np.uint8)
+
+
+def test_nvfp4_block_scale_bytes_are_e4m3_numbers():
+    """The reader's scale decoding against the library's float8 (e4m3) type, for every allowed byte: a record whose
+    codes are all 1.0 (code 2) and whose gate scale bytes run through 0..0x7E."""
+    d, I = 2048, 128                      # 128 blocks of 16 per gate row
+    two = np.full((I, d), 2)
+    bg = np.tile(np.arange(128) % 0x7F, (I, 1))
+    bg[1] = 0x7E - np.arange(128) % 0x7F
+    bu = np.full((I, d // 16), 0x38)      # 1.0
+    bd = np.full((I // 16, d), 0x38)
+    rec = _record_nvfp4_by_definition(two, two, two, bg, bu, bd, (1.0, 1.0, 1.0))
+    wg, wu, wd = O.unpack_record(rec, d, I, "nvfp4")
+    lib = torch.arange(0, 0x7F, dtype=torch.uint8).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    assert lib[0x38] == 1.0 and lib[0x7E] == 448.0 and lib[0x01] == 2.0 ** -9    # the format's landmarks
+    assert np.array_equal(wg[:, 0], np.repeat(lib[bg[0]], 16))
+    assert np.array_equal(wg[:, 1], np.repeat(lib[bg[1]], 16))
+    assert np.array_equal(wu, np.ones((d, I))) and np.array_equal(wd, np.ones((I, d)))
+
+
+@pytest.mark.parametrize("d,I", [(256, 128), (1024, 256)])
+def test_unpack_nvfp4_record_by_definition(d, I):
+    rng = np.random.default_rng(4)
+    cg, cu, cd = (rng.integers(0, 16, size=(I, d)) for _ in range(3))
+    bg = rng.integers(0, 0x7F, size=(I, d // 16))
+    bu = rng.integers(0x20, 0x50, size=(I, d // 16))
+    bd = rng.integers(0, 0x7F, size=(I // 16, d))
+    scales = (0.75, 3.0e-3, 17.0)
+    rec = _record_nvfp4_by_definition(cg, cu, cd, bg, bu, bd, scales)
+    assert rec.size == W.LayerShape(d, I, 1, 1, "nvfp4").expert_bytes
+    wg, wu, wd = O.unpack_record(rec, d, I, "nvfp4")
+    val = np.array(FP4_VALUES)
+    lib = torch.arange(0, 0x7F, dtype=torch.uint8).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+
+    def deq(c, b, axis, s):
+        return np.where(c & 8, -1.0, 1.0) * val[c & 7] * np.repeat(lib[b], 16, axis=axis) * float(np.float32(s))
+
+    assert np.array_equal(wg, deq(cg, bg, 1, scales[0]).T)
+    assert np.array_equal(wu, deq(cu, bu, 1, scales[1]).T)
+    assert np.array_equal(wd, deq(cd, bd, 0, scales[2]))
+
+
+def test_generated_nvfp4_pool_quantiser_error_bound():
+    """The generator's records, read back by the oracle, against the fp32 draws.  The matrix scale maps the largest
+    magnitude to 6 * 448; a block's scale byte is its amax / (6 * matrix scale) rounded to e4m3 (relative error
+    <= 2**-4), so the grid step at the top of a block is at most 2 * (1 + 2**-4) * amax / 6 and every element lies
+    within half of that of its draw (elements above 6 * scale after a downward rounding of the scale saturate at
+    6 * scale >= amax * (1 - 2**-4))."""
+    shape = W.LayerShape(d=256, inter=128, n_experts=2, top_k=1, wdtype="nvfp4")
+    rec = W.make_records(shape, seed=0, layer=0, first=0, count=1)[0].numpy()
+    wg, wu, wd = O.unpack_record(rec, 256, 128, "nvfp4")
+    g = torch.Generator().manual_seed(W.mix64(0, 1, 0, 0))
+    w = (torch.randn((3, 128, 256), generator=g) * 0.02).double().numpy()
+    for got, ref, axis in ((wg.T, w[0], 1), (wu.T, w[1], 1), (wd, w[2], 0)):
+        blocks = np.abs(ref).reshape((128, 16, 16) if axis == 1 else (8, 16, 256))
+        amax = np.repeat(blocks.max(axis=2 if axis == 1 else 1), 16, axis=axis)
+        assert np.all(np.abs(got - ref) <= amax * (1 + 2.0 ** -4) / 6 + 1e-15)
+        assert np.all(np.abs(got) <= amax * (1 + 2.0 ** -4) + 1e-15)
+    assert np.count_nonzero(wg) > wg.size // 2
+    # finer blocks and finer scales than mxfp4: the error is smaller on the same draws
+    shape_mx = W.LayerShape(d=256, inter=128, n_experts=2, top_k=1, wdtype="mxfp4")
+    wg_mx = O.unpack_record(W.make_records(shape_mx, seed=0, layer=0, first=0, count=1)[0].numpy(), 256, 128, "mxfp4")[0]
+    assert np.abs(wg.T - w[0]).mean() < np.abs(wg_mx.T - w[0]).mean()
+
+
 def test_generated_mxfp4_pool_quantiser_error_bound():
     """The generator's records, read back by the oracle, are within half a grid step of the fp32 draws: the e2m1 grid
     step is at most 2 (between 4 and 6) times the block scale 2**(floor(log2(amax)) - 2), i.e. |w - deq| <= amax / 4."""
