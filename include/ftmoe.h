@@ -69,11 +69,24 @@
  *                   r+8.  Section C: order (ng, cb, w, g, j, half, m), i.e. per lane g 32 bytes = for each tile j and
  *                   column half the scales of the four 32-neuron blocks m of the 128-neuron group.
  *                   S = 3*inter*hidden/2 + 3*inter*hidden/32 bytes.  Shapes as for int4.
- *   Shape limits: bf16: hidden in {256, 512, 1024, 2048}, inter % 16 == 0; int4 and mxfp4: hidden in
+ *   FT_W_NVFP4    : two-level scaled FP4 (paper Sec. 5.1, expert representations): the same e2m1 codes with one
+ *                   unsigned e4m3 scale byte b (exponent field E = b >> 3, mantissa M = b & 7: 2^(E-7) * (1 + M/8),
+ *                   or 2^-6 * M/8 when E = 0; b <= 0x7E) per 16 consecutive elements of the contraction dimension and
+ *                   one float32 scale per matrix: weight = (+-magnitude) * block scale * matrix scale.  Differences
+ *                   from FT_W_MXFP4: in a gate/up tile row, nibble e of word j of chunk q is the code of hidden index
+ *                   128*grp + 32*j + 16*(e & 1) + 4*q + e/2, so that the even nibbles of the row's words j are one
+ *                   scale block and the odd nibbles the next (K = 16 tensor-core steps); a unit of section A is
+ *                   2304*G bytes with 128 scale bytes per tile = for r in 0..7 the eight block scales of row r, then
+ *                   those of row r+8.  Section B is unchanged (a 16-neuron unit is one scale block).  Section C:
+ *                   order (ng, cb, w, g, j, half, unit), per lane g 64 bytes = for each tile j and column half the
+ *                   scales of the eight 16-neuron blocks of the 128-neuron group.  Then the matrix scales of gate,
+ *                   up and down as three little-endian float32, zero-padded to 256 bytes.
+ *                   S = 3*inter*hidden/2 + 3*inter*hidden/16 + 256 bytes.  Shapes as for int4.
+ *   Shape limits: bf16: hidden in {256, 512, 1024, 2048}, inter % 16 == 0; int4, mxfp4 and nvfp4: hidden in
  *   {512, 1024, 2048, 4096, 7168, 8192}, inter % 128 == 0; n_experts <= 1024;
  *   top_k <= min(n_experts, 32); slots per table (slots_per_layer, or n_layers*slots_per_layer with global_pool)
  *   <= 6144.  The tensor-core prefill path (gemm_min_tokens > 0) needs slots_per_layer > 0, hidden % 256 == 0 and
- *   inter % 256 == 0; int4 and mxfp4 experts on that path are first expanded, once per call, to bf16 records in a
+ *   inter % 256 == 0; 4-bit experts on that path are first expanded, once per call, to bf16 records in a
  *   scratch pool of slots_per_layer x 3*inter*hidden*2 bytes owned by the handle (not with global_pool).
  */
 #ifndef FTMOE_H_
@@ -100,7 +113,7 @@ typedef enum {
   FT_ERR_UNSUPPORTED = 8
 } ft_status_t;
 
-typedef enum { FT_W_BF16 = 0, FT_W_INT4_G128 = 1, FT_W_MXFP4 = 2 } ft_wdtype_t;
+typedef enum { FT_W_BF16 = 0, FT_W_INT4_G128 = 1, FT_W_MXFP4 = 2, FT_W_NVFP4 = 3 } ft_wdtype_t;
 
 /* How ft_moe_fill moves records.  Both give byte-identical slots. */
 typedef enum {

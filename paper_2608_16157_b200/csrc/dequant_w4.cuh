@@ -2,7 +2,8 @@
 // call, from their slot into a bf16 record in tile order (the layout the GEMMs' tensor maps read, see
 // include/ftmoe.h) in a per-layer scratch pool.  With hundreds of tokens per expert the expansion (one pass over
 // the record) is small beside the GEMMs, and the GEMMs then run on exact bf16 activations: int4 weights are rounded
-// to bf16 after the multiplication by their scale (11-12 significant bits -> 8), MXFP4 weights are exact in bf16.
+// to bf16 after the multiplication by their scale (11-12 significant bits -> 8), MXFP4 weights are exact in bf16,
+// NVFP4 weights are rounded after the multiplication by the block scale and the matrix scale.
 // One thread produces one 16-byte chunk of the destination (8 weights), in destination order, so that the writes
 // are coalesced; the 4-byte source words come from L2.
 #pragma once
@@ -26,12 +27,16 @@ __device__ __forceinline__ float w4_code_value(uint32_t nib, bool mx) {
   return (nib & 8u) ? -mag : mag;
 }
 
-template <bool MX>
+// value of an unsigned e4m3 byte (see nv4_scale in ffn_mx4.cuh)
+__device__ __forceinline__ float w4_ue4m3(uint32_t b) { return __uint_as_float((b & 0x7Fu) << 20) * 0x1p120f; }
+
+template <int FMT>   // 0: int4-g128, 1: MXFP4, 2: NVFP4
 __global__ void __launch_bounds__(256) dequant_w4_kernel(DequantParams p) {
+  constexpr bool MX = FMT != 0, NV = FMT == 2;
   const int d = p.d, I = p.inter;
   const uint32_t G = (uint32_t)d / 128u, NG = (uint32_t)I / 128u, NBLK = (uint32_t)I / 16u;
   const uint32_t NWD = min(16u, (uint32_t)d / 64u), CBW = 64u * NWD, CB = (uint32_t)d / CBW;
-  const size_t UA = (size_t)(MX ? 2176u : 2112u) * G;
+  const size_t UA = (size_t)(NV ? 2304u : MX ? 2176u : 2112u) * G;
   const size_t sec_b = (size_t)NBLK * UA, sec_c = sec_b + (size_t)I * d / 2;
   const size_t S16 = (size_t)3 * I * d * 2;
   const uint32_t chunks_unit = 6u * (uint32_t)d;                // 16-byte chunks of a 96*d-byte destination unit
@@ -41,6 +46,11 @@ __global__ void __launch_bounds__(256) dequant_w4_kernel(DequantParams p) {
   if (item >= *p.n_items) return;
   const uint32_t u = blockIdx.x;
   const uint8_t *rec = p.items[item].w;
+  float ms[3] = {1.f, 1.f, 1.f};   // NVFP4: the matrix scales
+  if (NV) {
+    const float *tail = reinterpret_cast<const float *>(rec + sec_c + (size_t)I * d / 16);
+    ms[0] = tail[0]; ms[1] = tail[1]; ms[2] = tail[2];
+  }
   uint8_t *dst_unit = p.scratch + (size_t)p.items[item].slot * S16 + (size_t)u * 96u * d;
   for (uint32_t k = threadIdx.x; k < chunks_unit; k += blockDim.x) {
     uint8_t *dst = dst_unit + (size_t)k * 16u;
@@ -52,6 +62,18 @@ __global__ void __launch_bounds__(256) dequant_w4_kernel(DequantParams p) {
       const uint32_t q = pos ^ ((r & 7u) >> 1);                 // chunk q of the row is stored at position pos
       const uint32_t grp = t >> 2, j = t & 3u;                  // hidden indices 128 grp + 32 j + 8 q + 0..7
       const uint8_t *unit = rec + (size_t)u * UA;
+      if (NV) {
+        // hidden indices 8q .. 8q+7 of block j: half q>>1 of the block (= the nibble parity), bytes 0..3 of word j of
+        // the source chunks 2(q&1) and 2(q&1)+1
+        const uint8_t *row = unit + (size_t)mm * 1024u * G + grp * 1024u + r * 64u + j * 4u;
+        const uint32_t wa = *reinterpret_cast<const uint32_t *>(row + (2u * (q & 1u)) * 16u);
+        const uint32_t wb = *reinterpret_cast<const uint32_t *>(row + (2u * (q & 1u) + 1u) * 16u);
+        const uint32_t hf = q >> 1;
+        const uint32_t b = unit[2048u * G + mm * 128u * G + grp * 128u + (r & 7u) * 16u + (r >> 3) * 8u + 2u * j + hf];
+        const float scale = w4_ue4m3(b) * ms[mm];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[e] = scale * w4_code_value(((e < 4 ? wa : wb) >> (8 * (e & 3) + 4 * (int)hf)) & 15u, true);
+      } else {
       const uint32_t w = *reinterpret_cast<const uint32_t *>(unit + (size_t)mm * 1024u * G + grp * 1024u + r * 64u + q * 16u + j * 4u);
       float scale;
       if (MX) {
@@ -63,6 +85,7 @@ __global__ void __launch_bounds__(256) dequant_w4_kernel(DequantParams p) {
       }
 #pragma unroll
       for (int e = 0; e < 8; ++e) v[e] = scale * w4_code_value((w >> (4 * e)) & 15u, MX);
+      }
     } else {
       // ---- down part: tile ct of 16 columns x the unit's 16 neurons, rows of 32 bytes, swizzled ----
       const uint32_t kk = k - 4u * d;
@@ -74,7 +97,9 @@ __global__ void __launch_bounds__(256) dequant_w4_kernel(DequantParams p) {
       const uint8_t *src = rec + sec_b + ((((size_t)(cb * NG + ng) * 8u + uu) * NWD + wq) * 32u + 4u * rr + 2u * nhalf) * 16u + 4u * j;
       const uint32_t w0 = *reinterpret_cast<const uint32_t *>(src), w1 = *reinterpret_cast<const uint32_t *>(src + 16);
       float scale;
-      if (MX) {
+      if (NV) {
+        scale = w4_ue4m3(rec[sec_c + ((size_t)(ng * CB + cb) * NWD + wq) * 512u + 64u * rr + 16u * j + 8u * cg + uu]) * ms[2];
+      } else if (MX) {
         const uint32_t b = rec[sec_c + ((size_t)(ng * CB + cb) * NWD + wq) * 256u + 32u * rr + 8u * j + 4u * cg + (uu >> 1)];
         scale = __uint_as_float(b << 23);
       } else {

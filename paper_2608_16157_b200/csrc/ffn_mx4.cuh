@@ -17,6 +17,8 @@
 #pragma once
 #include <cuda_fp8.h>
 
+#include <type_traits>
+
 #include "ffn_w4.cuh"
 
 namespace ftmoe {
@@ -34,6 +36,18 @@ __device__ __forceinline__ void mma_e4m3_first(float (&c)[4], uint32_t a0, uint3
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
 }
 
+// K = 16 form (one 16-element scale block of an NVFP4 record): a0 = row g, a1 = row g+8, b0 = the token's 4 bytes.
+__device__ __forceinline__ void mma_e4m3_k16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.e4m3.e4m3.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(b0));
+}
+__device__ __forceinline__ void mma_e4m3_k16_first(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.e4m3.e4m3.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%7,%7,%7,%7};"
+      : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
+      : "r"(a0), "r"(a1), "r"(b0), "f"(0.f));
+}
+
 constexpr float kMx4ActMax = 256.f;        // activations of a group are scaled so that the largest magnitude is this
 constexpr float kMx4CodeScale = 64.f;      // the e4m3 placement of a code is code * 2^-6
 
@@ -47,6 +61,12 @@ __device__ __forceinline__ uint32_t mx4_odd(uint32_t w, uint32_t k80, uint32_t k
 // 2^(b - 127) of byte j of a word of four scale bytes.
 __device__ __forceinline__ float mx4_scale(uint32_t w, int j) {
   return __uint_as_float(j < 3 ? ((w << (23 - 8 * j)) & 0x7F800000u) : ((w >> 1) & 0x7F800000u));
+}
+// The unsigned e4m3 number of byte k of a word of four NVFP4 block scales: its bits moved to the float's exponent
+// and mantissa top give the value * 2^-120 (an exact float, subnormal bytes included), the product restores it.
+__device__ __forceinline__ float nv4_scale(uint32_t w, int k) {
+  const uint32_t bits = (k < 3 ? (w << (20 - 8 * k)) : (w >> 4)) & 0x07F00000u;
+  return __uint_as_float(bits) * 0x1p120f;
 }
 // e4m3 rounding of two floats (satfinite), low byte = a.
 __device__ __forceinline__ uint32_t mx4_to_e4m3x2(float a, float b) {
@@ -72,6 +92,18 @@ __device__ __forceinline__ uint4 mx4_split8(const float (&f)[8]) {
   o.w = ((lo[0] >> 8) & 0xff) | (((lo[1] >> 8) & 0xff) << 8) | (((lo[2] >> 8) & 0xff) << 16) | (((lo[3] >> 8) & 0xff) << 24);
   return o;
 }
+// 8 scaled values (consecutive elements) -> hi bytes of elements 0..3, of 4..7, lo bytes of 0..3, of 4..7.
+__device__ __forceinline__ uint4 nv4_split8(const float (&f)[8]) {
+  uint32_t hi[4], lo[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    hi[k] = mx4_to_e4m3x2(f[2 * k], f[2 * k + 1]);
+    const float2 back = mx4_from_e4m3x2(hi[k]);
+    lo[k] = mx4_to_e4m3x2(f[2 * k] - back.x, f[2 * k + 1] - back.y);
+  }
+  return make_uint4((hi[0] & 0xffff) | (hi[1] << 16), (hi[2] & 0xffff) | (hi[3] << 16),
+                    (lo[0] & 0xffff) | (lo[1] << 16), (lo[2] & 0xffff) | (lo[3] << 16));
+}
 __device__ __forceinline__ void mx4_group_scale(float m, bool bad, float &scale, float &inv) {
   if (bad) { scale = __int_as_float(0x7fc00000); inv = 0.f; }
   else if (m < 1e-30f) { scale = 0.f; inv = 0.f; }
@@ -87,14 +119,19 @@ inline size_t mx4_gateup_smem_bytes(int max_items, int d) {
 // ... of the down kernel: per warp 2 slots of (h operands 2048 | 256 bytes of weight scales | 64 bytes of per-token
 // scales) | items | pref.
 constexpr uint32_t kMx4DownSlot = 2048 + 256 + 64;
-inline size_t mx4_down_smem_bytes(int max_items) {
-  return (size_t)kW4Warps * 2 * kMx4DownSlot + (size_t)max_items * sizeof(WorkItem) + ((size_t)max_items + 1) * 4 + 16;
+constexpr uint32_t kNv4DownSlot = 2048 + 512 + 64;   // NVFP4: 512 bytes of weight scales (one per 16 neurons)
+inline size_t mx4_down_smem_bytes(int max_items, bool nv) {
+  return (size_t)kW4Warps * 2 * (nv ? kNv4DownSlot : kMx4DownSlot) + (size_t)max_items * sizeof(WorkItem) +
+         ((size_t)max_items + 1) * 4 + 16;
 }
 
-template <int G>   // groups of 128 of the hidden dimension: d = 128 G
+// NV: NVFP4 records (an e4m3 scale per 16 elements, a float32 scale per matrix; the even codes of a word row are
+// one scale block, the odd codes the next, see include/ftmoe.h) instead of MXFP4 ones.
+template <int G, bool NV>   // groups of 128 of the hidden dimension: d = 128 G
 __global__ void __launch_bounds__(kW4Threads, 1) mx4_gateup_kernel(W4Params p) {
   constexpr int d = kGroup * G;
-  constexpr uint32_t kUA = 2176u * G;               // bytes of a unit: gate tiles, up tiles, gate scales, up scales
+  constexpr uint32_t kST = NV ? 128u : 64u;         // scale bytes of a tile
+  constexpr uint32_t kUA = (2048u + 2u * kST) * G;  // bytes of a unit: gate tiles, up tiles, gate scales, up scales
   constexpr uint32_t kXStride = 2u * d + 64u;
   constexpr int kBS = kW4BlockSteps;
   constexpr int kBlocks = G / kBS;
@@ -144,7 +181,19 @@ __global__ void __launch_bounds__(kW4Threads, 1) mx4_gateup_kernel(W4Params p) {
       mx4_group_scale(m, bad, scale, inv);
 #pragma unroll
       for (int e = 0; e < 8; ++e) f[e] *= inv;
-      *reinterpret_cast<uint4 *>(s_x + j * kXStride + 16 * c8) = mx4_split8(f);
+      if constexpr (NV) {
+        // elements 8 c8 .. 8 c8 + 7 are in half hf of their block of 32; lane q of the MMA reads, for word j4, the 16
+        // bytes (hi of half 0 | hi of half 1 | lo of half 0 | lo of half 1) of elements 4q .. 4q+3 of each half
+        const uint4 sp = nv4_split8(f);
+        const int blk32 = c8 >> 2, hf = (c8 >> 1) & 1, q0 = 2 * (c8 & 1);
+        uint32_t *row = reinterpret_cast<uint32_t *>(s_x + j * kXStride + 64 * blk32);
+        row[4 * q0 + hf] = sp.x;
+        row[4 * (q0 + 1) + hf] = sp.y;
+        row[4 * q0 + 2 + hf] = sp.z;
+        row[4 * (q0 + 1) + 2 + hf] = sp.w;
+      } else {
+        *reinterpret_cast<uint4 *>(s_x + j * kXStride + 16 * c8) = mx4_split8(f);
+      }
       if ((lane & 15) == 0) s_sx[j * G + c8 / 16] = scale;
     }
   };
@@ -155,8 +204,15 @@ __global__ void __launch_bounds__(kW4Threads, 1) mx4_gateup_kernel(W4Params p) {
 
   // The warp that completes a group of 128 neurons of a pass splits its h for the down kernel:
   // lane = (token, quarter): the quarter's two units of 16 neurons = one scale block of the down weights.
-  auto convert_group = [&](uint32_t grp) {
+  const size_t tail = (size_t)(p.inter / 16) * kUA + (size_t)p.inter * d / 2 + (size_t)p.inter * d / 16;   // NV only
+  auto convert_group = [&](uint32_t grp, const uint8_t *rec) {
     const int tok = lane >> 2, qt = lane & 3;
+    float cs_g = kMx4CodeScale, cs_u = kMx4CodeScale;
+    if constexpr (NV) {
+      const float2 ms = __ldg(reinterpret_cast<const float2 *>(rec + tail));   // matrix scales of gate and up
+      cs_g *= ms.x;
+      cs_u *= ms.y;
+    }
     float *src = p.hraw + ((size_t)grp * 8 + 2 * qt) * 256 + tok * 16;   // per unit: gate sums [8][16], up sums [8][16]
     float v[2][16];
 #pragma unroll
@@ -167,8 +223,8 @@ __global__ void __launch_bounds__(kW4Threads, 1) mx4_gateup_kernel(W4Params p) {
         float4 a = __ldcg(pg), b = __ldcg(pu_);
         __stcg(pg, make_float4(0.f, 0.f, 0.f, 0.f));   // the sums start from zero in the next call
         __stcg(pu_, make_float4(0.f, 0.f, 0.f, 0.f));
-        a.x *= kMx4CodeScale; a.y *= kMx4CodeScale; a.z *= kMx4CodeScale; a.w *= kMx4CodeScale;
-        b.x *= kMx4CodeScale; b.y *= kMx4CodeScale; b.z *= kMx4CodeScale; b.w *= kMx4CodeScale;
+        a.x *= cs_g; a.y *= cs_g; a.z *= cs_g; a.w *= cs_g;
+        b.x *= cs_u; b.y *= cs_u; b.z *= cs_u; b.w *= cs_u;
         v[u][4 * k4] = __fdividef(a.x, 1.f + __expf(-a.x)) * b.x;
         v[u][4 * k4 + 1] = __fdividef(a.y, 1.f + __expf(-a.y)) * b.y;
         v[u][4 * k4 + 2] = __fdividef(a.z, 1.f + __expf(-a.z)) * b.z;
@@ -208,20 +264,23 @@ __global__ void __launch_bounds__(kW4Threads, 1) mx4_gateup_kernel(W4Params p) {
     if (qt == 0) p.hs[(size_t)grp * 8 + tok] = make_float2(scale, 0.f);
   };
 
-  auto run = [&](const uint8_t *base, int ks0, int n_pieces, uint32_t hrow0) {
+  auto run = [&](const uint8_t *rec, const uint8_t *base, int ks0, int n_pieces, uint32_t hrow0) {
     uint4 buf[4 * kBS];     // per step: gate rows g, g+8; up rows g, g+8
-    uint2 sc[2 * kBS];      // per step: the four block scales of rows g (.x) and g+8 (.y), gate then up
+    // per step: the block scales of rows g and g+8, gate then up (MXFP4: four each in .x and .y; NVFP4: eight each
+    // in .x .y and .z .w)
+    using ScaleT = typename std::conditional<NV, uint4, uint2>::type;
+    ScaleT sc[2 * kBS];
     const uint8_t *nptr = base + ks0 * (G / kKS) * 1024 + g * 64 + q * 16;
-    const uint8_t *nsc = base + 2048u * G + ks0 * (G / kKS) * 64 + g * 8;
+    const uint8_t *nsc = base + 2048u * G + ks0 * (G / kKS) * kST + g * (kST / 8);
     int nblk = ks0 * kBlocksP, blocks_left = n_pieces * kBlocksP;
     auto advance = [&]() {
       nptr += kBS * 1024;
-      nsc += kBS * 64;
+      nsc += kBS * kST;
       --blocks_left;
       if (++nblk == kBlocks) {   // on to the next unit
         nblk = 0;
         nptr += kUA - 1024u * G;
-        nsc += kUA - 64u * G;
+        nsc += kUA - kST * G;
       }
     };
     auto request = [&](int si, const uint8_t *tp, const uint8_t *sp) {
@@ -229,8 +288,13 @@ __global__ void __launch_bounds__(kW4Threads, 1) mx4_gateup_kernel(W4Params p) {
       buf[4 * si + 1] = ld_stream_16(tp + si * 1024 + 512);
       buf[4 * si + 2] = ld_stream_16(tp + si * 1024 + 1024 * G);
       buf[4 * si + 3] = ld_stream_16(tp + si * 1024 + 1024 * G + 512);
-      sc[2 * si] = ld_stream_8(sp + si * 64);
-      sc[2 * si + 1] = ld_stream_8(sp + si * 64 + 64 * G);
+      if constexpr (NV) {
+        sc[2 * si] = ld_stream_16(sp + si * kST);
+        sc[2 * si + 1] = ld_stream_16(sp + si * kST + kST * G);
+      } else {
+        sc[2 * si] = ld_stream_8(sp + si * kST);
+        sc[2 * si + 1] = ld_stream_8(sp + si * kST + kST * G);
+      }
     };
 #pragma unroll
     for (int si = 0; si < kBS; ++si) request(si, nptr, nsc);
@@ -251,11 +315,41 @@ __global__ void __launch_bounds__(kW4Threads, 1) mx4_gateup_kernel(W4Params p) {
           const uint32_t ghi[4] = {buf[4 * si + 1].x, buf[4 * si + 1].y, buf[4 * si + 1].z, buf[4 * si + 1].w};
           const uint32_t ulo[4] = {buf[4 * si + 2].x, buf[4 * si + 2].y, buf[4 * si + 2].z, buf[4 * si + 2].w};
           const uint32_t uhi[4] = {buf[4 * si + 3].x, buf[4 * si + 3].y, buf[4 * si + 3].z, buf[4 * si + 3].w};
-          const uint2 gs = sc[2 * si], us = sc[2 * si + 1];
+          const ScaleT gs = sc[2 * si], us = sc[2 * si + 1];
           float sg[4] = {0.f, 0.f, 0.f, 0.f}, su[4] = {0.f, 0.f, 0.f, 0.f};   // the step's sums, before the activation scale
 #pragma unroll
           for (int j = 0; j < 4; ++j) {   // word j = scale block j of the group: hidden indices 32j + 8q + 0..7
             const uint4 xv = lds_v4(xa + si * 256u + j * 64u);
+            if constexpr (NV) {
+              // even codes = block 2j, odd codes = block 2j+1 of the group, each with its own scale per row
+              float e0[4], e1[4];
+              {
+                const uint32_t a0 = mx4_even(glo[j], k80, k1c), a1 = mx4_even(ghi[j], k80, k1c);
+                const uint32_t a2 = mx4_odd(glo[j], k80, k1c), a3 = mx4_odd(ghi[j], k80, k1c);
+                mma_e4m3_k16_first(e0, a0, a1, xv.x);
+                mma_e4m3_k16(e0, a0, a1, xv.z);
+                mma_e4m3_k16_first(e1, a2, a3, xv.y);
+                mma_e4m3_k16(e1, a2, a3, xv.w);
+              }
+              const uint32_t wlo = j < 2 ? gs.x : gs.y, whi = j < 2 ? gs.z : gs.w;
+              const float l0 = nv4_scale(wlo, 2 * (j & 1)), l1 = nv4_scale(wlo, 2 * (j & 1) + 1);
+              const float h0 = nv4_scale(whi, 2 * (j & 1)), h1 = nv4_scale(whi, 2 * (j & 1) + 1);
+              sg[0] += l0 * e0[0] + l1 * e1[0]; sg[1] += l0 * e0[1] + l1 * e1[1];
+              sg[2] += h0 * e0[2] + h1 * e1[2]; sg[3] += h0 * e0[3] + h1 * e1[3];
+              {
+                const uint32_t a0 = mx4_even(ulo[j], k80, k1c), a1 = mx4_even(uhi[j], k80, k1c);
+                const uint32_t a2 = mx4_odd(ulo[j], k80, k1c), a3 = mx4_odd(uhi[j], k80, k1c);
+                mma_e4m3_k16_first(e0, a0, a1, xv.x);
+                mma_e4m3_k16(e0, a0, a1, xv.z);
+                mma_e4m3_k16_first(e1, a2, a3, xv.y);
+                mma_e4m3_k16(e1, a2, a3, xv.w);
+              }
+              const uint32_t vlo = j < 2 ? us.x : us.y, vhi = j < 2 ? us.z : us.w;
+              const float m0 = nv4_scale(vlo, 2 * (j & 1)), m1 = nv4_scale(vlo, 2 * (j & 1) + 1);
+              const float n0 = nv4_scale(vhi, 2 * (j & 1)), n1 = nv4_scale(vhi, 2 * (j & 1) + 1);
+              su[0] += m0 * e0[0] + m1 * e1[0]; su[1] += m0 * e0[1] + m1 * e1[1];
+              su[2] += n0 * e0[2] + n1 * e1[2]; su[3] += n0 * e0[3] + n1 * e1[3];
+            } else {
             float ga[4], ua[4];
             {
               const uint32_t a0 = mx4_even(glo[j], k80, k1c), a1 = mx4_even(ghi[j], k80, k1c);
@@ -273,6 +367,7 @@ __global__ void __launch_bounds__(kW4Threads, 1) mx4_gateup_kernel(W4Params p) {
             const float u_lo = mx4_scale(us.x, j), u_hi = mx4_scale(us.y, j);
             sg[0] += g_lo * ga[0]; sg[1] += g_lo * ga[1]; sg[2] += g_hi * ga[2]; sg[3] += g_hi * ga[3];
             su[0] += u_lo * ua[0]; su[1] += u_lo * ua[1]; su[2] += u_hi * ua[2]; su[3] += u_hi * ua[3];
+            }
           }
           if (more) request(si, rp, rs);   // refill the step just consumed
           const float sx0 = my_s0[xg + si], sx1 = my_s1[xg + si];
@@ -296,7 +391,7 @@ __global__ void __launch_bounds__(kW4Threads, 1) mx4_gateup_kernel(W4Params p) {
       old = __shfl_sync(0xffffffffu, old, 0);
       if (old == 8 * kKS - 1) {
         __threadfence();
-        convert_group(hrow_i >> 3);
+        convert_group(hrow_i >> 3, rec);
         if (lane == 0) p.hcount[hrow_i >> 3] = 0;
       }
       if (++ks == kKS) { ks = 0; ++hrow_i; }
@@ -337,17 +432,19 @@ __global__ void __launch_bounds__(kW4Threads, 1) mx4_gateup_kernel(W4Params p) {
       const uint32_t lo = max(wf, pu * PP), hi = min(we, (pu + 1) * PP);
       if (lo < hi) {
         const uint32_t rel = lo - pu * PP;
-        run(it.w + (size_t)(rel / kKS) * kUA, (int)(rel % kKS), (int)(hi - lo), pu * NBLK + rel / kKS);
+        run(it.w, it.w + (size_t)(rel / kKS) * kUA, (int)(rel % kKS), (int)(hi - lo), pu * NBLK + rel / kKS);
       }
     }
   }
 }
 
-template <int NWD>   // warps that own output columns: a column block is 64 * NWD columns
+template <int NWD, bool NV>   // warps that own output columns: a column block is 64 * NWD columns
 __global__ void __launch_bounds__(kW4Threads, 1) mx4_down_kernel(W4Params p, int d) {
+  constexpr uint32_t kSlot = NV ? kNv4DownSlot : kMx4DownSlot;
+  constexpr uint32_t kSW = NV ? 512u : 256u;   // weight scale bytes of a chunk and warp
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char *s_h = smem;                                                // [16 warps][2 slots]
-  WorkItem *s_items = reinterpret_cast<WorkItem *>(smem + kW4Warps * 2 * kMx4DownSlot);
+  WorkItem *s_items = reinterpret_cast<WorkItem *>(smem + kW4Warps * 2 * kSlot);
   int32_t *s_pref = reinterpret_cast<int32_t *>(s_items + p.max_items);
   __shared__ int s_last;
 
@@ -363,7 +460,8 @@ __global__ void __launch_bounds__(kW4Threads, 1) mx4_down_kernel(W4Params p, int
   __syncthreads();
   const uint32_t NBLK = (uint32_t)p.inter / 16u, NG = (uint32_t)p.inter / 128u;
   const uint32_t G = (uint32_t)d / 128u, CB = (uint32_t)d / (64u * NWD);
-  const size_t sec_b = (size_t)NBLK * 2176u * G, sec_c = sec_b + (size_t)p.inter * d / 2;
+  const size_t sec_b = (size_t)NBLK * (NV ? 2304u : 2176u) * G, sec_c = sec_b + (size_t)p.inter * d / 2;
+  const size_t tail = sec_c + (size_t)p.inter * d / 16;   // NV only: the matrix scales
   const uint32_t per_pass = CB * NG;
   const bool dense = p.T <= kQ4Tokens;
   asm volatile("griddepcontrol.wait;" ::: "memory");   // from here on the gate/up kernel's h is needed
@@ -374,7 +472,7 @@ __global__ void __launch_bounds__(kW4Threads, 1) mx4_down_kernel(W4Params p, int
     const uint32_t rfirst0 = w4_first(t0, gridDim.x, blockIdx.x), rcount0 = w4_first(t0, gridDim.x, blockIdx.x + 1) - rfirst0;
     const uint32_t rfirst1 = t0 + w4_first(t1, gridDim.x, blockIdx.x);
     const uint32_t rcount1 = t0 + w4_first(t1, gridDim.x, blockIdx.x + 1) - rfirst1;
-    const uint32_t my_h = smem_u32(s_h) + (uint32_t)warp * 2u * kMx4DownSlot;
+    const uint32_t my_h = smem_u32(s_h) + (uint32_t)warp * 2u * kSlot;
     const uint32_t k1c = p.mask, k80 = p.flip;
 
     struct Ck { const uint8_t *rec; uint32_t pu, cb, ng; int item; };
@@ -410,17 +508,17 @@ __global__ void __launch_bounds__(kW4Threads, 1) mx4_down_kernel(W4Params p, int
     auto stage = [&](const Ck &c, uint32_t slot) {
       const size_t grp = (size_t)c.pu * NG + c.ng;
       const uint8_t *hsrc = p.hq + grp * 2048;
-      const uint32_t dst = my_h + slot * kMx4DownSlot;
+      const uint32_t dst = my_h + slot * kSlot;
 #pragma unroll
       for (int i = 0; i < 4; ++i)
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (i * 32 + lane) * 16u), "l"(hsrc + (i * 32 + lane) * 16)
                      : "memory");
-      if (lane < 16)
+      if (NV || lane < 16)
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 2048u + lane * 16u),
-                     "l"(c.rec + sec_c + ((size_t)(c.ng * CB + c.cb) * NWD + warp) * 256u + lane * 16u)
+                     "l"(c.rec + sec_c + ((size_t)(c.ng * CB + c.cb) * NWD + warp) * kSW + lane * 16u)
                      : "memory");
-      else if (lane < 20)   // (scale, unused) of the 8 tokens: 64 bytes, of which the scales are used
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 2304u + (lane - 16) * 16u),
+      if (lane >= 16 && lane < 20)   // (scale, unused) of the 8 tokens: 64 bytes, of which the scales are used
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 2048u + kSW + (lane - 16) * 16u),
                      "l"(reinterpret_cast<const uint8_t *>(p.hs + grp * 8) + (lane - 16) * 16)
                      : "memory");
     };
@@ -453,7 +551,7 @@ __global__ void __launch_bounds__(kW4Threads, 1) mx4_down_kernel(W4Params p, int
         }
       }
     };
-    auto flush = [&](uint32_t cb) {
+    auto flush = [&](uint32_t cb, const uint8_t *rec) {
       int tok_a, tok_b;
       float gw_a, gw_b;
       if (dense) {
@@ -471,8 +569,10 @@ __global__ void __launch_bounds__(kW4Threads, 1) mx4_down_kernel(W4Params p, int
         gw_a = __shfl_sync(0xffffffffu, my_w, 2 * q);
         gw_b = __shfl_sync(0xffffffffu, my_w, 2 * q + 1);
       }
-      gw_a *= kMx4CodeScale;
-      gw_b *= kMx4CodeScale;
+      float cs = kMx4CodeScale;
+      if constexpr (NV) cs *= __ldg(reinterpret_cast<const float *>(rec + tail) + 2);   // matrix scale of down
+      gw_a *= cs;
+      gw_b *= cs;
       const int col0 = (int)cb * 64 * NWD + warp * 64 + g;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
@@ -506,10 +606,15 @@ __global__ void __launch_bounds__(kW4Threads, 1) mx4_down_kernel(W4Params p, int
       const uint8_t *refill = h1 ? weights_of(c1) : nullptr;
       asm volatile("cp.async.wait_group 1;" ::: "memory");
       __syncwarp();
-      const uint32_t hs_base = my_h + slot * kMx4DownSlot;
-      // weight scales of the chunk: word 2j + half = the four 32-neuron blocks of (tile j, column g + 8 half)
-      const uint4 sa = lds_v4(hs_base + 2048u + g * 32u), sb = lds_v4(hs_base + 2048u + g * 32u + 16u);
-      const uint32_t sw[8] = {sa.x, sa.y, sa.z, sa.w, sb.x, sb.y, sb.z, sb.w};
+      const uint32_t hs_base = my_h + slot * kSlot;
+      // weight scales of the chunk.  MXFP4: word 2j + half = the four 32-neuron blocks of (tile j, column g + 8 half);
+      // NVFP4: words 4j + 2 half, + 1 = the eight 16-neuron blocks
+      uint32_t sw[NV ? 16 : 8];
+#pragma unroll
+      for (int i = 0; i < (NV ? 4 : 2); ++i) {
+        const uint4 sv = lds_v4(hs_base + 2048u + g * (kSW / 8u) + 16u * i);
+        sw[4 * i] = sv.x; sw[4 * i + 1] = sv.y; sw[4 * i + 2] = sv.z; sw[4 * i + 3] = sv.w;
+      }
       float ct[4][4];   // the chunk's sums, before the activation scale
 #pragma unroll
       for (int j = 0; j < 4; ++j) { ct[j][0] = ct[j][1] = ct[j][2] = ct[j][3] = 0.f; }
@@ -522,18 +627,31 @@ __global__ void __launch_bounds__(kW4Threads, 1) mx4_down_kernel(W4Params p, int
         for (int j = 0; j < 4; ++j) {   // tile j: columns g (even codes) and g+8 (odd codes)
           const uint32_t a0 = mx4_even(w0[j], k80, k1c), a1 = mx4_odd(w0[j], k80, k1c);
           const uint32_t a2 = mx4_even(w1[j], k80, k1c), a3 = mx4_odd(w1[j], k80, k1c);
+          if constexpr (NV) {
+            float e0[4], e1[4];   // unit 2m and unit 2m+1: one scale block each
+            mma_e4m3_k16_first(e0, a0, a1, hv.x);
+            mma_e4m3_k16(e0, a0, a1, hv.z);
+            mma_e4m3_k16_first(e1, a2, a3, hv.y);
+            mma_e4m3_k16(e1, a2, a3, hv.w);
+            const uint32_t wlo = sw[4 * j + (m >> 1)], whi = sw[4 * j + 2 + (m >> 1)];
+            const float l0 = nv4_scale(wlo, 2 * (m & 1)), l1 = nv4_scale(wlo, 2 * (m & 1) + 1);
+            const float h0 = nv4_scale(whi, 2 * (m & 1)), h1 = nv4_scale(whi, 2 * (m & 1) + 1);
+            ct[j][0] += l0 * e0[0] + l1 * e1[0]; ct[j][1] += l0 * e0[1] + l1 * e1[1];
+            ct[j][2] += h0 * e0[2] + h1 * e1[2]; ct[j][3] += h0 * e0[3] + h1 * e1[3];
+          } else {
           float acc[4];
           mma_e4m3_first(acc, a0, a1, a2, a3, hv.x, hv.y);
           mma_e4m3(acc, a0, a1, a2, a3, hv.z, hv.w);
           const float s_lo = mx4_scale(sw[2 * j], m), s_hi = mx4_scale(sw[2 * j + 1], m);
           ct[j][0] += s_lo * acc[0]; ct[j][1] += s_lo * acc[1]; ct[j][2] += s_hi * acc[2]; ct[j][3] += s_hi * acc[3];
+          }
         }
         if (refill) {
           buf[2 * m] = ld_stream_16(refill + (size_t)(2 * m) * NWD * 512u);
           buf[2 * m + 1] = ld_stream_16(refill + (size_t)(2 * m + 1) * NWD * 512u);
         }
       }
-      const uint4 tb = lds_v4(hs_base + 2304u + q * 16u);   // tokens 2q, 2q+1: (scale, unused) each
+      const uint4 tb = lds_v4(hs_base + 2048u + kSW + q * 16u);   // tokens 2q, 2q+1: (scale, unused) each
       __syncwarp();   // every lane has read the slot: it may be overwritten
       const float sh0 = __uint_as_float(tb.x), sh1 = __uint_as_float(tb.z);
 #pragma unroll
@@ -541,7 +659,7 @@ __global__ void __launch_bounds__(kW4Threads, 1) mx4_down_kernel(W4Params p, int
         dtot[j][0] += ct[j][0] * sh0; dtot[j][1] += ct[j][1] * sh1; dtot[j][2] += ct[j][2] * sh0; dtot[j][3] += ct[j][3] * sh1;
       }
       if (!h1 || c1.pu != c0.pu || c1.cb != c0.cb) {
-        flush(c0.cb);
+        flush(c0.cb, c0.rec);
         zero_tot();
         if (h1 && c1.pu != c0.pu) begin_pass(c1);
       }

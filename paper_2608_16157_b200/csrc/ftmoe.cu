@@ -165,6 +165,10 @@ size_t expert_bytes_of(const ft_moe_config_t *c) {
     if (d % 512 || d > 8192 || I % 128) return 0;   // (same shapes as int4)
     return 3 * I * d / 2 + 3 * I * d / 32;
   }
+  if (c->wdtype == FT_W_NVFP4) {
+    if (d % 512 || d > 8192 || I % 128) return 0;   // (same shapes as int4)
+    return 3 * I * d / 2 + 3 * I * d / 16 + 256;
+  }
   if (c->wdtype == FT_W_INT4_G128) {
     if (d % 512 || d > 8192 || I % 128) return 0;   // (the kernels further restrict d, see w4_shape_ok)
     return 3 * I * d / 2 + (2 * I * (d / 128) + (I / 128) * d) * 2;
@@ -526,7 +530,8 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
       c.max_tokens <= 0 || (c.n_shared != 0 && c.n_shared != 1) || c.device < 0 ||
       (c.fill_mode != FT_FILL_COPY_ENGINE && c.fill_mode != FT_FILL_SM))
     return FT_ERR_INVALID_ARG;
-  if (c.wdtype != FT_W_BF16 && c.wdtype != FT_W_INT4_G128 && c.wdtype != FT_W_MXFP4) return FT_ERR_INVALID_ARG;
+  if (c.wdtype != FT_W_BF16 && c.wdtype != FT_W_INT4_G128 && c.wdtype != FT_W_MXFP4 && c.wdtype != FT_W_NVFP4)
+    return FT_ERR_INVALID_ARG;
   if (c.bw_fill_MBps == 0 || c.bw_zc_MBps == 0 || c.bw_hbm_MBps == 0 || c.reuse_credit < 0 ||
       c.zc_tokens_per_pass < 1 || c.hbm_tokens_per_pass < 1 || c.gemm_min_tokens < 0 || c.split_min_pairs < 0)
     return FT_ERR_INVALID_ARG;
@@ -656,7 +661,7 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
   FT_TRY(cudaMalloc(&h->done_dev, 4));
   FT_TRY(cudaMemset(h->done_dev, 0, 4));
   FT_TRY(cudaFuncSetAttribute(fill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFillStages * (int)kFillChunk));
-  if (c.wdtype == FT_W_INT4_G128 || c.wdtype == FT_W_MXFP4) {
+  if (c.wdtype != FT_W_BF16) {
     const size_t passes = (P + 7) / 8 + 2 * E + 2;
     FT_TRY(cudaMalloc(&h->w4_hraw, passes * (c.inter / 16) * 1024));
     FT_TRY(cudaMemset(h->w4_hraw, 0, passes * (c.inter / 16) * 1024));
@@ -684,15 +689,16 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
     FT_TRY(cudaFuncSetAttribute(w4_gateup_half_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
     FT_TRY(cudaFuncSetAttribute(w4_down_half_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
     FT_TRY(cudaFuncSetAttribute(w4_down_half_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb));
-    const int sbm = (int)mx4_down_smem_bytes(2 * kMaxExperts + 1);
-    FT_TRY(cudaFuncSetAttribute(mx4_gateup_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
-    FT_TRY(cudaFuncSetAttribute(mx4_gateup_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
-    FT_TRY(cudaFuncSetAttribute(mx4_gateup_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
-    FT_TRY(cudaFuncSetAttribute(mx4_gateup_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
-    FT_TRY(cudaFuncSetAttribute(mx4_gateup_kernel<56>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
-    FT_TRY(cudaFuncSetAttribute(mx4_gateup_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
-    FT_TRY(cudaFuncSetAttribute(mx4_down_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, sbm));
-    FT_TRY(cudaFuncSetAttribute(mx4_down_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sbm));
+    const int sbm = (int)mx4_down_smem_bytes(2 * kMaxExperts + 1, false), sbn = (int)mx4_down_smem_bytes(2 * kMaxExperts + 1, true);
+#define FT_MX_ATTR(G)                                                                                                   \
+  FT_TRY(cudaFuncSetAttribute(mx4_gateup_kernel<G, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));           \
+  FT_TRY(cudaFuncSetAttribute(mx4_gateup_kernel<G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, sa));
+    FT_MX_ATTR(4) FT_MX_ATTR(8) FT_MX_ATTR(16) FT_MX_ATTR(32) FT_MX_ATTR(56) FT_MX_ATTR(64)
+#undef FT_MX_ATTR
+    FT_TRY(cudaFuncSetAttribute(mx4_down_kernel<8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, sbm));
+    FT_TRY(cudaFuncSetAttribute(mx4_down_kernel<16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, sbm));
+    FT_TRY(cudaFuncSetAttribute(mx4_down_kernel<8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, sbn));
+    FT_TRY(cudaFuncSetAttribute(mx4_down_kernel<16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, sbn));
   }
   if (c.wdtype == FT_W_BF16) {
     // the limit is a property of the function on this device, not of the handle: always the largest size any
@@ -1059,7 +1065,8 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   qp.pref = sc.res_pref;
   qp.max_items = 2 * c.n_experts + 1;
   qp.x = x_bf; qp.perm = sc.perm; qp.topk_w = sc.topk_w;
-  const bool mx = c.wdtype == FT_W_MXFP4;
+  const bool nv = c.wdtype == FT_W_NVFP4;
+  const bool mx = c.wdtype == FT_W_MXFP4 || nv;   // the floating-point 4-bit formats share their kernels
   qp.overlap = h->overlap;
   if (mx) { qp.mask = 0x1C1C1C1Cu; qp.flip = 0x80808080u; }   // (see ffn_mx4.cuh)
   else { qp.mask = 0x0F0F0F0Fu; qp.flip = 0x08080808u; }
@@ -1072,7 +1079,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   const bool half = !mx && L.T <= kW4HalfTokens;   // int4 with at most 4 tokens: one MMA per pair of weight words
   const size_t sa = mx ? mx4_gateup_smem_bytes(qp.max_items, c.hidden)
                        : half ? w4_gateup_half_smem_bytes(qp.max_items, c.hidden) : w4_gateup_smem_bytes(qp.max_items, c.hidden);
-  const size_t sb = mx ? mx4_down_smem_bytes(qp.max_items)
+  const size_t sb = mx ? mx4_down_smem_bytes(qp.max_items, nv)
                        : half ? w4_down_half_smem_bytes(qp.max_items) : w4_down_smem_bytes(qp.max_items);
   const int grid = h->sm_count;
   {
@@ -1085,14 +1092,16 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     lc.attrs = at; lc.numAttrs = h->overlap ? 1 : 0;
     cudaError_t le;
     if (mx) {
+#define FT_MX_LAUNCH(G) (nv ? cudaLaunchKernelEx(&lc, mx4_gateup_kernel<G, true>, qp) : cudaLaunchKernelEx(&lc, mx4_gateup_kernel<G, false>, qp))
       switch (c.hidden) {
-        case 512: le = cudaLaunchKernelEx(&lc, mx4_gateup_kernel<4>, qp); break;
-        case 1024: le = cudaLaunchKernelEx(&lc, mx4_gateup_kernel<8>, qp); break;
-        case 2048: le = cudaLaunchKernelEx(&lc, mx4_gateup_kernel<16>, qp); break;
-        case 4096: le = cudaLaunchKernelEx(&lc, mx4_gateup_kernel<32>, qp); break;
-        case 7168: le = cudaLaunchKernelEx(&lc, mx4_gateup_kernel<56>, qp); break;
-        default: le = cudaLaunchKernelEx(&lc, mx4_gateup_kernel<64>, qp); break;
+        case 512: le = FT_MX_LAUNCH(4); break;
+        case 1024: le = FT_MX_LAUNCH(8); break;
+        case 2048: le = FT_MX_LAUNCH(16); break;
+        case 4096: le = FT_MX_LAUNCH(32); break;
+        case 7168: le = FT_MX_LAUNCH(56); break;
+        default: le = FT_MX_LAUNCH(64); break;
       }
+#undef FT_MX_LAUNCH
     } else if (half) {
       switch (c.hidden) {
         case 512: le = cudaLaunchKernelEx(&lc, w4_gateup_half_kernel<4>, qp); break;
@@ -1124,9 +1133,12 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = at; lc.numAttrs = 1;
-    if (mx) {
-      if (c.hidden == 512) FT_CUDA(cudaLaunchKernelEx(&lc, mx4_down_kernel<8>, qp, c.hidden));
-      else FT_CUDA(cudaLaunchKernelEx(&lc, mx4_down_kernel<16>, qp, c.hidden));
+    if (nv) {
+      if (c.hidden == 512) FT_CUDA(cudaLaunchKernelEx(&lc, mx4_down_kernel<8, true>, qp, c.hidden));
+      else FT_CUDA(cudaLaunchKernelEx(&lc, mx4_down_kernel<16, true>, qp, c.hidden));
+    } else if (mx) {
+      if (c.hidden == 512) FT_CUDA(cudaLaunchKernelEx(&lc, mx4_down_kernel<8, false>, qp, c.hidden));
+      else FT_CUDA(cudaLaunchKernelEx(&lc, mx4_down_kernel<16, false>, qp, c.hidden));
     } else if (half) {
       if (c.hidden == 512) FT_CUDA(cudaLaunchKernelEx(&lc, w4_down_half_kernel<8>, qp, c.hidden));
       else FT_CUDA(cudaLaunchKernelEx(&lc, w4_down_half_kernel<16>, qp, c.hidden));
@@ -1150,8 +1162,9 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     {
       TimeScope ts(h, st, FT_TIME_GATHER);
       const dim3 dg((unsigned)(c.inter / 16), (unsigned)std::min(c.n_experts, c.slots_per_layer));
-      if (mx) dequant_w4_kernel<true><<<dg, 256, 0, st>>>(dp);
-      else dequant_w4_kernel<false><<<dg, 256, 0, st>>>(dp);
+      if (nv) dequant_w4_kernel<2><<<dg, 256, 0, st>>>(dp);
+      else if (mx) dequant_w4_kernel<1><<<dg, 256, 0, st>>>(dp);
+      else dequant_w4_kernel<0><<<dg, 256, 0, st>>>(dp);
     }
     h->launches++;
     return launch_gemm_path(h, layer, L, sc, x_bf, y_dev, st);

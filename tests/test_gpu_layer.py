@@ -108,7 +108,7 @@ def test_results_do_not_depend_on_residency():
     assert torch.equal(ys["fill"], ys["hit"]) or (ys["fill"] - ys["hit"]).abs().max() <= 1e-2 * scale
 
 
-@pytest.mark.parametrize("wdtype", ["int4", "mxfp4"])
+@pytest.mark.parametrize("wdtype", ["int4", "mxfp4", "nvfp4"])
 @pytest.mark.parametrize("n_shared", [0, 1])
 @pytest.mark.parametrize("T", [1, 4, 7])
 def test_int4_group_dequant_and_shared_expert(n_shared, T, wdtype):
@@ -119,7 +119,7 @@ def test_int4_group_dequant_and_shared_expert(n_shared, T, wdtype):
     pr.close()
 
 
-@pytest.mark.parametrize("wdtype", ["int4", "mxfp4"])
+@pytest.mark.parametrize("wdtype", ["int4", "mxfp4", "nvfp4"])
 @pytest.mark.parametrize("T", [9, 24, 40])
 def test_int4_resident_experts_with_many_tokens_and_shared_expert(T, wdtype):
     """More than 8 tokens per slot-resident 4-bit expert (several weight passes) and the shared expert at T > 8."""
@@ -133,7 +133,7 @@ def test_int4_resident_experts_with_many_tokens_and_shared_expert(T, wdtype):
     pr.close()
 
 
-@pytest.mark.parametrize("wdtype", ["int4", "mxfp4"])
+@pytest.mark.parametrize("wdtype", ["int4", "mxfp4", "nvfp4"])
 @pytest.mark.parametrize("scale_log2", [-10, 10])
 def test_int4_activation_range(scale_log2, wdtype):
     """The 4-bit kernels re-express activations and h per (token, group of 128) against the group's largest magnitude,
@@ -147,7 +147,7 @@ def test_int4_activation_range(scale_log2, wdtype):
     pr.close()
 
 
-@pytest.mark.parametrize("wdtype", ["int4", "mxfp4"])
+@pytest.mark.parametrize("wdtype", ["int4", "mxfp4", "nvfp4"])
 def test_int4_activation_outlier_in_a_group(wdtype):
     """One element 1000 x larger than the rest of its quantisation group: the group's re-expressed form (15-bit fixed
     point, or two fp8 numbers, against the group's largest magnitude) keeps the result within the tolerance."""
@@ -159,6 +159,29 @@ def test_int4_activation_outlier_in_a_group(wdtype):
         x[2, :] = 0.0                                # and an all-zero token
         pr.step(0, W.normal_logits(6, 8, 12, step), x.to(torch.bfloat16))
     pr.close()
+
+
+def test_nvfp4_small_and_subnormal_block_scales():
+    """NVFP4 records written by definition whose gate and down block scales are the 15 smallest e4m3 numbers (exponent
+    field 0 or 1: the subnormal bytes included) under a matrix scale of 2^9, so that an error in the decoding of
+    those bytes would show in y."""
+    from tests.test_oracle_ffn import _record_nvfp4_by_definition
+    d, I, E = 512, 128, 4
+    shape = W.LayerShape(d=d, inter=I, n_experts=E, top_k=2, wdtype="nvfp4")
+    rng = np.random.default_rng(21)
+    pool = B.HostPool(E * shape.expert_bytes)
+    recs = pool.tensor.view(E, shape.expert_bytes).numpy()
+    for e in range(E):
+        cg, cu, cd = (rng.integers(0, 16, size=(I, d)) for _ in range(3))
+        bg = rng.integers(1, 16, size=(I, d // 16))
+        bu = rng.integers(0x2C, 0x3C, size=(I, d // 16))
+        bd = rng.integers(1, 16, size=(I // 16, d))
+        recs[e] = _record_nvfp4_by_definition(cg, cu, cd, bg, bu, bd, (512.0 * 0.05, 0.02, 512.0 * 0.05))
+    pr = Pair(shape, n_slots=2, max_tokens=8, seed=21, pool=pool)
+    for step in range(2):
+        pr.step(0, W.normal_logits(5, E, 21, step), W.noise_x(5, d, 21, step, 0), check_slots=True)
+    pr.close()
+    pool.free()
 
 
 def test_plan_and_permutation_are_deterministic():
@@ -262,9 +285,9 @@ def test_qwen3_shaped_decode_two_layers(batch):
     pr.close()
 
 
-@pytest.mark.parametrize("shape", [W.DSV3_INT4, W.DSV3_MXFP4], ids=["int4", "mxfp4"])
+@pytest.mark.parametrize("shape", [W.DSV3_INT4, W.DSV3_MXFP4, W.DSV3_NVFP4], ids=["int4", "mxfp4", "nvfp4"])
 def test_dsv3_shaped_int4_decode_one_layer(shape):
-    """d=7168, 256 routed experts (int4 group 128, or mxfp4) + 1 shared expert, I=2048, top-8, 64 slots, batch 4."""
+    """d=7168, 256 routed experts (int4 group 128, mxfp4 or nvfp4) + 1 shared expert, I=2048, top-8, 64 slots, batch 4."""
     steps = 3
     pr = Pair(shape, n_slots=64, max_tokens=8, n_layers=1, seed=0, gen_device="cuda")
     logits = W.ar1_logits(1, steps, 4, 256, rho=0.9, alpha=1.2, seed=0)
