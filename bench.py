@@ -185,9 +185,10 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    dsv3 = args.workload in ("dsv3", "dsv3_mxfp4")
-    mxfp4 = args.workload == "dsv3_mxfp4"
-    shape = (W.DSV3_MXFP4 if mxfp4 else W.DSV3_INT4) if dsv3 else W.QWEN3_30B
+    dsv3 = args.workload in ("dsv3", "dsv3_mxfp4", "dsv3_nvfp4")
+    mxfp4 = args.workload in ("dsv3_mxfp4", "dsv3_nvfp4")    # the floating-point 4-bit formats share their kernels
+    fp4_name = "nvfp4" if args.workload == "dsv3_nvfp4" else "mxfp4"
+    shape = {"dsv3": W.DSV3_INT4, "dsv3_mxfp4": W.DSV3_MXFP4, "dsv3_nvfp4": W.DSV3_NVFP4}[args.workload] if dsv3 else W.QWEN3_30B
     RHO, ALPHA = (0.9, 1.2) if dsv3 else (0.8, 1.1)
     L = (4 if args.layers == 48 else args.layers) if dsv3 else args.layers
     E, k, d = shape.n_experts, shape.top_k, shape.d
@@ -218,7 +219,7 @@ def run_ours(args):
         cfg = Bd.make_config(hidden=d, inter=shape.inter, n_experts=E, top_k=k, n_layers=L, slots_per_layer=Ns,
                              max_tokens=max(B, 8), host_pool_ptr=pool.ptr.value, host_pool_bytes=pool.n_bytes,
                              fill_mode=fill_mode, device=local,
-                             wdtype={"int4": Bd.FT_W_INT4_G128, "mxfp4": Bd.FT_W_MXFP4, "bf16": Bd.FT_W_BF16}[shape.wdtype],
+                             wdtype={"int4": Bd.FT_W_INT4_G128, "mxfp4": Bd.FT_W_MXFP4, "nvfp4": Bd.FT_W_NVFP4, "bf16": Bd.FT_W_BF16}[shape.wdtype],
                              n_shared=shape.n_shared, shared_ptr=None if shared is None else shared.data_ptr(),
                              global_pool=args.global_pool, **bw)
         return Bd.FtMoe(cfg)
@@ -495,10 +496,10 @@ def run_ours(args):
         line = {
             "metric": "moe_decode_tok_per_s", "value": value, "unit": "tok/s", "n_gpus": world, "steps": K,
             "warmup": Wn, "ms_per_step": main["ms"] / K, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": ("mxfp4 weights, bf16 activations, fp32 accumulate" if mxfp4 else
+            "vs_baseline": None, "dtype": (fp4_name + " weights, bf16 activations, fp32 accumulate" if mxfp4 else
                                          "int4 weights, bf16 activations, fp32 accumulate") if dsv3 else "bf16",
             "data": "synthetic",
-            "config": {"workload": ("decode DeepSeek-V3-shaped mxfp4 MoE stack (config 3 shapes)" if mxfp4 else
+            "config": {"workload": ("decode DeepSeek-V3-shaped " + fp4_name + " MoE stack (config 3 shapes)" if mxfp4 else
                                     "decode DeepSeek-V3-shaped int4 MoE stack (config 3)" if dsv3 else
                                     "decode Qwen3-30B-A3B-shaped MoE stack (config 1)"), "batch": B, "layers": L,
                        "hidden": d, "experts": E, "inter": shape.inter, "top_k": k, "slots_per_layer": Ns,
@@ -611,7 +612,7 @@ def prefill_passes(args, dev, L, cal=None, shape=None, Ns=None):
     common = dict(hidden=d, inter=I, n_experts=E, top_k=k, n_layers=L, slots_per_layer=Ns, max_tokens=T,
                   host_pool_ptr=pool.ptr.value, host_pool_bytes=pool.n_bytes,
                   fill_mode=Bd.FT_FILL_SM if args.fill == "sm" else Bd.FT_FILL_COPY_ENGINE,
-                  wdtype={"int4": Bd.FT_W_INT4_G128, "mxfp4": Bd.FT_W_MXFP4, "bf16": Bd.FT_W_BF16}[shape.wdtype],
+                  wdtype={"int4": Bd.FT_W_INT4_G128, "mxfp4": Bd.FT_W_MXFP4, "nvfp4": Bd.FT_W_NVFP4, "bf16": Bd.FT_W_BF16}[shape.wdtype],
                   gemm_min_tokens=args.gemm_min_tokens)
     if shape.n_shared:
         shared = W.make_shared_records(shape, L, SEED, device=dev)
@@ -800,7 +801,7 @@ def sub_int4(args, dev, cal, wdtype="int4"):
     import torch
     from paper_2608_16157_b200 import binding as Bd
     from paper_2608_16157_b200 import workload as W
-    shape = W.DSV3_INT4 if wdtype == "int4" else W.DSV3_MXFP4
+    shape = {"int4": W.DSV3_INT4, "mxfp4": W.DSV3_MXFP4, "nvfp4": W.DSV3_NVFP4}[wdtype]
     L, E, k, d, B, Ns = 4, shape.n_experts, shape.top_k, shape.d, 4, 64
     S = shape.expert_bytes
     warm, K = 48, 16
@@ -810,7 +811,7 @@ def sub_int4(args, dev, cal, wdtype="int4"):
     moe = Bd.FtMoe(Bd.make_config(hidden=d, inter=shape.inter, n_experts=E, top_k=k, n_layers=L, slots_per_layer=Ns,
                                   max_tokens=8, host_pool_ptr=pool.ptr.value, host_pool_bytes=pool.n_bytes,
                                   fill_mode=Bd.FT_FILL_SM,
-                                  wdtype=Bd.FT_W_INT4_G128 if wdtype == "int4" else Bd.FT_W_MXFP4, n_shared=1,
+                                  wdtype={"int4": Bd.FT_W_INT4_G128, "mxfp4": Bd.FT_W_MXFP4, "nvfp4": Bd.FT_W_NVFP4}[wdtype], n_shared=1,
                                   shared_ptr=shared.data_ptr(), bw_fill=max(cal["fill_MBps"], 1),
                                   bw_zc=max(cal["zc_MBps"], 1), bw_zc_residual=0, bw_hbm=max(cal["hbm_MBps"], 1)))
     stream = torch.cuda.current_stream()
@@ -877,10 +878,11 @@ def sub_int4(args, dev, cal, wdtype="int4"):
     t0_us, nb0 = statistics.median(us[0][1:]), sum(nbytes[0][1:]) / len(nbytes[0][1:])
     gbps0 = nb0 / (t0_us * 1e-6) / 1e9
     return {"config": "decode, config 3: d=7168, 256 %s experts + 1 shared, I=2048, top-8, 4 layers, 64 slots "
-                      "per layer, batch 4, rho 0.9, alpha 1.2" % ("int4-g128" if wdtype == "int4" else "mxfp4"),
-            "kernels": "w4_gateup_kernel + w4_down_kernel" if wdtype == "int4" else "mx4_gateup_kernel + mx4_down_kernel",
-            "bound": "hbm" if wdtype == "int4" else "alu (logic pipe: 7 instructions per 8 weights plus a scale per MMA); "
-                     "reported against the HBM peak",
+                      "per layer, batch 4, rho 0.9, alpha 1.2" % ("int4-g128" if wdtype == "int4" else wdtype),
+            "kernels": "w4_gateup_kernel + w4_down_kernel" if wdtype == "int4" else
+                       "mx4_gateup_kernel + mx4_down_kernel" + (" (NVFP4 instances)" if wdtype == "nvfp4" else ""),
+            "bound": "hbm" if wdtype == "int4" else "alu (logic pipe: 7 instructions per 8 weights plus a scale per MMA"
+                     + (", one K=16 MMA per 16-element scale block" if wdtype == "nvfp4" else "") + "); reported against the HBM peak",
             "tok_per_s": B * K / (ms * 1e-3), "ms_per_step": ms / K,
             "fills_per_step": (st1["fills"] - st0["fills"]) / K, "cache_warm_steps": warm,
             "GBps": gbps, "frac": gbps / hbm_peak, "peak": hbm_peak, "peak_source": peak_kind,
@@ -897,7 +899,12 @@ def sub_mxfp4(args, dev, cal):
     return sub_int4(args, dev, cal, "mxfp4")
 
 
-SUBRECORDS = {"int4": sub_int4, "mxfp4": sub_mxfp4, "prefill": sub_prefill, "prefill_mxfp4": sub_prefill_mxfp4}
+def sub_nvfp4(args, dev, cal):
+    return sub_int4(args, dev, cal, "nvfp4")
+
+
+SUBRECORDS = {"int4": sub_int4, "mxfp4": sub_mxfp4, "nvfp4": sub_nvfp4, "prefill": sub_prefill,
+              "prefill_mxfp4": sub_prefill_mxfp4}
 
 
 def run_sweep(args):
@@ -997,7 +1004,7 @@ def main():
     ap.add_argument("--sweep-batches", default="1,16,64")
     ap.add_argument("--global-pool", type=int, default=0, help="1: one slot pool and LRU clock shared by all layers")
     ap.add_argument("--graph", type=int, default=1, help="replay each decode step as one CUDA graph (SM fill only)")
-    ap.add_argument("--workload", default="qwen", choices=["qwen", "dsv3", "dsv3_mxfp4"])
+    ap.add_argument("--workload", default="qwen", choices=["qwen", "dsv3", "dsv3_mxfp4", "dsv3_nvfp4"])
     ap.add_argument("--mode", default="decode", choices=["decode", "prefill", "sweep"])
     ap.add_argument("--tokens", type=int, default=4096)
     ap.add_argument("--gemm-min-tokens", type=int, default=32)
@@ -1017,7 +1024,7 @@ def main():
     ap.add_argument("--only-batch", action="store_true")
     ap.add_argument("--cache-warm-steps", type=int, default=64,
                     help="untimed steps from the empty cache before warm-up and timing (steady-state headline)")
-    ap.add_argument("--sub", default="int4,mxfp4,prefill,prefill_mxfp4", help="bounded sub-records added to the decode line (N=1 only)")
+    ap.add_argument("--sub", default="int4,mxfp4,nvfp4,prefill,prefill_mxfp4", help="bounded sub-records added to the decode line (N=1 only)")
     ap.add_argument("--overlap", type=int, default=0,
                     help="launch mode of the streaming kernel in the timed region (ft_moe_set_launch_overlap)")
     args = ap.parse_args()

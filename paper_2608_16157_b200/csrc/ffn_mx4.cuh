@@ -1,5 +1,5 @@
 // Steps 5+6 for MXFP4 experts (e2m1 codes, one power-of-two scale byte per 32 elements of the contraction
-// dimension) at decode-sized token counts.  Same structure, work distribution and buffers as the int4 kernels of
+// dimension; paper Sec. 5.1) at decode-sized token counts.  Same structure, work distribution and buffers as the int4 kernels of
 // ffn_w4.cuh (every warp of the gate/up kernel streams its share of half-unit pieces; the down kernel walks chunks of 128
 // neurons x 1024 columns; weights go from global memory straight into registers); what differs is the arithmetic:
 //   * an e2m1 code is a 4-bit float, and placing its bits (s, e1 e0, m) at bits (7, 4 3, 2) of a byte gives the fp8
@@ -11,6 +11,10 @@
 //   * the bf16 activations of a (token, group of 128) are scaled to |a| <= 256 and split into two e4m3 numbers,
 //     a = hi + lo with lo the e4m3 rounding of a - hi (7-8 significant bits, like bf16, down to 2^-17 of the group's
 //     largest magnitude); both MMAs accumulate into the same registers.
+// NVFP4 experts (an unsigned e4m3 scale per 16 elements, a float32 scale per matrix) run through the same kernels
+// (template flag NV): their records keep the codes of one 16-element block in the even nibbles of a word row and
+// those of the next block in the odd nibbles, so that each block is one K = 16 fp8 MMA; the scale byte becomes a
+// float by a shift, a mask and a multiplication by 2^120.
 // The per-MMA scale multiplications and the seven-instruction unpack make these kernels bound by the logic pipe, not
 // by HBM (about half the rate of the int4 kernels); the hardware's own route for this format is the block-scaled
 // tcgen05 MMA, which reads packed fp4 and scale factors without any unpacking.
