@@ -278,6 +278,15 @@ def unpack_record(rec: np.ndarray, d: int, inter: int, wdtype: str):
                                              + (n%128)//16
       matrix scales (gate, up, down): three little-endian float32 at UA*I/16 + I*d/2 + I*d/16, then zeros up to
                                       256 bytes.
+    mxfp4tc record: the mxfp4 numbers (codes, one power-of-two scale byte per 32 elements of the contraction
+    dimension) stored as operand images of the block-scaled tensor-core instruction.  Section A: for each group of
+    128 neurons ng and each 128 hidden indices st a block of 17408 bytes = gate image (8192), up image (8192), gate
+    scales (512), up scales (512); section B: for each group of 128 output columns cg and each 128 neurons st a block
+    of 8704 bytes = image (8192), scales (512).  In an image, the code of (row r, contraction index 128*st + k),
+    k < 128, is a nibble (low when k is even) of byte 4096*(k//64) + 2048*((k%64)//32) + 128*(r//8) + 16*(r%8)
+    + (k%32)//2; the scale of (row r, block 4*st + b) is byte 16*(r%32) + 4*(r//32) + b of the 512.  Rows are neurons
+    (section A) or output columns (section B).
+      block of (ng, st):  17408*(ng*(d//128) + st);   block of (cg, st):  17408*(I//128)*(d//128) + 8704*(cg*(I//128) + st)
     """
     rec = np.ascontiguousarray(rec).view(np.uint8).reshape(-1)
     n = inter * d
@@ -361,6 +370,38 @@ def unpack_record(rec: np.ndarray, d: int, inter: int, wdtype: str):
         a_down = UA * U + ((((cb * NG + ng) * 8 + uu) * nwd + w) * 32 + 4 * g + q) * 16 + 4 * j + e // 2
         s_down = UA * U + inter * d // 2 + ((ng * CB + cb) * nwd + w) * 256 + 32 * g + 8 * j + 4 * half + (n % 128) // 32
         wd = fp4(a_down, e % 2 == 0) * pow2(s_down)
+        return wg, wu, wd
+    if wdtype == "mxfp4tc":
+        NG, KS = inter // 128, d // 128
+        assert rec.size == 3 * inter * d // 2 + 3 * inter * d // 32
+        magnitude = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
+
+        def fp4(addr, lo):
+            b = rec[addr].astype(np.int64)
+            c = np.where(lo, b & 0xF, b >> 4)
+            return np.where(c & 8, -1.0, 1.0) * magnitude[c & 7]
+
+        def pow2(addr):
+            return np.exp2(rec[addr].astype(np.float64) - 127.0)
+
+        def in_image(r, k):      # byte of (row r < 128, k < 128) in an 8192-byte image
+            return 4096 * (k // 64) + 2048 * ((k % 64) // 32) + 128 * (r // 8) + 16 * (r % 8) + (k % 32) // 2
+
+        def in_scales(r, b):
+            return 16 * (r % 32) + 4 * (r // 32) + b
+
+        i = np.arange(d, dtype=np.int64)[:, None]          # gate/up are returned [d, I]
+        nn = np.arange(inter, dtype=np.int64)[None, :]
+        blk = 17408 * ((nn // 128) * KS + i // 128)
+        lo = (i % 2 == 0) & (nn >= 0)
+        a_gate = blk + in_image(nn % 128, i % 128)
+        s_gate = blk + 16384 + in_scales(nn % 128, (i % 128) // 32)
+        wg = fp4(a_gate, lo) * pow2(s_gate)
+        wu = fp4(a_gate + 8192, lo) * pow2(s_gate + 512)
+        n = np.arange(inter, dtype=np.int64)[:, None]      # down is returned [I, d]
+        c = np.arange(d, dtype=np.int64)[None, :]
+        blk = 17408 * NG * KS + 8704 * ((c // 128) * NG + n // 128)
+        wd = fp4(blk + in_image(c % 128, n % 128), (n % 2 == 0) & (c >= 0)) * pow2(blk + 8192 + in_scales(c % 128, (n % 128) // 32))
         return wg, wu, wd
     if wdtype == "nvfp4":
         G, NG, U = d // GROUP, inter // GROUP, inter // 16

@@ -42,6 +42,13 @@ flattened identifier of Sec. 4.2 of the paper):
           C. order (ng, cb, w, g, j, half, m): per lane ``g`` 32 bytes = for each tile ``j`` and column half the four
              32-neuron blocks ``m`` of the 128-neuron group.
           ``S = 3*I*d/2 + 3*I*d/32``.
+``mxfp4tc`` the ``mxfp4`` numbers as operand images of the block-scaled tensor-core instruction (K-major core
+          matrices of 8 rows x 16 bytes, scale factors in groups of 128 rows x 4 blocks).  Section A: per (group of
+          128 neurons, 128 hidden indices) 17408 bytes = gate image, up image (8192 each), gate scales, up scales (512
+          each); section B: per (group of 128 output columns, 128 neurons) 8704 bytes = image, scales.  Byte of (row
+          ``r``, index ``k`` < 128) in an image: ``4096*(k//64) + 2048*((k%64)//32) + 128*(r//8) + 16*(r%8) +
+          (k%32)//2`` (low nibble = even ``k``); scale of (row ``r``, block ``b``): ``16*(r%32) + 4*(r//32) + b``.
+          ``S`` as for ``mxfp4``.
 ``nvfp4`` the same e2m1 codes with one unsigned e4m3 scale byte per block of 16 consecutive elements along the
           contraction dimension and one float32 scale per matrix.  Differences from ``mxfp4``:
           A. ``2304*G`` bytes per unit; in a gate/up tile row the code of hidden index ``128*grp + 32*j + 16*(e & 1)
@@ -78,7 +85,7 @@ class LayerShape:
     inter: int        # expert intermediate size I
     n_experts: int    # routed experts E
     top_k: int
-    wdtype: str = "bf16"   # "bf16" | "int4" | "mxfp4" | "nvfp4"
+    wdtype: str = "bf16"   # "bf16" | "int4" | "mxfp4" | "mxfp4tc" | "nvfp4"
     n_shared: int = 0      # always-resident shared experts (0 or 1)
 
     @property
@@ -89,7 +96,7 @@ class LayerShape:
             payload = 3 * self.inter * self.d // 2
             scales = (2 * self.inter * (self.d // GROUP) + (self.inter // GROUP) * self.d) * 2
             return payload + scales
-        if self.wdtype == "mxfp4":
+        if self.wdtype in ("mxfp4", "mxfp4tc"):
             return 3 * self.inter * self.d // 2 + 3 * self.inter * self.d // MX_BLOCK
         if self.wdtype == "nvfp4":
             return 3 * self.inter * self.d // 2 + 3 * self.inter * self.d // NV_BLOCK + NV_TAIL
@@ -101,6 +108,7 @@ TINY = LayerShape(d=256, inter=128, n_experts=8, top_k=2)
 QWEN3_30B = LayerShape(d=2048, inter=768, n_experts=128, top_k=8)
 DSV3_INT4 = LayerShape(d=7168, inter=2048, n_experts=256, top_k=8, wdtype="int4", n_shared=1)
 DSV3_MXFP4 = LayerShape(d=7168, inter=2048, n_experts=256, top_k=8, wdtype="mxfp4", n_shared=1)
+DSV3_MXFP4TC = LayerShape(d=7168, inter=2048, n_experts=256, top_k=8, wdtype="mxfp4tc", n_shared=1)
 DSV3_NVFP4 = LayerShape(d=7168, inter=2048, n_experts=256, top_k=8, wdtype="nvfp4", n_shared=1)
 
 
@@ -216,6 +224,26 @@ def _pack_mxfp4_record(cg, cu, cd, bg, bu, bd) -> torch.Tensor:
     ng2, cb2, w2, g2, j2, half, m = torch.meshgrid(ar(NG), ar(CB), ar(nwd), ar(8), ar(4), ar(2), ar(4), indexing="ij")
     sec_c = bd[4 * ng2 + m, cb2 * cbw + (4 * w2 + j2) * 16 + g2 + 8 * half].reshape(-1)
     return torch.cat([sec_a, sec_b, sec_c])
+
+
+def _pack_mxfp4tc_record(cg, cu, cd, bg, bu, bd) -> torch.Tensor:
+    """The inputs of ``_pack_mxfp4_record`` -> the record of operand images (see the module text), uint8 flat."""
+    I, d = cg.shape
+    NG, KS = I // 128, d // 128
+
+    def images(c, R, Kd):      # codes [R rows][Kd] -> [R/128][Kd/128][8192]
+        t = c.reshape(R // 128, 16, 8, Kd // 128, 2, 2, 16, 2)        # rg, r8, r, st, step, kcore, byte, nibble
+        t = t.permute(0, 3, 4, 5, 1, 2, 6, 7)                          # rg, st, step, kcore, r8, r, byte, nibble
+        return (t[..., 0] | (t[..., 1] << 4)).reshape(R // 128, Kd // 128, 8192)
+
+    def scales(b_, R, Kd):     # scale bytes [R][Kd/32] -> [R/128][Kd/128][512]: (r%32)*16 + (r//32)*4 + b
+        t = b_.reshape(R // 128, 4, 32, Kd // 128, 4)                  # rg, r//32, r%32, st, b
+        return t.permute(0, 3, 2, 1, 4).reshape(R // 128, Kd // 128, 512)
+
+    sec_a = torch.cat([images(cg, I, d), images(cu, I, d), scales(bg, I, d), scales(bu, I, d)], dim=2).reshape(-1)
+    # down: rows are output columns, the contraction index is the neuron
+    sec_b = torch.cat([images(cd.t().contiguous(), d, I), scales(bd.t().contiguous(), d, I)], dim=2).reshape(-1)
+    return torch.cat([sec_a, sec_b])
 
 
 def _e2m1_codes(v: torch.Tensor) -> torch.Tensor:
@@ -347,6 +375,11 @@ def make_records(shape: LayerShape, seed: int, layer: int, first: int, count: in
             cu, bu = _quantise_mxfp4(w[1], 1)
             cd, bd = _quantise_mxfp4(w[2], 0)
             out[j] = _pack_mxfp4_record(cg, cu, cd, bg, bu, bd)
+        elif shape.wdtype == "mxfp4tc":
+            cg, bg = _quantise_mxfp4(w[0], 1)
+            cu, bu = _quantise_mxfp4(w[1], 1)
+            cd, bd = _quantise_mxfp4(w[2], 0)
+            out[j] = _pack_mxfp4tc_record(cg, cu, cd, bg, bu, bd)
         elif shape.wdtype == "nvfp4":
             cg, bg, mg = _quantise_nvfp4(w[0], 1)
             cu, bu, mu = _quantise_nvfp4(w[1], 1)

@@ -309,6 +309,71 @@ def test_generated_nvfp4_pool_quantiser_error_bound():
     assert np.abs(wg.T - w[0]).mean() < np.abs(wg_mx.T - w[0]).mean()
 
 
+def _record_mxfp4tc_by_definition(cg, cu, cd, bg, bu, bd):
+    """The inputs of `_record_mxfp4_by_definition`, written as operand images block by block."""
+    I, d = cg.shape
+    out = bytearray()
+
+    def image(code_of):           # code_of(r, k): r < 128 rows, k < 128 contraction indices
+        for step in range(2):
+            for kcore in range(2):
+                for r8 in range(16):
+                    for r in range(8):
+                        for byte in range(16):
+                            k = 64 * step + 32 * kcore + 2 * byte
+                            yield (int(code_of(8 * r8 + r, k)) & 0xF) | ((int(code_of(8 * r8 + r, k + 1)) & 0xF) << 4)
+
+    def scale_atom(scale_of):     # scale_of(r, b): b < 4 blocks of 32
+        for r32 in range(32):
+            for rq in range(4):
+                for b in range(4):
+                    yield int(scale_of(32 * rq + r32, b))
+
+    for ng in range(I // 128):
+        for st in range(d // 128):
+            for c_ in (cg, cu):
+                out += bytes(image(lambda r, k: c_[128 * ng + r, 128 * st + k]))
+            for b_ in (bg, bu):
+                out += bytes(scale_atom(lambda r, b: b_[128 * ng + r, 4 * st + b]))
+    for cgp in range(d // 128):
+        for st in range(I // 128):
+            out += bytes(image(lambda r, k: cd[128 * st + k, 128 * cgp + r]))
+            out += bytes(scale_atom(lambda r, b: bd[4 * st + b, 128 * cgp + r]))
+    return np.frombuffer(bytes(out), dtype=np.uint8)
+
+
+def test_unpack_mxfp4tc_record_by_definition():
+    d, I = 256, 128
+    rng = np.random.default_rng(5)
+    cg, cu, cd = (rng.integers(0, 16, size=(I, d)) for _ in range(3))
+    bg = rng.integers(120, 131, size=(I, d // 32))
+    bu = rng.integers(110, 127, size=(I, d // 32))
+    bd = rng.integers(125, 135, size=(I // 32, d))
+    rec = _record_mxfp4tc_by_definition(cg, cu, cd, bg, bu, bd)
+    assert rec.size == W.LayerShape(d, I, 1, 1, "mxfp4tc").expert_bytes
+    wg, wu, wd = O.unpack_record(rec, d, I, "mxfp4tc")
+    val = np.array(FP4_VALUES)
+
+    def deq(c, b, axis):
+        return np.where(c & 8, -1.0, 1.0) * val[c & 7] * np.repeat(np.exp2(b.astype(np.float64) - 127), 32, axis=axis)
+
+    assert np.array_equal(wg, deq(cg, bg, 1).T)
+    assert np.array_equal(wu, deq(cu, bu, 1).T)
+    assert np.array_equal(wd, deq(cd, bd, 0))
+    # the same numbers in the register-fragment order of the mxfp4 record read back identically
+    wg2, wu2, wd2 = O.unpack_record(_record_mxfp4_by_definition(cg, cu, cd, bg, bu, bd), d, I, "mxfp4")
+    assert np.array_equal(wg, wg2) and np.array_equal(wu, wu2) and np.array_equal(wd, wd2)
+
+
+def test_generated_mxfp4tc_pool_equals_generated_mxfp4_pool():
+    """Both layouts are packed from the same quantiser output: the generator's records decode to the same weights."""
+    for d, I in ((256, 128), (512, 256)):
+        a = W.make_records(W.LayerShape(d, I, 2, 1, "mxfp4tc"), seed=3, layer=1, first=1, count=1)[0].numpy()
+        b = W.make_records(W.LayerShape(d, I, 2, 1, "mxfp4"), seed=3, layer=1, first=1, count=1)[0].numpy()
+        for x, y in zip(O.unpack_record(a, d, I, "mxfp4tc"), O.unpack_record(b, d, I, "mxfp4")):
+            assert np.array_equal(x, y) and np.count_nonzero(x) > x.size // 2
+
+
 def test_generated_mxfp4_pool_quantiser_error_bound():
     """The generator's records, read back by the oracle, are within half a grid step of the fp32 draws: the e2m1 grid
     step is at most 2 (between 4 and 6) times the block scale 2**(floor(log2(amax)) - 2), i.e. |w - deq| <= amax / 4."""
