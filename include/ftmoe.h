@@ -69,6 +69,17 @@
  *                   r+8.  Section C: order (ng, cb, w, g, j, half, m), i.e. per lane g 32 bytes = for each tile j and
  *                   column half the scales of the four 32-neuron blocks m of the 128-neuron group.
  *                   S = 3*inter*hidden/2 + 3*inter*hidden/32 bytes.  Shapes as for int4.
+ *   FT_W_MXFP4_TC : the numbers of FT_W_MXFP4 stored as operand images of the block-scaled tensor-core instruction
+ *                   (tcgen05.mma kind::mxf4: packed e2m1 operands in K-major core matrices of 8 rows x 16 bytes, scale
+ *                   factors in groups of 128 rows x 4 blocks), so that the decode kernels feed the record's bytes to
+ *                   the instruction as they are.  Section A: for each group of 128 neurons ng and each 128 hidden
+ *                   indices st (in that order) 17408 bytes = gate image (8192), up image (8192), gate scales (512), up
+ *                   scales (512).  Section B: for each group of 128 output columns cg and each 128 neurons st 8704
+ *                   bytes = image, scales.  In an image the code of (row r < 128, contraction index k < 128) is a
+ *                   nibble (low when k is even) of byte 4096*(k/64) + 2048*((k%64)/32) + 128*(r/8) + 16*(r%8) +
+ *                   (k%32)/2; the scale byte of (row r, block b < 4) is byte 16*(r%32) + 4*(r/32) + b.  Rows are
+ *                   neurons (A) or output columns (B).  S as for FT_W_MXFP4.  Decode-sized calls only: max_tokens
+ *                   <= 8 and gemm_min_tokens = 0, else FT_ERR_UNSUPPORTED.
  *   FT_W_NVFP4    : two-level scaled FP4 (paper Sec. 5.1, expert representations): the same e2m1 codes with one
  *                   unsigned e4m3 scale byte b (exponent field E = b >> 3, mantissa M = b & 7: 2^(E-7) * (1 + M/8),
  *                   or 2^-6 * M/8 when E = 0; b <= 0x7E) per 16 consecutive elements of the contraction dimension and
@@ -113,7 +124,7 @@ typedef enum {
   FT_ERR_UNSUPPORTED = 8
 } ft_status_t;
 
-typedef enum { FT_W_BF16 = 0, FT_W_INT4_G128 = 1, FT_W_MXFP4 = 2, FT_W_NVFP4 = 3 } ft_wdtype_t;
+typedef enum { FT_W_BF16 = 0, FT_W_INT4_G128 = 1, FT_W_MXFP4 = 2, FT_W_NVFP4 = 3, FT_W_MXFP4_TC = 4 } ft_wdtype_t;
 
 /* How ft_moe_fill moves records.  Both give byte-identical slots. */
 typedef enum {

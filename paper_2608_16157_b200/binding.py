@@ -15,7 +15,7 @@ from . import build as _build
 FT_OK = 0
 FT_ERR_INVALID_ARG, FT_ERR_NOT_PINNED, FT_ERR_OOM, FT_ERR_CUDA = 1, 2, 3, 4
 FT_ERR_STATE, FT_ERR_TIMEOUT, FT_ERR_NONFINITE, FT_ERR_UNSUPPORTED = 5, 6, 7, 8
-FT_W_BF16, FT_W_INT4_G128, FT_W_MXFP4, FT_W_NVFP4 = 0, 1, 2, 3
+FT_W_BF16, FT_W_INT4_G128, FT_W_MXFP4, FT_W_NVFP4, FT_W_MXFP4_TC = 0, 1, 2, 3, 4
 FT_FILL_COPY_ENGINE, FT_FILL_SM = 0, 1
 STAT_NAMES = ("steps", "routed", "hits", "misses", "fills", "zc", "evictions", "pairs", "pairs_resident",
               "pairs_gemm")

@@ -1,0 +1,623 @@
+// Steps 5+6 for MXFP4 experts stored as tensor-core operand images (FT_W_MXFP4_TC), decode-sized calls (T <= 8):
+// the block-scaled 5th-generation tensor-core instruction tcgen05.mma kind::mxf4 multiplies packed e2m1 weights by
+// e2m1 activations, both with one power-of-two scale per 32 elements held in tensor memory, so the weights need no
+// unpacking at all: a record's bytes go from HBM (or, for zero-copy experts, from the mapped host pool) to shared
+// memory by bulk copies and are consumed there by the instruction (paper Sec. 5.1 expert representations; Sec. 3.2
+// grouped evaluation of the resident and the zero-copy experts).
+//   * Activations keep their precision by bit slicing along N: a (token, block of 32) is written as a sum of
+//     kTcTerms block-scaled e2m1 vectors, term i being the e2m1 rounding of what the terms before it left over,
+//     each with its own scale (the smallest power of two that brings the leftover's largest magnitude to <= 6).
+//     Every term removes at least a factor 3 of the block's largest leftover, so 6 terms leave <= 2^-9.5 of the
+//     block's largest magnitude; the terms of the 8 tokens are the N = 48 columns of the MMA (column 8 i + token),
+//     and the epilogue adds a token's 6 columns.  The tensor pipe has room for this: the kernels are HBM-bound.
+//   * Gate/up kernel: M = 128 neurons of the gate and of the up matrix per tile, K split into two halves (a CTA
+//     keeps the activation image of one half in shared memory: CTAs of even index the first half, of odd index the
+//     second), each CTA an equal share of (tile, 128-index stage) steps of its half.  One producer thread issues the
+//     bulk copies (17408 bytes per stage: gate image, up image, gate scales, up scales) into a ring, one thread
+//     copies the stage's scale factors to tensor memory (tcgen05.cp) and issues the four MMAs, four warps read the
+//     accumulators of a finished tile (tcgen05.ld), add a token's terms and add the partial sums into the per-unit
+//     fp32 accumulators in global memory; the CTA whose contribution completes a group of 128 neurons applies
+//     SiLU(gate) * up and writes the group's h as the bit-sliced activation image of the down kernel.
+//   * Down kernel: M = 128 output columns per tile, K = the neurons; same ring; the epilogue multiplies by the gate
+//     weight and adds into the fp32 output accumulator; the last CTA rounds it to bf16.
+// Every mbarrier wait is bounded (see async.cuh); a CTA whose wait runs out latches the timeout status, stops
+// issuing work, lets its copies in flight land, frees its tensor memory and returns.
+#pragma once
+#include "async.cuh"
+#include "ffn_w4.cuh"
+#include "gemm_tc.cuh"
+
+namespace ftmoe {
+
+constexpr int kTcTerms = 6;                 // e2m1 terms per activation
+constexpr int kTcN = 8 * kTcTerms;          // MMA columns: 8 tokens x terms
+constexpr uint32_t kTcStepB = kTcN * 32u;   // bytes of the activation image of one K = 64 step
+constexpr uint32_t kTcStageA = 17408u;      // gate/up stage: two images of 8192 bytes, two scale atoms of 512
+constexpr uint32_t kTcStageD = 8704u;       // down stage: one image, one scale atom
+constexpr int kTcThreads = 192;             // warp 0: producer, warp 1: MMA issuer, warps 2..5: epilogue
+constexpr int kTcMaxStages = 16;
+constexpr size_t kTcSmem = 232448 - 1024;   // dynamic shared memory the two kernels may use (1 KiB left for static data)
+
+// Activation images in global memory (written by tc_quant_x_kernel / by the gate/up kernel's group conversion).
+// Gate/up operand: for each K half: [d/128 steps][kTcStepB] then [d/256 scale atoms][512].
+__host__ __device__ inline size_t tc_x_half_bytes(int d) { return (size_t)(d / 128) * kTcStepB + (size_t)(d / 256) * 512; }
+// Down operand of one pass: [inter/64 steps][kTcStepB] then [inter/128 scale atoms][512].
+__host__ __device__ inline size_t tc_h_pass_bytes(int inter) { return (size_t)(inter / 64) * kTcStepB + (size_t)(inter / 128) * 512; }
+
+// e2m1 rounding of v in [0, 6] (nearest, ties away from zero on the magnitude): value and 3-bit code.
+__device__ __forceinline__ void tc_e2m1(float v, float &val, uint32_t &code) {
+  v = fminf(v, 6.f);
+  if (v < 1.f) {
+    val = 0.5f * rintf(2.f * v);
+  } else {
+    val = __uint_as_float((__float_as_uint(v) + 0x00200000u) & 0xFFC00000u);   // keep one mantissa bit
+    val = fminf(val, 6.f);
+  }
+  if (val < 1.f) {
+    code = val == 0.5f ? 1u : 0u;
+  } else {
+    const uint32_t b = __float_as_uint(val);
+    code = (((b >> 23) - 126u) << 1) | ((b >> 22) & 1u);
+  }
+}
+
+// One bit-slicing term of 8 values held by each of the 4 lanes of a quad (the quad = one block of 32): returns the 8
+// codes (nibble e = element e) and the scale byte, and subtracts the term from r[].  bad: a non-finite input.
+__device__ __forceinline__ void tc_term(float (&r)[8], bool bad, uint32_t &codes, uint32_t &scale_byte) {
+  float m = 0.f;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) m = fmaxf(m, fabsf(r[e]));
+  m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+  m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+  codes = 0u;
+  if (bad) { scale_byte = 255u; return; }           // the scale format's NaN: the token's outputs become NaN
+  if (m < 1e-37f) { scale_byte = 127u; return; }    // nothing left: zeros
+  const uint32_t tb = __float_as_uint(m * (1.f / 6.f));
+  uint32_t ex = (tb >> 23) + ((tb & 0x007FFFFFu) ? 1u : 0u);   // smallest power of two >= m / 6
+  ex = min(max(ex, 1u), 253u);
+  scale_byte = ex;
+  const float scale = __uint_as_float(ex << 23), inv = __uint_as_float((254u - ex) << 23);
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    float val;
+    uint32_t c;
+    tc_e2m1(fabsf(r[e]) * inv, val, c);
+    if (r[e] < 0.f) { val = -val; c |= 8u; }
+    r[e] -= val * scale;
+    codes |= c << (4 * e);
+  }
+}
+
+// x [T][d] bf16 -> the gate/up kernel's activation images of both K halves.  One thread per 8 consecutive hidden
+// indices of a token slot (slots >= T are written as zeros); a quad of lanes is one block of 32.
+struct TcQuantParams {
+  const __nv_bfloat16 *x;
+  uint8_t *xq;      // [2 halves][tc_x_half_bytes(d)]
+  int T, d;
+};
+__global__ void __launch_bounds__(256) tc_quant_x_kernel(TcQuantParams p) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int per_tok = p.d / 8;
+  const int i = blockIdx.x * 256 + threadIdx.x;
+  if (i >= 8 * per_tok) return;
+  const int tok = i / per_tok, c8 = i - tok * per_tok;   // hidden indices 8 c8 .. 8 c8 + 7
+  float r[8];
+  bool bad = false;
+  if (tok < p.T) {
+    const uint4 v = *reinterpret_cast<const uint4 *>(p.x + (size_t)tok * p.d + 8 * c8);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      r[2 * e] = __uint_as_float(w[e] << 16);
+      r[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) bad |= !(fabsf(r[e]) <= 3.0e38f);
+  } else {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) r[e] = 0.f;
+  }
+  bad = (__shfl_xor_sync(0xffffffffu, (int)bad, 1) | __shfl_xor_sync(0xffffffffu, (int)bad, 2) | (int)bad) != 0;
+  const int half_k = p.d / 2;
+  const int k = 8 * c8, half = k >= half_k ? 1 : 0, kk = k - half * half_k;
+  uint8_t *img = p.xq + (size_t)half * tc_x_half_bytes(p.d);
+  uint8_t *sf = img + (size_t)(p.d / 128) * kTcStepB;
+  const int step = kk >> 6, kcore = (kk >> 5) & 1, word = (kk & 31) >> 3;
+#pragma unroll
+  for (int t = 0; t < kTcTerms; ++t) {
+    uint32_t codes, sb;
+    tc_term(r, bad, codes, sb);
+    *reinterpret_cast<uint32_t *>(img + (size_t)step * kTcStepB + kcore * (kTcN * 16) + t * 128 + tok * 16 + word * 4) = codes;
+    if ((threadIdx.x & 3) == 0) {
+      const int n = 8 * t + tok, blk = kk >> 5;   // scale of (column n, block blk of the half)
+      sf[(size_t)(blk >> 2) * 512 + (n & 31) * 16 + (n >> 5) * 4 + (blk & 3)] = (uint8_t)sb;
+    }
+  }
+}
+
+
+struct TcParams {
+  W4Params w;          // the work lists, the hand-over buffers (hraw, hcount, hq) and the output, as for the other 4-bit kernels
+  const uint8_t *xq;   // activation images of the two K halves (tc_quant_x_kernel)
+  int d;
+  int n_stages;        // ring stages (what fits in shared memory, at most kTcMaxStages)
+};
+
+// ---- PTX wrappers of the block-scaled path ----
+__device__ __forceinline__ uint64_t tc_desc(uint32_t smem_addr, uint32_t lbo, uint32_t sbo) {
+  return umma_desc(smem_addr, lbo, sbo, 0);   // K-major core matrices of 8 rows x 16 bytes, no swizzle
+}
+__device__ __forceinline__ void tc_cp_scales(uint32_t tmem_col, uint32_t smem_addr) {
+  // 32 rows x 16 bytes -> lanes 0..31 x 4 columns, repeated for the four lane quarters
+  asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(tmem_col), "l"(tc_desc(smem_addr, 0, 128)) : "memory");
+}
+// D[128 x kTcN] (+)= A[128 x 64] * B[kTcN x 64]^T, e2m1 operands, one ue8m0 scale per 32 elements; sf_id = 0 or 2:
+// which two of a scale word's four bytes belong to this K step.
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t sf_id, uint32_t sfa,
+                                       uint32_t sfb, uint32_t accumulate) {
+  const uint32_t idesc = (sf_id << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTcN >> 3) << 17) | (1u << 23) |
+                         ((128u >> 4) << 24) | (sf_id << 29);
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%6], p;\n}\n" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa | (sf_id << 30)), "r"(sfb | (sf_id << 30))
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+}
+// The kTcN columns of this thread's accumulator row -> one sum per token.
+__device__ __forceinline__ void tc_row_sums(uint32_t taddr, float (&v)[8]) {
+#pragma unroll
+  for (int t = 0; t < 8; ++t) v[t] = 0.f;
+#pragma unroll
+  for (int c = 0; c < kTcN; c += 16) {
+    uint32_t r[16];
+    tmem_ld16(taddr + c, r);
+    tmem_ld_wait();
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v[j & 7] += __uint_as_float(r[j]);
+  }
+}
+__device__ __forceinline__ void tc_epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// Shared memory of the gate/up kernel: activation image of the K half | its scale atoms | ring | barriers | flags |
+// items | pref.
+inline size_t tc_gateup_fixed_bytes(int max_items, int d) {
+  return tc_x_half_bytes(d) + 64 * 8 + 64 + (size_t)max_items * sizeof(WorkItem) + ((size_t)max_items + 1) * 4 + 128;
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
+  const W4Params &p = q.w;
+  const int d = q.d, NS = q.n_stages;
+  const uint32_t KS = (uint32_t)d / 128u, SPH = KS / 2u;          // stages of a tile; of a K half
+  const uint32_t NG = (uint32_t)p.inter / 128u, NBLK = (uint32_t)p.inter / 16u;
+  extern __shared__ __align__(128) unsigned char smem[];
+  unsigned char *s_b = smem;                                        // [2 SPH steps][kTcStepB]
+  unsigned char *s_sfb = s_b + (size_t)2 * SPH * kTcStepB;          // [SPH][512]
+  unsigned char *s_ring = s_sfb + (size_t)SPH * 512;
+  uint64_t *s_bar = reinterpret_cast<uint64_t *>(s_ring + (size_t)NS * kTcStageA);
+  uint32_t *s_tmem = reinterpret_cast<uint32_t *>(s_bar + 64);
+  volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
+  volatile int *s_last = s_abort + 1;
+  WorkItem *s_items = reinterpret_cast<WorkItem *>(s_tmem + 16);
+  int32_t *s_pref = reinterpret_cast<int32_t *>(s_items + p.max_items);
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const uint32_t bar0 = smem_u32(s_bar);
+  auto full_bar = [&](uint32_t s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](uint32_t s) { return bar0 + 8u * (kTcMaxStages + s); };
+  auto tfull_bar = [&](uint32_t b) { return bar0 + 8u * (2 * kTcMaxStages + b); };
+  auto tempty_bar = [&](uint32_t b) { return bar0 + 8u * (2 * kTcMaxStages + 2 + b); };
+  const uint32_t x_bar = bar0 + 8u * (2 * kTcMaxStages + 4);
+  if (tid == 0) {
+    for (int s = 0; s < NS; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+    mbar_init(x_bar, 1);
+    *s_abort = 0;
+    *s_last = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  const int n_items = *p.n_items, n_zc = *p.n_zc;
+  for (int i = tid; i <= p.max_items; i += kTcThreads) s_pref[i] = p.pref[i];
+  {
+    const uint4 *src = reinterpret_cast<const uint4 *>(p.items);
+    uint4 *dst = reinterpret_cast<uint4 *>(s_items);
+    for (int i = tid; i < 2 * p.max_items; i += kTcThreads) dst[i] = src[i];
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(s_tmem)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *s_tmem;
+  const uint32_t t_sfa = tmem + 256u, t_sfb = tmem + 384u;
+
+  // this CTA's share: CTAs of even index work on the first K half, of odd index on the second; within a half and
+  // within each of the two pass ranges (resident passes, then zero-copy passes) an equal number of stages per CTA
+  const uint32_t half = blockIdx.x & 1u, ci = blockIdx.x >> 1, nc = gridDim.x >> 1;
+  uint32_t pass0[2], s_begin[2], s_end[2];
+  pass0[0] = 0u;
+  pass0[1] = (uint32_t)s_pref[n_items];
+  {
+    const uint32_t np0 = pass0[1], np1 = (uint32_t)s_pref[n_items + n_zc] - pass0[1];
+    const uint32_t t0 = np0 * NG * SPH, t1 = np1 * NG * SPH;
+    s_begin[0] = w4_first(t0, nc, ci); s_end[0] = w4_first(t0, nc, ci + 1);
+    s_begin[1] = w4_first(t1, nc, ci); s_end[1] = w4_first(t1, nc, ci + 1);
+  }
+  // body(pass, ng, st0, n): a run of n stages, starting at stage st0 of the half, of tile (pass, ng)
+  auto walk = [&](auto body) {
+    for (int r = 0; r < 2; ++r)
+      for (uint32_t s = s_begin[r]; s < s_end[r];) {
+        const uint32_t tile = s / SPH, st0 = s - tile * SPH, n = min(SPH - st0, s_end[r] - s);
+        if (!body(pass0[r] + tile / NG, tile % NG, st0, n)) return;
+        s += n;
+      }
+  };
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ---- producer: the weights do not depend on the preceding kernels; the activation image does ----
+      uint32_t it = 0;
+      bool x_sent = false;
+      auto send_x = [&]() {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        const uint32_t bytes = (uint32_t)tc_x_half_bytes(d);
+        mbar_expect_tx(x_bar, bytes);
+        const uint8_t *src = q.xq + (size_t)half * bytes;
+        for (uint32_t o = 0; o < bytes; o += 16384u) bulk_g2s(smem_u32(s_b) + o, src + o, min(16384u, bytes - o), x_bar);
+        x_sent = true;
+      };
+      walk([&](uint32_t pass, uint32_t ng, uint32_t st0, uint32_t n) {
+        const uint8_t *rec = s_items[w4_find_item(s_pref, n_items + n_zc, pass)].w;
+        const uint8_t *src = rec + ((size_t)ng * KS + half * SPH + st0) * kTcStageA;
+        for (uint32_t s = 0; s < n; ++s, ++it) {
+          const uint32_t slot = it % (uint32_t)NS;
+          if (!mbar_wait(empty_bar(slot), ((it / (uint32_t)NS) & 1u) ^ 1u, s_abort, p.status)) return false;
+          mbar_expect_tx(full_bar(slot), kTcStageA);
+          bulk_g2s(smem_u32(s_ring) + slot * kTcStageA, src + (size_t)s * kTcStageA, kTcStageA, full_bar(slot));
+          if (!x_sent && it + 1 == (uint32_t)NS) send_x();   // after the first ring fill
+        }
+        return true;
+      });
+      if (!x_sent) send_x();
+      // the copies issued must have landed before this CTA's shared memory is released
+      for (uint32_t k = it > (uint32_t)NS ? it - (uint32_t)NS : 0u; k < it; ++k)
+        (void)mbar_wait(full_bar(k % (uint32_t)NS), (k / (uint32_t)NS) & 1u, s_abort, p.status);
+      (void)mbar_wait(x_bar, 0u, s_abort, p.status);
+      abort_drain(s_abort);
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ---- MMA issuer ----
+      bool ok = mbar_wait(x_bar, 0u, s_abort, p.status);
+      if (ok) {
+        tc_fence_after();
+        for (uint32_t a = 0; a < SPH; ++a) tc_cp_scales(t_sfb + 4u * a, smem_u32(s_sfb) + a * 512u);
+      }
+      uint32_t it = 0, seg = 0;
+      if (ok)
+        walk([&](uint32_t, uint32_t, uint32_t st0, uint32_t n) {
+          const uint32_t buf = seg & 1u;
+          if (!mbar_wait(tempty_bar(buf), ((seg >> 1) & 1u) ^ 1u, s_abort, p.status)) return false;
+          tc_fence_after();
+          const uint32_t dg = tmem + buf * 128u, du = dg + 64u;
+          for (uint32_t s = 0; s < n; ++s, ++it) {
+            const uint32_t slot = it % (uint32_t)NS;
+            if (!mbar_wait(full_bar(slot), (it / (uint32_t)NS) & 1u, s_abort, p.status)) return false;
+            tc_fence_after();
+            const uint32_t st = smem_u32(s_ring) + slot * kTcStageA;
+            tc_cp_scales(t_sfa + slot * 8u, st + 16384u);
+            tc_cp_scales(t_sfa + slot * 8u + 4u, st + 16896u);
+#pragma unroll
+            for (uint32_t step = 0; step < 2; ++step) {
+              const uint64_t bd = tc_desc(smem_u32(s_b) + ((st0 + s) * 2u + step) * kTcStepB, kTcN * 16u, 128u);
+              const uint32_t sfb = t_sfb + 4u * (st0 + s), acc = (s | step) ? 1u : 0u;
+              tc_mma(dg, tc_desc(st + step * 4096u, 2048u, 128u), bd, 2u * step, t_sfa + slot * 8u, sfb, acc);
+              tc_mma(du, tc_desc(st + 8192u + step * 4096u, 2048u, 128u), bd, 2u * step, t_sfa + slot * 8u + 4u, sfb, acc);
+            }
+            umma_commit(empty_bar(slot));   // the stage may be refilled once these MMAs have read it
+          }
+          umma_commit(tfull_bar(buf));
+          ++seg;
+          return true;
+        });
+    }
+  } else {
+    // ---- epilogue: thread = accumulator row (neuron of the tile) ----
+    const int ew = warp & 3, row = ew * 32 + lane, et = (warp - 2) * 32 + lane;
+    uint32_t seg = 0;
+    walk([&](uint32_t pass, uint32_t ng, uint32_t, uint32_t n) {
+      const uint32_t buf = seg & 1u;
+      bool ok = true;
+      if (lane == 0) ok = mbar_wait(tfull_bar(buf), (seg >> 1) & 1u, s_abort, p.status);
+      ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+      if (ok) {
+        tc_fence_after();
+        const uint32_t trow = tmem + buf * 128u + ((uint32_t)(ew * 32) << 16);
+        float gsum[8], usum[8];
+        tc_row_sums(trow, gsum);
+        tc_row_sums(trow + 64u, usum);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar(buf));
+        float *hacc = p.hraw + ((size_t)pass * NBLK + 8u * ng + (uint32_t)(row >> 4)) * 256 + (row & 15);
+        for (int t = 0; t < p.T; ++t) {
+          red_add_f32(hacc + t * 16, gsum[t]);
+          red_add_f32(hacc + 128 + t * 16, usum[t]);
+        }
+        __threadfence();
+      }
+      tc_epi_barrier();
+      if (et == 0 && !*s_abort) {
+        const int old = atomicAdd(p.hcount + pass * NG + ng, (int)n);
+        *s_last = (old + (int)n == (int)KS) ? 1 : 0;
+      }
+      tc_epi_barrier();
+      if (*s_abort) return false;
+      if (*s_last) {
+        // this CTA's stages completed the group: h = SiLU(gate) * up, bit-sliced into the down kernel's operand
+        __threadfence();
+        const int tok = et >> 4, sub = et & 15;   // 8 neurons 8 sub .. 8 sub + 7 of the group, one token
+        float *src = p.hraw + ((size_t)pass * NBLK + 8u * ng + (uint32_t)(sub >> 1)) * 256 + tok * 16 + (sub & 1) * 8;
+        float h[8];
+#pragma unroll
+        for (int k4 = 0; k4 < 2; ++k4) {
+          float4 *pg = reinterpret_cast<float4 *>(src) + k4, *pu = reinterpret_cast<float4 *>(src + 128) + k4;
+          const float4 a = __ldcg(pg), b = __ldcg(pu);
+          __stcg(pg, make_float4(0.f, 0.f, 0.f, 0.f));   // the sums start from zero in the next call
+          __stcg(pu, make_float4(0.f, 0.f, 0.f, 0.f));
+          h[4 * k4] = __fdividef(a.x, 1.f + __expf(-a.x)) * b.x;
+          h[4 * k4 + 1] = __fdividef(a.y, 1.f + __expf(-a.y)) * b.y;
+          h[4 * k4 + 2] = __fdividef(a.z, 1.f + __expf(-a.z)) * b.z;
+          h[4 * k4 + 3] = __fdividef(a.w, 1.f + __expf(-a.w)) * b.w;
+        }
+        bool bad = false;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) bad |= !(fabsf(h[e]) <= 3.0e38f);
+        bad = (__shfl_xor_sync(0xffffffffu, (int)bad, 1) | __shfl_xor_sync(0xffffffffu, (int)bad, 2) | (int)bad) != 0;
+        uint8_t *img = p.hq + (size_t)pass * tc_h_pass_bytes(p.inter);
+        uint8_t *sf = img + (size_t)(p.inter / 64) * kTcStepB + (size_t)ng * 512;
+        uint8_t *dst = img + (size_t)(2u * ng + (uint32_t)(sub >> 3)) * kTcStepB + ((sub >> 2) & 1) * (kTcN * 16) + tok * 16 + (sub & 3) * 4;
+#pragma unroll
+        for (int t = 0; t < kTcTerms; ++t) {
+          uint32_t codes, sb;
+          tc_term(h, bad, codes, sb);
+          *reinterpret_cast<uint32_t *>(dst + t * 128) = codes;
+          if ((sub & 3) == 0) {
+            const int nn = 8 * t + tok;
+            sf[(nn & 31) * 16 + (nn >> 5) * 4 + (sub >> 2)] = (uint8_t)sb;
+          }
+        }
+        if (et == 0) p.hcount[pass * NG + ng] = 0;
+      }
+      ++seg;
+      return true;
+    });
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+}
+
+
+// Shared memory of the down kernel: activation image of the current pass and its scale atoms | ring | barriers |
+// flags | items | pref.
+inline size_t tc_down_fixed_bytes(int max_items, int inter) {
+  return tc_h_pass_bytes(inter) + 64 * 8 + 64 + (size_t)max_items * sizeof(WorkItem) + ((size_t)max_items + 1) * 4 + 128;
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
+  const W4Params &p = q.w;
+  const int d = q.d, NS = q.n_stages;
+  const uint32_t DS = (uint32_t)p.inter / 128u;        // stages (and scale atoms) of a tile
+  const uint32_t CG = (uint32_t)d / 128u, NG = (uint32_t)p.inter / 128u, KSA = (uint32_t)d / 128u;
+  const uint32_t h_bytes = (uint32_t)tc_h_pass_bytes(p.inter);
+  extern __shared__ __align__(128) unsigned char smem[];
+  unsigned char *s_b = smem;                                        // [2 DS steps][kTcStepB] | [DS][512]
+  unsigned char *s_ring = s_b + h_bytes;
+  uint64_t *s_bar = reinterpret_cast<uint64_t *>(s_ring + (size_t)NS * kTcStageD);
+  uint32_t *s_tmem = reinterpret_cast<uint32_t *>(s_bar + 64);
+  volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
+  WorkItem *s_items = reinterpret_cast<WorkItem *>(s_tmem + 16);
+  int32_t *s_pref = reinterpret_cast<int32_t *>(s_items + p.max_items);
+  __shared__ int s_final;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t bar0 = smem_u32(s_bar);
+  auto full_bar = [&](uint32_t s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](uint32_t s) { return bar0 + 8u * (kTcMaxStages + s); };
+  auto tfull_bar = [&](uint32_t b) { return bar0 + 8u * (2 * kTcMaxStages + b); };
+  auto tempty_bar = [&](uint32_t b) { return bar0 + 8u * (2 * kTcMaxStages + 2 + b); };
+  const uint32_t hfull_bar = bar0 + 8u * (2 * kTcMaxStages + 4), hempty_bar = bar0 + 8u * (2 * kTcMaxStages + 5);
+  if (tid == 0) {
+    for (int s = 0; s < NS; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+    mbar_init(hfull_bar, 1);
+    mbar_init(hempty_bar, 1);
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  const int n_items = *p.n_items, n_zc = *p.n_zc;
+  for (int i = tid; i <= p.max_items; i += kTcThreads) s_pref[i] = p.pref[i];
+  {
+    const uint4 *src = reinterpret_cast<const uint4 *>(p.items);
+    uint4 *dst = reinterpret_cast<uint4 *>(s_items);
+    for (int i = tid; i < 2 * p.max_items; i += kTcThreads) dst[i] = src[i];
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(s_tmem)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *s_tmem;
+  const uint32_t t_sfa = tmem + 128u, t_sfb = tmem + 192u;
+  const size_t sec_b = (size_t)NG * KSA * kTcStageA;   // the down section follows the gate/up section
+
+  uint32_t pass0[2], s_begin[2], s_end[2];
+  pass0[0] = 0u;
+  pass0[1] = (uint32_t)s_pref[n_items];
+  {
+    const uint32_t np0 = pass0[1], np1 = (uint32_t)s_pref[n_items + n_zc] - pass0[1];
+    const uint32_t t0 = np0 * CG * DS, t1 = np1 * CG * DS;
+    s_begin[0] = w4_first(t0, gridDim.x, blockIdx.x); s_end[0] = w4_first(t0, gridDim.x, blockIdx.x + 1);
+    s_begin[1] = w4_first(t1, gridDim.x, blockIdx.x); s_end[1] = w4_first(t1, gridDim.x, blockIdx.x + 1);
+  }
+  // body(pass, cg, st0, n): a run of n stages of tile (pass, column group cg), starting at stage st0
+  auto walk = [&](auto body) {
+    for (int r = 0; r < 2; ++r)
+      for (uint32_t s = s_begin[r]; s < s_end[r];) {
+        const uint32_t tile = s / DS, st0 = s - tile * DS, n = min(DS - st0, s_end[r] - s);
+        if (!body(pass0[r] + tile / CG, tile % CG, st0, n)) return;
+        s += n;
+      }
+  };
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ---- producer ----
+      asm volatile("griddepcontrol.wait;" ::: "memory");   // h is written by the gate/up kernel
+      uint32_t it = 0, n_h = 0, cur = 0xffffffffu;
+      walk([&](uint32_t pass, uint32_t cg, uint32_t st0, uint32_t n) {
+        if (pass != cur) {
+          // the pass's h image replaces the previous one once the MMAs that read that have completed
+          if (n_h && !mbar_wait(hempty_bar, (n_h - 1u) & 1u, s_abort, p.status)) return false;
+          mbar_expect_tx(hfull_bar, h_bytes);
+          const uint8_t *src = p.hq + (size_t)pass * h_bytes;
+          for (uint32_t o = 0; o < h_bytes; o += 16384u) bulk_g2s(smem_u32(s_b) + o, src + o, min(16384u, h_bytes - o), hfull_bar);
+          cur = pass;
+          ++n_h;
+        }
+        const uint8_t *rec = s_items[w4_find_item(s_pref, n_items + n_zc, pass)].w;
+        const uint8_t *src = rec + sec_b + ((size_t)cg * DS + st0) * kTcStageD;
+        for (uint32_t s = 0; s < n; ++s, ++it) {
+          const uint32_t slot = it % (uint32_t)NS;
+          if (!mbar_wait(empty_bar(slot), ((it / (uint32_t)NS) & 1u) ^ 1u, s_abort, p.status)) return false;
+          mbar_expect_tx(full_bar(slot), kTcStageD);
+          bulk_g2s(smem_u32(s_ring) + slot * kTcStageD, src + (size_t)s * kTcStageD, kTcStageD, full_bar(slot));
+        }
+        return true;
+      });
+      for (uint32_t k = it > (uint32_t)NS ? it - (uint32_t)NS : 0u; k < it; ++k)
+        (void)mbar_wait(full_bar(k % (uint32_t)NS), (k / (uint32_t)NS) & 1u, s_abort, p.status);
+      if (n_h) (void)mbar_wait(hfull_bar, (n_h - 1u) & 1u, s_abort, p.status);
+      abort_drain(s_abort);
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ---- MMA issuer ----
+      uint32_t it = 0, seg = 0, n_h = 0, cur = 0xffffffffu;
+      walk([&](uint32_t pass, uint32_t, uint32_t st0, uint32_t n) {
+        if (pass != cur) {
+          if (n_h) umma_commit(hempty_bar);   // arrives when every MMA issued so far has completed
+          if (!mbar_wait(hfull_bar, n_h & 1u, s_abort, p.status)) return false;
+          tc_fence_after();
+          for (uint32_t a = 0; a < DS; ++a) tc_cp_scales(t_sfb + 4u * a, smem_u32(s_b) + 2u * DS * kTcStepB + a * 512u);
+          cur = pass;
+          ++n_h;
+        }
+        const uint32_t buf = seg & 1u;
+        if (!mbar_wait(tempty_bar(buf), ((seg >> 1) & 1u) ^ 1u, s_abort, p.status)) return false;
+        tc_fence_after();
+        const uint32_t dd = tmem + buf * 64u;
+        for (uint32_t s = 0; s < n; ++s, ++it) {
+          const uint32_t slot = it % (uint32_t)NS;
+          if (!mbar_wait(full_bar(slot), (it / (uint32_t)NS) & 1u, s_abort, p.status)) return false;
+          tc_fence_after();
+          const uint32_t st = smem_u32(s_ring) + slot * kTcStageD;
+          tc_cp_scales(t_sfa + slot * 4u, st + 8192u);
+#pragma unroll
+          for (uint32_t step = 0; step < 2; ++step) {
+            const uint64_t bd = tc_desc(smem_u32(s_b) + ((st0 + s) * 2u + step) * kTcStepB, kTcN * 16u, 128u);
+            tc_mma(dd, tc_desc(st + step * 4096u, 2048u, 128u), bd, 2u * step, t_sfa + slot * 4u, t_sfb + 4u * (st0 + s),
+                   (s | step) ? 1u : 0u);
+          }
+          umma_commit(empty_bar(slot));
+        }
+        umma_commit(tfull_bar(buf));
+        ++seg;
+        return true;
+      });
+    }
+  } else {
+    // ---- epilogue: thread = output column of the tile ----
+    const int ew = warp & 3, row = ew * 32 + lane;
+    uint32_t seg = 0;
+    walk([&](uint32_t pass, uint32_t cg, uint32_t, uint32_t) {
+      const uint32_t buf = seg & 1u;
+      // gate weights of the pass's tokens (0 for the tokens that are not routed to this expert)
+      float gw[8];
+#pragma unroll
+      for (int t = 0; t < 8; ++t) gw[t] = 0.f;
+      {
+        const WorkItem &wi = s_items[w4_find_item(s_pref, n_items + n_zc, pass)];
+        if (wi.expert >= 0) {
+          for (int j = 0; j < wi.n_tok && j < 8; ++j) {
+            const int pr = p.perm[wi.off + j];
+            const float wv = p.topk_w[pr];
+            const int tk = pr / p.top_k;
+#pragma unroll
+            for (int t = 0; t < 8; ++t)
+              if (t == tk) gw[t] = wv;
+          }
+        } else {
+#pragma unroll
+          for (int t = 0; t < 8; ++t) gw[t] = t < p.T ? 1.f : 0.f;
+        }
+      }
+      bool ok = true;
+      if (lane == 0) ok = mbar_wait(tfull_bar(buf), (seg >> 1) & 1u, s_abort, p.status);
+      ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+      if (!ok) return false;
+      tc_fence_after();
+      float v[8];
+      tc_row_sums(tmem + buf * 64u + ((uint32_t)(ew * 32) << 16), v);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(buf));
+      float *yc = p.y_acc + 128u * cg + row;
+#pragma unroll
+      for (int t = 0; t < 8; ++t)
+        if (gw[t] != 0.f) red_add_f32(yc + (size_t)t * d, gw[t] * v[t]);
+      ++seg;
+      return true;
+    });
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+
+  // ---- the last CTA to finish rounds the accumulator to bf16 and clears it ----
+  if (!p.finalize) return;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const uint32_t prev = atomicAdd(p.done, 1u);
+    s_final = (prev == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (!s_final) return;
+  __threadfence();
+  const int n4 = p.T * (d / 4);
+  for (int i = tid; i < n4; i += kTcThreads) {
+    const float4 v = __ldcg(reinterpret_cast<const float4 *>(p.y_acc) + i);
+    __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b2 = __floats2bfloat162_rn(v.z, v.w);
+    uint2 o;
+    o.x = *reinterpret_cast<uint32_t *>(&a);
+    o.y = *reinterpret_cast<uint32_t *>(&b2);
+    reinterpret_cast<uint2 *>(p.y)[i] = o;
+    reinterpret_cast<float4 *>(p.y_acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  if (tid == 0) *p.done = 0u;
+}
+
+}  // namespace ftmoe

@@ -12,6 +12,7 @@
 #include "ffn_stream.cuh"
 #include "dequant_w4.cuh"
 #include "ffn_mx4.cuh"
+#include "ffn_mx4tc.cuh"
 #include "ffn_w4.cuh"
 #include "ffn_w4_half.cuh"
 #include "gemm_tc.cuh"
@@ -97,6 +98,7 @@ struct ft_moe {
   float *w4_hraw = nullptr;
   int32_t *w4_hcount = nullptr;
   uint8_t *w4_hq = nullptr;
+  uint8_t *tc_xq = nullptr;      // FT_W_MXFP4_TC: the bit-sliced activation images of a call (two K halves)
   float2 *w4_hs = nullptr;
   int last_fill_layer = -1;
   int overlap = 0;                      // launch mode of the streaming kernel (see FfnStreamParams::overlap)
@@ -161,7 +163,7 @@ size_t expert_bytes_of(const ft_moe_config_t *c) {
     if ((d != 256 && d != 512 && d != 1024 && d != 2048) || I % 16) return 0;
     return 3 * I * d * 2;
   }
-  if (c->wdtype == FT_W_MXFP4) {
+  if (c->wdtype == FT_W_MXFP4 || c->wdtype == FT_W_MXFP4_TC) {
     if (d % 512 || d > 8192 || I % 128) return 0;   // (same shapes as int4)
     return 3 * I * d / 2 + 3 * I * d / 32;
   }
@@ -499,6 +501,7 @@ ft_status_t ft_moe_destroy(ft_moe_t *h) {
   cudaFree(h->w4_hraw);
   cudaFree(h->w4_hcount);
   cudaFree(h->w4_hq);
+  cudaFree(h->tc_xq);
   cudaFree(h->w4_hs);
   cudaFree(h->trace_dev);
   cudaFree(h->stage_logits);
@@ -530,7 +533,8 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
       c.max_tokens <= 0 || (c.n_shared != 0 && c.n_shared != 1) || c.device < 0 ||
       (c.fill_mode != FT_FILL_COPY_ENGINE && c.fill_mode != FT_FILL_SM))
     return FT_ERR_INVALID_ARG;
-  if (c.wdtype != FT_W_BF16 && c.wdtype != FT_W_INT4_G128 && c.wdtype != FT_W_MXFP4 && c.wdtype != FT_W_NVFP4)
+  if (c.wdtype != FT_W_BF16 && c.wdtype != FT_W_INT4_G128 && c.wdtype != FT_W_MXFP4 && c.wdtype != FT_W_NVFP4 &&
+      c.wdtype != FT_W_MXFP4_TC)
     return FT_ERR_INVALID_ARG;
   if (c.bw_fill_MBps == 0 || c.bw_zc_MBps == 0 || c.bw_hbm_MBps == 0 || c.reuse_credit < 0 ||
       c.zc_tokens_per_pass < 1 || c.hbm_tokens_per_pass < 1 || c.gemm_min_tokens < 0 || c.split_min_pairs < 0)
@@ -541,6 +545,8 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
       (c.slots_per_layer == 0 || c.hidden % 256 || c.inter % 256 || c.gemm_min_tokens < 8 ||
        (c.wdtype != FT_W_BF16 && c.global_pool)))   // (4-bit: the bf16 scratch mirrors one layer's slots)
     return FT_ERR_UNSUPPORTED;
+  // the tensor-core-image records are served by the decode-sized kernels only
+  if (c.wdtype == FT_W_MXFP4_TC && (c.max_tokens > kQ4Tokens || c.gemm_min_tokens != 0)) return FT_ERR_UNSUPPORTED;
   if (!c.host_pool || c.host_pool_bytes < (size_t)c.n_layers * c.n_experts * S) return FT_ERR_INVALID_ARG;
   if (c.n_shared && !c.shared_weights) return FT_ERR_INVALID_ARG;
   if ((long long)c.max_tokens * c.top_k > (1ll << 30)) return FT_ERR_INVALID_ARG;
@@ -667,7 +673,17 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
     FT_TRY(cudaMemset(h->w4_hraw, 0, passes * (c.inter / 16) * 1024));
     FT_TRY(cudaMalloc(&h->w4_hcount, passes * (c.inter / 128) * 4));
     FT_TRY(cudaMemset(h->w4_hcount, 0, passes * (c.inter / 128) * 4));
-    FT_TRY(cudaMalloc(&h->w4_hq, passes * (c.inter / 128) * 2048));
+    FT_TRY(cudaMalloc(&h->w4_hq, c.wdtype == FT_W_MXFP4_TC ? passes * tc_h_pass_bytes(c.inter) : passes * (c.inter / 128) * 2048));
+    if (c.wdtype == FT_W_MXFP4_TC) {
+      FT_TRY(cudaMemset(h->w4_hq, 0, passes * tc_h_pass_bytes(c.inter)));
+      FT_TRY(cudaMalloc(&h->tc_xq, 2 * tc_x_half_bytes(c.hidden)));
+      FT_TRY(cudaMemset(h->tc_xq, 0, 2 * tc_x_half_bytes(c.hidden)));
+      if (tc_gateup_fixed_bytes(2 * c.n_experts + 1, c.hidden) + 3 * kTcStageA > kTcSmem ||
+          tc_down_fixed_bytes(2 * c.n_experts + 1, c.inter) + 3 * kTcStageD > kTcSmem || c.inter / 128 > 80)
+        return fail(FT_ERR_UNSUPPORTED);
+      FT_TRY(cudaFuncSetAttribute(tc_gateup_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmem));
+      FT_TRY(cudaFuncSetAttribute(tc_down_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmem));
+    }
     FT_TRY(cudaMalloc(&h->w4_hs, passes * (c.inter / 128) * 64));
     // (limits are per function and device, not per handle: always the largest a CTA can have, and the handle's own
     // need is checked against it)
@@ -1058,6 +1074,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   }
   // int4 / mxfp4: gate/up kernel writes h, down kernel accumulates, its last CTA finalizes y
   if (c.slots_per_layer > 0 && L.fill_recorded) FT_CUDA(cudaStreamWaitEvent(st, L.ev_fill, 0));
+  if (c.wdtype == FT_W_MXFP4_TC && L.T > kQ4Tokens) return FT_ERR_UNSUPPORTED;
   W4Params qp;
   qp.items = sc.items_res;
   qp.n_items = &sc.plan_dev->n_res_items;
@@ -1076,6 +1093,45 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   qp.inter = c.inter; qp.top_k = c.top_k; qp.T = L.T;
   const bool own_finalize = !use_gemm && L.T > kFinalizeInKernelMaxTokens;
   qp.finalize = (use_gemm || own_finalize) ? 0 : 1;   // (the GEMM path's combine rounds y)
+  if (c.wdtype == FT_W_MXFP4_TC) {
+    // bit-sliced activation images, then the two block-scaled tensor-core kernels (programmatic dependents: their
+    // set-up and first weight copies overlap the kernel before them)
+    qp.finalize = 1;
+    TcQuantParams tq;
+    tq.x = x_bf; tq.xq = h->tc_xq; tq.T = L.T; tq.d = c.hidden;
+    {
+      TimeScope ts(h, st, FT_TIME_GATHER);
+      tc_quant_x_kernel<<<c.hidden / 256, 256, 0, st>>>(tq);
+    }
+    TcParams tp;
+    tp.w = qp; tp.xq = h->tc_xq; tp.d = c.hidden;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    const int grid = h->sm_count & ~1;   // CTAs of even / odd index work on the first / second half of the hidden dimension
+    {
+      TimeScope ts(h, st, FT_TIME_FFN_ZC);
+      const size_t fixed = tc_gateup_fixed_bytes(qp.max_items, c.hidden);
+      tp.n_stages = (int)std::min<size_t>(kTcMaxStages, (kTcSmem - fixed) / kTcStageA);
+      cudaLaunchConfig_t lc = {};
+      lc.gridDim = dim3(grid); lc.blockDim = dim3(kTcThreads); lc.stream = st;
+      lc.dynamicSmemBytes = fixed + (size_t)tp.n_stages * kTcStageA;
+      lc.attrs = at; lc.numAttrs = 1;
+      FT_CUDA(cudaLaunchKernelEx(&lc, tc_gateup_kernel, tp));
+    }
+    {
+      TimeScope ts(h, st, FT_TIME_FFN_RES);
+      const size_t fixed = tc_down_fixed_bytes(qp.max_items, c.inter);
+      tp.n_stages = (int)std::min<size_t>(kTcMaxStages, (kTcSmem - fixed) / kTcStageD);
+      cudaLaunchConfig_t lc = {};
+      lc.gridDim = dim3(h->sm_count); lc.blockDim = dim3(kTcThreads); lc.stream = st;
+      lc.dynamicSmemBytes = fixed + (size_t)tp.n_stages * kTcStageD;
+      lc.attrs = at; lc.numAttrs = 1;
+      FT_CUDA(cudaLaunchKernelEx(&lc, tc_down_kernel, tp));
+    }
+    h->launches += 3;
+    return FT_OK;
+  }
   const bool half = !mx && L.T <= kW4HalfTokens;   // int4 with at most 4 tokens: one MMA per pair of weight words
   const size_t sa = mx ? mx4_gateup_smem_bytes(qp.max_items, c.hidden)
                        : half ? w4_gateup_half_smem_bytes(qp.max_items, c.hidden) : w4_gateup_smem_bytes(qp.max_items, c.hidden);

@@ -33,7 +33,7 @@ class Pair:
         self.shared = None
         if shape.n_shared:
             self.shared = W.make_shared_records(shape, n_layers, seed, device=gen_device)
-        wd = {"bf16": B.FT_W_BF16, "int4": B.FT_W_INT4_G128, "mxfp4": B.FT_W_MXFP4, "nvfp4": B.FT_W_NVFP4}[shape.wdtype]
+        wd = {"bf16": B.FT_W_BF16, "int4": B.FT_W_INT4_G128, "mxfp4": B.FT_W_MXFP4, "nvfp4": B.FT_W_NVFP4, "mxfp4tc": B.FT_W_MXFP4_TC}[shape.wdtype]
         self.cfg = B.make_config(hidden=shape.d, inter=shape.inter, n_experts=shape.n_experts,
                                  top_k=shape.top_k, n_layers=n_layers, slots_per_layer=n_slots,
                                  max_tokens=max_tokens, host_pool_ptr=self.pool.ptr.value,

@@ -161,6 +161,18 @@ def test_int4_activation_outlier_in_a_group(wdtype):
     pr.close()
 
 
+@pytest.mark.parametrize("n_shared", [0, 1])
+@pytest.mark.parametrize("T", [1, 4, 8])
+def test_mxfp4_tensor_core_images_decode(n_shared, T):
+    """MXFP4 experts stored as operand images of the block-scaled tensor-core instruction: slot-resident, filled and
+    zero-copy experts (4 slots for 8 experts) and the shared expert, 1 to 8 tokens."""
+    shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2, wdtype="mxfp4tc", n_shared=n_shared)
+    pr = Pair(shape, n_slots=4, max_tokens=8, seed=5)
+    for step in range(3):
+        pr.step(0, W.normal_logits(T, 8, 5, step), W.noise_x(T, 512, 5, step, 0), check_slots=True)
+    pr.close()
+
+
 def test_nvfp4_small_and_subnormal_block_scales():
     """NVFP4 records written by definition whose gate and down block scales are the 15 smallest e4m3 numbers (exponent
     field 0 or 1: the subnormal bytes included) under a matrix scale of 2^9, so that an error in the decoding of
