@@ -801,7 +801,7 @@ def sub_int4(args, dev, cal, wdtype="int4"):
     import torch
     from paper_2608_16157_b200 import binding as Bd
     from paper_2608_16157_b200 import workload as W
-    shape = {"int4": W.DSV3_INT4, "mxfp4": W.DSV3_MXFP4, "nvfp4": W.DSV3_NVFP4}[wdtype]
+    shape = {"int4": W.DSV3_INT4, "mxfp4": W.DSV3_MXFP4, "nvfp4": W.DSV3_NVFP4, "mxfp4tc": W.DSV3_MXFP4TC}[wdtype]
     L, E, k, d, B, Ns = 4, shape.n_experts, shape.top_k, shape.d, 4, 64
     S = shape.expert_bytes
     warm, K = 48, 16
@@ -811,7 +811,8 @@ def sub_int4(args, dev, cal, wdtype="int4"):
     moe = Bd.FtMoe(Bd.make_config(hidden=d, inter=shape.inter, n_experts=E, top_k=k, n_layers=L, slots_per_layer=Ns,
                                   max_tokens=8, host_pool_ptr=pool.ptr.value, host_pool_bytes=pool.n_bytes,
                                   fill_mode=Bd.FT_FILL_SM,
-                                  wdtype={"int4": Bd.FT_W_INT4_G128, "mxfp4": Bd.FT_W_MXFP4, "nvfp4": Bd.FT_W_NVFP4}[wdtype], n_shared=1,
+                                  wdtype={"int4": Bd.FT_W_INT4_G128, "mxfp4": Bd.FT_W_MXFP4, "nvfp4": Bd.FT_W_NVFP4,
+                                          "mxfp4tc": Bd.FT_W_MXFP4_TC}[wdtype], n_shared=1,
                                   shared_ptr=shared.data_ptr(), bw_fill=max(cal["fill_MBps"], 1),
                                   bw_zc=max(cal["zc_MBps"], 1), bw_zc_residual=0, bw_hbm=max(cal["hbm_MBps"], 1)))
     stream = torch.cuda.current_stream()
@@ -880,8 +881,10 @@ def sub_int4(args, dev, cal, wdtype="int4"):
     return {"config": "decode, config 3: d=7168, 256 %s experts + 1 shared, I=2048, top-8, 4 layers, 64 slots "
                       "per layer, batch 4, rho 0.9, alpha 1.2" % ("int4-g128" if wdtype == "int4" else wdtype),
             "kernels": "w4_gateup_kernel + w4_down_kernel" if wdtype == "int4" else
+                       "tc_quant_x_kernel + tc_gateup_kernel + tc_down_kernel (tcgen05 kind::mxf4 block-scaled MMA on "
+                       "records stored as operand images)" if wdtype == "mxfp4tc" else
                        "mx4_gateup_kernel + mx4_down_kernel" + (" (NVFP4 instances)" if wdtype == "nvfp4" else ""),
-            "bound": "hbm" if wdtype == "int4" else "alu (logic pipe: 7 instructions per 8 weights plus a scale per MMA"
+            "bound": "hbm" if wdtype in ("int4", "mxfp4tc") else "alu (logic pipe: 7 instructions per 8 weights plus a scale per MMA"
                      + (", one K=16 MMA per 16-element scale block" if wdtype == "nvfp4" else "") + "); reported against the HBM peak",
             "tok_per_s": B * K / (ms * 1e-3), "ms_per_step": ms / K,
             "fills_per_step": (st1["fills"] - st0["fills"]) / K, "cache_warm_steps": warm,
@@ -899,11 +902,15 @@ def sub_mxfp4(args, dev, cal):
     return sub_int4(args, dev, cal, "mxfp4")
 
 
+def sub_mxfp4tc(args, dev, cal):
+    return sub_int4(args, dev, cal, "mxfp4tc")
+
+
 def sub_nvfp4(args, dev, cal):
     return sub_int4(args, dev, cal, "nvfp4")
 
 
-SUBRECORDS = {"int4": sub_int4, "mxfp4": sub_mxfp4, "nvfp4": sub_nvfp4, "prefill": sub_prefill,
+SUBRECORDS = {"int4": sub_int4, "mxfp4": sub_mxfp4, "mxfp4tc": sub_mxfp4tc, "nvfp4": sub_nvfp4, "prefill": sub_prefill,
               "prefill_mxfp4": sub_prefill_mxfp4}
 
 
@@ -1024,7 +1031,7 @@ def main():
     ap.add_argument("--only-batch", action="store_true")
     ap.add_argument("--cache-warm-steps", type=int, default=64,
                     help="untimed steps from the empty cache before warm-up and timing (steady-state headline)")
-    ap.add_argument("--sub", default="int4,mxfp4,nvfp4,prefill,prefill_mxfp4", help="bounded sub-records added to the decode line (N=1 only)")
+    ap.add_argument("--sub", default="int4,mxfp4,mxfp4tc,nvfp4,prefill,prefill_mxfp4", help="bounded sub-records added to the decode line (N=1 only)")
     ap.add_argument("--overlap", type=int, default=0,
                     help="launch mode of the streaming kernel in the timed region (ft_moe_set_launch_overlap)")
     args = ap.parse_args()

@@ -97,6 +97,8 @@ struct TcQuantParams {
 };
 __global__ void __launch_bounds__(256) tc_quant_x_kernel(TcQuantParams p) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // (when launched as a programmatic dependent: the images are still being read until the kernels before have completed)
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int per_tok = p.d / 8;
   const int i = blockIdx.x * 256 + threadIdx.x;
   if (i >= 8 * per_tok) return;
@@ -431,6 +433,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
   __shared__ int s_final;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const uint32_t bar0 = smem_u32(s_bar);
   auto full_bar = [&](uint32_t s) { return bar0 + 8u * s; };
   auto empty_bar = [&](uint32_t s) { return bar0 + 8u * (kTcMaxStages + s); };

@@ -1099,15 +1099,18 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     qp.finalize = 1;
     TcQuantParams tq;
     tq.x = x_bf; tq.xq = h->tc_xq; tq.T = L.T; tq.d = c.hidden;
-    {
-      TimeScope ts(h, st, FT_TIME_GATHER);
-      tc_quant_x_kernel<<<c.hidden / 256, 256, 0, st>>>(tq);
-    }
-    TcParams tp;
-    tp.w = qp; tp.xq = h->tc_xq; tp.d = c.hidden;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
+    {
+      TimeScope ts(h, st, FT_TIME_GATHER);
+      cudaLaunchConfig_t lc = {};
+      lc.gridDim = dim3(c.hidden / 256); lc.blockDim = dim3(256); lc.stream = st;
+      lc.attrs = at; lc.numAttrs = h->overlap ? 1 : 0;   // (it waits for the kernels before it by itself)
+      FT_CUDA(cudaLaunchKernelEx(&lc, tc_quant_x_kernel, tq));
+    }
+    TcParams tp;
+    tp.w = qp; tp.xq = h->tc_xq; tp.d = c.hidden;
     const int grid = h->sm_count & ~1;   // CTAs of even / odd index work on the first / second half of the hidden dimension
     {
       TimeScope ts(h, st, FT_TIME_FFN_ZC);

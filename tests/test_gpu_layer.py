@@ -173,6 +173,50 @@ def test_mxfp4_tensor_core_images_decode(n_shared, T):
     pr.close()
 
 
+@pytest.mark.parametrize("scale_log2", [-10, 10])
+def test_mxfp4_tensor_core_images_activation_range(scale_log2):
+    """The bit-sliced activations carry a power-of-two scale per (token, term, block of 32), so inputs scaled by
+    2^-10 and 2^10 meet the same tolerance."""
+    shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2, wdtype="mxfp4tc", n_shared=1)
+    pr = Pair(shape, n_slots=4, max_tokens=8, seed=8)
+    for step in range(2):
+        x = (W.noise_x(6, 512, 8, step, 0).float() * (2.0 ** scale_log2)).to(torch.bfloat16)
+        pr.step(0, W.normal_logits(6, 8, 8, step), x)
+    pr.close()
+
+
+def test_mxfp4_tensor_core_images_activation_outlier_in_a_block():
+    """One element 1000 x larger than the rest of its block, every token, and an all-zero token."""
+    shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2, wdtype="mxfp4tc", n_shared=1)
+    pr = Pair(shape, n_slots=4, max_tokens=8, seed=12)
+    for step in range(2):
+        x = W.noise_x(6, 512, 12, step, 0).float()
+        x[:, 5::128] *= 1000.0
+        x[2, :] = 0.0
+        pr.step(0, W.normal_logits(6, 8, 12, step), x.to(torch.bfloat16))
+    pr.close()
+
+
+def test_mxfp4_tensor_core_images_many_steps_device_fills_and_wide_shape():
+    """d=2048, I=768 (6 neuron groups, 16 stages per tile), 32 experts, top-4, 12 slots, device-driven fills, 12
+    steps of 8 tokens: evictions, zero-copy experts and tiles split between CTAs."""
+    shape = W.LayerShape(d=2048, inter=768, n_experts=32, top_k=4, wdtype="mxfp4tc")
+    pr = Pair(shape, n_slots=12, max_tokens=8, seed=14, fill_mode=B.FT_FILL_SM, gen_device="cuda")
+    ev = 0
+    for step in range(12):
+        _, r = pr.step(0, W.normal_logits(8, 32, 14, step), W.noise_x(8, 2048, 14, step, 0), fused=(step % 2 == 1))
+        ev += sum(1 for e in r.plan.fill_evicted if e >= 0)
+    assert ev > 0
+    pr.close()
+
+
+def test_mxfp4_tensor_core_images_refuse_many_token_handles():
+    shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2, wdtype="mxfp4tc")
+    with pytest.raises(B.FtMoeError) as ei:
+        Pair(shape, n_slots=4, max_tokens=16, seed=1)
+    assert ei.value.code == B.FT_ERR_UNSUPPORTED
+
+
 def test_nvfp4_small_and_subnormal_block_scales():
     """NVFP4 records written by definition whose gate and down block scales are the 15 smallest e4m3 numbers (exponent
     field 0 or 1: the subnormal bytes included) under a matrix scale of 2^9, so that an error in the decoding of
@@ -297,7 +341,8 @@ def test_qwen3_shaped_decode_two_layers(batch):
     pr.close()
 
 
-@pytest.mark.parametrize("shape", [W.DSV3_INT4, W.DSV3_MXFP4, W.DSV3_NVFP4], ids=["int4", "mxfp4", "nvfp4"])
+@pytest.mark.parametrize("shape", [W.DSV3_INT4, W.DSV3_MXFP4, W.DSV3_NVFP4, W.DSV3_MXFP4TC],
+                         ids=["int4", "mxfp4", "nvfp4", "mxfp4tc"])
 def test_dsv3_shaped_int4_decode_one_layer(shape):
     """d=7168, 256 routed experts (int4 group 128, mxfp4 or nvfp4) + 1 shared expert, I=2048, top-8, 64 slots, batch 4."""
     steps = 3
