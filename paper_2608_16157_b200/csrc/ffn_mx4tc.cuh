@@ -10,16 +10,20 @@
 //     Every term removes at least a factor 3 of the block's largest leftover, so 6 terms leave <= 2^-9.5 of the
 //     block's largest magnitude; the terms of the 8 tokens are the N = 48 columns of the MMA (column 8 i + token),
 //     and the epilogue adds a token's 6 columns.  The tensor pipe has room for this: the kernels are HBM-bound.
-//   * Gate/up kernel: M = 128 neurons of the gate and of the up matrix per tile, K split into two halves (a CTA
-//     keeps the activation image of one half in shared memory: CTAs of even index the first half, of odd index the
-//     second), each CTA an equal share of (tile, 128-index stage) steps of its half.  One producer thread issues the
-//     bulk copies (17408 bytes per stage: gate image, up image, gate scales, up scales) into a ring, one thread
-//     copies the stage's scale factors to tensor memory (tcgen05.cp) and issues the four MMAs, four warps read the
-//     accumulators of a finished tile (tcgen05.ld), add a token's terms and add the partial sums into the per-unit
-//     fp32 accumulators in global memory; the CTA whose contribution completes a group of 128 neurons applies
-//     SiLU(gate) * up and writes the group's h as the bit-sliced activation image of the down kernel.
-//   * Down kernel: M = 128 output columns per tile, K = the neurons; same ring; the epilogue multiplies by the gate
-//     weight and adds into the fp32 output accumulator; the last CTA rounds it to bf16.
+//   * Gate/up kernel: M = 128 neurons of the gate and of the up matrix per tile, K split into four parts (a CTA
+//     keeps the activation image of one part in shared memory: CTA i that of part i % 4, which leaves most of the
+//     shared memory to the ring), each CTA an equal share of (tile, 128-index stage) steps of its part.  A producer
+//     warp issues the bulk copies (17408 bytes per stage: gate image, up image, gate scales, up scales) into a
+//     ring; two issuing threads, one for the gate and one for the up matrix, copy the stage's scale factors to
+//     tensor memory (tcgen05.cp) and issue two MMAs each (an MMA of this shape occupies the tensor pipe for about
+//     136 clocks whatever N is, so the pipe is busy most of the time and the scalar work of one issuer must hide
+//     behind the MMAs of the other); four warps read the accumulators of a finished tile (tcgen05.ld), add a
+//     token's terms and add the partial sums into the per-unit fp32 accumulators in global memory; the CTA whose
+//     contribution completes a group of 128 neurons applies SiLU(gate) * up and writes the group's h as the
+//     bit-sliced activation image of the down kernel.
+//   * Down kernel: M = 128 output columns per tile, K = the neurons; same ring, the two issuers take the stages
+//     alternately and accumulate separately; the epilogue adds the two, multiplies by the gate weight and adds into
+//     the fp32 output accumulator; the last CTA rounds it to bf16.
 // Every mbarrier wait is bounded (see async.cuh); a CTA whose wait runs out latches the timeout status, stops
 // issuing work, lets its copies in flight land, frees its tensor memory and returns.
 #pragma once
@@ -34,13 +38,18 @@ constexpr int kTcN = 8 * kTcTerms;          // MMA columns: 8 tokens x terms
 constexpr uint32_t kTcStepB = kTcN * 32u;   // bytes of the activation image of one K = 64 step
 constexpr uint32_t kTcStageA = 17408u;      // gate/up stage: two images of 8192 bytes, two scale atoms of 512
 constexpr uint32_t kTcStageD = 8704u;       // down stage: one image, one scale atom
-constexpr int kTcThreads = 192;             // warp 0: producer, warp 1: MMA issuer, warps 2..5: epilogue
+constexpr int kTcLoaders = 128;             // warps 0..3 copy the records' stages into the ring, 16 bytes per cp.async
+constexpr int kTcThreads = kTcLoaders + 64 + 128;   // then warps 4 and 5: MMA issuers, warps 6..9: epilogue
 constexpr int kTcMaxStages = 16;
 constexpr size_t kTcSmem = 232448 - 1024;   // dynamic shared memory the two kernels may use (1 KiB left for static data)
 
 // Activation images in global memory (written by tc_quant_x_kernel / by the gate/up kernel's group conversion).
-// Gate/up operand: for each K half: [d/128 steps][kTcStepB] then [d/256 scale atoms][512].
-__host__ __device__ inline size_t tc_x_half_bytes(int d) { return (size_t)(d / 128) * kTcStepB + (size_t)(d / 256) * 512; }
+// Gate/up operand: for each of the kTcParts parts of the hidden dimension: [d/256 steps][kTcStepB] then
+// [d/512 scale atoms][512].
+constexpr int kTcParts = 4;
+__host__ __device__ inline size_t tc_x_part_bytes(int d) {
+  return (size_t)(d / (64 * kTcParts)) * kTcStepB + (size_t)(d / (128 * kTcParts)) * 512;
+}
 // Down operand of one pass: [inter/64 steps][kTcStepB] then [inter/128 scale atoms][512].
 __host__ __device__ inline size_t tc_h_pass_bytes(int inter) { return (size_t)(inter / 64) * kTcStepB + (size_t)(inter / 128) * 512; }
 
@@ -92,7 +101,7 @@ __device__ __forceinline__ void tc_term(float (&r)[8], bool bad, uint32_t &codes
 // indices of a token slot (slots >= T are written as zeros); a quad of lanes is one block of 32.
 struct TcQuantParams {
   const __nv_bfloat16 *x;
-  uint8_t *xq;      // [2 halves][tc_x_half_bytes(d)]
+  uint8_t *xq;      // [kTcParts][tc_x_part_bytes(d)]
   int T, d;
 };
 __global__ void __launch_bounds__(256) tc_quant_x_kernel(TcQuantParams p) {
@@ -120,10 +129,10 @@ __global__ void __launch_bounds__(256) tc_quant_x_kernel(TcQuantParams p) {
     for (int e = 0; e < 8; ++e) r[e] = 0.f;
   }
   bad = (__shfl_xor_sync(0xffffffffu, (int)bad, 1) | __shfl_xor_sync(0xffffffffu, (int)bad, 2) | (int)bad) != 0;
-  const int half_k = p.d / 2;
-  const int k = 8 * c8, half = k >= half_k ? 1 : 0, kk = k - half * half_k;
-  uint8_t *img = p.xq + (size_t)half * tc_x_half_bytes(p.d);
-  uint8_t *sf = img + (size_t)(p.d / 128) * kTcStepB;
+  const int part_k = p.d / kTcParts;
+  const int k = 8 * c8, part = k / part_k, kk = k - part * part_k;
+  uint8_t *img = p.xq + (size_t)part * tc_x_part_bytes(p.d);
+  uint8_t *sf = img + (size_t)(part_k / 64) * kTcStepB;
   const int step = kk >> 6, kcore = (kk >> 5) & 1, word = (kk & 31) >> 3;
 #pragma unroll
   for (int t = 0; t < kTcTerms; ++t) {
@@ -131,7 +140,7 @@ __global__ void __launch_bounds__(256) tc_quant_x_kernel(TcQuantParams p) {
     tc_term(r, bad, codes, sb);
     *reinterpret_cast<uint32_t *>(img + (size_t)step * kTcStepB + kcore * (kTcN * 16) + t * 128 + tok * 16 + word * 4) = codes;
     if ((threadIdx.x & 3) == 0) {
-      const int n = 8 * t + tok, blk = kk >> 5;   // scale of (column n, block blk of the half)
+      const int n = 8 * t + tok, blk = kk >> 5;   // scale of (column n, block blk of the part)
       sf[(size_t)(blk >> 2) * 512 + (n & 31) * 16 + (n >> 5) * 4 + (blk & 3)] = (uint8_t)sb;
     }
   }
@@ -140,7 +149,7 @@ __global__ void __launch_bounds__(256) tc_quant_x_kernel(TcQuantParams p) {
 
 struct TcParams {
   W4Params w;          // the work lists, the hand-over buffers (hraw, hcount, hq) and the output, as for the other 4-bit kernels
-  const uint8_t *xq;   // activation images of the two K halves (tc_quant_x_kernel)
+  const uint8_t *xq;   // activation images of the kTcParts parts of the hidden dimension (tc_quant_x_kernel)
   int d;
   int n_stages;        // ring stages (what fits in shared memory, at most kTcMaxStages)
 };
@@ -172,10 +181,8 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
         "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr));
 }
-// The kTcN columns of this thread's accumulator row -> one sum per token.
+// The kTcN columns of this thread's accumulator row -> one sum per token, added to v[].
 __device__ __forceinline__ void tc_row_sums(uint32_t taddr, float (&v)[8]) {
-#pragma unroll
-  for (int t = 0; t < 8; ++t) v[t] = 0.f;
 #pragma unroll
   for (int c = 0; c < kTcN; c += 16) {
     uint32_t r[16];
@@ -185,18 +192,43 @@ __device__ __forceinline__ void tc_row_sums(uint32_t taddr, float (&v)[8]) {
     for (int j = 0; j < 16; ++j) v[j & 7] += __uint_as_float(r[j]);
   }
 }
+__device__ __forceinline__ void tc_cp16(uint32_t dst, const void *src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+// Shared memory written by the loaders' copies is read by the tensor core: order the two kinds of access.
+__device__ __forceinline__ void tc_fence_copies() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// One stage is copied by one loader warp (the loader warps take the stages in turn): each lane copies its 16-byte
+// pieces and posts an arrival that fires when its copies have landed.  The arrival orders a warp's later copies
+// behind it, so a warp has one stage in flight; the stages in flight are those of the different loader warps.
+template <uint32_t BYTES>
+__device__ __forceinline__ void tc_load_stage(uint32_t dst, const uint8_t *src, int lane, uint32_t full_bar) {
+  constexpr uint32_t kPieces = BYTES / 16u;
+  static_assert(kPieces % 32u == 0, "whole warps");
+#pragma unroll
+  for (uint32_t c = 0; c < kPieces / 32u; ++c) tc_cp16(dst + (c * 32u + lane) * 16u, src + (c * 32u + lane) * 16u);
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(full_bar) : "memory");
+}
 __device__ __forceinline__ void tc_epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-// Shared memory of the gate/up kernel: activation image of the K half | its scale atoms | ring | barriers | flags |
-// items | pref.
-inline size_t tc_gateup_fixed_bytes(int max_items, int d) {
-  return tc_x_half_bytes(d) + 64 * 8 + 64 + (size_t)max_items * sizeof(WorkItem) + ((size_t)max_items + 1) * 4 + 128;
-}
+// Barriers of both kernels (8 bytes each): full[16] | empty[16] | tfull[2] | tempty[2] | four more.
+struct TcBars {
+  uint32_t base;
+  __device__ uint32_t full(uint32_t s) const { return base + 8u * s; }
+  __device__ uint32_t empty(uint32_t s) const { return base + 8u * (kTcMaxStages + s); }
+  __device__ uint32_t tfull(uint32_t b) const { return base + 8u * (2 * kTcMaxStages + b); }
+  __device__ uint32_t tempty(uint32_t b) const { return base + 8u * (2 * kTcMaxStages + 2 + b); }
+  __device__ uint32_t extra(uint32_t i) const { return base + 8u * (2 * kTcMaxStages + 4 + i); }
+};
+
+// Shared memory of the gate/up kernel: activation image of the CTA's part of K | its scale atoms | ring | barriers |
+// flags.
+inline size_t tc_gateup_fixed_bytes(int d) { return tc_x_part_bytes(d) + 64 * 8 + 64 + 128; }
 
 __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
   const W4Params &p = q.w;
-  const int d = q.d, NS = q.n_stages;
-  const uint32_t KS = (uint32_t)d / 128u, SPH = KS / 2u;          // stages of a tile; of a K half
+  const int d = q.d;
+  const uint32_t NS = (uint32_t)q.n_stages;
+  const uint32_t KS = (uint32_t)d / 128u, SPH = KS / kTcParts;    // stages of a tile; of one part of the hidden dimension
   const uint32_t NG = (uint32_t)p.inter / 128u, NBLK = (uint32_t)p.inter / 16u;
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char *s_b = smem;                                        // [2 SPH steps][kTcStepB]
@@ -206,33 +238,23 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
   uint32_t *s_tmem = reinterpret_cast<uint32_t *>(s_bar + 64);
   volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
   volatile int *s_last = s_abort + 1;
-  WorkItem *s_items = reinterpret_cast<WorkItem *>(s_tmem + 16);
-  int32_t *s_pref = reinterpret_cast<int32_t *>(s_items + p.max_items);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  const uint32_t bar0 = smem_u32(s_bar);
-  auto full_bar = [&](uint32_t s) { return bar0 + 8u * s; };
-  auto empty_bar = [&](uint32_t s) { return bar0 + 8u * (kTcMaxStages + s); };
-  auto tfull_bar = [&](uint32_t b) { return bar0 + 8u * (2 * kTcMaxStages + b); };
-  auto tempty_bar = [&](uint32_t b) { return bar0 + 8u * (2 * kTcMaxStages + 2 + b); };
-  const uint32_t x_bar = bar0 + 8u * (2 * kTcMaxStages + 4);
+  const TcBars bar{smem_u32(s_bar)};
+  const uint32_t x_bar = bar.extra(0), sfb_bar = bar.extra(1);
   if (tid == 0) {
-    for (int s = 0; s < NS; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+    for (uint32_t s = 0; s < NS; ++s) { mbar_init(bar.full(s), 32); mbar_init(bar.empty(s), 2); }
+    for (uint32_t b = 0; b < 2; ++b) { mbar_init(bar.tfull(b), 2); mbar_init(bar.tempty(b), 4); }
     mbar_init(x_bar, 1);
+    mbar_init(sfb_bar, 1);
     *s_abort = 0;
     *s_last = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  // (decode-sized calls: every list entry is one pass of at most 8 tokens, so pass = index into the list)
   const int n_items = *p.n_items, n_zc = *p.n_zc;
-  for (int i = tid; i <= p.max_items; i += kTcThreads) s_pref[i] = p.pref[i];
-  {
-    const uint4 *src = reinterpret_cast<const uint4 *>(p.items);
-    uint4 *dst = reinterpret_cast<uint4 *>(s_items);
-    for (int i = tid; i < 2 * p.max_items; i += kTcThreads) dst[i] = src[i];
-  }
-  if (warp == 1) {
+  if (warp == 4) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(s_tmem)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -240,21 +262,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
+  // tensor memory columns: accumulators (buffer b: gate at 128 b, up at 128 b + 64) | weight scales of the ring
+  // slots (gate 4 s, up 64 + 4 s) | activation scales of the part (4 per stage)
   const uint32_t t_sfa = tmem + 256u, t_sfb = tmem + 384u;
 
-  // this CTA's share: CTAs of even index work on the first K half, of odd index on the second; within a half and
-  // within each of the two pass ranges (resident passes, then zero-copy passes) an equal number of stages per CTA
-  const uint32_t half = blockIdx.x & 1u, ci = blockIdx.x >> 1, nc = gridDim.x >> 1;
+  // this CTA's share: CTA i works on part i % kTcParts of the hidden dimension; within a part and within each of the
+  // two pass ranges (resident passes, then zero-copy passes) an equal number of stages per CTA
+  const uint32_t part = blockIdx.x % kTcParts, ci = blockIdx.x / kTcParts, nc = gridDim.x / kTcParts;
   uint32_t pass0[2], s_begin[2], s_end[2];
   pass0[0] = 0u;
-  pass0[1] = (uint32_t)s_pref[n_items];
+  pass0[1] = (uint32_t)n_items;
   {
-    const uint32_t np0 = pass0[1], np1 = (uint32_t)s_pref[n_items + n_zc] - pass0[1];
-    const uint32_t t0 = np0 * NG * SPH, t1 = np1 * NG * SPH;
+    const uint32_t t0 = (uint32_t)n_items * NG * SPH, t1 = (uint32_t)n_zc * NG * SPH;
     s_begin[0] = w4_first(t0, nc, ci); s_end[0] = w4_first(t0, nc, ci + 1);
     s_begin[1] = w4_first(t1, nc, ci); s_end[1] = w4_first(t1, nc, ci + 1);
   }
-  // body(pass, ng, st0, n): a run of n stages, starting at stage st0 of the half, of tile (pass, ng)
+  // body(pass, ng, st0, n): a run of n stages, starting at stage st0 of the part, of tile (pass, ng)
   auto walk = [&](auto body) {
     for (int r = 0; r < 2; ++r)
       for (uint32_t s = s_begin[r]; s < s_end[r];) {
@@ -264,92 +287,100 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
       }
   };
 
-  if (warp == 0) {
-    if (lane == 0) {
-      // ---- producer: the weights do not depend on the preceding kernels; the activation image does ----
-      uint32_t it = 0;
-      bool x_sent = false;
-      auto send_x = [&]() {
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-        const uint32_t bytes = (uint32_t)tc_x_half_bytes(d);
-        mbar_expect_tx(x_bar, bytes);
-        const uint8_t *src = q.xq + (size_t)half * bytes;
-        for (uint32_t o = 0; o < bytes; o += 16384u) bulk_g2s(smem_u32(s_b) + o, src + o, min(16384u, bytes - o), x_bar);
-        x_sent = true;
-      };
-      walk([&](uint32_t pass, uint32_t ng, uint32_t st0, uint32_t n) {
-        const uint8_t *rec = s_items[w4_find_item(s_pref, n_items + n_zc, pass)].w;
-        const uint8_t *src = rec + ((size_t)ng * KS + half * SPH + st0) * kTcStageA;
-        for (uint32_t s = 0; s < n; ++s, ++it) {
-          const uint32_t slot = it % (uint32_t)NS;
-          if (!mbar_wait(empty_bar(slot), ((it / (uint32_t)NS) & 1u) ^ 1u, s_abort, p.status)) return false;
-          mbar_expect_tx(full_bar(slot), kTcStageA);
-          bulk_g2s(smem_u32(s_ring) + slot * kTcStageA, src + (size_t)s * kTcStageA, kTcStageA, full_bar(slot));
-          if (!x_sent && it + 1 == (uint32_t)NS) send_x();   // after the first ring fill
+  if (warp < 4) {
+    // ---- loaders: the weights do not depend on the preceding kernels; the activation image does ----
+    uint32_t it = 0;
+    bool x_sent = tid != 0;
+    auto send_x = [&]() {
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      const uint32_t bytes = (uint32_t)tc_x_part_bytes(d);
+      mbar_expect_tx(x_bar, bytes);
+      const uint8_t *src = q.xq + (size_t)part * bytes;
+      for (uint32_t o = 0; o < bytes; o += 16384u) bulk_g2s(smem_u32(s_b) + o, src + o, min(16384u, bytes - o), x_bar);
+      x_sent = true;
+    };
+    walk([&](uint32_t pass, uint32_t ng, uint32_t st0, uint32_t n) {
+      const uint8_t *src = p.items[pass].w + ((size_t)ng * KS + part * SPH + st0) * kTcStageA;
+      for (uint32_t s = 0; s < n; ++s, ++it, src += kTcStageA) {
+        const uint32_t slot = it % NS;
+        if (it % (kTcLoaders / 32) == (uint32_t)warp) {
+          bool ok = true;
+          if (lane == 0) ok = mbar_wait(bar.empty(slot), ((it / NS) & 1u) ^ 1u, s_abort, p.status);
+          if (!__shfl_sync(0xffffffffu, (int)ok, 0)) return false;
+          tc_load_stage<kTcStageA>(smem_u32(s_ring) + slot * kTcStageA, src, lane, bar.full(slot));
         }
-        return true;
-      });
-      if (!x_sent) send_x();
-      // the copies issued must have landed before this CTA's shared memory is released
-      for (uint32_t k = it > (uint32_t)NS ? it - (uint32_t)NS : 0u; k < it; ++k)
-        (void)mbar_wait(full_bar(k % (uint32_t)NS), (k / (uint32_t)NS) & 1u, s_abort, p.status);
+        if (!x_sent && it + 1 == NS) send_x();   // after the first ring fill
+      }
+      return true;
+    });
+    if (!x_sent) send_x();
+    // the copies issued must have landed before this CTA's shared memory is released
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    if (tid == 0) {
       (void)mbar_wait(x_bar, 0u, s_abort, p.status);
       abort_drain(s_abort);
     }
-  } else if (warp == 1) {
+  } else if (warp <= 5) {
     if (lane == 0) {
-      // ---- MMA issuer ----
-      bool ok = mbar_wait(x_bar, 0u, s_abort, p.status);
-      if (ok) {
-        tc_fence_after();
-        for (uint32_t a = 0; a < SPH; ++a) tc_cp_scales(t_sfb + 4u * a, smem_u32(s_sfb) + a * 512u);
+      // ---- MMA issuers: warp 4 the gate matrix, warp 5 the up matrix ----
+      const uint32_t mat = (uint32_t)warp - 4u;
+      bool ok;
+      if (mat == 0) {
+        ok = mbar_wait(x_bar, 0u, s_abort, p.status);
+        if (ok) {
+          tc_fence_after();
+          for (uint32_t a = 0; a < SPH; ++a) tc_cp_scales(t_sfb + 4u * a, smem_u32(s_sfb) + a * 512u);
+          umma_commit(sfb_bar);   // the other issuer's MMAs read these scales too
+        }
+      } else {
+        ok = mbar_wait(sfb_bar, 0u, s_abort, p.status);
+        if (ok) tc_fence_after();
       }
       uint32_t it = 0, seg = 0;
+      const uint32_t b_base = smem_u32(s_b), ring = smem_u32(s_ring) + mat * 8192u, t_sf = t_sfa + mat * 64u;
       if (ok)
         walk([&](uint32_t, uint32_t, uint32_t st0, uint32_t n) {
           const uint32_t buf = seg & 1u;
-          if (!mbar_wait(tempty_bar(buf), ((seg >> 1) & 1u) ^ 1u, s_abort, p.status)) return false;
+          if (!mbar_wait(bar.tempty(buf), ((seg >> 1) & 1u) ^ 1u, s_abort, p.status)) return false;
           tc_fence_after();
-          const uint32_t dg = tmem + buf * 128u, du = dg + 64u;
+          const uint32_t dacc = tmem + buf * 128u + mat * 64u;
           for (uint32_t s = 0; s < n; ++s, ++it) {
-            const uint32_t slot = it % (uint32_t)NS;
-            if (!mbar_wait(full_bar(slot), (it / (uint32_t)NS) & 1u, s_abort, p.status)) return false;
+            const uint32_t slot = it % NS;
+            if (!mbar_wait(bar.full(slot), (it / NS) & 1u, s_abort, p.status)) return false;
+            tc_fence_copies();
             tc_fence_after();
-            const uint32_t st = smem_u32(s_ring) + slot * kTcStageA;
-            tc_cp_scales(t_sfa + slot * 8u, st + 16384u);
-            tc_cp_scales(t_sfa + slot * 8u + 4u, st + 16896u);
+            const uint32_t st = ring + slot * kTcStageA;
+            tc_cp_scales(t_sf + slot * 4u, smem_u32(s_ring) + slot * kTcStageA + 16384u + mat * 512u);
 #pragma unroll
-            for (uint32_t step = 0; step < 2; ++step) {
-              const uint64_t bd = tc_desc(smem_u32(s_b) + ((st0 + s) * 2u + step) * kTcStepB, kTcN * 16u, 128u);
-              const uint32_t sfb = t_sfb + 4u * (st0 + s), acc = (s | step) ? 1u : 0u;
-              tc_mma(dg, tc_desc(st + step * 4096u, 2048u, 128u), bd, 2u * step, t_sfa + slot * 8u, sfb, acc);
-              tc_mma(du, tc_desc(st + 8192u + step * 4096u, 2048u, 128u), bd, 2u * step, t_sfa + slot * 8u + 4u, sfb, acc);
-            }
-            umma_commit(empty_bar(slot));   // the stage may be refilled once these MMAs have read it
+            for (uint32_t step = 0; step < 2; ++step)
+              tc_mma(dacc, tc_desc(st + step * 4096u, 2048u, 128u),
+                     tc_desc(b_base + ((st0 + s) * 2u + step) * kTcStepB, kTcN * 16u, 128u), 2u * step, t_sf + slot * 4u,
+                     t_sfb + 4u * (st0 + s), (s | step) ? 1u : 0u);
+            umma_commit(bar.empty(slot));   // (count 2) the stage may be refilled once both issuers' MMAs have read it
           }
-          umma_commit(tfull_bar(buf));
+          umma_commit(bar.tfull(buf));
           ++seg;
           return true;
         });
     }
   } else {
     // ---- epilogue: thread = accumulator row (neuron of the tile) ----
-    const int ew = warp & 3, row = ew * 32 + lane, et = (warp - 2) * 32 + lane;
+    const int ew = warp & 3, row = ew * 32 + lane, et = (warp - 6) * 32 + lane;
     uint32_t seg = 0;
     walk([&](uint32_t pass, uint32_t ng, uint32_t, uint32_t n) {
       const uint32_t buf = seg & 1u;
       bool ok = true;
-      if (lane == 0) ok = mbar_wait(tfull_bar(buf), (seg >> 1) & 1u, s_abort, p.status);
+      if (lane == 0) ok = mbar_wait(bar.tfull(buf), (seg >> 1) & 1u, s_abort, p.status);
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
       if (ok) {
         tc_fence_after();
         const uint32_t trow = tmem + buf * 128u + ((uint32_t)(ew * 32) << 16);
-        float gsum[8], usum[8];
+        float gsum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f}, usum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
         tc_row_sums(trow, gsum);
         tc_row_sums(trow + 64u, usum);
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(tempty_bar(buf));
+        if (lane == 0) mbar_arrive(bar.tempty(buf));
         float *hacc = p.hraw + ((size_t)pass * NBLK + 8u * ng + (uint32_t)(row >> 4)) * 256 + (row & 15);
         for (int t = 0; t < p.T; ++t) {
           red_add_f32(hacc + t * 16, gsum[t]);
@@ -393,9 +424,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
           uint32_t codes, sb;
           tc_term(h, bad, codes, sb);
           *reinterpret_cast<uint32_t *>(dst + t * 128) = codes;
-          if ((sub & 3) == 0) {
+          // the scale bytes of the token's four blocks (held by the lanes sub = 0, 4, 8, 12) leave as one word
+          const int base = lane & 16;
+          const uint32_t w4 = __shfl_sync(0xffffffffu, sb, base) | (__shfl_sync(0xffffffffu, sb, base + 4) << 8) |
+                              (__shfl_sync(0xffffffffu, sb, base + 8) << 16) | (__shfl_sync(0xffffffffu, sb, base + 12) << 24);
+          if (sub == 0) {
             const int nn = 8 * t + tok;
-            sf[(nn & 31) * 16 + (nn >> 5) * 4 + (sub >> 2)] = (uint8_t)sb;
+            *reinterpret_cast<uint32_t *>(sf + (nn & 31) * 16 + (nn >> 5) * 4) = w4;
           }
         }
         if (et == 0) p.hcount[pass * NG + ng] = 0;
@@ -406,19 +441,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+  if (warp == 4) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
 }
-
 
 // Shared memory of the down kernel: activation image of the current pass and its scale atoms | ring | barriers |
-// flags | items | pref.
-inline size_t tc_down_fixed_bytes(int max_items, int inter) {
-  return tc_h_pass_bytes(inter) + 64 * 8 + 64 + (size_t)max_items * sizeof(WorkItem) + ((size_t)max_items + 1) * 4 + 128;
-}
+// flags.
+inline size_t tc_down_fixed_bytes(int inter) { return tc_h_pass_bytes(inter) + 64 * 8 + 64 + 128; }
 
 __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
   const W4Params &p = q.w;
-  const int d = q.d, NS = q.n_stages;
+  const int d = q.d;
+  const uint32_t NS = (uint32_t)q.n_stages;
   const uint32_t DS = (uint32_t)p.inter / 128u;        // stages (and scale atoms) of a tile
   const uint32_t CG = (uint32_t)d / 128u, NG = (uint32_t)p.inter / 128u, KSA = (uint32_t)d / 128u;
   const uint32_t h_bytes = (uint32_t)tc_h_pass_bytes(p.inter);
@@ -428,34 +461,23 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
   uint64_t *s_bar = reinterpret_cast<uint64_t *>(s_ring + (size_t)NS * kTcStageD);
   uint32_t *s_tmem = reinterpret_cast<uint32_t *>(s_bar + 64);
   volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
-  WorkItem *s_items = reinterpret_cast<WorkItem *>(s_tmem + 16);
-  int32_t *s_pref = reinterpret_cast<int32_t *>(s_items + p.max_items);
   __shared__ int s_final;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  const uint32_t bar0 = smem_u32(s_bar);
-  auto full_bar = [&](uint32_t s) { return bar0 + 8u * s; };
-  auto empty_bar = [&](uint32_t s) { return bar0 + 8u * (kTcMaxStages + s); };
-  auto tfull_bar = [&](uint32_t b) { return bar0 + 8u * (2 * kTcMaxStages + b); };
-  auto tempty_bar = [&](uint32_t b) { return bar0 + 8u * (2 * kTcMaxStages + 2 + b); };
-  const uint32_t hfull_bar = bar0 + 8u * (2 * kTcMaxStages + 4), hempty_bar = bar0 + 8u * (2 * kTcMaxStages + 5);
+  const TcBars bar{smem_u32(s_bar)};
+  const uint32_t hfull_bar = bar.extra(0), hempty_bar = bar.extra(1), sfb_bar = bar.extra(2);
   if (tid == 0) {
-    for (int s = 0; s < NS; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+    for (uint32_t s = 0; s < NS; ++s) { mbar_init(bar.full(s), 32); mbar_init(bar.empty(s), 1); }
+    for (uint32_t b = 0; b < 2; ++b) { mbar_init(bar.tfull(b), 2); mbar_init(bar.tempty(b), 4); }
     mbar_init(hfull_bar, 1);
-    mbar_init(hempty_bar, 1);
+    mbar_init(hempty_bar, 2);
+    mbar_init(sfb_bar, 1);
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  const int n_items = *p.n_items, n_zc = *p.n_zc;
-  for (int i = tid; i <= p.max_items; i += kTcThreads) s_pref[i] = p.pref[i];
-  {
-    const uint4 *src = reinterpret_cast<const uint4 *>(p.items);
-    uint4 *dst = reinterpret_cast<uint4 *>(s_items);
-    for (int i = tid; i < 2 * p.max_items; i += kTcThreads) dst[i] = src[i];
-  }
-  if (warp == 1) {
+  const int n_items = *p.n_items, n_zc = *p.n_zc;   // (pass = index into the list, see the gate/up kernel)
+  if (warp == 4) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(s_tmem)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -463,15 +485,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
-  const uint32_t t_sfa = tmem + 128u, t_sfb = tmem + 192u;
+  // tensor memory columns: accumulators (buffer b: the even stages' at 128 b, the odd stages' at 128 b + 64) | weight
+  // scales of the ring slots (4 s) | activation scales of the pass (4 per stage)
+  const uint32_t t_sfa = tmem + 256u, t_sfb = tmem + 320u;
   const size_t sec_b = (size_t)NG * KSA * kTcStageA;   // the down section follows the gate/up section
 
   uint32_t pass0[2], s_begin[2], s_end[2];
   pass0[0] = 0u;
-  pass0[1] = (uint32_t)s_pref[n_items];
+  pass0[1] = (uint32_t)n_items;
   {
-    const uint32_t np0 = pass0[1], np1 = (uint32_t)s_pref[n_items + n_zc] - pass0[1];
-    const uint32_t t0 = np0 * CG * DS, t1 = np1 * CG * DS;
+    const uint32_t t0 = (uint32_t)n_items * CG * DS, t1 = (uint32_t)n_zc * CG * DS;
     s_begin[0] = w4_first(t0, gridDim.x, blockIdx.x); s_end[0] = w4_first(t0, gridDim.x, blockIdx.x + 1);
     s_begin[1] = w4_first(t1, gridDim.x, blockIdx.x); s_end[1] = w4_first(t1, gridDim.x, blockIdx.x + 1);
   }
@@ -485,68 +508,81 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
       }
   };
 
-  if (warp == 0) {
-    if (lane == 0) {
-      // ---- producer ----
-      asm volatile("griddepcontrol.wait;" ::: "memory");   // h is written by the gate/up kernel
-      uint32_t it = 0, n_h = 0, cur = 0xffffffffu;
-      walk([&](uint32_t pass, uint32_t cg, uint32_t st0, uint32_t n) {
-        if (pass != cur) {
-          // the pass's h image replaces the previous one once the MMAs that read that have completed
-          if (n_h && !mbar_wait(hempty_bar, (n_h - 1u) & 1u, s_abort, p.status)) return false;
+  if (warp < 4) {
+    // ---- loaders ----
+    if (tid == 0) asm volatile("griddepcontrol.wait;" ::: "memory");   // h is written by the gate/up kernel
+    uint32_t it = 0, n_h = 0, cur = 0xffffffffu;
+    walk([&](uint32_t pass, uint32_t cg, uint32_t st0, uint32_t n) {
+      if (pass != cur && tid == 0) {
+        // the pass's h image replaces the previous one once the MMAs that read that have completed (a wait that
+        // gives up latches the abort flag: every loader then leaves at its next wait)
+        if (!n_h || mbar_wait(hempty_bar, (n_h - 1u) & 1u, s_abort, p.status)) {
           mbar_expect_tx(hfull_bar, h_bytes);
-          const uint8_t *src = p.hq + (size_t)pass * h_bytes;
-          for (uint32_t o = 0; o < h_bytes; o += 16384u) bulk_g2s(smem_u32(s_b) + o, src + o, min(16384u, h_bytes - o), hfull_bar);
-          cur = pass;
+          const uint8_t *hsrc = p.hq + (size_t)pass * h_bytes;
+          for (uint32_t o = 0; o < h_bytes; o += 16384u) bulk_g2s(smem_u32(s_b) + o, hsrc + o, min(16384u, h_bytes - o), hfull_bar);
           ++n_h;
         }
-        const uint8_t *rec = s_items[w4_find_item(s_pref, n_items + n_zc, pass)].w;
-        const uint8_t *src = rec + sec_b + ((size_t)cg * DS + st0) * kTcStageD;
-        for (uint32_t s = 0; s < n; ++s, ++it) {
-          const uint32_t slot = it % (uint32_t)NS;
-          if (!mbar_wait(empty_bar(slot), ((it / (uint32_t)NS) & 1u) ^ 1u, s_abort, p.status)) return false;
-          mbar_expect_tx(full_bar(slot), kTcStageD);
-          bulk_g2s(smem_u32(s_ring) + slot * kTcStageD, src + (size_t)s * kTcStageD, kTcStageD, full_bar(slot));
+      }
+      cur = pass;
+      const uint8_t *src = p.items[pass].w + sec_b + ((size_t)cg * DS + st0) * kTcStageD;
+      for (uint32_t s = 0; s < n; ++s, ++it, src += kTcStageD) {
+        const uint32_t slot = it % NS;
+        if (it % (kTcLoaders / 32) == (uint32_t)warp) {
+          bool ok = true;
+          if (lane == 0) ok = mbar_wait(bar.empty(slot), ((it / NS) & 1u) ^ 1u, s_abort, p.status);
+          if (!__shfl_sync(0xffffffffu, (int)ok, 0)) return false;
+          tc_load_stage<kTcStageD>(smem_u32(s_ring) + slot * kTcStageD, src, lane, bar.full(slot));
         }
-        return true;
-      });
-      for (uint32_t k = it > (uint32_t)NS ? it - (uint32_t)NS : 0u; k < it; ++k)
-        (void)mbar_wait(full_bar(k % (uint32_t)NS), (k / (uint32_t)NS) & 1u, s_abort, p.status);
+      }
+      return true;
+    });
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    if (tid == 0) {
       if (n_h) (void)mbar_wait(hfull_bar, (n_h - 1u) & 1u, s_abort, p.status);
       abort_drain(s_abort);
     }
-  } else if (warp == 1) {
+  } else if (warp <= 5) {
     if (lane == 0) {
-      // ---- MMA issuer ----
+      // ---- MMA issuers: warp 4 takes the stages of even ring index, warp 5 the odd ones ----
+      const uint32_t me = (uint32_t)warp - 4u;
       uint32_t it = 0, seg = 0, n_h = 0, cur = 0xffffffffu;
+      const uint32_t b_base = smem_u32(s_b);
       walk([&](uint32_t pass, uint32_t, uint32_t st0, uint32_t n) {
         if (pass != cur) {
-          if (n_h) umma_commit(hempty_bar);   // arrives when every MMA issued so far has completed
-          if (!mbar_wait(hfull_bar, n_h & 1u, s_abort, p.status)) return false;
-          tc_fence_after();
-          for (uint32_t a = 0; a < DS; ++a) tc_cp_scales(t_sfb + 4u * a, smem_u32(s_b) + 2u * DS * kTcStepB + a * 512u);
+          if (n_h) umma_commit(hempty_bar);   // (count 2) arrives when every MMA this thread has issued so far has completed
+          if (me == 0) {
+            if (!mbar_wait(hfull_bar, n_h & 1u, s_abort, p.status)) return false;
+            tc_fence_after();
+            for (uint32_t a = 0; a < DS; ++a) tc_cp_scales(t_sfb + 4u * a, b_base + 2u * DS * kTcStepB + a * 512u);
+            umma_commit(sfb_bar);
+          } else {
+            if (!mbar_wait(sfb_bar, n_h & 1u, s_abort, p.status)) return false;
+            tc_fence_after();
+          }
           cur = pass;
           ++n_h;
         }
         const uint32_t buf = seg & 1u;
-        if (!mbar_wait(tempty_bar(buf), ((seg >> 1) & 1u) ^ 1u, s_abort, p.status)) return false;
+        if (!mbar_wait(bar.tempty(buf), ((seg >> 1) & 1u) ^ 1u, s_abort, p.status)) return false;
         tc_fence_after();
-        const uint32_t dd = tmem + buf * 64u;
+        const uint32_t dacc = tmem + buf * 128u + me * 64u;
+        uint32_t mine = 0;
         for (uint32_t s = 0; s < n; ++s, ++it) {
-          const uint32_t slot = it % (uint32_t)NS;
-          if (!mbar_wait(full_bar(slot), (it / (uint32_t)NS) & 1u, s_abort, p.status)) return false;
+          if ((it & 1u) != me) continue;
+          const uint32_t slot = it % NS;
+          if (!mbar_wait(bar.full(slot), (it / NS) & 1u, s_abort, p.status)) return false;
+          tc_fence_copies();
           tc_fence_after();
           const uint32_t st = smem_u32(s_ring) + slot * kTcStageD;
           tc_cp_scales(t_sfa + slot * 4u, st + 8192u);
 #pragma unroll
-          for (uint32_t step = 0; step < 2; ++step) {
-            const uint64_t bd = tc_desc(smem_u32(s_b) + ((st0 + s) * 2u + step) * kTcStepB, kTcN * 16u, 128u);
-            tc_mma(dd, tc_desc(st + step * 4096u, 2048u, 128u), bd, 2u * step, t_sfa + slot * 4u, t_sfb + 4u * (st0 + s),
-                   (s | step) ? 1u : 0u);
-          }
-          umma_commit(empty_bar(slot));
+          for (uint32_t step = 0; step < 2; ++step)
+            tc_mma(dacc, tc_desc(st + step * 4096u, 2048u, 128u), tc_desc(b_base + ((st0 + s) * 2u + step) * kTcStepB, kTcN * 16u, 128u),
+                   2u * step, t_sfa + slot * 4u, t_sfb + 4u * (st0 + s), (mine | step) ? 1u : 0u);
+          ++mine;
+          umma_commit(bar.empty(slot));
         }
-        umma_commit(tfull_bar(buf));
+        umma_commit(bar.tfull(buf));   // (count 2; immediate for an issuer without a stage in this run)
         ++seg;
         return true;
       });
@@ -554,15 +590,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
   } else {
     // ---- epilogue: thread = output column of the tile ----
     const int ew = warp & 3, row = ew * 32 + lane;
-    uint32_t seg = 0;
-    walk([&](uint32_t pass, uint32_t cg, uint32_t, uint32_t) {
+    uint32_t seg = 0, it = 0, gw_pass = 0xffffffffu;
+    float gw[8];
+    walk([&](uint32_t pass, uint32_t cg, uint32_t, uint32_t n) {
       const uint32_t buf = seg & 1u;
-      // gate weights of the pass's tokens (0 for the tokens that are not routed to this expert)
-      float gw[8];
+      if (pass != gw_pass) {
+        // gate weights of the pass's tokens (0 for the tokens that are not routed to this expert); a CTA's tiles
+        // mostly belong to one pass, so these dependent loads are rare
+        gw_pass = pass;
 #pragma unroll
-      for (int t = 0; t < 8; ++t) gw[t] = 0.f;
-      {
-        const WorkItem &wi = s_items[w4_find_item(s_pref, n_items + n_zc, pass)];
+        for (int t = 0; t < 8; ++t) gw[t] = 0.f;
+        const WorkItem wi = p.items[pass];
         if (wi.expert >= 0) {
           for (int j = 0; j < wi.n_tok && j < 8; ++j) {
             const int pr = p.perm[wi.off + j];
@@ -578,26 +616,31 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
         }
       }
       bool ok = true;
-      if (lane == 0) ok = mbar_wait(tfull_bar(buf), (seg >> 1) & 1u, s_abort, p.status);
+      if (lane == 0) ok = mbar_wait(bar.tfull(buf), (seg >> 1) & 1u, s_abort, p.status);
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
       if (!ok) return false;
       tc_fence_after();
-      float v[8];
-      tc_row_sums(tmem + buf * 64u + ((uint32_t)(ew * 32) << 16), v);
+      // the run's stages it .. it+n-1 went alternately to the two issuers: add the accumulators that were written
+      const bool has_even = n >= 2u || (it & 1u) == 0u, has_odd = n >= 2u || (it & 1u) == 1u;
+      float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      const uint32_t trow = tmem + buf * 128u + ((uint32_t)(ew * 32) << 16);
+      if (has_even) tc_row_sums(trow, v);
+      if (has_odd) tc_row_sums(trow + 64u, v);
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(buf));
+      if (lane == 0) mbar_arrive(bar.tempty(buf));
       float *yc = p.y_acc + 128u * cg + row;
 #pragma unroll
       for (int t = 0; t < 8; ++t)
         if (gw[t] != 0.f) red_add_f32(yc + (size_t)t * d, gw[t] * v[t]);
+      it += n;
       ++seg;
       return true;
     });
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+  if (warp == 4) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
 
   // ---- the last CTA to finish rounds the accumulator to bf16 and clears it ----
   if (!p.finalize) return;

@@ -676,10 +676,10 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
     FT_TRY(cudaMalloc(&h->w4_hq, c.wdtype == FT_W_MXFP4_TC ? passes * tc_h_pass_bytes(c.inter) : passes * (c.inter / 128) * 2048));
     if (c.wdtype == FT_W_MXFP4_TC) {
       FT_TRY(cudaMemset(h->w4_hq, 0, passes * tc_h_pass_bytes(c.inter)));
-      FT_TRY(cudaMalloc(&h->tc_xq, 2 * tc_x_half_bytes(c.hidden)));
-      FT_TRY(cudaMemset(h->tc_xq, 0, 2 * tc_x_half_bytes(c.hidden)));
-      if (tc_gateup_fixed_bytes(2 * c.n_experts + 1, c.hidden) + 3 * kTcStageA > kTcSmem ||
-          tc_down_fixed_bytes(2 * c.n_experts + 1, c.inter) + 3 * kTcStageD > kTcSmem || c.inter / 128 > 80)
+      FT_TRY(cudaMalloc(&h->tc_xq, kTcParts * tc_x_part_bytes(c.hidden)));
+      FT_TRY(cudaMemset(h->tc_xq, 0, kTcParts * tc_x_part_bytes(c.hidden)));
+      if (tc_gateup_fixed_bytes(c.hidden) + 3 * kTcStageA > kTcSmem ||
+          tc_down_fixed_bytes(c.inter) + 3 * kTcStageD > kTcSmem || c.inter / 128 > 48 || h->sm_count < kTcParts)
         return fail(FT_ERR_UNSUPPORTED);
       FT_TRY(cudaFuncSetAttribute(tc_gateup_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmem));
       FT_TRY(cudaFuncSetAttribute(tc_down_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmem));
@@ -1111,10 +1111,10 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     }
     TcParams tp;
     tp.w = qp; tp.xq = h->tc_xq; tp.d = c.hidden;
-    const int grid = h->sm_count & ~1;   // CTAs of even / odd index work on the first / second half of the hidden dimension
+    const int grid = h->sm_count - h->sm_count % kTcParts;   // CTA i works on part i % kTcParts of the hidden dimension
     {
       TimeScope ts(h, st, FT_TIME_FFN_ZC);
-      const size_t fixed = tc_gateup_fixed_bytes(qp.max_items, c.hidden);
+      const size_t fixed = tc_gateup_fixed_bytes(c.hidden);
       tp.n_stages = (int)std::min<size_t>(kTcMaxStages, (kTcSmem - fixed) / kTcStageA);
       cudaLaunchConfig_t lc = {};
       lc.gridDim = dim3(grid); lc.blockDim = dim3(kTcThreads); lc.stream = st;
@@ -1124,7 +1124,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     }
     {
       TimeScope ts(h, st, FT_TIME_FFN_RES);
-      const size_t fixed = tc_down_fixed_bytes(qp.max_items, c.inter);
+      const size_t fixed = tc_down_fixed_bytes(c.inter);
       tp.n_stages = (int)std::min<size_t>(kTcMaxStages, (kTcSmem - fixed) / kTcStageD);
       cudaLaunchConfig_t lc = {};
       lc.gridDim = dim3(h->sm_count); lc.blockDim = dim3(kTcThreads); lc.stream = st;
