@@ -152,6 +152,7 @@ struct TcParams {
   const uint8_t *xq;   // activation images of the kTcParts parts of the hidden dimension (tc_quant_x_kernel)
   int d;
   int n_stages;        // ring stages (what fits in shared memory, at most kTcMaxStages)
+  int *pass_done;      // per pass: groups of 128 neurons whose h the gate/up kernel has written (0 between calls)
 };
 
 // ---- PTX wrappers of the block-scaled path ----
@@ -433,7 +434,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
             *reinterpret_cast<uint32_t *>(sf + (nn & 31) * 16 + (nn >> 5) * 4) = w4;
           }
         }
-        if (et == 0) p.hcount[pass * NG + ng] = 0;
+        // publish: the down kernel starts a pass when all its groups are there (it does not wait for this grid to end)
+        __threadfence();
+        tc_epi_barrier();
+        if (et == 0) {
+          p.hcount[pass * NG + ng] = 0;
+          atomicAdd(q.pass_done + pass, 1);
+        }
       }
       ++seg;
       return true;
@@ -510,13 +517,29 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
 
   if (warp < 4) {
     // ---- loaders ----
-    if (tid == 0) asm volatile("griddepcontrol.wait;" ::: "memory");   // h is written by the gate/up kernel
     uint32_t it = 0, n_h = 0, cur = 0xffffffffu;
     walk([&](uint32_t pass, uint32_t cg, uint32_t st0, uint32_t n) {
       if (pass != cur && tid == 0) {
         // the pass's h image replaces the previous one once the MMAs that read that have completed (a wait that
         // gives up latches the abort flag: every loader then leaves at its next wait)
         if (!n_h || mbar_wait(hempty_bar, (n_h - 1u) & 1u, s_abort, p.status)) {
+          // h of this pass is written by the gate/up kernel, which precedes this kernel in the stream and is at least
+          // running (this kernel is its programmatic dependent): wait, bounded, for the pass's groups
+          {
+            const uint32_t limit = g_wait_polls;
+            uint32_t polls = 0;
+            int have;
+            do {
+              asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(have) : "l"(q.pass_done + pass) : "memory");
+              if (have >= (int)NG) break;
+              __nanosleep(64);
+            } while (++polls < limit && !*s_abort);
+            if (have < (int)NG && !*s_abort) {
+              *s_abort = 1;
+              atomicOr(p.status, kStatTimeout);
+            }
+            asm volatile("fence.proxy.async;" ::: "memory");   // the copies below read what those generic stores wrote
+          }
           mbar_expect_tx(hfull_bar, h_bytes);
           const uint8_t *hsrc = p.hq + (size_t)pass * h_bytes;
           for (uint32_t o = 0; o < h_bytes; o += 16384u) bulk_g2s(smem_u32(s_b) + o, hsrc + o, min(16384u, h_bytes - o), hfull_bar);
@@ -663,6 +686,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
     reinterpret_cast<uint2 *>(p.y)[i] = o;
     reinterpret_cast<float4 *>(p.y_acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
   }
+  for (int i = tid; i < n_items + n_zc; i += kTcThreads) q.pass_done[i] = 0;
   if (tid == 0) *p.done = 0u;
 }
 

@@ -98,7 +98,8 @@ struct ft_moe {
   float *w4_hraw = nullptr;
   int32_t *w4_hcount = nullptr;
   uint8_t *w4_hq = nullptr;
-  uint8_t *tc_xq = nullptr;      // FT_W_MXFP4_TC: the bit-sliced activation images of a call (two K halves)
+  uint8_t *tc_xq = nullptr;      // FT_W_MXFP4_TC: the bit-sliced activation images of a call
+  int *tc_pass_done = nullptr;   // FT_W_MXFP4_TC: per pass, the groups whose h is written (hand-over between the two kernels)
   float2 *w4_hs = nullptr;
   int last_fill_layer = -1;
   int overlap = 0;                      // launch mode of the streaming kernel (see FfnStreamParams::overlap)
@@ -502,6 +503,7 @@ ft_status_t ft_moe_destroy(ft_moe_t *h) {
   cudaFree(h->w4_hcount);
   cudaFree(h->w4_hq);
   cudaFree(h->tc_xq);
+  cudaFree(h->tc_pass_done);
   cudaFree(h->w4_hs);
   cudaFree(h->trace_dev);
   cudaFree(h->stage_logits);
@@ -678,6 +680,8 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
       FT_TRY(cudaMemset(h->w4_hq, 0, passes * tc_h_pass_bytes(c.inter)));
       FT_TRY(cudaMalloc(&h->tc_xq, kTcParts * tc_x_part_bytes(c.hidden)));
       FT_TRY(cudaMemset(h->tc_xq, 0, kTcParts * tc_x_part_bytes(c.hidden)));
+      FT_TRY(cudaMalloc(&h->tc_pass_done, passes * sizeof(int)));
+      FT_TRY(cudaMemset(h->tc_pass_done, 0, passes * sizeof(int)));
       if (tc_gateup_fixed_bytes(c.hidden) + 3 * kTcStageA > kTcSmem ||
           tc_down_fixed_bytes(c.inter) + 3 * kTcStageD > kTcSmem || c.inter / 128 > 48 || h->sm_count < kTcParts)
         return fail(FT_ERR_UNSUPPORTED);
@@ -759,6 +763,14 @@ ft_status_t ft_moe_reset(ft_moe_t *h, int layer) {
     }
   if (h->cfg.global_pool) FT_CUDA(cudaMemset(h->layers[0].clock, 0, 8));
   FT_CUDA(cudaMemset(h->y_acc, 0, (size_t)h->cfg.max_tokens * h->cfg.hidden * 4));
+  FT_CUDA(cudaMemset(h->done_dev, 0, 4));
+  if (h->w4_hraw) {   // the hand-over buffers of the 4-bit kernels (a call that gave up may have left partial sums)
+    const ft_moe_config_t &c = h->cfg;
+    const size_t passes = ((size_t)c.max_tokens * c.top_k + 7) / 8 + 2 * (size_t)c.n_experts + 2;
+    FT_CUDA(cudaMemset(h->w4_hraw, 0, passes * (c.inter / 16) * 1024));
+    FT_CUDA(cudaMemset(h->w4_hcount, 0, passes * (c.inter / 128) * 4));
+    if (h->tc_pass_done) FT_CUDA(cudaMemset(h->tc_pass_done, 0, passes * sizeof(int)));
+  }
   FT_CUDA(cudaDeviceSynchronize());
   return FT_OK;
 }
@@ -1110,7 +1122,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
       FT_CUDA(cudaLaunchKernelEx(&lc, tc_quant_x_kernel, tq));
     }
     TcParams tp;
-    tp.w = qp; tp.xq = h->tc_xq; tp.d = c.hidden;
+    tp.w = qp; tp.xq = h->tc_xq; tp.d = c.hidden; tp.pass_done = h->tc_pass_done;
     const int grid = h->sm_count - h->sm_count % kTcParts;   // CTA i works on part i % kTcParts of the hidden dimension
     {
       TimeScope ts(h, st, FT_TIME_FFN_ZC);
