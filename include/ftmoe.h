@@ -324,7 +324,9 @@ ft_status_t ft_moe_set_launch_overlap(ft_moe_t *h, int mode);
  * call that timed out is unspecified; ft_moe_sync_status reports FT_ERR_TIMEOUT once, and after ft_moe_reset
  * the handle works as before.  Waits for the device. */
 enum { FT_DEBUG_WITHHOLD_FILL = 1,      /* device-driven fill kernel (FT_FILL_SM) */
-       FT_DEBUG_WITHHOLD_GEMM = 4 };    /* prefill gate/up grouped GEMM */
+       FT_DEBUG_WITHHOLD_GEMM = 4,      /* prefill gate/up grouped GEMM */
+       FT_DEBUG_WITHHOLD_TC = 8 };      /* gate/up kernel of the FT_W_MXFP4_TC decode path (its down kernel then waits,
+                                           bounded, for h that never comes) */
 /* (The bf16 and int4 streaming kernels load weights straight into registers and contain no waits.) */
 ft_status_t ft_moe_debug_inject(ft_moe_t *h, uint32_t withhold_mask, uint32_t wait_polls);
 /* Number of kernels this handle has launched since create. */

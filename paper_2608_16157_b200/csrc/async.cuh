@@ -13,7 +13,7 @@ constexpr uint32_t kDefaultWaitPolls = 1u << 22;
 // Test hook (ft_moe_debug_inject): bits that make one producer withhold a single copy, so that the consumer's
 // bounded wait runs out and the error path can be exercised without faulting, trapping or hanging anything.
 static __device__ uint32_t g_debug_withhold = 0;
-constexpr uint32_t kWithholdFill = 1u, kWithholdGemm = 4u;
+constexpr uint32_t kWithholdFill = 1u, kWithholdGemm = 4u, kWithholdTc = 8u;
 
 // After a bounded wait has given up: give the copies this CTA has already issued time to land before its shared
 // memory is released (bounded: about 50 us).

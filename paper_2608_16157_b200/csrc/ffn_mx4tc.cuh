@@ -308,6 +308,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
           bool ok = true;
           if (lane == 0) ok = mbar_wait(bar.empty(slot), ((it / NS) & 1u) ^ 1u, s_abort, p.status);
           if (!__shfl_sync(0xffffffffu, (int)ok, 0)) return false;
+          if ((g_debug_withhold & kWithholdTc) && it == 0) continue;   // test hook: this stage never arrives
           tc_load_stage<kTcStageA>(smem_u32(s_ring) + slot * kTcStageA, src, lane, bar.full(slot));
         }
         if (!x_sent && it + 1 == NS) send_x();   // after the first ring fill

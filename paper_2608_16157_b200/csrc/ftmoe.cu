@@ -1431,7 +1431,7 @@ ft_status_t ft_moe_set_launch_overlap(ft_moe_t *h, int mode) {
 }
 
 ft_status_t ft_moe_debug_inject(ft_moe_t *h, uint32_t withhold_mask, uint32_t wait_polls) {
-  if (!h || (withhold_mask & ~7u)) return FT_ERR_INVALID_ARG;
+  if (!h || (withhold_mask & ~15u)) return FT_ERR_INVALID_ARG;
   FT_CUDA(cudaSetDevice(h->cfg.device));
   FT_CUDA(cudaDeviceSynchronize());
   const uint32_t polls = wait_polls ? wait_polls : kDefaultWaitPolls;

@@ -11,7 +11,7 @@ from tests.helpers import Pair
 
 pytestmark = pytest.mark.gpu
 
-FT_DEBUG_WITHHOLD_FILL, FT_DEBUG_WITHHOLD_GEMM = 1, 4
+FT_DEBUG_WITHHOLD_FILL, FT_DEBUG_WITHHOLD_GEMM, FT_DEBUG_WITHHOLD_TC = 1, 4, 8
 
 
 def _reset_both(pr):
@@ -58,4 +58,18 @@ def test_prefill_gemm_wait_runs_out_and_the_handle_recovers():
     _run_expect_timeout(pr, FT_DEBUG_WITHHOLD_GEMM, 128, logits, x)
     _reset_both(pr)
     pr.step(0, logits, x)
+    pr.close()
+
+
+def test_tensor_core_decode_waits_run_out_and_the_handle_recovers():
+    """FT_W_MXFP4_TC: one stage of the gate/up kernel's ring never arrives: its MMA issuers and epilogue give up, the
+    down kernel gives up waiting for h, both kernels return, the status says so, and after a reset (which also clears
+    the partial sums of the hand-over buffers) the handle is correct again."""
+    shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2, wdtype="mxfp4tc", n_shared=1)
+    pr = Pair(shape, n_slots=4, max_tokens=8, seed=9)
+    pr.step(0, W.normal_logits(6, 8, 9, 0), W.noise_x(6, 512, 9, 0, 0))
+    _run_expect_timeout(pr, FT_DEBUG_WITHHOLD_TC, 6, W.normal_logits(6, 8, 9, 1), W.noise_x(6, 512, 9, 1, 0))
+    _reset_both(pr)
+    for step in range(2):
+        pr.step(0, W.normal_logits(6, 8, 9, step), W.noise_x(6, 512, 9, step, 0), check_slots=True)
     pr.close()
