@@ -185,10 +185,11 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    dsv3 = args.workload in ("dsv3", "dsv3_mxfp4", "dsv3_nvfp4")
-    mxfp4 = args.workload in ("dsv3_mxfp4", "dsv3_nvfp4")    # the floating-point 4-bit formats share their kernels
-    fp4_name = "nvfp4" if args.workload == "dsv3_nvfp4" else "mxfp4"
-    shape = {"dsv3": W.DSV3_INT4, "dsv3_mxfp4": W.DSV3_MXFP4, "dsv3_nvfp4": W.DSV3_NVFP4}[args.workload] if dsv3 else W.QWEN3_30B
+    dsv3 = args.workload in ("dsv3", "dsv3_mxfp4", "dsv3_nvfp4", "dsv3_mxfp4tc")
+    mxfp4 = args.workload in ("dsv3_mxfp4", "dsv3_nvfp4", "dsv3_mxfp4tc")    # the floating-point 4-bit formats
+    fp4_name = {"dsv3_nvfp4": "nvfp4", "dsv3_mxfp4tc": "mxfp4 (tensor-core operand images)"}.get(args.workload, "mxfp4")
+    shape = {"dsv3": W.DSV3_INT4, "dsv3_mxfp4": W.DSV3_MXFP4, "dsv3_nvfp4": W.DSV3_NVFP4,
+             "dsv3_mxfp4tc": W.DSV3_MXFP4TC}[args.workload] if dsv3 else W.QWEN3_30B
     RHO, ALPHA = (0.9, 1.2) if dsv3 else (0.8, 1.1)
     L = (4 if args.layers == 48 else args.layers) if dsv3 else args.layers
     E, k, d = shape.n_experts, shape.top_k, shape.d
@@ -219,7 +220,8 @@ def run_ours(args):
         cfg = Bd.make_config(hidden=d, inter=shape.inter, n_experts=E, top_k=k, n_layers=L, slots_per_layer=Ns,
                              max_tokens=max(B, 8), host_pool_ptr=pool.ptr.value, host_pool_bytes=pool.n_bytes,
                              fill_mode=fill_mode, device=local,
-                             wdtype={"int4": Bd.FT_W_INT4_G128, "mxfp4": Bd.FT_W_MXFP4, "nvfp4": Bd.FT_W_NVFP4, "bf16": Bd.FT_W_BF16}[shape.wdtype],
+                             wdtype={"int4": Bd.FT_W_INT4_G128, "mxfp4": Bd.FT_W_MXFP4, "nvfp4": Bd.FT_W_NVFP4, "mxfp4tc": Bd.FT_W_MXFP4_TC,
+                                     "bf16": Bd.FT_W_BF16}[shape.wdtype],
                              n_shared=shape.n_shared, shared_ptr=None if shared is None else shared.data_ptr(),
                              global_pool=args.global_pool, **bw)
         return Bd.FtMoe(cfg)
@@ -514,7 +516,8 @@ def run_ours(args):
             "gpu_launches": main["launches"],
             "roofline": {
                 "bound": "hbm",
-                "kernel": ("mx4_gateup_kernel + mx4_down_kernel (one pass over each record)" if mxfp4 else
+                "kernel": ("tc_gateup_kernel + tc_down_kernel (one pass over each record)" if args.workload == "dsv3_mxfp4tc" else
+                           "mx4_gateup_kernel + mx4_down_kernel (one pass over each record)" if mxfp4 else
                            "w4_gateup_kernel + w4_down_kernel (one pass over each record)" if dsv3
                            else "ffn_stream_kernel (expert FFN over the HBM-resident records of a layer)"),
                 "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
@@ -612,7 +615,8 @@ def prefill_passes(args, dev, L, cal=None, shape=None, Ns=None):
     common = dict(hidden=d, inter=I, n_experts=E, top_k=k, n_layers=L, slots_per_layer=Ns, max_tokens=T,
                   host_pool_ptr=pool.ptr.value, host_pool_bytes=pool.n_bytes,
                   fill_mode=Bd.FT_FILL_SM if args.fill == "sm" else Bd.FT_FILL_COPY_ENGINE,
-                  wdtype={"int4": Bd.FT_W_INT4_G128, "mxfp4": Bd.FT_W_MXFP4, "nvfp4": Bd.FT_W_NVFP4, "bf16": Bd.FT_W_BF16}[shape.wdtype],
+                  wdtype={"int4": Bd.FT_W_INT4_G128, "mxfp4": Bd.FT_W_MXFP4, "nvfp4": Bd.FT_W_NVFP4, "mxfp4tc": Bd.FT_W_MXFP4_TC,
+                                     "bf16": Bd.FT_W_BF16}[shape.wdtype],
                   gemm_min_tokens=args.gemm_min_tokens)
     if shape.n_shared:
         shared = W.make_shared_records(shape, L, SEED, device=dev)
@@ -1011,7 +1015,7 @@ def main():
     ap.add_argument("--sweep-batches", default="1,16,64")
     ap.add_argument("--global-pool", type=int, default=0, help="1: one slot pool and LRU clock shared by all layers")
     ap.add_argument("--graph", type=int, default=1, help="replay each decode step as one CUDA graph (SM fill only)")
-    ap.add_argument("--workload", default="qwen", choices=["qwen", "dsv3", "dsv3_mxfp4", "dsv3_nvfp4"])
+    ap.add_argument("--workload", default="qwen", choices=["qwen", "dsv3", "dsv3_mxfp4", "dsv3_nvfp4", "dsv3_mxfp4tc"])
     ap.add_argument("--mode", default="decode", choices=["decode", "prefill", "sweep"])
     ap.add_argument("--tokens", type=int, default=4096)
     ap.add_argument("--gemm-min-tokens", type=int, default=32)
