@@ -34,6 +34,13 @@ def test_config_struct_matches_header_size_and_expert_bytes():
     cfg = B.make_config(hidden=7168, inter=2048, n_experts=256, top_k=8, slots_per_layer=64, max_tokens=8,
                         host_pool_ptr=None, host_pool_bytes=0, wdtype=B.FT_W_INT4_G128)
     assert B.ft_moe_expert_bytes(cfg) == 22708224
+    # the library's record sizes and the generator's agree for every weight format
+    from paper_2608_16157_b200 import workload as W
+    for wd, name in ((B.FT_W_MXFP4, "mxfp4"), (B.FT_W_MXFP4_TC, "mxfp4tc"), (B.FT_W_NVFP4, "nvfp4"), (B.FT_W_INT4_G128, "int4")):
+        for d, inter in ((7168, 2048), (512, 256)):
+            cfg = B.make_config(hidden=d, inter=inter, n_experts=8, top_k=2, slots_per_layer=4, max_tokens=8,
+                                host_pool_ptr=None, host_pool_bytes=0, wdtype=wd)
+            assert B.ft_moe_expert_bytes(cfg) == W.LayerShape(d, inter, 8, 2, name).expert_bytes
     cfg = B.make_config(hidden=100, inter=768, n_experts=128, top_k=8, slots_per_layer=64, max_tokens=8,
                         host_pool_ptr=None, host_pool_bytes=0)
     assert B.ft_moe_expert_bytes(cfg) == 0
