@@ -1,4 +1,4 @@
-// Steps 5+6 for MXFP4 experts stored as tensor-core operand images (FT_W_MXFP4_TC), decode-sized calls (T <= 8):
+// Steps 5+6 for MXFP4 experts stored as tensor-core operand images (FT_W_MXFP4_TC), 8 tokens of an expert per pass:
 // the block-scaled 5th-generation tensor-core instruction tcgen05.mma kind::mxf4 multiplies packed e2m1 weights by
 // e2m1 activations, both with one power-of-two scale per 32 elements held in tensor memory, so the weights need no
 // unpacking at all: a record's bytes go from HBM (or, for zero-copy experts, from the mapped host pool) to shared
@@ -10,6 +10,9 @@
 //     Every term removes at least a factor 3 of the block's largest leftover, so 6 terms leave <= 2^-9.5 of the
 //     block's largest magnitude; the terms of the 8 tokens are the N = 48 columns of the MMA (column 8 i + token),
 //     and the epilogue adds a token's 6 columns.  The tensor pipe has room for this: the kernels are HBM-bound.
+//     A call with at most 8 tokens has one activation image (its tokens, for every expert); a larger call one image
+//     per pass (8 tokens of the pass's expert, gathered through the expert-sorted permutation), which a CTA brings
+//     into shared memory when its tiles change pass.
 //   * Gate/up kernel: M = 128 neurons of the gate and of the up matrix per tile, K split into four parts (a CTA
 //     keeps the activation image of one part in shared memory: CTA i that of part i % 4, which leaves most of the
 //     shared memory to the ring), each CTA an equal share of (tile, 128-index stage) steps of its part.  A producer
@@ -97,25 +100,73 @@ __device__ __forceinline__ void tc_term(float (&r)[8], bool bad, uint32_t &codes
   }
 }
 
-// x [T][d] bf16 -> the gate/up kernel's activation images of both K halves.  One thread per 8 consecutive hidden
-// indices of a token slot (slots >= T are written as zeros); a quad of lanes is one block of 32.
-struct TcQuantParams {
-  const __nv_bfloat16 *x;
-  uint8_t *xq;      // [kTcParts][tc_x_part_bytes(d)]
-  int T, d;
+// Tokens of a pass: with at most 8 tokens in the call ("dense") the 8 columns are the call's tokens for every pass;
+// otherwise a pass serves 8 tokens of its list entry (pass = the entry's first pass + k: tokens 8k .. 8k+7 of the
+// entry, gathered through the expert-sorted permutation; the shared expert's entry holds the tokens themselves).
+struct TcPassTokens {
+  int nt;        // columns in use
+  int tok[8];    // token of column j, or -1
+  float w[8];    // its gate weight
 };
-__global__ void __launch_bounds__(256) tc_quant_x_kernel(TcQuantParams p) {
+__device__ __forceinline__ void tc_pass_tokens(const W4Params &p, bool dense, uint32_t pass, bool want_weights, TcPassTokens &o) {
+#pragma unroll
+  for (int j = 0; j < 8; ++j) { o.tok[j] = -1; o.w[j] = 0.f; }
+  const int n_lists = *p.n_items + *p.n_zc;
+  const int item = dense ? (int)pass : w4_find_item(p.pref, n_lists, pass);
+  const WorkItem wi = p.items[item];
+  const int tok0 = dense ? 0 : (int)(pass - (uint32_t)p.pref[item]) * 8;
+  const int cnt = min(8, wi.n_tok - tok0);
+  o.nt = dense ? p.T : cnt;
+  if (wi.expert < 0) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      if (j < cnt) { o.tok[j] = tok0 + j; o.w[j] = 1.f; }
+    return;
+  }
+  for (int j = 0; j < cnt; ++j) {
+    const int pr = p.perm[wi.off + tok0 + j];
+    const int tk = pr / p.top_k;
+    const float wv = want_weights ? p.topk_w[pr] : 1.f;
+    const int col = dense ? tk : j;       // dense: column = token
+#pragma unroll
+    for (int c = 0; c < 8; ++c)
+      if (c == col) { o.tok[c] = tk; o.w[c] = wv; }
+  }
+}
+
+// x [T][d] bf16 -> the gate/up kernel's activation images: image i (blockIdx.y) holds the 8 token columns of pass i
+// (dense: one image, columns = the call's tokens), each as kTcParts parts of the hidden dimension.  One thread per 8
+// consecutive hidden indices of a column (unused columns are written as zeros); a quad of lanes is one block of 32.
+struct TcQuantParams {
+  W4Params w;
+  const __nv_bfloat16 *x;
+  uint8_t *xq;      // [images][kTcParts][tc_x_part_bytes(d)]
+  int d, dense;
+};
+__global__ void __launch_bounds__(256) tc_quant_x_kernel(TcQuantParams q) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // (when launched as a programmatic dependent: the images are still being read until the kernels before have completed)
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  const int per_tok = p.d / 8;
+  const W4Params &p = q.w;
+  const uint32_t pass = blockIdx.y;
+  if (!q.dense && pass >= (uint32_t)p.pref[*p.n_items + *p.n_zc]) return;
+  const int per_tok = q.d / 8;
   const int i = blockIdx.x * 256 + threadIdx.x;
   if (i >= 8 * per_tok) return;
-  const int tok = i / per_tok, c8 = i - tok * per_tok;   // hidden indices 8 c8 .. 8 c8 + 7
+  const int col = i / per_tok, c8 = i - col * per_tok;   // hidden indices 8 c8 .. 8 c8 + 7 of column col
+  int tok;
+  if (q.dense) {
+    tok = col < p.T ? col : -1;
+  } else {
+    __shared__ TcPassTokens s_pt;
+    if (threadIdx.x == 0) tc_pass_tokens(p, false, pass, false, s_pt);
+    __syncthreads();
+    tok = s_pt.tok[col];
+  }
   float r[8];
   bool bad = false;
-  if (tok < p.T) {
-    const uint4 v = *reinterpret_cast<const uint4 *>(p.x + (size_t)tok * p.d + 8 * c8);
+  if (tok >= 0) {
+    const uint4 v = *reinterpret_cast<const uint4 *>(q.x + (size_t)tok * q.d + 8 * c8);
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
@@ -129,18 +180,18 @@ __global__ void __launch_bounds__(256) tc_quant_x_kernel(TcQuantParams p) {
     for (int e = 0; e < 8; ++e) r[e] = 0.f;
   }
   bad = (__shfl_xor_sync(0xffffffffu, (int)bad, 1) | __shfl_xor_sync(0xffffffffu, (int)bad, 2) | (int)bad) != 0;
-  const int part_k = p.d / kTcParts;
+  const int part_k = q.d / kTcParts;
   const int k = 8 * c8, part = k / part_k, kk = k - part * part_k;
-  uint8_t *img = p.xq + (size_t)part * tc_x_part_bytes(p.d);
+  uint8_t *img = q.xq + ((size_t)(q.dense ? 0u : pass) * kTcParts + part) * tc_x_part_bytes(q.d);
   uint8_t *sf = img + (size_t)(part_k / 64) * kTcStepB;
   const int step = kk >> 6, kcore = (kk >> 5) & 1, word = (kk & 31) >> 3;
 #pragma unroll
   for (int t = 0; t < kTcTerms; ++t) {
     uint32_t codes, sb;
     tc_term(r, bad, codes, sb);
-    *reinterpret_cast<uint32_t *>(img + (size_t)step * kTcStepB + kcore * (kTcN * 16) + t * 128 + tok * 16 + word * 4) = codes;
+    *reinterpret_cast<uint32_t *>(img + (size_t)step * kTcStepB + kcore * (kTcN * 16) + t * 128 + col * 16 + word * 4) = codes;
     if ((threadIdx.x & 3) == 0) {
-      const int n = 8 * t + tok, blk = kk >> 5;   // scale of (column n, block blk of the part)
+      const int n = 8 * t + col, blk = kk >> 5;   // scale of (column n, block blk of the part)
       sf[(size_t)(blk >> 2) * 512 + (n & 31) * 16 + (n >> 5) * 4 + (blk & 3)] = (uint8_t)sb;
     }
   }
@@ -149,7 +200,8 @@ __global__ void __launch_bounds__(256) tc_quant_x_kernel(TcQuantParams p) {
 
 struct TcParams {
   W4Params w;          // the work lists, the hand-over buffers (hraw, hcount, hq) and the output, as for the other 4-bit kernels
-  const uint8_t *xq;   // activation images of the kTcParts parts of the hidden dimension (tc_quant_x_kernel)
+  const uint8_t *xq;   // activation images (tc_quant_x_kernel): one per pass, or one for all passes when dense
+  int dense;           // at most 8 tokens in the call: the MMA's token columns are the call's tokens for every pass
   int d;
   int n_stages;        // ring stages (what fits in shared memory, at most kTcMaxStages)
   int *pass_done;      // per pass: groups of 128 neurons whose h the gate/up kernel has written (0 between calls)
@@ -243,18 +295,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const TcBars bar{smem_u32(s_bar)};
-  const uint32_t x_bar = bar.extra(0), sfb_bar = bar.extra(1);
+  const uint32_t x_bar = bar.extra(0), sfb_bar = bar.extra(1), xempty_bar = bar.extra(2);
   if (tid == 0) {
     for (uint32_t s = 0; s < NS; ++s) { mbar_init(bar.full(s), 32); mbar_init(bar.empty(s), 2); }
     for (uint32_t b = 0; b < 2; ++b) { mbar_init(bar.tfull(b), 2); mbar_init(bar.tempty(b), 4); }
     mbar_init(x_bar, 1);
     mbar_init(sfb_bar, 1);
+    mbar_init(xempty_bar, 2);
     *s_abort = 0;
     *s_last = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // (decode-sized calls: every list entry is one pass of at most 8 tokens, so pass = index into the list)
   const int n_items = *p.n_items, n_zc = *p.n_zc;
+  const bool dense = q.dense != 0;   // then every list entry is one pass: pass = index into the list
   if (warp == 4) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(s_tmem)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -272,9 +325,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
   const uint32_t part = blockIdx.x % kTcParts, ci = blockIdx.x / kTcParts, nc = gridDim.x / kTcParts;
   uint32_t pass0[2], s_begin[2], s_end[2];
   pass0[0] = 0u;
-  pass0[1] = (uint32_t)n_items;
+  pass0[1] = (uint32_t)p.pref[n_items];
   {
-    const uint32_t t0 = (uint32_t)n_items * NG * SPH, t1 = (uint32_t)n_zc * NG * SPH;
+    const uint32_t t0 = pass0[1] * NG * SPH, t1 = ((uint32_t)p.pref[n_items + n_zc] - pass0[1]) * NG * SPH;
     s_begin[0] = w4_first(t0, nc, ci); s_end[0] = w4_first(t0, nc, ci + 1);
     s_begin[1] = w4_first(t1, nc, ci); s_end[1] = w4_first(t1, nc, ci + 1);
   }
@@ -289,19 +342,33 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
   };
 
   if (warp < 4) {
-    // ---- loaders: the weights do not depend on the preceding kernels; the activation image does ----
-    uint32_t it = 0;
-    bool x_sent = tid != 0;
-    auto send_x = [&]() {
-      asm volatile("griddepcontrol.wait;" ::: "memory");
-      const uint32_t bytes = (uint32_t)tc_x_part_bytes(d);
-      mbar_expect_tx(x_bar, bytes);
-      const uint8_t *src = q.xq + (size_t)part * bytes;
-      for (uint32_t o = 0; o < bytes; o += 16384u) bulk_g2s(smem_u32(s_b) + o, src + o, min(16384u, bytes - o), x_bar);
-      x_sent = true;
+    // ---- loaders: the weights do not depend on the preceding kernels; the activation images do ----
+    // Thread 0 also brings the activation image (of the pass, or the one image of a dense call) into shared memory:
+    // the first one after the first ring fill (so that the weights start to stream while the kernel before still
+    // runs), a later one once the MMAs that read its predecessor have completed.
+    uint32_t it = 0, n_x = 0, cur = 0xffffffffu, pending = 0xffffffffu;
+    bool waited = false;
+    auto send_x = [&](uint32_t img) {
+      if (!waited) { asm volatile("griddepcontrol.wait;" ::: "memory"); waited = true; }
+      // (a wait that gives up latches the abort flag: every loader then leaves at its next wait)
+      if (!n_x || mbar_wait(xempty_bar, (n_x - 1u) & 1u, s_abort, p.status)) {
+        const uint32_t bytes = (uint32_t)tc_x_part_bytes(d);
+        mbar_expect_tx(x_bar, bytes);
+        const uint8_t *src = q.xq + ((size_t)img * kTcParts + part) * bytes;
+        for (uint32_t o = 0; o < bytes; o += 16384u) bulk_g2s(smem_u32(s_b) + o, src + o, min(16384u, bytes - o), x_bar);
+        ++n_x;
+      }
     };
     walk([&](uint32_t pass, uint32_t ng, uint32_t st0, uint32_t n) {
-      const uint8_t *src = p.items[pass].w + ((size_t)ng * KS + part * SPH + st0) * kTcStageA;
+      const uint32_t img = dense ? 0u : pass;
+      if (tid == 0 && img != cur) {
+        if (pending != 0xffffffffu) { send_x(pending); pending = 0xffffffffu; }
+        if (cur == 0xffffffffu) pending = img;   // the first image is sent below, after the first ring fill
+        else send_x(img);
+        cur = img;
+      }
+      const int item = dense ? (int)pass : w4_find_item(p.pref, n_items + n_zc, pass);
+      const uint8_t *src = p.items[item].w + ((size_t)ng * KS + part * SPH + st0) * kTcStageA;
       for (uint32_t s = 0; s < n; ++s, ++it, src += kTcStageA) {
         const uint32_t slot = it % NS;
         if (it % (kTcLoaders / 32) == (uint32_t)warp) {
@@ -311,37 +378,40 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
           if ((g_debug_withhold & kWithholdTc) && it == 0) continue;   // test hook: this stage never arrives
           tc_load_stage<kTcStageA>(smem_u32(s_ring) + slot * kTcStageA, src, lane, bar.full(slot));
         }
-        if (!x_sent && it + 1 == NS) send_x();   // after the first ring fill
+        if (tid == 0 && pending != 0xffffffffu && it + 1 == NS) { send_x(pending); pending = 0xffffffffu; }
       }
       return true;
     });
-    if (!x_sent) send_x();
+    if (tid == 0 && pending != 0xffffffffu) send_x(pending);
     // the copies issued must have landed before this CTA's shared memory is released
     asm volatile("cp.async.wait_all;" ::: "memory");
     if (tid == 0) {
-      (void)mbar_wait(x_bar, 0u, s_abort, p.status);
+      if (n_x) (void)mbar_wait(x_bar, (n_x - 1u) & 1u, s_abort, p.status);
       abort_drain(s_abort);
     }
   } else if (warp <= 5) {
     if (lane == 0) {
       // ---- MMA issuers: warp 4 the gate matrix, warp 5 the up matrix ----
       const uint32_t mat = (uint32_t)warp - 4u;
-      bool ok;
-      if (mat == 0) {
-        ok = mbar_wait(x_bar, 0u, s_abort, p.status);
-        if (ok) {
-          tc_fence_after();
-          for (uint32_t a = 0; a < SPH; ++a) tc_cp_scales(t_sfb + 4u * a, smem_u32(s_sfb) + a * 512u);
-          umma_commit(sfb_bar);   // the other issuer's MMAs read these scales too
-        }
-      } else {
-        ok = mbar_wait(sfb_bar, 0u, s_abort, p.status);
-        if (ok) tc_fence_after();
-      }
-      uint32_t it = 0, seg = 0;
+      uint32_t it = 0, seg = 0, n_x = 0, cur = 0xffffffffu;
       const uint32_t b_base = smem_u32(s_b), ring = smem_u32(s_ring) + mat * 8192u, t_sf = t_sfa + mat * 64u;
-      if (ok)
-        walk([&](uint32_t, uint32_t, uint32_t st0, uint32_t n) {
+      walk([&](uint32_t pass, uint32_t, uint32_t st0, uint32_t n) {
+          const uint32_t img = dense ? 0u : pass;
+          if (img != cur) {
+            // a new activation image: its scales go to tensor memory once the MMAs on the old one are done
+            if (n_x) umma_commit(xempty_bar);   // (count 2) arrives when every MMA this thread has issued so far has completed
+            if (mat == 0) {
+              if (!mbar_wait(x_bar, n_x & 1u, s_abort, p.status)) return false;
+              tc_fence_after();
+              for (uint32_t a = 0; a < SPH; ++a) tc_cp_scales(t_sfb + 4u * a, smem_u32(s_sfb) + a * 512u);
+              umma_commit(sfb_bar);   // the other issuer's MMAs read these scales too
+            } else {
+              if (!mbar_wait(sfb_bar, n_x & 1u, s_abort, p.status)) return false;
+              tc_fence_after();
+            }
+            cur = img;
+            ++n_x;
+          }
           const uint32_t buf = seg & 1u;
           if (!mbar_wait(bar.tempty(buf), ((seg >> 1) & 1u) ^ 1u, s_abort, p.status)) return false;
           tc_fence_after();
@@ -363,14 +433,20 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
           umma_commit(bar.tfull(buf));
           ++seg;
           return true;
-        });
+      });
     }
   } else {
     // ---- epilogue: thread = accumulator row (neuron of the tile) ----
     const int ew = warp & 3, row = ew * 32 + lane, et = (warp - 6) * 32 + lane;
-    uint32_t seg = 0;
+    uint32_t seg = 0, nt_pass = 0xffffffffu;
+    int nt = p.T;   // token columns of the pass in use
     walk([&](uint32_t pass, uint32_t ng, uint32_t, uint32_t n) {
       const uint32_t buf = seg & 1u;
+      if (!dense && pass != nt_pass) {
+        const int item = w4_find_item(p.pref, n_items + n_zc, pass);
+        nt = min(8, p.items[item].n_tok - (int)(pass - (uint32_t)p.pref[item]) * 8);
+        nt_pass = pass;
+      }
       bool ok = true;
       if (lane == 0) ok = mbar_wait(bar.tfull(buf), (seg >> 1) & 1u, s_abort, p.status);
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -384,7 +460,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
         __syncwarp();
         if (lane == 0) mbar_arrive(bar.tempty(buf));
         float *hacc = p.hraw + ((size_t)pass * NBLK + 8u * ng + (uint32_t)(row >> 4)) * 256 + (row & 15);
-        for (int t = 0; t < p.T; ++t) {
+        for (int t = 0; t < nt; ++t) {
           red_add_f32(hacc + t * 16, gsum[t]);
           red_add_f32(hacc + 128 + t * 16, usum[t]);
         }
@@ -484,7 +560,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  const int n_items = *p.n_items, n_zc = *p.n_zc;   // (pass = index into the list, see the gate/up kernel)
+  const int n_items = *p.n_items, n_zc = *p.n_zc;
+  const bool dense = q.dense != 0;   // then pass = index into the list, see the gate/up kernel
   if (warp == 4) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(s_tmem)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -500,9 +577,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
 
   uint32_t pass0[2], s_begin[2], s_end[2];
   pass0[0] = 0u;
-  pass0[1] = (uint32_t)n_items;
+  pass0[1] = (uint32_t)p.pref[n_items];
   {
-    const uint32_t t0 = (uint32_t)n_items * CG * DS, t1 = (uint32_t)n_zc * CG * DS;
+    const uint32_t t0 = pass0[1] * CG * DS, t1 = ((uint32_t)p.pref[n_items + n_zc] - pass0[1]) * CG * DS;
     s_begin[0] = w4_first(t0, gridDim.x, blockIdx.x); s_end[0] = w4_first(t0, gridDim.x, blockIdx.x + 1);
     s_begin[1] = w4_first(t1, gridDim.x, blockIdx.x); s_end[1] = w4_first(t1, gridDim.x, blockIdx.x + 1);
   }
@@ -548,7 +625,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
         }
       }
       cur = pass;
-      const uint8_t *src = p.items[pass].w + sec_b + ((size_t)cg * DS + st0) * kTcStageD;
+      const int item = dense ? (int)pass : w4_find_item(p.pref, n_items + n_zc, pass);
+      const uint8_t *src = p.items[item].w + sec_b + ((size_t)cg * DS + st0) * kTcStageD;
       for (uint32_t s = 0; s < n; ++s, ++it, src += kTcStageD) {
         const uint32_t slot = it % NS;
         if (it % (kTcLoaders / 32) == (uint32_t)warp) {
@@ -615,29 +693,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
     // ---- epilogue: thread = output column of the tile ----
     const int ew = warp & 3, row = ew * 32 + lane;
     uint32_t seg = 0, it = 0, gw_pass = 0xffffffffu;
-    float gw[8];
+    TcPassTokens pt;
     walk([&](uint32_t pass, uint32_t cg, uint32_t, uint32_t n) {
       const uint32_t buf = seg & 1u;
       if (pass != gw_pass) {
-        // gate weights of the pass's tokens (0 for the tokens that are not routed to this expert); a CTA's tiles
-        // mostly belong to one pass, so these dependent loads are rare
+        // the tokens of the pass's columns and their gate weights; a CTA's tiles mostly belong to one pass, so these
+        // dependent loads are rare
         gw_pass = pass;
-#pragma unroll
-        for (int t = 0; t < 8; ++t) gw[t] = 0.f;
-        const WorkItem wi = p.items[pass];
-        if (wi.expert >= 0) {
-          for (int j = 0; j < wi.n_tok && j < 8; ++j) {
-            const int pr = p.perm[wi.off + j];
-            const float wv = p.topk_w[pr];
-            const int tk = pr / p.top_k;
-#pragma unroll
-            for (int t = 0; t < 8; ++t)
-              if (t == tk) gw[t] = wv;
-          }
-        } else {
-#pragma unroll
-          for (int t = 0; t < 8; ++t) gw[t] = t < p.T ? 1.f : 0.f;
-        }
+        tc_pass_tokens(p, dense, pass, true, pt);
       }
       bool ok = true;
       if (lane == 0) ok = mbar_wait(bar.tfull(buf), (seg >> 1) & 1u, s_abort, p.status);
@@ -656,7 +719,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
       float *yc = p.y_acc + 128u * cg + row;
 #pragma unroll
       for (int t = 0; t < 8; ++t)
-        if (gw[t] != 0.f) red_add_f32(yc + (size_t)t * d, gw[t] * v[t]);
+        if (pt.tok[t] >= 0) red_add_f32(yc + (size_t)pt.tok[t] * d, pt.w[t] * v[t]);
       it += n;
       ++seg;
       return true;
@@ -666,8 +729,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
   __syncthreads();
   if (warp == 4) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
 
-  // ---- the last CTA to finish rounds the accumulator to bf16 and clears it ----
-  if (!p.finalize) return;
+  // ---- the last CTA to finish clears the passes' hand-over counters and, unless a finalize launch follows (more
+  // than 16 tokens), rounds the accumulator to bf16 and clears it ----
   __threadfence();
   __syncthreads();
   if (tid == 0) {
@@ -677,7 +740,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
   __syncthreads();
   if (!s_final) return;
   __threadfence();
-  const int n4 = p.T * (d / 4);
+  const int n4 = p.finalize ? p.T * (d / 4) : 0;
   for (int i = tid; i < n4; i += kTcThreads) {
     const float4 v = __ldcg(reinterpret_cast<const float4 *>(p.y_acc) + i);
     __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b2 = __floats2bfloat162_rn(v.z, v.w);
@@ -687,7 +750,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
     reinterpret_cast<uint2 *>(p.y)[i] = o;
     reinterpret_cast<float4 *>(p.y_acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
   }
-  for (int i = tid; i < n_items + n_zc; i += kTcThreads) q.pass_done[i] = 0;
+  for (int i = tid; i < p.pref[n_items + n_zc]; i += kTcThreads) q.pass_done[i] = 0;
   if (tid == 0) *p.done = 0u;
 }
 

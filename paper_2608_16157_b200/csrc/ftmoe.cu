@@ -547,8 +547,8 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
       (c.slots_per_layer == 0 || c.hidden % 256 || c.inter % 256 || c.gemm_min_tokens < 8 ||
        (c.wdtype != FT_W_BF16 && c.global_pool)))   // (4-bit: the bf16 scratch mirrors one layer's slots)
     return FT_ERR_UNSUPPORTED;
-  // the tensor-core-image records are served by the decode-sized kernels only
-  if (c.wdtype == FT_W_MXFP4_TC && (c.max_tokens > kQ4Tokens || c.gemm_min_tokens != 0)) return FT_ERR_UNSUPPORTED;
+  // the tensor-core-image records are served by the streaming (decode) kernels only
+  if (c.wdtype == FT_W_MXFP4_TC && c.gemm_min_tokens != 0) return FT_ERR_UNSUPPORTED;
   if (!c.host_pool || c.host_pool_bytes < (size_t)c.n_layers * c.n_experts * S) return FT_ERR_INVALID_ARG;
   if (c.n_shared && !c.shared_weights) return FT_ERR_INVALID_ARG;
   if ((long long)c.max_tokens * c.top_k > (1ll << 30)) return FT_ERR_INVALID_ARG;
@@ -678,8 +678,10 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
     FT_TRY(cudaMalloc(&h->w4_hq, c.wdtype == FT_W_MXFP4_TC ? passes * tc_h_pass_bytes(c.inter) : passes * (c.inter / 128) * 2048));
     if (c.wdtype == FT_W_MXFP4_TC) {
       FT_TRY(cudaMemset(h->w4_hq, 0, passes * tc_h_pass_bytes(c.inter)));
-      FT_TRY(cudaMalloc(&h->tc_xq, kTcParts * tc_x_part_bytes(c.hidden)));
-      FT_TRY(cudaMemset(h->tc_xq, 0, kTcParts * tc_x_part_bytes(c.hidden)));
+      // one activation image per pass, or a single one for handles that never see more than 8 tokens
+      const size_t n_img = c.max_tokens <= kQ4Tokens ? 1 : passes;
+      FT_TRY(cudaMalloc(&h->tc_xq, n_img * kTcParts * tc_x_part_bytes(c.hidden)));
+      FT_TRY(cudaMemset(h->tc_xq, 0, n_img * kTcParts * tc_x_part_bytes(c.hidden)));
       FT_TRY(cudaMalloc(&h->tc_pass_done, passes * sizeof(int)));
       FT_TRY(cudaMemset(h->tc_pass_done, 0, passes * sizeof(int)));
       if (tc_gateup_fixed_bytes(c.hidden) + 3 * kTcStageA > kTcSmem ||
@@ -1086,7 +1088,6 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   }
   // int4 / mxfp4: gate/up kernel writes h, down kernel accumulates, its last CTA finalizes y
   if (c.slots_per_layer > 0 && L.fill_recorded) FT_CUDA(cudaStreamWaitEvent(st, L.ev_fill, 0));
-  if (c.wdtype == FT_W_MXFP4_TC && L.T > kQ4Tokens) return FT_ERR_UNSUPPORTED;
   W4Params qp;
   qp.items = sc.items_res;
   qp.n_items = &sc.plan_dev->n_res_items;
@@ -1108,21 +1109,24 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   if (c.wdtype == FT_W_MXFP4_TC) {
     // bit-sliced activation images, then the two block-scaled tensor-core kernels (programmatic dependents: their
     // set-up and first weight copies overlap the kernel before them)
-    qp.finalize = 1;
+    const bool dense = L.T <= kQ4Tokens, tc_own_finalize = L.T > kFinalizeInKernelMaxTokens;
+    qp.finalize = tc_own_finalize ? 0 : 1;
     TcQuantParams tq;
-    tq.x = x_bf; tq.xq = h->tc_xq; tq.T = L.T; tq.d = c.hidden;
+    tq.w = qp; tq.x = x_bf; tq.xq = h->tc_xq; tq.d = c.hidden; tq.dense = dense ? 1 : 0;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
     {
       TimeScope ts(h, st, FT_TIME_GATHER);
       cudaLaunchConfig_t lc = {};
-      lc.gridDim = dim3(c.hidden / 256); lc.blockDim = dim3(256); lc.stream = st;
+      // (the number of passes is known on the device only: one block row per possible pass, the surplus returns at once)
+      const size_t max_passes = ((size_t)L.T * c.top_k + 7) / 8 + 2 * (size_t)c.n_experts + 2;
+      lc.gridDim = dim3(c.hidden / 256, dense ? 1u : (unsigned)max_passes); lc.blockDim = dim3(256); lc.stream = st;
       lc.attrs = at; lc.numAttrs = h->overlap ? 1 : 0;   // (it waits for the kernels before it by itself)
       FT_CUDA(cudaLaunchKernelEx(&lc, tc_quant_x_kernel, tq));
     }
     TcParams tp;
-    tp.w = qp; tp.xq = h->tc_xq; tp.d = c.hidden; tp.pass_done = h->tc_pass_done;
+    tp.w = qp; tp.xq = h->tc_xq; tp.d = c.hidden; tp.pass_done = h->tc_pass_done; tp.dense = dense ? 1 : 0;
     const int grid = h->sm_count - h->sm_count % kTcParts;   // CTA i works on part i % kTcParts of the hidden dimension
     {
       TimeScope ts(h, st, FT_TIME_FFN_ZC);
@@ -1145,6 +1149,12 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
       FT_CUDA(cudaLaunchKernelEx(&lc, tc_down_kernel, tp));
     }
     h->launches += 3;
+    if (tc_own_finalize) {
+      TimeScope ts(h, st, FT_TIME_FINALIZE);
+      const int n4 = L.T * (c.hidden / 4);
+      finalize_kernel<<<std::min((n4 + 255) / 256, h->sm_count * 8), 256, 0, st>>>(h->y_acc, qp.y, n4);
+      h->launches++;
+    }
     return FT_OK;
   }
   const bool half = !mx && L.T <= kW4HalfTokens;   // int4 with at most 4 tokens: one MMA per pair of weight words

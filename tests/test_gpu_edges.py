@@ -29,7 +29,7 @@ def test_256_experts_more_slots_than_experts_used():
     pr.close()
 
 
-@pytest.mark.parametrize("wdtype", ["bf16", "int4", "mxfp4", "nvfp4"])
+@pytest.mark.parametrize("wdtype", ["bf16", "int4", "mxfp4", "nvfp4", "mxfp4tc"])
 def test_zero_slots_everything_zero_copy_many_tokens(wdtype):
     """No cache at all: every expert is computed from the mapped host pool, more than 8 tokens per expert."""
     shape = W.LayerShape(d=512, inter=128, n_experts=4, top_k=2, wdtype=wdtype)

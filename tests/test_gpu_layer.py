@@ -119,7 +119,7 @@ def test_int4_group_dequant_and_shared_expert(n_shared, T, wdtype):
     pr.close()
 
 
-@pytest.mark.parametrize("wdtype", ["int4", "mxfp4", "nvfp4"])
+@pytest.mark.parametrize("wdtype", ["int4", "mxfp4", "nvfp4", "mxfp4tc"])
 @pytest.mark.parametrize("T", [9, 24, 40])
 def test_int4_resident_experts_with_many_tokens_and_shared_expert(T, wdtype):
     """More than 8 tokens per slot-resident 4-bit expert (several weight passes) and the shared expert at T > 8."""
@@ -210,10 +210,22 @@ def test_mxfp4_tensor_core_images_many_steps_device_fills_and_wide_shape():
     pr.close()
 
 
-def test_mxfp4_tensor_core_images_refuse_many_token_handles():
+def test_mxfp4_tensor_core_images_many_tokens_then_few_on_one_handle():
+    """A handle for up to 64 tokens: calls with 64, 20 and 3 tokens (one activation image per pass of 8 tokens of an
+    expert, or the single image of a call with at most 8 tokens), slots, fills and zero-copy experts."""
+    shape = W.LayerShape(d=1024, inter=256, n_experts=8, top_k=2, wdtype="mxfp4tc", n_shared=1)
+    pr = Pair(shape, n_slots=5, max_tokens=64, seed=16, fill_mode=B.FT_FILL_SM)
+    for step, T in enumerate((64, 20, 3, 64)):
+        _, r = pr.step(0, W.normal_logits(T, 8, 16, step), W.noise_x(T, 1024, 16, step, 0), fused=(step == 1))
+        if T == 64:
+            assert max(r.count) > 8
+    pr.close()
+
+
+def test_mxfp4_tensor_core_images_refuse_the_gemm_path():
     shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2, wdtype="mxfp4tc")
     with pytest.raises(B.FtMoeError) as ei:
-        Pair(shape, n_slots=4, max_tokens=16, seed=1)
+        Pair(shape, n_slots=4, max_tokens=64, seed=1, gemm_min_tokens=32)
     assert ei.value.code == B.FT_ERR_UNSUPPORTED
 
 
