@@ -314,7 +314,9 @@ ft_status_t ft_moe_set_split_min_pairs(ft_moe_t *h, int pairs);
  * latency is hidden.  2: as 1, but the grid waits only before its first write to the output accumulator, so its
  * weight streaming overlaps the tail of the preceding kernel; the caller asserts that x_dev, the slots and the plan
  * of this layer are not produced by that preceding kernel (e.g. forward calls of several already planned layers
- * issued back to back).  Takes effect at the next ft_moe_forward. */
+ * issued back to back).  For FT_W_MXFP4_TC handles mode 2 lets a call's first two kernels start while the call
+ * before is in its last kernel (calls with at most 8 tokens; not meant for replay from a captured graph, where the
+ * completion counts that order the calls are frozen).  Takes effect at the next ft_moe_forward. */
 ft_status_t ft_moe_set_launch_overlap(ft_moe_t *h, int mode);
 /* Test hook for the failure path of the bounded device-side waits (every wait of a kernel on an mbarrier gives up
  * after a limited number of polls, latches FT_ERR_TIMEOUT in the device status word, lets the copies already in

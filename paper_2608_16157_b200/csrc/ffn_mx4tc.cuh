@@ -134,6 +134,22 @@ __device__ __forceinline__ void tc_pass_tokens(const W4Params &p, bool dense, ui
   }
 }
 
+// Completion counts of the launches of a handle (cumulative numbers of CTAs that have finished: [0] gate/up kernels,
+// [1] down kernels).  A launch is given the counts all earlier launches add up to and waits for them, bounded, before
+// it touches what those launches use; in stream order the waits are satisfied on arrival, and they are what makes
+// launch overlap mode 2 (a call's first kernels start while the call before is still finishing) safe by construction.
+__device__ __forceinline__ bool tc_wait_count(const int *addr, int expect, uint32_t *status) {
+  const uint32_t limit = g_wait_polls;
+  for (uint32_t polls = 0; polls < limit; ++polls) {
+    int have;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(have) : "l"(addr) : "memory");
+    if ((int)((uint32_t)have - (uint32_t)expect) >= 0) return true;
+    __nanosleep(64);
+  }
+  atomicOr(status, kStatTimeout);
+  return false;
+}
+
 // x [T][d] bf16 -> the gate/up kernel's activation images: image i (blockIdx.y) holds the 8 token columns of pass i
 // (dense: one image, columns = the call's tokens), each as kTcParts parts of the hidden dimension.  One thread per 8
 // consecutive hidden indices of a column (unused columns are written as zeros); a quad of lanes is one block of 32.
@@ -142,12 +158,22 @@ struct TcQuantParams {
   const __nv_bfloat16 *x;
   uint8_t *xq;      // [images][kTcParts][tc_x_part_bytes(d)]
   int d, dense;
+  const int *gen;   // completion counts (see tc_wait_count)
+  int expect_gu;    // gate/up CTAs of all earlier calls: they read the images this kernel overwrites
+  int early;        // launch overlap mode 2: do not wait for the kernel before this one
 };
 __global__ void __launch_bounds__(256) tc_quant_x_kernel(TcQuantParams q) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  // (when launched as a programmatic dependent: the images are still being read until the kernels before have completed)
-  asm volatile("griddepcontrol.wait;" ::: "memory");
   const W4Params &p = q.w;
+  if (!q.early) {
+    // (when launched as a programmatic dependent: the images are still being read until the kernels before have completed)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+  } else {
+    // the caller's word: x, the plan and the slots are not produced by the kernel before; the images were last read
+    // by the gate/up kernel of the call before
+    if (threadIdx.x == 0) (void)tc_wait_count(q.gen, q.expect_gu, p.status);
+    __syncthreads();
+  }
   const uint32_t pass = blockIdx.y;
   if (!q.dense && pass >= (uint32_t)p.pref[*p.n_items + *p.n_zc]) return;
   const int per_tok = q.d / 8;
@@ -205,6 +231,8 @@ struct TcParams {
   int d;
   int n_stages;        // ring stages (what fits in shared memory, at most kTcMaxStages)
   int *pass_done;      // per pass: groups of 128 neurons whose h the gate/up kernel has written (0 between calls)
+  int *gen;            // completion counts (see tc_wait_count)
+  int expect_gu, expect_dn;   // gate/up CTAs, down CTAs of all earlier calls
 };
 
 // ---- PTX wrappers of the block-scaled path ----
@@ -440,6 +468,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
     const int ew = warp & 3, row = ew * 32 + lane, et = (warp - 6) * 32 + lane;
     uint32_t seg = 0, nt_pass = 0xffffffffu;
     int nt = p.T;   // token columns of the pass in use
+    // the hand-over buffers (partial sums, arrival counters, h images, pass counters) are free once the gate/up and
+    // down kernels of the earlier calls have completed
+    if (et == 0 && !(tc_wait_count(q.gen, q.expect_gu, p.status) && tc_wait_count(q.gen + 1, q.expect_dn, p.status))) *s_abort = 1;
+    tc_epi_barrier();
     walk([&](uint32_t pass, uint32_t ng, uint32_t, uint32_t n) {
       const uint32_t buf = seg & 1u;
       if (!dense && pass != nt_pass) {
@@ -526,6 +558,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
   tc_fence_before();
   __syncthreads();
   if (warp == 4) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+  if (tid == 0) {
+    __threadfence();
+    atomicAdd(q.gen, 1);
+  }
 }
 
 // Shared memory of the down kernel: activation image of the current pass and its scale atoms | ring | barriers |
@@ -694,6 +730,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
     const int ew = warp & 3, row = ew * 32 + lane;
     uint32_t seg = 0, it = 0, gw_pass = 0xffffffffu;
     TcPassTokens pt;
+    // the output accumulator is free once the down kernels of the earlier calls (their last CTA rounds and clears it)
+    // have completed
+    if (warp == 6 && lane == 0 && !tc_wait_count(q.gen + 1, q.expect_dn, p.status)) *s_abort = 1;
+    tc_epi_barrier();
     walk([&](uint32_t pass, uint32_t cg, uint32_t, uint32_t n) {
       const uint32_t buf = seg & 1u;
       if (pass != gw_pass) {
@@ -738,7 +778,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
     s_final = (prev == gridDim.x - 1);
   }
   __syncthreads();
-  if (!s_final) return;
+  if (!s_final) {
+    if (tid == 0) atomicAdd(q.gen + 1, 1);   // (after the fence above: this CTA's adds are visible)
+    return;
+  }
   __threadfence();
   const int n4 = p.finalize ? p.T * (d / 4) : 0;
   for (int i = tid; i < n4; i += kTcThreads) {
@@ -751,7 +794,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
     reinterpret_cast<float4 *>(p.y_acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
   }
   for (int i = tid; i < p.pref[n_items + n_zc]; i += kTcThreads) q.pass_done[i] = 0;
-  if (tid == 0) *p.done = 0u;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    *p.done = 0u;
+    __threadfence();
+    atomicAdd(q.gen + 1, 1);
+  }
 }
 
 }  // namespace ftmoe

@@ -100,6 +100,8 @@ struct ft_moe {
   uint8_t *w4_hq = nullptr;
   uint8_t *tc_xq = nullptr;      // FT_W_MXFP4_TC: the bit-sliced activation images of a call
   int *tc_pass_done = nullptr;   // FT_W_MXFP4_TC: per pass, the groups whose h is written (hand-over between the two kernels)
+  int *tc_gen = nullptr;         // FT_W_MXFP4_TC: cumulative counts of finished gate/up and down CTAs
+  uint32_t tc_calls = 0;         // FT_W_MXFP4_TC: forward calls so far
   float2 *w4_hs = nullptr;
   int last_fill_layer = -1;
   int overlap = 0;                      // launch mode of the streaming kernel (see FfnStreamParams::overlap)
@@ -504,6 +506,7 @@ ft_status_t ft_moe_destroy(ft_moe_t *h) {
   cudaFree(h->w4_hq);
   cudaFree(h->tc_xq);
   cudaFree(h->tc_pass_done);
+  cudaFree(h->tc_gen);
   cudaFree(h->w4_hs);
   cudaFree(h->trace_dev);
   cudaFree(h->stage_logits);
@@ -684,6 +687,8 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
       FT_TRY(cudaMemset(h->tc_xq, 0, n_img * kTcParts * tc_x_part_bytes(c.hidden)));
       FT_TRY(cudaMalloc(&h->tc_pass_done, passes * sizeof(int)));
       FT_TRY(cudaMemset(h->tc_pass_done, 0, passes * sizeof(int)));
+      FT_TRY(cudaMalloc(&h->tc_gen, 2 * sizeof(int)));
+      FT_TRY(cudaMemset(h->tc_gen, 0, 2 * sizeof(int)));
       if (tc_gateup_fixed_bytes(c.hidden) + 3 * kTcStageA > kTcSmem ||
           tc_down_fixed_bytes(c.inter) + 3 * kTcStageD > kTcSmem || c.inter / 128 > 48 || h->sm_count < kTcParts)
         return fail(FT_ERR_UNSUPPORTED);
@@ -771,7 +776,11 @@ ft_status_t ft_moe_reset(ft_moe_t *h, int layer) {
     const size_t passes = ((size_t)c.max_tokens * c.top_k + 7) / 8 + 2 * (size_t)c.n_experts + 2;
     FT_CUDA(cudaMemset(h->w4_hraw, 0, passes * (c.inter / 16) * 1024));
     FT_CUDA(cudaMemset(h->w4_hcount, 0, passes * (c.inter / 128) * 4));
-    if (h->tc_pass_done) FT_CUDA(cudaMemset(h->tc_pass_done, 0, passes * sizeof(int)));
+    if (h->tc_pass_done) {
+      FT_CUDA(cudaMemset(h->tc_pass_done, 0, passes * sizeof(int)));
+      FT_CUDA(cudaMemset(h->tc_gen, 0, 2 * sizeof(int)));
+      h->tc_calls = 0;
+    }
   }
   FT_CUDA(cudaDeviceSynchronize());
   return FT_OK;
@@ -1112,7 +1121,14 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     const bool dense = L.T <= kQ4Tokens, tc_own_finalize = L.T > kFinalizeInKernelMaxTokens;
     qp.finalize = tc_own_finalize ? 0 : 1;
     TcQuantParams tq;
+    const int grid = h->sm_count - h->sm_count % kTcParts;   // CTA i works on part i % kTcParts of the hidden dimension
+    const int expect_gu = (int)(h->tc_calls * (uint32_t)grid), expect_dn = (int)(h->tc_calls * (uint32_t)h->sm_count);
+    h->tc_calls++;
     tq.w = qp; tq.x = x_bf; tq.xq = h->tc_xq; tq.d = c.hidden; tq.dense = dense ? 1 : 0;
+    tq.gen = h->tc_gen; tq.expect_gu = expect_gu;
+    // overlap mode 2: the call's first kernels start while the call before is finishing (the completion counts order
+    // what they share); only for calls whose down kernel rounds y itself and that have a single activation image
+    tq.early = (h->overlap == 2 && dense && !tc_own_finalize) ? 1 : 0;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
@@ -1127,7 +1143,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     }
     TcParams tp;
     tp.w = qp; tp.xq = h->tc_xq; tp.d = c.hidden; tp.pass_done = h->tc_pass_done; tp.dense = dense ? 1 : 0;
-    const int grid = h->sm_count - h->sm_count % kTcParts;   // CTA i works on part i % kTcParts of the hidden dimension
+    tp.gen = h->tc_gen; tp.expect_gu = expect_gu; tp.expect_dn = expect_dn;
     {
       TimeScope ts(h, st, FT_TIME_FFN_ZC);
       const size_t fixed = tc_gateup_fixed_bytes(c.hidden);

@@ -11,9 +11,12 @@ from tests.helpers import Pair, bits, check_output
 pytestmark = pytest.mark.gpu
 
 
+@pytest.mark.parametrize("wdtype", ["bf16", "mxfp4tc"])
 @pytest.mark.parametrize("T", [3, 8, 21])
-def test_forward_calls_of_planned_layers_back_to_back_in_every_overlap_mode(T):
-    shape = W.LayerShape(d=1024, inter=256, n_experts=16, top_k=4)
+def test_forward_calls_of_planned_layers_back_to_back_in_every_overlap_mode(T, wdtype):
+    """(For the tensor-core MXFP4 path mode 2 lets a call's activation slicing and gate/up kernel start while the call
+    before is still in its down kernel; completion counts order what the calls share.)"""
+    shape = W.LayerShape(d=1024, inter=256, n_experts=16, top_k=4, wdtype=wdtype)
     L = 4
     pr = Pair(shape, n_slots=8, max_tokens=32, n_layers=L, seed=13, fill_mode=B.FT_FILL_SM)
     dev = pr.dev
