@@ -318,7 +318,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
   uint64_t *s_bar = reinterpret_cast<uint64_t *>(s_ring + (size_t)NS * kTcStageA);
   uint32_t *s_tmem = reinterpret_cast<uint32_t *>(s_bar + 64);
   volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
-  volatile int *s_last = s_abort + 1;
+  volatile int *s_last = s_abort + 1, *s_stop = s_abort + 2;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -499,12 +499,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
         __threadfence();
       }
       tc_epi_barrier();
-      if (et == 0 && !*s_abort) {
-        const int old = atomicAdd(p.hcount + pass * NG + ng, (int)n);
-        *s_last = (old + (int)n == (int)KS) ? 1 : 0;
+      if (et == 0) {
+        // (one thread decides for all whether to go on, so that the 128 threads leave together)
+        *s_stop = *s_abort;
+        *s_last = 0;
+        if (!*s_stop) {
+          const int old = atomicAdd(p.hcount + pass * NG + ng, (int)n);
+          *s_last = (old + (int)n == (int)KS) ? 1 : 0;
+        }
       }
       tc_epi_barrier();
-      if (*s_abort) return false;
+      if (*s_stop) return false;
       if (*s_last) {
         // this CTA's stages completed the group: h = SiLU(gate) * up, bit-sliced into the down kernel's operand
         __threadfence();
