@@ -2,7 +2,8 @@
 // call, from their slot into a bf16 record in tile order (the layout the GEMMs' tensor maps read, see
 // include/ftmoe.h) in a per-layer scratch pool.  With hundreds of tokens per expert the expansion (one pass over
 // the record) is small beside the GEMMs, and the GEMMs then run on exact bf16 activations: int4 weights are rounded
-// to bf16 after the multiplication by their scale (11-12 significant bits -> 8), MXFP4 weights are exact in bf16,
+// to bf16 after the multiplication by their scale (11-12 significant bits -> 8), MXFP4 weights (in either record
+// order) are exact in bf16,
 // NVFP4 weights are rounded after the multiplication by the block scale and the matrix scale.
 // One thread produces one 16-byte chunk of the destination (8 weights), in destination order, so that the writes
 // are coalesced; the 4-byte source words come from L2.
@@ -30,9 +31,9 @@ __device__ __forceinline__ float w4_code_value(uint32_t nib, bool mx) {
 // value of an unsigned e4m3 byte (see nv4_scale in ffn_mx4.cuh)
 __device__ __forceinline__ float w4_ue4m3(uint32_t b) { return __uint_as_float((b & 0x7Fu) << 20) * 0x1p120f; }
 
-template <int FMT>   // 0: int4-g128, 1: MXFP4, 2: NVFP4
+template <int FMT>   // 0: int4-g128, 1: MXFP4, 2: NVFP4, 3: MXFP4 stored as tensor-core operand images
 __global__ void __launch_bounds__(256) dequant_w4_kernel(DequantParams p) {
-  constexpr bool MX = FMT != 0, NV = FMT == 2;
+  constexpr bool MX = FMT != 0, NV = FMT == 2, TC = FMT == 3;
   const int d = p.d, I = p.inter;
   const uint32_t G = (uint32_t)d / 128u, NG = (uint32_t)I / 128u, NBLK = (uint32_t)I / 16u;
   const uint32_t NWD = min(16u, (uint32_t)d / 64u), CBW = 64u * NWD, CB = (uint32_t)d / CBW;
@@ -62,7 +63,17 @@ __global__ void __launch_bounds__(256) dequant_w4_kernel(DequantParams p) {
       const uint32_t q = pos ^ ((r & 7u) >> 1);                 // chunk q of the row is stored at position pos
       const uint32_t grp = t >> 2, j = t & 3u;                  // hidden indices 128 grp + 32 j + 8 q + 0..7
       const uint8_t *unit = rec + (size_t)u * UA;
-      if (NV) {
+      if (TC) {
+        // operand images: block of (128 neurons ng, 128 hidden indices st) = gate image, up image, gate scales, up
+        // scales; the 8 codes of hidden indices 8q .. 8q+7 of block j are one word of the row
+        const uint32_t row = 16u * (u & 7u) + r, kb = 32u * j + 8u * q;       // row of the 128, index in the 128
+        const uint8_t *blk = rec + ((size_t)(u >> 3) * G + grp) * 17408u;
+        const uint32_t w = *reinterpret_cast<const uint32_t *>(blk + mm * 8192u + 4096u * (kb >> 6) + 2048u * ((kb & 63u) >> 5) +
+                                                               128u * (row >> 3) + 16u * (row & 7u) + ((kb & 31u) >> 1));
+        const float scale = __uint_as_float((uint32_t)blk[16384u + mm * 512u + 16u * (row & 31u) + 4u * (row >> 5) + j] << 23);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[e] = scale * w4_code_value((w >> (4 * e)) & 15u, true);
+      } else if (NV) {
         // hidden indices 8q .. 8q+7 of block j: half q>>1 of the block (= the nibble parity), bytes 0..3 of word j of
         // the source chunks 2(q&1) and 2(q&1)+1
         const uint8_t *row = unit + (size_t)mm * 1024u * G + grp * 1024u + r * 64u + j * 4u;
@@ -95,9 +106,23 @@ __global__ void __launch_bounds__(256) dequant_w4_kernel(DequantParams p) {
       const uint32_t ng = u >> 3, uu = u & 7u;
       const uint32_t cb = c >> cbw_shift, tt = (c - (cb << cbw_shift)) >> 4, wq = tt >> 2, j = tt & 3u;
       const uint8_t *src = rec + sec_b + ((((size_t)(cb * NG + ng) * 8u + uu) * NWD + wq) * 32u + 4u * rr + 2u * nhalf) * 16u + 4u * j;
-      const uint32_t w0 = *reinterpret_cast<const uint32_t *>(src), w1 = *reinterpret_cast<const uint32_t *>(src + 16);
+      uint32_t w0 = 0u, w1 = 0u;
+      if (!TC) { w0 = *reinterpret_cast<const uint32_t *>(src); w1 = *reinterpret_cast<const uint32_t *>(src + 16); }
       float scale;
-      if (NV) {
+      if (TC) {
+        // section B: block of (128 columns cgp, 128 neurons ng); the unit's 16 neurons are 8 bytes of the column's row
+        const uint32_t rowc = c & 127u, kb = 16u * uu + 8u * nhalf;            // column of the 128, first neuron in the 128
+        const uint8_t *blk = rec + (size_t)(I / 128u) * G * 17408u + ((size_t)(c >> 7) * NG + ng) * 8704u;
+        const uint32_t wv = *reinterpret_cast<const uint32_t *>(blk + 4096u * (kb >> 6) + 2048u * ((kb & 63u) >> 5) + 128u * (rowc >> 3) +
+                                                                16u * (rowc & 7u) + ((kb & 31u) >> 1));
+        scale = __uint_as_float((uint32_t)blk[8192u + 16u * (rowc & 31u) + 4u * (rowc >> 5) + (kb >> 5)] << 23);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = scale * w4_code_value((wv >> (4 * i)) & 15u, true);
+        uint4 o;
+        o.x = pack_bf16(v[0], v[1]); o.y = pack_bf16(v[2], v[3]); o.z = pack_bf16(v[4], v[5]); o.w = pack_bf16(v[6], v[7]);
+        *reinterpret_cast<uint4 *>(dst) = o;
+        continue;
+      } else if (NV) {
         scale = w4_ue4m3(rec[sec_c + ((size_t)(ng * CB + cb) * NWD + wq) * 512u + 64u * rr + 16u * j + 8u * cg + uu]) * ms[2];
       } else if (MX) {
         const uint32_t b = rec[sec_c + ((size_t)(ng * CB + cb) * NWD + wq) * 256u + 32u * rr + 8u * j + 4u * cg + (uu >> 1)];

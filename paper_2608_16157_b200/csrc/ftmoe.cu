@@ -550,8 +550,6 @@ ft_status_t ft_moe_create(const ft_moe_config_t *cfg, ft_moe_t **out) {
       (c.slots_per_layer == 0 || c.hidden % 256 || c.inter % 256 || c.gemm_min_tokens < 8 ||
        (c.wdtype != FT_W_BF16 && c.global_pool)))   // (4-bit: the bf16 scratch mirrors one layer's slots)
     return FT_ERR_UNSUPPORTED;
-  // the tensor-core-image records are served by the streaming (decode) kernels only
-  if (c.wdtype == FT_W_MXFP4_TC && c.gemm_min_tokens != 0) return FT_ERR_UNSUPPORTED;
   if (!c.host_pool || c.host_pool_bytes < (size_t)c.n_layers * c.n_experts * S) return FT_ERR_INVALID_ARG;
   if (c.n_shared && !c.shared_weights) return FT_ERR_INVALID_ARG;
   if ((long long)c.max_tokens * c.top_k > (1ll << 30)) return FT_ERR_INVALID_ARG;
@@ -1118,8 +1116,8 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
   if (c.wdtype == FT_W_MXFP4_TC) {
     // bit-sliced activation images, then the two block-scaled tensor-core kernels (programmatic dependents: their
     // set-up and first weight copies overlap the kernel before them)
-    const bool dense = L.T <= kQ4Tokens, tc_own_finalize = L.T > kFinalizeInKernelMaxTokens;
-    qp.finalize = tc_own_finalize ? 0 : 1;
+    const bool dense = L.T <= kQ4Tokens, tc_own_finalize = !use_gemm && L.T > kFinalizeInKernelMaxTokens;
+    qp.finalize = (use_gemm || tc_own_finalize) ? 0 : 1;   // (the GEMM path's combine rounds y)
     TcQuantParams tq;
     const int grid = h->sm_count - h->sm_count % kTcParts;   // CTA i works on part i % kTcParts of the hidden dimension
     const int expect_gu = (int)(h->tc_calls * (uint32_t)grid), expect_dn = (int)(h->tc_calls * (uint32_t)h->sm_count);
@@ -1128,7 +1126,7 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
     tq.gen = h->tc_gen; tq.expect_gu = expect_gu;
     // overlap mode 2: the call's first kernels start while the call before is finishing (the completion counts order
     // what they share); only for calls whose down kernel rounds y itself and that have a single activation image
-    tq.early = (h->overlap == 2 && dense && !tc_own_finalize) ? 1 : 0;
+    tq.early = (h->overlap == 2 && dense && !tc_own_finalize && !use_gemm) ? 1 : 0;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
@@ -1170,6 +1168,19 @@ ft_status_t ft_moe_forward(ft_moe_t *h, int layer, const void *x_dev, void *y_de
       const int n4 = L.T * (c.hidden / 4);
       finalize_kernel<<<std::min((n4 + 255) / 256, h->sm_count * 8), 256, 0, st>>>(h->y_acc, qp.y, n4);
       h->launches++;
+    }
+    if (use_gemm) {
+      // the experts of the GEMM list: expanded from their operand images to bf16 records, then the grouped GEMMs
+      DequantParams dp;
+      dp.items = sc.items_gemm; dp.n_items = &sc.plan_dev->n_gemm_items; dp.scratch = h->wq_scratch;
+      dp.d = c.hidden; dp.inter = c.inter;
+      {
+        TimeScope ts(h, st, FT_TIME_GATHER);
+        const dim3 dg((unsigned)(c.inter / 16), (unsigned)std::min(c.n_experts, c.slots_per_layer));
+        dequant_w4_kernel<3><<<dg, 256, 0, st>>>(dp);
+      }
+      h->launches++;
+      return launch_gemm_path(h, layer, L, sc, x_bf, y_dev, st);
     }
     return FT_OK;
   }

@@ -222,13 +222,6 @@ def test_mxfp4_tensor_core_images_many_tokens_then_few_on_one_handle():
     pr.close()
 
 
-def test_mxfp4_tensor_core_images_refuse_the_gemm_path():
-    shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2, wdtype="mxfp4tc")
-    with pytest.raises(B.FtMoeError) as ei:
-        Pair(shape, n_slots=4, max_tokens=64, seed=1, gemm_min_tokens=32)
-    assert ei.value.code == B.FT_ERR_UNSUPPORTED
-
-
 def test_nvfp4_small_and_subnormal_block_scales():
     """NVFP4 records written by definition whose gate and down block scales are the 15 smallest e4m3 numbers (exponent
     field 0 or 1: the subnormal bytes included) under a matrix scale of 2^9, so that an error in the decoding of

@@ -16,7 +16,7 @@ def _zipf_logits(T, E, seed, step, alpha=1.1):
     return (rng.standard_normal((T, E)) + b).astype(np.float32)
 
 
-@pytest.mark.parametrize("wdtype", ["bf16", "int4", "mxfp4", "nvfp4"])
+@pytest.mark.parametrize("wdtype", ["bf16", "int4", "mxfp4", "nvfp4", "mxfp4tc"])
 @pytest.mark.parametrize("T,n_slots", [(300, 8), (1000, 6), (129, 3)])
 def test_prefill_grouped_gemm_matches_oracle(T, n_slots, wdtype):
     """Experts with >= 32 tokens and a slot go through the tensor-core GEMMs (4-bit experts after their expansion to
@@ -34,7 +34,7 @@ def test_prefill_grouped_gemm_matches_oracle(T, n_slots, wdtype):
     pr.close()
 
 
-@pytest.mark.parametrize("wdtype", ["int4", "mxfp4", "nvfp4"])
+@pytest.mark.parametrize("wdtype", ["int4", "mxfp4", "nvfp4", "mxfp4tc"])
 def test_prefill_4bit_wide_hidden_size(wdtype):
     """d=7168, I=2048 (the 4-bit decode configuration's layer shape), 8 experts, 256 tokens: K = 7168 in the gate/up
     GEMM, 56 column tiles in the down GEMM, weights from the bf16 scratch records."""
@@ -46,7 +46,7 @@ def test_prefill_4bit_wide_hidden_size(wdtype):
     pr.close()
 
 
-@pytest.mark.parametrize("wdtype", ["bf16", "mxfp4"])
+@pytest.mark.parametrize("wdtype", ["bf16", "mxfp4", "mxfp4tc"])
 def test_prefill_then_decode_on_the_same_handle(wdtype):
     shape = W.LayerShape(d=512, inter=256, n_experts=8, top_k=2, wdtype=wdtype)
     pr = Pair(shape, n_slots=8, max_tokens=512, seed=33, gemm_min_tokens=32)
@@ -57,7 +57,7 @@ def test_prefill_then_decode_on_the_same_handle(wdtype):
     pr.close()
 
 
-@pytest.mark.parametrize("wdtype", ["int4", "mxfp4", "nvfp4"])
+@pytest.mark.parametrize("wdtype", ["int4", "mxfp4", "nvfp4", "mxfp4tc"])
 def test_prefill_4bit_after_resize(wdtype):
     """The bf16 scratch pool the GEMMs read 4-bit experts from holds one record per slot of a layer, so a resize to
     more slots must grow it (and rebind the weight tensor maps): 3 slots -> 8 slots -> 2 slots."""
