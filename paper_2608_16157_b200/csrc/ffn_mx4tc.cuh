@@ -30,6 +30,8 @@
 // Every mbarrier wait is bounded (see async.cuh); a CTA whose wait runs out latches the timeout status, stops
 // issuing work, lets its copies in flight land, frees its tensor memory and returns.
 #pragma once
+#include <cuda_fp4.h>
+
 #include "async.cuh"
 #include "ffn_w4.cuh"
 #include "gemm_tc.cuh"
@@ -56,25 +58,9 @@ __host__ __device__ inline size_t tc_x_part_bytes(int d) {
 // Down operand of one pass: [inter/64 steps][kTcStepB] then [inter/128 scale atoms][512].
 __host__ __device__ inline size_t tc_h_pass_bytes(int inter) { return (size_t)(inter / 64) * kTcStepB + (size_t)(inter / 128) * 512; }
 
-// e2m1 rounding of v in [0, 6] (nearest, ties away from zero on the magnitude): value and 3-bit code.
-__device__ __forceinline__ void tc_e2m1(float v, float &val, uint32_t &code) {
-  v = fminf(v, 6.f);
-  if (v < 1.f) {
-    val = 0.5f * rintf(2.f * v);
-  } else {
-    val = __uint_as_float((__float_as_uint(v) + 0x00200000u) & 0xFFC00000u);   // keep one mantissa bit
-    val = fminf(val, 6.f);
-  }
-  if (val < 1.f) {
-    code = val == 0.5f ? 1u : 0u;
-  } else {
-    const uint32_t b = __float_as_uint(val);
-    code = (((b >> 23) - 126u) << 1) | ((b >> 22) & 1u);
-  }
-}
-
 // One bit-slicing term of 8 values held by each of the 4 lanes of a quad (the quad = one block of 32): returns the 8
 // codes (nibble e = element e) and the scale byte, and subtracts the term from r[].  bad: a non-finite input.
+// The e2m1 rounding (nearest, saturating at 6) and the way back are the hardware's conversions.
 __device__ __forceinline__ void tc_term(float (&r)[8], bool bad, uint32_t &codes, uint32_t &scale_byte) {
   float m = 0.f;
 #pragma unroll
@@ -90,13 +76,13 @@ __device__ __forceinline__ void tc_term(float (&r)[8], bool bad, uint32_t &codes
   scale_byte = ex;
   const float scale = __uint_as_float(ex << 23), inv = __uint_as_float((254u - ex) << 23);
 #pragma unroll
-  for (int e = 0; e < 8; ++e) {
-    float val;
-    uint32_t c;
-    tc_e2m1(fabsf(r[e]) * inv, val, c);
-    if (r[e] < 0.f) { val = -val; c |= 8u; }
-    r[e] -= val * scale;
-    codes |= c << (4 * e);
+  for (int k = 0; k < 4; ++k) {
+    const __nv_fp4x2_storage_t c = __nv_cvt_float2_to_fp4x2(make_float2(r[2 * k] * inv, r[2 * k + 1] * inv), __NV_E2M1, cudaRoundNearest);
+    const __half2_raw hb = __nv_cvt_fp4x2_to_halfraw2(c, __NV_E2M1);
+    const float2 back = __half22float2(*reinterpret_cast<const __half2 *>(&hb));
+    r[2 * k] -= back.x * scale;
+    r[2 * k + 1] -= back.y * scale;
+    codes |= (uint32_t)c << (8 * k);
   }
 }
 
