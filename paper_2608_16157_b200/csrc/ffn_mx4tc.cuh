@@ -43,8 +43,9 @@ constexpr int kTcN = 8 * kTcTerms;          // MMA columns: 8 tokens x terms
 constexpr uint32_t kTcStepB = kTcN * 32u;   // bytes of the activation image of one K = 64 step
 constexpr uint32_t kTcStageA = 17408u;      // gate/up stage: two images of 8192 bytes, two scale atoms of 512
 constexpr uint32_t kTcStageD = 8704u;       // down stage: one image, one scale atom
-constexpr int kTcLoaders = 128;             // warps 0..3 copy the records' stages into the ring, 16 bytes per cp.async
-constexpr int kTcThreads = kTcLoaders + 64 + 128;   // then warps 4 and 5: MMA issuers, warps 6..9: epilogue
+constexpr int kTcLoaders = 128;             // the first kTcLW warps copy the records' stages into the ring, 16 bytes per cp.async
+constexpr int kTcLW = kTcLoaders / 32;      // (a loader warp has one stage in flight; eight warps measured slower than four)
+constexpr int kTcThreads = kTcLoaders + 64 + 128;   // then two warps: MMA issuers, four warps: epilogue
 constexpr int kTcMaxStages = 16;
 constexpr size_t kTcSmem = 232448 - 1024;   // dynamic shared memory the two kernels may use (1 KiB left for static data)
 
@@ -322,7 +323,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
   }
   const int n_items = *p.n_items, n_zc = *p.n_zc;
   const bool dense = q.dense != 0;   // then every list entry is one pass: pass = index into the list
-  if (warp == 4) {
+  if (warp == kTcLW) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(s_tmem)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -355,7 +356,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
       }
   };
 
-  if (warp < 4) {
+  if (warp < kTcLW) {
     // ---- loaders: the weights do not depend on the preceding kernels; the activation images do ----
     // Thread 0 also brings the activation image (of the pass, or the one image of a dense call) into shared memory:
     // the first one after the first ring fill (so that the weights start to stream while the kernel before still
@@ -403,10 +404,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
       if (n_x) (void)mbar_wait(x_bar, (n_x - 1u) & 1u, s_abort, p.status);
       abort_drain(s_abort);
     }
-  } else if (warp <= 5) {
+  } else if (warp <= kTcLW + 1) {
     if (lane == 0) {
-      // ---- MMA issuers: warp 4 the gate matrix, warp 5 the up matrix ----
-      const uint32_t mat = (uint32_t)warp - 4u;
+      // ---- MMA issuers: the first of the two warps the gate matrix, the second the up matrix ----
+      const uint32_t mat = (uint32_t)(warp - kTcLW);
       uint32_t it = 0, seg = 0, n_x = 0, cur = 0xffffffffu;
       const uint32_t b_base = smem_u32(s_b), ring = smem_u32(s_ring) + mat * 8192u, t_sf = t_sfa + mat * 64u;
       walk([&](uint32_t pass, uint32_t, uint32_t st0, uint32_t n) {
@@ -451,7 +452,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
     }
   } else {
     // ---- epilogue: thread = accumulator row (neuron of the tile) ----
-    const int ew = warp & 3, row = ew * 32 + lane, et = (warp - 6) * 32 + lane;
+    const int ew = warp & 3, row = ew * 32 + lane, et = (warp - kTcLW - 2) * 32 + lane;
     uint32_t seg = 0, nt_pass = 0xffffffffu;
     int nt = p.T;   // token columns of the pass in use
     // the hand-over buffers (partial sums, arrival counters, h images, pass counters) are free once the gate/up and
@@ -548,7 +549,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_gateup_kernel(TcParams q) {
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 4) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+  if (warp == kTcLW) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
   if (tid == 0) {
     __threadfence();
     atomicAdd(q.gen, 1);
@@ -589,7 +590,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
   }
   const int n_items = *p.n_items, n_zc = *p.n_zc;
   const bool dense = q.dense != 0;   // then pass = index into the list, see the gate/up kernel
-  if (warp == 4) {
+  if (warp == kTcLW) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(s_tmem)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -620,7 +621,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
       }
   };
 
-  if (warp < 4) {
+  if (warp < kTcLW) {
     // ---- loaders ----
     uint32_t it = 0, n_h = 0, cur = 0xffffffffu;
     walk([&](uint32_t pass, uint32_t cg, uint32_t st0, uint32_t n) {
@@ -670,10 +671,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
       if (n_h) (void)mbar_wait(hfull_bar, (n_h - 1u) & 1u, s_abort, p.status);
       abort_drain(s_abort);
     }
-  } else if (warp <= 5) {
+  } else if (warp <= kTcLW + 1) {
     if (lane == 0) {
-      // ---- MMA issuers: warp 4 takes the stages of even ring index, warp 5 the odd ones ----
-      const uint32_t me = (uint32_t)warp - 4u;
+      // ---- MMA issuers: the first warp takes the stages of even ring index, the second the odd ones ----
+      const uint32_t me = (uint32_t)(warp - kTcLW);
       uint32_t it = 0, seg = 0, n_h = 0, cur = 0xffffffffu;
       const uint32_t b_base = smem_u32(s_b);
       walk([&](uint32_t pass, uint32_t, uint32_t st0, uint32_t n) {
@@ -723,7 +724,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
     TcPassTokens pt;
     // the output accumulator is free once the down kernels of the earlier calls (their last CTA rounds and clears it)
     // have completed
-    if (warp == 6 && lane == 0 && !tc_wait_count(q.gen + 1, q.expect_dn, p.status)) *s_abort = 1;
+    if (warp == kTcLW + 2 && lane == 0 && !tc_wait_count(q.gen + 1, q.expect_dn, p.status)) *s_abort = 1;
     tc_epi_barrier();
     walk([&](uint32_t pass, uint32_t cg, uint32_t, uint32_t n) {
       const uint32_t buf = seg & 1u;
@@ -758,7 +759,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_down_kernel(TcParams q) {
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 4) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+  if (warp == kTcLW) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
 
   // ---- the last CTA to finish clears the passes' hand-over counters and, unless a finalize launch follows (more
   // than 16 tokens), rounds the accumulator to bf16 and clears it ----
