@@ -78,9 +78,10 @@
  *                   bytes = image, scales.  In an image the code of (row r < 128, contraction index k < 128) is a
  *                   nibble (low when k is even) of byte 4096*(k/64) + 2048*((k%64)/32) + 128*(r/8) + 16*(r%8) +
  *                   (k%32)/2; the scale byte of (row r, block b < 4) is byte 16*(r%32) + 4*(r/32) + b.  Rows are
- *                   neurons (A) or output columns (B).  S as for FT_W_MXFP4.  The streaming kernels serve any token count (8 tokens of
- *                   an expert per weight pass); on the tensor-core prefill path the experts are expanded to bf16
- *                   records like the other 4-bit formats.
+ *                   neurons (A) or output columns (B).  S as for FT_W_MXFP4.  The streaming kernels serve any token
+ *                   count (8 tokens of an expert per weight pass; the bf16 activations are re-expressed as sums of
+ *                   six block-scaled e2m1 vectors, error <= 3^-6 of a block's largest magnitude); on the tensor-core
+ *                   prefill path the experts are expanded to bf16 records like the other 4-bit formats.
  *   FT_W_NVFP4    : two-level scaled FP4 (paper Sec. 5.1, expert representations): the same e2m1 codes with one
  *                   unsigned e4m3 scale byte b (exponent field E = b >> 3, mantissa M = b & 7: 2^(E-7) * (1 + M/8),
  *                   or 2^-6 * M/8 when E = 0; b <= 0x7E) per 16 consecutive elements of the contraction dimension and
